@@ -1,0 +1,435 @@
+"""CPU oracle for one TwIST training round.  TEST INFRASTRUCTURE ONLY.
+
+A plain, slow, obviously-correct numpy implementation (float64 arithmetic) of
+what the CUDA hot path computes: Algorithm 1 blueprints, dispatcher gather,
+local forward/backward/SGD steps on the dense slices, and the aggregator's
+coverage-normalised average.  It shares no code with the CUDA library and does
+not import it; only tests, the smoke check and the bench's cpu_baseline leg may
+call it.  The product path never routes through this module.
+
+Every function cites the passage of the paper it follows.  TwIST is an
+iteration, not a shortcut to a closed form, so each function takes the
+algorithm's steps in the paper's order and notation.
+
+Storage convention (a choice of this build, the paper fixes only mathematical
+shapes in its Problem formulation): every partitioned matrix is stored with one
+row per neuron / head-dimension and d_model contiguous, so a block is a run of
+whole rows ("a block is a chunk of parameters in memory", Sec. 3.1):
+    W_up, W_gate : [F, d]   (paper's W^ffn,  rows = hidden neurons)
+    W_down       : [F, d]   (paper's C^ffn transposed, rows = hidden neurons)
+    W_qkv        : [(H + 2 H_kv) d_head, d]  (transposed W^Q_h | W^K_h | W^V_h, head after head)
+    W_o          : [H d_head, d]             (paper's C^attn as printed)
+
+Parity pins: see tests/test_oracle_*.py.  The particular random stream of the
+sampler (which blocks a given seed picks) is fixed by this file's hash, not by
+the paper: "parity unpinned" for the stream itself; its distribution, its
+post-conditions and every other function are pinned.  A whole round at scale has
+no worked numeric example in the paper: "parity unpinned" beyond the per-step pins.
+"""
+from __future__ import annotations
+
+import numpy as np
+from scipy.special import erf
+
+FFN_RELU, FFN_GELU, FFN_SWIGLU = 0, 1, 2
+MODE_COVER, MODE_IID = 0, 1
+KIND_FFN, KIND_HEAD = 0, 1
+STREAM_PERM, STREAM_FILL = 0, 1
+
+_U64 = np.uint64
+_GOLDEN = _U64(0x9E3779B97F4A7C15)
+_M1 = _U64(0xBF58476D1CE4E5B9)
+_M2 = _U64(0x94D049BB133111EB)
+
+
+# ----------------------------------------------------------------------------------------
+# Counter-based integer hash used for every random draw of the sampler.
+# The paper leaves the generator open (Algorithm 1 calls it "unique_choice" and
+# Sec. 3.1 says "uniformly at random"); this build fixes a 64-bit avalanche
+# mixer (the published splitmix64 finaliser) applied to the counter tuple.
+# ----------------------------------------------------------------------------------------
+
+def mix64(z):
+    """One avalanche round on uint64 (wrapping arithmetic)."""
+    z = np.asarray(z, dtype=_U64)
+    with np.errstate(over="ignore"):
+        z = (z ^ (z >> _U64(30))) * _M1
+        z = (z ^ (z >> _U64(27))) * _M2
+        return z ^ (z >> _U64(31))
+
+
+def block_keys(seed, rnd, layer, kind, stream, s, n_full):
+    """Sort keys of blocks 0..n_full-1 for one (seed, round, layer, kind, stream, subnet).
+
+    key(b) = (hash48 << 16) | b : the upper 48 bits are random, the lower 16 are the
+    block index, so keys are distinct and "smallest key, ties by smaller b" is a
+    plain integer order.  Requires n_full <= 65536.
+    """
+    assert 0 < n_full <= 65536
+    with np.errstate(over="ignore"):
+        h = mix64(_U64(seed) + _GOLDEN)
+        h = mix64(h + _U64(rnd))
+        h = mix64(h + _U64((layer << 16) | (kind << 8) | stream))
+        h = mix64(h + _U64(s))
+        b = np.arange(n_full, dtype=_U64)
+        k = mix64(h + b)
+    return (k & ~_U64(0xFFFF)) | b
+
+
+def feasible(n_full, n_subnets, n_sub, n_common, mode=MODE_COVER):
+    """Size constraints of Sec. 3.1: N_sub <= N_full and N_full - |C| <= S (N_sub - |C|).
+    The IID mode (independent random subnets, no coverage guarantee) only needs
+    |C| <= N_sub <= N_full."""
+    if not (n_common <= n_sub <= n_full):
+        return False
+    if mode == MODE_COVER:
+        return n_full - n_common <= n_subnets * (n_sub - n_common)
+    return True
+
+
+def sample_blueprint(n_full, n_subnets, n_sub, common, seed, rnd, layer, kind, mode=MODE_COVER):
+    """Algorithm 1 ("Generate Training Subnet Blueprint"): returns A [S, N_sub], rows sorted.
+
+    Steps, in the algorithm's order:
+      1. every row starts with the common blocks C;
+      2. the non-common blocks C' are enumerated -- here in a seeded uniformly random
+         order (the text says subnets are generated uniformly at random) -- and the
+         i-th goes to subnet i mod S, so every block is assigned at least once;
+      3. each subnet s draws N_empty = N_sub - |filled_s| further distinct blocks
+         uniformly from those it does not hold yet: the N_empty candidates with the
+         smallest fill key of stream (s);
+      4. each row is sorted.
+    IID mode skips step 2 (used where N_sub is below the feasibility bound).
+    """
+    common = np.asarray(sorted(set(int(c) for c in common)), dtype=np.int64)
+    if not feasible(n_full, n_subnets, n_sub, len(common), mode):
+        raise ValueError("infeasible subnet size")
+    is_common = np.zeros(n_full, dtype=bool)
+    is_common[common] = True
+    filled = np.zeros((n_subnets, n_full), dtype=bool)
+    filled[:, common] = True                                            # step 1
+    if mode == MODE_COVER:                                              # step 2
+        kp = block_keys(seed, rnd, layer, kind, STREAM_PERM, 0, n_full)
+        non_common = np.flatnonzero(~is_common)
+        order = non_common[np.argsort(kp[non_common], kind="stable")]
+        for i, b in enumerate(order):
+            filled[i % n_subnets, b] = True
+    A = np.zeros((n_subnets, n_sub), dtype=np.int32)
+    for s in range(n_subnets):                                          # step 3
+        n_empty = n_sub - int(filled[s].sum())
+        assert n_empty >= 0
+        kf = block_keys(seed, rnd, layer, kind, STREAM_FILL, s, n_full)
+        cand = np.flatnonzero(~filled[s])
+        chosen = cand[np.argsort(kf[cand], kind="stable")[:n_empty]]
+        row = filled[s].copy()
+        row[chosen] = True
+        A[s] = np.flatnonzero(row)                                      # step 4 (ascending)
+    return A
+
+
+def cover_and_pos(A, n_full, counts=None):
+    """Derived index data for the aggregator (Sec. 3.3): per block the bitmask of
+    subnets holding it, the coverage count (the formula's denominator), and
+    pos[s, b] = rank of b inside row A[s] (-1 if absent).  `counts[s]` limits row s
+    to its first counts[s] entries (ragged KV-group rows)."""
+    S = len(A)
+    cover = np.zeros(n_full, dtype=np.uint32)
+    pos = np.full((S, n_full), -1, dtype=np.int32)
+    for s in range(S):
+        row = np.asarray(A[s])[: (len(A[s]) if counts is None else counts[s])]
+        cover[row] |= np.uint32(1 << s)
+        pos[s, row] = np.arange(len(row), dtype=np.int32)
+    count = np.array([bin(int(c)).count("1") for c in cover], dtype=np.int32)
+    return cover, count, pos
+
+
+def kv_groups(head_idx, n_heads, n_kv_heads):
+    """Grouped-query attention (not in the paper, which is plain multi-head): KV group
+    g = h // (H / H_kv) belongs to subnet s iff any of its query heads does.  Returns
+    kv_idx [S, H_kv] (sorted kept groups, padded with -1) and kv_count [S]."""
+    S = len(head_idx)
+    per = n_heads // n_kv_heads
+    kv_idx = np.full((S, n_kv_heads), -1, dtype=np.int32)
+    kv_count = np.zeros(S, dtype=np.int32)
+    for s in range(S):
+        g = np.unique(np.asarray(head_idx[s]) // per)
+        kv_idx[s, : len(g)] = g
+        kv_count[s] = len(g)
+    return kv_idx, kv_count
+
+
+# ----------------------------------------------------------------------------------------
+# Dispatcher (Sec. 3.2): kept blocks are concatenated into dense sub-matrices.
+# ----------------------------------------------------------------------------------------
+
+def block_rows_of(blocks, block_rows, row_offset=0):
+    blocks = np.asarray(blocks, dtype=np.int64)
+    return (row_offset + blocks[:, None] * block_rows + np.arange(block_rows)[None, :]).reshape(-1)
+
+
+def gather_rows(W_full, blocks, block_rows, row_offset=0):
+    """slice = rows of the kept blocks, in blueprint order, concatenated densely."""
+    return W_full[block_rows_of(blocks, block_rows, row_offset)].copy()
+
+
+# ----------------------------------------------------------------------------------------
+# Rounding points of the bf16 data flow (weights, stored activations and stored
+# activation gradients are bf16; every product-sum is accumulated wide).
+# ----------------------------------------------------------------------------------------
+
+def round_bf16(x):
+    """float64 -> nearest bf16 (ties to even), returned as float64."""
+    u = np.ascontiguousarray(x, dtype=np.float32).view(np.uint32)
+    r = (u + np.uint32(0x7FFF) + ((u >> np.uint32(16)) & np.uint32(1))) & np.uint32(0xFFFF0000)
+    return r.view(np.float32).astype(np.float64)
+
+
+def _q(x, lowp):
+    return round_bf16(x) if lowp else np.asarray(x, dtype=np.float64)
+
+
+def act_scale(n_full, n_sub):
+    """Activation-shift correction of Sec. 3.4: sqrt(N_full / N_sub)."""
+    return float(np.sqrt(n_full / n_sub))
+
+
+# ----------------------------------------------------------------------------------------
+# FFN block on a dense slice.  Paper (App. A, Feedforward): y = C relu(W x).
+# GELU (exact, x Phi(x)) and SwiGLU (silu(gate) * up) are the workloads' variants.
+# ----------------------------------------------------------------------------------------
+
+def _sigmoid(z):
+    return 1.0 / (1.0 + np.exp(-z))
+
+
+def _act(pre, kind):
+    if kind == FFN_RELU:
+        return np.maximum(pre, 0.0)
+    if kind == FFN_GELU:
+        return 0.5 * pre * (1.0 + erf(pre / np.sqrt(2.0)))
+    raise ValueError(kind)
+
+
+def _act_grad(pre, kind):
+    if kind == FFN_RELU:
+        return (pre > 0.0).astype(np.float64)
+    if kind == FFN_GELU:
+        return 0.5 * (1.0 + erf(pre / np.sqrt(2.0))) + pre * np.exp(-0.5 * pre * pre) / np.sqrt(2.0 * np.pi)
+    raise ValueError(kind)
+
+
+def ffn_fwd(X, W_up, W_gate, W_down, kind, alpha, lowp):
+    """Y = alpha * act(X W_up^T) W_down  (MLP)  or  alpha * (silu(X W_gate^T) * (X W_up^T)) W_down.
+    Returns Y [T, d] and the tensors kept for the backward pass (stored precision)."""
+    U = X @ W_up.T
+    if kind == FFN_SWIGLU:
+        G = X @ W_gate.T
+        Hh = (G * _sigmoid(G)) * U
+        saved = {"G": _q(G, lowp), "U": _q(U, lowp), "Hh": _q(Hh, lowp)}
+    else:
+        saved = {"U": _q(U, lowp), "Hh": _q(_act(U, kind), lowp)}
+    Y = _q(alpha * (saved["Hh"] @ W_down), lowp)
+    return Y, saved
+
+
+def ffn_bwd(dY, X, saved, W_up, W_gate, W_down, kind, alpha, lowp):
+    """Exact chain rule through ffn_fwd.  Returns dX and dW_up, dW_gate, dW_down ([f', d] each)."""
+    dHh = alpha * (dY @ W_down.T)
+    dW_down = alpha * (saved["Hh"].T @ dY)
+    if kind == FFN_SWIGLU:
+        G, U = saved["G"], saved["U"]
+        sg = _sigmoid(G)
+        dG = _q(dHh * U * (sg * (1.0 + G * (1.0 - sg))), lowp)
+        dU = _q(dHh * (G * sg), lowp)
+        dX = _q(dG @ W_gate + dU @ W_up, lowp)
+        return dX, dU.T @ X, dG.T @ X, dW_down
+    dU = _q(dHh * _act_grad(saved["U"], kind), lowp)
+    dX = _q(dU @ W_up, lowp)
+    return dX, dU.T @ X, None, dW_down
+
+
+# ----------------------------------------------------------------------------------------
+# Attention projections on a dense slice (App. A, Multi-Head Attention):
+# Q_h = X W^Q_h (and K, V), Y_attn = Concat(heads) C^attn.
+# ----------------------------------------------------------------------------------------
+
+def qkv_fwd(X, W_qkv, lowp):
+    return _q(X @ W_qkv.T, lowp)
+
+
+def qkv_bwd(dQKV, X, W_qkv, lowp):
+    return _q(dQKV @ W_qkv, lowp), dQKV.T @ X
+
+
+def o_fwd(A, W_o, alpha, lowp):
+    return _q(alpha * (A @ W_o), lowp)
+
+
+def o_bwd(dY, A, W_o, alpha, lowp):
+    return _q(alpha * (dY @ W_o.T), lowp), alpha * (A.T @ dY)
+
+
+# ----------------------------------------------------------------------------------------
+# Loss and optimiser of the local steps: mean squared error, plain SGD.
+# ----------------------------------------------------------------------------------------
+
+def mse(Y, Tgt, lowp, valid_cols=None):
+    """loss = mean over the T x width elements of (y - t)^2 (no 1/2); dY = 2 (y - t) / (T width).
+    valid_cols restricts both to the leading columns (zero gradient elsewhere)."""
+    T, width = Y.shape
+    vc = width if valid_cols is None else valid_cols
+    diff = np.zeros_like(Y, dtype=np.float64)
+    diff[:, :vc] = Y[:, :vc] - Tgt[:, :vc]
+    n = T * vc
+    return float(np.sum(diff * diff) / n), _q(2.0 * diff / n, lowp)
+
+
+def sgd(master, dW, lr, lowp):
+    """master <- master - lr dW; returns (new master, compute copy in stored precision)."""
+    new = master - lr * dW
+    return new, _q(new, lowp)
+
+
+# ----------------------------------------------------------------------------------------
+# Aggregator (Sec. 3.3): p <- sum_i p_i 1[p in W_i] / sum_i 1[p in W_i].
+# ----------------------------------------------------------------------------------------
+
+def aggregate(W_full, subs, blueprints, block_rows, live_mask=None, row_offset=0):
+    """Average each partitioned row over the (live) subnets that hold it; rows held by
+    no live subnet keep their value (the formula is 0/0 there).  Sum in ascending s."""
+    out = np.array(W_full, dtype=np.float64, copy=True)
+    acc = np.zeros_like(out)
+    cnt = np.zeros(out.shape[0], dtype=np.int64)
+    for s, (sub, blocks) in enumerate(zip(subs, blueprints)):
+        if live_mask is not None and not (live_mask >> s) & 1:
+            continue
+        rows = block_rows_of(blocks, block_rows, row_offset)
+        acc[rows] += np.asarray(sub, dtype=np.float64)[: len(rows)]
+        cnt[rows] += 1
+    held = cnt > 0
+    out[held] = acc[held] / cnt[held][:, None]
+    return out
+
+
+# ----------------------------------------------------------------------------------------
+# One round on one layer, BLOCKWISE composition: the FFN block, the QKV projection and
+# the output projection of a layer are independent regression problems, each with its
+# own N(0,1) inputs and targets.  Overview of a round: Sec. 3 (generate blueprints,
+# dispatch, local training for the repartition interval, aggregate, resample).
+# ----------------------------------------------------------------------------------------
+
+def layer_blueprints(spec, rnd, layer):
+    """Blueprints of one layer for one round: FFN blocks, heads, KV groups."""
+    out = {}
+    out["ffn"] = sample_blueprint(spec.d_ff // spec.ffn_block, spec.n_subnets, spec.ffn_keep, spec.common_ffn,
+                                  spec.seed_mask, rnd, layer, KIND_FFN, spec.sample_mode)
+    if spec.n_heads:
+        out["head"] = sample_blueprint(spec.n_heads, spec.n_subnets, spec.head_keep, spec.common_heads,
+                                       spec.seed_mask, rnd, layer, KIND_HEAD, spec.sample_mode)
+        out["kv_idx"], out["kv_count"] = kv_groups(out["head"], spec.n_heads, spec.n_kv_heads)
+    return out
+
+
+def gather_layer(spec, full, bp, s):
+    """Dense slices of subnet s for one layer (full: dict gate/up/down/qkv/o -> [rows, d])."""
+    sl = {}
+    sl["up"] = gather_rows(full["up"], bp["ffn"][s], spec.ffn_block)
+    sl["down"] = gather_rows(full["down"], bp["ffn"][s], spec.ffn_block)
+    if spec.ffn_kind == FFN_SWIGLU:
+        sl["gate"] = gather_rows(full["gate"], bp["ffn"][s], spec.ffn_block)
+    if spec.n_heads:
+        dh, H, Hkv = spec.d_head, spec.n_heads, spec.n_kv_heads
+        kv = bp["kv_idx"][s][: bp["kv_count"][s]]
+        sl["qkv"] = np.concatenate([gather_rows(full["qkv"], bp["head"][s], dh),
+                                    gather_rows(full["qkv"], kv, dh, H * dh),
+                                    gather_rows(full["qkv"], kv, dh, (H + Hkv) * dh)], axis=0)
+        sl["o"] = gather_rows(full["o"], bp["head"][s], dh)
+    return sl
+
+
+def local_steps_blockwise(spec, sl, get_batch, rnd, s, lowp):
+    """K local SGD steps of subnet s on its slices `sl` (masters, float64; updated in
+    place).  get_batch(kind, rnd, s, k, width) -> [T, width].  Returns the losses
+    {block: [K]}.  Batch kinds: 0 X, 1 target of width d, 2 target of QKV width, 3 A."""
+    d = spec.d_model
+    alpha_f = act_scale(spec.d_ff // spec.ffn_block, spec.ffn_keep)
+    losses = {"ffn": [], "qkv": [], "o": []}
+    for k in range(spec.local_steps):
+        X = get_batch(0, rnd, s, k, d).astype(np.float64)
+        Td = get_batch(1, rnd, s, k, d).astype(np.float64)
+        cw = {m: _q(v, lowp) for m, v in sl.items()}            # compute copies
+        Y, saved = ffn_fwd(X, cw["up"], cw.get("gate"), cw["down"], spec.ffn_kind, alpha_f, lowp)
+        loss, dY = mse(Y, Td, lowp)
+        _, dWu, dWg, dWd = ffn_bwd(dY, X, saved, cw["up"], cw.get("gate"), cw["down"], spec.ffn_kind, alpha_f, lowp)
+        losses["ffn"].append(loss)
+        sl["up"], _ = sgd(sl["up"], dWu, spec.lr, lowp)
+        sl["down"], _ = sgd(sl["down"], dWd, spec.lr, lowp)
+        if dWg is not None:
+            sl["gate"], _ = sgd(sl["gate"], dWg, spec.lr, lowp)
+        if spec.n_heads:
+            alpha_a = act_scale(spec.n_heads, spec.head_keep)
+            nq = sl["qkv"].shape[0]
+            Tq = get_batch(2, rnd, s, k, nq).astype(np.float64)
+            QKV = qkv_fwd(X, cw["qkv"], lowp)
+            loss, dQKV = mse(QKV, Tq, lowp)
+            _, dWq = qkv_bwd(dQKV, X, cw["qkv"], lowp)
+            losses["qkv"].append(loss)
+            sl["qkv"], _ = sgd(sl["qkv"], dWq, spec.lr, lowp)
+            A = get_batch(3, rnd, s, k, sl["o"].shape[0]).astype(np.float64)
+            Yo = o_fwd(A, cw["o"], alpha_a, lowp)
+            loss, dYo = mse(Yo, Td, lowp)
+            _, dWo = o_bwd(dYo, A, cw["o"], alpha_a, lowp)
+            losses["o"].append(loss)
+            sl["o"], _ = sgd(sl["o"], dWo, spec.lr, lowp)
+    return losses
+
+
+def aggregate_layer(spec, full, slices, bp):
+    """Aggregator over all partitioned matrices of one layer; returns the new full dict."""
+    S = spec.n_subnets
+    new = {}
+    for m in ("up", "down") + (("gate",) if spec.ffn_kind == FFN_SWIGLU else ()):
+        new[m] = aggregate(full[m], [slices[s][m] for s in range(S)], bp["ffn"], spec.ffn_block)
+    if spec.n_heads:
+        dh, H, Hkv = spec.d_head, spec.n_heads, spec.n_kv_heads
+        a_sub = spec.head_keep * dh
+        kvs = [bp["kv_idx"][s][: bp["kv_count"][s]] for s in range(S)]
+        qkv = aggregate(full["qkv"], [slices[s]["qkv"][:a_sub] for s in range(S)], bp["head"], dh)
+        qkv = aggregate(qkv, [slices[s]["qkv"][a_sub:a_sub + len(kvs[s]) * dh] for s in range(S)], kvs, dh,
+                        row_offset=H * dh)
+        qkv = aggregate(qkv, [slices[s]["qkv"][a_sub + len(kvs[s]) * dh:] for s in range(S)], kvs, dh,
+                        row_offset=(H + Hkv) * dh)
+        new["qkv"] = qkv
+        new["o"] = aggregate(full["o"], [slices[s]["o"] for s in range(S)], bp["head"], dh)
+    return new
+
+
+def round_blockwise_layer(spec, full, get_batch, rnd, layer, lowp):
+    """One full round on one layer: blueprint -> gather -> K local steps per subnet ->
+    aggregate.  Returns (new full weights of the layer, blueprints, losses per subnet)."""
+    bp = layer_blueprints(spec, rnd, layer)
+    slices, losses = [], []
+    for s in range(spec.n_subnets):
+        sl = {m: np.asarray(v, dtype=np.float64) for m, v in gather_layer(spec, full, bp, s).items()}
+        losses.append(local_steps_blockwise(spec, sl, get_batch, rnd, s, lowp))
+        slices.append(sl)
+    new = aggregate_layer(spec, full, slices, bp)
+    if lowp:   # the stored full model is bf16; the next round's gather reads the rounded shadow
+        new_shadow = {m: round_bf16(v) for m, v in new.items()}
+    else:
+        new_shadow = new
+    return new, new_shadow, bp, losses
+
+
+# ----------------------------------------------------------------------------------------
+# Parameter-count model of App. C (used to pin the byte counts of gather / aggregate).
+# ----------------------------------------------------------------------------------------
+
+def n_attn_params(d_attn, d_model, bias=True):
+    """N_attn = 4 d_attn d_model (+ 3 d_attn + d_model with biases)."""
+    return 4 * d_attn * d_model + ((3 * d_attn + d_model) if bias else 0)
+
+
+def n_ffn_params(d_ffn, d_model, bias=True):
+    """N_ffn = 2 d_ffn d_model (+ d_ffn + d_model with biases)."""
+    return 2 * d_ffn * d_model + ((d_ffn + d_model) if bias else 0)
