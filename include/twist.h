@@ -1,0 +1,240 @@
+/*
+ * twist.h -- C ABI of the B200-native (sm_100a) hot path of one TwIST training round.
+ *
+ * One round (paper Sec. 3, overview of the system): sample S structured subnet
+ * blueprints (Algorithm 1), gather the kept blocks of every partitioned weight
+ * matrix into dense slices (dispatcher, Sec. 3.2), run K local forward/backward
+ * SGD steps per subnet on the slices, average every parameter over the subnets
+ * that hold it (aggregator, Sec. 3.3), resample.
+ *
+ * General conventions
+ *  - Every function returns a status (TWIST_OK == 0, negative on error), never
+ *    throws, never exits.  Except where a function says otherwise it allocates
+ *    nothing, does not synchronise, and only enqueues work on `stream`
+ *    (a cudaStream_t passed as void*; NULL is the default stream).
+ *  - "device" pointers are CUDA device memory owned by the caller; they must stay
+ *    valid until the stream has run the call.  "host" pointers are read during the
+ *    call only.  Base pointers must be 16-byte aligned.
+ *  - Storage layout: every partitioned matrix is row-major with one row per hidden
+ *    neuron / head dimension and d_model contiguous ("a block is a chunk of
+ *    parameters in memory", Sec. 3.1):
+ *        W_gate, W_up, W_down : [F, d];  W_qkv : [(H + 2 H_kv) d_head, d];  W_o : [H d_head, d].
+ *    up/gate/qkv rows are output features (y = x W^T), down/o rows are input features (y = h W).
+ *    Slices and activations of the S subnets are packed [S][rows][cols], dense.
+ *  - dtype TWIST_BF16: weights, stored activations and stored activation gradients are
+ *    bf16; products accumulate in fp32; each slice has an fp32 master copy that SGD
+ *    updates.  dtype TWIST_FP32: everything is fp32 and the slice is its own master.
+ *  - Row widths (d_model, f_sub, a_sub, ...) must be multiples of 8 elements in bf16.
+ *  - Kernels that wait on hardware barriers bound every wait; on expiry they record
+ *    TWIST_ERR_DEVICE_TIMEOUT in a device status word (read it with twist_device_status)
+ *    and return instead of hanging.
+ */
+#ifndef TWIST_H_
+#define TWIST_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+  TWIST_OK = 0,
+  TWIST_ERR_NULL = -1,           /* a required pointer is NULL */
+  TWIST_ERR_SHAPE = -2,          /* a size is non-positive, misaligned or inconsistent */
+  TWIST_ERR_INFEASIBLE = -3,     /* N_sub violates the size bound of Sec. 3.1 */
+  TWIST_ERR_BAD_INDEX = -4,      /* an index array entry is out of range / unsorted */
+  TWIST_ERR_UNSUPPORTED = -5,    /* valid request outside what the kernels implement */
+  TWIST_ERR_WORKSPACE = -6,      /* workspace missing or too small */
+  TWIST_ERR_CUDA = -7,           /* a CUDA runtime/driver call failed (see twist_last_cuda_error) */
+  TWIST_ERR_DEVICE_TIMEOUT = -8  /* a bounded device-side wait expired */
+};
+
+enum { TWIST_FP32 = 0, TWIST_BF16 = 1 };
+enum { TWIST_FFN_RELU = 0, TWIST_FFN_GELU = 1, TWIST_FFN_SWIGLU = 2 };
+enum { TWIST_MODE_COVER = 0, TWIST_MODE_IID = 1 };
+enum { TWIST_KIND_FFN = 0, TWIST_KIND_HEAD = 1 };
+enum { TWIST_PROJ_QKV = 0, TWIST_PROJ_O = 1 };
+
+#define TWIST_MAX_SUBNETS 32
+#define TWIST_MAX_BLOCKS 16384   /* blocks per layer and kind the sampler kernel handles */
+#define TWIST_MAX_COMMON 256     /* common blocks |C| per layer and kind */
+
+uint32_t twist_abi_version(void);
+const char* twist_strerror(int32_t status);
+/* Text of the last CUDA error this library saw on the calling thread ("" if none). */
+const char* twist_last_cuda_error(void);
+/* Reads (and clears) the device status word.  Synchronises the device.  *code is TWIST_OK or
+ * TWIST_ERR_DEVICE_TIMEOUT. */
+int32_t twist_device_status(int32_t* code);
+
+/* ---------------------------------------------------------------------------------------------
+ * twist_sample_masks -- subnet generator, Algorithm 1 ("Generate Training Subnet Blueprint").
+ *
+ * For each of n_layers consecutive layers (layer_begin ...) and one block kind, builds the
+ * blueprint A [S][n_sub] (rows sorted ascending):  common blocks C, then a seeded random
+ * order of the non-common blocks dealt round-robin to the subnets (every block is held at
+ * least once), then each subnet fills up to n_sub with distinct random blocks it lacks, then
+ * sort.  TWIST_MODE_IID skips the round-robin deal (independent random subnets; used where
+ * n_sub is below the bound of Sec. 3.1).  Random draws are a counter-based 64-bit hash of
+ * (seed, round, layer, kind, stream, subnet, block); results are a pure function of those.
+ * Also writes the index data the aggregator (Sec. 3.3) needs: cover[l][b] = bitmask of the
+ * subnets holding block b, pos[l][s][b] = rank of b in A[s] or -1.
+ *
+ *  common      host, n_common sorted distinct block ids (may be NULL when n_common == 0)
+ *  idx         device out, int32 [n_layers][S][n_sub]
+ *  cover       device out, uint32 [n_layers][n_full]
+ *  pos         device out, int32 [n_layers][S][n_full]
+ * Errors: INFEASIBLE when (n_full + (S-1)|C|)/S <= n_sub <= n_full fails in COVER mode (IID
+ * needs |C| <= n_sub <= n_full); UNSUPPORTED when n_full > TWIST_MAX_BLOCKS, S > 32 or
+ * n_common > TWIST_MAX_COMMON; BAD_INDEX when `common` is unsorted or out of range.
+ */
+int32_t twist_sample_masks(uint64_t seed, uint64_t round, int32_t layer_begin, int32_t n_layers, int32_t kind,
+                           int32_t n_full, int32_t n_subnets, int32_t n_sub,
+                           const int32_t* common, int32_t n_common, int32_t sample_mode,
+                           int32_t* idx, uint32_t* cover, int32_t* pos, void* stream);
+
+/* KV groups under grouped-query attention (an extension; the paper's attention is plain
+ * multi-head, App. A): group g = h / (n_heads / n_kv_heads) is held by subnet s iff one of its
+ * query heads is.  Writes kv_idx [n_layers][S][n_kv_heads] (sorted kept groups, then -1),
+ * kv_count [n_layers][S], kv_cols [n_layers][S] = kv_count * d_head (valid K or V columns of the
+ * subnet's projection), kv_cover [n_layers][n_kv_heads], kv_pos [n_layers][S][n_kv_heads]; all device. */
+int32_t twist_kv_groups(const int32_t* head_idx, int32_t n_layers, int32_t n_subnets, int32_t head_keep,
+                        int32_t n_heads, int32_t n_kv_heads, int32_t d_head, int32_t* kv_idx, int32_t* kv_count,
+                        int32_t* kv_cols, uint32_t* kv_cover, int32_t* kv_pos, void* stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * twist_gather_subnets -- dispatcher, Sec. 3.2: the kept blocks of a matrix are concatenated
+ * into one dense sub-matrix per subnet.
+ *
+ * One call moves up to TWIST_MAX_SEGMENTS row ranges ("segments", e.g. gate, up, down, Q, K, V,
+ * O of one layer) in a single launch.  For segment g, subnet s, kept entry j < n_keep and
+ * i < block_rows:
+ *   dst[s*dst_subnet_stride + (dst_row_offset + j*block_rows + i)*d + :]
+ *       = src[(src_row_offset + idx[s*idx_stride + j]*block_rows + i)*d + :]
+ * (bit copy); the same values widened to fp32 go to dst_master when it is not NULL.  Entries
+ * j >= count[s] (count may be NULL = all valid) are written as zeros (padding of ragged KV rows).
+ */
+#define TWIST_MAX_SEGMENTS 8
+typedef struct {
+  const void* src;            /* device, full matrix [rows_full][d] in `dtype` */
+  void* dst;                  /* device, slices in `dtype` */
+  float* dst_master;          /* device fp32 copy of dst (same geometry) or NULL */
+  const int32_t* idx;         /* device int32 [S][idx_stride], kept block ids */
+  const int32_t* count;       /* device int32 [S] valid entries per subnet, or NULL */
+  int32_t idx_stride;
+  int32_t n_keep;             /* entries written per subnet */
+  int32_t block_rows;         /* rows per block */
+  int32_t reserved;
+  int64_t src_row_offset;     /* first row of the partitioned range inside src */
+  int64_t dst_subnet_stride;  /* elements between consecutive subnets in dst / dst_master */
+  int64_t dst_row_offset;     /* first destination row inside a subnet's slice */
+} twist_gather_segment;
+
+int32_t twist_gather_subnets(const twist_gather_segment* segs /*host*/, int32_t n_segs, int32_t n_subnets,
+                             int32_t d, int32_t dtype, void* stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * twist_aggregate -- aggregator, Sec. 3.3:  p <- sum_i p_i 1[p in W_i] / sum_i 1[p in W_i].
+ *
+ * For every block b of a segment whose cover mask (restricted to live_subnets) is non-zero,
+ * each of its rows becomes the fp32 sum, in ascending subnet order, of the subnets' master rows
+ * divided (IEEE division) by the number of subnets summed.  The result is written to dst_f32
+ * (if not NULL) and, rounded to nearest-even, to dst (bf16 dtype) -- the copy the next gather
+ * reads.  Blocks held by no live subnet are neither read nor written.  One writer per row, fixed
+ * order, no atomics: results are deterministic.
+ *   src (subnet s, block b at rank pos[s][b]) row i:
+ *       sub[s*sub_subnet_stride + (sub_row_offset + pos[s*n_full + b]*block_rows + i)*d + :]
+ */
+typedef struct {
+  void* dst;                  /* device, full matrix in `dtype` (bf16: rounded shadow; fp32: the result) */
+  float* dst_f32;             /* device fp32 full-precision result (bf16 dtype only), may be NULL */
+  const float* sub;           /* device fp32 slices (masters in bf16 dtype, the slices in fp32 dtype) */
+  const uint32_t* cover;      /* device uint32 [n_full] */
+  const int32_t* pos;         /* device int32 [S][n_full] */
+  int32_t n_full;             /* blocks in this segment */
+  int32_t block_rows;
+  int64_t dst_row_offset;     /* first row of the partitioned range inside dst */
+  int64_t sub_subnet_stride;  /* elements between subnets in sub */
+  int64_t sub_row_offset;     /* first row of this segment inside a subnet's slice */
+} twist_aggregate_segment;
+
+int32_t twist_aggregate(const twist_aggregate_segment* segs /*host*/, int32_t n_segs, int32_t n_subnets,
+                        int32_t d, int32_t dtype, uint32_t live_subnets, void* stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * Local training on the dense slices (workers of Sec. 4.1 "True TwIST"; FFN of App. A:
+ * y = C relu(W x); the GELU and SwiGLU variants are the workloads').  All S subnets run in one
+ * grouped launch per contraction.  out_scale is the activation-shift correction sqrt(N_full/N_sub)
+ * of Sec. 3.4 (pass 1 to disable it).
+ *
+ * twist_subnet_ffn_fwd:
+ *   MLP:    pre = X W_up^T;                 hh = act(pre);               Y = out_scale * hh W_down
+ *   SwiGLU: pre = [X W_gate^T | X W_up^T];  hh = silu(G) * U;            Y = out_scale * hh W_down
+ * twist_subnet_ffn_bwd (exact chain rule):
+ *   dHh = out_scale * dY W_down^T;  dpre = dHh * act'(pre)  (SwiGLU: dG = dHh U silu'(G), dU = dHh silu(G));
+ *   dX = dpre W_gu;  dW_gu = dpre^T X;  dW_down = out_scale * hh^T dY;
+ *   if lr != 0:  master -= lr * dW (fp32), compute copy = round(master)   [plain SGD]
+ */
+typedef struct {
+  int32_t ffn_kind, dtype, n_subnets, tokens, d_model, f_sub;
+  float out_scale, lr;
+  const void* x;        /* device [S][T][d] */
+  void* w_gu;           /* device [S][g*f_sub][d], g = 2 (SwiGLU: gate rows then up rows) or 1 */
+  void* w_down;         /* device [S][f_sub][d] */
+  float* w_gu_master;   /* device fp32 masters (bf16 dtype, bwd only) */
+  float* w_down_master;
+  void* pre;            /* device [S][T][g*f_sub]  fwd: out, bwd: in */
+  void* hh;             /* device [S][T][f_sub]    fwd: out, bwd: in */
+  void* y;              /* device [S][T][d]        fwd: out */
+  const void* dy;       /* device [S][T][d]        bwd: in */
+  void* dpre;           /* device [S][T][g*f_sub]  bwd: out (gradient w.r.t. pre) */
+  void* dx;             /* device [S][T][d]        bwd: out, may be NULL */
+  float* dw_gu;         /* device fp32 [S][g*f_sub][d] gradient dump, may be NULL (required in fp32 dtype) */
+  float* dw_down;       /* device fp32 [S][f_sub][d]   gradient dump, may be NULL (required in fp32 dtype) */
+} twist_ffn_args;
+
+int32_t twist_subnet_ffn_fwd(const twist_ffn_args* a /*host*/, void* stream);
+int32_t twist_subnet_ffn_bwd(const twist_ffn_args* a /*host*/, void* stream);
+
+/* Attention projections on the kept heads (App. A, Multi-Head Attention: Q_h = X W^Q_h ...,
+ * Y_attn = Concat(heads) C^attn).
+ *   which == TWIST_PROJ_QKV:  out [S][T][n] = out_scale * in [S][T][d] W^T,  W [S][n][d],  n = a_sub + 2 kv_sub
+ *                             (the paper scales only the block output: pass out_scale = 1 here)
+ *   which == TWIST_PROJ_O:    out [S][T][d] = out_scale * in [S][T][n] W,  W [S][n][d],  n = a_sub
+ * bwd: d_in (may be NULL), dW = (QKV) d_out^T in | (O) out_scale * in^T d_out, SGD as above. */
+typedef struct {
+  int32_t which, dtype, n_subnets, tokens, d_model, n;
+  float out_scale, lr;
+  const void* in;       /* device */
+  void* w;              /* device [S][n][d] */
+  float* w_master;      /* device fp32 master (bf16 dtype, bwd only) */
+  void* out;            /* fwd: out */
+  const void* d_out;    /* bwd: in */
+  void* d_in;           /* bwd: out, may be NULL */
+  float* dw;            /* device fp32 [S][n][d] gradient dump, may be NULL (required in fp32 dtype) */
+} twist_proj_args;
+
+int32_t twist_subnet_attn_proj_fwd(const twist_proj_args* a /*host*/, void* stream);
+int32_t twist_subnet_attn_proj_bwd(const twist_proj_args* a /*host*/, void* stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * Loss of the local steps: mean squared error against a target, per subnet, and its gradient.
+ *   loss[s] = mean over the valid elements of (y - t)^2;   dy = 2 (y - t) / n_valid  (zero where invalid)
+ * Valid columns: all `width` columns when valid_cols is NULL.  Otherwise columns [0, seg_begin) are
+ * valid and the remaining columns form groups of seg_width columns each, of which the first
+ * valid_cols[s] (device int32 [S]) are valid -- the zero-padded K and V column groups of a subnet
+ * that kept fewer KV groups than the maximum.  (seg_begin = 0, seg_width = width gives a prefix mask.)
+ *  ws / ws_bytes: device scratch of at least twist_mse_workspace_bytes(S) bytes (per-block partial
+ *  sums; summed in a fixed order, so the loss is deterministic).
+ */
+size_t twist_mse_workspace_bytes(int32_t n_subnets);
+int32_t twist_mse_fwd_bwd(const void* y, const void* tgt, void* dy, float* loss, int32_t n_subnets, int32_t tokens,
+                          int32_t width, const int32_t* valid_cols, int32_t seg_begin, int32_t seg_width,
+                          int32_t dtype, void* ws, size_t ws_bytes, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TWIST_H_ */

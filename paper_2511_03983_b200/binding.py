@@ -1,0 +1,222 @@
+"""Thin ctypes binding of the C ABI in include/twist.h (argument marshalling only).
+
+Every function has the name of its C entry point.  Tensors are torch CUDA tensors
+(torch is used for device memory and streams only); the binding passes their
+data pointers and the current CUDA stream.  A non-zero status raises TwistError.
+The shared library must exist: there is no CPU fallback.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional, Sequence
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libtwist.so")
+
+OK = 0
+ERR_NULL, ERR_SHAPE, ERR_INFEASIBLE, ERR_BAD_INDEX, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_DEVICE_TIMEOUT = \
+    -1, -2, -3, -4, -5, -6, -7, -8
+FP32, BF16 = 0, 1
+FFN_RELU, FFN_GELU, FFN_SWIGLU = 0, 1, 2
+MODE_COVER, MODE_IID = 0, 1
+KIND_FFN, KIND_HEAD = 0, 1
+PROJ_QKV, PROJ_O = 0, 1
+MAX_SEGMENTS = 8
+
+EXPORTS = [
+    "twist_abi_version", "twist_strerror", "twist_last_cuda_error", "twist_device_status", "twist_sample_masks",
+    "twist_kv_groups", "twist_gather_subnets", "twist_aggregate", "twist_subnet_ffn_fwd", "twist_subnet_ffn_bwd",
+    "twist_subnet_attn_proj_fwd", "twist_subnet_attn_proj_bwd", "twist_mse_workspace_bytes", "twist_mse_fwd_bwd",
+]
+
+
+class TwistError(RuntimeError):
+    def __init__(self, status: int, where: str, detail: str = ""):
+        self.status = status
+        super().__init__(f"{where}: status {status} ({detail})")
+
+
+class GatherSegment(C.Structure):
+    _fields_ = [("src", C.c_void_p), ("dst", C.c_void_p), ("dst_master", C.c_void_p), ("idx", C.c_void_p),
+                ("count", C.c_void_p), ("idx_stride", C.c_int32), ("n_keep", C.c_int32), ("block_rows", C.c_int32),
+                ("reserved", C.c_int32), ("src_row_offset", C.c_int64), ("dst_subnet_stride", C.c_int64),
+                ("dst_row_offset", C.c_int64)]
+
+
+class AggregateSegment(C.Structure):
+    _fields_ = [("dst", C.c_void_p), ("dst_f32", C.c_void_p), ("sub", C.c_void_p), ("cover", C.c_void_p),
+                ("pos", C.c_void_p), ("n_full", C.c_int32), ("block_rows", C.c_int32), ("dst_row_offset", C.c_int64),
+                ("sub_subnet_stride", C.c_int64), ("sub_row_offset", C.c_int64)]
+
+
+class FfnArgs(C.Structure):
+    _fields_ = [("ffn_kind", C.c_int32), ("dtype", C.c_int32), ("n_subnets", C.c_int32), ("tokens", C.c_int32),
+                ("d_model", C.c_int32), ("f_sub", C.c_int32), ("out_scale", C.c_float), ("lr", C.c_float),
+                ("x", C.c_void_p), ("w_gu", C.c_void_p), ("w_down", C.c_void_p), ("w_gu_master", C.c_void_p),
+                ("w_down_master", C.c_void_p), ("pre", C.c_void_p), ("hh", C.c_void_p), ("y", C.c_void_p),
+                ("dy", C.c_void_p), ("dpre", C.c_void_p), ("dx", C.c_void_p), ("dw_gu", C.c_void_p),
+                ("dw_down", C.c_void_p)]
+
+
+class ProjArgs(C.Structure):
+    _fields_ = [("which", C.c_int32), ("dtype", C.c_int32), ("n_subnets", C.c_int32), ("tokens", C.c_int32),
+                ("d_model", C.c_int32), ("n", C.c_int32), ("out_scale", C.c_float), ("lr", C.c_float),
+                ("in_", C.c_void_p), ("w", C.c_void_p), ("w_master", C.c_void_p), ("out", C.c_void_p),
+                ("d_out", C.c_void_p), ("d_in", C.c_void_p), ("dw", C.c_void_p)]
+
+
+_lib_handle = None
+
+
+def lib() -> C.CDLL:
+    """Loads libtwist.so (once).  Fails loudly when it has not been built."""
+    global _lib_handle
+    if _lib_handle is None:
+        if not os.path.exists(LIB_PATH):
+            raise FileNotFoundError(
+                f"{LIB_PATH} is missing: build it with `python -m paper_2511_03983_b200.build` (there is no fallback)")
+        h = C.CDLL(LIB_PATH)
+        h.twist_abi_version.restype = C.c_uint32
+        h.twist_strerror.restype = C.c_char_p
+        h.twist_strerror.argtypes = [C.c_int32]
+        h.twist_last_cuda_error.restype = C.c_char_p
+        h.twist_device_status.argtypes = [C.POINTER(C.c_int32)]
+        h.twist_sample_masks.argtypes = [C.c_uint64, C.c_uint64, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int32,
+                                         C.c_int32, C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p,
+                                         C.c_void_p, C.c_void_p]
+        h.twist_kv_groups.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int32,
+                                      C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+        h.twist_gather_subnets.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_void_p]
+        h.twist_aggregate.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_uint32, C.c_void_p]
+        for name in ("twist_subnet_ffn_fwd", "twist_subnet_ffn_bwd", "twist_subnet_attn_proj_fwd",
+                     "twist_subnet_attn_proj_bwd"):
+            getattr(h, name).argtypes = [C.c_void_p, C.c_void_p]
+        h.twist_mse_workspace_bytes.restype = C.c_size_t
+        h.twist_mse_workspace_bytes.argtypes = [C.c_int32]
+        h.twist_mse_fwd_bwd.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32,
+                                        C.c_int32, C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_size_t,
+                                        C.c_void_p]
+        for name in EXPORTS:
+            f = getattr(h, name)
+            if name not in ("twist_abi_version", "twist_strerror", "twist_last_cuda_error",
+                            "twist_mse_workspace_bytes"):
+                f.restype = C.c_int32
+        _lib_handle = h
+    return _lib_handle
+
+
+def _check(status: int, where: str):
+    if status != OK:
+        h = lib()
+        detail = h.twist_strerror(status).decode()
+        if status == ERR_CUDA:
+            detail += ": " + h.twist_last_cuda_error().decode()
+        raise TwistError(status, where, detail)
+
+
+def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
+    if t is None:
+        return None
+    assert t.is_cuda and t.is_contiguous(), "device tensors must be contiguous CUDA tensors"
+    return t.data_ptr()
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def twist_abi_version() -> int:
+    return lib().twist_abi_version()
+
+
+def twist_device_status() -> int:
+    code = C.c_int32(0)
+    _check(lib().twist_device_status(C.byref(code)), "twist_device_status")
+    return code.value
+
+
+def twist_sample_masks(seed, rnd, layer_begin, n_layers, kind, n_full, n_subnets, n_sub, common: Sequence[int],
+                       sample_mode, idx, cover, pos):
+    arr = (C.c_int32 * max(1, len(common)))(*common)
+    _check(lib().twist_sample_masks(seed, rnd, layer_begin, n_layers, kind, n_full, n_subnets, n_sub,
+                                    C.cast(arr, C.c_void_p) if len(common) else None, len(common), sample_mode,
+                                    _ptr(idx), _ptr(cover), _ptr(pos), _stream()), "twist_sample_masks")
+
+
+def twist_kv_groups(head_idx, n_layers, n_subnets, head_keep, n_heads, n_kv_heads, d_head, kv_idx, kv_count, kv_cols,
+                    kv_cover, kv_pos):
+    _check(lib().twist_kv_groups(_ptr(head_idx), n_layers, n_subnets, head_keep, n_heads, n_kv_heads, d_head,
+                                 _ptr(kv_idx), _ptr(kv_count), _ptr(kv_cols), _ptr(kv_cover), _ptr(kv_pos), _stream()),
+           "twist_kv_groups")
+
+
+def gather_segment(src, dst, dst_master, idx, count, idx_stride, n_keep, block_rows, src_row_offset,
+                   dst_subnet_stride, dst_row_offset) -> GatherSegment:
+    """Marshals one twist_gather_segment.  src/dst/... may be tensors or raw device addresses (ints)."""
+    a = lambda v: v if (v is None or isinstance(v, int)) else _ptr(v)
+    return GatherSegment(a(src), a(dst), a(dst_master), a(idx), a(count), idx_stride, n_keep, block_rows, 0,
+                         src_row_offset, dst_subnet_stride, dst_row_offset)
+
+
+def twist_gather_subnets(segs: Sequence[GatherSegment], n_subnets, d, dtype):
+    arr = (GatherSegment * len(segs))(*segs)
+    _check(lib().twist_gather_subnets(C.cast(arr, C.c_void_p), len(segs), n_subnets, d, dtype, _stream()),
+           "twist_gather_subnets")
+
+
+def aggregate_segment(dst, dst_f32, sub, cover, pos, n_full, block_rows, dst_row_offset, sub_subnet_stride,
+                      sub_row_offset) -> AggregateSegment:
+    a = lambda v: v if (v is None or isinstance(v, int)) else _ptr(v)
+    return AggregateSegment(a(dst), a(dst_f32), a(sub), a(cover), a(pos), n_full, block_rows, dst_row_offset,
+                            sub_subnet_stride, sub_row_offset)
+
+
+def twist_aggregate(segs: Sequence[AggregateSegment], n_subnets, d, dtype, live_subnets=0xFFFFFFFF):
+    arr = (AggregateSegment * len(segs))(*segs)
+    _check(lib().twist_aggregate(C.cast(arr, C.c_void_p), len(segs), n_subnets, d, dtype, live_subnets, _stream()),
+           "twist_aggregate")
+
+
+def ffn_args(ffn_kind, dtype, n_subnets, tokens, d_model, f_sub, out_scale, lr=0.0, **t) -> FfnArgs:
+    names = ["x", "w_gu", "w_down", "w_gu_master", "w_down_master", "pre", "hh", "y", "dy", "dpre", "dx", "dw_gu",
+             "dw_down"]
+    unknown = set(t) - set(names)
+    assert not unknown, unknown
+    return FfnArgs(ffn_kind, dtype, n_subnets, tokens, d_model, f_sub, out_scale, lr, *[_ptr(t.get(n)) for n in names])
+
+
+def twist_subnet_ffn_fwd(a: FfnArgs):
+    _check(lib().twist_subnet_ffn_fwd(C.byref(a), _stream()), "twist_subnet_ffn_fwd")
+
+
+def twist_subnet_ffn_bwd(a: FfnArgs):
+    _check(lib().twist_subnet_ffn_bwd(C.byref(a), _stream()), "twist_subnet_ffn_bwd")
+
+
+def proj_args(which, dtype, n_subnets, tokens, d_model, n, out_scale, lr=0.0, **t) -> ProjArgs:
+    names = ["in_", "w", "w_master", "out", "d_out", "d_in", "dw"]
+    unknown = set(t) - set(names)
+    assert not unknown, unknown
+    return ProjArgs(which, dtype, n_subnets, tokens, d_model, n, out_scale, lr, *[_ptr(t.get(n)) for n in names])
+
+
+def twist_subnet_attn_proj_fwd(a: ProjArgs):
+    _check(lib().twist_subnet_attn_proj_fwd(C.byref(a), _stream()), "twist_subnet_attn_proj_fwd")
+
+
+def twist_subnet_attn_proj_bwd(a: ProjArgs):
+    _check(lib().twist_subnet_attn_proj_bwd(C.byref(a), _stream()), "twist_subnet_attn_proj_bwd")
+
+
+def twist_mse_workspace_bytes(n_subnets: int) -> int:
+    return lib().twist_mse_workspace_bytes(n_subnets)
+
+
+def twist_mse_fwd_bwd(y, tgt, dy, loss, n_subnets, tokens, width, valid_cols, seg_begin, seg_width, dtype, ws):
+    _check(lib().twist_mse_fwd_bwd(_ptr(y), _ptr(tgt), _ptr(dy), _ptr(loss), n_subnets, tokens, width,
+                                   _ptr(valid_cols), seg_begin, seg_width, dtype, _ptr(ws),
+                                   ws.numel() * ws.element_size(), _stream()),
+           "twist_mse_fwd_bwd")

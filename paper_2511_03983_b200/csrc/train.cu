@@ -1,0 +1,215 @@
+// twist_subnet_ffn_fwd/bwd and twist_subnet_attn_proj_fwd/bwd: the local training step of the
+// S subnets on their dense slices (FFN of App. A: y = C act(W x); projections of the multi-head
+// attention definition).  bf16: grouped tcgen05 GEMMs with fused epilogues.  fp32: plain SIMT
+// kernels (tiny correctness workload only).
+#include "gemm_sm100.cuh"
+#include "glue.cuh"
+
+namespace twist {
+namespace {
+
+#define TWIST_TRY(expr)               \
+  do {                                \
+    int rc__ = (expr);                \
+    if (rc__ != TWIST_OK) return rc__;\
+  } while (0)
+
+int check_ffn(const twist_ffn_args* a) {
+  if (!a) return TWIST_ERR_NULL;
+  if (a->n_subnets <= 0 || a->tokens <= 0 || a->d_model <= 0 || a->f_sub <= 0) return TWIST_ERR_SHAPE;
+  if (a->ffn_kind < TWIST_FFN_RELU || a->ffn_kind > TWIST_FFN_SWIGLU) return TWIST_ERR_SHAPE;
+  if (a->dtype != TWIST_FP32 && a->dtype != TWIST_BF16) return TWIST_ERR_SHAPE;
+  if (a->dtype == TWIST_BF16 && (a->d_model % 8 || a->f_sub % 8)) return TWIST_ERR_SHAPE;
+  return TWIST_OK;
+}
+
+GemmParams base_params(int M, int N, int K, int groups, float scale) {
+  GemmParams p;
+  memset(&p, 0, sizeof(p));
+  p.M = M; p.N = N; p.K = K; p.groups = groups; p.scale = scale;
+  return p;
+}
+
+}  // namespace
+}  // namespace twist
+
+using namespace twist;
+
+extern "C" int32_t twist_subnet_ffn_fwd(const twist_ffn_args* a, void* stream) {
+  TWIST_TRY(check_ffn(a));
+  if (!a->x || !a->w_gu || !a->w_down || !a->pre || !a->hh || !a->y) return TWIST_ERR_NULL;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int S = a->n_subnets, T = a->tokens, d = a->d_model, f = a->f_sub;
+  const bool swiglu = a->ffn_kind == TWIST_FFN_SWIGLU;
+  const int gf = swiglu ? 2 * f : f;
+  if (a->dtype == TWIST_FP32) {
+    const float* x = static_cast<const float*>(a->x);
+    float* pre = static_cast<float*>(a->pre);
+    float* hh = static_cast<float*>(a->hh);
+    TWIST_TRY(sgemm_f32(false, true, x, static_cast<const float*>(a->w_gu), pre, T, gf, d, d, d, gf, (long long)T * d,
+                        (long long)gf * d, (long long)T * gf, S, 1.f, st));
+    TWIST_TRY(act_fwd_f32(pre, hh, (long long)S * T, f, a->ffn_kind, st));
+    return sgemm_f32(false, false, hh, static_cast<const float*>(a->w_down), static_cast<float*>(a->y), T, d, f, f, d,
+                     d, (long long)T * f, (long long)f * d, (long long)T * d, S, a->out_scale, st);
+  }
+  // pre (and hh) = epilogue(X W_gu^T)
+  GemmParams p = base_params(T, f, d, S, 1.f);
+  p.out0 = static_cast<__nv_bfloat16*>(a->pre);
+  p.out1 = static_cast<__nv_bfloat16*>(a->hh);
+  p.b_split = f;
+  p.act_kind = a->ffn_kind;
+  TWIST_TRY(launch_gemm_bf16(0, swiglu ? EPI_SWIGLU_FWD : EPI_ACT_FWD, GemmOperand{a->x, T, d},
+                             GemmOperand{a->w_gu, gf, d}, p, st));
+  // Y = out_scale * hh W_down
+  GemmParams q = base_params(T, d, f, S, a->out_scale);
+  q.out0 = static_cast<__nv_bfloat16*>(a->y);
+  return launch_gemm_bf16(1, EPI_STORE, GemmOperand{a->hh, T, f}, GemmOperand{a->w_down, f, d}, q, st);
+}
+
+extern "C" int32_t twist_subnet_ffn_bwd(const twist_ffn_args* a, void* stream) {
+  TWIST_TRY(check_ffn(a));
+  if (!a->x || !a->w_gu || !a->w_down || !a->pre || !a->hh || !a->dy || !a->dpre) return TWIST_ERR_NULL;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int S = a->n_subnets, T = a->tokens, d = a->d_model, f = a->f_sub;
+  const bool swiglu = a->ffn_kind == TWIST_FFN_SWIGLU;
+  const int gf = swiglu ? 2 * f : f;
+  if (a->dtype == TWIST_FP32) {
+    if (!a->dw_gu || !a->dw_down) return TWIST_ERR_NULL;
+    const float* x = static_cast<const float*>(a->x);
+    const float* dy = static_cast<const float*>(a->dy);
+    const float* pre = static_cast<const float*>(a->pre);
+    const float* hh = static_cast<const float*>(a->hh);
+    float* dpre = static_cast<float*>(a->dpre);
+    float* wgu = static_cast<float*>(a->w_gu);
+    float* wd = static_cast<float*>(a->w_down);
+    // dHh = out_scale * dY W_down^T, parked in dpre (SwiGLU: in the "up" half), then through the activation in place
+    TWIST_TRY(sgemm_f32(false, true, dy, wd, dpre + (swiglu ? f : 0), T, f, d, d, d, gf, (long long)T * d,
+                        (long long)f * d, (long long)T * gf, S, a->out_scale, st));
+    TWIST_TRY(act_bwd_f32(pre, dpre, (long long)S * T, f, a->ffn_kind, st));
+    if (a->dx)
+      TWIST_TRY(sgemm_f32(false, false, dpre, wgu, static_cast<float*>(a->dx), T, d, gf, gf, d, d, (long long)T * gf,
+                          (long long)gf * d, (long long)T * d, S, 1.f, st));
+    TWIST_TRY(sgemm_f32(true, false, dpre, x, a->dw_gu, gf, d, T, gf, d, d, (long long)T * gf, (long long)T * d,
+                        (long long)gf * d, S, 1.f, st));
+    TWIST_TRY(sgemm_f32(true, false, hh, dy, a->dw_down, f, d, T, f, d, d, (long long)T * f, (long long)T * d,
+                        (long long)f * d, S, a->out_scale, st));
+    if (a->lr != 0.f) {
+      TWIST_TRY(sgd_f32(wgu, a->dw_gu, a->lr, (long long)S * gf * d, st));
+      TWIST_TRY(sgd_f32(wd, a->dw_down, a->lr, (long long)S * f * d, st));
+    }
+    return TWIST_OK;
+  }
+  if (a->lr != 0.f && (!a->w_gu_master || !a->w_down_master)) return TWIST_ERR_NULL;
+  // dpre = act'(pre) * (out_scale * dY W_down^T)
+  GemmParams p = base_params(T, f, d, S, a->out_scale);
+  p.out0 = static_cast<__nv_bfloat16*>(a->dpre);
+  p.in0 = static_cast<const __nv_bfloat16*>(a->pre);
+  p.act_kind = a->ffn_kind;
+  TWIST_TRY(launch_gemm_bf16(0, swiglu ? EPI_DSWIGLU : EPI_DACT, GemmOperand{a->dy, T, d}, GemmOperand{a->w_down, f, d},
+                             p, st));
+  // dX = dpre W_gu   (before the weights are updated)
+  if (a->dx) {
+    GemmParams q = base_params(T, d, gf, S, 1.f);
+    q.out0 = static_cast<__nv_bfloat16*>(a->dx);
+    TWIST_TRY(launch_gemm_bf16(1, EPI_STORE, GemmOperand{a->dpre, T, gf}, GemmOperand{a->w_gu, gf, d}, q, st));
+  }
+  // dW_down = out_scale * hh^T dY, fused SGD
+  GemmParams r = base_params(f, d, T, S, a->out_scale);
+  r.out0 = static_cast<__nv_bfloat16*>(a->w_down);
+  r.master = a->w_down_master;
+  r.dw = a->dw_down;
+  r.lr = a->lr;
+  TWIST_TRY(launch_gemm_bf16(2, EPI_SGD, GemmOperand{a->hh, T, f}, GemmOperand{a->dy, T, d}, r, st));
+  // dW_gu = dpre^T X, fused SGD
+  GemmParams u = base_params(gf, d, T, S, 1.f);
+  u.out0 = static_cast<__nv_bfloat16*>(a->w_gu);
+  u.master = a->w_gu_master;
+  u.dw = a->dw_gu;
+  u.lr = a->lr;
+  return launch_gemm_bf16(2, EPI_SGD, GemmOperand{a->dpre, T, gf}, GemmOperand{a->x, T, d}, u, st);
+}
+
+static int check_proj(const twist_proj_args* a) {
+  if (!a) return TWIST_ERR_NULL;
+  if (a->n_subnets <= 0 || a->tokens <= 0 || a->d_model <= 0 || a->n <= 0) return TWIST_ERR_SHAPE;
+  if (a->which != TWIST_PROJ_QKV && a->which != TWIST_PROJ_O) return TWIST_ERR_SHAPE;
+  if (a->dtype != TWIST_FP32 && a->dtype != TWIST_BF16) return TWIST_ERR_SHAPE;
+  if (a->dtype == TWIST_BF16 && (a->d_model % 8 || a->n % 8)) return TWIST_ERR_SHAPE;
+  return TWIST_OK;
+}
+
+extern "C" int32_t twist_subnet_attn_proj_fwd(const twist_proj_args* a, void* stream) {
+  TWIST_TRY(check_proj(a));
+  if (!a->in || !a->w || !a->out) return TWIST_ERR_NULL;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int S = a->n_subnets, T = a->tokens, d = a->d_model, n = a->n;
+  if (a->dtype == TWIST_FP32) {
+    const float* in = static_cast<const float*>(a->in);
+    const float* w = static_cast<const float*>(a->w);
+    float* out = static_cast<float*>(a->out);
+    if (a->which == TWIST_PROJ_QKV)
+      return sgemm_f32(false, true, in, w, out, T, n, d, d, d, n, (long long)T * d, (long long)n * d, (long long)T * n,
+                       S, a->out_scale, st);
+    return sgemm_f32(false, false, in, w, out, T, d, n, n, d, d, (long long)T * n, (long long)n * d, (long long)T * d, S,
+                     a->out_scale, st);
+  }
+  if (a->which == TWIST_PROJ_QKV) {
+    GemmParams p = base_params(T, n, d, S, a->out_scale);
+    p.out0 = static_cast<__nv_bfloat16*>(a->out);
+    return launch_gemm_bf16(0, EPI_STORE, GemmOperand{a->in, T, d}, GemmOperand{a->w, n, d}, p, st);
+  }
+  GemmParams p = base_params(T, d, n, S, a->out_scale);
+  p.out0 = static_cast<__nv_bfloat16*>(a->out);
+  return launch_gemm_bf16(1, EPI_STORE, GemmOperand{a->in, T, n}, GemmOperand{a->w, n, d}, p, st);
+}
+
+extern "C" int32_t twist_subnet_attn_proj_bwd(const twist_proj_args* a, void* stream) {
+  TWIST_TRY(check_proj(a));
+  if (!a->in || !a->w || !a->d_out) return TWIST_ERR_NULL;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int S = a->n_subnets, T = a->tokens, d = a->d_model, n = a->n;
+  const bool qkv = a->which == TWIST_PROJ_QKV;
+  const int w_in = qkv ? d : n;       // width of `in`
+  const int w_out = qkv ? n : d;      // width of `d_out`
+  if (a->dtype == TWIST_FP32) {
+    if (!a->dw) return TWIST_ERR_NULL;
+    const float* in = static_cast<const float*>(a->in);
+    const float* dout = static_cast<const float*>(a->d_out);
+    float* w = static_cast<float*>(a->w);
+    if (a->d_in) {
+      if (qkv)   // dX = dQKV W
+        TWIST_TRY(sgemm_f32(false, false, dout, w, static_cast<float*>(a->d_in), T, d, n, n, d, d, (long long)T * n,
+                            (long long)n * d, (long long)T * d, S, a->out_scale, st));
+      else       // dA = out_scale * dY W^T
+        TWIST_TRY(sgemm_f32(false, true, dout, w, static_cast<float*>(a->d_in), T, n, d, d, d, n, (long long)T * d,
+                            (long long)n * d, (long long)T * n, S, a->out_scale, st));
+    }
+    if (qkv)     // dW [n][d] = dQKV^T X
+      TWIST_TRY(sgemm_f32(true, false, dout, in, a->dw, n, d, T, n, d, d, (long long)T * n, (long long)T * d,
+                          (long long)n * d, S, a->out_scale, st));
+    else         // dW [n][d] = out_scale * A^T dY
+      TWIST_TRY(sgemm_f32(true, false, in, dout, a->dw, n, d, T, n, d, d, (long long)T * n, (long long)T * d,
+                          (long long)n * d, S, a->out_scale, st));
+    if (a->lr != 0.f) TWIST_TRY(sgd_f32(w, a->dw, a->lr, (long long)S * n * d, st));
+    return TWIST_OK;
+  }
+  if (a->lr != 0.f && !a->w_master) return TWIST_ERR_NULL;
+  if (a->d_in) {
+    if (qkv) {
+      GemmParams p = base_params(T, d, n, S, a->out_scale);
+      p.out0 = static_cast<__nv_bfloat16*>(a->d_in);
+      TWIST_TRY(launch_gemm_bf16(1, EPI_STORE, GemmOperand{a->d_out, T, n}, GemmOperand{a->w, n, d}, p, st));
+    } else {
+      GemmParams p = base_params(T, n, d, S, a->out_scale);
+      p.out0 = static_cast<__nv_bfloat16*>(a->d_in);
+      TWIST_TRY(launch_gemm_bf16(0, EPI_STORE, GemmOperand{a->d_out, T, d}, GemmOperand{a->w, n, d}, p, st));
+    }
+  }
+  GemmParams r = base_params(n, d, T, S, a->out_scale);
+  r.out0 = static_cast<__nv_bfloat16*>(a->w);
+  r.master = a->w_master;
+  r.dw = a->dw;
+  r.lr = a->lr;
+  if (qkv) return launch_gemm_bf16(2, EPI_SGD, GemmOperand{a->d_out, T, w_out}, GemmOperand{a->in, T, w_in}, r, st);
+  return launch_gemm_bf16(2, EPI_SGD, GemmOperand{a->in, T, w_in}, GemmOperand{a->d_out, T, w_out}, r, st);
+}

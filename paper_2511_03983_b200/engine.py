@@ -1,0 +1,230 @@
+"""Sequencing of one TwIST round on one GPU (BLOCKWISE composition).
+
+This module only allocates device buffers (torch) and calls the C ABI in order:
+sample masks -> per layer { gather -> K local steps (forward, MSE, backward with fused
+SGD) for the FFN block, the QKV projection and the output projection -> aggregate }.
+Every arithmetic step runs in the CUDA library; nothing here computes on tensors.
+
+Layers are streamed: slices, masters and activations exist for one layer at a time,
+which is what lets the 7B-shaped workloads fit (per layer ~2.4 GB of slices + masters
+at S=8, keep 25%, instead of 78 GB for all 32 layers).
+"""
+from __future__ import annotations
+
+import math
+from typing import Dict, List, Optional
+
+import torch
+
+from . import binding as B
+from .inputs import DTYPE_BF16, FFN_SWIGLU, Workload
+
+
+def _tdtype(w: Workload):
+    return torch.bfloat16 if w.dtype == DTYPE_BF16 else torch.float32
+
+
+class RoundEngine:
+    BLOCKS = ("ffn", "qkv", "o")
+
+    def __init__(self, w: Workload, device: str = "cuda", keep_f32_full: bool = False, compute_dx: bool = True,
+                 dump_grads: bool = False):
+        self.w, self.dev = w, torch.device(device)
+        self.compute_dx, self.dump_grads = compute_dx, dump_grads or w.dtype != DTYPE_BF16
+        td, dev = _tdtype(w), self.dev
+        S, T, d, f = w.n_subnets, w.tokens, w.d_model, w.f_sub
+        self.g = 2 if w.ffn_kind == FFN_SWIGLU else 1
+        gf = self.g * f
+        L, F = w.n_layers, w.d_ff
+        self.has_attn = w.n_heads > 0
+        bf16 = w.dtype == DTYPE_BF16
+        # full model (the central model of the paper's server)
+        self.full: Dict[str, torch.Tensor] = {"up": torch.empty(L, F, d, dtype=td, device=dev),
+                                              "down": torch.empty(L, F, d, dtype=td, device=dev)}
+        if self.g == 2:
+            self.full["gate"] = torch.empty(L, F, d, dtype=td, device=dev)
+        if self.has_attn:
+            H, Hkv, dh = w.n_heads, w.n_kv_heads, w.d_head
+            self.kv_max = min(Hkv, w.head_keep)
+            self.a_sub = w.head_keep * dh
+            self.nq = self.a_sub + 2 * self.kv_max * dh
+            self.full["qkv"] = torch.empty(L, (H + 2 * Hkv) * dh, d, dtype=td, device=dev)
+            self.full["o"] = torch.empty(L, H * dh, d, dtype=td, device=dev)
+        self.full_f32 = ({m: torch.empty(v.shape, dtype=torch.float32, device=dev) for m, v in self.full.items()}
+                         if (keep_f32_full and bf16) else None)
+        # blueprints and aggregator index data, all layers
+        nb = w.n_ffn_blocks
+        i32 = dict(dtype=torch.int32, device=dev)
+        self.idx_ffn = torch.empty(L, S, w.ffn_keep, **i32)
+        self.cover_ffn = torch.empty(L, nb, **i32)
+        self.pos_ffn = torch.empty(L, S, nb, **i32)
+        if self.has_attn:
+            self.idx_head = torch.empty(L, S, w.head_keep, **i32)
+            self.cover_head = torch.empty(L, w.n_heads, **i32)
+            self.pos_head = torch.empty(L, S, w.n_heads, **i32)
+            self.kv_idx = torch.empty(L, S, w.n_kv_heads, **i32)
+            self.kv_count = torch.empty(L, S, **i32)
+            self.kv_cols = torch.empty(L, S, **i32)
+            self.kv_cover = torch.empty(L, w.n_kv_heads, **i32)
+            self.kv_pos = torch.empty(L, S, w.n_kv_heads, **i32)
+        # slices of one layer (+ fp32 masters in bf16 mode)
+        def sl(rows):
+            t = torch.empty(S, rows, d, dtype=td, device=dev)
+            return t, (torch.empty(S, rows, d, dtype=torch.float32, device=dev) if bf16 else None)
+        self.w_gu, self.w_gu_m = sl(gf)
+        self.w_down, self.w_down_m = sl(f)
+        if self.has_attn:
+            self.w_qkv, self.w_qkv_m = sl(self.nq)
+            self.w_o, self.w_o_m = sl(self.a_sub)
+        # activations of one (layer, step)
+        act = lambda width: torch.empty(S, T, width, dtype=td, device=dev)
+        self.pre, self.dpre, self.hh = act(gf), act(gf), act(f)
+        self.y, self.dy = act(d), act(d)
+        self.dx = act(d) if compute_dx else None
+        if self.has_attn:
+            self.qkv_out, self.dqkv = act(self.nq), act(self.nq)
+            self.da = act(self.a_sub) if compute_dx else None
+        f32 = lambda *shape: torch.empty(*shape, dtype=torch.float32, device=dev)
+        self.dw_gu = f32(S, gf, d) if self.dump_grads else None
+        self.dw_down = f32(S, f, d) if self.dump_grads else None
+        if self.has_attn:
+            self.dw_qkv = f32(S, self.nq, d) if self.dump_grads else None
+            self.dw_o = f32(S, self.a_sub, d) if self.dump_grads else None
+        self.loss = torch.zeros(L, 3, max(1, w.local_steps), S, dtype=torch.float32, device=dev)
+        self.ws = torch.empty(B.twist_mse_workspace_bytes(S), dtype=torch.uint8, device=dev)
+        self.alpha_f = math.sqrt(w.n_ffn_blocks / w.ffn_keep)
+        self.alpha_a = math.sqrt(w.n_heads / w.head_keep) if self.has_attn else 1.0
+        # batches: lists over the local step k of [S][T][width] tensors
+        self.X: List[torch.Tensor] = []
+        self.Td: List[torch.Tensor] = []
+        self.Tq: List[torch.Tensor] = []
+        self.A: List[torch.Tensor] = []
+        self.launches = 0
+
+    # ------------------------------------------------------------------ steps of the round
+    def sample_masks(self, rnd: int):
+        w = self.w
+        B.twist_sample_masks(w.seed_mask, rnd, 0, w.n_layers, B.KIND_FFN, w.n_ffn_blocks, w.n_subnets, w.ffn_keep,
+                             list(w.common_ffn), w.sample_mode, self.idx_ffn, self.cover_ffn, self.pos_ffn)
+        self.launches += 2
+        if self.has_attn:
+            B.twist_sample_masks(w.seed_mask, rnd, 0, w.n_layers, B.KIND_HEAD, w.n_heads, w.n_subnets, w.head_keep,
+                                 list(w.common_heads), w.sample_mode, self.idx_head, self.cover_head, self.pos_head)
+            B.twist_kv_groups(self.idx_head, w.n_layers, w.n_subnets, w.head_keep, w.n_heads, w.n_kv_heads, w.d_head,
+                              self.kv_idx, self.kv_count, self.kv_cols, self.kv_cover, self.kv_pos)
+            self.launches += 4
+
+    def gather_layer(self, l: int, which=("ffn", "attn")):
+        w, d = self.w, self.w.d_model
+        f, gf = w.f_sub, self.g * w.f_sub
+        segs = []
+        if "ffn" in which:
+            if self.g == 2:
+                segs.append(B.gather_segment(self.full["gate"][l], self.w_gu, self.w_gu_m, self.idx_ffn[l], None,
+                                             w.ffn_keep, w.ffn_keep, w.ffn_block, 0, gf * d, 0))
+            segs.append(B.gather_segment(self.full["up"][l], self.w_gu, self.w_gu_m, self.idx_ffn[l], None,
+                                         w.ffn_keep, w.ffn_keep, w.ffn_block, 0, gf * d, f if self.g == 2 else 0))
+            segs.append(B.gather_segment(self.full["down"][l], self.w_down, self.w_down_m, self.idx_ffn[l], None,
+                                         w.ffn_keep, w.ffn_keep, w.ffn_block, 0, f * d, 0))
+        if self.has_attn and "attn" in which:
+            H, Hkv, dh = w.n_heads, w.n_kv_heads, w.d_head
+            qkv = self.full["qkv"][l]
+            segs.append(B.gather_segment(qkv, self.w_qkv, self.w_qkv_m, self.idx_head[l], None, w.head_keep,
+                                         w.head_keep, dh, 0, self.nq * d, 0))
+            segs.append(B.gather_segment(qkv, self.w_qkv, self.w_qkv_m, self.kv_idx[l], self.kv_count[l], Hkv,
+                                         self.kv_max, dh, H * dh, self.nq * d, self.a_sub))
+            segs.append(B.gather_segment(qkv, self.w_qkv, self.w_qkv_m, self.kv_idx[l], self.kv_count[l], Hkv,
+                                         self.kv_max, dh, (H + Hkv) * dh, self.nq * d, self.a_sub + self.kv_max * dh))
+            segs.append(B.gather_segment(self.full["o"][l], self.w_o, self.w_o_m, self.idx_head[l], None, w.head_keep,
+                                         w.head_keep, dh, 0, self.a_sub * d, 0))
+        B.twist_gather_subnets(segs, w.n_subnets, d, w.dtype)
+        self.launches += 1
+
+    def aggregate_layer(self, l: int, live: int = 0xFFFFFFFF, which=("ffn", "attn")):
+        w, d = self.w, self.w.d_model
+        f, gf = w.f_sub, self.g * w.f_sub
+        bf16 = w.dtype == DTYPE_BF16
+        f32 = (lambda m: self.full_f32[m][l]) if self.full_f32 is not None else (lambda m: None)
+        sub = lambda lo, master: master if bf16 else lo
+        nb = w.n_ffn_blocks
+        segs = []
+        if "ffn" in which:
+            if self.g == 2:
+                segs.append(B.aggregate_segment(self.full["gate"][l], f32("gate"), sub(self.w_gu, self.w_gu_m),
+                                                self.cover_ffn[l], self.pos_ffn[l], nb, w.ffn_block, 0, gf * d, 0))
+            segs.append(B.aggregate_segment(self.full["up"][l], f32("up"), sub(self.w_gu, self.w_gu_m),
+                                            self.cover_ffn[l], self.pos_ffn[l], nb, w.ffn_block, 0, gf * d,
+                                            f if self.g == 2 else 0))
+            segs.append(B.aggregate_segment(self.full["down"][l], f32("down"), sub(self.w_down, self.w_down_m),
+                                            self.cover_ffn[l], self.pos_ffn[l], nb, w.ffn_block, 0, f * d, 0))
+        if self.has_attn and "attn" in which:
+            H, Hkv, dh = w.n_heads, w.n_kv_heads, w.d_head
+            q_sub = sub(self.w_qkv, self.w_qkv_m)
+            segs.append(B.aggregate_segment(self.full["qkv"][l], f32("qkv"), q_sub, self.cover_head[l],
+                                            self.pos_head[l], H, dh, 0, self.nq * d, 0))
+            segs.append(B.aggregate_segment(self.full["qkv"][l], f32("qkv"), q_sub, self.kv_cover[l], self.kv_pos[l],
+                                            Hkv, dh, H * dh, self.nq * d, self.a_sub))
+            segs.append(B.aggregate_segment(self.full["qkv"][l], f32("qkv"), q_sub, self.kv_cover[l], self.kv_pos[l],
+                                            Hkv, dh, (H + Hkv) * dh, self.nq * d, self.a_sub + self.kv_max * dh))
+            segs.append(B.aggregate_segment(self.full["o"][l], f32("o"), sub(self.w_o, self.w_o_m), self.cover_head[l],
+                                            self.pos_head[l], H, dh, 0, self.a_sub * d, 0))
+        B.twist_aggregate(segs, w.n_subnets, d, w.dtype, live)
+        self.launches += 1
+
+    def _mse(self, y, tgt, dy, loss, width, valid_cols=None, seg_begin=0, seg_width=0):
+        w = self.w
+        B.twist_mse_fwd_bwd(y, tgt, dy, loss, w.n_subnets, w.tokens, width, valid_cols, seg_begin, seg_width, w.dtype,
+                            self.ws)
+        self.launches += 2
+
+    def ffn_step(self, l: int, k: int, lr: Optional[float] = None):
+        w = self.w
+        lr = w.lr if lr is None else lr
+        a = B.ffn_args(w.ffn_kind, w.dtype, w.n_subnets, w.tokens, w.d_model, w.f_sub, self.alpha_f, lr,
+                       x=self.X[k], w_gu=self.w_gu, w_down=self.w_down, w_gu_master=self.w_gu_m,
+                       w_down_master=self.w_down_m, pre=self.pre, hh=self.hh, y=self.y, dy=self.dy, dpre=self.dpre,
+                       dx=self.dx, dw_gu=self.dw_gu, dw_down=self.dw_down)
+        B.twist_subnet_ffn_fwd(a)
+        self._mse(self.y, self.Td[k], self.dy, self.loss[l, 0, k], w.d_model)
+        B.twist_subnet_ffn_bwd(a)
+        bf16 = w.dtype == DTYPE_BF16
+        self.launches += (2 + 3 + (1 if self.compute_dx else 0)) if bf16 else (3 + 4 + (1 if self.compute_dx else 0) + 2)
+
+    def qkv_step(self, l: int, k: int, lr: Optional[float] = None):
+        w = self.w
+        lr = w.lr if lr is None else lr
+        a = B.proj_args(B.PROJ_QKV, w.dtype, w.n_subnets, w.tokens, w.d_model, self.nq, 1.0, lr, in_=self.X[k],
+                        w=self.w_qkv, w_master=self.w_qkv_m, out=self.qkv_out, d_out=self.dqkv, d_in=self.dx,
+                        dw=self.dw_qkv)
+        B.twist_subnet_attn_proj_fwd(a)
+        ragged = self.w.n_kv_heads != self.w.n_heads
+        self._mse(self.qkv_out, self.Tq[k], self.dqkv, self.loss[l, 1, k], self.nq,
+                  self.kv_cols[l] if ragged else None, self.a_sub, self.kv_max * w.d_head)
+        B.twist_subnet_attn_proj_bwd(a)
+        self.launches += 1 + 1 + (1 if self.compute_dx else 0) + (0 if w.dtype == DTYPE_BF16 else 1)
+
+    def o_step(self, l: int, k: int, lr: Optional[float] = None):
+        w = self.w
+        lr = w.lr if lr is None else lr
+        a = B.proj_args(B.PROJ_O, w.dtype, w.n_subnets, w.tokens, w.d_model, self.a_sub, self.alpha_a, lr,
+                        in_=self.A[k], w=self.w_o, w_master=self.w_o_m, out=self.y, d_out=self.dy, d_in=self.da,
+                        dw=self.dw_o)
+        B.twist_subnet_attn_proj_fwd(a)
+        self._mse(self.y, self.Td[k], self.dy, self.loss[l, 2, k], w.d_model)
+        B.twist_subnet_attn_proj_bwd(a)
+        self.launches += 1 + 1 + (1 if self.compute_dx else 0) + (0 if w.dtype == DTYPE_BF16 else 1)
+
+    def run_layer(self, l: int):
+        self.gather_layer(l)
+        for k in range(self.w.local_steps):
+            self.ffn_step(l, k)
+            if self.has_attn:
+                self.qkv_step(l, k)
+                self.o_step(l, k)
+        self.aggregate_layer(l)
+
+    def run_round(self, rnd: int):
+        """One full round: resample every layer's blueprints, then stream the layers."""
+        self.sample_masks(rnd)
+        for l in range(self.w.n_layers):
+            self.run_layer(l)

@@ -1,0 +1,76 @@
+"""The C-ABI library loads and exports every symbol include/twist.h declares; host-side
+argument checks return the documented status codes without touching a GPU."""
+import ctypes as C
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _declared():
+    text = open(os.path.join(ROOT, "include", "twist.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(twist_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol():
+    from paper_2511_03983_b200 import binding as B
+    names = _declared()
+    assert len(names) >= 14
+    h = B.lib()
+    for n in names:
+        assert hasattr(h, n), n
+    assert sorted(B.EXPORTS) == names
+    assert B.twist_abi_version() == 1
+
+
+def test_status_strings():
+    from paper_2511_03983_b200 import binding as B
+    h = B.lib()
+    assert h.twist_strerror(0) == b"ok"
+    for code in range(-8, 0):
+        assert len(h.twist_strerror(code)) > 3
+
+
+def test_host_side_argument_checks():
+    from paper_2511_03983_b200 import binding as B
+    h = B.lib()
+    dummy = C.c_void_p(0x1000)   # never dereferenced: every call below fails validation first
+    # sampler: null, shape, unsupported, infeasible (size bound of Sec. 3.1), bad common list
+    f = h.twist_sample_masks
+    assert f(1, 0, 0, 1, 0, 12, 4, 6, None, 0, 0, None, dummy, dummy, None) == B.ERR_NULL
+    assert f(1, 0, 0, 1, 0, 0, 4, 6, None, 0, 0, dummy, dummy, dummy, None) == B.ERR_SHAPE
+    assert f(1, 0, 0, 1, 0, 20000, 4, 6000, None, 0, 0, dummy, dummy, dummy, None) == B.ERR_UNSUPPORTED
+    assert f(1, 0, 0, 1, 0, 12, 33, 6, None, 0, 0, dummy, dummy, dummy, None) == B.ERR_UNSUPPORTED
+    assert f(1, 0, 0, 1, 0, 11008, 2, 2752, None, 0, B.MODE_COVER, dummy, dummy, dummy, None) == B.ERR_INFEASIBLE
+    assert f(1, 0, 0, 1, 0, 12, 4, 13, None, 0, B.MODE_IID, dummy, dummy, dummy, None) == B.ERR_INFEASIBLE
+    bad = (C.c_int32 * 2)(5, 3)
+    assert f(1, 0, 0, 1, 0, 12, 4, 6, C.cast(bad, C.c_void_p), 2, 0, dummy, dummy, dummy, None) == B.ERR_BAD_INDEX
+    # gather / aggregate
+    assert h.twist_gather_subnets(None, 1, 2, 64, B.BF16, None) == B.ERR_NULL
+    seg = B.GatherSegment(0x1000, 0x2000, None, 0x3000, None, 4, 4, 1, 0, 0, 256, 0)
+    arr = (B.GatherSegment * 1)(seg)
+    assert h.twist_gather_subnets(C.cast(arr, C.c_void_p), 1, 2, 63, B.BF16, None) == B.ERR_SHAPE     # row not 16 B
+    assert h.twist_gather_subnets(C.cast(arr, C.c_void_p), 9, 2, 64, B.BF16, None) == B.ERR_SHAPE     # too many segments
+    assert h.twist_aggregate(None, 1, 2, 64, B.BF16, 3, None) == B.ERR_NULL
+    # local steps
+    a = B.FfnArgs(B.FFN_SWIGLU, B.BF16, 2, 128, 64, 100, 1.0, 0.0)       # f_sub not a multiple of 8
+    assert h.twist_subnet_ffn_fwd(C.byref(a), None) == B.ERR_SHAPE
+    a = B.FfnArgs(B.FFN_SWIGLU, B.BF16, 2, 128, 64, 128, 1.0, 0.0)       # all pointers NULL
+    assert h.twist_subnet_ffn_fwd(C.byref(a), None) == B.ERR_NULL
+    assert h.twist_subnet_ffn_bwd(C.byref(a), None) == B.ERR_NULL
+    p = B.ProjArgs(7, B.BF16, 2, 128, 64, 64, 1.0, 0.0)
+    assert h.twist_subnet_attn_proj_fwd(C.byref(p), None) == B.ERR_SHAPE
+    # mse workspace
+    assert B.twist_mse_workspace_bytes(4) == 4 * 1024 * 4
+    assert h.twist_mse_fwd_bwd(dummy, dummy, dummy, dummy, 2, 8, 64, None, 0, 0, B.BF16, None, 0, None) == B.ERR_WORKSPACE
+
+
+def test_missing_library_fails_loudly(monkeypatch, tmp_path):
+    from paper_2511_03983_b200 import binding as B
+    monkeypatch.setattr(B, "_lib_handle", None)
+    monkeypatch.setattr(B, "LIB_PATH", str(tmp_path / "nope.so"))
+    with pytest.raises(FileNotFoundError):
+        B.lib()

@@ -1,0 +1,414 @@
+"""Parity of the CUDA path (through the C ABI) with the CPU oracle on the same seeded inputs.
+
+Bars: masks, index data and gather output bit-exact; aggregate within 1e-6 relative per
+element; bf16 GEMM outputs and gradients within 2e-2 relative Frobenius error of the fp64
+oracle (which mirrors the bf16 rounding points of stored tensors); fp32 path within 1e-4.
+"""
+import math
+from dataclasses import replace
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import twist_oracle as o
+from paper_2511_03983_b200 import inputs as I
+
+pytestmark = pytest.mark.gpu
+
+GEMM_TOL = 2e-2
+AGG_TOL = 1e-6
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_2511_03983_b200 import binding
+    binding.lib()
+    return binding
+
+
+def dev(x, dtype=None):
+    t = torch.from_numpy(np.ascontiguousarray(x))
+    if dtype is not None:
+        t = t.to(dtype)
+    return t.cuda()
+
+
+def host(t):
+    return t.detach().float().cpu().numpy().astype(np.float64) if t.is_floating_point() else t.detach().cpu().numpy()
+
+
+def rel_fro(got, want):
+    return float(np.linalg.norm(got - want) / max(np.linalg.norm(want), 1e-300))
+
+
+def check_status(B):
+    assert B.twist_device_status() == 0
+
+
+# --------------------------------------------------------------------------------------------- sampler
+
+def _gpu_masks(B, seed, rnd, layer_begin, n_layers, kind, n_full, S, n_sub, common, mode):
+    idx = torch.full((n_layers, S, n_sub), -7, dtype=torch.int32, device="cuda")
+    cover = torch.full((n_layers, n_full), -7, dtype=torch.int32, device="cuda")
+    pos = torch.full((n_layers, S, n_full), -7, dtype=torch.int32, device="cuda")
+    B.twist_sample_masks(seed, rnd, layer_begin, n_layers, kind, n_full, S, n_sub, common, mode, idx, cover, pos)
+    torch.cuda.synchronize()
+    return idx.cpu().numpy(), cover.cpu().numpy().view(np.uint32), pos.cpu().numpy()
+
+
+@pytest.mark.parametrize("n_full,S,n_sub,common,mode,kind,n_layers", [
+    (256, 2, 128, [], 0, 0, 1),            # config 1
+    (3072, 4, 1536, [], 0, 0, 12),         # config 2 FFN
+    (12, 4, 6, [], 0, 1, 12),              # config 2 heads
+    (5632, 4, 2816, [], 0, 0, 3),          # config 3 FFN
+    (32, 4, 16, [], 0, 1, 22),             # config 3 heads
+    (11008, 8, 2752, [], 0, 0, 3),         # config 4 FFN
+    (32, 8, 8, [], 0, 1, 32),              # config 4 heads
+    (11008, 2, 2752, [], 1, 0, 2),         # config 5 cells (IID)
+    (11008, 16, 8256, [], 1, 0, 2),
+    (11008, 4, 5504, [], 1, 0, 1),
+    (100, 7, 16, [3], 0, 0, 2), (12, 3, 6, [0, 7], 0, 1, 2), (40, 3, 17, [1, 2, 39], 1, 0, 2),   # common blocks
+    (16384, 2, 8192, [], 0, 0, 1),         # maximum block count
+    (7, 1, 7, [], 0, 0, 1), (1, 1, 1, [], 0, 1, 1), (33, 32, 2, [], 0, 0, 1),   # degenerate
+])
+def test_masks_bit_exact(B, n_full, S, n_sub, common, mode, kind, n_layers):
+    seed, rnd, l0 = 3000 + n_full, 2, 5
+    idx, cover, pos = _gpu_masks(B, seed, rnd, l0, n_layers, kind, n_full, S, n_sub, common, mode)
+    for l in range(n_layers):
+        A = o.sample_blueprint(n_full, S, n_sub, common, seed, rnd, l0 + l, kind, mode)
+        assert np.array_equal(idx[l], A), (l,)
+        c, _, p = o.cover_and_pos(A, n_full)
+        assert np.array_equal(cover[l], c)
+        assert np.array_equal(pos[l], p)
+    check_status(B)
+
+
+def test_kv_groups_bit_exact(B):
+    H, Hkv, S, keep, L, dh = 32, 4, 4, 3, 6, 64       # few kept heads so that some groups are dropped
+    idx, _, _ = _gpu_masks(B, 17, 0, 0, L, 1, H, S, keep, [], I.MODE_IID)
+    t = lambda *s: torch.full(s, -7, dtype=torch.int32, device="cuda")
+    kv_idx, kv_count, kv_cols, kv_cover, kv_pos = t(L, S, Hkv), t(L, S), t(L, S), t(L, Hkv), t(L, S, Hkv)
+    B.twist_kv_groups(dev(idx), L, S, keep, H, Hkv, dh, kv_idx, kv_count, kv_cols, kv_cover, kv_pos)
+    torch.cuda.synchronize()
+    saw_ragged = False
+    for l in range(L):
+        want_idx, want_count = o.kv_groups(idx[l], H, Hkv)
+        assert np.array_equal(kv_idx[l].cpu().numpy(), want_idx)
+        assert np.array_equal(kv_count[l].cpu().numpy(), want_count)
+        assert np.array_equal(kv_cols[l].cpu().numpy(), want_count * dh)
+        c, _, p = o.cover_and_pos(want_idx, Hkv, counts=want_count)
+        assert np.array_equal(kv_cover[l].cpu().numpy().view(np.uint32), c)
+        assert np.array_equal(kv_pos[l].cpu().numpy(), p)
+        saw_ragged |= bool(np.any(want_count < Hkv))
+    assert saw_ragged
+
+
+# --------------------------------------------------------------------------------------------- gather / aggregate
+
+@pytest.mark.parametrize("dtype,d,n_full,S,n_sub,br", [
+    (I.DTYPE_BF16, 4096, 512, 8, 128, 1), (I.DTYPE_BF16, 328, 300, 3, 101, 1), (I.DTYPE_BF16, 768, 12, 4, 6, 64),
+    (I.DTYPE_FP32, 64, 256, 2, 128, 1), (I.DTYPE_FP32, 100, 37, 5, 9, 3), (I.DTYPE_BF16, 8, 5, 2, 3, 1),
+])
+def test_gather_bit_exact_and_aggregate_parity(B, dtype, d, n_full, S, n_sub, br):
+    td = torch.bfloat16 if dtype == I.DTYPE_BF16 else torch.float32
+    W = I.normal(11, 1, (n_full * br + 5, d), 0.02, dtype)          # 5 extra rows: src_row_offset = 2
+    A = o.sample_blueprint(n_full, S, n_sub, [], 5, 0, 0, 0, o.MODE_IID)
+    cover, count, pos = o.cover_and_pos(A, n_full)
+    Wd = dev(W, td)
+    rows = n_sub * br
+    pad_rows = 3                                                     # slice rows before the segment
+    sub = torch.zeros(S, pad_rows + rows, d, dtype=td, device="cuda")
+    master = torch.zeros(S, pad_rows + rows, d, dtype=torch.float32, device="cuda") if dtype == I.DTYPE_BF16 else None
+    seg = B.gather_segment(Wd, sub, master, dev(A), None, n_sub, n_sub, br, 2, (pad_rows + rows) * d, pad_rows)
+    B.twist_gather_subnets([seg], S, d, dtype)
+    torch.cuda.synchronize()
+    for s in range(S):
+        want = o.gather_rows(W, A[s], br, row_offset=2)
+        got = sub[s, pad_rows:].float().cpu().numpy()
+        assert np.array_equal(got.view(np.uint32), want.astype(np.float32).view(np.uint32))
+        assert torch.all(sub[s, :pad_rows] == 0)
+        if master is not None:
+            assert np.array_equal(master[s, pad_rows:].cpu().numpy().view(np.uint32), want.astype(np.float32).view(np.uint32))
+
+    # "train": perturb the fp32 masters / slices with seeded noise, then aggregate
+    noise = I.normal(12, 2, (S, pad_rows + rows, d), 0.01, I.DTYPE_FP32)
+    trained = (master if master is not None else sub).float() + dev(noise)
+    trained = trained.contiguous()
+    for live in (0xFFFFFFFF, 0b101 & ((1 << S) - 1)):
+        full = Wd.clone()
+        full_f32 = torch.full((n_full * br + 5, d), 123.0, dtype=torch.float32, device="cuda") if dtype == I.DTYPE_BF16 else None
+        seg = B.aggregate_segment(full, full_f32, trained, dev(cover.view(np.int32)), dev(pos), n_full, br, 2,
+                                  (pad_rows + rows) * d, pad_rows)
+        B.twist_aggregate([seg], S, d, dtype, live)
+        torch.cuda.synchronize()
+        tr = trained.cpu().numpy().astype(np.float64)
+        want = o.aggregate(W.astype(np.float64), [tr[s, pad_rows:] for s in range(S)], A, br, live_mask=live, row_offset=2)
+        live_cnt = np.array([bin(int(c) & live).count("1") for c in cover])
+        held_rows = np.repeat(live_cnt > 0, br)
+        res = (full_f32 if full_f32 is not None else full).cpu().numpy().astype(np.float64)[2:2 + n_full * br]
+        w_rows = want[2:2 + n_full * br]
+        # relative to the mean magnitude of the averaged values (an fp32 sum that cancels cannot be
+        # relatively exact in its own, much smaller, magnitude)
+        mag = o.aggregate(np.abs(W.astype(np.float64)), [np.abs(tr[s, pad_rows:]) for s in range(S)], A, br,
+                          live_mask=live, row_offset=2)[2:2 + n_full * br]
+        err = np.abs(res[held_rows] - w_rows[held_rows]) / np.maximum(mag[held_rows], 1e-30)
+        assert err.max() <= AGG_TOL, err.max()
+        if full_f32 is not None:      # untouched rows keep their values in both outputs; bf16 shadow = RNE(fp32 result)
+            assert torch.all(full_f32[2:2 + n_full * br][torch.from_numpy(~held_rows).cuda()] == 123.0)
+            assert torch.equal(full[2:2 + n_full * br][torch.from_numpy(held_rows).cuda()],
+                               full_f32[2:2 + n_full * br][torch.from_numpy(held_rows).cuda()].to(torch.bfloat16))
+        assert torch.equal(full[2:2 + n_full * br][torch.from_numpy(~held_rows).cuda()],
+                           Wd[2:2 + n_full * br][torch.from_numpy(~held_rows).cuda()])
+        assert torch.equal(full[:2], Wd[:2]) and torch.equal(full[2 + n_full * br:], Wd[2 + n_full * br:])
+    check_status(B)
+
+
+def test_gather_ragged_counts_zero_fill(B):
+    d, S, Hkv, dh = 64, 3, 4, 8
+    W = I.normal(13, 1, (Hkv * dh, d), 0.02, I.DTYPE_BF16)
+    kv_idx = np.array([[0, 2, -1, -1], [1, -1, -1, -1], [0, 1, 2, 3]], dtype=np.int32)
+    kv_count = np.array([2, 1, 4], dtype=np.int32)
+    sub = torch.full((S, Hkv * dh, d), 9.0, dtype=torch.bfloat16, device="cuda")
+    master = torch.full((S, Hkv * dh, d), 9.0, dtype=torch.float32, device="cuda")
+    seg = B.gather_segment(dev(W, torch.bfloat16), sub, master, dev(kv_idx), dev(kv_count), Hkv, Hkv, dh, 0, Hkv * dh * d, 0)
+    B.twist_gather_subnets([seg], S, d, I.DTYPE_BF16)
+    torch.cuda.synchronize()
+    for s in range(S):
+        n = kv_count[s] * dh
+        want = o.gather_rows(W, kv_idx[s][: kv_count[s]], dh)
+        assert np.array_equal(sub[s, :n].float().cpu().numpy(), want)
+        assert torch.all(sub[s, n:] == 0) and torch.all(master[s, n:] == 0)
+
+
+# --------------------------------------------------------------------------------------------- MSE glue
+
+@pytest.mark.parametrize("dtype", [I.DTYPE_BF16, I.DTYPE_FP32])
+def test_mse_parity(B, dtype):
+    S, T, width = 3, 77, 72
+    td = torch.bfloat16 if dtype == I.DTYPE_BF16 else torch.float32
+    Y = I.normal(21, 1, (S, T, width), 1.0, dtype)
+    Tg = I.normal(21, 2, (S, T, width), 1.0, dtype)
+    ws = torch.empty(B.twist_mse_workspace_bytes(S), dtype=torch.uint8, device="cuda")
+    for valid, seg_begin, seg_width in [(None, 0, 0), (np.array([8, 16, 24], dtype=np.int32), 24, 24),
+                                        (np.array([72, 40, 8], dtype=np.int32), 0, 72)]:
+        dy = torch.empty(S, T, width, dtype=td, device="cuda")
+        loss = torch.empty(S, dtype=torch.float32, device="cuda")
+        B.twist_mse_fwd_bwd(dev(Y, td), dev(Tg, td), dy, loss, S, T, width, None if valid is None else dev(valid),
+                            seg_begin, seg_width, dtype, ws)
+        torch.cuda.synchronize()
+        for s in range(S):
+            if valid is None:
+                cols = np.arange(width)
+            else:
+                cols = np.array([c for c in range(width) if c < seg_begin or (c - seg_begin) % seg_width < valid[s]])
+            want_loss, want_dy = o.mse(Y[s][:, cols].astype(np.float64), Tg[s][:, cols].astype(np.float64),
+                                       lowp=dtype == I.DTYPE_BF16)
+            got = host(dy[s])
+            assert abs(loss[s].item() - want_loss) <= 1e-5 * want_loss
+            assert rel_fro(got[:, cols], want_dy) < (1e-2 if dtype == I.DTYPE_BF16 else 1e-6)
+            other = np.setdiff1d(np.arange(width), cols)
+            assert np.all(got[:, other] == 0)
+
+
+# --------------------------------------------------------------------------------------------- FFN / projections
+
+def _ffn_case(B, kind, dtype, S, T, d, f, alpha, lr, seed):
+    lowp = dtype == I.DTYPE_BF16
+    td = torch.bfloat16 if lowp else torch.float32
+    g = 2 if kind == I.FFN_SWIGLU else 1
+    X = I.normal(seed, 1, (S, T, d), 1.0, dtype)
+    Wgu = I.normal(seed, 2, (S, g * f, d), 0.05, dtype)
+    Wd = I.normal(seed, 3, (S, f, d), 0.05, dtype)
+    dY = I.normal(seed, 4, (S, T, d), 1e-3, dtype)
+    t = lambda *s: torch.zeros(*s, dtype=td, device="cuda")
+    w_gu, w_down = dev(Wgu, td), dev(Wd, td)
+    m_gu, m_down = (w_gu.float(), w_down.float()) if lowp else (None, None)
+    pre, hh, y, dpre, dx = t(S, T, g * f), t(S, T, f), t(S, T, d), t(S, T, g * f), t(S, T, d)
+    dw_gu = torch.zeros(S, g * f, d, dtype=torch.float32, device="cuda")
+    dw_down = torch.zeros(S, f, d, dtype=torch.float32, device="cuda")
+    a = B.ffn_args(kind, dtype, S, T, d, f, alpha, lr, x=dev(X, td), w_gu=w_gu, w_down=w_down, w_gu_master=m_gu,
+                   w_down_master=m_down, pre=pre, hh=hh, y=y, dy=dev(dY, td), dpre=dpre, dx=dx, dw_gu=dw_gu,
+                   dw_down=dw_down)
+    B.twist_subnet_ffn_fwd(a)
+    B.twist_subnet_ffn_bwd(a)
+    torch.cuda.synchronize()
+    check_status(B)
+    tol = GEMM_TOL if lowp else 1e-4
+    for s in range(S):
+        Wg_s = Wgu[s, :f].astype(np.float64) if g == 2 else None
+        Wu_s = Wgu[s, (g - 1) * f:].astype(np.float64)
+        Wd_s = Wd[s].astype(np.float64)
+        Xs, dYs = X[s].astype(np.float64), dY[s].astype(np.float64)
+        Yw, saved = o.ffn_fwd(Xs, Wu_s, Wg_s, Wd_s, kind, alpha, lowp)
+        dXw, dWu, dWg, dWd = o.ffn_bwd(dYs, Xs, saved, Wu_s, Wg_s, Wd_s, kind, alpha, lowp)
+        pre_w = np.concatenate([saved["G"], saved["U"]], axis=1) if g == 2 else saved["U"]
+        dWgu = np.concatenate([dWg, dWu], axis=0) if g == 2 else dWu
+        assert rel_fro(host(pre[s]), pre_w) < tol, ("pre", s)
+        assert rel_fro(host(hh[s]), saved["Hh"]) < tol, ("hh", s)
+        assert rel_fro(host(y[s]), Yw) < tol, ("y", s)
+        assert rel_fro(host(dx[s]), dXw) < tol, ("dx", s)
+        assert rel_fro(host(dw_gu[s]), dWgu) < tol, ("dw_gu", s)
+        assert rel_fro(host(dw_down[s]), dWd) < tol, ("dw_down", s)
+        if lr != 0:
+            new_gu, new_gu_c = o.sgd(Wgu[s].astype(np.float64), dWgu, lr, lowp)
+            new_d, new_d_c = o.sgd(Wd_s, dWd, lr, lowp)
+            upd = host(m_gu[s] if lowp else w_gu[s]) - Wgu[s]
+            assert rel_fro(upd, new_gu - Wgu[s]) < tol, ("sgd gu", s)
+            upd = host(m_down[s] if lowp else w_down[s]) - Wd[s]
+            assert rel_fro(upd, new_d - Wd[s]) < tol, ("sgd down", s)
+            if lowp:   # compute copy is the nearest-even rounding of the device's own master
+                assert torch.equal(w_gu[s], m_gu[s].to(torch.bfloat16))
+                assert torch.equal(w_down[s], m_down[s].to(torch.bfloat16))
+
+
+@pytest.mark.parametrize("kind", [I.FFN_RELU, I.FFN_GELU, I.FFN_SWIGLU])
+def test_ffn_fp32_parity(B, kind):
+    _ffn_case(B, kind, I.DTYPE_FP32, S=2, T=37, d=24, f=20, alpha=1.5, lr=0.5, seed=31)
+
+
+@pytest.mark.parametrize("kind,S,T,d,f", [
+    (I.FFN_SWIGLU, 2, 256, 256, 256),      # whole tiles
+    (I.FFN_SWIGLU, 3, 200, 328, 344),      # ragged M, K and N tails, several tiles
+    (I.FFN_GELU, 2, 333, 192, 520),
+    (I.FFN_RELU, 2, 128, 64, 128),         # config-1 shape in bf16
+    (I.FFN_SWIGLU, 1, 520, 1032, 688),     # > 4 k-blocks: the ring wraps; 3 n-tiles in dX
+])
+def test_ffn_bf16_parity(B, kind, S, T, d, f):
+    _ffn_case(B, kind, I.DTYPE_BF16, S, T, d, f, alpha=2.0, lr=0.5, seed=41)
+
+
+@pytest.mark.parametrize("dtype,S,T,d,n", [(I.DTYPE_FP32, 2, 33, 24, 16), (I.DTYPE_BF16, 2, 200, 328, 200),
+                                           (I.DTYPE_BF16, 3, 384, 768, 1152), (I.DTYPE_BF16, 1, 130, 64, 72)])
+def test_proj_parity(B, dtype, S, T, d, n):
+    lowp = dtype == I.DTYPE_BF16
+    td = torch.bfloat16 if lowp else torch.float32
+    tol = GEMM_TOL if lowp else 1e-4
+    lr = 0.5
+    for which, alpha in ((B.PROJ_QKV, 1.0), (B.PROJ_O, 1.7)):
+        w_in, w_out = (d, n) if which == B.PROJ_QKV else (n, d)
+        Xin = I.normal(51, 1 + which, (S, T, w_in), 1.0, dtype)
+        W = I.normal(51, 3 + which, (S, n, d), 0.05, dtype)
+        dO = I.normal(51, 5 + which, (S, T, w_out), 1e-3, dtype)
+        w = dev(W, td)
+        m = w.float() if lowp else None
+        out = torch.zeros(S, T, w_out, dtype=td, device="cuda")
+        d_in = torch.zeros(S, T, w_in, dtype=td, device="cuda")
+        dw = torch.zeros(S, n, d, dtype=torch.float32, device="cuda")
+        a = B.proj_args(which, dtype, S, T, d, n, alpha, lr, in_=dev(Xin, td), w=w, w_master=m, out=out,
+                        d_out=dev(dO, td), d_in=d_in, dw=dw)
+        B.twist_subnet_attn_proj_fwd(a)
+        B.twist_subnet_attn_proj_bwd(a)
+        torch.cuda.synchronize()
+        check_status(B)
+        for s in range(S):
+            Xs, Ws, dOs = (v[s].astype(np.float64) for v in (Xin, W, dO))
+            if which == B.PROJ_QKV:
+                want_out = o.qkv_fwd(Xs, Ws, lowp)
+                want_din, want_dw = o.qkv_bwd(dOs, Xs, Ws, lowp)
+            else:
+                want_out = o.o_fwd(Xs, Ws, alpha, lowp)
+                want_din, want_dw = o.o_bwd(dOs, Xs, Ws, alpha, lowp)
+            assert rel_fro(host(out[s]), want_out) < tol, (which, "out")
+            assert rel_fro(host(d_in[s]), want_din) < tol, (which, "d_in")
+            assert rel_fro(host(dw[s]), want_dw) < tol, (which, "dw")
+            upd = host(m[s] if lowp else w[s]) - W[s]
+            assert rel_fro(upd, -lr * want_dw) < tol, (which, "sgd")
+
+
+# --------------------------------------------------------------------------------------------- whole rounds
+
+def _load_full(eng, w):
+    td = torch.bfloat16 if w.dtype == I.DTYPE_BF16 else torch.float32
+    mats = {"gate": I.MAT_GATE, "up": I.MAT_UP, "down": I.MAT_DOWN, "qkv": I.MAT_QKV, "o": I.MAT_O}
+    full_np = []
+    for l in range(w.n_layers):
+        layer = {}
+        for m in eng.full:
+            layer[m] = I.weight(w, l, mats[m])
+            eng.full[m][l].copy_(dev(layer[m], td))
+        full_np.append(layer)
+    return full_np
+
+
+def _load_batches(eng, w, rnd):
+    td = torch.bfloat16 if w.dtype == I.DTYPE_BF16 else torch.float32
+    S = w.n_subnets
+    eng.X, eng.Td, eng.Tq, eng.A = [], [], [], []
+    store = {}
+    for k in range(w.local_steps):
+        for kind, width, dst in ((I.BATCH_X, w.d_model, eng.X), (I.BATCH_TGT_D, w.d_model, eng.Td)) + (
+                ((I.BATCH_TGT_QKV, eng.nq, eng.Tq), (I.BATCH_A, eng.a_sub, eng.A)) if eng.has_attn else ()):
+            arr = np.stack([I.batch(w, kind, rnd, s, k, width) for s in range(S)])
+            store[(kind, k)] = arr
+            dst.append(dev(arr, td))
+    return store
+
+
+def _run_round_and_compare(B, w, rnd=0, tol_dw=5e-2):
+    from paper_2511_03983_b200.engine import RoundEngine
+    lowp = w.dtype == I.DTYPE_BF16
+    eng = RoundEngine(w, keep_f32_full=True)
+    full_np = _load_full(eng, w)
+    store = _load_batches(eng, w, rnd)
+    before = {m: v.clone() for m, v in eng.full.items()}
+    eng.run_round(rnd)
+    torch.cuda.synchronize()
+    check_status(B)
+    ragged = eng.has_attn and w.n_kv_heads != w.n_heads
+    for l in range(w.n_layers):
+        bp = o.layer_blueprints(w, rnd, l)
+
+        def get_batch(kind, rnd_, s, k, width):
+            arr = store[(kind, k)][s]
+            if kind == I.BATCH_TGT_QKV and ragged:     # device layout [Q | K pad | V pad] -> oracle [Q | K | V]
+                kc = bp["kv_count"][s] * w.d_head
+                kvw = eng.kv_max * w.d_head
+                return np.concatenate([arr[:, :eng.a_sub], arr[:, eng.a_sub:eng.a_sub + kc],
+                                       arr[:, eng.a_sub + kvw:eng.a_sub + kvw + kc]], axis=1)
+            return arr
+
+        full64 = {m: v.astype(np.float64) for m, v in full_np[l].items()}
+        new, new_shadow, _, losses = o.round_blockwise_layer(w, full64, get_batch, rnd, l, lowp)
+        assert np.array_equal(eng.idx_ffn[l].cpu().numpy(), bp["ffn"])
+        for m in eng.full:
+            res = (eng.full_f32[m][l] if lowp else eng.full[m][l]).cpu().numpy().astype(np.float64)
+            delta_w, delta_g = new[m] - full64[m], res - full64[m]
+            # fp32: the update is ~1e-4 of the weight, so the fp32 storage of W bounds the accuracy of the
+            # difference at ~1e-3; the weights themselves must agree to fp32 rounding.
+            assert rel_fro(delta_g, delta_w) < (tol_dw if lowp else 1e-3), (l, m, rel_fro(delta_g, delta_w))
+            if not lowp:
+                assert np.max(np.abs(res - new[m])) <= 2e-7 * np.max(np.abs(new[m])), (l, m)
+        for bi, name in enumerate(("ffn", "qkv", "o")[: 3 if eng.has_attn else 1]):
+            got = eng.loss[l, bi, : w.local_steps].cpu().numpy()
+            want = np.array([losses[s][name] for s in range(w.n_subnets)]).T
+            assert np.allclose(got, want, rtol=2e-2 if lowp else 1e-4), (l, name)
+    return eng, before
+
+
+def test_config1_fp32_round_matches_oracle_everywhere(B):
+    _run_round_and_compare(B, I.PRESETS[1])
+
+
+@pytest.mark.parametrize("cfg,dims", [
+    (2, dict(d_model=192, d_ff=520, d_head=16, tokens=200, n_layers=2, local_steps=2)),
+    (3, dict(d_model=256, d_ff=688, d_head=8, tokens=256, n_layers=2, local_steps=2)),
+    (4, dict(d_model=328, d_ff=1376, d_head=8, tokens=200, n_layers=1, local_steps=2)),
+])
+def test_scaled_twin_rounds_match_oracle(B, cfg, dims):
+    w = I.scaled_twin(I.PRESETS[cfg], **dims)
+    _run_round_and_compare(B, w)
+
+
+def test_round_with_zero_lr_is_identity_on_the_bf16_model(B):
+    from paper_2511_03983_b200.engine import RoundEngine
+    w = replace(I.scaled_twin(I.PRESETS[4], d_model=128, d_ff=512, d_head=8, tokens=128, n_layers=1, local_steps=1),
+                lr=0.0)
+    eng = RoundEngine(w)
+    _load_full(eng, w)
+    _load_batches(eng, w, 0)
+    before = {m: v.clone() for m, v in eng.full.items()}
+    eng.run_round(0)
+    torch.cuda.synchronize()
+    for m in before:      # aggregation of identical (untrained) subnets is the identity
+        assert torch.equal(before[m], eng.full[m]), m
