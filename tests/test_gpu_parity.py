@@ -391,7 +391,7 @@ def test_config1_fp32_round_matches_oracle_everywhere(B):
 
 
 @pytest.mark.parametrize("cfg,dims", [
-    (2, dict(d_model=192, d_ff=520, d_head=16, tokens=200, n_layers=2, local_steps=2)),
+    (2, dict(d_model=192, d_ff=528, d_head=16, tokens=200, n_layers=2, local_steps=2)),
     (3, dict(d_model=256, d_ff=688, d_head=8, tokens=256, n_layers=2, local_steps=2)),
     (4, dict(d_model=328, d_ff=1376, d_head=8, tokens=200, n_layers=1, local_steps=2)),
 ])
