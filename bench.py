@@ -1,0 +1,379 @@
+#!/usr/bin/env python
+"""Benchmark of one TwIST training round (BLOCKWISE) through the C ABI on B200.
+
+A "step" is one whole round of the hot path over one batch of synthetic input:
+sample masks -> per layer { gather -> K local steps (FFN block, QKV projection, output
+projection: forward, MSE, backward with fused SGD; all S subnets per launch) -> aggregate }.
+Metric: tokens/s per round, tokens = S * K * T.
+
+Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle instead (a bounded
+sample per step, extrapolated to a round; rank 0 only).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "twist_round_tokens_per_s"
+UNIT = "tokens/s"
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return {"hbm_gbs": p["hbm_gbs"], "bf16_tflops": p["bf16_tflops"],
+                "bf16_tflops_sustained": p.get("bf16_tflops_sustained", p["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+# ------------------------------------------------------------------------------------------------
+# algorithmic work of one round (what the method must do; the dense model would need more)
+# ------------------------------------------------------------------------------------------------
+
+def round_work(w, nq_valid=None):
+    """FLOPs of the grouped GEMMs and bytes of gather / aggregate for one round."""
+    S, K, T, d, L = w.n_subnets, w.local_steps, w.tokens, w.d_model, w.n_layers
+    f = w.f_sub
+    flops_ffn = 6.0 * T * d * f * w.nmat                      # fwd 2 + bwd 4 per weight element per token
+    a = w.a_sub
+    kv = (min(w.n_kv_heads, w.head_keep) * w.d_head) if w.n_heads else 0
+    nq = (a + 2 * kv) if nq_valid is None else nq_valid
+    flops_attn = 6.0 * T * d * (nq + a) if w.n_heads else 0.0
+    gemm_flops = (flops_ffn + flops_attn) * S * K * L
+    kept = (w.nmat * f + (nq + a if w.n_heads else 0)) * d    # kept elements per subnet per layer
+    gather_bytes = (2 + 2 + 4) * kept * S * L                 # read bf16, write bf16, write fp32 master
+    # aggregate: read every subnet's master (4 B) + write fp32 result and bf16 shadow for every covered element
+    full = (w.nmat * w.d_ff + ((w.n_heads + 2 * w.n_kv_heads + w.n_heads) * w.d_head if w.n_heads else 0)) * d
+    agg_bytes = 4 * kept * S * L + (4 + 2) * full * L         # cover mode: every element is covered
+    return {"gemm_flops": gemm_flops, "gather_bytes": gather_bytes, "aggregate_bytes": agg_bytes}
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.rows, self.proc, self.gpu = [], None, gpu_index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.gpu), f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "200"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            threading.Thread(target=self._read, daemon=True).start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.25)
+        self.proc.terminate()          # the exact process this object started
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            pass
+        sm = sorted(float(r[1]) for r in self.rows if len(r) >= 9 and r[1].replace(".", "").isdigit())
+        mx = [float(r[2]) for r in self.rows if len(r) >= 9 and r[2].replace(".", "").isdigit()]
+        reasons = set()
+        for r in self.rows:
+            if len(r) >= 9:
+                for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[5:9]):
+                    if v.lower().startswith("active"):
+                        reasons.add(name)
+        return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# ------------------------------------------------------------------------------------------------
+# CPU oracle timing (reported baseline and `--impl reference` arm)
+# ------------------------------------------------------------------------------------------------
+
+def oracle_round_estimate(w, tokens_sample=128, seed=7):
+    """Times the oracle, as it stands, on a bounded sample of the workload: ONE layer, all S
+    subnets, ONE local step on `tokens_sample` tokens per subnet, plus that layer's blueprint,
+    gather and aggregate at full size.  The per-round figure scales the local-step time by
+    K * T / tokens_sample and everything by the layer count (extrapolated)."""
+    import numpy as np
+    from dataclasses import replace
+    from oracle import twist_oracle as o
+    from paper_2511_03983_b200 import inputs as I
+
+    lowp = w.dtype == I.DTYPE_BF16
+    ws = replace(w, n_layers=1, local_steps=1, tokens=tokens_sample)
+    mats = {"gate": I.MAT_GATE, "up": I.MAT_UP, "down": I.MAT_DOWN, "qkv": I.MAT_QKV, "o": I.MAT_O}
+    names = ["up", "down"] + (["gate"] if w.ffn_kind == I.FFN_SWIGLU else []) + (["qkv", "o"] if w.n_heads else [])
+    full = {m: I.weight(ws, 0, mats[m]).astype(np.float64) for m in names}
+    cache = {}
+
+    def get_batch(kind, rnd, s, k, width):
+        key = (kind, s, width)
+        if key not in cache:
+            cache[key] = I.batch(ws, kind, rnd, s, k, width).astype(np.float64)
+        return cache[key]
+
+    t0 = time.perf_counter()
+    bp = o.layer_blueprints(ws, 0, 0)
+    t1 = time.perf_counter()
+    slices = [{m: np.asarray(v, dtype=np.float64) for m, v in o.gather_layer(ws, full, bp, s).items()}
+              for s in range(ws.n_subnets)]
+    t2 = time.perf_counter()
+    for s in range(ws.n_subnets):     # warm the batch cache outside the timed local steps
+        get_batch(0, 0, s, 0, w.d_model), get_batch(1, 0, s, 0, w.d_model)
+        if w.n_heads:
+            get_batch(2, 0, s, 0, slices[s]["qkv"].shape[0]), get_batch(3, 0, s, 0, slices[s]["o"].shape[0])
+    t3 = time.perf_counter()
+    for s in range(ws.n_subnets):
+        o.local_steps_blockwise(ws, slices[s], get_batch, 0, s, lowp)
+    t4 = time.perf_counter()
+    o.aggregate_layer(ws, full, slices, bp)
+    t5 = time.perf_counter()
+    t_mask, t_gather, t_local, t_agg = t1 - t0, t2 - t1, t4 - t3, t5 - t4
+    per_round = w.n_layers * (t_mask + t_gather + t_agg + t_local * w.local_steps * (w.tokens / tokens_sample))
+    cores = os.cpu_count() or 1
+    try:
+        from threadpoolctl import threadpool_info
+        cores = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+    except Exception:
+        pass
+    return {
+        "value": w.tokens_per_round / per_round, "unit": UNIT, "cores": cores, "kind": "oracle",
+        "sample": (f"1 of {w.n_layers} layers, all S={w.n_subnets} subnets, 1 local step on {tokens_sample} of "
+                   f"{w.tokens} tokens per subnet (numpy fp64), blueprint+gather+aggregate of that layer at full "
+                   f"size; extrapolated to a round: layers x (mask {t_mask:.3f}s + gather {t_gather:.3f}s + aggregate "
+                   f"{t_agg:.3f}s + local {t_local:.3f}s x K x T/{tokens_sample})"),
+        "sample_seconds": round(t5 - t0, 3), "round_seconds_extrapolated": round(per_round, 1),
+    }
+
+
+def run_reference(args, w):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    times, last = [], None
+    for i in range(args.warmup + args.steps):
+        last = oracle_round_estimate(w, tokens_sample=args.oracle_tokens)
+        if i >= args.warmup:
+            times.append(last["round_seconds_extrapolated"])
+    ms = 1e3 * sum(times) / len(times)
+    value = w.tokens_per_round / (ms / 1e3)
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f64", "data": "synthetic", "config": workload_config(w, args),
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": last["cores"], "kind": "oracle", "sample": last["sample"]},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def workload_config(w, args):
+    return {"workload": f"configs[{args.config - 1}] {w.name}: BLOCKWISE round, L={w.n_layers} d={w.d_model} "
+                        f"F={w.d_ff} f'={w.f_sub} H'={w.head_keep}/{w.n_heads} S={w.n_subnets} T={w.tokens} K={w.local_steps}",
+            "tokens_per_round": w.tokens_per_round, "mode": "blockwise, layers streamed",
+            "l2_policy": "inputs larger than L2 (every tensor a kernel reads is >= 4x the 126 MB L2)"
+                         if w.d_model >= 2048 else "working set exceeds L2 across the layers of a round",
+            "parallelism": "replicas only" if args.gpus > 1 else "single GPU"}
+
+
+# ------------------------------------------------------------------------------------------------
+# CUDA arm
+# ------------------------------------------------------------------------------------------------
+
+def run_ours(args, w):
+    import torch
+    import torch.distributed as dist
+
+    from paper_2511_03983_b200 import binding as B
+    from paper_2511_03983_b200 import inputs as I
+    from paper_2511_03983_b200.engine import RoundEngine
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the CUDA path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    B.lib()
+    bf16 = w.dtype == I.DTYPE_BF16
+    td = torch.bfloat16 if bf16 else torch.float32
+    eng = RoundEngine(w, keep_f32_full=True, compute_dx=True)
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(w.seed_w + 7919 * rank)
+    for m, v in eng.full.items():                         # weights ~ N(0, 0.02^2), one matrix at a time
+        for l in range(w.n_layers):
+            v[l].copy_((torch.randn(v[l].shape, generator=gen, device="cuda", dtype=torch.float32) * 0.02).to(td))
+    gen.manual_seed(w.seed_x + 7919 * rank)
+    S, T, K = w.n_subnets, w.tokens, w.local_steps
+    widths = [("X", w.d_model), ("Td", w.d_model)] + ([("Tq", eng.nq), ("A", eng.a_sub)] if eng.has_attn else [])
+    host = {}
+    for name, width in widths:
+        lst = getattr(eng, name)
+        for k in range(K):
+            t = torch.empty(S, T, width, dtype=td, device="cuda")
+            for s in range(S):
+                t[s].copy_(torch.randn(T, width, generator=gen, device="cuda", dtype=torch.float32).to(td))
+            lst.append(t)
+    h2d_bytes = sum(t.numel() * t.element_size() for name, _ in widths for t in getattr(eng, name))
+    d2h_bytes = eng.loss.numel() * 4
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- device-resident timing -------------------------------------------------------------
+    rnd = 0
+    for _ in range(args.warmup):
+        eng.run_round(rnd)
+        rnd += 1
+    barrier()
+    eng.launches = 0
+    eng.timing = True
+    eng.events.clear()
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e0.record()
+    for _ in range(args.steps):
+        eng.run_round(rnd)
+        rnd += 1
+    e1.record()
+    barrier()
+    clocks = sampler.stop() if rank == 0 else None
+    ms_total = e0.elapsed_time(e1)
+    launches = eng.launches
+    phases = eng.phase_ms()
+    eng.timing = False
+    status = B.twist_device_status()
+    if status != 0:
+        raise SystemExit(f"device status {status}: a bounded device wait expired")
+    t_ms = torch.tensor([ms_total], dtype=torch.float64, device="cuda")
+    if world > 1:
+        dist.all_reduce(t_ms, op=dist.ReduceOp.MAX)
+    ms_per_step = t_ms.item() / args.steps
+    value = world * w.tokens_per_round / (ms_per_step / 1e3)
+
+    # ---- end-to-end: host buffers, copies inside the timed region --------------------------------
+    e2e = None
+    if not args.no_e2e:
+        pinned = {}
+        for name, _ in widths:
+            pinned[name] = [t.cpu().pin_memory() for t in getattr(eng, name)]
+        loss_host = torch.empty(eng.loss.shape, dtype=torch.float32).pin_memory()
+        n_e2e = max(1, min(args.steps, args.e2e_steps))
+        barrier()
+        e0.record()
+        for _ in range(n_e2e):
+            for name, _ in widths:
+                for dst, src in zip(getattr(eng, name), pinned[name]):
+                    dst.copy_(src, non_blocking=True)
+            eng.run_round(rnd)
+            rnd += 1
+            loss_host.copy_(eng.loss, non_blocking=True)
+        e1.record()
+        barrier()
+        t_ms = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device="cuda")
+        if world > 1:
+            dist.all_reduce(t_ms, op=dist.ReduceOp.MAX)
+        e2e = {"value": world * w.tokens_per_round / (t_ms.item() / n_e2e / 1e3), "unit": UNIT,
+               "h2d_bytes_per_step": h2d_bytes, "d2h_bytes_per_step": d2h_bytes, "steps": n_e2e,
+               "note": "pinned host batches copied in, per-subnet losses copied out, every step"}
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peaks = measured_peaks()
+    work = round_work(w)
+    gemm_names = [n for n in ("ffn_fwd", "ffn_bwd", "qkv_fwd", "qkv_bwd", "o_fwd", "o_bwd") if n in phases]
+    gemm_ms = sum(phases[n][0] for n in gemm_names)
+    gemm_launches_per_round = w.n_layers * K * ((2 + 4) + ((1 + 2 + 1 + 2) if eng.has_attn else 0))
+    roofline, phase_out = None, {}
+    for n, (ms, calls) in phases.items():
+        phase_out[n] = {"ms_per_step": ms / args.steps, "calls_per_step": calls // args.steps}
+    if bf16 and gemm_ms > 0:
+        tflops = work["gemm_flops"] * args.steps / (gemm_ms / 1e3) / 1e12
+        peak = peaks["bf16_tflops_sustained"]
+        roofline = {"bound": "tensor", "kernel": "gemm_kernel (grouped tcgen05 GEMM, all layouts/epilogues)",
+                    "achieved": tflops, "peak": peak, "unit": "TFLOP/s", "frac": tflops / peak,
+                    "peak_source": f"bf16_tflops_sustained of {peaks['source']}", "traffic": None,
+                    "flops_per_launch": work["gemm_flops"] / gemm_launches_per_round,
+                    "avg_launch_ms": gemm_ms / args.steps / gemm_launches_per_round,
+                    "share_of_step": gemm_ms / ms_total}
+    hbm = {}
+    for name, key in (("gather", "gather_bytes"), ("aggregate", "aggregate_bytes")):
+        if name in phases and phases[name][0] > 0:
+            gbs = work[key] * args.steps / (phases[name][0] / 1e3) / 1e9
+            hbm[name] = {"achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"],
+                         "bytes_per_launch": work[key] / w.n_layers}
+    if roofline is None and "aggregate" in hbm:
+        roofline = dict(bound="hbm", kernel="aggregate_rows_kernel", traffic=None, **hbm["aggregate"])
+
+    cpu = None
+    if not args.no_cpu_baseline:
+        cpu = oracle_round_estimate(w, tokens_sample=args.oracle_tokens)
+        cpu = {k: cpu[k] for k in ("value", "unit", "cores", "kind", "sample")}
+
+    out = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+           "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+           "dtype": "bf16" if bf16 else "f32", "data": "synthetic", "config": workload_config(w, args),
+           "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline, "hbm_kernels": hbm,
+           "phases": phase_out, "cpu_baseline": cpu}
+    print(json.dumps(out))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=2)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", type=int, default=4, help="workload 1..5 (default 4: the 7B-shaped round)")
+    ap.add_argument("--oracle-tokens", type=int, default=128)
+    ap.add_argument("--e2e-steps", type=int, default=1)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--layers", type=int, default=0, help="override the layer count (profiling on a small case)")
+    ap.add_argument("--tokens", type=int, default=0, help="override tokens per subnet-step (profiling on a small case)")
+    ap.add_argument("--local-steps", type=int, default=0)
+    args = ap.parse_args()
+    from dataclasses import replace
+    from paper_2511_03983_b200 import inputs as I
+    w = I.PRESETS[args.config]
+    if args.layers:
+        w = replace(w, n_layers=args.layers, name=w.name + f"-L{args.layers}")
+    if args.tokens:
+        w = replace(w, tokens=args.tokens, name=w.name + f"-T{args.tokens}")
+    if args.local_steps:
+        w = replace(w, local_steps=args.local_steps, name=w.name + f"-K{args.local_steps}")
+    if args.impl == "reference":
+        run_reference(args, w)
+    else:
+        run_ours(args, w)
+
+
+if __name__ == "__main__":
+    main()

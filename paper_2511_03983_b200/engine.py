@@ -12,7 +12,8 @@ at S=8, keep 25%, instead of 78 GB for all 32 layers).
 from __future__ import annotations
 
 import math
-from typing import Dict, List, Optional
+from contextlib import contextmanager
+from typing import Dict, List, Optional, Tuple
 
 import torch
 
@@ -100,19 +101,39 @@ class RoundEngine:
         self.Tq: List[torch.Tensor] = []
         self.A: List[torch.Tensor] = []
         self.launches = 0
+        # optional per-phase CUDA-event timing (events on the launching stream)
+        self.timing = False
+        self.events: Dict[str, List[Tuple[torch.cuda.Event, torch.cuda.Event]]] = {}
+
+    @contextmanager
+    def _timed(self, name: str):
+        if not self.timing:
+            yield
+            return
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        yield
+        b.record()
+        self.events.setdefault(name, []).append((a, b))
+
+    def phase_ms(self) -> Dict[str, Tuple[float, int]]:
+        """Total milliseconds and number of timed calls per phase (call after a synchronize)."""
+        return {k: (sum(a.elapsed_time(b) for a, b in v), len(v)) for k, v in self.events.items()}
 
     # ------------------------------------------------------------------ steps of the round
     def sample_masks(self, rnd: int):
         w = self.w
-        B.twist_sample_masks(w.seed_mask, rnd, 0, w.n_layers, B.KIND_FFN, w.n_ffn_blocks, w.n_subnets, w.ffn_keep,
-                             list(w.common_ffn), w.sample_mode, self.idx_ffn, self.cover_ffn, self.pos_ffn)
-        self.launches += 2
-        if self.has_attn:
-            B.twist_sample_masks(w.seed_mask, rnd, 0, w.n_layers, B.KIND_HEAD, w.n_heads, w.n_subnets, w.head_keep,
-                                 list(w.common_heads), w.sample_mode, self.idx_head, self.cover_head, self.pos_head)
-            B.twist_kv_groups(self.idx_head, w.n_layers, w.n_subnets, w.head_keep, w.n_heads, w.n_kv_heads, w.d_head,
-                              self.kv_idx, self.kv_count, self.kv_cols, self.kv_cover, self.kv_pos)
-            self.launches += 4
+        with self._timed("sample_masks"):
+            B.twist_sample_masks(w.seed_mask, rnd, 0, w.n_layers, B.KIND_FFN, w.n_ffn_blocks, w.n_subnets, w.ffn_keep,
+                                 list(w.common_ffn), w.sample_mode, self.idx_ffn, self.cover_ffn, self.pos_ffn)
+            self.launches += 2
+            if self.has_attn:
+                B.twist_sample_masks(w.seed_mask, rnd, 0, w.n_layers, B.KIND_HEAD, w.n_heads, w.n_subnets,
+                                     w.head_keep, list(w.common_heads), w.sample_mode, self.idx_head, self.cover_head,
+                                     self.pos_head)
+                B.twist_kv_groups(self.idx_head, w.n_layers, w.n_subnets, w.head_keep, w.n_heads, w.n_kv_heads,
+                                  w.d_head, self.kv_idx, self.kv_count, self.kv_cols, self.kv_cover, self.kv_pos)
+                self.launches += 4
 
     def gather_layer(self, l: int, which=("ffn", "attn")):
         w, d = self.w, self.w.d_model
@@ -137,7 +158,8 @@ class RoundEngine:
                                          self.kv_max, dh, (H + Hkv) * dh, self.nq * d, self.a_sub + self.kv_max * dh))
             segs.append(B.gather_segment(self.full["o"][l], self.w_o, self.w_o_m, self.idx_head[l], None, w.head_keep,
                                          w.head_keep, dh, 0, self.a_sub * d, 0))
-        B.twist_gather_subnets(segs, w.n_subnets, d, w.dtype)
+        with self._timed("gather"):
+            B.twist_gather_subnets(segs, w.n_subnets, d, w.dtype)
         self.launches += 1
 
     def aggregate_layer(self, l: int, live: int = 0xFFFFFFFF, which=("ffn", "attn")):
@@ -168,13 +190,15 @@ class RoundEngine:
                                             Hkv, dh, (H + Hkv) * dh, self.nq * d, self.a_sub + self.kv_max * dh))
             segs.append(B.aggregate_segment(self.full["o"][l], f32("o"), sub(self.w_o, self.w_o_m), self.cover_head[l],
                                             self.pos_head[l], H, dh, 0, self.a_sub * d, 0))
-        B.twist_aggregate(segs, w.n_subnets, d, w.dtype, live)
+        with self._timed("aggregate"):
+            B.twist_aggregate(segs, w.n_subnets, d, w.dtype, live)
         self.launches += 1
 
     def _mse(self, y, tgt, dy, loss, width, valid_cols=None, seg_begin=0, seg_width=0):
         w = self.w
-        B.twist_mse_fwd_bwd(y, tgt, dy, loss, w.n_subnets, w.tokens, width, valid_cols, seg_begin, seg_width, w.dtype,
-                            self.ws)
+        with self._timed("mse"):
+            B.twist_mse_fwd_bwd(y, tgt, dy, loss, w.n_subnets, w.tokens, width, valid_cols, seg_begin, seg_width,
+                                w.dtype, self.ws)
         self.launches += 2
 
     def ffn_step(self, l: int, k: int, lr: Optional[float] = None):
@@ -184,9 +208,11 @@ class RoundEngine:
                        x=self.X[k], w_gu=self.w_gu, w_down=self.w_down, w_gu_master=self.w_gu_m,
                        w_down_master=self.w_down_m, pre=self.pre, hh=self.hh, y=self.y, dy=self.dy, dpre=self.dpre,
                        dx=self.dx, dw_gu=self.dw_gu, dw_down=self.dw_down)
-        B.twist_subnet_ffn_fwd(a)
+        with self._timed("ffn_fwd"):
+            B.twist_subnet_ffn_fwd(a)
         self._mse(self.y, self.Td[k], self.dy, self.loss[l, 0, k], w.d_model)
-        B.twist_subnet_ffn_bwd(a)
+        with self._timed("ffn_bwd"):
+            B.twist_subnet_ffn_bwd(a)
         bf16 = w.dtype == DTYPE_BF16
         self.launches += (2 + 3 + (1 if self.compute_dx else 0)) if bf16 else (3 + 4 + (1 if self.compute_dx else 0) + 2)
 
@@ -196,11 +222,13 @@ class RoundEngine:
         a = B.proj_args(B.PROJ_QKV, w.dtype, w.n_subnets, w.tokens, w.d_model, self.nq, 1.0, lr, in_=self.X[k],
                         w=self.w_qkv, w_master=self.w_qkv_m, out=self.qkv_out, d_out=self.dqkv, d_in=self.dx,
                         dw=self.dw_qkv)
-        B.twist_subnet_attn_proj_fwd(a)
+        with self._timed("qkv_fwd"):
+            B.twist_subnet_attn_proj_fwd(a)
         ragged = self.w.n_kv_heads != self.w.n_heads
         self._mse(self.qkv_out, self.Tq[k], self.dqkv, self.loss[l, 1, k], self.nq,
                   self.kv_cols[l] if ragged else None, self.a_sub, self.kv_max * w.d_head)
-        B.twist_subnet_attn_proj_bwd(a)
+        with self._timed("qkv_bwd"):
+            B.twist_subnet_attn_proj_bwd(a)
         self.launches += 1 + 1 + (1 if self.compute_dx else 0) + (0 if w.dtype == DTYPE_BF16 else 1)
 
     def o_step(self, l: int, k: int, lr: Optional[float] = None):
@@ -209,9 +237,11 @@ class RoundEngine:
         a = B.proj_args(B.PROJ_O, w.dtype, w.n_subnets, w.tokens, w.d_model, self.a_sub, self.alpha_a, lr,
                         in_=self.A[k], w=self.w_o, w_master=self.w_o_m, out=self.y, d_out=self.dy, d_in=self.da,
                         dw=self.dw_o)
-        B.twist_subnet_attn_proj_fwd(a)
+        with self._timed("o_fwd"):
+            B.twist_subnet_attn_proj_fwd(a)
         self._mse(self.y, self.Td[k], self.dy, self.loss[l, 2, k], w.d_model)
-        B.twist_subnet_attn_proj_bwd(a)
+        with self._timed("o_bwd"):
+            B.twist_subnet_attn_proj_bwd(a)
         self.launches += 1 + 1 + (1 if self.compute_dx else 0) + (0 if w.dtype == DTYPE_BF16 else 1)
 
     def run_layer(self, l: int):
