@@ -234,6 +234,35 @@ int32_t twist_mse_fwd_bwd(const void* y, const void* tgt, void* dy, float* loss,
                           int32_t width, const int32_t* valid_cols, int32_t seg_begin, int32_t seg_width,
                           int32_t dtype, void* ws, size_t ws_bytes, void* stream);
 
+/* ---------------------------------------------------------------------------------------------
+ * twist_mse_fwd_bwd_noalloc -- the same loss and gradient as twist_mse_fwd_bwd, for callers that
+ * cannot provide scratch memory.  (The paper has no counterpart: this entry point exists for the
+ * integration, not for the method.)
+ *
+ * Who needs it: code that runs where device allocation is forbidden or unavailable -- inside a
+ * region where cudaMalloc would synchronise or fail (a latency-critical serving loop, a callback, a
+ * host that hands this library a fixed set of buffers and nothing else), or a plug-in with no
+ * allocator of its own.  twist_mse_fwd_bwd needs a caller-provided workspace for its per-block
+ * partial sums; this variant keeps those partial sums in an array that lives inside the library.
+ *
+ * Limits and behaviour
+ *  - The array is fixed-size device memory (TWIST_NOALLOC_MAX_SUBNETS x 1024 floats = 128 KB) that
+ *    every GPU which loads the library holds until the process exits.
+ *  - n_subnets > TWIST_NOALLOC_MAX_SUBNETS returns TWIST_ERR_UNSUPPORTED; nothing is launched.
+ *  - No cudaMalloc, cudaFree or other allocating call is made, here or in a library on its behalf.
+ *  - The first call on each device looks up the array's device address (once per device, with that
+ *    device current).  Make that first call outside any stream capture.
+ *  - All calls share the one array, which keeps whatever the previous call left in it.  Nothing in it
+ *    has to start at zero: each call overwrites every partial sum it later reads.  Two calls that
+ *    overlap on the GPU (different streams, or different host threads without ordering) race on the
+ *    array and give wrong losses; order them on one stream or with events.
+ *  - Arguments, results and error codes are otherwise those of twist_mse_fwd_bwd.
+ */
+#define TWIST_NOALLOC_MAX_SUBNETS 32
+int32_t twist_mse_fwd_bwd_noalloc(const void* y, const void* tgt, void* dy, float* loss, int32_t n_subnets,
+                                  int32_t tokens, int32_t width, const int32_t* valid_cols, int32_t seg_begin,
+                                  int32_t seg_width, int32_t dtype, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

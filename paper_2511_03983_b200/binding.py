@@ -30,6 +30,7 @@ EXPORTS = [
     "twist_abi_version", "twist_strerror", "twist_last_cuda_error", "twist_device_status", "twist_sample_masks",
     "twist_kv_groups", "twist_gather_subnets", "twist_aggregate", "twist_subnet_ffn_fwd", "twist_subnet_ffn_bwd",
     "twist_subnet_attn_proj_fwd", "twist_subnet_attn_proj_bwd", "twist_mse_workspace_bytes", "twist_mse_fwd_bwd",
+    "twist_mse_fwd_bwd_noalloc",
 ]
 
 
@@ -99,6 +100,8 @@ def lib() -> C.CDLL:
         h.twist_mse_fwd_bwd.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32,
                                         C.c_int32, C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_size_t,
                                         C.c_void_p]
+        h.twist_mse_fwd_bwd_noalloc.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32,
+                                                C.c_int32, C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_void_p]
         for name in EXPORTS:
             f = getattr(h, name)
             if name not in ("twist_abi_version", "twist_strerror", "twist_last_cuda_error",
@@ -220,3 +223,12 @@ def twist_mse_fwd_bwd(y, tgt, dy, loss, n_subnets, tokens, width, valid_cols, se
                                    _ptr(valid_cols), seg_begin, seg_width, dtype, _ptr(ws),
                                    ws.numel() * ws.element_size(), _stream()),
            "twist_mse_fwd_bwd")
+
+
+def twist_mse_fwd_bwd_noalloc(y, tgt, dy, loss, n_subnets, tokens, width, valid_cols, seg_begin, seg_width, dtype):
+    """Loss and gradient like twist_mse_fwd_bwd, but with the library's built-in scratch: for callers
+    that must not (or cannot) allocate device memory.  At most 32 subnets; calls must not overlap on
+    the GPU; make the first call on a device outside stream capture."""
+    _check(lib().twist_mse_fwd_bwd_noalloc(_ptr(y), _ptr(tgt), _ptr(dy), _ptr(loss), n_subnets, tokens, width,
+                                           _ptr(valid_cols), seg_begin, seg_width, dtype, _stream()),
+           "twist_mse_fwd_bwd_noalloc")

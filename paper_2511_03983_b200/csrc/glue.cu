@@ -235,3 +235,45 @@ extern "C" int32_t twist_mse_fwd_bwd(const void* y, const void* tgt, void* dy, f
   TWIST_LAUNCH_CHECK();
   return TWIST_OK;
 }
+
+// ---------------------------------------------------------------------------------------------
+// Allocation-free variant of the loss.  Its partial sums live in a file-scope device array, so a
+// caller that cannot allocate (or was given no workspace to pass on) can still compute the loss.
+// In host code `g_noalloc_partials` is only a handle for the runtime, not a device address: the
+// address is looked up once per device and that pointer is what the kernels receive.
+// ---------------------------------------------------------------------------------------------
+static __device__ __align__(256) float g_noalloc_partials[TWIST_NOALLOC_MAX_SUBNETS * twist::kMseBlocks];
+
+namespace {
+constexpr int kMaxDevices = 64;
+float* g_noalloc_addr[kMaxDevices] = {nullptr};   // per device; written once, racing first calls write the same value
+
+// Device address of the scratch array on the current device (first call per device does the lookup).
+int noalloc_scratch(float** out) {
+  int dev = -1;
+  TWIST_CUDA_TRY(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= kMaxDevices) return TWIST_ERR_UNSUPPORTED;
+  if (!g_noalloc_addr[dev]) {
+    void* p = nullptr;
+    TWIST_CUDA_TRY(cudaGetSymbolAddress(&p, g_noalloc_partials));
+    if (!p) return TWIST_ERR_CUDA;
+    g_noalloc_addr[dev] = static_cast<float*>(p);
+  }
+  *out = g_noalloc_addr[dev];
+  return TWIST_OK;
+}
+}  // namespace
+
+extern "C" int32_t twist_mse_fwd_bwd_noalloc(const void* y, const void* tgt, void* dy, float* loss, int32_t n_subnets,
+                                             int32_t tokens, int32_t width, const int32_t* valid_cols,
+                                             int32_t seg_begin, int32_t seg_width, int32_t dtype, void* stream) {
+  if (n_subnets > TWIST_NOALLOC_MAX_SUBNETS) return TWIST_ERR_UNSUPPORTED;   // beyond the built-in scratch
+  if (n_subnets <= 0) return TWIST_ERR_SHAPE;
+  float* scratch = nullptr;
+  int rc = noalloc_scratch(&scratch);
+  if (rc != TWIST_OK) return rc;
+  // Every partial sum that the finishing kernel reads is written by this call's first kernel, so the
+  // contents left by an earlier call never need clearing.
+  return twist_mse_fwd_bwd(y, tgt, dy, loss, n_subnets, tokens, width, valid_cols, seg_begin, seg_width, dtype, scratch,
+                           (size_t)TWIST_NOALLOC_MAX_SUBNETS * twist::kMseBlocks * sizeof(float), stream);
+}
