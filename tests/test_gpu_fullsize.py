@@ -1,0 +1,192 @@
+"""Parity at the full sizes of the 7B-shaped workload (S=8, T=32768, d=4096, F=11008 -> f'=2752,
+8 of 32 heads), in the launch configuration bench.py times, on outputs the oracle can compute one
+by one: sampled token rows of every activation, sampled weight rows of every fused-SGD update
+(full-length contractions over all 32768 tokens), whole blueprints, whole gathered slices of
+sampled subnets, and the whole aggregate.  Inputs are seeded draws made on the device; the oracle
+reads the same bytes.  One layer, one local step."""
+from dataclasses import replace
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import twist_oracle as o
+from paper_2511_03983_b200 import inputs as I
+
+pytestmark = pytest.mark.gpu
+
+TOL = 2e-2
+SUBNETS = (1, 6)          # subnets whose activations / updates are checked
+N_ROWS, N_WROWS = 40, 12  # sampled token rows, sampled weight rows
+
+
+def rel_fro(got, want):
+    return float(np.linalg.norm(got - want) / max(np.linalg.norm(want), 1e-300))
+
+
+def f64(t):
+    return t.detach().float().cpu().numpy().astype(np.float64)
+
+
+@pytest.fixture(scope="module")
+def setup():
+    from paper_2511_03983_b200 import binding as B
+    from paper_2511_03983_b200.engine import RoundEngine
+    B.lib()
+    w = replace(I.PRESETS[4], n_layers=1, local_steps=1)
+    eng = RoundEngine(w, keep_f32_full=True)
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(w.seed_w)
+    for m, v in eng.full.items():
+        v[0].copy_((torch.randn(v[0].shape, generator=gen, device="cuda") * 0.02).to(torch.bfloat16))
+    gen.manual_seed(w.seed_x)
+    S, T, d = w.n_subnets, w.tokens, w.d_model
+    rnd = lambda width, std=1.0: (torch.randn(S, T, width, generator=gen, device="cuda") * std).to(torch.bfloat16)
+    eng.X, eng.Td, eng.Tq, eng.A = [rnd(d)], [rnd(d)], [rnd(eng.nq)], [rnd(eng.a_sub)]
+    full_np = {m: v[0].float().cpu().numpy() for m, v in eng.full.items()}
+    eng.sample_masks(0)
+    eng.gather_layer(0)
+    torch.cuda.synchronize()
+    bp = o.layer_blueprints(w, 0, 0)
+    rng = np.random.default_rng(5)
+    rows = np.sort(rng.choice(T, N_ROWS, replace=False))
+    return dict(B=B, eng=eng, w=w, full=full_np, bp=bp, rows=rows, rng=rng, gen=gen, rnd=rnd)
+
+
+def test_blueprints_and_index_data_bit_exact(setup):
+    eng, w, bp = setup["eng"], setup["w"], setup["bp"]
+    assert np.array_equal(eng.idx_ffn[0].cpu().numpy(), bp["ffn"])
+    assert np.array_equal(eng.idx_head[0].cpu().numpy(), bp["head"])
+    c, _, p = o.cover_and_pos(bp["ffn"], w.n_ffn_blocks)
+    assert np.array_equal(eng.cover_ffn[0].cpu().numpy().view(np.uint32), c)
+    assert np.array_equal(eng.pos_ffn[0].cpu().numpy(), p)
+    c, _, p = o.cover_and_pos(bp["head"], w.n_heads)
+    assert np.array_equal(eng.cover_head[0].cpu().numpy().view(np.uint32), c)
+    assert np.array_equal(eng.pos_head[0].cpu().numpy(), p)
+    assert np.array_equal(eng.kv_idx[0].cpu().numpy()[:, : w.head_keep], bp["kv_idx"][:, : w.head_keep])
+    assert np.array_equal(eng.kv_count[0].cpu().numpy(), bp["kv_count"])
+
+
+def test_gathered_slices_bit_exact(setup):
+    eng, w, bp, full = setup["eng"], setup["w"], setup["bp"], setup["full"]
+    f = w.f_sub
+    for s in SUBNETS:
+        sl = o.gather_layer(w, full, bp, s)
+        want = {"w_gu": np.concatenate([sl["gate"], sl["up"]]), "w_down": sl["down"], "w_qkv": sl["qkv"], "w_o": sl["o"]}
+        for name, arr in want.items():
+            got16 = getattr(eng, name)[s].float().cpu().numpy()
+            got32 = getattr(eng, name + "_m")[s].cpu().numpy()
+            assert np.array_equal(got16.view(np.uint32), arr.view(np.uint32)), (s, name)
+            assert np.array_equal(got32.view(np.uint32), arr.view(np.uint32)), (s, name, "master")
+
+
+def _sl64(setup, s):
+    sl = o.gather_layer(setup["w"], setup["full"], setup["bp"], s)
+    return {m: v.astype(np.float64) for m, v in sl.items()}
+
+
+def test_ffn_forward_backward_sampled(setup):
+    B, eng, w, rows, rng = setup["B"], setup["eng"], setup["w"], setup["rows"], setup["rng"]
+    S, T, d, f = w.n_subnets, w.tokens, w.d_model, w.f_sub
+    lr = w.lr
+    dY = setup["rnd"](d, 1e-4)
+    a = B.ffn_args(w.ffn_kind, w.dtype, S, T, d, f, eng.alpha_f, lr, x=eng.X[0], w_gu=eng.w_gu, w_down=eng.w_down,
+                   w_gu_master=eng.w_gu_m, w_down_master=eng.w_down_m, pre=eng.pre, hh=eng.hh, y=eng.y, dy=dY,
+                   dpre=eng.dpre, dx=eng.dx)
+    B.twist_subnet_ffn_fwd(a)
+    B.twist_subnet_ffn_bwd(a)
+    torch.cuda.synchronize()
+    assert B.twist_device_status() == 0
+    for s in SUBNETS:
+        sl = _sl64(setup, s)
+        X = f64(eng.X[0][s])
+        dYs = f64(dY[s])
+        # sampled token rows: every activation of the chain
+        Yw, saved = o.ffn_fwd(X[rows], sl["up"], sl["gate"], sl["down"], w.ffn_kind, eng.alpha_f, True)
+        dXw, _, _, _ = o.ffn_bwd(dYs[rows], X[rows], saved, sl["up"], sl["gate"], sl["down"], w.ffn_kind, eng.alpha_f, True)
+        r = torch.from_numpy(rows).cuda()
+        assert rel_fro(f64(eng.pre[s][r]), np.concatenate([saved["G"], saved["U"]], axis=1)) < TOL
+        assert rel_fro(f64(eng.hh[s][r]), saved["Hh"]) < TOL
+        assert rel_fro(f64(eng.y[s][r]), Yw) < TOL
+        assert rel_fro(f64(eng.dx[s][r]), dXw) < TOL
+        # sampled neurons: weight gradients with the full-length contraction over all T tokens; the
+        # FFN is separable per neuron except for Y and dX, so restricting the slices to J is exact
+        J = np.sort(rng.choice(f, N_WROWS, replace=False))
+        _, savedJ = o.ffn_fwd(X, sl["up"][J], sl["gate"][J], sl["down"][J], w.ffn_kind, eng.alpha_f, True)
+        _, dWu, dWg, dWd = o.ffn_bwd(dYs, X, savedJ, sl["up"][J], sl["gate"][J], sl["down"][J], w.ffn_kind,
+                                     eng.alpha_f, True)
+        Jt = torch.from_numpy(J).cuda()
+        upd_gate = f64(eng.w_gu_m[s][Jt]) - sl["gate"][J]
+        upd_up = f64(eng.w_gu_m[s][Jt + f]) - sl["up"][J]
+        upd_down = f64(eng.w_down_m[s][Jt]) - sl["down"][J]
+        assert rel_fro(upd_gate, -lr * dWg) < TOL, (s, "gate")
+        assert rel_fro(upd_up, -lr * dWu) < TOL, (s, "up")
+        assert rel_fro(upd_down, -lr * dWd) < TOL, (s, "down")
+        assert torch.equal(eng.w_gu[s][Jt], eng.w_gu_m[s][Jt].to(torch.bfloat16))
+
+
+def test_projections_forward_backward_sampled(setup):
+    B, eng, w, rows, rng = setup["B"], setup["eng"], setup["w"], setup["rows"], setup["rng"]
+    S, T, d = w.n_subnets, w.tokens, w.d_model
+    lr = w.lr
+    dQ = setup["rnd"](eng.nq, 1e-4)
+    dYo = setup["rnd"](d, 1e-4)
+    aq = B.proj_args(B.PROJ_QKV, w.dtype, S, T, d, eng.nq, 1.0, lr, in_=eng.X[0], w=eng.w_qkv, w_master=eng.w_qkv_m,
+                     out=eng.qkv_out, d_out=dQ, d_in=eng.dx)
+    B.twist_subnet_attn_proj_fwd(aq)
+    B.twist_subnet_attn_proj_bwd(aq)
+    ao = B.proj_args(B.PROJ_O, w.dtype, S, T, d, eng.a_sub, eng.alpha_a, lr, in_=eng.A[0], w=eng.w_o, w_master=eng.w_o_m,
+                     out=eng.y, d_out=dYo, d_in=eng.da)
+    B.twist_subnet_attn_proj_fwd(ao)
+    B.twist_subnet_attn_proj_bwd(ao)
+    torch.cuda.synchronize()
+    assert B.twist_device_status() == 0
+    r = torch.from_numpy(rows).cuda()
+    for s in SUBNETS:
+        sl = _sl64(setup, s)
+        X, A = f64(eng.X[0][s]), f64(eng.A[0][s])
+        dQs, dYs = f64(dQ[s]), f64(dYo[s])
+        assert rel_fro(f64(eng.qkv_out[s][r]), o.qkv_fwd(X[rows], sl["qkv"], True)) < TOL
+        assert rel_fro(f64(eng.dx[s][r]), o.qkv_bwd(dQs[rows], X[rows], sl["qkv"], True)[0]) < TOL
+        assert rel_fro(f64(eng.y[s][r]), o.o_fwd(A[rows], sl["o"], eng.alpha_a, True)) < TOL
+        assert rel_fro(f64(eng.da[s][r]), o.o_bwd(dYs[rows], A[rows], sl["o"], eng.alpha_a, True)[0]) < TOL
+        J = np.sort(rng.choice(eng.nq, N_WROWS, replace=False))
+        _, dWq = o.qkv_bwd(dQs[:, J], X, sl["qkv"][J], True)
+        assert rel_fro(f64(eng.w_qkv_m[s][torch.from_numpy(J).cuda()]) - sl["qkv"][J], -lr * dWq) < TOL
+        J = np.sort(rng.choice(eng.a_sub, N_WROWS, replace=False))
+        _, dWo = o.o_bwd(dYs, A[:, J], sl["o"][J], eng.alpha_a, True)
+        assert rel_fro(f64(eng.w_o_m[s][torch.from_numpy(J).cuda()]) - sl["o"][J], -lr * dWo) < TOL
+
+
+def test_aggregate_whole_layer(setup):
+    eng, w, bp, full, gen = setup["eng"], setup["w"], setup["bp"], setup["full"], setup["gen"]
+    S = w.n_subnets
+    # seeded "trained" masters (the oracle reads the same bytes)
+    for m in (eng.w_gu_m, eng.w_down_m, eng.w_qkv_m, eng.w_o_m):
+        m.copy_(torch.randn(m.shape, generator=gen, device="cuda") * 0.02)
+    eng.aggregate_layer(0)
+    torch.cuda.synchronize()
+    f, a_sub, dh, H = w.f_sub, eng.a_sub, w.d_head, w.n_heads
+    gu, down, qkv, wo = (t.cpu().numpy().astype(np.float64) for t in (eng.w_gu_m, eng.w_down_m, eng.w_qkv_m, eng.w_o_m))
+    kvs = [bp["kv_idx"][s][: bp["kv_count"][s]] for s in range(S)]
+    cases = [
+        ("gate", [gu[s, :f] for s in range(S)], bp["ffn"], 1, 0, slice(0, w.d_ff)),
+        ("up", [gu[s, f:] for s in range(S)], bp["ffn"], 1, 0, slice(0, w.d_ff)),
+        ("down", [down[s] for s in range(S)], bp["ffn"], 1, 0, slice(0, w.d_ff)),
+        ("qkv", [qkv[s, :a_sub] for s in range(S)], bp["head"], dh, 0, slice(0, H * dh)),
+        ("qkv", [qkv[s, a_sub:2 * a_sub] for s in range(S)], kvs, dh, H * dh, slice(H * dh, 2 * H * dh)),
+        ("qkv", [qkv[s, 2 * a_sub:] for s in range(S)], kvs, dh, 2 * H * dh, slice(2 * H * dh, 3 * H * dh)),
+        ("o", [wo[s] for s in range(S)], bp["head"], dh, 0, slice(0, H * dh)),
+    ]
+    for name, subs, blue, br, off, rows in cases:
+        before = full[name].astype(np.float64)
+        want = o.aggregate(before, subs, blue, br, row_offset=off)[rows]
+        mag = o.aggregate(np.abs(before), [np.abs(v) for v in subs], blue, br, row_offset=off)[rows]
+        got = eng.full_f32[name][0].cpu().numpy().astype(np.float64)[rows]
+        held = np.any(want != before[rows], axis=1)
+        assert held.any()
+        err = np.abs(got[held] - want[held]) / np.maximum(mag[held], 1e-30)
+        assert err.max() <= 1e-6, (name, err.max())
+        shadow = eng.full[name][0][rows]
+        assert torch.equal(shadow[torch.from_numpy(held).cuda()],
+                           eng.full_f32[name][0][rows][torch.from_numpy(held).cuda()].to(torch.bfloat16))
