@@ -214,7 +214,7 @@ def run_ours(args, w):
     B.lib()
     bf16 = w.dtype == I.DTYPE_BF16
     td = torch.bfloat16 if bf16 else torch.float32
-    eng = RoundEngine(w, keep_f32_full=True, compute_dx=True)
+    eng = RoundEngine(w, keep_f32_full=True, compute_dx=True, fuse_loss=True, store_outputs=False)
     gen = torch.Generator(device="cuda")
     gen.manual_seed(w.seed_w + 7919 * rank)
     for m, v in eng.full.items():                         # weights ~ N(0, 0.02^2), one matrix at a time

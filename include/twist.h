@@ -187,13 +187,26 @@ typedef struct {
   float* w_down_master;
   void* pre;            /* device [S][T][g*f_sub]  fwd: out, bwd: in */
   void* hh;             /* device [S][T][f_sub]    fwd: out, bwd: in */
-  void* y;              /* device [S][T][d]        fwd: out */
-  const void* dy;       /* device [S][T][d]        bwd: in */
+  void* y;              /* device [S][T][d]        fwd: out (may be NULL with fused loss, bf16 dtype) */
+  const void* dy;       /* device [S][T][d]        bwd: in (written by a forward call with fused loss) */
   void* dpre;           /* device [S][T][g*f_sub]  bwd: out (gradient w.r.t. pre) */
   void* dx;             /* device [S][T][d]        bwd: out, may be NULL */
   float* dw_gu;         /* device fp32 [S][g*f_sub][d] gradient dump, may be NULL (required in fp32 dtype) */
   float* dw_down;       /* device fp32 [S][f_sub][d]   gradient dump, may be NULL (required in fp32 dtype) */
+  /* Optional fused loss of the forward call (see "Fused loss" below); all NULL / 0 to leave it out. */
+  const void* tgt;      /* device [S][T][d] regression target */
+  float* loss;          /* device fp32 [S]: out */
+  void* loss_ws;        /* device scratch, at least twist_fused_loss_workspace_bytes(S, T, d) bytes */
+  size_t loss_ws_bytes;
 } twist_ffn_args;
+
+/* Fused loss.  When `tgt` is set, twist_subnet_ffn_fwd / twist_subnet_attn_proj_fwd also evaluate the loss
+ * of twist_mse_fwd_bwd on their output inside the producing kernel: loss[s] is written, and the
+ * gradient of the loss with respect to the output is written where the backward call reads it
+ * (twist_ffn_args.dy, twist_proj_args.d_out), exactly as if twist_mse_fwd_bwd had been called on the
+ * stored output.  The output itself (y / out) may then be NULL: it is not stored.  Results are
+ * deterministic (fixed summation order). */
+size_t twist_fused_loss_workspace_bytes(int32_t n_subnets, int32_t tokens, int32_t width);
 
 int32_t twist_subnet_ffn_fwd(const twist_ffn_args* a /*host*/, void* stream);
 int32_t twist_subnet_ffn_bwd(const twist_ffn_args* a /*host*/, void* stream);
@@ -210,10 +223,17 @@ typedef struct {
   const void* in;       /* device */
   void* w;              /* device [S][n][d] */
   float* w_master;      /* device fp32 master (bf16 dtype, bwd only) */
-  void* out;            /* fwd: out */
-  const void* d_out;    /* bwd: in */
+  void* out;            /* fwd: out (may be NULL with fused loss, bf16 dtype) */
+  const void* d_out;    /* bwd: in (written by a forward call with fused loss) */
   void* d_in;           /* bwd: out, may be NULL */
   float* dw;            /* device fp32 [S][n][d] gradient dump, may be NULL (required in fp32 dtype) */
+  /* Optional fused loss of the forward call (see "Fused loss"); all NULL / 0 to leave it out. */
+  const void* tgt;      /* device, same shape as the output */
+  float* loss;          /* device fp32 [S]: out */
+  void* loss_ws;        /* device scratch, at least twist_fused_loss_workspace_bytes(S, T, output width) bytes */
+  size_t loss_ws_bytes;
+  const int32_t* valid_cols;   /* column mask of twist_mse_fwd_bwd (device int32 [S]) or NULL */
+  int32_t seg_begin, seg_width;
 } twist_proj_args;
 
 int32_t twist_subnet_attn_proj_fwd(const twist_proj_args* a /*host*/, void* stream);

@@ -30,7 +30,7 @@ EXPORTS = [
     "twist_abi_version", "twist_strerror", "twist_last_cuda_error", "twist_device_status", "twist_sample_masks",
     "twist_kv_groups", "twist_gather_subnets", "twist_aggregate", "twist_subnet_ffn_fwd", "twist_subnet_ffn_bwd",
     "twist_subnet_attn_proj_fwd", "twist_subnet_attn_proj_bwd", "twist_mse_workspace_bytes", "twist_mse_fwd_bwd",
-    "twist_mse_fwd_bwd_noalloc",
+    "twist_mse_fwd_bwd_noalloc", "twist_fused_loss_workspace_bytes",
 ]
 
 
@@ -59,14 +59,17 @@ class FfnArgs(C.Structure):
                 ("x", C.c_void_p), ("w_gu", C.c_void_p), ("w_down", C.c_void_p), ("w_gu_master", C.c_void_p),
                 ("w_down_master", C.c_void_p), ("pre", C.c_void_p), ("hh", C.c_void_p), ("y", C.c_void_p),
                 ("dy", C.c_void_p), ("dpre", C.c_void_p), ("dx", C.c_void_p), ("dw_gu", C.c_void_p),
-                ("dw_down", C.c_void_p)]
+                ("dw_down", C.c_void_p), ("tgt", C.c_void_p), ("loss", C.c_void_p), ("loss_ws", C.c_void_p),
+                ("loss_ws_bytes", C.c_size_t)]
 
 
 class ProjArgs(C.Structure):
     _fields_ = [("which", C.c_int32), ("dtype", C.c_int32), ("n_subnets", C.c_int32), ("tokens", C.c_int32),
                 ("d_model", C.c_int32), ("n", C.c_int32), ("out_scale", C.c_float), ("lr", C.c_float),
                 ("in_", C.c_void_p), ("w", C.c_void_p), ("w_master", C.c_void_p), ("out", C.c_void_p),
-                ("d_out", C.c_void_p), ("d_in", C.c_void_p), ("dw", C.c_void_p)]
+                ("d_out", C.c_void_p), ("d_in", C.c_void_p), ("dw", C.c_void_p), ("tgt", C.c_void_p),
+                ("loss", C.c_void_p), ("loss_ws", C.c_void_p), ("loss_ws_bytes", C.c_size_t),
+                ("valid_cols", C.c_void_p), ("seg_begin", C.c_int32), ("seg_width", C.c_int32)]
 
 
 _lib_handle = None
@@ -97,6 +100,8 @@ def lib() -> C.CDLL:
             getattr(h, name).argtypes = [C.c_void_p, C.c_void_p]
         h.twist_mse_workspace_bytes.restype = C.c_size_t
         h.twist_mse_workspace_bytes.argtypes = [C.c_int32]
+        h.twist_fused_loss_workspace_bytes.restype = C.c_size_t
+        h.twist_fused_loss_workspace_bytes.argtypes = [C.c_int32, C.c_int32, C.c_int32]
         h.twist_mse_fwd_bwd.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32,
                                         C.c_int32, C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_size_t,
                                         C.c_void_p]
@@ -105,7 +110,7 @@ def lib() -> C.CDLL:
         for name in EXPORTS:
             f = getattr(h, name)
             if name not in ("twist_abi_version", "twist_strerror", "twist_last_cuda_error",
-                            "twist_mse_workspace_bytes"):
+                            "twist_mse_workspace_bytes", "twist_fused_loss_workspace_bytes"):
                 f.restype = C.c_int32
         _lib_handle = h
     return _lib_handle
@@ -183,12 +188,18 @@ def twist_aggregate(segs: Sequence[AggregateSegment], n_subnets, d, dtype, live_
            "twist_aggregate")
 
 
+def _ws_bytes(ws) -> int:
+    return 0 if ws is None else ws.numel() * ws.element_size()
+
+
 def ffn_args(ffn_kind, dtype, n_subnets, tokens, d_model, f_sub, out_scale, lr=0.0, **t) -> FfnArgs:
+    """Marshals twist_ffn_args.  tgt / loss / loss_ws request the fused loss of the forward call."""
     names = ["x", "w_gu", "w_down", "w_gu_master", "w_down_master", "pre", "hh", "y", "dy", "dpre", "dx", "dw_gu",
-             "dw_down"]
+             "dw_down", "tgt", "loss", "loss_ws"]
     unknown = set(t) - set(names)
     assert not unknown, unknown
-    return FfnArgs(ffn_kind, dtype, n_subnets, tokens, d_model, f_sub, out_scale, lr, *[_ptr(t.get(n)) for n in names])
+    return FfnArgs(ffn_kind, dtype, n_subnets, tokens, d_model, f_sub, out_scale, lr, *[_ptr(t.get(n)) for n in names],
+                   _ws_bytes(t.get("loss_ws")))
 
 
 def twist_subnet_ffn_fwd(a: FfnArgs):
@@ -199,11 +210,14 @@ def twist_subnet_ffn_bwd(a: FfnArgs):
     _check(lib().twist_subnet_ffn_bwd(C.byref(a), _stream()), "twist_subnet_ffn_bwd")
 
 
-def proj_args(which, dtype, n_subnets, tokens, d_model, n, out_scale, lr=0.0, **t) -> ProjArgs:
-    names = ["in_", "w", "w_master", "out", "d_out", "d_in", "dw"]
-    unknown = set(t) - set(names)
+def proj_args(which, dtype, n_subnets, tokens, d_model, n, out_scale, lr=0.0, seg_begin=0, seg_width=0, **t) -> ProjArgs:
+    """Marshals twist_proj_args.  tgt / loss / loss_ws (and the optional column mask valid_cols,
+    seg_begin, seg_width) request the fused loss of the forward call."""
+    names = ["in_", "w", "w_master", "out", "d_out", "d_in", "dw", "tgt", "loss", "loss_ws"]
+    unknown = set(t) - set(names) - {"valid_cols"}
     assert not unknown, unknown
-    return ProjArgs(which, dtype, n_subnets, tokens, d_model, n, out_scale, lr, *[_ptr(t.get(n)) for n in names])
+    return ProjArgs(which, dtype, n_subnets, tokens, d_model, n, out_scale, lr, *[_ptr(t.get(n)) for n in names],
+                    _ws_bytes(t.get("loss_ws")), _ptr(t.get("valid_cols")), seg_begin, seg_width)
 
 
 def twist_subnet_attn_proj_fwd(a: ProjArgs):
@@ -216,6 +230,10 @@ def twist_subnet_attn_proj_bwd(a: ProjArgs):
 
 def twist_mse_workspace_bytes(n_subnets: int) -> int:
     return lib().twist_mse_workspace_bytes(n_subnets)
+
+
+def twist_fused_loss_workspace_bytes(n_subnets: int, tokens: int, width: int) -> int:
+    return lib().twist_fused_loss_workspace_bytes(n_subnets, tokens, width)
 
 
 def twist_mse_fwd_bwd(y, tgt, dy, loss, n_subnets, tokens, width, valid_cols, seg_begin, seg_width, dtype, ws):

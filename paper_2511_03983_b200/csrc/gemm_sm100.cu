@@ -42,22 +42,130 @@ int make_map(CUtensorMap* map, const GemmOperand& op, int groups, int box_rows) 
   return TWIST_OK;
 }
 
+// CTA pairs that can be resident at once (one CTA per SM, pairs on neighbouring SMs); queried once per
+// kernel instance and device.  More tiles than pairs: the persistent pairs stride over the tile list.
+template <int AM, int BM_, int EPI>
+int resident_pairs(int* out) {
+  static int cached[64] = {0};
+  int dev = 0;
+  TWIST_CUDA_TRY(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= 64) return TWIST_ERR_UNSUPPORTED;
+  if (cached[dev] == 0) {
+    TWIST_CUDA_TRY(cudaFuncSetAttribute(gemm_kernel<AM, BM_, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        gemm_smem_bytes(EPI != EPI_SGD)));
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = dim3(2 * (sm_count() / 2));
+    cfg.blockDim = dim3(kGemmThreads);
+    cfg.dynamicSmemBytes = gemm_smem_bytes(EPI != EPI_SGD);
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeClusterDimension;
+    attr.val.clusterDim.x = 2; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, gemm_kernel<AM, BM_, EPI>, &cfg) != cudaSuccess || n <= 0) {
+      cudaGetLastError();
+      n = sm_count() / 2;
+    }
+    cached[dev] = n < sm_count() / 2 ? n : sm_count() / 2;
+  }
+  *out = cached[dev];
+  return TWIST_OK;
+}
+
+// 3-D map over a bf16 tensor [groups][rows][cols] whose rows are `row_stride` elements apart, for the
+// epilogue's 32 x 32 boxes (64-byte rows in shared memory, 64-byte swizzle).  Loads read zeros outside
+// the tensor, stores write nothing there.
+int make_box_map(CUtensorMap* map, const void* ptr, int rows, int cols, long long row_stride, int groups) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) { note_cuda_error(cudaErrorUnknown, "cuTensorMapEncodeTiled entry point"); return TWIST_ERR_CUDA; }
+  if (!ptr || !aligned16(ptr) || (row_stride * 2) % 16 != 0) return TWIST_ERR_SHAPE;
+  cuuint64_t dims[3] = {(cuuint64_t)cols, (cuuint64_t)rows, (cuuint64_t)groups};
+  cuuint64_t strides[2] = {(cuuint64_t)row_stride * 2, (cuuint64_t)rows * (cuuint64_t)row_stride * 2};
+  cuuint32_t box[3] = {32, 32, 1};
+  cuuint32_t estr[3] = {1, 1, 1};
+  CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    note_cuda_error(cudaErrorInvalidValue, "cuTensorMapEncodeTiled (epilogue box)");
+    return TWIST_ERR_CUDA;
+  }
+  return TWIST_OK;
+}
+
+// Tensor maps of the boxes each epilogue reads and writes (layout of EpiMaps in the kernel header).
+int make_epilogue_maps(int epi, const GemmParams& p, const CUtensorMap& filler, EpiMaps* e) {
+  for (int i = 0; i < 4; ++i) e->m[i] = filler;          // unused entries stay valid descriptors
+  const int M = p.M, N = p.N, G = p.groups;
+  int rc = TWIST_OK;
+  auto mk = [&](int i, const void* ptr, int cols, long long stride) {
+    if (rc == TWIST_OK) rc = make_box_map(&e->m[i], ptr, M, cols, stride, G);
+  };
+  switch (epi) {
+    case EPI_STORE: mk(0, p.out0, N, N); break;
+    case EPI_MSE:
+      mk(0, p.in0, N, N); mk(1, p.out1, N, N);
+      if (p.out0) mk(2, p.out0, N, N);
+      break;
+    case EPI_SWIGLU_FWD: mk(0, p.out0, N, 2LL * N); mk(1, p.out0 + N, N, 2LL * N); mk(2, p.out1, N, N); break;
+    case EPI_ACT_FWD: mk(0, p.out0, N, N); mk(1, p.out1, N, N); break;
+    case EPI_DSWIGLU:
+      mk(0, p.in0, N, 2LL * N); mk(1, p.in0 + N, N, 2LL * N);
+      mk(2, p.out0, N, 2LL * N); mk(3, p.out0 + N, N, 2LL * N);
+      break;
+    case EPI_DACT: mk(0, p.in0, N, N); mk(1, p.out0, N, N); break;
+    default: break;                                        // EPI_SGD: plain global accesses
+  }
+  return rc;
+}
+
 template <int AM, int BM_, int EPI>
 int launch(const CUtensorMap& ta, const CUtensorMap& tb, const GemmParams& p, cudaStream_t st) {
-  static bool configured = false;
-  if (!configured) {
-    TWIST_CUDA_TRY(cudaFuncSetAttribute(gemm_kernel<AM, BM_, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                        kGemmSmemBytes));
-    configured = true;
-  }
+  int pairs = 0;
+  int rc = resident_pairs<AM, BM_, EPI>(&pairs);
+  if (rc != TWIST_OK) return rc;
   const int tiles = p.groups * p.m_tiles * p.n_tiles;
-  const int grid = tiles < sm_count() ? tiles : sm_count();
-  gemm_kernel<AM, BM_, EPI><<<grid, kGemmThreads, kGemmSmemBytes, st>>>(ta, tb, p);
+  const int grid = 2 * (tiles < pairs ? tiles : pairs);
+  EpiMaps te;
+  rc = make_epilogue_maps(EPI, p, ta, &te);
+  if (rc != TWIST_OK) return rc;
+  gemm_kernel<AM, BM_, EPI><<<grid, kGemmThreads, gemm_smem_bytes(EPI != EPI_SGD), st>>>(ta, tb, te, p);
   TWIST_LAUNCH_CHECK();
   return TWIST_OK;
 }
 
+// loss[g] = (sum of the group's partial sums, fixed order) / (tokens * valid columns of the group)
+__global__ void fused_loss_finish_kernel(const float* __restrict__ partial, long long per_group, int tokens, int width,
+                                         const int32_t* __restrict__ valid_cols, int seg_begin, int seg_width,
+                                         float* __restrict__ loss) {
+  const int g = blockIdx.x, lane = threadIdx.x;
+  const float* src = partial + (long long)g * per_group;
+  double acc = 0.0;
+  for (long long i = lane; i < per_group; i += 32) acc += (double)src[i];
+  for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+  if (lane == 0) {
+    const int vc = valid_cols ? valid_cols[g] : seg_width;
+    const long long n_valid = seg_begin + (long long)((width - seg_begin) / seg_width) * vc;
+    loss[g] = (float)(acc / ((double)tokens * (double)n_valid));
+  }
+}
+
 }  // namespace
+
+size_t fused_loss_partials(int groups, int M, int N) {
+  const size_t m_tiles = (size_t)(M + kBM - 1) / kBM, n_tiles = (size_t)(N + kBN - 1) / kBN;
+  return (size_t)groups * m_tiles * n_tiles * 8;
+}
+
+int finish_fused_loss(const float* partial, int groups, int M, int N, const int32_t* valid_cols, int seg_begin,
+                      int seg_width, float* loss, cudaStream_t st) {
+  const long long per_group = (long long)(fused_loss_partials(groups, M, N) / (size_t)groups);
+  fused_loss_finish_kernel<<<groups, 32, 0, st>>>(partial, per_group, M, N, valid_cols, seg_begin, seg_width, loss);
+  TWIST_LAUNCH_CHECK();
+  return TWIST_OK;
+}
 
 int launch_gemm_bf16(int layout, int epi, const GemmOperand& A, const GemmOperand& B, GemmParams p, cudaStream_t st) {
   if (!A.ptr || !B.ptr) return TWIST_ERR_NULL;
@@ -67,7 +175,7 @@ int launch_gemm_bf16(int layout, int epi, const GemmOperand& A, const GemmOperan
   const int a_major = layout == 2 ? MAJOR_MN : MAJOR_K;
   const int b_major = layout == 0 ? MAJOR_K : MAJOR_MN;
   p.m_tiles = (p.M + kBM - 1) / kBM;
-  p.n_tiles = epi == EPI_SWIGLU_FWD ? (p.N + kBN / 2 - 1) / (kBN / 2) : (p.N + kBN - 1) / kBN;
+  p.n_tiles = epi == EPI_SWIGLU_FWD ? (p.N + kCtaN - 1) / kCtaN : (p.N + kBN - 1) / kBN;
   if ((long long)p.groups * p.m_tiles * p.n_tiles > 0x7fffffffLL) return TWIST_ERR_UNSUPPORTED;
   p.status = device_status_ptr();
   if (!p.status) return TWIST_ERR_CUDA;
@@ -83,10 +191,12 @@ int launch_gemm_bf16(int layout, int epi, const GemmOperand& A, const GemmOperan
       case EPI_ACT_FWD: return launch<MAJOR_K, MAJOR_K, EPI_ACT_FWD>(ta, tb, p, st);
       case EPI_DSWIGLU: return launch<MAJOR_K, MAJOR_K, EPI_DSWIGLU>(ta, tb, p, st);
       case EPI_DACT: return launch<MAJOR_K, MAJOR_K, EPI_DACT>(ta, tb, p, st);
+      case EPI_MSE: return launch<MAJOR_K, MAJOR_K, EPI_MSE>(ta, tb, p, st);
       default: return TWIST_ERR_UNSUPPORTED;
     }
   }
   if (layout == 1 && epi == EPI_STORE) return launch<MAJOR_K, MAJOR_MN, EPI_STORE>(ta, tb, p, st);
+  if (layout == 1 && epi == EPI_MSE) return launch<MAJOR_K, MAJOR_MN, EPI_MSE>(ta, tb, p, st);
   if (layout == 2 && epi == EPI_SGD) return launch<MAJOR_MN, MAJOR_MN, EPI_SGD>(ta, tb, p, st);
   return TWIST_ERR_UNSUPPORTED;
 }

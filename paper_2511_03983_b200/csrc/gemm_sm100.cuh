@@ -1,6 +1,13 @@
 // Grouped bf16 GEMM for sm_100a: TMA -> shared-memory ring -> tcgen05.mma (fp32 accumulators in
-// tensor memory, double buffered) -> fused epilogues.  One persistent CTA per SM walks the tile list
-// of all S subnets ("groups"), so the S independent problems of a local-training step are one launch.
+// tensor memory, double buffered) -> fused epilogues.  Persistent CTA pairs (clusters of two CTAs on
+// neighbouring SMs, one pair-wide 256 x 256 tile at a time) walk the tile list of all S subnets
+// ("groups"), so the S independent problems of a local-training step are one launch.
+//
+// A pair shares one tile: CTA r of the pair loads the A rows [128 r, 128 r + 128) and the B columns
+// [128 r, 128 r + 128) of the tile into its own shared memory, and the leader (r = 0) issues
+// tcgen05.mma.cta_group::2, which reads both CTAs' shared memory and writes each CTA's 128 accumulator
+// rows into that CTA's tensor memory.  Per SM and k-block this moves 32 KB from L2 instead of the
+// 48 KB a single-CTA 128 x 256 tile needs; no load is multicast.
 //
 //   D[g] (M x N) = op(A[g]) op(B[g]),  contraction length K, for g < groups.
 // Operands are dense row-major [groups][rows][cols] bf16.  "K-major" = the contraction index is the
@@ -10,8 +17,11 @@
 //   NN (A K-major, B MN-major)  h W              : down / o forward, dX
 //   TN (A MN-major, B MN-major) act^T other      : every weight gradient (contraction over tokens)
 //
-// Warp roles (192 threads): warps 0-3 epilogue (warp w owns TMEM lanes 32w..32w+31), warp 4 TMA
-// producer (one lane), warp 5 TMEM allocator + MMA issuer (one lane).
+// Warp roles (192 threads per CTA): warps 0-3 epilogue (warp w owns TMEM lanes 32w..32w+31), warp 4 TMA
+// producer (one lane), warp 5 TMEM allocator (both CTAs) + MMA issuer (one lane, leader CTA only).
+// Barriers: both producers' copies complete on the leader's "full" barrier; the leader's
+// tcgen05.commit signals "stage empty" and "accumulator full" in both CTAs; the epilogue warps of both
+// CTAs arrive on the leader's "accumulator empty" barrier.
 // Every mbarrier wait is bounded in wall time; on expiry the CTA records a timeout and leaves.
 #pragma once
 #include <cuda.h>
@@ -21,16 +31,29 @@
 namespace twist {
 
 enum { MAJOR_K = 0, MAJOR_MN = 1 };
-enum { EPI_STORE = 0, EPI_SWIGLU_FWD = 1, EPI_ACT_FWD = 2, EPI_DSWIGLU = 3, EPI_DACT = 4, EPI_SGD = 5 };
+enum { EPI_STORE = 0, EPI_SWIGLU_FWD = 1, EPI_ACT_FWD = 2, EPI_DSWIGLU = 3, EPI_DACT = 4, EPI_SGD = 5, EPI_MSE = 6 };
 
-constexpr int kBM = 128, kBN = 256, kBK = 64, kStages = 4, kUmmaK = 16;
-constexpr int kABytes = kBM * kBK * 2;            // 16 KB
-constexpr int kBBytes = kBN * kBK * 2;            // 32 KB
-constexpr int kStageBytes = kABytes + kBBytes;    // 48 KB
+constexpr int kBM = 256, kBN = 256, kBK = 64, kUmmaK = 16;   // tile of a CTA pair
+constexpr int kCtaM = kBM / 2, kCtaN = kBN / 2;   // rows of A / columns of B that one CTA of the pair loads
+constexpr int kABytes = kCtaM * kBK * 2;          // 16 KB
+constexpr int kBBytes = kCtaN * kBK * 2;          // 16 KB
+constexpr int kStageBytes = kABytes + kBBytes;    // 32 KB per CTA and stage
 constexpr int kGemmThreads = 192;
-constexpr int kGemmSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
-constexpr int kTmemCols = 512;                    // two 128 x 256 fp32 accumulators
-constexpr int kRasterGroupM = 16;                 // m-tiles per raster group (L2 reuse of A and B tiles)
+// Epilogue staging: every epilogue warp owns 16 KB in which 32-row x 32-column bf16 boxes (2 KB, 64-byte rows,
+// 64-byte swizzle) travel between global memory and the warp by TMA: operands the epilogue reads arrive as boxes,
+// results leave as boxes, so every global access of the epilogue is a full-line bulk transfer.
+constexpr int kEpiBoxBytes = 32 * 32 * 2;
+constexpr int kEpiWarpBytes = 16384;
+constexpr int kEpiBytes = 4 * kEpiWarpBytes;
+constexpr int kCtrlBytes = 384;
+// Operand ring: 5 stages of 32 KB beside the epilogue staging.  The weight-gradient kernel stages nothing and
+// could hold 7, but measured no faster with them (it is bound by power, not by latency), so it keeps 5 too.
+__host__ __device__ constexpr int gemm_stages(bool /*staged_epilogue*/) { return 5; }
+__host__ __device__ constexpr int gemm_smem_bytes(bool staged_epilogue) {
+  return gemm_stages(staged_epilogue) * kStageBytes + (staged_epilogue ? kEpiBytes : 0) + 1024 /*alignment slack*/ + kCtrlBytes;
+}
+constexpr int kTmemCols = 512;                    // two 128 x 256 fp32 accumulators per CTA
+constexpr int kRasterGroupM = 8;                  // m-tiles per raster group (L2 reuse of A and B tiles)
 
 struct GemmParams {
   int M, N, K;          // per group.  EPI_SWIGLU_FWD: N = f_sub (neurons); the tile holds 128 gate + 128 up columns
@@ -39,13 +62,34 @@ struct GemmParams {
   int b_split;          // EPI_SWIGLU_FWD: row of the first "up" weight inside B (= f_sub)
   int act_kind;         // TWIST_FFN_*
   float scale, lr;
-  __nv_bfloat16* out0;  // STORE: D [g][M][N].  *_FWD: pre.  D*: dpre.  SGD: bf16 compute copy of the weights
-  __nv_bfloat16* out1;  // *_FWD: hh [g][M][f_sub]
-  const __nv_bfloat16* in0;   // DSWIGLU / DACT: pre
+  __nv_bfloat16* out0;  // STORE: D [g][M][N].  *_FWD: pre.  D*: dpre.  SGD: bf16 compute copy of the weights.  MSE: D or null
+  __nv_bfloat16* out1;  // *_FWD: hh [g][M][f_sub].  MSE: gradient of the loss w.r.t. D, [g][M][N]
+  const __nv_bfloat16* in0;   // DSWIGLU / DACT: pre.  MSE: target [g][M][N]
   float* master;        // SGD: fp32 master weights [g][M][N] (updated when lr != 0)
-  float* dw;            // SGD: optional fp32 gradient dump [g][M][N]
+  float* dw;            // SGD: optional fp32 gradient dump [g][M][N].  MSE: partial sums, 8 per tile (2 CTAs x 4 warps)
+  const int32_t* valid_cols;   // MSE: valid columns per column group and subnet [groups], or null (all valid)
+  int seg_begin, seg_width;    // MSE: columns [0, seg_begin) valid, then groups of seg_width columns (see twist_mse_fwd_bwd)
   int* status;          // device status word
 };
+
+// Tensor maps of the epilogue's boxes (box = 32 columns x 32 rows of a dense bf16 [groups][M][cols] tensor):
+//   STORE: 0 D.            MSE: 0 target (in), 1 dD (out), 2 D (out, optional).
+//   SWIGLU_FWD: 0 G, 1 U (the two halves of pre), 2 hh.        ACT_FWD: 0 pre, 1 hh.
+//   DSWIGLU: 0 G, 1 U (in), 2 dG, 3 dU (out).                  DACT: 0 pre (in), 1 dpre (out).
+struct EpiMaps { CUtensorMap m[4]; };
+
+// Boxes per chunk buffer, how many of them are read from global memory first, and buffers per warp.
+__host__ __device__ constexpr int epi_slots(int epi) {
+  return epi == EPI_SWIGLU_FWD ? 3 : (epi == EPI_MSE || epi == EPI_ACT_FWD || epi == EPI_DSWIGLU) ? 2 : 1;
+}
+__host__ __device__ constexpr int epi_in_slots(int epi) {
+  return epi == EPI_DSWIGLU ? 2 : (epi == EPI_MSE || epi == EPI_DACT) ? 1 : 0;
+}
+__host__ __device__ constexpr int epi_bufs(int epi) { return epi_slots(epi) == 3 ? 2 : 4; }
+
+// Registers of one 32-column chunk of accumulator words.
+template <int EPI> struct EpiAcc { uint32_t r0[32]; };
+template <> struct EpiAcc<EPI_SWIGLU_FWD> { uint32_t r0[32], r1[32]; };
 
 // ---------------------------------------------------------------------------------------------
 // PTX wrappers
@@ -65,10 +109,28 @@ __device__ inline uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
   uint32_t done;
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
       "selp.u32 %0, 1, 0, p;\n\t}"
       : "=r"(done) : "r"(bar), "r"(parity) : "memory");
   return done;
+}
+// Cluster helpers: rank of this CTA in its pair, address of a shared-memory location of CTA `rank`
+// in the cluster-wide shared window, arrival on a barrier given by such an address, cluster barrier.
+__device__ inline uint32_t cluster_rank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ inline uint32_t map_to_cta(uint32_t saddr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(saddr), "r"(rank));
+  return r;
+}
+__device__ inline void mbar_arrive_cluster(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ inline void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
 __device__ inline uint64_t global_timer_ns() {
   uint64_t t;
@@ -92,10 +154,35 @@ __device__ inline bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* ab
   }
 }
 
+// Tiled copy into this CTA's shared memory; completion bytes are counted on `bar`, which may be a
+// barrier of the other CTA of the pair (cluster-window address).
 __device__ inline void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2) : "memory");
+}
+// Tiled copy into this CTA's shared memory, completion counted on a barrier of this CTA.
+__device__ inline void tma_load_3d_local(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2) {
   asm volatile(
       "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
       ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2) : "memory");
+}
+// Tiled store of a shared-memory box; elements outside the tensor are not written.
+__device__ inline void tma_store_3d(const CUtensorMap* map, uint32_t src, int c0, int c1, int c2) {
+  asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%2, %3, %4}], [%1];"
+               ::"l"(map), "r"(src), "r"(c0), "r"(c1), "r"(c2) : "memory");
+}
+__device__ inline void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+template <int N>
+__device__ inline void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
+__device__ inline void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ inline uint4 lds128(uint32_t a) {
+  uint4 v;
+  asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(a));
+  return v;
+}
+__device__ inline void sts128(uint32_t a, uint4 v) {
+  asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(a), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
 }
 __device__ inline void tma_prefetch_desc(const CUtensorMap* map) {
   asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
@@ -103,14 +190,18 @@ __device__ inline void tma_prefetch_desc(const CUtensorMap* map) {
 
 __device__ inline void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ inline void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ inline void tc_commit(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+// Arrives, once the MMAs issued so far have completed, on the barrier at this shared-memory offset in
+// both CTAs of the pair.
+__device__ inline void tc_commit_pair(uint32_t bar) {
+  const uint16_t both = 3;
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+               ::"r"(bar), "h"(both) : "memory");
 }
 __device__ inline void tc_mma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
       "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
       ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
 }
 __device__ inline void tc_ld32(uint32_t taddr, uint32_t (&r)[32]) {
@@ -132,7 +223,7 @@ __device__ inline uint64_t smem_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_
          (1ull << 46) | (2ull << 61);
 }
 
-// Instruction descriptor: fp32 accumulate, bf16 x bf16, M = 128, N = 256, operand majors as given.
+// Instruction descriptor: fp32 accumulate, bf16 x bf16, M = 256 (over the CTA pair), N = 256, operand majors as given.
 __host__ __device__ constexpr uint32_t instr_desc(int a_major, int b_major) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)a_major << 15) | ((uint32_t)b_major << 16) |
          ((uint32_t)(kBN >> 3) << 17) | ((uint32_t)(kBM >> 4) << 24);
@@ -164,6 +255,10 @@ __device__ inline void load_row32(const __nv_bfloat16* src, uint32_t (&w)[16], i
   }
 }
 
+// 1 / (1 + e^-x) with the hardware exponential and approximate reciprocal (error ~1e-7 relative, far below
+// the bf16 rounding of every value it feeds); the IEEE division costs several times the rest of the epilogue.
+__device__ inline float sigmoid_fast(float x) { return __fdividef(1.f, 1.f + __expf(-x)); }
+
 __device__ inline float act_fwd(float x, int kind) {
   return kind == TWIST_FFN_RELU ? fmaxf(x, 0.f) : 0.5f * x * (1.f + erff(x * 0.70710678118654752f));
 }
@@ -188,14 +283,21 @@ __device__ inline void tile_coords(const GemmParams& p, int tile, int& g, int& m
 }
 
 template <int A_MAJOR, int B_MAJOR, int EPI>
-__global__ void __launch_bounds__(kGemmThreads, 1)
-gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const GemmParams p) {
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 1)
+gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+            const __grid_constant__ EpiMaps tmE, const GemmParams p) {
+  constexpr bool kStaged = EPI != EPI_SGD;
+  constexpr int kStages = gemm_stages(kStaged);
   extern __shared__ unsigned char smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   unsigned char* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
-  const uint32_t bar_base = smem_base + kStages * kStageBytes;
-  volatile uint32_t* ctrl = reinterpret_cast<volatile uint32_t*>(smem_gen + kStages * kStageBytes);
-  // control block (in 4-byte words): full[4] @0, empty[4] @8, tmem_full[2] @16, tmem_empty[2] @20, tmem ptr @24, abort @25
+  const uint32_t epi_base = smem_base + kStages * kStageBytes;
+  const uint32_t bar_base = epi_base + (kStaged ? kEpiBytes : 0);
+  volatile uint32_t* ctrl = reinterpret_cast<volatile uint32_t*>(smem_gen + kStages * kStageBytes + (kStaged ? kEpiBytes : 0));
+  // control block: 8-byte barriers full[kStages], empty[kStages], tmem_full[2], tmem_empty[2]; then the TMEM base
+  // address and the abort flag (4 bytes each, within the first 160 bytes for at most 7 stages); at byte 192 the
+  // 16 "box arrived" barriers of the epilogue warps (4 per warp).  Same offsets in both CTAs of the pair.
+  auto in_bar = [&](int w, uint32_t buf) { return bar_base + 192u + 8u * (4u * w + buf); };
   auto full_bar = [&](int i) { return bar_base + 8u * i; };
   auto empty_bar = [&](int i) { return bar_base + 8u * (kStages + i); };
   auto tfull_bar = [&](int i) { return bar_base + 8u * (2 * kStages + i); };
@@ -204,6 +306,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   volatile int* abort_flag = reinterpret_cast<volatile int*>(ctrl + 2 * (2 * kStages + 4) + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_rank();               // 0: leader of the pair (issues the MMAs)
+  const int pair = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
   const int total_tiles = p.groups * p.m_tiles * p.n_tiles;
   const int num_kb = (p.K + kBK - 1) / kBK;
 
@@ -211,37 +315,43 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     tma_prefetch_desc(&tmA);
     tma_prefetch_desc(&tmB);
     for (int i = 0; i < kStages; ++i) { mbar_init(full_bar(i), 1); mbar_init(empty_bar(i), 1); }
-    for (int i = 0; i < 2; ++i) { mbar_init(tfull_bar(i), 1); mbar_init(tempty_bar(i), 4); }
+    for (int i = 0; i < 2; ++i) { mbar_init(tfull_bar(i), 1); mbar_init(tempty_bar(i), 8); }   // 4 epilogue warps x 2 CTAs
+    if (kStaged)
+      for (int w = 0; w < 4; ++w)
+        for (int b = 0; b < 4; ++b) mbar_init(in_bar(w, b), 1);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
-  if (warp == 5) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+  if (warp == 5) {   // the same warp of both CTAs allocates the pair's tensor memory together
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;"
                  ::"r"(smem_u32(const_cast<uint32_t*>(tmem_slot))), "r"((uint32_t)kTmemCols) : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
   }
   tc_fence_before();
   __syncthreads();
+  cluster_sync_all();          // the peer's barriers exist before anything is signalled across the pair
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
   if (warp == 4) {
-    // ------------------------------------------------------------------ TMA producer
+    // ------------------------------------------------------------------ TMA producer (both CTAs)
     if (lane == 0) {
       uint32_t it = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
+      for (int tile = pair; ok && tile < total_tiles; tile += num_pairs) {
         int g, mt, nt;
         tile_coords(p, tile, g, mt, nt);
-        const int m0 = mt * kBM;
-        const int n0 = nt * (EPI == EPI_SWIGLU_FWD ? kBN / 2 : kBN);
+        const int m0 = mt * kBM + (int)rank * kCtaM;
+        // B rows (K-major) / columns (MN-major) of this CTA.  SwiGLU forward: the leader loads 128 gate
+        // rows, the peer the matching 128 up rows, so accumulator columns 0..127 are G and 128..255 are U.
+        const int n0 = (EPI == EPI_SWIGLU_FWD) ? (rank ? p.b_split : 0) + nt * kCtaN : nt * kBN + (int)rank * kCtaN;
         for (int kb = 0; kb < num_kb; ++kb, ++it) {
           const int stage = it % kStages;
           const uint32_t phase = (it / kStages) & 1u;
           if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status)) { ok = false; break; }
-          const uint32_t bar = full_bar(stage);
-          mbar_expect_tx(bar, kStageBytes);
+          if (rank == 0) mbar_expect_tx(full_bar(stage), 2 * kStageBytes);   // both CTAs' bytes
+          const uint32_t bar = map_to_cta(full_bar(stage), 0);
           const uint32_t a_dst = smem_base + stage * kStageBytes;
           const uint32_t b_dst = a_dst + kABytes;
           const int k0 = kb * kBK;
@@ -249,23 +359,20 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             tma_load_3d(a_dst, &tmA, bar, k0, m0, g);                       // box 64 (K) x 128 rows
           } else {
 #pragma unroll
-            for (int j = 0; j < kBM / 64; ++j) tma_load_3d(a_dst + j * 8192, &tmA, bar, m0 + 64 * j, k0, g);   // 64 (M) x 64 (K)
+            for (int j = 0; j < kCtaM / 64; ++j) tma_load_3d(a_dst + j * 8192, &tmA, bar, m0 + 64 * j, k0, g);   // 64 (M) x 64 (K)
           }
           if (B_MAJOR == MAJOR_K) {
-            const int r0 = n0;
-            const int r1 = (EPI == EPI_SWIGLU_FWD) ? p.b_split + n0 : n0 + 128;
-            tma_load_3d(b_dst, &tmB, bar, k0, r0, g);                       // box 64 (K) x 128 rows
-            tma_load_3d(b_dst + 16384, &tmB, bar, k0, r1, g);
+            tma_load_3d(b_dst, &tmB, bar, k0, n0, g);                       // box 64 (K) x 128 rows
           } else {
 #pragma unroll
-            for (int j = 0; j < kBN / 64; ++j) tma_load_3d(b_dst + j * 8192, &tmB, bar, n0 + 64 * j, k0, g);   // 64 (N) x 64 (K)
+            for (int j = 0; j < kCtaN / 64; ++j) tma_load_3d(b_dst + j * 8192, &tmB, bar, n0 + 64 * j, k0, g);   // 64 (N) x 64 (K)
           }
         }
       }
     }
   } else if (warp == 5) {
-    // ------------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
+    // ------------------------------------------------------------------ MMA issuer (leader CTA only)
+    if (lane == 0 && rank == 0) {
       constexpr uint32_t idesc = instr_desc(A_MAJOR, B_MAJOR);
       constexpr uint32_t a_lbo = A_MAJOR == MAJOR_K ? 16u : (uint32_t)kBK * 128u;
       constexpr uint32_t b_lbo = B_MAJOR == MAJOR_K ? 16u : (uint32_t)kBK * 128u;
@@ -273,7 +380,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       constexpr uint32_t b_kstep = B_MAJOR == MAJOR_K ? (kUmmaK * 2) : (kUmmaK * 128);
       uint32_t it = 0, tl = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x, ++tl) {
+      for (int tile = pair; ok && tile < total_tiles; tile += num_pairs, ++tl) {
         const uint32_t slot = tl & 1u, acc_phase = (tl >> 1) & 1u;
         if (!mbar_wait(tempty_bar(slot), acc_phase ^ 1u, abort_flag, p.status)) { ok = false; break; }
         tc_fence_after();
@@ -292,184 +399,277 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             tc_mma_bf16(d_tmem, a_desc + (uint64_t)((k * a_kstep) >> 4), b_desc + (uint64_t)((k * b_kstep) >> 4), idesc,
                         (kb | k) != 0 ? 1u : 0u);
           }
-          tc_commit(empty_bar(stage));          // frees the stage when these MMAs have read it
+          tc_commit_pair(empty_bar(stage));      // frees the stage in both CTAs when these MMAs have read it
         }
-        if (ok) tc_commit(tfull_bar(slot));     // accumulator complete
+        if (ok) tc_commit_pair(tfull_bar(slot)); // accumulator complete, in both CTAs
       }
     }
   } else {
     // ------------------------------------------------------------------ epilogue warps 0..3
+    // Thread (warp w, lane l) owns accumulator row 32 w + l of this CTA and walks it in chunks of 32 columns;
+    // the tensor-memory load of chunk c + 1 is in flight while chunk c is processed.
+    constexpr int kChunks = (EPI == EPI_SWIGLU_FWD) ? kCtaN / 32 : kBN / 32;
+    constexpr int kTileN = (EPI == EPI_SWIGLU_FWD) ? kCtaN : kBN;     // output columns (neurons) per tile
+    const uint32_t tempty_leader[2] = {map_to_cta(tempty_bar(0), 0), map_to_cta(tempty_bar(1), 0)};
     uint32_t tl = 0;
     bool ok = true;
-    for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x, ++tl) {
-      int g, mt, nt;
-      tile_coords(p, tile, g, mt, nt);
-      const uint32_t slot = tl & 1u, acc_phase = (tl >> 1) & 1u;
-      if (!mbar_wait(tfull_bar(slot), acc_phase, abort_flag, p.status)) { ok = false; break; }
-      tc_fence_after();
-      const int row = mt * kBM + warp * 32 + lane;
-      const bool row_ok = row < p.M;
-      const uint32_t t_row = tmem_base + slot * kBN + ((uint32_t)(warp * 32) << 16);
-      const long long grow = (long long)g * p.M + row;      // row index over all groups
 
-      if (EPI == EPI_STORE) {
-        const int n0 = nt * kBN;
-        __nv_bfloat16* out = p.out0 + grow * p.N;
-        for (int c = 0; c < kBN / 32; ++c) {
-          const int n = n0 + 32 * c;
-          if (n >= p.N) break;
-          uint32_t r[32];
-          tc_ld32(t_row + 32 * c, r);
-          tc_wait_ld();
-          if (row_ok) {
-            uint32_t w[16];
+    if constexpr (EPI == EPI_SGD) {
+      // Weight-gradient tiles (contraction over all tokens, so this epilogue is rare): plain vector accesses
+      // to the fp32 master rows; the master values of the next chunk are loaded ahead.
+      for (int tile = pair; ok && tile < total_tiles; tile += num_pairs, ++tl) {
+        int g, mt, nt;
+        tile_coords(p, tile, g, mt, nt);
+        const uint32_t slot = tl & 1u, acc_phase = (tl >> 1) & 1u;
+        const int row = mt * kBM + (int)rank * kCtaM + warp * 32 + lane;
+        const bool row_ok = row < p.M;
+        const uint32_t t_row = tmem_base + slot * kBN + ((uint32_t)(warp * 32) << 16);
+        const long long grow = (long long)g * p.M + row;      // row index over all groups
+        const int n_base = nt * kBN;
+        float4 mv[2][8];
+        EpiAcc<EPI> acc[2];
+        auto load_master = [&](int c, float4 (&m)[8]) {
+          const int n = n_base + 32 * c;
+          const int valid = (row_ok && n < p.N && p.lr != 0.f) ? min(32, p.N - n) : 0;
+          const float4* src = reinterpret_cast<const float4*>(p.master + grow * p.N + n);
 #pragma unroll
-            for (int q = 0; q < 16; ++q)
-              w[q] = pack2(p.scale * __uint_as_float(r[2 * q]), p.scale * __uint_as_float(r[2 * q + 1]));
-            store_row32(out + n, w, min(32, p.N - n));
+          for (int q = 0; q < 8; ++q) m[q] = (4 * q < valid) ? src[q] : make_float4(0.f, 0.f, 0.f, 0.f);
+        };
+        load_master(0, mv[0]);
+        if (!mbar_wait(tfull_bar(slot), acc_phase, abort_flag, p.status)) { ok = false; break; }
+        tc_fence_after();
+        tc_ld32(t_row, acc[0].r0);
+#pragma unroll
+        for (int c = 0; c < kChunks; ++c) {
+          tc_wait_ld();
+          if (c + 1 < kChunks) {
+            tc_ld32(t_row + 32 * (c + 1), acc[(c + 1) & 1].r0);
+            load_master(c + 1, mv[(c + 1) & 1]);
           }
-        }
-      } else if (EPI == EPI_SWIGLU_FWD) {
-        const int j0 = nt * (kBN / 2);
-        const int f = p.N;
-        __nv_bfloat16* pre = p.out0 + grow * (2LL * f);
-        __nv_bfloat16* hh = p.out1 + grow * f;
-        for (int c = 0; c < kBN / 64; ++c) {
-          const int j = j0 + 32 * c;
-          if (j >= f) break;
-          uint32_t rg[32], ru[32];
-          tc_ld32(t_row + 32 * c, rg);
-          tc_ld32(t_row + kBN / 2 + 32 * c, ru);
-          tc_wait_ld();
-          if (row_ok) {
-            uint32_t wg[16], wu[16], wh[16];
-#pragma unroll
-            for (int q = 0; q < 16; ++q) {
-              const float g0 = __uint_as_float(rg[2 * q]), g1 = __uint_as_float(rg[2 * q + 1]);
-              const float u0 = __uint_as_float(ru[2 * q]), u1 = __uint_as_float(ru[2 * q + 1]);
-              wg[q] = pack2(g0, g1);
-              wu[q] = pack2(u0, u1);
-              wh[q] = pack2(g0 / (1.f + __expf(-g0)) * u0, g1 / (1.f + __expf(-g1)) * u1);
-            }
-            const int valid = min(32, f - j);
-            store_row32(pre + j, wg, valid);
-            store_row32(pre + f + j, wu, valid);
-            store_row32(hh + j, wh, valid);
-          }
-        }
-      } else if (EPI == EPI_ACT_FWD) {
-        const int n0 = nt * kBN;
-        __nv_bfloat16* pre = p.out0 + grow * p.N;
-        __nv_bfloat16* hh = p.out1 + grow * p.N;
-        for (int c = 0; c < kBN / 32; ++c) {
-          const int n = n0 + 32 * c;
-          if (n >= p.N) break;
-          uint32_t r[32];
-          tc_ld32(t_row + 32 * c, r);
-          tc_wait_ld();
-          if (row_ok) {
-            uint32_t wp[16], wh[16];
-#pragma unroll
-            for (int q = 0; q < 16; ++q) {
-              const float a0 = __uint_as_float(r[2 * q]), a1 = __uint_as_float(r[2 * q + 1]);
-              wp[q] = pack2(a0, a1);
-              wh[q] = pack2(act_fwd(a0, p.act_kind), act_fwd(a1, p.act_kind));
-            }
+          const int n = n_base + 32 * c;
+          if (row_ok && n < p.N) {
             const int valid = min(32, p.N - n);
-            store_row32(pre + n, wp, valid);
-            store_row32(hh + n, wh, valid);
-          }
-        }
-      } else if (EPI == EPI_DSWIGLU) {
-        const int n0 = nt * kBN;
-        const int f = p.N;
-        const __nv_bfloat16* pre = p.in0 + grow * (2LL * f);
-        __nv_bfloat16* dpre = p.out0 + grow * (2LL * f);
-        for (int c = 0; c < kBN / 32; ++c) {
-          const int j = n0 + 32 * c;
-          if (j >= f) break;
-          uint32_t r[32];
-          tc_ld32(t_row + 32 * c, r);
-          tc_wait_ld();
-          if (row_ok) {
-            const int valid = min(32, f - j);
-            uint32_t pg[16], pu[16], wg[16], wu[16];
-            load_row32(pre + j, pg, valid);
-            load_row32(pre + f + j, pu, valid);
-#pragma unroll
-            for (int q = 0; q < 16; ++q) {
-              float dg[2], du[2];
-#pragma unroll
-              for (int h = 0; h < 2; ++h) {
-                const float dh = p.scale * __uint_as_float(r[2 * q + h]);
-                const float gt = h ? bf_hi(pg[q]) : bf_lo(pg[q]);
-                const float up = h ? bf_hi(pu[q]) : bf_lo(pu[q]);
-                const float sg = 1.f / (1.f + __expf(-gt));
-                dg[h] = dh * up * (sg * (1.f + gt * (1.f - sg)));
-                du[h] = dh * (gt * sg);
-              }
-              wg[q] = pack2(dg[0], dg[1]);
-              wu[q] = pack2(du[0], du[1]);
-            }
-            store_row32(dpre + j, wg, valid);
-            store_row32(dpre + f + j, wu, valid);
-          }
-        }
-      } else if (EPI == EPI_DACT) {
-        const int n0 = nt * kBN;
-        const __nv_bfloat16* pre = p.in0 + grow * p.N;
-        __nv_bfloat16* dpre = p.out0 + grow * p.N;
-        for (int c = 0; c < kBN / 32; ++c) {
-          const int n = n0 + 32 * c;
-          if (n >= p.N) break;
-          uint32_t r[32];
-          tc_ld32(t_row + 32 * c, r);
-          tc_wait_ld();
-          if (row_ok) {
-            const int valid = min(32, p.N - n);
-            uint32_t pp[16], w[16];
-            load_row32(pre + n, pp, valid);
-#pragma unroll
-            for (int q = 0; q < 16; ++q)
-              w[q] = pack2(p.scale * __uint_as_float(r[2 * q]) * act_grad(bf_lo(pp[q]), p.act_kind),
-                           p.scale * __uint_as_float(r[2 * q + 1]) * act_grad(bf_hi(pp[q]), p.act_kind));
-            store_row32(dpre + n, w, valid);
-          }
-        }
-      } else {   // EPI_SGD: acc = dW tile; master -= lr * scale * acc; compute copy = bf16(master)
-        const int n0 = nt * kBN;
-        float* master = p.master + grow * p.N;
-        float* dw = p.dw ? p.dw + grow * p.N : nullptr;
-        __nv_bfloat16* w16 = p.out0 + grow * p.N;
-        for (int c = 0; c < kBN / 32; ++c) {
-          const int n = n0 + 32 * c;
-          if (n >= p.N) break;
-          uint32_t r[32];
-          tc_ld32(t_row + 32 * c, r);
-          tc_wait_ld();
-          if (row_ok) {
-            const int valid = min(32, p.N - n);
+            const uint32_t* r = acc[c & 1].r0;
+            float* master = p.master + grow * p.N + n;
+            float* dw = p.dw ? p.dw + grow * p.N + n : nullptr;
+            __nv_bfloat16* w16 = p.out0 + grow * p.N + n;
 #pragma unroll
             for (int q = 0; q < 8; ++q) {
               if (4 * q < valid) {
-                float4 gq = make_float4(p.scale * __uint_as_float(r[4 * q]), p.scale * __uint_as_float(r[4 * q + 1]),
-                                        p.scale * __uint_as_float(r[4 * q + 2]), p.scale * __uint_as_float(r[4 * q + 3]));
-                if (dw) *reinterpret_cast<float4*>(dw + n + 4 * q) = gq;
-                if (p.lr != 0.f) {
-                  float4 m = *reinterpret_cast<const float4*>(master + n + 4 * q);
+                const float4 gq = make_float4(p.scale * __uint_as_float(r[4 * q]), p.scale * __uint_as_float(r[4 * q + 1]),
+                                              p.scale * __uint_as_float(r[4 * q + 2]), p.scale * __uint_as_float(r[4 * q + 3]));
+                if (dw) *reinterpret_cast<float4*>(dw + 4 * q) = gq;
+                if (p.lr != 0.f) {      // master -= lr * dW (fp32); compute copy = bf16(master)
+                  float4 m = mv[c & 1][q];
                   m.x -= p.lr * gq.x; m.y -= p.lr * gq.y; m.z -= p.lr * gq.z; m.w -= p.lr * gq.w;
-                  *reinterpret_cast<float4*>(master + n + 4 * q) = m;
-                  *reinterpret_cast<uint2*>(w16 + n + 4 * q) = make_uint2(pack2(m.x, m.y), pack2(m.z, m.w));
+                  *reinterpret_cast<float4*>(master + 4 * q) = m;
+                  *reinterpret_cast<uint2*>(w16 + 4 * q) = make_uint2(pack2(m.x, m.y), pack2(m.z, m.w));
                 }
               }
             }
           }
         }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive_cluster(tempty_leader[slot]);      // accumulator slot free again
       }
-      // accumulator slot free again
-      tc_fence_before();
+    } else {
+      // Staged epilogues.  Chunk number gc (counted over all tiles of this CTA) uses buffer gc % kBufs of the
+      // warp: kSlots boxes of 2 KB.  Boxes the chunk reads are requested kBufs - 1 chunks ahead, results are
+      // written over them in place (each thread touches only its own row) and leave as bulk stores; a buffer
+      // is refilled or rewritten only after the bulk store that last read it has finished reading.
+      constexpr int kSlots = epi_slots(EPI), kIn = epi_in_slots(EPI), kBufs = epi_bufs(EPI);
+      const uint32_t wbase = epi_base + (uint32_t)warp * kEpiWarpBytes;
+      auto box = [&](uint32_t gc, int slot) { return wbase + ((gc & (kBufs - 1)) * kSlots + slot) * kEpiBoxBytes; };
+      // 16-byte piece q (0..3) of this thread's row inside a box (64-byte rows, 64-byte swizzle)
+      const uint32_t row_off = (uint32_t)lane * 64u;
+      const uint32_t sw = ((uint32_t)lane >> 1) & 3u;
+      auto piece = [&](uint32_t box_addr, int q) { return box_addr + row_off + ((((uint32_t)q) ^ sw) << 4); };
+      // (group, first row of this warp, first column) of chunk gc; false past the CTA's last tile
+      auto chunk_coords = [&](uint32_t gc, int& g, int& row0, int& n) {
+        const int tile = pair + (int)(gc / kChunks) * num_pairs;
+        if (tile >= total_tiles) return false;
+        int mt, nt;
+        tile_coords(p, tile, g, mt, nt);
+        row0 = mt * kBM + (int)rank * kCtaM + warp * 32;
+        n = nt * kTileN + 32 * (int)(gc % kChunks);
+        return true;
+      };
+      auto request_inputs = [&](uint32_t gc) {      // lane 0 only
+        int g, row0, n;
+        if (kIn == 0 || !chunk_coords(gc, g, row0, n)) return;
+        const uint32_t bar = in_bar(warp, gc & (kBufs - 1));
+        mbar_expect_tx(bar, kIn * kEpiBoxBytes);
+#pragma unroll
+        for (int i = 0; i < kIn; ++i) tma_load_3d_local(box(gc, i), &tmE.m[i], bar, n, row0, g);
+      };
+      if (lane == 0) {
+        for (uint32_t gc = 0; gc + 1 < (uint32_t)kBufs; ++gc) request_inputs(gc);
+      }
+
+      for (int tile = pair; ok && tile < total_tiles; tile += num_pairs, ++tl) {
+        int g, mt, nt;
+        tile_coords(p, tile, g, mt, nt);
+        const uint32_t slot = tl & 1u, acc_phase = (tl >> 1) & 1u;
+        const int row0 = mt * kBM + (int)rank * kCtaM + warp * 32;
+        const bool row_ok = row0 + lane < p.M;
+        const uint32_t t_row = tmem_base + slot * kBN + ((uint32_t)(warp * 32) << 16);
+        const int n_base = nt * kTileN;
+        EpiAcc<EPI> acc[2];
+        float loss_acc = 0.f, kfac = 0.f;
+        int vc = 0;
+        if constexpr (EPI == EPI_MSE) {
+          vc = p.valid_cols ? p.valid_cols[g] : p.seg_width;
+          const int n_valid = p.seg_begin + ((p.N - p.seg_begin) / p.seg_width) * vc;
+          kfac = 2.0f / ((float)p.M * (float)n_valid);
+        }
+        auto load_acc = [&](int c, EpiAcc<EPI>& a) {
+          tc_ld32(t_row + 32 * c, a.r0);
+          if constexpr (EPI == EPI_SWIGLU_FWD) tc_ld32(t_row + kCtaN + 32 * c, a.r1);
+        };
+        if (!mbar_wait(tfull_bar(slot), acc_phase, abort_flag, p.status)) { ok = false; break; }
+        tc_fence_after();
+        load_acc(0, acc[0]);
+#pragma unroll
+        for (int c = 0; c < kChunks; ++c) {
+          const uint32_t gc = tl * kChunks + c;
+          const int n = n_base + 32 * c;
+          if (kIn > 0) {      // this chunk's boxes have arrived
+            if (!mbar_wait(in_bar(warp, gc & (kBufs - 1)), (gc / kBufs) & 1u, abort_flag, p.status)) { ok = false; break; }
+          } else {            // the bulk store that last read this buffer is done with it
+            if (lane == 0) bulk_wait_read<kBufs - 1>();
+            __syncwarp();
+          }
+          tc_wait_ld();
+          if (c + 1 < kChunks) load_acc(c + 1, acc[(c + 1) & 1]);
+          const EpiAcc<EPI>& a = acc[c & 1];
+          const uint32_t b0 = box(gc, 0), b1 = box(gc, kSlots > 1 ? 1 : 0), b2 = box(gc, kSlots > 2 ? 2 : 0);
+
+          // ---- compute this thread's 32 columns; results go to the boxes, 8 columns (16 bytes) at a time
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            const uint32_t* r = a.r0 + 8 * q;
+            if constexpr (EPI == EPI_STORE) {
+              sts128(piece(b0, q), make_uint4(pack2(p.scale * __uint_as_float(r[0]), p.scale * __uint_as_float(r[1])),
+                                              pack2(p.scale * __uint_as_float(r[2]), p.scale * __uint_as_float(r[3])),
+                                              pack2(p.scale * __uint_as_float(r[4]), p.scale * __uint_as_float(r[5])),
+                                              pack2(p.scale * __uint_as_float(r[6]), p.scale * __uint_as_float(r[7]))));
+            } else if constexpr (EPI == EPI_MSE) {
+              const uint4 tv = lds128(piece(b0, q));
+              const uint32_t tw[4] = {tv.x, tv.y, tv.z, tv.w};
+              // validity is constant over aligned groups of 8 columns (seg_begin, seg_width, vc are multiples of 8)
+              const int col = n + 8 * q;
+              const bool cv = row_ok && col < p.N && (col < p.seg_begin || (col - p.seg_begin) % p.seg_width < vc);
+              uint32_t wy[4], wd[4];
+#pragma unroll
+              for (int h = 0; h < 4; ++h) {
+                wy[h] = pack2(p.scale * __uint_as_float(r[2 * h]), p.scale * __uint_as_float(r[2 * h + 1]));
+                const float d0 = cv ? bf_lo(wy[h]) - bf_lo(tw[h]) : 0.f;
+                const float d1 = cv ? bf_hi(wy[h]) - bf_hi(tw[h]) : 0.f;
+                loss_acc += d0 * d0 + d1 * d1;
+                wd[h] = pack2(kfac * d0, kfac * d1);
+              }
+              sts128(piece(b0, q), make_uint4(wd[0], wd[1], wd[2], wd[3]));
+              if (p.out0) sts128(piece(b1, q), make_uint4(wy[0], wy[1], wy[2], wy[3]));
+            } else if constexpr (EPI == EPI_SWIGLU_FWD) {
+              const uint32_t* ru = a.r1 + 8 * q;
+              uint32_t wg[4], wu[4], wh[4];
+#pragma unroll
+              for (int h = 0; h < 4; ++h) {
+                const float g0 = __uint_as_float(r[2 * h]), g1 = __uint_as_float(r[2 * h + 1]);
+                const float u0 = __uint_as_float(ru[2 * h]), u1 = __uint_as_float(ru[2 * h + 1]);
+                wg[h] = pack2(g0, g1);
+                wu[h] = pack2(u0, u1);
+                wh[h] = pack2(g0 * sigmoid_fast(g0) * u0, g1 * sigmoid_fast(g1) * u1);
+              }
+              sts128(piece(b0, q), make_uint4(wg[0], wg[1], wg[2], wg[3]));
+              sts128(piece(b1, q), make_uint4(wu[0], wu[1], wu[2], wu[3]));
+              sts128(piece(b2, q), make_uint4(wh[0], wh[1], wh[2], wh[3]));
+            } else if constexpr (EPI == EPI_ACT_FWD) {
+              uint32_t wp[4], wh[4];
+#pragma unroll
+              for (int h = 0; h < 4; ++h) {
+                const float a0 = __uint_as_float(r[2 * h]), a1 = __uint_as_float(r[2 * h + 1]);
+                wp[h] = pack2(a0, a1);
+                wh[h] = pack2(act_fwd(a0, p.act_kind), act_fwd(a1, p.act_kind));
+              }
+              sts128(piece(b0, q), make_uint4(wp[0], wp[1], wp[2], wp[3]));
+              sts128(piece(b1, q), make_uint4(wh[0], wh[1], wh[2], wh[3]));
+            } else if constexpr (EPI == EPI_DSWIGLU) {
+              const uint4 gv = lds128(piece(b0, q)), uv = lds128(piece(b1, q));
+              const uint32_t pg[4] = {gv.x, gv.y, gv.z, gv.w}, pu[4] = {uv.x, uv.y, uv.z, uv.w};
+              uint32_t wg[4], wu[4];
+#pragma unroll
+              for (int h = 0; h < 4; ++h) {
+                float dg[2], du[2];
+#pragma unroll
+                for (int e = 0; e < 2; ++e) {
+                  const float dh = p.scale * __uint_as_float(r[2 * h + e]);
+                  const float gt = e ? bf_hi(pg[h]) : bf_lo(pg[h]);
+                  const float up = e ? bf_hi(pu[h]) : bf_lo(pu[h]);
+                  const float sg = sigmoid_fast(gt);
+                  dg[e] = dh * up * (sg * (1.f + gt * (1.f - sg)));
+                  du[e] = dh * (gt * sg);
+                }
+                wg[h] = pack2(dg[0], dg[1]);
+                wu[h] = pack2(du[0], du[1]);
+              }
+              sts128(piece(b0, q), make_uint4(wg[0], wg[1], wg[2], wg[3]));
+              sts128(piece(b1, q), make_uint4(wu[0], wu[1], wu[2], wu[3]));
+            } else {   // EPI_DACT
+              const uint4 pv = lds128(piece(b0, q));
+              const uint32_t pp[4] = {pv.x, pv.y, pv.z, pv.w};
+              uint32_t w[4];
+#pragma unroll
+              for (int h = 0; h < 4; ++h)
+                w[h] = pack2(p.scale * __uint_as_float(r[2 * h]) * act_grad(bf_lo(pp[h]), p.act_kind),
+                             p.scale * __uint_as_float(r[2 * h + 1]) * act_grad(bf_hi(pp[h]), p.act_kind));
+              sts128(piece(b0, q), make_uint4(w[0], w[1], w[2], w[3]));
+            }
+          }
+
+          // ---- the boxes leave by bulk store (rows / columns outside the tensor are clipped)
+          fence_async_smem();
+          __syncwarp();
+          if (lane == 0) {
+            const int rr = row0, gg = g;
+            if constexpr (EPI == EPI_STORE) {
+              tma_store_3d(&tmE.m[0], b0, n, rr, gg);
+            } else if constexpr (EPI == EPI_MSE) {
+              tma_store_3d(&tmE.m[1], b0, n, rr, gg);
+              if (p.out0) tma_store_3d(&tmE.m[2], b1, n, rr, gg);
+            } else if constexpr (EPI == EPI_SWIGLU_FWD) {
+              tma_store_3d(&tmE.m[0], b0, n, rr, gg);
+              tma_store_3d(&tmE.m[1], b1, n, rr, gg);
+              tma_store_3d(&tmE.m[2], b2, n, rr, gg);
+            } else if constexpr (EPI == EPI_ACT_FWD) {
+              tma_store_3d(&tmE.m[0], b0, n, rr, gg);
+              tma_store_3d(&tmE.m[1], b1, n, rr, gg);
+            } else if constexpr (EPI == EPI_DSWIGLU) {
+              tma_store_3d(&tmE.m[2], b0, n, rr, gg);
+              tma_store_3d(&tmE.m[3], b1, n, rr, gg);
+            } else {
+              tma_store_3d(&tmE.m[1], b0, n, rr, gg);
+            }
+            bulk_commit();
+            if (kIn > 0) {     // the previous chunk's store has finished reading its buffer: refill it
+              bulk_wait_read<1>();
+              request_inputs(gc + kBufs - 1);
+            }
+          }
+        }
+        if (!ok) break;
+        // accumulator slot free again
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive_cluster(tempty_leader[slot]);
+        if constexpr (EPI == EPI_MSE) {   // per-warp partial sum of squared errors, fixed order
+          for (int o = 16; o > 0; o >>= 1) loss_acc += __shfl_xor_sync(0xffffffffu, loss_acc, o);
+          if (lane == 0) p.dw[((long long)tile * 2 + rank) * 4 + warp] = loss_acc;
+        }
+      }
+      if (lane == 0) bulk_wait_read<0>();      // shared memory stays valid until the last store has read it
       __syncwarp();
-      if (lane == 0) mbar_arrive(tempty_bar(slot));
     }
   }
 
@@ -482,9 +682,12 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     while (global_timer_ns() - t0 < 2000000ull) __nanosleep(1000);
     __syncthreads();
   }
+  // Neither CTA leaves (nor frees tensor memory) while the other may still signal its barriers, read
+  // its shared memory or write its accumulators.
+  cluster_sync_all();
   if (warp == 5) {
     tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)kTmemCols) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)kTmemCols) : "memory");
   }
 }
 
@@ -497,5 +700,11 @@ struct GemmOperand {
 
 // layout: 0 NT, 1 NN, 2 TN.  Returns a TWIST_* status.
 int launch_gemm_bf16(int layout, int epi, const GemmOperand& A, const GemmOperand& B, GemmParams p, cudaStream_t st);
+
+// EPI_MSE: number of fp32 partial sums the kernel writes (GemmParams::dw) for `groups` problems of M x N,
+// and the fixed-order reduction of those partials into loss[groups].
+size_t fused_loss_partials(int groups, int M, int N);
+int finish_fused_loss(const float* partial, int groups, int M, int N, const int32_t* valid_cols, int seg_begin,
+                      int seg_width, float* loss, cudaStream_t st);
 
 }  // namespace twist

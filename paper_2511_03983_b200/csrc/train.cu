@@ -23,6 +23,34 @@ int check_ffn(const twist_ffn_args* a) {
   return TWIST_OK;
 }
 
+// Checks the fused-loss arguments of a forward call; *fused tells whether the loss is requested.
+int check_fused(const void* tgt, float* loss, const void* dgrad, void* ws, size_t ws_bytes, int S, int T, int width,
+                const int32_t* valid_cols, int seg_begin, int seg_width, bool* fused) {
+  *fused = tgt != nullptr;
+  if (!*fused) return TWIST_OK;
+  if (!loss || !dgrad) return TWIST_ERR_NULL;
+  if (!ws || ws_bytes < twist_fused_loss_workspace_bytes(S, T, width)) return TWIST_ERR_WORKSPACE;
+  if (valid_cols && (seg_begin < 0 || seg_begin >= width || seg_width <= 0 || (width - seg_begin) % seg_width != 0 ||
+                     seg_begin % 8 != 0 || seg_width % 8 != 0))
+    return TWIST_ERR_SHAPE;
+  return TWIST_OK;
+}
+
+// Output GEMM of a forward call with the loss fused into its epilogue (bf16).
+int launch_fused_loss(int layout, const GemmOperand& A, const GemmOperand& B, GemmParams p, void* out, const void* tgt,
+                      void* dgrad, float* loss, void* ws, const int32_t* valid_cols, int seg_begin, int seg_width,
+                      cudaStream_t st) {
+  p.out0 = static_cast<__nv_bfloat16*>(out);
+  p.out1 = static_cast<__nv_bfloat16*>(dgrad);
+  p.in0 = static_cast<const __nv_bfloat16*>(tgt);
+  p.dw = static_cast<float*>(ws);
+  p.valid_cols = valid_cols;
+  p.seg_begin = valid_cols ? seg_begin : 0;
+  p.seg_width = valid_cols ? seg_width : p.N;
+  TWIST_TRY(launch_gemm_bf16(layout, EPI_MSE, A, B, p, st));
+  return finish_fused_loss(p.dw, p.groups, p.M, p.N, valid_cols, p.seg_begin, p.seg_width, loss, st);
+}
+
 GemmParams base_params(int M, int N, int K, int groups, float scale) {
   GemmParams p;
   memset(&p, 0, sizeof(p));
@@ -35,9 +63,20 @@ GemmParams base_params(int M, int N, int K, int groups, float scale) {
 
 using namespace twist;
 
+extern "C" size_t twist_fused_loss_workspace_bytes(int32_t n_subnets, int32_t tokens, int32_t width) {
+  if (n_subnets <= 0 || tokens <= 0 || width <= 0) return 0;
+  const size_t a = fused_loss_partials(n_subnets, tokens, width) * sizeof(float);
+  const size_t b = twist_mse_workspace_bytes(n_subnets);      // the fp32 dtype runs the stand-alone loss kernels
+  return a > b ? a : b;
+}
+
 extern "C" int32_t twist_subnet_ffn_fwd(const twist_ffn_args* a, void* stream) {
   TWIST_TRY(check_ffn(a));
-  if (!a->x || !a->w_gu || !a->w_down || !a->pre || !a->hh || !a->y) return TWIST_ERR_NULL;
+  bool fused = false;
+  TWIST_TRY(check_fused(a->tgt, a->loss, a->dy, a->loss_ws, a->loss_ws_bytes, a->n_subnets, a->tokens, a->d_model,
+                        nullptr, 0, 0, &fused));
+  if (!a->x || !a->w_gu || !a->w_down || !a->pre || !a->hh || (!a->y && !fused)) return TWIST_ERR_NULL;
+  if (a->dtype == TWIST_FP32 && !a->y) return TWIST_ERR_NULL;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const int S = a->n_subnets, T = a->tokens, d = a->d_model, f = a->f_sub;
   const bool swiglu = a->ffn_kind == TWIST_FFN_SWIGLU;
@@ -49,8 +88,11 @@ extern "C" int32_t twist_subnet_ffn_fwd(const twist_ffn_args* a, void* stream) {
     TWIST_TRY(sgemm_f32(false, true, x, static_cast<const float*>(a->w_gu), pre, T, gf, d, d, d, gf, (long long)T * d,
                         (long long)gf * d, (long long)T * gf, S, 1.f, st));
     TWIST_TRY(act_fwd_f32(pre, hh, (long long)S * T, f, a->ffn_kind, st));
-    return sgemm_f32(false, false, hh, static_cast<const float*>(a->w_down), static_cast<float*>(a->y), T, d, f, f, d,
-                     d, (long long)T * f, (long long)f * d, (long long)T * d, S, a->out_scale, st);
+    TWIST_TRY(sgemm_f32(false, false, hh, static_cast<const float*>(a->w_down), static_cast<float*>(a->y), T, d, f, f, d,
+                        d, (long long)T * f, (long long)f * d, (long long)T * d, S, a->out_scale, st));
+    if (!fused) return TWIST_OK;
+    return twist_mse_fwd_bwd(a->y, a->tgt, const_cast<void*>(a->dy), a->loss, S, T, d, nullptr, 0, 0, TWIST_FP32,
+                             a->loss_ws, a->loss_ws_bytes, stream);
   }
   // pre (and hh) = epilogue(X W_gu^T)
   GemmParams p = base_params(T, f, d, S, 1.f);
@@ -60,8 +102,11 @@ extern "C" int32_t twist_subnet_ffn_fwd(const twist_ffn_args* a, void* stream) {
   p.act_kind = a->ffn_kind;
   TWIST_TRY(launch_gemm_bf16(0, swiglu ? EPI_SWIGLU_FWD : EPI_ACT_FWD, GemmOperand{a->x, T, d},
                              GemmOperand{a->w_gu, gf, d}, p, st));
-  // Y = out_scale * hh W_down
+  // Y = out_scale * hh W_down  (+ loss and dY in the same epilogue when requested)
   GemmParams q = base_params(T, d, f, S, a->out_scale);
+  if (fused)
+    return launch_fused_loss(1, GemmOperand{a->hh, T, f}, GemmOperand{a->w_down, f, d}, q, a->y, a->tgt,
+                             const_cast<void*>(a->dy), a->loss, a->loss_ws, nullptr, 0, 0, st);
   q.out0 = static_cast<__nv_bfloat16*>(a->y);
   return launch_gemm_bf16(1, EPI_STORE, GemmOperand{a->hh, T, f}, GemmOperand{a->w_down, f, d}, q, st);
 }
@@ -140,27 +185,37 @@ static int check_proj(const twist_proj_args* a) {
 
 extern "C" int32_t twist_subnet_attn_proj_fwd(const twist_proj_args* a, void* stream) {
   TWIST_TRY(check_proj(a));
-  if (!a->in || !a->w || !a->out) return TWIST_ERR_NULL;
-  cudaStream_t st = static_cast<cudaStream_t>(stream);
   const int S = a->n_subnets, T = a->tokens, d = a->d_model, n = a->n;
+  const bool qkv = a->which == TWIST_PROJ_QKV;
+  const int w_out = qkv ? n : d;      // width of the output
+  bool fused = false;
+  TWIST_TRY(check_fused(a->tgt, a->loss, a->d_out, a->loss_ws, a->loss_ws_bytes, S, T, w_out, a->valid_cols,
+                        a->seg_begin, a->seg_width, &fused));
+  if (!a->in || !a->w || (!a->out && !fused)) return TWIST_ERR_NULL;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (a->dtype == TWIST_FP32) {
+    if (!a->out) return TWIST_ERR_NULL;
     const float* in = static_cast<const float*>(a->in);
     const float* w = static_cast<const float*>(a->w);
     float* out = static_cast<float*>(a->out);
-    if (a->which == TWIST_PROJ_QKV)
-      return sgemm_f32(false, true, in, w, out, T, n, d, d, d, n, (long long)T * d, (long long)n * d, (long long)T * n,
-                       S, a->out_scale, st);
-    return sgemm_f32(false, false, in, w, out, T, d, n, n, d, d, (long long)T * n, (long long)n * d, (long long)T * d, S,
-                     a->out_scale, st);
+    if (qkv)
+      TWIST_TRY(sgemm_f32(false, true, in, w, out, T, n, d, d, d, n, (long long)T * d, (long long)n * d,
+                          (long long)T * n, S, a->out_scale, st));
+    else
+      TWIST_TRY(sgemm_f32(false, false, in, w, out, T, d, n, n, d, d, (long long)T * n, (long long)n * d,
+                          (long long)T * d, S, a->out_scale, st));
+    if (!fused) return TWIST_OK;
+    return twist_mse_fwd_bwd(out, a->tgt, const_cast<void*>(a->d_out), a->loss, S, T, w_out, a->valid_cols,
+                             a->seg_begin, a->seg_width, TWIST_FP32, a->loss_ws, a->loss_ws_bytes, stream);
   }
-  if (a->which == TWIST_PROJ_QKV) {
-    GemmParams p = base_params(T, n, d, S, a->out_scale);
-    p.out0 = static_cast<__nv_bfloat16*>(a->out);
-    return launch_gemm_bf16(0, EPI_STORE, GemmOperand{a->in, T, d}, GemmOperand{a->w, n, d}, p, st);
-  }
-  GemmParams p = base_params(T, d, n, S, a->out_scale);
+  const GemmOperand A{a->in, T, qkv ? d : n}, W{a->w, n, d};
+  GemmParams p = qkv ? base_params(T, n, d, S, a->out_scale) : base_params(T, d, n, S, a->out_scale);
+  const int layout = qkv ? 0 : 1;
+  if (fused)
+    return launch_fused_loss(layout, A, W, p, a->out, a->tgt, const_cast<void*>(a->d_out), a->loss, a->loss_ws,
+                             a->valid_cols, a->seg_begin, a->seg_width, st);
   p.out0 = static_cast<__nv_bfloat16*>(a->out);
-  return launch_gemm_bf16(1, EPI_STORE, GemmOperand{a->in, T, n}, GemmOperand{a->w, n, d}, p, st);
+  return launch_gemm_bf16(layout, EPI_STORE, A, W, p, st);
 }
 
 extern "C" int32_t twist_subnet_attn_proj_bwd(const twist_proj_args* a, void* stream) {

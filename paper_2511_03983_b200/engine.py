@@ -29,9 +29,14 @@ class RoundEngine:
     BLOCKS = ("ffn", "qkv", "o")
 
     def __init__(self, w: Workload, device: str = "cuda", keep_f32_full: bool = False, compute_dx: bool = True,
-                 dump_grads: bool = False):
+                 dump_grads: bool = False, fuse_loss: bool = True, store_outputs: bool = True):
+        """fuse_loss: evaluate the loss inside the forward call's output kernel (otherwise with the
+        stand-alone twist_mse_fwd_bwd).  store_outputs=False (fused loss, bf16 only) skips storing the
+        block outputs, which nothing reads once the loss gradient exists."""
         self.w, self.dev = w, torch.device(device)
         self.compute_dx, self.dump_grads = compute_dx, dump_grads or w.dtype != DTYPE_BF16
+        self.fuse_loss = fuse_loss
+        self.store_outputs = store_outputs or not fuse_loss or w.dtype != DTYPE_BF16
         td, dev = _tdtype(w), self.dev
         S, T, d, f = w.n_subnets, w.tokens, w.d_model, w.f_sub
         self.g = 2 if w.ffn_kind == FFN_SWIGLU else 1
@@ -92,7 +97,9 @@ class RoundEngine:
             self.dw_qkv = f32(S, self.nq, d) if self.dump_grads else None
             self.dw_o = f32(S, self.a_sub, d) if self.dump_grads else None
         self.loss = torch.zeros(L, 3, max(1, w.local_steps), S, dtype=torch.float32, device=dev)
-        self.ws = torch.empty(B.twist_mse_workspace_bytes(S), dtype=torch.uint8, device=dev)
+        ws_bytes = max(B.twist_mse_workspace_bytes(S),
+                       B.twist_fused_loss_workspace_bytes(S, T, max(d, self.nq if self.has_attn else 0)))
+        self.ws = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
         self.alpha_f = math.sqrt(w.n_ffn_blocks / w.ffn_keep)
         self.alpha_a = math.sqrt(w.n_heads / w.head_keep) if self.has_attn else 1.0
         # batches: lists over the local step k of [S][T][width] tensors
@@ -204,13 +211,18 @@ class RoundEngine:
     def ffn_step(self, l: int, k: int, lr: Optional[float] = None):
         w = self.w
         lr = w.lr if lr is None else lr
+        fused = dict(tgt=self.Td[k], loss=self.loss[l, 0, k], loss_ws=self.ws) if self.fuse_loss else {}
         a = B.ffn_args(w.ffn_kind, w.dtype, w.n_subnets, w.tokens, w.d_model, w.f_sub, self.alpha_f, lr,
                        x=self.X[k], w_gu=self.w_gu, w_down=self.w_down, w_gu_master=self.w_gu_m,
-                       w_down_master=self.w_down_m, pre=self.pre, hh=self.hh, y=self.y, dy=self.dy, dpre=self.dpre,
-                       dx=self.dx, dw_gu=self.dw_gu, dw_down=self.dw_down)
+                       w_down_master=self.w_down_m, pre=self.pre, hh=self.hh,
+                       y=self.y if self.store_outputs else None, dy=self.dy, dpre=self.dpre,
+                       dx=self.dx, dw_gu=self.dw_gu, dw_down=self.dw_down, **fused)
         with self._timed("ffn_fwd"):
             B.twist_subnet_ffn_fwd(a)
-        self._mse(self.y, self.Td[k], self.dy, self.loss[l, 0, k], w.d_model)
+        if self.fuse_loss:
+            self.launches += 1 if w.dtype == DTYPE_BF16 else 2
+        else:
+            self._mse(self.y, self.Td[k], self.dy, self.loss[l, 0, k], w.d_model)
         with self._timed("ffn_bwd"):
             B.twist_subnet_ffn_bwd(a)
         bf16 = w.dtype == DTYPE_BF16
@@ -219,14 +231,19 @@ class RoundEngine:
     def qkv_step(self, l: int, k: int, lr: Optional[float] = None):
         w = self.w
         lr = w.lr if lr is None else lr
+        ragged = self.w.n_kv_heads != self.w.n_heads
+        mask = dict(valid_cols=self.kv_cols[l], seg_begin=self.a_sub, seg_width=self.kv_max * w.d_head) if ragged else {}
+        fused = dict(tgt=self.Tq[k], loss=self.loss[l, 1, k], loss_ws=self.ws, **mask) if self.fuse_loss else {}
         a = B.proj_args(B.PROJ_QKV, w.dtype, w.n_subnets, w.tokens, w.d_model, self.nq, 1.0, lr, in_=self.X[k],
-                        w=self.w_qkv, w_master=self.w_qkv_m, out=self.qkv_out, d_out=self.dqkv, d_in=self.dx,
-                        dw=self.dw_qkv)
+                        w=self.w_qkv, w_master=self.w_qkv_m, out=self.qkv_out if self.store_outputs else None,
+                        d_out=self.dqkv, d_in=self.dx, dw=self.dw_qkv, **fused)
         with self._timed("qkv_fwd"):
             B.twist_subnet_attn_proj_fwd(a)
-        ragged = self.w.n_kv_heads != self.w.n_heads
-        self._mse(self.qkv_out, self.Tq[k], self.dqkv, self.loss[l, 1, k], self.nq,
-                  self.kv_cols[l] if ragged else None, self.a_sub, self.kv_max * w.d_head)
+        if self.fuse_loss:
+            self.launches += 1 if w.dtype == DTYPE_BF16 else 2
+        else:
+            self._mse(self.qkv_out, self.Tq[k], self.dqkv, self.loss[l, 1, k], self.nq,
+                      self.kv_cols[l] if ragged else None, self.a_sub, self.kv_max * w.d_head)
         with self._timed("qkv_bwd"):
             B.twist_subnet_attn_proj_bwd(a)
         self.launches += 1 + 1 + (1 if self.compute_dx else 0) + (0 if w.dtype == DTYPE_BF16 else 1)
@@ -234,12 +251,16 @@ class RoundEngine:
     def o_step(self, l: int, k: int, lr: Optional[float] = None):
         w = self.w
         lr = w.lr if lr is None else lr
+        fused = dict(tgt=self.Td[k], loss=self.loss[l, 2, k], loss_ws=self.ws) if self.fuse_loss else {}
         a = B.proj_args(B.PROJ_O, w.dtype, w.n_subnets, w.tokens, w.d_model, self.a_sub, self.alpha_a, lr,
-                        in_=self.A[k], w=self.w_o, w_master=self.w_o_m, out=self.y, d_out=self.dy, d_in=self.da,
-                        dw=self.dw_o)
+                        in_=self.A[k], w=self.w_o, w_master=self.w_o_m, out=self.y if self.store_outputs else None,
+                        d_out=self.dy, d_in=self.da, dw=self.dw_o, **fused)
         with self._timed("o_fwd"):
             B.twist_subnet_attn_proj_fwd(a)
-        self._mse(self.y, self.Td[k], self.dy, self.loss[l, 2, k], w.d_model)
+        if self.fuse_loss:
+            self.launches += 1 if w.dtype == DTYPE_BF16 else 2
+        else:
+            self._mse(self.y, self.Td[k], self.dy, self.loss[l, 2, k], w.d_model)
         with self._timed("o_bwd"):
             B.twist_subnet_attn_proj_bwd(a)
         self.launches += 1 + 1 + (1 if self.compute_dx else 0) + (0 if w.dtype == DTYPE_BF16 else 1)

@@ -316,6 +316,75 @@ def test_proj_parity(B, dtype, S, T, d, n):
             assert rel_fro(upd, -lr * want_dw) < tol, (which, "sgd")
 
 
+# --------------------------------------------------------------------------------------------- fused loss
+
+@pytest.mark.parametrize("S,T,d,f", [(2, 200, 328, 344), (3, 520, 264, 136)])
+def test_fused_loss_equals_standalone_loss_ffn(B, S, T, d, f):
+    """The loss evaluated in the forward call's output kernel gives the gradient twist_mse_fwd_bwd gives on
+    the stored output, bit for bit, and the same loss up to summation order; both match the oracle."""
+    td, dtype, kind, alpha = torch.bfloat16, I.DTYPE_BF16, I.FFN_SWIGLU, 2.0
+    X = I.normal(61, 1, (S, T, d), 1.0, dtype)
+    Wgu = I.normal(61, 2, (S, 2 * f, d), 0.05, dtype)
+    Wd = I.normal(61, 3, (S, f, d), 0.05, dtype)
+    Tg = I.normal(61, 4, (S, T, d), 1.0, dtype)
+    t = lambda *s: torch.zeros(*s, dtype=td, device="cuda")
+    pre, hh, y, dy_a, dy_b = t(S, T, 2 * f), t(S, T, f), t(S, T, d), t(S, T, d), t(S, T, d)
+    loss_a = torch.zeros(S, dtype=torch.float32, device="cuda")
+    loss_b = torch.zeros(S, dtype=torch.float32, device="cuda")
+    ws = torch.empty(B.twist_fused_loss_workspace_bytes(S, T, d), dtype=torch.uint8, device="cuda")
+    common = dict(x=dev(X, td), w_gu=dev(Wgu, td), w_down=dev(Wd, td), pre=pre, hh=hh)
+    B.twist_subnet_ffn_fwd(B.ffn_args(kind, dtype, S, T, d, f, alpha, 0.0, y=y, **common))
+    B.twist_mse_fwd_bwd(y, dev(Tg, td), dy_a, loss_a, S, T, d, None, 0, 0, dtype, ws)
+    y2 = t(S, T, d)
+    B.twist_subnet_ffn_fwd(B.ffn_args(kind, dtype, S, T, d, f, alpha, 0.0, y=y2, dy=dy_b, tgt=dev(Tg, td), loss=loss_b,
+                                      loss_ws=ws, **common))
+    dy_c = t(S, T, d)     # the output need not be stored
+    B.twist_subnet_ffn_fwd(B.ffn_args(kind, dtype, S, T, d, f, alpha, 0.0, y=None, dy=dy_c, tgt=dev(Tg, td),
+                                      loss=loss_b, loss_ws=ws, **common))
+    torch.cuda.synchronize()
+    check_status(B)
+    assert torch.equal(y, y2) and torch.equal(dy_a, dy_b) and torch.equal(dy_a, dy_c)
+    assert torch.allclose(loss_a, loss_b, rtol=1e-5, atol=0)
+    for s in range(S):
+        Yw, _ = o.ffn_fwd(X[s].astype(np.float64), Wgu[s, f:].astype(np.float64), Wgu[s, :f].astype(np.float64),
+                          Wd[s].astype(np.float64), kind, alpha, True)
+        want_loss, want_dy = o.mse(Yw, Tg[s].astype(np.float64), True)
+        assert abs(loss_b[s].item() - want_loss) <= 2e-2 * want_loss
+        assert rel_fro(host(dy_b[s]), want_dy) < GEMM_TOL
+
+
+def test_fused_loss_equals_standalone_loss_proj_with_column_mask(B):
+    td, dtype = torch.bfloat16, I.DTYPE_BF16
+    S, T, d = 3, 300, 200
+    a_sub, kvw = 64, 48                   # [Q 64 | K 48 | V 48], valid K/V columns per subnet below
+    n = a_sub + 2 * kvw
+    valid = dev(np.array([48, 16, 32], dtype=np.int32))
+    Xin = I.normal(71, 1, (S, T, d), 1.0, dtype)
+    W = I.normal(71, 2, (S, n, d), 0.05, dtype)
+    Tg = I.normal(71, 3, (S, T, n), 1.0, dtype)
+    out = torch.zeros(S, T, n, dtype=td, device="cuda")
+    d_a, d_b = torch.zeros_like(out), torch.zeros_like(out)
+    loss_a = torch.zeros(S, dtype=torch.float32, device="cuda")
+    loss_b = torch.zeros(S, dtype=torch.float32, device="cuda")
+    ws = torch.empty(B.twist_fused_loss_workspace_bytes(S, T, max(n, d)), dtype=torch.uint8, device="cuda")
+    for which, width, w_in, mask in ((B.PROJ_QKV, n, d, True), (B.PROJ_O, d, n, False)):
+        xin = dev(Xin, td) if which == B.PROJ_QKV else dev(Tg, td)       # O projection: input of width n
+        tg = dev(Tg, td) if which == B.PROJ_QKV else dev(Xin, td)
+        o1 = torch.zeros(S, T, width, dtype=td, device="cuda")
+        g1, g2 = torch.zeros_like(o1), torch.zeros_like(o1)
+        kw = dict(valid_cols=valid, seg_begin=a_sub, seg_width=kvw) if mask else {}
+        B.twist_subnet_attn_proj_fwd(B.proj_args(which, dtype, S, T, d, n, 1.3, 0.0, in_=xin, w=dev(W, td), out=o1))
+        B.twist_mse_fwd_bwd(o1, tg, g1, loss_a, S, T, width, valid if mask else None, a_sub if mask else 0,
+                            kvw if mask else 0, dtype, ws)
+        torch.cuda.synchronize()
+        B.twist_subnet_attn_proj_fwd(B.proj_args(which, dtype, S, T, d, n, 1.3, 0.0, in_=xin, w=dev(W, td), out=None,
+                                                 d_out=g2, tgt=tg, loss=loss_b, loss_ws=ws, **kw))
+        torch.cuda.synchronize()
+        check_status(B)
+        assert torch.equal(g1, g2), which
+        assert torch.allclose(loss_a, loss_b, rtol=1e-5, atol=0), which
+
+
 # --------------------------------------------------------------------------------------------- whole rounds
 
 def _load_full(eng, w):
@@ -345,10 +414,10 @@ def _load_batches(eng, w, rnd):
     return store
 
 
-def _run_round_and_compare(B, w, rnd=0, tol_dw=5e-2):
+def _run_round_and_compare(B, w, rnd=0, tol_dw=5e-2, **engine_kw):
     from paper_2511_03983_b200.engine import RoundEngine
     lowp = w.dtype == I.DTYPE_BF16
-    eng = RoundEngine(w, keep_f32_full=True)
+    eng = RoundEngine(w, keep_f32_full=True, **engine_kw)
     full_np = _load_full(eng, w)
     store = _load_batches(eng, w, rnd)
     before = {m: v.clone() for m, v in eng.full.items()}
@@ -398,6 +467,12 @@ def test_config1_fp32_round_matches_oracle_everywhere(B):
 def test_scaled_twin_rounds_match_oracle(B, cfg, dims):
     w = I.scaled_twin(I.PRESETS[cfg], **dims)
     _run_round_and_compare(B, w)
+
+
+@pytest.mark.parametrize("engine_kw", [dict(fuse_loss=False), dict(store_outputs=False)])
+def test_scaled_twin_round_with_standalone_loss_and_without_stored_outputs(B, engine_kw):
+    w = I.scaled_twin(I.PRESETS[3], d_model=256, d_ff=688, d_head=8, tokens=256, n_layers=1, local_steps=2)
+    _run_round_and_compare(B, w, **engine_kw)
 
 
 def test_round_with_zero_lr_is_identity_on_the_bf16_model(B):
