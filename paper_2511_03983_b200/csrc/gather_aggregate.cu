@@ -1,8 +1,11 @@
 // twist_gather_subnets (dispatcher, Sec. 3.2) and twist_aggregate (aggregator, Sec. 3.3).
-// Both are HBM-bandwidth kernels: one warp moves one whole row with 16-byte accesses per lane,
-// several independent loads in flight per lane, streaming stores.  Rows are >= 1.5 KB in every
-// workload (8 KB at d_model = 4096 in bf16), so every access is fully coalesced.
+// Both are HBM-bandwidth kernels over whole rows (>= 1.5 KB in every workload, 8 KB at d_model = 4096
+// in bf16).  The gather moves rows with the bulk-copy engine: global -> shared memory -> global, the
+// fp32 master widened in shared memory on the way, so that the SMs issue almost no global-memory
+// instructions.  The aggregate is one warp per row with 16-byte accesses per lane and several
+// independent loads in flight.
 #include "common.cuh"
+#include "ptx.cuh"
 
 namespace twist {
 namespace {
@@ -47,14 +50,49 @@ __device__ inline uint4 widen_hi(uint4 v) {   // bf16 elements 4..7
 
 constexpr int kUnroll = 4;
 
-// One warp per destination row.  ELEM = 2 (bf16) or 4 (fp32) bytes.
+constexpr int kGatherWarps = 8;          // warps per CTA
+constexpr int kGatherPieceBytes = 4096;  // a row travels in pieces of at most this many bytes
+
+// Work item = (destination row, piece of the row); one warp per item at a time, two buffers per warp so
+// the load of the next item overlaps the widening and the stores of the current one.
+// Shared memory per warp and buffer: the piece as loaded [piece bytes] and, when masters are written,
+// its fp32 widening [2 x piece bytes].  ELEM = 2 (bf16) or 4 (fp32) bytes.
 template <int ELEM>
-__global__ void __launch_bounds__(256) gather_rows_kernel(const __grid_constant__ GatherParams p) {
-  const int lane = threadIdx.x & 31;
-  const long long warp0 = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-  const long long nwarps = ((long long)gridDim.x * blockDim.x) >> 5;
-  const int chunks = p.d * ELEM / 16;                 // 16-byte chunks per row
-  for (long long r = warp0; r < p.total_rows; r += nwarps) {
+__global__ void __launch_bounds__(kGatherWarps * 32) gather_rows_kernel(const __grid_constant__ GatherParams p,
+                                                                        int piece_bytes, int pieces, int buf_bytes,
+                                                                        int* status) {
+  extern __shared__ __align__(128) unsigned char gsm[];
+  __shared__ __align__(8) unsigned long long bars[kGatherWarps][2];
+  __shared__ int abort_flag;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (threadIdx.x == 0) abort_flag = 0;
+  if (lane == 0) {
+    mbar_init(smem_u32(&bars[warp][0]), 1);
+    mbar_init(smem_u32(&bars[warp][1]), 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    fence_async_smem();
+  }
+  __syncthreads();
+  const uint32_t wbase = smem_u32(gsm) + (uint32_t)warp * 2u * (uint32_t)buf_bytes;
+  const int row_bytes = p.d * ELEM;
+  const long long items = p.total_rows * pieces;
+  const long long wid0 = (long long)blockIdx.x * kGatherWarps + warp;
+  const long long stride = (long long)gridDim.x * kGatherWarps;
+
+  // Item `it` decoded.  The kept-block index is loaded here but only used when the item's copy is requested,
+  // one iteration later, so that its latency (it is rarely cached) stays off the critical path.
+  struct Item {
+    const char* src_base;   // null: a padding row, written as zeros
+    long long src_row;      // row of the source piece before the block index is applied
+    int block_rows, idxv, off;
+    char* dst; char* mst; int bytes;
+  };
+  auto decode = [&](long long it) {
+    Item o;
+    o.src_base = nullptr; o.src_row = 0; o.block_rows = 0; o.idxv = 0; o.off = 0; o.dst = nullptr; o.mst = nullptr; o.bytes = 0;
+    if (it >= items) return o;
+    const long long r = it / pieces;
+    const int pc = (int)(it - r * pieces);
     int g = 0;
     while (g + 1 < p.n_segs && r >= p.row_end[g]) ++g;
     const twist_gather_segment& sg = p.seg[g];
@@ -64,36 +102,76 @@ __global__ void __launch_bounds__(256) gather_rows_kernel(const __grid_constant_
     const int rem = (int)(rl - (long long)s * rows_per_subnet);
     const int j = rem / sg.block_rows, i = rem - j * sg.block_rows;
     const bool valid = sg.count ? (j < sg.count[s]) : true;
-    const long long dst_row = sg.dst_row_offset + rem;
-    uint4* dst = reinterpret_cast<uint4*>(static_cast<char*>(sg.dst) +
-                                          ((long long)s * sg.dst_subnet_stride + dst_row * p.d) * ELEM);
-    uint4* mst = sg.dst_master ? reinterpret_cast<uint4*>(sg.dst_master + (long long)s * sg.dst_subnet_stride +
-                                                          dst_row * p.d)
-                               : nullptr;
-    const uint4* src = nullptr;
+    const long long dst_elem = (long long)s * sg.dst_subnet_stride + (sg.dst_row_offset + rem) * p.d;
+    o.off = pc * piece_bytes;
+    o.bytes = min(piece_bytes, row_bytes - o.off);
+    o.dst = static_cast<char*>(sg.dst) + dst_elem * ELEM + o.off;
+    o.mst = (ELEM == 2 && sg.dst_master) ? reinterpret_cast<char*>(sg.dst_master + dst_elem) + 2 * o.off : nullptr;
     if (valid) {
-      const long long src_row = sg.src_row_offset + (long long)sg.idx[(long long)s * sg.idx_stride + j] * sg.block_rows + i;
-      src = reinterpret_cast<const uint4*>(static_cast<const char*>(sg.src) + src_row * p.d * ELEM);
+      o.src_base = static_cast<const char*>(sg.src);
+      o.src_row = sg.src_row_offset + i;
+      o.block_rows = sg.block_rows;
+      asm volatile("ld.global.nc.s32 %0, [%1];" : "=r"(o.idxv) : "l"(sg.idx + (long long)s * sg.idx_stride + j));
     }
-    for (int c0 = lane; c0 < chunks; c0 += 32 * kUnroll) {
-      uint4 v[kUnroll];
-#pragma unroll
-      for (int u = 0; u < kUnroll; ++u) {
-        const int c = c0 + 32 * u;
-        v[u] = (valid && c < chunks) ? ld_nc(src + c) : make_uint4(0, 0, 0, 0);
+    return o;
+  };
+  auto request = [&](const Item& o, int b) {          // lane 0
+    if (!o.src_base) return;
+    const uint32_t bar = smem_u32(&bars[warp][b]);
+    const char* src = o.src_base + (o.src_row + (long long)o.idxv * o.block_rows) * row_bytes + o.off;
+    mbar_expect_tx(bar, (uint32_t)o.bytes);
+    bulk_load(wbase + (uint32_t)b * buf_bytes, src, (uint32_t)o.bytes, bar);
+  };
+
+  uint32_t uses0 = 0, uses1 = 0;                       // completed phases of each buffer's barrier
+  Item cur = decode(wid0);
+  if (lane == 0 && wid0 < items) request(cur, 0);
+  Item nxt = decode(wid0 + stride);
+  int n = 0;
+  for (long long it = wid0; it < items; it += stride, ++n) {
+    const int b = n & 1;
+    const Item nxt2 = decode(it + 2 * stride);         // its index load is in flight during this iteration
+    if (lane == 0) {
+      bulk_wait_read<0>();                             // the stores that read the other buffer are done with it
+      if (it + stride < items) request(nxt, b ^ 1);
+    }
+    const uint32_t in = wbase + (uint32_t)b * buf_bytes;
+    if (cur.src_base) {
+      const uint32_t parity = (b ? uses1 : uses0) & 1u;
+      // warp-uniform outcome: either every lane goes on or every lane leaves
+      if (!__all_sync(0xffffffffu, mbar_wait(smem_u32(&bars[warp][b]), parity, &abort_flag, status))) break;
+      if (b) ++uses1; else ++uses0;
+      if (lane == 0) bulk_store(cur.dst, in, (uint32_t)cur.bytes);
+      if (cur.mst) {                                   // exact widening bf16 -> fp32, staged in shared memory
+        const uint32_t out = in + (uint32_t)piece_bytes;
+        for (int c = lane; c < cur.bytes / 16; c += 32) {
+          const uint4 v = lds128(in + 16u * c);
+          sts128(out + 32u * c, widen_lo(v));
+          sts128(out + 32u * c + 16u, widen_hi(v));
+        }
+        fence_async_smem();
+        __syncwarp();
+        if (lane == 0) bulk_store(cur.mst, out, 2u * (uint32_t)cur.bytes);
       }
-#pragma unroll
-      for (int u = 0; u < kUnroll; ++u) {
-        const int c = c0 + 32 * u;
-        if (c < chunks) {
-          st_cs(dst + c, v[u]);
-          if (ELEM == 2 && mst) {
-            st_cs(mst + 2 * c, widen_lo(v[u]));
-            st_cs(mst + 2 * c + 1, widen_hi(v[u]));
-          }
+      if (lane == 0) bulk_commit();
+    } else {                                           // padding row: zeros, plain stores
+      for (int c = lane; c < cur.bytes / 16; c += 32) {
+        st_cs(reinterpret_cast<uint4*>(cur.dst) + c, make_uint4(0, 0, 0, 0));
+        if (cur.mst) {
+          st_cs(reinterpret_cast<uint4*>(cur.mst) + 2 * c, make_uint4(0, 0, 0, 0));
+          st_cs(reinterpret_cast<uint4*>(cur.mst) + 2 * c + 1, make_uint4(0, 0, 0, 0));
         }
       }
     }
+    __syncwarp();
+    cur = nxt;
+    nxt = nxt2;
+  }
+  if (lane == 0) bulk_wait_read<0>();
+  __syncthreads();
+  if (abort_flag) {     // a wait expired: let a copy that may still be in flight land before shared memory is released
+    const uint64_t t0 = global_timer_ns();
+    while (global_timer_ns() - t0 < 2000000ull) __nanosleep(1000);
   }
 }
 
@@ -102,7 +180,9 @@ __device__ inline uint32_t pack_bf16x2_rn(float lo, float hi) {
   return *reinterpret_cast<uint32_t*>(&t);
 }
 
-// One warp per full-model row: fp32 sum over the covering subnets in ascending order, IEEE divide.
+// One warp per full-model row: 16-byte accesses per lane, several independent loads in flight; fp32 sum over the
+// covering subnets in ascending order, correctly rounded quotient.  (A bulk-copy version of this kernel, like the
+// gather's, measured slower: 2 KB pieces keep too few bytes in flight per SM.)
 template <bool BF16>
 __global__ void __launch_bounds__(256) aggregate_rows_kernel(const __grid_constant__ AggParams p) {
   const int lane = threadIdx.x & 31;
@@ -125,7 +205,14 @@ __global__ void __launch_bounds__(256) aggregate_rows_kernel(const __grid_consta
       mine = reinterpret_cast<const float4*>(sg.sub + (long long)s * sg.sub_subnet_stride + srow * p.d);
     }
     const long long drow = sg.dst_row_offset + rl;
+    // Quotient by the coverage count: reciprocal product corrected with the exact remainder, which gives
+    // the correctly rounded quotient (the same bits as an IEEE division) at a fraction of its cost.
     const float denom = (float)cnt;
+    const float rden = 1.0f / denom;
+    auto quot = [&](float a) {
+      const float q = a * rden;
+      return fmaf(fmaf(-q, denom, a), rden, q);
+    };
     for (int c0 = lane; c0 < chunks; c0 += 32 * kUnroll) {
       float4 acc[kUnroll];
 #pragma unroll
@@ -148,7 +235,7 @@ __global__ void __launch_bounds__(256) aggregate_rows_kernel(const __grid_consta
       for (int u = 0; u < kUnroll; ++u) {
         const int c = c0 + 32 * u;
         if (c < chunks) {
-          float4 q = make_float4(acc[u].x / denom, acc[u].y / denom, acc[u].z / denom, acc[u].w / denom);
+          float4 q = make_float4(quot(acc[u].x), quot(acc[u].y), quot(acc[u].z), quot(acc[u].w));
           uint4 qb = make_uint4(__float_as_uint(q.x), __float_as_uint(q.y), __float_as_uint(q.z), __float_as_uint(q.w));
           if (BF16) {
             if (sg.dst_f32) st_cs(reinterpret_cast<uint4*>(sg.dst_f32 + drow * p.d) + c, qb);
@@ -200,9 +287,34 @@ extern "C" int32_t twist_gather_subnets(const twist_gather_segment* segs, int32_
   p.d = d;
   p.total_rows = total;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  const int grid = grid_for_rows(total);
-  if (dtype == TWIST_BF16) gather_rows_kernel<2><<<grid, 256, 0, st>>>(p);
-  else gather_rows_kernel<4><<<grid, 256, 0, st>>>(p);
+  bool any_master = false;
+  for (int g = 0; g < n_segs; ++g) any_master |= segs[g].dst_master != nullptr;
+  const int row_bytes = d * elem;
+  const int piece_bytes = row_bytes < kGatherPieceBytes ? row_bytes : kGatherPieceBytes;
+  const int pieces = (row_bytes + piece_bytes - 1) / piece_bytes;
+  const int buf_bytes = piece_bytes * (any_master ? 3 : 1);          // the piece + its fp32 widening
+  const int smem = kGatherWarps * 2 * buf_bytes;
+  static bool configured = false;
+  if (!configured) {
+    TWIST_CUDA_TRY(cudaFuncSetAttribute(gather_rows_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        kGatherWarps * 2 * 3 * kGatherPieceBytes));
+    TWIST_CUDA_TRY(cudaFuncSetAttribute(gather_rows_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        kGatherWarps * 2 * kGatherPieceBytes));
+    configured = true;
+  }
+  // persistent grid: as many CTAs per SM as the shared memory allows (at most 8), or fewer for small inputs
+  int per_sm = (220 * 1024) / (smem + 1024);
+  per_sm = per_sm < 1 ? 1 : (per_sm > 8 ? 8 : per_sm);
+  const long long items = total * pieces;
+  const long long want = (items + kGatherWarps - 1) / kGatherWarps;
+  const long long cap = (long long)sm_count() * per_sm;
+  const int grid = (int)(want < cap ? (want > 0 ? want : 1) : cap);
+  int* status = device_status_ptr();
+  if (!status) return TWIST_ERR_CUDA;
+  if (dtype == TWIST_BF16)
+    gather_rows_kernel<2><<<grid, kGatherWarps * 32, smem, st>>>(p, piece_bytes, pieces, buf_bytes, status);
+  else
+    gather_rows_kernel<4><<<grid, kGatherWarps * 32, smem, st>>>(p, piece_bytes, pieces, buf_bytes, status);
   TWIST_LAUNCH_CHECK();
   return TWIST_OK;
 }

@@ -27,6 +27,7 @@
 #include <cuda.h>
 
 #include "common.cuh"
+#include "ptx.cuh"
 
 namespace twist {
 
@@ -94,26 +95,6 @@ template <> struct EpiAcc<EPI_SWIGLU_FWD> { uint32_t r0[32], r1[32]; };
 // ---------------------------------------------------------------------------------------------
 // PTX wrappers
 // ---------------------------------------------------------------------------------------------
-__device__ inline uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ inline void mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ inline void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ inline void mbar_arrive(uint32_t bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ inline uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
-  uint32_t done;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(done) : "r"(bar), "r"(parity) : "memory");
-  return done;
-}
 // Cluster helpers: rank of this CTA in its pair, address of a shared-memory location of CTA `rank`
 // in the cluster-wide shared window, arrival on a barrier given by such an address, cluster barrier.
 __device__ inline uint32_t cluster_rank() {
@@ -132,28 +113,6 @@ __device__ inline void mbar_arrive_cluster(uint32_t cluster_addr) {
 __device__ inline void cluster_sync_all() {
   asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
-__device__ inline uint64_t global_timer_ns() {
-  uint64_t t;
-  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-  return t;
-}
-
-// Bounded wait: gives up after ~2 s of wall time or as soon as another role of the CTA gave up.
-__device__ inline bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status) {
-  if (mbar_try_wait(bar, parity)) return true;
-  const uint64_t t0 = global_timer_ns();
-  for (uint32_t it = 1;; ++it) {
-    if (mbar_try_wait(bar, parity)) return true;
-    if ((it & 255u) == 0) {
-      if (*abort_flag || global_timer_ns() - t0 > 2000000000ull) {
-        *abort_flag = 1;
-        atomicExch(status, (int)TWIST_ERR_DEVICE_TIMEOUT);
-        return false;
-      }
-    }
-  }
-}
-
 // Tiled copy into this CTA's shared memory; completion bytes are counted on `bar`, which may be a
 // barrier of the other CTA of the pair (cluster-window address).
 __device__ inline void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2) {
@@ -171,18 +130,6 @@ __device__ inline void tma_load_3d_local(uint32_t dst, const CUtensorMap* map, u
 __device__ inline void tma_store_3d(const CUtensorMap* map, uint32_t src, int c0, int c1, int c2) {
   asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%2, %3, %4}], [%1];"
                ::"l"(map), "r"(src), "r"(c0), "r"(c1), "r"(c2) : "memory");
-}
-__device__ inline void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
-template <int N>
-__device__ inline void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
-__device__ inline void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-__device__ inline uint4 lds128(uint32_t a) {
-  uint4 v;
-  asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(a));
-  return v;
-}
-__device__ inline void sts128(uint32_t a, uint4 v) {
-  asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(a), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
 }
 __device__ inline void tma_prefetch_desc(const CUtensorMap* map) {
   asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
@@ -436,7 +383,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           for (int q = 0; q < 8; ++q) m[q] = (4 * q < valid) ? src[q] : make_float4(0.f, 0.f, 0.f, 0.f);
         };
         load_master(0, mv[0]);
-        if (!mbar_wait(tfull_bar(slot), acc_phase, abort_flag, p.status)) { ok = false; break; }
+        if (!__all_sync(0xffffffffu, mbar_wait(tfull_bar(slot), acc_phase, abort_flag, p.status))) { ok = false; break; }
         tc_fence_after();
         tc_ld32(t_row, acc[0].r0);
 #pragma unroll
@@ -527,7 +474,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           tc_ld32(t_row + 32 * c, a.r0);
           if constexpr (EPI == EPI_SWIGLU_FWD) tc_ld32(t_row + kCtaN + 32 * c, a.r1);
         };
-        if (!mbar_wait(tfull_bar(slot), acc_phase, abort_flag, p.status)) { ok = false; break; }
+        if (!__all_sync(0xffffffffu, mbar_wait(tfull_bar(slot), acc_phase, abort_flag, p.status))) { ok = false; break; }
         tc_fence_after();
         load_acc(0, acc[0]);
 #pragma unroll
@@ -535,7 +482,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           const uint32_t gc = tl * kChunks + c;
           const int n = n_base + 32 * c;
           if (kIn > 0) {      // this chunk's boxes have arrived
-            if (!mbar_wait(in_bar(warp, gc & (kBufs - 1)), (gc / kBufs) & 1u, abort_flag, p.status)) { ok = false; break; }
+            if (!__all_sync(0xffffffffu, mbar_wait(in_bar(warp, gc & (kBufs - 1)), (gc / kBufs) & 1u, abort_flag, p.status))) { ok = false; break; }
           } else {            // the bulk store that last read this buffer is done with it
             if (lane == 0) bulk_wait_read<kBufs - 1>();
             __syncwarp();
