@@ -218,9 +218,14 @@ def _act_grad(pre, kind):
     raise ValueError(kind)
 
 
-def ffn_fwd(X, W_up, W_gate, W_down, kind, alpha, lowp):
+def _plus(v, residual):
+    return v if residual is None else v + residual
+
+
+def ffn_fwd(X, W_up, W_gate, W_down, kind, alpha, lowp, residual=None):
     """Y = alpha * act(X W_up^T) W_down  (MLP)  or  alpha * (silu(X W_gate^T) * (X W_up^T)) W_down.
-    Returns Y [T, d] and the tensors kept for the backward pass (stored precision)."""
+    Returns Y [T, d] and the tensors kept for the backward pass (stored precision).
+    `residual` (App. A, Transformer Layer Architecture, final output) is added before Y is stored."""
     U = X @ W_up.T
     if kind == FFN_SWIGLU:
         G = X @ W_gate.T
@@ -228,12 +233,13 @@ def ffn_fwd(X, W_up, W_gate, W_down, kind, alpha, lowp):
         saved = {"G": _q(G, lowp), "U": _q(U, lowp), "Hh": _q(Hh, lowp)}
     else:
         saved = {"U": _q(U, lowp), "Hh": _q(_act(U, kind), lowp)}
-    Y = _q(alpha * (saved["Hh"] @ W_down), lowp)
+    Y = _q(_plus(alpha * (saved["Hh"] @ W_down), residual), lowp)
     return Y, saved
 
 
-def ffn_bwd(dY, X, saved, W_up, W_gate, W_down, kind, alpha, lowp):
-    """Exact chain rule through ffn_fwd.  Returns dX and dW_up, dW_gate, dW_down ([f', d] each)."""
+def ffn_bwd(dY, X, saved, W_up, W_gate, W_down, kind, alpha, lowp, residual=None):
+    """Exact chain rule through ffn_fwd.  Returns dX and dW_up, dW_gate, dW_down ([f', d] each).
+    `residual`: gradient arriving over the skip connection, added to dX before it is stored."""
     dHh = alpha * (dY @ W_down.T)
     dW_down = alpha * (saved["Hh"].T @ dY)
     if kind == FFN_SWIGLU:
@@ -241,10 +247,10 @@ def ffn_bwd(dY, X, saved, W_up, W_gate, W_down, kind, alpha, lowp):
         sg = _sigmoid(G)
         dG = _q(dHh * U * (sg * (1.0 + G * (1.0 - sg))), lowp)
         dU = _q(dHh * (G * sg), lowp)
-        dX = _q(dG @ W_gate + dU @ W_up, lowp)
+        dX = _q(_plus(dG @ W_gate + dU @ W_up, residual), lowp)
         return dX, dU.T @ X, dG.T @ X, dW_down
     dU = _q(dHh * _act_grad(saved["U"], kind), lowp)
-    dX = _q(dU @ W_up, lowp)
+    dX = _q(_plus(dU @ W_up, residual), lowp)
     return dX, dU.T @ X, None, dW_down
 
 
@@ -257,12 +263,12 @@ def qkv_fwd(X, W_qkv, lowp):
     return _q(X @ W_qkv.T, lowp)
 
 
-def qkv_bwd(dQKV, X, W_qkv, lowp):
-    return _q(dQKV @ W_qkv, lowp), dQKV.T @ X
+def qkv_bwd(dQKV, X, W_qkv, lowp, residual=None):
+    return _q(_plus(dQKV @ W_qkv, residual), lowp), dQKV.T @ X
 
 
-def o_fwd(A, W_o, alpha, lowp):
-    return _q(alpha * (A @ W_o), lowp)
+def o_fwd(A, W_o, alpha, lowp, residual=None):
+    return _q(_plus(alpha * (A @ W_o), residual), lowp)
 
 
 def o_bwd(dY, A, W_o, alpha, lowp):
@@ -419,6 +425,151 @@ def round_blockwise_layer(spec, full, get_batch, rnd, layer, lowp):
     else:
         new_shadow = new
     return new, new_shadow, bp, losses
+
+
+# ----------------------------------------------------------------------------------------
+# Attention core on the kept heads (App. A, Multi-Head Attention):
+#   head_h = softmax(Q_h K_h^T / sqrt(d_head)) V_h,
+# applied per sequence with a causal mask (the workloads are causal language-model shapes:
+# position n attends positions <= n).  Grouped-query attention (an extension): kept head hq
+# reads the K/V columns of its KV group, head_kv[hq] = position of that group among the
+# subnet's kept groups.
+# Layout of QKV [T, a' + 2 kvw]: Q of the kept heads, then K of the kept groups, then V.
+# ----------------------------------------------------------------------------------------
+
+def _causal_softmax(scores):
+    n = scores.shape[0]
+    masked = np.where(np.tril(np.ones((n, n), dtype=bool)), scores, -np.inf)
+    masked = masked - masked.max(axis=1, keepdims=True)
+    e = np.exp(masked)
+    return e / e.sum(axis=1, keepdims=True)
+
+
+def attn_core_fwd(QKV, n_seqs, seq_len, d_head, head_kv, kv_width, lowp):
+    """A [T, a'] = concatenated heads; T = n_seqs * seq_len rows, sequence after sequence."""
+    H = len(head_kv)
+    a = H * d_head
+    A = np.zeros((n_seqs * seq_len, a), dtype=np.float64)
+    for b in range(n_seqs):
+        rows = slice(b * seq_len, (b + 1) * seq_len)
+        for hq in range(H):
+            g = int(head_kv[hq])
+            Q = QKV[rows, hq * d_head:(hq + 1) * d_head]
+            K = QKV[rows, a + g * d_head:a + (g + 1) * d_head]
+            V = QKV[rows, a + kv_width + g * d_head:a + kv_width + (g + 1) * d_head]
+            P = _causal_softmax(Q @ K.T / np.sqrt(d_head))
+            A[rows, hq * d_head:(hq + 1) * d_head] = P @ V
+    return _q(A, lowp)
+
+
+def attn_core_bwd(dA, QKV, n_seqs, seq_len, d_head, head_kv, kv_width, lowp):
+    """Exact chain rule through attn_core_fwd: with P the softmax and dP = dO V^T,
+    dV = P^T dO,  dS = P * (dP - rowsum(dP * P)),  dQ = dS K / sqrt(d),  dK = dS^T Q / sqrt(d);
+    heads that share a KV group add up in dK and dV."""
+    H = len(head_kv)
+    a = H * d_head
+    dQKV = np.zeros_like(QKV, dtype=np.float64)
+    for b in range(n_seqs):
+        rows = slice(b * seq_len, (b + 1) * seq_len)
+        for hq in range(H):
+            g = int(head_kv[hq])
+            qc = slice(hq * d_head, (hq + 1) * d_head)
+            kc = slice(a + g * d_head, a + (g + 1) * d_head)
+            vc = slice(a + kv_width + g * d_head, a + kv_width + (g + 1) * d_head)
+            Q, K, V, dO = QKV[rows, qc], QKV[rows, kc], QKV[rows, vc], dA[rows, qc]
+            P = _causal_softmax(Q @ K.T / np.sqrt(d_head))
+            dP = dO @ V.T
+            dS = P * (dP - np.sum(dP * P, axis=1, keepdims=True))
+            dQKV[rows, qc] += dS @ K / np.sqrt(d_head)
+            dQKV[rows, kc] += dS.T @ Q / np.sqrt(d_head)
+            dQKV[rows, vc] += P.T @ dO
+    return _q(dQKV, lowp)
+
+
+# ----------------------------------------------------------------------------------------
+# STACK composition: the chained transformer of App. A (Transformer Layer Architecture),
+# without layer normalisation, biases and embeddings (not on this path):
+#   x <- x + alpha_a * Concat(heads) C^attn ;  x <- x + alpha_f * FFN(x)   for every layer,
+# one MSE loss on the final x.  alpha = sqrt(N_full / N_sub) scales each block's output
+# before the residual addition (Sec. 3.4).
+# ----------------------------------------------------------------------------------------
+
+def head_kv_positions(bp, spec, s):
+    """Position of each kept head's KV group among subnet s's kept groups."""
+    per = spec.n_heads // spec.n_kv_heads
+    groups = list(bp["kv_idx"][s][: bp["kv_count"][s]])
+    return np.array([groups.index(h // per) for h in bp["head"][s]], dtype=np.int64)
+
+
+def stack_fwd(spec, layers, head_kv, X0, n_seqs, seq_len, lowp):
+    """layers[l] = compute copies {gate, up, down, qkv, o} of one subnet; head_kv[l] as above.
+    Returns the final x and what the backward pass needs per layer."""
+    alpha_f = act_scale(spec.d_ff // spec.ffn_block, spec.ffn_keep)
+    alpha_a = act_scale(spec.n_heads, spec.head_keep)
+    x, saved = X0, []
+    for l, W in enumerate(layers):
+        kvw = (W["qkv"].shape[0] - W["o"].shape[0]) // 2
+        QKV = qkv_fwd(x, W["qkv"], lowp)
+        A = attn_core_fwd(QKV, n_seqs, seq_len, spec.d_head, head_kv[l], kvw, lowp)
+        x_mid = o_fwd(A, W["o"], alpha_a, lowp, residual=x)
+        x_out, ffn_saved = ffn_fwd(x_mid, W["up"], W.get("gate"), W["down"], spec.ffn_kind, alpha_f, lowp,
+                                   residual=x_mid)
+        saved.append({"x": x, "QKV": QKV, "A": A, "x_mid": x_mid, "ffn": ffn_saved, "kvw": kvw})
+        x = x_out
+    return x, saved
+
+
+def stack_bwd(spec, layers, head_kv, saved, dX, n_seqs, seq_len, lowp):
+    """Gradients of every layer's slices for the loss gradient dX at the output; also returns
+    the gradient with respect to the input.  The gradient of each residual sum flows both
+    through the block and over the skip connection."""
+    alpha_f = act_scale(spec.d_ff // spec.ffn_block, spec.ffn_keep)
+    alpha_a = act_scale(spec.n_heads, spec.head_keep)
+    grads = [None] * len(layers)
+    dx = dX
+    for l in reversed(range(len(layers))):
+        W, sv = layers[l], saved[l]
+        dx_mid, dWu, dWg, dWd = ffn_bwd(dx, sv["x_mid"], sv["ffn"], W["up"], W.get("gate"), W["down"],
+                                        spec.ffn_kind, alpha_f, lowp, residual=dx)
+        dA, dWo = o_bwd(dx_mid, sv["A"], W["o"], alpha_a, lowp)
+        dQKV = attn_core_bwd(dA, sv["QKV"], n_seqs, seq_len, spec.d_head, head_kv[l], sv["kvw"], lowp)
+        dx, dWq = qkv_bwd(dQKV, sv["x"], W["qkv"], lowp, residual=dx_mid)
+        grads[l] = {"up": dWu, "gate": dWg, "down": dWd, "qkv": dWq, "o": dWo}
+    return grads, dx
+
+
+def local_steps_stack(spec, slices, head_kv, get_batch, rnd, s, n_seqs, seq_len, lowp):
+    """K local SGD steps of subnet s through the whole stack (masters `slices[l]`, float64,
+    updated in place).  Batch kinds: 0 input X of width d, 1 target of width d.  Returns the losses."""
+    losses = []
+    for k in range(spec.local_steps):
+        X0 = get_batch(0, rnd, s, k, spec.d_model).astype(np.float64)
+        Tgt = get_batch(1, rnd, s, k, spec.d_model).astype(np.float64)
+        layers = [{m: _q(v, lowp) for m, v in sl.items()} for sl in slices]
+        xL, saved = stack_fwd(spec, layers, head_kv, X0, n_seqs, seq_len, lowp)
+        loss, dX = mse(xL, Tgt, lowp)
+        grads, _ = stack_bwd(spec, layers, head_kv, saved, dX, n_seqs, seq_len, lowp)
+        losses.append(loss)
+        for sl, g in zip(slices, grads):
+            for m in sl:
+                sl[m], _ = sgd(sl[m], g[m], spec.lr, lowp)
+    return losses
+
+
+def round_stack(spec, full, get_batch, rnd, n_seqs, seq_len, lowp):
+    """One full round in STACK composition.  full[l] = dict of the layer's full matrices.
+    Returns (new full weights per layer, blueprints per layer, losses per subnet)."""
+    L = spec.n_layers
+    bps = [layer_blueprints(spec, rnd, l) for l in range(L)]
+    all_slices, losses = [], []
+    for s in range(spec.n_subnets):
+        slices = [{m: np.asarray(v, dtype=np.float64) for m, v in gather_layer(spec, full[l], bps[l], s).items()}
+                  for l in range(L)]
+        head_kv = [head_kv_positions(bps[l], spec, s) for l in range(L)]
+        losses.append(local_steps_stack(spec, slices, head_kv, get_batch, rnd, s, n_seqs, seq_len, lowp))
+        all_slices.append(slices)
+    new = [aggregate_layer(spec, full[l], [all_slices[s][l] for s in range(spec.n_subnets)], bps[l]) for l in range(L)]
+    return new, bps, losses
 
 
 # ----------------------------------------------------------------------------------------
