@@ -198,6 +198,12 @@ typedef struct {
   float* loss;          /* device fp32 [S]: out */
   void* loss_ws;        /* device scratch, at least twist_fused_loss_workspace_bytes(S, T, d) bytes */
   size_t loss_ws_bytes;
+  /* Optional skip connections of the chained transformer layer (App. A, Transformer Layer Architecture:
+   * Y = Y_attnlayer + Y_ffn).  fwd: y = y_residual + out_scale * hh W_down;  bwd: dx = dx_residual + dpre W_gu
+   * (the gradient arriving over the skip connection).  Each sum is rounded once.  NULL: no addend.
+   * Not combinable with the fused loss. */
+  const void* y_residual;   /* device [S][T][d] */
+  const void* dx_residual;  /* device [S][T][d] */
 } twist_ffn_args;
 
 /* Fused loss.  When `tgt` is set, twist_subnet_ffn_fwd / twist_subnet_attn_proj_fwd also evaluate the loss
@@ -234,10 +240,44 @@ typedef struct {
   size_t loss_ws_bytes;
   const int32_t* valid_cols;   /* column mask of twist_mse_fwd_bwd (device int32 [S]) or NULL */
   int32_t seg_begin, seg_width;
+  /* Optional skip connections (App. A: Y_attnlayer = X + Y_attn).  TWIST_PROJ_O fwd: out = out_residual + out_scale * in W;
+   * TWIST_PROJ_QKV bwd: d_in = d_in_residual + d_out W.  NULL: no addend.  Not combinable with the fused loss. */
+  const void* out_residual;    /* device [S][T][d] */
+  const void* d_in_residual;   /* device [S][T][d] */
 } twist_proj_args;
 
 int32_t twist_subnet_attn_proj_fwd(const twist_proj_args* a /*host*/, void* stream);
 int32_t twist_subnet_attn_proj_bwd(const twist_proj_args* a /*host*/, void* stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * Attention core of the kept heads (App. A, Multi-Head Attention: head_h = softmax(Q_h K_h^T / sqrt(d_head)) V_h),
+ * the step between the QKV projection and the output projection in the chained (STACK) composition of
+ * the transformer layer.  Causal within each of the n_seqs sequences of seq_len tokens (T = n_seqs * seq_len).
+ *   qkv    [S][T][a' + 2 kv_max d_head]: Q of the kept heads | K of the kept KV positions | V of the same
+ *   out    [S][T][a'], a' = head_keep * d_head: the concatenated heads
+ *   lse    [S][head_keep][T] fp32: log-sum-exp of each score row (fwd: out; bwd: in)
+ * bwd:  d_qkv [S][T][a' + 2 kv_max d_head] from d_out [S][T][a'] (exact chain rule; the probabilities are recomputed
+ *       from lse); delta [S][head_keep][T] is fp32 scratch.  K/V positions a subnet does not hold
+ *       (kv position >= kv_count[s]) get zero gradient.
+ * Grouped-query sharing (an extension, the paper's attention is plain multi-head): when head_idx is set, kept head hq
+ * of subnet s reads KV position kv_pos[s][head_idx[s][hq] / (n_heads / n_kv_heads)]; heads that share a position add
+ * up in dK and dV.  head_idx == NULL: head hq reads position hq (kv_max must equal head_keep).
+ * dtype TWIST_BF16 only; d_head in {8, 16, 32, 64, 128}.  fp32 arithmetic, deterministic (one writer per result). */
+typedef struct {
+  int32_t dtype, n_subnets, n_seqs, seq_len, head_keep, kv_max, d_head, n_heads, n_kv_heads;
+  const void* qkv;           /* device */
+  void* out;                 /* device  fwd: out, bwd: in */
+  float* lse;                /* device */
+  const void* d_out;         /* device  bwd: in */
+  void* d_qkv;               /* device  bwd: out */
+  float* delta;              /* device  bwd: scratch */
+  const int32_t* head_idx;   /* device int32 [S][head_keep] or NULL */
+  const int32_t* kv_pos;     /* device int32 [S][n_kv_heads] (required with head_idx) */
+  const int32_t* kv_count;   /* device int32 [S] or NULL (every subnet holds kv_max positions) */
+} twist_attn_core_args;
+
+int32_t twist_attn_core_fwd(const twist_attn_core_args* a /*host*/, void* stream);
+int32_t twist_attn_core_bwd(const twist_attn_core_args* a /*host*/, void* stream);
 
 /* ---------------------------------------------------------------------------------------------
  * Loss of the local steps: mean squared error against a target, per subnet, and its gradient.

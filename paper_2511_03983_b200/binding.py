@@ -30,7 +30,7 @@ EXPORTS = [
     "twist_abi_version", "twist_strerror", "twist_last_cuda_error", "twist_device_status", "twist_sample_masks",
     "twist_kv_groups", "twist_gather_subnets", "twist_aggregate", "twist_subnet_ffn_fwd", "twist_subnet_ffn_bwd",
     "twist_subnet_attn_proj_fwd", "twist_subnet_attn_proj_bwd", "twist_mse_workspace_bytes", "twist_mse_fwd_bwd",
-    "twist_mse_fwd_bwd_noalloc", "twist_fused_loss_workspace_bytes",
+    "twist_mse_fwd_bwd_noalloc", "twist_fused_loss_workspace_bytes", "twist_attn_core_fwd", "twist_attn_core_bwd",
 ]
 
 
@@ -60,7 +60,7 @@ class FfnArgs(C.Structure):
                 ("w_down_master", C.c_void_p), ("pre", C.c_void_p), ("hh", C.c_void_p), ("y", C.c_void_p),
                 ("dy", C.c_void_p), ("dpre", C.c_void_p), ("dx", C.c_void_p), ("dw_gu", C.c_void_p),
                 ("dw_down", C.c_void_p), ("tgt", C.c_void_p), ("loss", C.c_void_p), ("loss_ws", C.c_void_p),
-                ("loss_ws_bytes", C.c_size_t)]
+                ("loss_ws_bytes", C.c_size_t), ("y_residual", C.c_void_p), ("dx_residual", C.c_void_p)]
 
 
 class ProjArgs(C.Structure):
@@ -69,7 +69,16 @@ class ProjArgs(C.Structure):
                 ("in_", C.c_void_p), ("w", C.c_void_p), ("w_master", C.c_void_p), ("out", C.c_void_p),
                 ("d_out", C.c_void_p), ("d_in", C.c_void_p), ("dw", C.c_void_p), ("tgt", C.c_void_p),
                 ("loss", C.c_void_p), ("loss_ws", C.c_void_p), ("loss_ws_bytes", C.c_size_t),
-                ("valid_cols", C.c_void_p), ("seg_begin", C.c_int32), ("seg_width", C.c_int32)]
+                ("valid_cols", C.c_void_p), ("seg_begin", C.c_int32), ("seg_width", C.c_int32),
+                ("out_residual", C.c_void_p), ("d_in_residual", C.c_void_p)]
+
+
+class AttnCoreArgs(C.Structure):
+    _fields_ = [("dtype", C.c_int32), ("n_subnets", C.c_int32), ("n_seqs", C.c_int32), ("seq_len", C.c_int32),
+                ("head_keep", C.c_int32), ("kv_max", C.c_int32), ("d_head", C.c_int32), ("n_heads", C.c_int32),
+                ("n_kv_heads", C.c_int32), ("qkv", C.c_void_p), ("out", C.c_void_p), ("lse", C.c_void_p),
+                ("d_out", C.c_void_p), ("d_qkv", C.c_void_p), ("delta", C.c_void_p), ("head_idx", C.c_void_p),
+                ("kv_pos", C.c_void_p), ("kv_count", C.c_void_p)]
 
 
 _lib_handle = None
@@ -96,7 +105,7 @@ def lib() -> C.CDLL:
         h.twist_gather_subnets.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_void_p]
         h.twist_aggregate.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_uint32, C.c_void_p]
         for name in ("twist_subnet_ffn_fwd", "twist_subnet_ffn_bwd", "twist_subnet_attn_proj_fwd",
-                     "twist_subnet_attn_proj_bwd"):
+                     "twist_subnet_attn_proj_bwd", "twist_attn_core_fwd", "twist_attn_core_bwd"):
             getattr(h, name).argtypes = [C.c_void_p, C.c_void_p]
         h.twist_mse_workspace_bytes.restype = C.c_size_t
         h.twist_mse_workspace_bytes.argtypes = [C.c_int32]
@@ -196,10 +205,10 @@ def ffn_args(ffn_kind, dtype, n_subnets, tokens, d_model, f_sub, out_scale, lr=0
     """Marshals twist_ffn_args.  tgt / loss / loss_ws request the fused loss of the forward call."""
     names = ["x", "w_gu", "w_down", "w_gu_master", "w_down_master", "pre", "hh", "y", "dy", "dpre", "dx", "dw_gu",
              "dw_down", "tgt", "loss", "loss_ws"]
-    unknown = set(t) - set(names)
+    unknown = set(t) - set(names) - {"y_residual", "dx_residual"}
     assert not unknown, unknown
     return FfnArgs(ffn_kind, dtype, n_subnets, tokens, d_model, f_sub, out_scale, lr, *[_ptr(t.get(n)) for n in names],
-                   _ws_bytes(t.get("loss_ws")))
+                   _ws_bytes(t.get("loss_ws")), _ptr(t.get("y_residual")), _ptr(t.get("dx_residual")))
 
 
 def twist_subnet_ffn_fwd(a: FfnArgs):
@@ -214,10 +223,11 @@ def proj_args(which, dtype, n_subnets, tokens, d_model, n, out_scale, lr=0.0, se
     """Marshals twist_proj_args.  tgt / loss / loss_ws (and the optional column mask valid_cols,
     seg_begin, seg_width) request the fused loss of the forward call."""
     names = ["in_", "w", "w_master", "out", "d_out", "d_in", "dw", "tgt", "loss", "loss_ws"]
-    unknown = set(t) - set(names) - {"valid_cols"}
+    unknown = set(t) - set(names) - {"valid_cols", "out_residual", "d_in_residual"}
     assert not unknown, unknown
     return ProjArgs(which, dtype, n_subnets, tokens, d_model, n, out_scale, lr, *[_ptr(t.get(n)) for n in names],
-                    _ws_bytes(t.get("loss_ws")), _ptr(t.get("valid_cols")), seg_begin, seg_width)
+                    _ws_bytes(t.get("loss_ws")), _ptr(t.get("valid_cols")), seg_begin, seg_width,
+                    _ptr(t.get("out_residual")), _ptr(t.get("d_in_residual")))
 
 
 def twist_subnet_attn_proj_fwd(a: ProjArgs):
@@ -226,6 +236,23 @@ def twist_subnet_attn_proj_fwd(a: ProjArgs):
 
 def twist_subnet_attn_proj_bwd(a: ProjArgs):
     _check(lib().twist_subnet_attn_proj_bwd(C.byref(a), _stream()), "twist_subnet_attn_proj_bwd")
+
+
+def attn_core_args(dtype, n_subnets, n_seqs, seq_len, head_keep, kv_max, d_head, n_heads=0, n_kv_heads=0,
+                   **t) -> AttnCoreArgs:
+    names = ["qkv", "out", "lse", "d_out", "d_qkv", "delta", "head_idx", "kv_pos", "kv_count"]
+    unknown = set(t) - set(names)
+    assert not unknown, unknown
+    return AttnCoreArgs(dtype, n_subnets, n_seqs, seq_len, head_keep, kv_max, d_head, n_heads, n_kv_heads,
+                        *[_ptr(t.get(n)) for n in names])
+
+
+def twist_attn_core_fwd(a: AttnCoreArgs):
+    _check(lib().twist_attn_core_fwd(C.byref(a), _stream()), "twist_attn_core_fwd")
+
+
+def twist_attn_core_bwd(a: AttnCoreArgs):
+    _check(lib().twist_attn_core_bwd(C.byref(a), _stream()), "twist_attn_core_bwd")
 
 
 def twist_mse_workspace_bytes(n_subnets: int) -> int:

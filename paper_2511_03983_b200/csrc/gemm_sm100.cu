@@ -115,7 +115,8 @@ int make_epilogue_maps(int epi, const GemmParams& p, const CUtensorMap& filler, 
       mk(0, p.in0, N, 2LL * N); mk(1, p.in0 + N, N, 2LL * N);
       mk(2, p.out0, N, 2LL * N); mk(3, p.out0 + N, N, 2LL * N);
       break;
-    case EPI_DACT: mk(0, p.in0, N, N); mk(1, p.out0, N, N); break;
+    case EPI_DACT:
+    case EPI_RESID: mk(0, p.in0, N, N); mk(1, p.out0, N, N); break;
     default: break;                                        // EPI_SGD: plain global accesses
   }
   return rc;
@@ -197,6 +198,7 @@ int launch_gemm_bf16(int layout, int epi, const GemmOperand& A, const GemmOperan
   }
   if (layout == 1 && epi == EPI_STORE) return launch<MAJOR_K, MAJOR_MN, EPI_STORE>(ta, tb, p, st);
   if (layout == 1 && epi == EPI_MSE) return launch<MAJOR_K, MAJOR_MN, EPI_MSE>(ta, tb, p, st);
+  if (layout == 1 && epi == EPI_RESID) return launch<MAJOR_K, MAJOR_MN, EPI_RESID>(ta, tb, p, st);
   if (layout == 2 && epi == EPI_SGD) return launch<MAJOR_MN, MAJOR_MN, EPI_SGD>(ta, tb, p, st);
   return TWIST_ERR_UNSUPPORTED;
 }

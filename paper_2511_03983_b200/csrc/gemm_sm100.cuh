@@ -32,7 +32,7 @@
 namespace twist {
 
 enum { MAJOR_K = 0, MAJOR_MN = 1 };
-enum { EPI_STORE = 0, EPI_SWIGLU_FWD = 1, EPI_ACT_FWD = 2, EPI_DSWIGLU = 3, EPI_DACT = 4, EPI_SGD = 5, EPI_MSE = 6 };
+enum { EPI_STORE = 0, EPI_SWIGLU_FWD = 1, EPI_ACT_FWD = 2, EPI_DSWIGLU = 3, EPI_DACT = 4, EPI_SGD = 5, EPI_MSE = 6, EPI_RESID = 7 };
 
 constexpr int kBM = 256, kBN = 256, kBK = 64, kUmmaK = 16;   // tile of a CTA pair
 constexpr int kCtaM = kBM / 2, kCtaN = kBN / 2;   // rows of A / columns of B that one CTA of the pair loads
@@ -65,7 +65,7 @@ struct GemmParams {
   float scale, lr;
   __nv_bfloat16* out0;  // STORE: D [g][M][N].  *_FWD: pre.  D*: dpre.  SGD: bf16 compute copy of the weights.  MSE: D or null
   __nv_bfloat16* out1;  // *_FWD: hh [g][M][f_sub].  MSE: gradient of the loss w.r.t. D, [g][M][N]
-  const __nv_bfloat16* in0;   // DSWIGLU / DACT: pre.  MSE: target [g][M][N]
+  const __nv_bfloat16* in0;   // DSWIGLU / DACT: pre.  MSE: target [g][M][N].  RESID: addend [g][M][N]
   float* master;        // SGD: fp32 master weights [g][M][N] (updated when lr != 0)
   float* dw;            // SGD: optional fp32 gradient dump [g][M][N].  MSE: partial sums, 8 per tile (2 CTAs x 4 warps)
   const int32_t* valid_cols;   // MSE: valid columns per column group and subnet [groups], or null (all valid)
@@ -77,6 +77,7 @@ struct GemmParams {
 //   STORE: 0 D.            MSE: 0 target (in), 1 dD (out), 2 D (out, optional).
 //   SWIGLU_FWD: 0 G, 1 U (the two halves of pre), 2 hh.        ACT_FWD: 0 pre, 1 hh.
 //   DSWIGLU: 0 G, 1 U (in), 2 dG, 3 dU (out).                  DACT: 0 pre (in), 1 dpre (out).
+//   RESID: 0 addend (in), 1 D (out).
 struct EpiMaps { CUtensorMap m[4]; };
 
 // Boxes per chunk buffer, how many of them are read from global memory first, and buffers per warp.
@@ -84,7 +85,7 @@ __host__ __device__ constexpr int epi_slots(int epi) {
   return epi == EPI_SWIGLU_FWD ? 3 : (epi == EPI_MSE || epi == EPI_ACT_FWD || epi == EPI_DSWIGLU) ? 2 : 1;
 }
 __host__ __device__ constexpr int epi_in_slots(int epi) {
-  return epi == EPI_DSWIGLU ? 2 : (epi == EPI_MSE || epi == EPI_DACT) ? 1 : 0;
+  return epi == EPI_DSWIGLU ? 2 : (epi == EPI_MSE || epi == EPI_DACT || epi == EPI_RESID) ? 1 : 0;
 }
 __host__ __device__ constexpr int epi_bufs(int epi) { return epi_slots(epi) == 3 ? 2 : 4; }
 
@@ -563,6 +564,15 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
               }
               sts128(piece(b0, q), make_uint4(wg[0], wg[1], wg[2], wg[3]));
               sts128(piece(b1, q), make_uint4(wu[0], wu[1], wu[2], wu[3]));
+            } else if constexpr (EPI == EPI_RESID) {   // D = addend + scale * acc, rounded once
+              const uint4 av = lds128(piece(b0, q));
+              const uint32_t aw[4] = {av.x, av.y, av.z, av.w};
+              uint32_t w[4];
+#pragma unroll
+              for (int h = 0; h < 4; ++h)
+                w[h] = pack2(fmaf(p.scale, __uint_as_float(r[2 * h]), bf_lo(aw[h])),
+                             fmaf(p.scale, __uint_as_float(r[2 * h + 1]), bf_hi(aw[h])));
+              sts128(piece(b0, q), make_uint4(w[0], w[1], w[2], w[3]));
             } else {   // EPI_DACT
               const uint4 pv = lds128(piece(b0, q));
               const uint32_t pp[4] = {pv.x, pv.y, pv.z, pv.w};
@@ -595,7 +605,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             } else if constexpr (EPI == EPI_DSWIGLU) {
               tma_store_3d(&tmE.m[2], b0, n, rr, gg);
               tma_store_3d(&tmE.m[3], b1, n, rr, gg);
-            } else {
+            } else {   // DACT, RESID
               tma_store_3d(&tmE.m[1], b0, n, rr, gg);
             }
             bulk_commit();

@@ -77,6 +77,7 @@ extern "C" int32_t twist_subnet_ffn_fwd(const twist_ffn_args* a, void* stream) {
                         nullptr, 0, 0, &fused));
   if (!a->x || !a->w_gu || !a->w_down || !a->pre || !a->hh || (!a->y && !fused)) return TWIST_ERR_NULL;
   if (a->dtype == TWIST_FP32 && !a->y) return TWIST_ERR_NULL;
+  if (a->y_residual && (fused || a->dtype == TWIST_FP32)) return TWIST_ERR_UNSUPPORTED;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const int S = a->n_subnets, T = a->tokens, d = a->d_model, f = a->f_sub;
   const bool swiglu = a->ffn_kind == TWIST_FFN_SWIGLU;
@@ -108,7 +109,9 @@ extern "C" int32_t twist_subnet_ffn_fwd(const twist_ffn_args* a, void* stream) {
     return launch_fused_loss(1, GemmOperand{a->hh, T, f}, GemmOperand{a->w_down, f, d}, q, a->y, a->tgt,
                              const_cast<void*>(a->dy), a->loss, a->loss_ws, nullptr, 0, 0, st);
   q.out0 = static_cast<__nv_bfloat16*>(a->y);
-  return launch_gemm_bf16(1, EPI_STORE, GemmOperand{a->hh, T, f}, GemmOperand{a->w_down, f, d}, q, st);
+  q.in0 = static_cast<const __nv_bfloat16*>(a->y_residual);
+  return launch_gemm_bf16(1, a->y_residual ? EPI_RESID : EPI_STORE, GemmOperand{a->hh, T, f}, GemmOperand{a->w_down, f, d},
+                          q, st);
 }
 
 extern "C" int32_t twist_subnet_ffn_bwd(const twist_ffn_args* a, void* stream) {
@@ -120,6 +123,7 @@ extern "C" int32_t twist_subnet_ffn_bwd(const twist_ffn_args* a, void* stream) {
   const int gf = swiglu ? 2 * f : f;
   if (a->dtype == TWIST_FP32) {
     if (!a->dw_gu || !a->dw_down) return TWIST_ERR_NULL;
+    if (a->dx_residual) return TWIST_ERR_UNSUPPORTED;
     const float* x = static_cast<const float*>(a->x);
     const float* dy = static_cast<const float*>(a->dy);
     const float* pre = static_cast<const float*>(a->pre);
@@ -145,6 +149,7 @@ extern "C" int32_t twist_subnet_ffn_bwd(const twist_ffn_args* a, void* stream) {
     return TWIST_OK;
   }
   if (a->lr != 0.f && (!a->w_gu_master || !a->w_down_master)) return TWIST_ERR_NULL;
+  if (a->dx_residual && !a->dx) return TWIST_ERR_NULL;
   // dpre = act'(pre) * (out_scale * dY W_down^T)
   GemmParams p = base_params(T, f, d, S, a->out_scale);
   p.out0 = static_cast<__nv_bfloat16*>(a->dpre);
@@ -156,7 +161,9 @@ extern "C" int32_t twist_subnet_ffn_bwd(const twist_ffn_args* a, void* stream) {
   if (a->dx) {
     GemmParams q = base_params(T, d, gf, S, 1.f);
     q.out0 = static_cast<__nv_bfloat16*>(a->dx);
-    TWIST_TRY(launch_gemm_bf16(1, EPI_STORE, GemmOperand{a->dpre, T, gf}, GemmOperand{a->w_gu, gf, d}, q, st));
+    q.in0 = static_cast<const __nv_bfloat16*>(a->dx_residual);
+    TWIST_TRY(launch_gemm_bf16(1, a->dx_residual ? EPI_RESID : EPI_STORE, GemmOperand{a->dpre, T, gf},
+                               GemmOperand{a->w_gu, gf, d}, q, st));
   }
   // dW_down = out_scale * hh^T dY, fused SGD
   GemmParams r = base_params(f, d, T, S, a->out_scale);
@@ -192,6 +199,7 @@ extern "C" int32_t twist_subnet_attn_proj_fwd(const twist_proj_args* a, void* st
   TWIST_TRY(check_fused(a->tgt, a->loss, a->d_out, a->loss_ws, a->loss_ws_bytes, S, T, w_out, a->valid_cols,
                         a->seg_begin, a->seg_width, &fused));
   if (!a->in || !a->w || (!a->out && !fused)) return TWIST_ERR_NULL;
+  if (a->out_residual && (fused || qkv || a->dtype == TWIST_FP32)) return TWIST_ERR_UNSUPPORTED;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (a->dtype == TWIST_FP32) {
     if (!a->out) return TWIST_ERR_NULL;
@@ -215,7 +223,8 @@ extern "C" int32_t twist_subnet_attn_proj_fwd(const twist_proj_args* a, void* st
     return launch_fused_loss(layout, A, W, p, a->out, a->tgt, const_cast<void*>(a->d_out), a->loss, a->loss_ws,
                              a->valid_cols, a->seg_begin, a->seg_width, st);
   p.out0 = static_cast<__nv_bfloat16*>(a->out);
-  return launch_gemm_bf16(layout, EPI_STORE, A, W, p, st);
+  p.in0 = static_cast<const __nv_bfloat16*>(a->out_residual);
+  return launch_gemm_bf16(layout, a->out_residual ? EPI_RESID : EPI_STORE, A, W, p, st);
 }
 
 extern "C" int32_t twist_subnet_attn_proj_bwd(const twist_proj_args* a, void* stream) {
@@ -228,6 +237,7 @@ extern "C" int32_t twist_subnet_attn_proj_bwd(const twist_proj_args* a, void* st
   const int w_out = qkv ? n : d;      // width of `d_out`
   if (a->dtype == TWIST_FP32) {
     if (!a->dw) return TWIST_ERR_NULL;
+    if (a->d_in_residual) return TWIST_ERR_UNSUPPORTED;
     const float* in = static_cast<const float*>(a->in);
     const float* dout = static_cast<const float*>(a->d_out);
     float* w = static_cast<float*>(a->w);
@@ -249,11 +259,14 @@ extern "C" int32_t twist_subnet_attn_proj_bwd(const twist_proj_args* a, void* st
     return TWIST_OK;
   }
   if (a->lr != 0.f && !a->w_master) return TWIST_ERR_NULL;
+  if (a->d_in_residual && (!qkv || !a->d_in)) return TWIST_ERR_UNSUPPORTED;
   if (a->d_in) {
     if (qkv) {
       GemmParams p = base_params(T, d, n, S, a->out_scale);
       p.out0 = static_cast<__nv_bfloat16*>(a->d_in);
-      TWIST_TRY(launch_gemm_bf16(1, EPI_STORE, GemmOperand{a->d_out, T, n}, GemmOperand{a->w, n, d}, p, st));
+      p.in0 = static_cast<const __nv_bfloat16*>(a->d_in_residual);
+      TWIST_TRY(launch_gemm_bf16(1, a->d_in_residual ? EPI_RESID : EPI_STORE, GemmOperand{a->d_out, T, n},
+                                 GemmOperand{a->w, n, d}, p, st));
     } else {
       GemmParams p = base_params(T, n, d, S, a->out_scale);
       p.out0 = static_cast<__nv_bfloat16*>(a->d_in);

@@ -279,3 +279,115 @@ class RoundEngine:
         self.sample_masks(rnd)
         for l in range(self.w.n_layers):
             self.run_layer(l)
+
+
+class StackEngine(RoundEngine):
+    """One TwIST round in the chained (STACK) composition: every local step runs all layers,
+    x <- x + alpha_a * O(core(QKV(x))),  x <- x + alpha_f * FFN(x),  with one loss on the final x.
+
+    All layers' slices and saved activations are resident at once (the backward pass needs them), so
+    this engine is for the stack-shaped workloads whose activations fit; the streamed RoundEngine
+    covers the per-block workloads.  Like RoundEngine it only allocates buffers and calls the C ABI.
+    """
+
+    def __init__(self, w: Workload, n_seqs: int, seq_len: int, device: str = "cuda", keep_f32_full: bool = False):
+        assert w.n_heads > 0 and w.dtype == DTYPE_BF16 and n_seqs * seq_len == w.tokens
+        super().__init__(w, device=device, keep_f32_full=keep_f32_full, compute_dx=True, fuse_loss=False)
+        self.n_seqs, self.seq_len = n_seqs, seq_len
+        S, T, d, L = w.n_subnets, w.tokens, w.d_model, w.n_layers
+        gf, f = self.g * w.f_sub, w.f_sub
+        dev, bf = self.dev, torch.bfloat16
+        names = ("w_gu", "w_gu_m", "w_down", "w_down_m", "w_qkv", "w_qkv_m", "w_o", "w_o_m")
+        self.slices = [{n: (getattr(self, n) if l == 0 else torch.empty_like(getattr(self, n))) for n in names}
+                       for l in range(L)]
+        act = lambda width: torch.empty(S, T, width, dtype=bf, device=dev)
+        self.x = [act(d) for _ in range(L + 1)]
+        self.x_mid = [act(d) for _ in range(L)]
+        self.qkv_l = [act(self.nq) for _ in range(L)]
+        self.a_l = [act(self.a_sub) for _ in range(L)]
+        self.pre_l = [act(gf) for _ in range(L)]
+        self.hh_l = [act(f) for _ in range(L)]
+        self.lse = [torch.empty(S, w.head_keep, T, dtype=torch.float32, device=dev) for _ in range(L)]
+        self.delta = torch.empty(S, w.head_keep, T, dtype=torch.float32, device=dev)
+        self.grad = [act(d), act(d)]            # gradient w.r.t. the residual stream (ping-pong)
+        self.stack_loss = torch.zeros(max(1, w.local_steps), S, dtype=torch.float32, device=dev)
+        self.gqa = w.n_kv_heads != w.n_heads
+
+    def _bind(self, l: int):
+        for n, t in self.slices[l].items():
+            setattr(self, n, t)
+
+    def _core_args(self, l: int, **t):
+        w = self.w
+        extra = dict(head_idx=self.idx_head[l], kv_pos=self.kv_pos[l], kv_count=self.kv_count[l]) if self.gqa else {}
+        return B.attn_core_args(w.dtype, w.n_subnets, self.n_seqs, self.seq_len, w.head_keep, self.kv_max, w.d_head,
+                                w.n_heads, w.n_kv_heads, **extra, **t)
+
+    def forward(self, k: int):
+        w = self.w
+        S, T, d = w.n_subnets, w.tokens, w.d_model
+        self.x[0].copy_(self.X[k])
+        for l in range(w.n_layers):
+            self._bind(l)
+            with self._timed("qkv_fwd"):
+                B.twist_subnet_attn_proj_fwd(B.proj_args(B.PROJ_QKV, w.dtype, S, T, d, self.nq, 1.0, 0.0, in_=self.x[l],
+                                                         w=self.w_qkv, out=self.qkv_l[l]))
+            with self._timed("core_fwd"):
+                B.twist_attn_core_fwd(self._core_args(l, qkv=self.qkv_l[l], out=self.a_l[l], lse=self.lse[l]))
+            with self._timed("o_fwd"):
+                B.twist_subnet_attn_proj_fwd(B.proj_args(B.PROJ_O, w.dtype, S, T, d, self.a_sub, self.alpha_a, 0.0,
+                                                         in_=self.a_l[l], w=self.w_o, out=self.x_mid[l],
+                                                         out_residual=self.x[l]))
+            with self._timed("ffn_fwd"):
+                B.twist_subnet_ffn_fwd(B.ffn_args(w.ffn_kind, w.dtype, S, T, d, w.f_sub, self.alpha_f, 0.0,
+                                                  x=self.x_mid[l], w_gu=self.w_gu, w_down=self.w_down, pre=self.pre_l[l],
+                                                  hh=self.hh_l[l], y=self.x[l + 1], y_residual=self.x_mid[l]))
+            self.launches += 5
+
+    def backward(self, k: int, lr: Optional[float] = None):
+        w = self.w
+        lr = w.lr if lr is None else lr
+        S, T, d = w.n_subnets, w.tokens, w.d_model
+        g, g_mid = self.grad
+        for l in reversed(range(w.n_layers)):
+            self._bind(l)
+            with self._timed("ffn_bwd"):
+                B.twist_subnet_ffn_bwd(B.ffn_args(w.ffn_kind, w.dtype, S, T, d, w.f_sub, self.alpha_f, lr,
+                                                  x=self.x_mid[l], w_gu=self.w_gu, w_down=self.w_down,
+                                                  w_gu_master=self.w_gu_m, w_down_master=self.w_down_m,
+                                                  pre=self.pre_l[l], hh=self.hh_l[l], dy=g, dpre=self.dpre, dx=g_mid,
+                                                  dx_residual=g, dw_gu=self.dw_gu, dw_down=self.dw_down))
+            with self._timed("o_bwd"):
+                B.twist_subnet_attn_proj_bwd(B.proj_args(B.PROJ_O, w.dtype, S, T, d, self.a_sub, self.alpha_a, lr,
+                                                         in_=self.a_l[l], w=self.w_o, w_master=self.w_o_m, d_out=g_mid,
+                                                         d_in=self.da, dw=self.dw_o))
+            with self._timed("core_bwd"):
+                B.twist_attn_core_bwd(self._core_args(l, qkv=self.qkv_l[l], out=self.a_l[l], lse=self.lse[l],
+                                                      d_out=self.da, d_qkv=self.dqkv, delta=self.delta))
+            with self._timed("qkv_bwd"):
+                B.twist_subnet_attn_proj_bwd(B.proj_args(B.PROJ_QKV, w.dtype, S, T, d, self.nq, 1.0, lr, in_=self.x[l],
+                                                         w=self.w_qkv, w_master=self.w_qkv_m, d_out=self.dqkv, d_in=g,
+                                                         d_in_residual=g_mid, dw=self.dw_qkv))
+            self.launches += 4 + 2 + 3 + 2
+
+    def local_step(self, k: int, lr: Optional[float] = None):
+        w = self.w
+        self.forward(k)
+        with self._timed("mse"):
+            B.twist_mse_fwd_bwd(self.x[w.n_layers], self.Td[k], self.grad[0], self.stack_loss[k], w.n_subnets, w.tokens,
+                                w.d_model, None, 0, 0, w.dtype, self.ws)
+        self.launches += 2
+        self.backward(k, lr)
+
+    def run_round(self, rnd: int):
+        """Resample, gather every layer, K local steps through the whole stack, aggregate every layer."""
+        w = self.w
+        self.sample_masks(rnd)
+        for l in range(w.n_layers):
+            self._bind(l)
+            self.gather_layer(l)
+        for k in range(w.local_steps):
+            self.local_step(k)
+        for l in range(w.n_layers):
+            self._bind(l)
+            self.aggregate_layer(l)
