@@ -183,6 +183,13 @@ def run_reference(args, w):
 
 
 def workload_config(w, args):
+    if getattr(args, "mode", "blockwise") == "stack":
+        return {"workload": f"configs[{args.config - 1}] {w.name}: STACK round (chained layers, causal attention core, "
+                            f"{w.n_seqs} sequences of {w.tokens // w.n_seqs}), L={w.n_layers} d={w.d_model} F={w.d_ff} "
+                            f"f'={w.f_sub} H'={w.head_keep}/{w.n_heads} S={w.n_subnets} T={w.tokens} K={w.local_steps}",
+                "tokens_per_round": w.tokens_per_round, "mode": "stack, all layers resident",
+                "l2_policy": "working set exceeds L2 across the layers of a round",
+                "parallelism": "replicas only" if args.gpus > 1 else "single GPU"}
     return {"workload": f"configs[{args.config - 1}] {w.name}: BLOCKWISE round, L={w.n_layers} d={w.d_model} "
                         f"F={w.d_ff} f'={w.f_sub} H'={w.head_keep}/{w.n_heads} S={w.n_subnets} T={w.tokens} K={w.local_steps}",
             "tokens_per_round": w.tokens_per_round, "mode": "blockwise, layers streamed",
@@ -201,7 +208,7 @@ def run_ours(args, w):
 
     from paper_2511_03983_b200 import binding as B
     from paper_2511_03983_b200 import inputs as I
-    from paper_2511_03983_b200.engine import RoundEngine
+    from paper_2511_03983_b200.engine import RoundEngine, StackEngine
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -214,7 +221,13 @@ def run_ours(args, w):
     B.lib()
     bf16 = w.dtype == I.DTYPE_BF16
     td = torch.bfloat16 if bf16 else torch.float32
-    eng = RoundEngine(w, keep_f32_full=True, compute_dx=True, fuse_loss=True, store_outputs=False)
+    stack = args.mode == "stack"
+    if stack:
+        if not (w.n_heads and bf16 and w.tokens % w.n_seqs == 0):
+            raise SystemExit("--mode stack needs a bf16 workload with attention heads")
+        eng = StackEngine(w, w.n_seqs, w.tokens // w.n_seqs, keep_f32_full=True)
+    else:
+        eng = RoundEngine(w, keep_f32_full=True, compute_dx=True, fuse_loss=True, store_outputs=False)
     gen = torch.Generator(device="cuda")
     gen.manual_seed(w.seed_w + 7919 * rank)
     for m, v in eng.full.items():                         # weights ~ N(0, 0.02^2), one matrix at a time
@@ -222,7 +235,8 @@ def run_ours(args, w):
             v[l].copy_((torch.randn(v[l].shape, generator=gen, device="cuda", dtype=torch.float32) * 0.02).to(td))
     gen.manual_seed(w.seed_x + 7919 * rank)
     S, T, K = w.n_subnets, w.tokens, w.local_steps
-    widths = [("X", w.d_model), ("Td", w.d_model)] + ([("Tq", eng.nq), ("A", eng.a_sub)] if eng.has_attn else [])
+    widths = [("X", w.d_model), ("Td", w.d_model)] + ([("Tq", eng.nq), ("A", eng.a_sub)]
+                                                      if (eng.has_attn and not stack) else [])
     host = {}
     for name, width in widths:
         lst = getattr(eng, name)
@@ -232,7 +246,8 @@ def run_ours(args, w):
                 t[s].copy_(torch.randn(T, width, generator=gen, device="cuda", dtype=torch.float32).to(td))
             lst.append(t)
     h2d_bytes = sum(t.numel() * t.element_size() for name, _ in widths for t in getattr(eng, name))
-    d2h_bytes = eng.loss.numel() * 4
+    loss_dev = eng.stack_loss if stack else eng.loss
+    d2h_bytes = loss_dev.numel() * 4
 
     def barrier():
         if world > 1:
@@ -279,7 +294,7 @@ def run_ours(args, w):
         pinned = {}
         for name, _ in widths:
             pinned[name] = [t.cpu().pin_memory() for t in getattr(eng, name)]
-        loss_host = torch.empty(eng.loss.shape, dtype=torch.float32).pin_memory()
+        loss_host = torch.empty(loss_dev.shape, dtype=torch.float32).pin_memory()
         n_e2e = max(1, min(args.steps, args.e2e_steps))
         barrier()
         e0.record()
@@ -289,7 +304,7 @@ def run_ours(args, w):
                     dst.copy_(src, non_blocking=True)
             eng.run_round(rnd)
             rnd += 1
-            loss_host.copy_(eng.loss, non_blocking=True)
+            loss_host.copy_(loss_dev, non_blocking=True)
         e1.record()
         barrier()
         t_ms = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device="cuda")
@@ -322,11 +337,14 @@ def run_ours(args, w):
                     "avg_launch_ms": gemm_ms / args.steps / gemm_launches_per_round,
                     "share_of_step": gemm_ms / ms_total}
     hbm = {}
+    # DRAM bytes per launch from the committed ncu capture of one 7B-shaped layer (profiles/); only that launch shape
+    ncu_traffic = {"gather": 3.09e9, "aggregate": 2.79e9} if (args.config == 4 and not stack) else {}
     for name, key in (("gather", "gather_bytes"), ("aggregate", "aggregate_bytes")):
         if name in phases and phases[name][0] > 0:
             gbs = work[key] * args.steps / (phases[name][0] / 1e3) / 1e9
-            hbm[name] = {"achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"],
-                         "bytes_per_launch": work[key] / w.n_layers}
+            hbm[name] = {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                         "frac": gbs / peaks["hbm_gbs"], "bytes_per_launch": work[key] / w.n_layers,
+                         "traffic": ncu_traffic.get(name)}
     if roofline is None and "aggregate" in hbm:
         roofline = dict(bound="hbm", kernel="aggregate_rows_kernel", traffic=None, **hbm["aggregate"])
 
@@ -345,6 +363,69 @@ def run_ours(args, w):
         dist.destroy_process_group()
 
 
+def run_sweep(args):
+    """Workload 5: the gather / aggregate sweep over S x keep on the 7B FFN shapes (IID masks, K=1, 1024 tokens per
+    subnet).  One JSON line whose `cells` give the gather and scatter-average GB/s of every cell."""
+    import torch
+    from dataclasses import replace
+    from paper_2511_03983_b200 import binding as B
+    from paper_2511_03983_b200 import inputs as I
+    from paper_2511_03983_b200.engine import RoundEngine
+
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    B.lib()
+    peaks = measured_peaks()
+    cells = []
+    for w in I.sweep_cfg5():
+        if args.layers:
+            w = replace(w, n_layers=args.layers)
+        eng = RoundEngine(w, keep_f32_full=True, compute_dx=True, fuse_loss=True, store_outputs=False)
+        gen = torch.Generator(device="cuda")
+        gen.manual_seed(w.seed_w)
+        for m, v in eng.full.items():
+            for l in range(w.n_layers):
+                v[l].copy_((torch.randn(v[l].shape, generator=gen, device="cuda", dtype=torch.float32) * 0.02).to(v.dtype))
+        for name in ("X", "Td"):
+            getattr(eng, name).append(torch.randn(w.n_subnets, w.tokens, w.d_model, generator=gen, device="cuda",
+                                                  dtype=torch.float32).to(torch.bfloat16))
+        for r in range(max(1, args.warmup)):
+            eng.run_round(r)
+        torch.cuda.synchronize()
+        eng.timing = True
+        eng.events.clear()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for r in range(args.steps):
+            eng.run_round(100 + r)
+        e1.record()
+        torch.cuda.synchronize()
+        ph = eng.phase_ms()
+        if B.twist_device_status() != 0:
+            raise SystemExit("device status: a bounded device wait expired")
+        kept = w.nmat * w.f_sub * w.d_model                                      # kept elements per subnet and layer
+        covered = int((eng.cover_ffn != 0).sum().item()) * w.ffn_block * w.d_model * w.nmat   # last round, all layers
+        gather_b = 8.0 * kept * w.n_subnets * w.n_layers
+        agg_b = 4.0 * kept * w.n_subnets * w.n_layers + 6.0 * covered
+        g_gbs = gather_b * args.steps / (ph["gather"][0] / 1e3) / 1e9
+        a_gbs = agg_b * args.steps / (ph["aggregate"][0] / 1e3) / 1e9
+        cells.append({"S": w.n_subnets, "keep": round(w.ffn_keep / w.n_ffn_blocks, 2), "gather_gbs": round(g_gbs, 1),
+                      "aggregate_gbs": round(a_gbs, 1), "gather_frac": round(g_gbs / peaks["hbm_gbs"], 3),
+                      "aggregate_frac": round(a_gbs / peaks["hbm_gbs"], 3),
+                      "covered_fraction": round(covered / (w.nmat * w.d_ff * w.d_model * w.n_layers), 4),
+                      "round_ms": round(e0.elapsed_time(e1) / args.steps, 2),
+                      "tokens_per_s": round(w.tokens_per_round / (e0.elapsed_time(e1) / args.steps / 1e3), 1)})
+        del eng
+        torch.cuda.empty_cache()
+    print(json.dumps({"metric": "gather_and_aggregate_gbs", "unit": "GB/s", "peak": peaks["hbm_gbs"],
+                      "peak_source": f"hbm_gbs of {peaks['source']}", "steps": args.steps, "warmup": max(1, args.warmup),
+                      "config": {"workload": "configs[4] gather/aggregate sweep on the 7B FFN shapes: d=4096 F=11008 "
+                                             f"L={args.layers or 32} bf16 weights, fp32 aggregate, IID masks, K=1, "
+                                             "1024 tokens per subnet",
+                                 "bytes": "gather 8 B per kept element (2 read, 2 write, 4 master); aggregate 4 B per "
+                                          "kept master element + 6 B per covered element"},
+                      "cells": cells}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -359,6 +440,9 @@ def main():
     ap.add_argument("--layers", type=int, default=0, help="override the layer count (profiling on a small case)")
     ap.add_argument("--tokens", type=int, default=0, help="override tokens per subnet-step (profiling on a small case)")
     ap.add_argument("--local-steps", type=int, default=0)
+    ap.add_argument("--mode", default="blockwise", choices=["blockwise", "stack"],
+                    help="stack: chained layers with the attention core (workloads 2 and 3)")
+    ap.add_argument("--sweep", action="store_true", help="workload 5: all 12 (S, keep) cells, gather / aggregate GB/s")
     args = ap.parse_args()
     from dataclasses import replace
     from paper_2511_03983_b200 import inputs as I
@@ -371,6 +455,8 @@ def main():
         w = replace(w, local_steps=args.local_steps, name=w.name + f"-K{args.local_steps}")
     if args.impl == "reference":
         run_reference(args, w)
+    elif args.sweep:
+        run_sweep(args)
     else:
         run_ours(args, w)
 

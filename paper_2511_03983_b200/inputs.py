@@ -51,6 +51,7 @@ class Workload:
     seed_mask: int = 3000
     common_ffn: Tuple[int, ...] = field(default_factory=tuple)
     common_heads: Tuple[int, ...] = field(default_factory=tuple)
+    n_seqs: int = 1       # sequences per batch (tokens = n_seqs * sequence length); matters to the attention core only
 
     @property
     def n_ffn_blocks(self) -> int:
@@ -84,14 +85,14 @@ PRESETS: Dict[int, Workload] = {
           rounds=1, dtype=DTYPE_FP32, sample_mode=MODE_COVER, seed_w=1001, seed_x=2001, seed_mask=3001),
     2: _w("cfg2-gpt2-small-gelu-bf16", n_layers=12, d_model=768, n_heads=12, n_kv_heads=12, d_head=64, d_ff=3072,
           ffn_kind=FFN_GELU, n_subnets=4, ffn_keep=1536, head_keep=6, ffn_block=1, tokens=8 * 1024, local_steps=4,
-          rounds=10, dtype=DTYPE_BF16, sample_mode=MODE_COVER, seed_w=1002, seed_x=2002, seed_mask=3002),
+          n_seqs=8, rounds=10, dtype=DTYPE_BF16, sample_mode=MODE_COVER, seed_w=1002, seed_x=2002, seed_mask=3002),
     3: _w("cfg3-tinyllama-swiglu-gqa-bf16", n_layers=22, d_model=2048, n_heads=32, n_kv_heads=4, d_head=64,
           d_ff=5632, ffn_kind=FFN_SWIGLU, n_subnets=4, ffn_keep=2816, head_keep=16, ffn_block=1,
-          tokens=16 * 2048, local_steps=8, rounds=5, dtype=DTYPE_BF16, sample_mode=MODE_COVER,
+          tokens=16 * 2048, local_steps=8, n_seqs=16, rounds=5, dtype=DTYPE_BF16, sample_mode=MODE_COVER,
           seed_w=1003, seed_x=2003, seed_mask=3003),
     4: _w("cfg4-llama7b-swiglu-bf16", n_layers=32, d_model=4096, n_heads=32, n_kv_heads=32, d_head=128,
           d_ff=11008, ffn_kind=FFN_SWIGLU, n_subnets=8, ffn_keep=2752, head_keep=8, ffn_block=1,
-          tokens=8 * 4096, local_steps=4, rounds=3, dtype=DTYPE_BF16, sample_mode=MODE_COVER,
+          tokens=8 * 4096, local_steps=4, n_seqs=8, rounds=3, dtype=DTYPE_BF16, sample_mode=MODE_COVER,
           seed_w=1004, seed_x=2004, seed_mask=3004),
     # config 5 is a sweep over (S, keep); this entry is its S=8, keep=0.25 cell, see sweep_cfg5().
     5: _w("cfg5-7b-ffn-gather-aggregate-sweep", n_layers=32, d_model=4096, n_heads=0, n_kv_heads=0, d_head=0,
