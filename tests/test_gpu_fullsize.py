@@ -190,3 +190,94 @@ def test_aggregate_whole_layer(setup):
         shadow = eng.full[name][0][rows]
         assert torch.equal(shadow[torch.from_numpy(held).cuda()],
                            eng.full_f32[name][0][rows][torch.from_numpy(held).cuda()].to(torch.bfloat16))
+
+
+def test_fused_loss_at_full_size(setup):
+    """The bench's forward call: loss and dY formed in the output epilogue, y not stored.  dY must equal, bit for
+    bit, what the stand-alone loss kernel gives on the stored y; sampled rows of it and the loss match the oracle."""
+    B, eng, w, rows = setup["B"], setup["eng"], setup["w"], setup["rows"]
+    S, T, d, f = w.n_subnets, w.tokens, w.d_model, w.f_sub
+    # earlier tests trained the slices and aggregated into the full model: restore the seeded model and gather again
+    for m, v in setup["full"].items():
+        eng.full[m][0].copy_(torch.from_numpy(v).to(torch.bfloat16))
+    eng.gather_layer(0)
+    common = dict(x=eng.X[0], w_gu=eng.w_gu, w_down=eng.w_down, pre=eng.pre, hh=eng.hh)
+    loss_a = torch.zeros(S, dtype=torch.float32, device="cuda")
+    loss_b = torch.zeros(S, dtype=torch.float32, device="cuda")
+    dy_b = torch.empty_like(eng.dy)
+    B.twist_subnet_ffn_fwd(B.ffn_args(w.ffn_kind, w.dtype, S, T, d, f, eng.alpha_f, 0.0, y=eng.y, **common))
+    B.twist_mse_fwd_bwd(eng.y, eng.Td[0], eng.dy, loss_a, S, T, d, None, 0, 0, w.dtype, eng.ws)
+    B.twist_subnet_ffn_fwd(B.ffn_args(w.ffn_kind, w.dtype, S, T, d, f, eng.alpha_f, 0.0, y=None, dy=dy_b, tgt=eng.Td[0],
+                                      loss=loss_b, loss_ws=eng.ws, **common))
+    torch.cuda.synchronize()
+    assert B.twist_device_status() == 0
+    assert torch.equal(eng.dy, dy_b)
+    assert torch.allclose(loss_a, loss_b, rtol=1e-5, atol=0)
+    r = torch.from_numpy(rows).cuda()
+    for s in SUBNETS:
+        sl = _sl64(setup, s)
+        Yw, _ = o.ffn_fwd(f64(eng.X[0][s][r]), sl["up"], sl["gate"], sl["down"], w.ffn_kind, eng.alpha_f, True)
+        want_dy = o.round_bf16(2.0 * (Yw - f64(eng.Td[0][s][r])) / (T * d))
+        assert rel_fro(f64(dy_b[s][r]), want_dy) < TOL
+        # the reduction: mean squared error over ALL T x d elements, recomputed in fp64 from the stored y
+        diff = eng.y[s].double() - eng.Td[0][s].double()
+        want_loss = float((diff * diff).sum().item()) / (T * d)
+        assert abs(loss_b[s].item() - want_loss) <= 1e-5 * want_loss
+
+
+@pytest.mark.parametrize("cfg", [2, 3])
+def test_attention_core_at_stack_workload_sizes(cfg):
+    """The softmax core at the full sizes of the stack-shaped workloads (8 x 1024 tokens, 6 of 12 heads; 16 x 2048
+    tokens, 16 of 32 heads in 4 KV groups).  The oracle evaluates whole (subnet, sequence) pairs for the heads of a
+    sampled KV position: every output row, dQ, and the dK / dV of that position summed over its heads."""
+    from paper_2511_03983_b200 import binding as B
+    B.lib()
+    w = I.PRESETS[cfg]
+    S, n_seqs, N, H, dh = w.n_subnets, w.n_seqs, w.tokens // w.n_seqs, w.head_keep, w.d_head
+    T = w.tokens
+    bp = o.layer_blueprints(w, 0, 0)
+    gqa = w.n_kv_heads != w.n_heads
+    kv_max = min(w.n_kv_heads, H)
+    a, kvw = H * dh, kv_max * dh
+    nq = a + 2 * kvw
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(77 + cfg)
+    qkv = torch.randn(S, T, nq, generator=gen, device="cuda").to(torch.bfloat16)
+    d_out = torch.randn(S, T, a, generator=gen, device="cuda").to(torch.bfloat16)
+    out = torch.zeros(S, T, a, dtype=torch.bfloat16, device="cuda")
+    d_qkv = torch.zeros(S, T, nq, dtype=torch.bfloat16, device="cuda")
+    lse = torch.zeros(S, H, T, dtype=torch.float32, device="cuda")
+    delta = torch.zeros(S, H, T, dtype=torch.float32, device="cuda")
+    extra = {}
+    if gqa:
+        _, _, kv_pos = o.cover_and_pos(bp["kv_idx"], w.n_kv_heads, counts=bp["kv_count"])
+        extra = dict(head_idx=torch.from_numpy(bp["head"].astype(np.int32)).cuda(),
+                     kv_pos=torch.from_numpy(kv_pos.astype(np.int32)).cuda(),
+                     kv_count=torch.from_numpy(bp["kv_count"].astype(np.int32)).cuda())
+    args = B.attn_core_args(B.BF16, S, n_seqs, N, H, kv_max, dh, w.n_heads, w.n_kv_heads, qkv=qkv, out=out, lse=lse,
+                            d_out=d_out, d_qkv=d_qkv, delta=delta, **extra)
+    B.twist_attn_core_fwd(args)
+    B.twist_attn_core_bwd(args)
+    torch.cuda.synchronize()
+    assert B.twist_device_status() == 0
+    rng = np.random.default_rng(11)
+    for s, b in ((0, 0), (S - 1, n_seqs - 1)):
+        head_kv = o.head_kv_positions(bp, w, s) if gqa else np.arange(H)
+        g = int(rng.choice(np.unique(head_kv)))
+        heads = [hq for hq in range(H) if head_kv[hq] == g]
+        rows = slice(b * N, (b + 1) * N)
+        # a sub-problem with only these heads and this one KV position
+        qcols = np.concatenate([np.arange(hq * dh, (hq + 1) * dh) for hq in heads])
+        kcols = np.arange(a + g * dh, a + (g + 1) * dh)
+        vcols = kcols + kvw
+        Z = f64(qkv[s, rows])[:, np.concatenate([qcols, kcols, vcols])]
+        dA = f64(d_out[s, rows])[:, qcols]
+        hk = [0] * len(heads)
+        want = o.attn_core_fwd(Z, 1, N, dh, hk, dh, True)
+        assert rel_fro(f64(out[s, rows])[:, qcols], want) < TOL
+        dZ = o.attn_core_bwd(dA, Z, 1, N, dh, hk, dh, True)
+        got = f64(d_qkv[s, rows])[:, np.concatenate([qcols, kcols, vcols])]
+        nqh = len(qcols)
+        assert rel_fro(got[:, :nqh], dZ[:, :nqh]) < TOL, "dq"
+        assert rel_fro(got[:, nqh:nqh + dh], dZ[:, nqh:nqh + dh]) < TOL, "dk"
+        assert rel_fro(got[:, nqh + dh:], dZ[:, nqh + dh:]) < TOL, "dv"
