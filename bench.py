@@ -58,6 +58,30 @@ def round_work(w, nq_valid=None):
     return {"gemm_flops": gemm_flops, "gather_bytes": gather_bytes, "aggregate_bytes": agg_bytes}
 
 
+# ------------------------------------------------------------------------------------------------
+# N > 1: independent replicas, one process per GPU (the path has no exchange step between GPUs).
+# ------------------------------------------------------------------------------------------------
+
+def replica_seed(base: int, rank: int) -> int:
+    """Every replica draws its own weights and batches."""
+    return base + 7919 * rank
+
+
+def max_over_ranks(ms_local: float, device="cuda") -> float:
+    """Step time of the job = the slowest replica's (all-reduce MAX when a process group is up)."""
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms_local], dtype=torch.float64, device=device)
+    if dist.is_available() and dist.is_initialized() and dist.get_world_size() > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return t.item()
+
+
+def whole_job_value(tokens_per_round: int, world: int, ms_per_step: float) -> float:
+    """Tokens per second of all replicas together."""
+    return world * tokens_per_round / (ms_per_step / 1e3)
+
+
 class ClockSampler:
     """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
     Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
@@ -229,11 +253,11 @@ def run_ours(args, w):
     else:
         eng = RoundEngine(w, keep_f32_full=True, compute_dx=True, fuse_loss=True, store_outputs=False)
     gen = torch.Generator(device="cuda")
-    gen.manual_seed(w.seed_w + 7919 * rank)
+    gen.manual_seed(replica_seed(w.seed_w, rank))
     for m, v in eng.full.items():                         # weights ~ N(0, 0.02^2), one matrix at a time
         for l in range(w.n_layers):
             v[l].copy_((torch.randn(v[l].shape, generator=gen, device="cuda", dtype=torch.float32) * 0.02).to(td))
-    gen.manual_seed(w.seed_x + 7919 * rank)
+    gen.manual_seed(replica_seed(w.seed_x, rank))
     S, T, K = w.n_subnets, w.tokens, w.local_steps
     widths = [("X", w.d_model), ("Td", w.d_model)] + ([("Tq", eng.nq), ("A", eng.a_sub)]
                                                       if (eng.has_attn and not stack) else [])
@@ -282,11 +306,8 @@ def run_ours(args, w):
     status = B.twist_device_status()
     if status != 0:
         raise SystemExit(f"device status {status}: a bounded device wait expired")
-    t_ms = torch.tensor([ms_total], dtype=torch.float64, device="cuda")
-    if world > 1:
-        dist.all_reduce(t_ms, op=dist.ReduceOp.MAX)
-    ms_per_step = t_ms.item() / args.steps
-    value = world * w.tokens_per_round / (ms_per_step / 1e3)
+    ms_per_step = max_over_ranks(ms_total) / args.steps
+    value = whole_job_value(w.tokens_per_round, world, ms_per_step)
 
     # ---- end-to-end: host buffers, copies inside the timed region --------------------------------
     e2e = None
@@ -307,10 +328,8 @@ def run_ours(args, w):
             loss_host.copy_(loss_dev, non_blocking=True)
         e1.record()
         barrier()
-        t_ms = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device="cuda")
-        if world > 1:
-            dist.all_reduce(t_ms, op=dist.ReduceOp.MAX)
-        e2e = {"value": world * w.tokens_per_round / (t_ms.item() / n_e2e / 1e3), "unit": UNIT,
+        e2e_ms = max_over_ranks(e0.elapsed_time(e1)) / n_e2e
+        e2e = {"value": whole_job_value(w.tokens_per_round, world, e2e_ms), "unit": UNIT,
                "h2d_bytes_per_step": h2d_bytes, "d2h_bytes_per_step": d2h_bytes, "steps": n_e2e,
                "note": "pinned host batches copied in, per-subnet losses copied out, every step"}
 
