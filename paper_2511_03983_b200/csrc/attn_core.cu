@@ -3,12 +3,14 @@
 // head_h = softmax(Q_h K_h^T / sqrt(d_head)) V_h), causal within each sequence, with optional
 // grouped-query sharing of K/V.  Needed by the chained (STACK) composition only.
 //
+// d_head = 64 runs on the tensor cores (attn_core_tc.cu); the kernels in this file serve the other head sizes (and
+// the delta reduction of every size).
 // These are plain fp32 SIMT kernels (bf16 storage, fp32 arithmetic): one group of G threads owns
 // one query (forward, dQ) or one key (dK/dV) with DPT = d_head / G of its dimensions in registers;
 // the other side streams through shared memory in tiles of 64 rows.  The forward keeps a running
 // maximum and sum (one rescale per 8 keys) and stores the log-sum-exp; the backward recomputes
 // the probabilities from it.  Every result has one writer: deterministic, no atomics.
-#include "common.cuh"
+#include "attn_core.cuh"
 
 namespace twist {
 namespace {
@@ -23,21 +25,6 @@ __device__ inline uint32_t pack2(float lo, float hi) {
   __nv_bfloat162 t = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<uint32_t*>(&t);
 }
-
-struct AttnParams {
-  const __nv_bfloat16* qkv;   // [S][T][nq]
-  __nv_bfloat16* out;         // [S][T][a_sub]
-  float* lse;                 // [S][H'][T]   natural-log sum of exp(scores)
-  const __nv_bfloat16* d_out; // [S][T][a_sub]
-  __nv_bfloat16* d_qkv;       // [S][T][nq]
-  float* delta;               // [S][H'][T]   rowsum(dA * A)
-  const int32_t* head_idx;    // [S][H'] kept head ids, or null (no KV sharing: head hq reads KV position hq)
-  const int32_t* kv_pos;      // [S][H_kv] position of a KV group among the subnet's kept groups
-  const int32_t* kv_count;    // [S] kept KV groups, or null (= kv_max)
-  int n_seqs, seq_len, heads, kv_max, d_head, per_group, n_kv_heads;
-  int a_sub, nq, T;
-  float scale_log2;           // log2(e) / sqrt(d_head)
-};
 
 __device__ inline int kv_position(const AttnParams& p, int s, int hq) {
   if (!p.head_idx) return hq;
@@ -350,6 +337,7 @@ int run(const AttnParams& p, int n_subnets, bool backward, cudaStream_t st) {
   const long long n = (long long)n_subnets * p.heads * p.T;
   attn_delta_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(p, n);
   TWIST_LAUNCH_CHECK();
+  if (DPT * G == 64) return attn_bwd_tc(p, n_subnets, st);                         // tensor-core dQ and dK/dV
   attn_dq_kernel<DPT, G><<<grid_q, kAttnThreads, 0, st>>>(p);
   TWIST_LAUNCH_CHECK();
   const dim3 grid_k(grid_q.x, p.kv_max, grid_q.z);
@@ -363,7 +351,9 @@ int dispatch(const AttnParams& p, int n_subnets, bool backward, cudaStream_t st)
     case 8: return run<8, 1>(p, n_subnets, backward, st);
     case 16: return run<16, 1>(p, n_subnets, backward, st);
     case 32: return run<32, 1>(p, n_subnets, backward, st);
-    case 64: return run<32, 2>(p, n_subnets, backward, st);
+    case 64:
+      if (!backward) return attn_fwd_tc(p, n_subnets, st);                          // tensor-core forward
+      return run<32, 2>(p, n_subnets, backward, st);
     case 128: return run<32, 4>(p, n_subnets, backward, st);
     default: return TWIST_ERR_UNSUPPORTED;
   }

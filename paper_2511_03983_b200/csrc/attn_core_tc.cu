@@ -1,0 +1,658 @@
+// Tensor-core forward of the attention core (App. A: head_h = softmax(Q_h K_h^T / sqrt(d_head)) V_h, causal per
+// sequence) for d_head = 64, on tcgen05 with accumulators in tensor memory.
+//
+// One CTA per (block of 128 queries, kept head, sequence).  Per block of 128 keys:
+//   S = Q K^T        one 128 x 128 x 64 MMA chain, Q and K tiles brought by TMA (K-major, 128-byte swizzle)
+//   softmax          thread = query row: the row of S is read from tensor memory twice (maximum, then
+//                    exponentials), running maximum / sum kept in registers, P written to shared memory as the
+//                    bf16 A operand of the next MMA
+//   O_blk = P V      128 x 64 x 128 MMA chain, V as the MN-major B operand (rows = keys as they lie in memory)
+//   O = O * corr + O_blk in registers (64 fp32 per thread), so tensor memory never needs rescaling.
+// The MMA of the next block's S is issued as soon as P of the current block is consumed, so it overlaps the
+// threads' accumulation of O.  Warps 0-3: softmax / output; warp 4, one lane: TMA and MMA issue.
+// Backward (same tile sizes; probabilities recomputed from the stored log-sum-exp, dS = P (dP - delta)):
+//   dQ kernel     one CTA per query block: per key block S = Q K^T and dP = dO V^T into tensor memory, the threads
+//                 write dS (bf16) to shared memory, dQ += dS K accumulates in tensor memory over the key blocks.
+//   dK/dV kernel  one CTA per (key block, KV position): for every kept head that reads the position and every
+//                 query block at or after the key block, S and dP as above, the threads write P and dS, and
+//                 dV += P^T dO, dK += dS^T Q accumulate in tensor memory (P and dS are read as MN-major A
+//                 operands: the same bytes, no transpose).
+// Every wait is bounded; on expiry the CTA records TWIST_ERR_DEVICE_TIMEOUT and leaves.
+#include "attn_core.cuh"
+#include "ptx.cuh"
+
+namespace twist {
+namespace {
+
+constexpr int kDh = 64;                 // head dimension of this kernel
+constexpr int kBq = 128, kBk = 128;     // queries per CTA, keys per block
+constexpr int kTileBytes = 128 * kDh * 2;            // a 128-row tile of Q, K or V: 16 KB
+constexpr int kPBytes = kBq * kBk * 2;               // P: 32 KB (two 64-key halves of 16 KB)
+constexpr int kFwdThreads = 160;
+constexpr int kFwdSmem = kTileBytes * 5 + kPBytes + 1024 + 128;   // Q, K[2], V[2], P, alignment, barriers
+constexpr int kFwdTmemCols = 256;       // S: columns 0..127, O_blk: columns 128..191
+
+__device__ inline void mma1(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ inline void commit1(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// fp32 accumulate, bf16 x bf16, M x N tile, operand majors (0: K-major, 1: MN-major)
+__host__ __device__ constexpr uint32_t idesc_bf16(int a_major, int b_major, int M, int N) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)a_major << 15) | ((uint32_t)b_major << 16) |
+         ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+}
+__device__ inline uint32_t pack2(float lo, float hi) {
+  __nv_bfloat162 t = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&t);
+}
+__device__ inline int kv_position(const AttnParams& p, int s, int hq) {
+  if (!p.head_idx) return hq;
+  const int g = p.head_idx[(long long)s * p.heads + hq] / p.per_group;
+  return p.kv_pos[(long long)s * p.n_kv_heads + g];
+}
+
+// qkv viewed as [S * n_seqs][seq_len][nq]: rows past the end of a sequence read as zeros.
+__global__ void __launch_bounds__(kFwdThreads) attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQKV,
+                                                                  const AttnParams p, int* status) {
+  extern __shared__ unsigned char smem_raw[];
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  unsigned char* gen = smem_raw + (base - smem_u32(smem_raw));
+  const uint32_t q_s = base, k_s = base + kTileBytes, v_s = base + 3 * kTileBytes, p_s = base + 5 * kTileBytes;
+  const uint32_t bar0 = p_s + kPBytes;
+  volatile uint32_t* ctrl = reinterpret_cast<volatile uint32_t*>(gen + 5 * kTileBytes + kPBytes);
+  // barriers (8 bytes each): 0 q_full, 1-2 kv_full, 3-4 kv_free, 5 s_full, 6 p_ready, 7 o_full; then TMEM base, abort flag
+  auto bar = [&](int i) { return bar0 + 8u * i; };
+  volatile uint32_t* tmem_slot = ctrl + 16;
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(ctrl + 17);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int qb = blockIdx.x, hq = blockIdx.y, s = blockIdx.z / p.n_seqs, b = blockIdx.z - s * p.n_seqs;
+  const int nblk = qb + 1;                               // causal: key blocks 0 .. qb
+  if (threadIdx.x == 128) {
+    tma_prefetch_desc(&tmQKV);
+    for (int i = 0; i < 8; ++i) mbar_init(bar(i), i == 6 ? 128 : 1);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    fence_async_smem();
+  }
+  if (warp == 4) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                 ::"r"(smem_u32(const_cast<uint32_t*>(tmem_slot))), "r"((uint32_t)kFwdTmemCols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tmem_slot;
+  const uint32_t tm_s = tmem, tm_o = tmem + 128;
+
+  if (warp == 4) {
+    if (lane == 0) {
+      const int kvp = kv_position(p, s, hq);
+      const int z = blockIdx.z;
+      const int k_col = p.a_sub + kvp * kDh, v_col = k_col + p.kv_max * kDh;
+      auto load_kv = [&](int j) {
+        const int st = j & 1;
+        mbar_expect_tx(bar(1 + st), 2 * kTileBytes);
+        tma_load_3d_local(k_s + st * kTileBytes, &tmQKV, bar(1 + st), k_col, j * kBk, z);
+        tma_load_3d_local(v_s + st * kTileBytes, &tmQKV, bar(1 + st), v_col, j * kBk, z);
+      };
+      mbar_expect_tx(bar(0), kTileBytes);
+      tma_load_3d_local(q_s, &tmQKV, bar(0), hq * kDh, qb * kBq, z);
+      load_kv(0);
+      if (nblk > 1) load_kv(1);
+      constexpr uint32_t idesc_s = idesc_bf16(0, 0, kBq, kBk);       // S = Q K^T : both K-major
+      constexpr uint32_t idesc_o = idesc_bf16(0, 1, kBq, kDh);       // O = P V   : V MN-major
+      auto mma_s = [&](int j) {
+        const uint64_t a = smem_desc(q_s, 16u, 1024u), bd = smem_desc(k_s + (j & 1) * kTileBytes, 16u, 1024u);
+#pragma unroll
+        for (int k = 0; k < kDh / 16; ++k) mma1(tm_s, a + 2u * k, bd + 2u * k, idesc_s, k != 0);
+        commit1(bar(5));
+      };
+      bool ok = mbar_wait(bar(0), 0, abort_flag, status) && mbar_wait(bar(1), 0, abort_flag, status);
+      if (ok) {
+        tc_fence_after();
+        mma_s(0);
+      }
+      for (int j = 0; ok && j < nblk; ++j) {
+        const int st = j & 1;
+        if (!mbar_wait(bar(6), j & 1, abort_flag, status)) break;                 // P of block j is in shared memory
+        tc_fence_after();
+        const uint64_t bd = smem_desc(v_s + st * kTileBytes, (uint32_t)kDh * 128u, 1024u);
+#pragma unroll
+        for (int k = 0; k < kBk / 16; ++k) {
+          const uint64_t a = smem_desc(p_s + (k >> 2) * (kPBytes / 2), 16u, 1024u) + 2u * (k & 3);
+          mma1(tm_o, a, bd + (uint64_t)((k * 16 * 128) >> 4), idesc_o, k != 0);
+        }
+        commit1(bar(7));                                                          // O_blk complete
+        commit1(bar(3 + st));                                                     // K/V stage free
+        if (j + 1 < nblk) {
+          if (!mbar_wait(bar(1 + ((j + 1) & 1)), ((j + 1) >> 1) & 1, abort_flag, status)) break;
+          tc_fence_after();
+          mma_s(j + 1);                                                           // overlaps the threads' work on O
+        }
+        if (j + 2 < nblk) {
+          if (!mbar_wait(bar(3 + st), (j >> 1) & 1, abort_flag, status)) break;
+          load_kv(j + 2);
+        }
+      }
+    }
+  } else {
+    // ---- softmax warps: thread = query row
+    const int r = warp * 32 + lane;
+    const int qi = qb * kBq + r;
+    const uint32_t t_s = tm_s + ((uint32_t)(warp * 32) << 16), t_o = tm_o + ((uint32_t)(warp * 32) << 16);
+    // 16-byte piece c (0..7) of this row inside a 64-key half of P (128-byte rows, 128-byte swizzle)
+    const uint32_t p_row = p_s + (uint32_t)(r >> 3) * 1024u + (uint32_t)(r & 7) * 128u;
+    const uint32_t sw = (uint32_t)(r & 7);
+    float o[kDh];
+#pragma unroll
+    for (int i = 0; i < kDh; ++i) o[i] = 0.f;
+    float m = -INFINITY, l = 0.f;
+    bool ok = true;
+    for (int j = 0; j < nblk; ++j) {
+      if (!__all_sync(0xffffffffu, mbar_wait(bar(5), j & 1, abort_flag, status))) { ok = false; break; }
+      tc_fence_after();
+      const int k_lim = (j == qb) ? qi - j * kBk : kBk;                           // columns <= k_lim are visible
+      // pass 1: row maximum (scores scaled into the log2 domain)
+      float mx = -INFINITY;
+#pragma unroll
+      for (int c = 0; c < kBk / 32; ++c) {
+        uint32_t v[32];
+        tc_ld32(t_s + 32 * c, v);
+        tc_wait_ld();
+#pragma unroll
+        for (int i = 0; i < 32; ++i)
+          if (32 * c + i <= k_lim) mx = fmaxf(mx, __uint_as_float(v[i]));
+      }
+      const float m_new = fmaxf(m, mx * p.scale_log2);
+      const float corr = exp2f(m - m_new);
+      l *= corr;
+      // pass 2: exponentials -> P (bf16) in shared memory, row sum
+#pragma unroll
+      for (int c = 0; c < kBk / 32; ++c) {
+        uint32_t v[32];
+        tc_ld32(t_s + 32 * c, v);
+        tc_wait_ld();
+        uint32_t w[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+          const float p0 = (32 * c + 2 * i <= k_lim) ? exp2f(fmaf(__uint_as_float(v[2 * i]), p.scale_log2, -m_new)) : 0.f;
+          const float p1 = (32 * c + 2 * i + 1 <= k_lim) ? exp2f(fmaf(__uint_as_float(v[2 * i + 1]), p.scale_log2, -m_new)) : 0.f;
+          l += p0 + p1;
+          w[i] = pack2(p0, p1);
+        }
+        const uint32_t half = p_row + (uint32_t)(c >> 1) * (kPBytes / 2);
+#pragma unroll
+        for (int q4 = 0; q4 < 4; ++q4) {
+          const uint32_t piece = (uint32_t)((c & 1) * 4 + q4);
+          sts128(half + ((piece ^ sw) << 4), make_uint4(w[4 * q4], w[4 * q4 + 1], w[4 * q4 + 2], w[4 * q4 + 3]));
+        }
+      }
+      fence_async_smem();                                                         // P: generic writes -> MMA reads
+      tc_fence_before();
+      mbar_arrive(bar(6));
+      if (!__all_sync(0xffffffffu, mbar_wait(bar(7), j & 1, abort_flag, status))) { ok = false; break; }
+      tc_fence_after();
+#pragma unroll
+      for (int c = 0; c < kDh / 32; ++c) {
+        uint32_t v[32];
+        tc_ld32(t_o + 32 * c, v);
+        tc_wait_ld();
+#pragma unroll
+        for (int i = 0; i < 32; ++i) o[32 * c + i] = fmaf(o[32 * c + i], corr, __uint_as_float(v[i]));
+      }
+      m = m_new;
+    }
+    if (ok && qi < p.seq_len) {
+      const float inv = 1.f / l;
+      const long long row = (long long)s * p.T + (long long)b * p.seq_len + qi;
+      uint4* dst = reinterpret_cast<uint4*>(p.out + row * p.a_sub + hq * kDh);
+#pragma unroll
+      for (int c = 0; c < kDh / 8; ++c)
+        dst[c] = make_uint4(pack2(o[8 * c] * inv, o[8 * c + 1] * inv), pack2(o[8 * c + 2] * inv, o[8 * c + 3] * inv),
+                            pack2(o[8 * c + 4] * inv, o[8 * c + 5] * inv), pack2(o[8 * c + 6] * inv, o[8 * c + 7] * inv));
+      p.lse[((long long)s * p.heads + hq) * p.T + (long long)b * p.seq_len + qi] = (m + log2f(l)) * 0.6931471805599453f;
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (*abort_flag) {     // a wait expired: let copies that may still be in flight land before shared memory is released
+    const uint64_t t0 = global_timer_ns();
+    while (global_timer_ns() - t0 < 2000000ull) __nanosleep(1000);
+    __syncthreads();
+  }
+  if (warp == 4) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"((uint32_t)kFwdTmemCols) : "memory");
+  }
+}
+
+// 16-byte pieces of row r of a [128 rows][2 x 64 columns] bf16 operand tile (two halves of 16 KB, 128-byte rows,
+// 128-byte swizzle): the layout of P and dS, readable as a K-major A operand (rows = M) or an MN-major one (rows = K).
+__device__ inline void store_row_chunk32(uint32_t tile, int r, int c, const uint32_t (&w)[16]) {
+  const uint32_t half = tile + (uint32_t)(c >> 1) * (kPBytes / 2) + (uint32_t)(r >> 3) * 1024u + (uint32_t)(r & 7) * 128u;
+  const uint32_t sw = (uint32_t)(r & 7);
+#pragma unroll
+  for (int q4 = 0; q4 < 4; ++q4) {
+    const uint32_t piece = (uint32_t)((c & 1) * 4 + q4);
+    sts128(half + ((piece ^ sw) << 4), make_uint4(w[4 * q4], w[4 * q4 + 1], w[4 * q4 + 2], w[4 * q4 + 3]));
+  }
+}
+
+constexpr int kBwdTmemCols = 512;
+constexpr int kDqSmem = kTileBytes * 6 + kPBytes + 1024 + 128;        // Q, dO, K[2], V[2], dS
+constexpr int kDkvSmem = kTileBytes * 6 + 2 * kPBytes + 1024 + 256;   // K, V, Q[2], dO[2], P, dS
+
+// ---- dQ: grid (query blocks, kept heads, S * n_seqs)
+__global__ void __launch_bounds__(kFwdThreads) attn_dq_tc_kernel(const __grid_constant__ CUtensorMap tmQKV,
+                                                                 const __grid_constant__ CUtensorMap tmDO,
+                                                                 const AttnParams p, int* status) {
+  extern __shared__ unsigned char smem_raw[];
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  unsigned char* gen = smem_raw + (base - smem_u32(smem_raw));
+  const uint32_t q_s = base, do_s = base + kTileBytes, k_s = base + 2 * kTileBytes, v_s = base + 4 * kTileBytes,
+                 ds_s = base + 6 * kTileBytes;
+  const uint32_t bar0 = ds_s + kPBytes;
+  volatile uint32_t* ctrl = reinterpret_cast<volatile uint32_t*>(gen + 6 * kTileBytes + kPBytes);
+  // barriers: 0 q_full, 1-2 kv_full, 3-4 kv_free, 5 sdp_full, 6 ds_ready, 7 dq_full
+  auto bar = [&](int i) { return bar0 + 8u * i; };
+  volatile uint32_t* tmem_slot = ctrl + 16;
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(ctrl + 17);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int qb = blockIdx.x, hq = blockIdx.y, s = blockIdx.z / p.n_seqs, b = blockIdx.z - s * p.n_seqs;
+  const int nblk = qb + 1;
+  if (threadIdx.x == 128) {
+    tma_prefetch_desc(&tmQKV);
+    tma_prefetch_desc(&tmDO);
+    for (int i = 0; i < 8; ++i) mbar_init(bar(i), i == 6 ? 128 : 1);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    fence_async_smem();
+  }
+  if (warp == 4) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                 ::"r"(smem_u32(const_cast<uint32_t*>(tmem_slot))), "r"((uint32_t)kBwdTmemCols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tmem_slot;
+  const uint32_t tm_s = tmem, tm_dp = tmem + 128, tm_dq = tmem + 256;
+
+  if (warp == 4) {
+    if (lane == 0) {
+      const int kvp = kv_position(p, s, hq);
+      const int z = blockIdx.z;
+      const int k_col = p.a_sub + kvp * kDh, v_col = k_col + p.kv_max * kDh;
+      auto load_kv = [&](int j) {
+        const int st = j & 1;
+        mbar_expect_tx(bar(1 + st), 2 * kTileBytes);
+        tma_load_3d_local(k_s + st * kTileBytes, &tmQKV, bar(1 + st), k_col, j * kBk, z);
+        tma_load_3d_local(v_s + st * kTileBytes, &tmQKV, bar(1 + st), v_col, j * kBk, z);
+      };
+      mbar_expect_tx(bar(0), 2 * kTileBytes);
+      tma_load_3d_local(q_s, &tmQKV, bar(0), hq * kDh, qb * kBq, z);
+      tma_load_3d_local(do_s, &tmDO, bar(0), hq * kDh, qb * kBq, z);
+      load_kv(0);
+      if (nblk > 1) load_kv(1);
+      constexpr uint32_t idesc_s = idesc_bf16(0, 0, kBq, kBk);       // S = Q K^T, dP = dO V^T : both K-major
+      constexpr uint32_t idesc_q = idesc_bf16(0, 1, kBq, kDh);       // dQ = dS K : K as the MN-major B operand
+      auto mma_sdp = [&](int j) {
+        const uint64_t aq = smem_desc(q_s, 16u, 1024u), ao = smem_desc(do_s, 16u, 1024u);
+        const uint64_t bk = smem_desc(k_s + (j & 1) * kTileBytes, 16u, 1024u), bv = smem_desc(v_s + (j & 1) * kTileBytes, 16u, 1024u);
+#pragma unroll
+        for (int k = 0; k < kDh / 16; ++k) mma1(tm_s, aq + 2u * k, bk + 2u * k, idesc_s, k != 0);
+#pragma unroll
+        for (int k = 0; k < kDh / 16; ++k) mma1(tm_dp, ao + 2u * k, bv + 2u * k, idesc_s, k != 0);
+        commit1(bar(5));
+      };
+      bool ok = mbar_wait(bar(0), 0, abort_flag, status) && mbar_wait(bar(1), 0, abort_flag, status);
+      if (ok) {
+        tc_fence_after();
+        mma_sdp(0);
+      }
+      for (int j = 0; ok && j < nblk; ++j) {
+        const int st = j & 1;
+        if (!mbar_wait(bar(6), j & 1, abort_flag, status)) break;                 // dS of block j is in shared memory
+        tc_fence_after();
+        const uint64_t bd = smem_desc(k_s + st * kTileBytes, (uint32_t)kDh * 128u, 1024u);
+#pragma unroll
+        for (int k = 0; k < kBk / 16; ++k) {
+          const uint64_t a = smem_desc(ds_s + (k >> 2) * (kPBytes / 2), 16u, 1024u) + 2u * (k & 3);
+          mma1(tm_dq, a, bd + (uint64_t)((k * 16 * 128) >> 4), idesc_q, (j | k) != 0);
+        }
+        commit1(bar(3 + st));
+        if (j + 1 == nblk) commit1(bar(7));
+        if (j + 1 < nblk) {
+          if (!mbar_wait(bar(1 + ((j + 1) & 1)), ((j + 1) >> 1) & 1, abort_flag, status)) break;
+          tc_fence_after();
+          mma_sdp(j + 1);
+        }
+        if (j + 2 < nblk) {
+          if (!mbar_wait(bar(3 + st), (j >> 1) & 1, abort_flag, status)) break;
+          load_kv(j + 2);
+        }
+      }
+    }
+  } else {
+    const int r = warp * 32 + lane;
+    const int qi = qb * kBq + r;
+    const bool row_ok = qi < p.seq_len;
+    const uint32_t lane_off = (uint32_t)(warp * 32) << 16;
+    const long long stat = ((long long)s * p.heads + hq) * p.T + (long long)b * p.seq_len + qi;
+    const float lse2 = row_ok ? p.lse[stat] * 1.4426950408889634f : 0.f;
+    const float dl = row_ok ? p.delta[stat] : 0.f;
+    bool ok = true;
+    for (int j = 0; j < nblk; ++j) {
+      if (!__all_sync(0xffffffffu, mbar_wait(bar(5), j & 1, abort_flag, status))) { ok = false; break; }
+      tc_fence_after();
+      const int k_lim = !row_ok ? -1 : ((j == qb) ? qi - j * kBk : kBk);
+#pragma unroll
+      for (int c = 0; c < kBk / 32; ++c) {
+        uint32_t vs[32], vd[32];
+        tc_ld32(tm_s + lane_off + 32 * c, vs);
+        tc_ld32(tm_dp + lane_off + 32 * c, vd);
+        tc_wait_ld();
+        uint32_t w[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+          float d2[2];
+#pragma unroll
+          for (int e = 0; e < 2; ++e) {
+            const int col = 32 * c + 2 * i + e;
+            const float pr = col <= k_lim ? exp2f(fmaf(__uint_as_float(vs[2 * i + e]), p.scale_log2, -lse2)) : 0.f;
+            d2[e] = pr * (__uint_as_float(vd[2 * i + e]) - dl);
+          }
+          w[i] = pack2(d2[0], d2[1]);
+        }
+        store_row_chunk32(ds_s, r, c, w);
+      }
+      fence_async_smem();
+      tc_fence_before();
+      mbar_arrive(bar(6));
+    }
+    if (ok && __all_sync(0xffffffffu, mbar_wait(bar(7), 0, abort_flag, status))) {
+      tc_fence_after();
+      const float sc = p.scale_log2 * 0.6931471805599453f;                         // 1 / sqrt(d_head)
+      const long long row = (long long)s * p.T + (long long)b * p.seq_len + qi;
+      uint4* dst = reinterpret_cast<uint4*>(p.d_qkv + row * p.nq + hq * kDh);
+#pragma unroll
+      for (int c = 0; c < kDh / 32; ++c) {
+        uint32_t v[32];
+        tc_ld32(tm_dq + lane_off + 32 * c, v);
+        tc_wait_ld();
+        if (row_ok) {
+#pragma unroll
+          for (int q4 = 0; q4 < 4; ++q4)
+            dst[4 * c + q4] = make_uint4(pack2(sc * __uint_as_float(v[8 * q4]), sc * __uint_as_float(v[8 * q4 + 1])),
+                                         pack2(sc * __uint_as_float(v[8 * q4 + 2]), sc * __uint_as_float(v[8 * q4 + 3])),
+                                         pack2(sc * __uint_as_float(v[8 * q4 + 4]), sc * __uint_as_float(v[8 * q4 + 5])),
+                                         pack2(sc * __uint_as_float(v[8 * q4 + 6]), sc * __uint_as_float(v[8 * q4 + 7])));
+        }
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (*abort_flag) {
+    const uint64_t t0 = global_timer_ns();
+    while (global_timer_ns() - t0 < 2000000ull) __nanosleep(1000);
+    __syncthreads();
+  }
+  if (warp == 4) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"((uint32_t)kBwdTmemCols) : "memory");
+  }
+}
+
+// ---- dK, dV: grid (key blocks, KV positions, S * n_seqs)
+__global__ void __launch_bounds__(kFwdThreads) attn_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmQKV,
+                                                                  const __grid_constant__ CUtensorMap tmDO,
+                                                                  const AttnParams p, int* status) {
+  extern __shared__ unsigned char smem_raw[];
+  __shared__ int match[64];
+  __shared__ int n_match_s;
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  unsigned char* gen = smem_raw + (base - smem_u32(smem_raw));
+  const uint32_t k_s = base, v_s = base + kTileBytes, q_s = base + 2 * kTileBytes, do_s = base + 4 * kTileBytes,
+                 p_s = base + 6 * kTileBytes, ds_s = p_s + kPBytes;
+  const uint32_t bar0 = ds_s + kPBytes;
+  volatile uint32_t* ctrl = reinterpret_cast<volatile uint32_t*>(gen + 6 * kTileBytes + 2 * kPBytes);
+  // barriers: 0 kv_full, 1-2 q_full, 3-4 q_free, 5 sdp_full, 6 pds_ready, 7 acc_full
+  auto bar = [&](int i) { return bar0 + 8u * i; };
+  volatile uint32_t* tmem_slot = ctrl + 16;
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(ctrl + 17);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int kb = blockIdx.x, kvp = blockIdx.y, s = blockIdx.z / p.n_seqs, b = blockIdx.z - s * p.n_seqs;
+  const int nqb = (p.seq_len + kBq - 1) / kBq;
+  const int held = p.kv_count ? p.kv_count[s] : p.kv_max;
+  if (threadIdx.x == 128) {
+    tma_prefetch_desc(&tmQKV);
+    tma_prefetch_desc(&tmDO);
+    for (int i = 0; i < 8; ++i) mbar_init(bar(i), i == 6 ? 128 : 1);
+    *abort_flag = 0;
+    int n = 0;
+    if (kvp < held)
+      for (int hq = 0; hq < p.heads && n < 64; ++hq)
+        if (kv_position(p, s, hq) == kvp) match[n++] = hq;
+    n_match_s = n;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    fence_async_smem();
+  }
+  if (warp == 4) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                 ::"r"(smem_u32(const_cast<uint32_t*>(tmem_slot))), "r"((uint32_t)kBwdTmemCols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tmem_slot;
+  const uint32_t tm_s = tmem, tm_dp = tmem + 128, tm_dv = tmem + 256, tm_dk = tmem + 320;
+  const int per_head = nqb - kb;                         // query blocks kb .. nqb-1
+  const int total = n_match_s * per_head;                // units (head, query block)
+
+  if (warp == 4) {
+    if (lane == 0 && total > 0) {
+      const int z = blockIdx.z;
+      auto load_q = [&](int n) {
+        const int st = n & 1, hq = match[n / per_head], i = kb + n % per_head;
+        mbar_expect_tx(bar(1 + st), 2 * kTileBytes);
+        tma_load_3d_local(q_s + st * kTileBytes, &tmQKV, bar(1 + st), hq * kDh, i * kBq, z);
+        tma_load_3d_local(do_s + st * kTileBytes, &tmDO, bar(1 + st), hq * kDh, i * kBq, z);
+      };
+      mbar_expect_tx(bar(0), 2 * kTileBytes);
+      tma_load_3d_local(k_s, &tmQKV, bar(0), p.a_sub + kvp * kDh, kb * kBk, z);
+      tma_load_3d_local(v_s, &tmQKV, bar(0), p.a_sub + (p.kv_max + kvp) * kDh, kb * kBk, z);
+      load_q(0);
+      if (total > 1) load_q(1);
+      constexpr uint32_t idesc_s = idesc_bf16(0, 0, kBq, kBk);       // S = Q K^T, dP = dO V^T
+      constexpr uint32_t idesc_t = idesc_bf16(1, 1, kBk, kDh);       // dV = P^T dO, dK = dS^T Q : both MN-major
+      auto mma_sdp = [&](int n) {
+        const int st = n & 1;
+        const uint64_t aq = smem_desc(q_s + st * kTileBytes, 16u, 1024u), ao = smem_desc(do_s + st * kTileBytes, 16u, 1024u);
+        const uint64_t bk = smem_desc(k_s, 16u, 1024u), bv = smem_desc(v_s, 16u, 1024u);
+#pragma unroll
+        for (int k = 0; k < kDh / 16; ++k) mma1(tm_s, aq + 2u * k, bk + 2u * k, idesc_s, k != 0);
+#pragma unroll
+        for (int k = 0; k < kDh / 16; ++k) mma1(tm_dp, ao + 2u * k, bv + 2u * k, idesc_s, k != 0);
+        commit1(bar(5));
+      };
+      bool ok = mbar_wait(bar(0), 0, abort_flag, status) && mbar_wait(bar(1), 0, abort_flag, status);
+      if (ok) {
+        tc_fence_after();
+        mma_sdp(0);
+      }
+      for (int n = 0; ok && n < total; ++n) {
+        const int st = n & 1;
+        if (!mbar_wait(bar(6), n & 1, abort_flag, status)) break;                 // P and dS of unit n are in shared memory
+        tc_fence_after();
+        // A = P^T / dS^T: rows of the tile are the contraction index (queries), 64 keys per 128-byte row, the two
+        // 64-key halves 16 KB apart; B = dO / Q with rows = queries.
+        const uint64_t ap = smem_desc(p_s, (uint32_t)(kPBytes / 2), 1024u), ad = smem_desc(ds_s, (uint32_t)(kPBytes / 2), 1024u);
+        const uint64_t bo = smem_desc(do_s + st * kTileBytes, (uint32_t)kDh * 128u, 1024u);
+        const uint64_t bq = smem_desc(q_s + st * kTileBytes, (uint32_t)kDh * 128u, 1024u);
+#pragma unroll
+        for (int k = 0; k < kBq / 16; ++k) mma1(tm_dv, ap + (uint64_t)(k * 128), bo + (uint64_t)(k * 128), idesc_t, (n | k) != 0);
+#pragma unroll
+        for (int k = 0; k < kBq / 16; ++k) mma1(tm_dk, ad + (uint64_t)(k * 128), bq + (uint64_t)(k * 128), idesc_t, (n | k) != 0);
+        commit1(bar(3 + st));
+        if (n + 1 == total) commit1(bar(7));
+        if (n + 1 < total) {
+          if (!mbar_wait(bar(1 + ((n + 1) & 1)), ((n + 1) >> 1) & 1, abort_flag, status)) break;
+          tc_fence_after();
+          mma_sdp(n + 1);
+        }
+        if (n + 2 < total) {
+          if (!mbar_wait(bar(3 + st), (n >> 1) & 1, abort_flag, status)) break;
+          load_q(n + 2);
+        }
+      }
+    }
+  } else {
+    const int r = warp * 32 + lane;
+    const uint32_t lane_off = (uint32_t)(warp * 32) << 16;
+    bool ok = true;
+    for (int n = 0; n < total; ++n) {
+      const int hq = match[n / per_head], i = kb + n % per_head;
+      const int qi = i * kBq + r;
+      const bool row_ok = qi < p.seq_len;
+      const long long stat = ((long long)s * p.heads + hq) * p.T + (long long)b * p.seq_len + qi;
+      const float lse2 = row_ok ? p.lse[stat] * 1.4426950408889634f : 0.f;
+      const float dl = row_ok ? p.delta[stat] : 0.f;
+      if (!__all_sync(0xffffffffu, mbar_wait(bar(5), n & 1, abort_flag, status))) { ok = false; break; }
+      tc_fence_after();
+      const int k_lim = !row_ok ? -1 : ((i == kb) ? r : kBk);                     // diagonal block: keys <= query
+#pragma unroll
+      for (int c = 0; c < kBk / 32; ++c) {
+        uint32_t vs[32], vd[32];
+        tc_ld32(tm_s + lane_off + 32 * c, vs);
+        tc_ld32(tm_dp + lane_off + 32 * c, vd);
+        tc_wait_ld();
+        uint32_t wp[16], wd[16];
+#pragma unroll
+        for (int e = 0; e < 16; ++e) {
+          float pr[2], d2[2];
+#pragma unroll
+          for (int h = 0; h < 2; ++h) {
+            const int col = 32 * c + 2 * e + h;
+            pr[h] = col <= k_lim ? exp2f(fmaf(__uint_as_float(vs[2 * e + h]), p.scale_log2, -lse2)) : 0.f;
+            d2[h] = pr[h] * (__uint_as_float(vd[2 * e + h]) - dl);
+          }
+          wp[e] = pack2(pr[0], pr[1]);
+          wd[e] = pack2(d2[0], d2[1]);
+        }
+        store_row_chunk32(p_s, r, c, wp);
+        store_row_chunk32(ds_s, r, c, wd);
+      }
+      fence_async_smem();
+      tc_fence_before();
+      mbar_arrive(bar(6));
+    }
+    // accumulator rows are keys now: thread r owns key kb * 128 + r
+    const int kj = kb * kBk + r;
+    const long long row = (long long)s * p.T + (long long)b * p.seq_len + kj;
+    uint4* dst_k = reinterpret_cast<uint4*>(p.d_qkv + row * p.nq + p.a_sub + kvp * kDh);
+    uint4* dst_v = reinterpret_cast<uint4*>(p.d_qkv + row * p.nq + p.a_sub + (p.kv_max + kvp) * kDh);
+    if (total == 0) {                                    // a KV position this subnet does not hold: zero gradient
+      if (kj < p.seq_len)
+        for (int c = 0; c < kDh / 8; ++c) { dst_k[c] = make_uint4(0, 0, 0, 0); dst_v[c] = make_uint4(0, 0, 0, 0); }
+    } else if (ok && __all_sync(0xffffffffu, mbar_wait(bar(7), 0, abort_flag, status))) {
+      tc_fence_after();
+      const float sc = p.scale_log2 * 0.6931471805599453f;
+#pragma unroll
+      for (int c = 0; c < kDh / 32; ++c) {
+        uint32_t vv[32], vk[32];
+        tc_ld32(tm_dv + lane_off + 32 * c, vv);
+        tc_ld32(tm_dk + lane_off + 32 * c, vk);
+        tc_wait_ld();
+        if (kj < p.seq_len) {
+#pragma unroll
+          for (int q4 = 0; q4 < 4; ++q4) {
+            dst_v[4 * c + q4] = make_uint4(pack2(__uint_as_float(vv[8 * q4]), __uint_as_float(vv[8 * q4 + 1])),
+                                           pack2(__uint_as_float(vv[8 * q4 + 2]), __uint_as_float(vv[8 * q4 + 3])),
+                                           pack2(__uint_as_float(vv[8 * q4 + 4]), __uint_as_float(vv[8 * q4 + 5])),
+                                           pack2(__uint_as_float(vv[8 * q4 + 6]), __uint_as_float(vv[8 * q4 + 7])));
+            dst_k[4 * c + q4] = make_uint4(pack2(sc * __uint_as_float(vk[8 * q4]), sc * __uint_as_float(vk[8 * q4 + 1])),
+                                           pack2(sc * __uint_as_float(vk[8 * q4 + 2]), sc * __uint_as_float(vk[8 * q4 + 3])),
+                                           pack2(sc * __uint_as_float(vk[8 * q4 + 4]), sc * __uint_as_float(vk[8 * q4 + 5])),
+                                           pack2(sc * __uint_as_float(vk[8 * q4 + 6]), sc * __uint_as_float(vk[8 * q4 + 7])));
+          }
+        }
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (*abort_flag) {
+    const uint64_t t0 = global_timer_ns();
+    while (global_timer_ns() - t0 < 2000000ull) __nanosleep(1000);
+    __syncthreads();
+  }
+  if (warp == 4) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"((uint32_t)kBwdTmemCols) : "memory");
+  }
+}
+
+}  // namespace
+
+// Map over a bf16 activation [S * n_seqs][seq_len][width], box = 64 columns x 128 rows of one sequence.
+static int sequence_map(CUtensorMap* tm, const void* ptr, int width, const AttnParams& p, int n_subnets) {
+  const unsigned long long dims[3] = {(unsigned long long)width, (unsigned long long)p.seq_len,
+                                      (unsigned long long)n_subnets * p.n_seqs};
+  const unsigned long long strides[2] = {(unsigned long long)width * 2, (unsigned long long)p.seq_len * width * 2};
+  const unsigned box[3] = {64, 128, 1};
+  return encode_map_3d_bf16(tm, ptr, dims, strides, box, 128);
+}
+
+int attn_bwd_tc(const AttnParams& p, int n_subnets, cudaStream_t st) {
+  if (p.d_head != kDh || p.nq % 8 != 0) return TWIST_ERR_UNSUPPORTED;
+  CUtensorMap tq, tdo;
+  int rc = sequence_map(&tq, p.qkv, p.nq, p, n_subnets);
+  if (rc != TWIST_OK) return rc;
+  rc = sequence_map(&tdo, p.d_out, p.a_sub, p, n_subnets);
+  if (rc != TWIST_OK) return rc;
+  static bool configured = false;
+  if (!configured) {
+    TWIST_CUDA_TRY(cudaFuncSetAttribute(attn_dq_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kDqSmem));
+    TWIST_CUDA_TRY(cudaFuncSetAttribute(attn_dkv_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kDkvSmem));
+    configured = true;
+  }
+  int* status = device_status_ptr();
+  if (!status) return TWIST_ERR_CUDA;
+  const int nb = (p.seq_len + kBq - 1) / kBq;
+  attn_dq_tc_kernel<<<dim3(nb, p.heads, n_subnets * p.n_seqs), kFwdThreads, kDqSmem, st>>>(tq, tdo, p, status);
+  TWIST_LAUNCH_CHECK();
+  attn_dkv_tc_kernel<<<dim3(nb, p.kv_max, n_subnets * p.n_seqs), kFwdThreads, kDkvSmem, st>>>(tq, tdo, p, status);
+  TWIST_LAUNCH_CHECK();
+  return TWIST_OK;
+}
+
+int attn_fwd_tc(const AttnParams& p, int n_subnets, cudaStream_t st) {
+  if (p.d_head != kDh || p.nq % 8 != 0) return TWIST_ERR_UNSUPPORTED;
+  CUtensorMap tm;
+  int rc = sequence_map(&tm, p.qkv, p.nq, p, n_subnets);
+  if (rc != TWIST_OK) return rc;
+  static bool configured = false;
+  if (!configured) {
+    TWIST_CUDA_TRY(cudaFuncSetAttribute(attn_fwd_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kFwdSmem));
+    configured = true;
+  }
+  int* status = device_status_ptr();
+  if (!status) return TWIST_ERR_CUDA;
+  const dim3 grid((p.seq_len + kBq - 1) / kBq, p.heads, n_subnets * p.n_seqs);
+  attn_fwd_tc_kernel<<<grid, kFwdThreads, kFwdSmem, st>>>(tm, p, status);
+  TWIST_LAUNCH_CHECK();
+  return TWIST_OK;
+}
+
+}  // namespace twist

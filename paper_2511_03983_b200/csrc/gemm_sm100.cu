@@ -155,6 +155,25 @@ __global__ void fused_loss_finish_kernel(const float* __restrict__ partial, long
 
 }  // namespace
 
+int encode_map_3d_bf16(CUtensorMap* map, const void* ptr, const unsigned long long dims[3],
+                       const unsigned long long strides[2], const unsigned box[3], int swizzle_bytes) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) { note_cuda_error(cudaErrorUnknown, "cuTensorMapEncodeTiled entry point"); return TWIST_ERR_CUDA; }
+  if (!ptr || !aligned16(ptr) || strides[0] % 16 || strides[1] % 16) return TWIST_ERR_SHAPE;
+  cuuint64_t d[3] = {dims[0], dims[1], dims[2]};
+  cuuint64_t st[2] = {strides[0], strides[1]};
+  cuuint32_t bx[3] = {box[0], box[1], box[2]};
+  cuuint32_t estr[3] = {1, 1, 1};
+  CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), d, st, bx, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B,
+                  CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    note_cuda_error(cudaErrorInvalidValue, "cuTensorMapEncodeTiled");
+    return TWIST_ERR_CUDA;
+  }
+  return TWIST_OK;
+}
+
 size_t fused_loss_partials(int groups, int M, int N) {
   const size_t m_tiles = (size_t)(M + kBM - 1) / kBM, n_tiles = (size_t)(N + kBN - 1) / kBN;
   return (size_t)groups * m_tiles * n_tiles * 8;
