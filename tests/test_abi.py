@@ -66,6 +66,21 @@ def test_host_side_argument_checks():
     # mse workspace
     assert B.twist_mse_workspace_bytes(4) == 4 * 1024 * 4
     assert h.twist_mse_fwd_bwd(dummy, dummy, dummy, dummy, 2, 8, 64, None, 0, 0, B.BF16, None, 0, None) == B.ERR_WORKSPACE
+    # attention core
+    assert h.twist_attn_core_fwd(None, None) == B.ERR_NULL
+    ac = B.AttnCoreArgs(B.FP32, 2, 1, 64, 2, 2, 64, 0, 0, 0x1000, 0x2000, 0x3000)
+    assert h.twist_attn_core_fwd(C.byref(ac), None) == B.ERR_UNSUPPORTED                 # bf16 only
+    ac = B.AttnCoreArgs(B.BF16, 2, 1, 64, 2, 2, 48, 0, 0, 0x1000, 0x2000, 0x3000)
+    assert h.twist_attn_core_fwd(C.byref(ac), None) == B.ERR_UNSUPPORTED                 # head size
+    ac = B.AttnCoreArgs(B.BF16, 2, 1, 64, 4, 2, 64, 0, 0, 0x1000, 0x2000, 0x3000)
+    assert h.twist_attn_core_fwd(C.byref(ac), None) == B.ERR_SHAPE                       # kv_max != head_keep without sharing
+    ac = B.AttnCoreArgs(B.BF16, 2, 1, 64, 2, 2, 64, 0, 0, 0x1000, 0x2000, None)
+    assert h.twist_attn_core_fwd(C.byref(ac), None) == B.ERR_NULL                        # lse missing
+    # skip connections are not combinable with the fused loss
+    a = B.FfnArgs(B.FFN_SWIGLU, B.BF16, 2, 128, 64, 96, 1.0, 0.0, 0x1000, 0x1000, 0x1000, None, None, 0x1000, 0x1000,
+                  0x1000, 0x1000, None, None, None, None, 0x1000, 0x1000, 0x1000, 1 << 30, 0x1000, None)
+    assert h.twist_subnet_ffn_fwd(C.byref(a), None) == B.ERR_UNSUPPORTED
+
 
 
 def test_missing_library_fails_loudly(monkeypatch, tmp_path):
