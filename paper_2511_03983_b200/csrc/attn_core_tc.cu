@@ -29,7 +29,7 @@ constexpr int kBq = 128, kBk = 128;     // queries per CTA, keys per block
 constexpr int kTileBytes = 128 * kDh * 2;            // a 128-row tile of Q, K or V: 16 KB
 constexpr int kPBytes = kBq * kBk * 2;               // P: 32 KB (two 64-key halves of 16 KB)
 constexpr int kFwdThreads = 160;
-constexpr int kFwdSmem = kTileBytes * 5 + kPBytes + 1024 + 128;   // Q, K[2], V[2], P, alignment, barriers
+constexpr int kFwdSmem = kTileBytes * 4 + kPBytes + 1024 + 128;   // Q, K[2], V, P, alignment, barriers: two CTAs per SM
 constexpr int kFwdTmemCols = 256;       // S: columns 0..127, O_blk: columns 128..191
 
 __device__ inline void mma1(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
@@ -58,15 +58,16 @@ __device__ inline int kv_position(const AttnParams& p, int s, int hq) {
 }
 
 // qkv viewed as [S * n_seqs][seq_len][nq]: rows past the end of a sequence read as zeros.
-__global__ void __launch_bounds__(kFwdThreads) attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQKV,
-                                                                  const AttnParams p, int* status) {
+__global__ void __launch_bounds__(kFwdThreads, 2) attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQKV,
+                                                                     const AttnParams p, int* status) {
   extern __shared__ unsigned char smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   unsigned char* gen = smem_raw + (base - smem_u32(smem_raw));
-  const uint32_t q_s = base, k_s = base + kTileBytes, v_s = base + 3 * kTileBytes, p_s = base + 5 * kTileBytes;
+  const uint32_t q_s = base, k_s = base + kTileBytes, v_s = base + 3 * kTileBytes, p_s = base + 4 * kTileBytes;
   const uint32_t bar0 = p_s + kPBytes;
-  volatile uint32_t* ctrl = reinterpret_cast<volatile uint32_t*>(gen + 5 * kTileBytes + kPBytes);
-  // barriers (8 bytes each): 0 q_full, 1-2 kv_full, 3-4 kv_free, 5 s_full, 6 p_ready, 7 o_full; then TMEM base, abort flag
+  volatile uint32_t* ctrl = reinterpret_cast<volatile uint32_t*>(gen + 4 * kTileBytes + kPBytes);
+  // Two CTAs share an SM (their startup, softmax and MMA phases interleave), so K is double-buffered and V is not.
+  // barriers (8 bytes each): 0 q_full, 1-2 k_full, 3 v_full, 4 v_free, 5 s_full, 6 p_ready, 7 o_full; then TMEM base, abort flag
   auto bar = [&](int i) { return bar0 + 8u * i; };
   volatile uint32_t* tmem_slot = ctrl + 16;
   volatile int* abort_flag = reinterpret_cast<volatile int*>(ctrl + 17);
@@ -97,16 +98,20 @@ __global__ void __launch_bounds__(kFwdThreads) attn_fwd_tc_kernel(const __grid_c
       const int kvp = kv_position(p, s, hq);
       const int z = blockIdx.z;
       const int k_col = p.a_sub + kvp * kDh, v_col = k_col + p.kv_max * kDh;
-      auto load_kv = [&](int j) {
+      auto load_k = [&](int j) {
         const int st = j & 1;
-        mbar_expect_tx(bar(1 + st), 2 * kTileBytes);
+        mbar_expect_tx(bar(1 + st), kTileBytes);
         tma_load_3d_local(k_s + st * kTileBytes, &tmQKV, bar(1 + st), k_col, j * kBk, z);
-        tma_load_3d_local(v_s + st * kTileBytes, &tmQKV, bar(1 + st), v_col, j * kBk, z);
+      };
+      auto load_v = [&](int j) {
+        mbar_expect_tx(bar(3), kTileBytes);
+        tma_load_3d_local(v_s, &tmQKV, bar(3), v_col, j * kBk, z);
       };
       mbar_expect_tx(bar(0), kTileBytes);
       tma_load_3d_local(q_s, &tmQKV, bar(0), hq * kDh, qb * kBq, z);
-      load_kv(0);
-      if (nblk > 1) load_kv(1);
+      load_k(0);
+      load_v(0);
+      if (nblk > 1) load_k(1);
       constexpr uint32_t idesc_s = idesc_bf16(0, 0, kBq, kBk);       // S = Q K^T : both K-major
       constexpr uint32_t idesc_o = idesc_bf16(0, 1, kBq, kDh);       // O = P V   : V MN-major
       auto mma_s = [&](int j) {
@@ -121,25 +126,24 @@ __global__ void __launch_bounds__(kFwdThreads) attn_fwd_tc_kernel(const __grid_c
         mma_s(0);
       }
       for (int j = 0; ok && j < nblk; ++j) {
-        const int st = j & 1;
-        if (!mbar_wait(bar(6), j & 1, abort_flag, status)) break;                 // P of block j is in shared memory
+        if (!mbar_wait(bar(6), j & 1, abort_flag, status)) break;                 // P of block j is in shared memory:
+        if (j + 2 < nblk) load_k(j + 2);                                          // S(j) was read, so K(j)'s buffer is free
+        if (!mbar_wait(bar(3), j & 1, abort_flag, status)) break;                 // V of block j
         tc_fence_after();
-        const uint64_t bd = smem_desc(v_s + st * kTileBytes, (uint32_t)kDh * 128u, 1024u);
+        const uint64_t bd = smem_desc(v_s, (uint32_t)kDh * 128u, 1024u);
 #pragma unroll
         for (int k = 0; k < kBk / 16; ++k) {
           const uint64_t a = smem_desc(p_s + (k >> 2) * (kPBytes / 2), 16u, 1024u) + 2u * (k & 3);
           mma1(tm_o, a, bd + (uint64_t)((k * 16 * 128) >> 4), idesc_o, k != 0);
         }
         commit1(bar(7));                                                          // O_blk complete
-        commit1(bar(3 + st));                                                     // K/V stage free
+        commit1(bar(4));                                                          // V buffer free
         if (j + 1 < nblk) {
           if (!mbar_wait(bar(1 + ((j + 1) & 1)), ((j + 1) >> 1) & 1, abort_flag, status)) break;
           tc_fence_after();
           mma_s(j + 1);                                                           // overlaps the threads' work on O
-        }
-        if (j + 2 < nblk) {
-          if (!mbar_wait(bar(3 + st), (j >> 1) & 1, abort_flag, status)) break;
-          load_kv(j + 2);
+          if (!mbar_wait(bar(4), j & 1, abort_flag, status)) break;
+          load_v(j + 1);
         }
       }
     }
