@@ -251,11 +251,55 @@ __device__ inline void store_row_chunk32(uint32_t tile, int r, int c, const uint
 }
 
 constexpr int kBwdTmemCols = 512;
-constexpr int kDqSmem = kTileBytes * 6 + kPBytes + 1024 + 128;        // Q, dO, K[2], V[2], dS
-constexpr int kDkvSmem = kTileBytes * 6 + 2 * kPBytes + 1024 + 256;   // K, V, Q[2], dO[2], P, dS
+constexpr int kBwdThreads = 288;        // 8 element-wise warps (two per tensor-memory lane quarter) + the control warp
+constexpr int kDqSmem = kTileBytes * 6 + 2 * kPBytes + 1024 + 128;    // Q, dO, K[2], V[2], dS[2]
+constexpr int kDkvSmem = kTileBytes * 6 + 4 * kPBytes + 1024 + 256;   // K, V, Q[2], dO[2], P[2], dS[2]
 
-// ---- dQ: grid (query blocks, kept heads, S * n_seqs)
-__global__ void __launch_bounds__(kFwdThreads) attn_dq_tc_kernel(const __grid_constant__ CUtensorMap tmQKV,
+// Element-wise step shared by the two backward kernels: for this thread's row and its 64 columns (two 32-column
+// chunks starting at chunk c0) of S and dP in tensor memory, P = exp2(S * scale - lse2) where visible (column <=
+// k_lim), dS = P * (dP - dl); dS (and P when WRITE_P) go to the operand tiles in shared memory.
+template <bool WRITE_P>
+__device__ inline void probs_and_ds(uint32_t t_s, uint32_t t_dp, int c0, int r, int k_lim, float scale_log2, float lse2,
+                                    float dl, uint32_t p_tile, uint32_t ds_tile) {
+#pragma unroll
+  for (int cc = 0; cc < 2; ++cc) {
+    const int c = c0 + cc;
+    uint32_t vs[32], vd[32];
+    tc_ld32(t_s + 32 * c, vs);
+    tc_ld32(t_dp + 32 * c, vd);
+    tc_wait_ld();
+    uint32_t wp[16], wd[16];
+#pragma unroll
+    for (int e = 0; e < 16; ++e) {
+      float pr[2], d2[2];
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        const int col = 32 * c + 2 * e + h;
+        pr[h] = col <= k_lim ? exp2f(fmaf(__uint_as_float(vs[2 * e + h]), scale_log2, -lse2)) : 0.f;
+        d2[h] = pr[h] * (__uint_as_float(vd[2 * e + h]) - dl);
+      }
+      wp[e] = pack2(pr[0], pr[1]);
+      wd[e] = pack2(d2[0], d2[1]);
+    }
+    if (WRITE_P) store_row_chunk32(p_tile, r, c, wp);
+    store_row_chunk32(ds_tile, r, c, wd);
+  }
+}
+
+// Stores 32 accumulator columns (scaled) of this thread's row as bf16.
+__device__ inline void store_acc32(__nv_bfloat16* dst, const uint32_t (&v)[32], float sc) {
+  uint4* d = reinterpret_cast<uint4*>(dst);
+#pragma unroll
+  for (int q4 = 0; q4 < 4; ++q4)
+    d[q4] = make_uint4(pack2(sc * __uint_as_float(v[8 * q4]), sc * __uint_as_float(v[8 * q4 + 1])),
+                       pack2(sc * __uint_as_float(v[8 * q4 + 2]), sc * __uint_as_float(v[8 * q4 + 3])),
+                       pack2(sc * __uint_as_float(v[8 * q4 + 4]), sc * __uint_as_float(v[8 * q4 + 5])),
+                       pack2(sc * __uint_as_float(v[8 * q4 + 6]), sc * __uint_as_float(v[8 * q4 + 7])));
+}
+
+// ---- dQ: grid (query blocks, kept heads, S * n_seqs).  S / dP of block j + 1 are issued before dQ += dS K of block j
+// (dS is double-buffered), so the MMAs of one block run while the threads work on the next.
+__global__ void __launch_bounds__(kBwdThreads) attn_dq_tc_kernel(const __grid_constant__ CUtensorMap tmQKV,
                                                                  const __grid_constant__ CUtensorMap tmDO,
                                                                  const AttnParams p, int* status) {
   extern __shared__ unsigned char smem_raw[];
@@ -263,8 +307,8 @@ __global__ void __launch_bounds__(kFwdThreads) attn_dq_tc_kernel(const __grid_co
   unsigned char* gen = smem_raw + (base - smem_u32(smem_raw));
   const uint32_t q_s = base, do_s = base + kTileBytes, k_s = base + 2 * kTileBytes, v_s = base + 4 * kTileBytes,
                  ds_s = base + 6 * kTileBytes;
-  const uint32_t bar0 = ds_s + kPBytes;
-  volatile uint32_t* ctrl = reinterpret_cast<volatile uint32_t*>(gen + 6 * kTileBytes + kPBytes);
+  const uint32_t bar0 = ds_s + 2 * kPBytes;
+  volatile uint32_t* ctrl = reinterpret_cast<volatile uint32_t*>(gen + 6 * kTileBytes + 2 * kPBytes);
   // barriers: 0 q_full, 1-2 kv_full, 3-4 kv_free, 5 sdp_full, 6 ds_ready, 7 dq_full
   auto bar = [&](int i) { return bar0 + 8u * i; };
   volatile uint32_t* tmem_slot = ctrl + 16;
@@ -272,15 +316,15 @@ __global__ void __launch_bounds__(kFwdThreads) attn_dq_tc_kernel(const __grid_co
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int qb = blockIdx.x, hq = blockIdx.y, s = blockIdx.z / p.n_seqs, b = blockIdx.z - s * p.n_seqs;
   const int nblk = qb + 1;
-  if (threadIdx.x == 128) {
+  if (threadIdx.x == 256) {
     tma_prefetch_desc(&tmQKV);
     tma_prefetch_desc(&tmDO);
-    for (int i = 0; i < 8; ++i) mbar_init(bar(i), i == 6 ? 128 : 1);
+    for (int i = 0; i < 8; ++i) mbar_init(bar(i), i == 6 ? 256 : 1);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     fence_async_smem();
   }
-  if (warp == 4) {
+  if (warp == 8) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
                  ::"r"(smem_u32(const_cast<uint32_t*>(tmem_slot))), "r"((uint32_t)kBwdTmemCols) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -291,7 +335,7 @@ __global__ void __launch_bounds__(kFwdThreads) attn_dq_tc_kernel(const __grid_co
   const uint32_t tmem = *tmem_slot;
   const uint32_t tm_s = tmem, tm_dp = tmem + 128, tm_dq = tmem + 256;
 
-  if (warp == 4) {
+  if (warp == 8) {
     if (lane == 0) {
       const int kvp = kv_position(p, s, hq);
       const int z = blockIdx.z;
@@ -325,21 +369,22 @@ __global__ void __launch_bounds__(kFwdThreads) attn_dq_tc_kernel(const __grid_co
       }
       for (int j = 0; ok && j < nblk; ++j) {
         const int st = j & 1;
-        if (!mbar_wait(bar(6), j & 1, abort_flag, status)) break;                 // dS of block j is in shared memory
-        tc_fence_after();
-        const uint64_t bd = smem_desc(k_s + st * kTileBytes, (uint32_t)kDh * 128u, 1024u);
-#pragma unroll
-        for (int k = 0; k < kBk / 16; ++k) {
-          const uint64_t a = smem_desc(ds_s + (k >> 2) * (kPBytes / 2), 16u, 1024u) + 2u * (k & 3);
-          mma1(tm_dq, a, bd + (uint64_t)((k * 16 * 128) >> 4), idesc_q, (j | k) != 0);
-        }
-        commit1(bar(3 + st));
-        if (j + 1 == nblk) commit1(bar(7));
+        if (!mbar_wait(bar(6), j & 1, abort_flag, status)) break;                 // dS of block j is in shared memory,
+        tc_fence_after();                                                         // S / dP of block j have been read
         if (j + 1 < nblk) {
           if (!mbar_wait(bar(1 + ((j + 1) & 1)), ((j + 1) >> 1) & 1, abort_flag, status)) break;
           tc_fence_after();
           mma_sdp(j + 1);
         }
+        const uint64_t bd = smem_desc(k_s + st * kTileBytes, (uint32_t)kDh * 128u, 1024u);
+        const uint32_t ds_j = ds_s + st * kPBytes;
+#pragma unroll
+        for (int k = 0; k < kBk / 16; ++k) {
+          const uint64_t a = smem_desc(ds_j + (k >> 2) * (kPBytes / 2), 16u, 1024u) + 2u * (k & 3);
+          mma1(tm_dq, a, bd + (uint64_t)((k * 16 * 128) >> 4), idesc_q, (j | k) != 0);
+        }
+        commit1(bar(3 + st));
+        if (j + 1 == nblk) commit1(bar(7));
         if (j + 2 < nblk) {
           if (!mbar_wait(bar(3 + st), (j >> 1) & 1, abort_flag, status)) break;
           load_kv(j + 2);
@@ -347,10 +392,11 @@ __global__ void __launch_bounds__(kFwdThreads) attn_dq_tc_kernel(const __grid_co
       }
     }
   } else {
-    const int r = warp * 32 + lane;
+    const int quarter = warp & 3, half = warp >> 2;
+    const int r = quarter * 32 + lane;
     const int qi = qb * kBq + r;
     const bool row_ok = qi < p.seq_len;
-    const uint32_t lane_off = (uint32_t)(warp * 32) << 16;
+    const uint32_t lane_off = (uint32_t)(quarter * 32) << 16;
     const long long stat = ((long long)s * p.heads + hq) * p.T + (long long)b * p.seq_len + qi;
     const float lse2 = row_ok ? p.lse[stat] * 1.4426950408889634f : 0.f;
     const float dl = row_ok ? p.delta[stat] : 0.f;
@@ -359,48 +405,20 @@ __global__ void __launch_bounds__(kFwdThreads) attn_dq_tc_kernel(const __grid_co
       if (!__all_sync(0xffffffffu, mbar_wait(bar(5), j & 1, abort_flag, status))) { ok = false; break; }
       tc_fence_after();
       const int k_lim = !row_ok ? -1 : ((j == qb) ? qi - j * kBk : kBk);
-#pragma unroll
-      for (int c = 0; c < kBk / 32; ++c) {
-        uint32_t vs[32], vd[32];
-        tc_ld32(tm_s + lane_off + 32 * c, vs);
-        tc_ld32(tm_dp + lane_off + 32 * c, vd);
-        tc_wait_ld();
-        uint32_t w[16];
-#pragma unroll
-        for (int i = 0; i < 16; ++i) {
-          float d2[2];
-#pragma unroll
-          for (int e = 0; e < 2; ++e) {
-            const int col = 32 * c + 2 * i + e;
-            const float pr = col <= k_lim ? exp2f(fmaf(__uint_as_float(vs[2 * i + e]), p.scale_log2, -lse2)) : 0.f;
-            d2[e] = pr * (__uint_as_float(vd[2 * i + e]) - dl);
-          }
-          w[i] = pack2(d2[0], d2[1]);
-        }
-        store_row_chunk32(ds_s, r, c, w);
-      }
+      probs_and_ds<false>(tm_s + lane_off, tm_dp + lane_off, 2 * half, r, k_lim, p.scale_log2, lse2, dl, 0u,
+                          ds_s + (j & 1) * kPBytes);
       fence_async_smem();
       tc_fence_before();
       mbar_arrive(bar(6));
     }
     if (ok && __all_sync(0xffffffffu, mbar_wait(bar(7), 0, abort_flag, status))) {
       tc_fence_after();
-      const float sc = p.scale_log2 * 0.6931471805599453f;                         // 1 / sqrt(d_head)
-      const long long row = (long long)s * p.T + (long long)b * p.seq_len + qi;
-      uint4* dst = reinterpret_cast<uint4*>(p.d_qkv + row * p.nq + hq * kDh);
-#pragma unroll
-      for (int c = 0; c < kDh / 32; ++c) {
-        uint32_t v[32];
-        tc_ld32(tm_dq + lane_off + 32 * c, v);
-        tc_wait_ld();
-        if (row_ok) {
-#pragma unroll
-          for (int q4 = 0; q4 < 4; ++q4)
-            dst[4 * c + q4] = make_uint4(pack2(sc * __uint_as_float(v[8 * q4]), sc * __uint_as_float(v[8 * q4 + 1])),
-                                         pack2(sc * __uint_as_float(v[8 * q4 + 2]), sc * __uint_as_float(v[8 * q4 + 3])),
-                                         pack2(sc * __uint_as_float(v[8 * q4 + 4]), sc * __uint_as_float(v[8 * q4 + 5])),
-                                         pack2(sc * __uint_as_float(v[8 * q4 + 6]), sc * __uint_as_float(v[8 * q4 + 7])));
-        }
+      uint32_t v[32];
+      tc_ld32(tm_dq + lane_off + 32 * half, v);
+      tc_wait_ld();
+      if (row_ok) {
+        const long long row = (long long)s * p.T + (long long)b * p.seq_len + qi;
+        store_acc32(p.d_qkv + row * p.nq + hq * kDh + 32 * half, v, p.scale_log2 * 0.6931471805599453f);   // / sqrt(d_head)
       }
     }
   }
@@ -411,14 +429,15 @@ __global__ void __launch_bounds__(kFwdThreads) attn_dq_tc_kernel(const __grid_co
     while (global_timer_ns() - t0 < 2000000ull) __nanosleep(1000);
     __syncthreads();
   }
-  if (warp == 4) {
+  if (warp == 8) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"((uint32_t)kBwdTmemCols) : "memory");
   }
 }
 
-// ---- dK, dV: grid (key blocks, KV positions, S * n_seqs)
-__global__ void __launch_bounds__(kFwdThreads) attn_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmQKV,
+// ---- dK, dV: grid (key blocks, KV positions, S * n_seqs).  Units (kept head, query block) stream through; S / dP
+// of unit n + 1 are issued before dV += P^T dO, dK += dS^T Q of unit n (P and dS are double-buffered).
+__global__ void __launch_bounds__(kBwdThreads) attn_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmQKV,
                                                                   const __grid_constant__ CUtensorMap tmDO,
                                                                   const AttnParams p, int* status) {
   extern __shared__ unsigned char smem_raw[];
@@ -427,9 +446,9 @@ __global__ void __launch_bounds__(kFwdThreads) attn_dkv_tc_kernel(const __grid_c
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   unsigned char* gen = smem_raw + (base - smem_u32(smem_raw));
   const uint32_t k_s = base, v_s = base + kTileBytes, q_s = base + 2 * kTileBytes, do_s = base + 4 * kTileBytes,
-                 p_s = base + 6 * kTileBytes, ds_s = p_s + kPBytes;
-  const uint32_t bar0 = ds_s + kPBytes;
-  volatile uint32_t* ctrl = reinterpret_cast<volatile uint32_t*>(gen + 6 * kTileBytes + 2 * kPBytes);
+                 p_s = base + 6 * kTileBytes, ds_s = p_s + 2 * kPBytes;
+  const uint32_t bar0 = ds_s + 2 * kPBytes;
+  volatile uint32_t* ctrl = reinterpret_cast<volatile uint32_t*>(gen + 6 * kTileBytes + 4 * kPBytes);
   // barriers: 0 kv_full, 1-2 q_full, 3-4 q_free, 5 sdp_full, 6 pds_ready, 7 acc_full
   auto bar = [&](int i) { return bar0 + 8u * i; };
   volatile uint32_t* tmem_slot = ctrl + 16;
@@ -438,10 +457,10 @@ __global__ void __launch_bounds__(kFwdThreads) attn_dkv_tc_kernel(const __grid_c
   const int kb = blockIdx.x, kvp = blockIdx.y, s = blockIdx.z / p.n_seqs, b = blockIdx.z - s * p.n_seqs;
   const int nqb = (p.seq_len + kBq - 1) / kBq;
   const int held = p.kv_count ? p.kv_count[s] : p.kv_max;
-  if (threadIdx.x == 128) {
+  if (threadIdx.x == 256) {
     tma_prefetch_desc(&tmQKV);
     tma_prefetch_desc(&tmDO);
-    for (int i = 0; i < 8; ++i) mbar_init(bar(i), i == 6 ? 128 : 1);
+    for (int i = 0; i < 8; ++i) mbar_init(bar(i), i == 6 ? 256 : 1);
     *abort_flag = 0;
     int n = 0;
     if (kvp < held)
@@ -451,7 +470,7 @@ __global__ void __launch_bounds__(kFwdThreads) attn_dkv_tc_kernel(const __grid_c
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     fence_async_smem();
   }
-  if (warp == 4) {
+  if (warp == 8) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
                  ::"r"(smem_u32(const_cast<uint32_t*>(tmem_slot))), "r"((uint32_t)kBwdTmemCols) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -464,7 +483,7 @@ __global__ void __launch_bounds__(kFwdThreads) attn_dkv_tc_kernel(const __grid_c
   const int per_head = nqb - kb;                         // query blocks kb .. nqb-1
   const int total = n_match_s * per_head;                // units (head, query block)
 
-  if (warp == 4) {
+  if (warp == 8) {
     if (lane == 0 && total > 0) {
       const int z = blockIdx.z;
       auto load_q = [&](int n) {
@@ -497,11 +516,17 @@ __global__ void __launch_bounds__(kFwdThreads) attn_dkv_tc_kernel(const __grid_c
       }
       for (int n = 0; ok && n < total; ++n) {
         const int st = n & 1;
-        if (!mbar_wait(bar(6), n & 1, abort_flag, status)) break;                 // P and dS of unit n are in shared memory
-        tc_fence_after();
+        if (!mbar_wait(bar(6), n & 1, abort_flag, status)) break;                 // P and dS of unit n are in shared memory,
+        tc_fence_after();                                                         // S / dP of unit n have been read
+        if (n + 1 < total) {
+          if (!mbar_wait(bar(1 + ((n + 1) & 1)), ((n + 1) >> 1) & 1, abort_flag, status)) break;
+          tc_fence_after();
+          mma_sdp(n + 1);
+        }
         // A = P^T / dS^T: rows of the tile are the contraction index (queries), 64 keys per 128-byte row, the two
         // 64-key halves 16 KB apart; B = dO / Q with rows = queries.
-        const uint64_t ap = smem_desc(p_s, (uint32_t)(kPBytes / 2), 1024u), ad = smem_desc(ds_s, (uint32_t)(kPBytes / 2), 1024u);
+        const uint64_t ap = smem_desc(p_s + st * kPBytes, (uint32_t)(kPBytes / 2), 1024u);
+        const uint64_t ad = smem_desc(ds_s + st * kPBytes, (uint32_t)(kPBytes / 2), 1024u);
         const uint64_t bo = smem_desc(do_s + st * kTileBytes, (uint32_t)kDh * 128u, 1024u);
         const uint64_t bq = smem_desc(q_s + st * kTileBytes, (uint32_t)kDh * 128u, 1024u);
 #pragma unroll
@@ -510,11 +535,6 @@ __global__ void __launch_bounds__(kFwdThreads) attn_dkv_tc_kernel(const __grid_c
         for (int k = 0; k < kBq / 16; ++k) mma1(tm_dk, ad + (uint64_t)(k * 128), bq + (uint64_t)(k * 128), idesc_t, (n | k) != 0);
         commit1(bar(3 + st));
         if (n + 1 == total) commit1(bar(7));
-        if (n + 1 < total) {
-          if (!mbar_wait(bar(1 + ((n + 1) & 1)), ((n + 1) >> 1) & 1, abort_flag, status)) break;
-          tc_fence_after();
-          mma_sdp(n + 1);
-        }
         if (n + 2 < total) {
           if (!mbar_wait(bar(3 + st), (n >> 1) & 1, abort_flag, status)) break;
           load_q(n + 2);
@@ -522,8 +542,9 @@ __global__ void __launch_bounds__(kFwdThreads) attn_dkv_tc_kernel(const __grid_c
       }
     }
   } else {
-    const int r = warp * 32 + lane;
-    const uint32_t lane_off = (uint32_t)(warp * 32) << 16;
+    const int quarter = warp & 3, half = warp >> 2;
+    const int r = quarter * 32 + lane;
+    const uint32_t lane_off = (uint32_t)(quarter * 32) << 16;
     bool ok = true;
     for (int n = 0; n < total; ++n) {
       const int hq = match[n / per_head], i = kb + n % per_head;
@@ -535,62 +556,28 @@ __global__ void __launch_bounds__(kFwdThreads) attn_dkv_tc_kernel(const __grid_c
       if (!__all_sync(0xffffffffu, mbar_wait(bar(5), n & 1, abort_flag, status))) { ok = false; break; }
       tc_fence_after();
       const int k_lim = !row_ok ? -1 : ((i == kb) ? r : kBk);                     // diagonal block: keys <= query
-#pragma unroll
-      for (int c = 0; c < kBk / 32; ++c) {
-        uint32_t vs[32], vd[32];
-        tc_ld32(tm_s + lane_off + 32 * c, vs);
-        tc_ld32(tm_dp + lane_off + 32 * c, vd);
-        tc_wait_ld();
-        uint32_t wp[16], wd[16];
-#pragma unroll
-        for (int e = 0; e < 16; ++e) {
-          float pr[2], d2[2];
-#pragma unroll
-          for (int h = 0; h < 2; ++h) {
-            const int col = 32 * c + 2 * e + h;
-            pr[h] = col <= k_lim ? exp2f(fmaf(__uint_as_float(vs[2 * e + h]), p.scale_log2, -lse2)) : 0.f;
-            d2[h] = pr[h] * (__uint_as_float(vd[2 * e + h]) - dl);
-          }
-          wp[e] = pack2(pr[0], pr[1]);
-          wd[e] = pack2(d2[0], d2[1]);
-        }
-        store_row_chunk32(p_s, r, c, wp);
-        store_row_chunk32(ds_s, r, c, wd);
-      }
+      probs_and_ds<true>(tm_s + lane_off, tm_dp + lane_off, 2 * half, r, k_lim, p.scale_log2, lse2, dl,
+                         p_s + (n & 1) * kPBytes, ds_s + (n & 1) * kPBytes);
       fence_async_smem();
       tc_fence_before();
       mbar_arrive(bar(6));
     }
-    // accumulator rows are keys now: thread r owns key kb * 128 + r
+    // accumulator rows are keys now: thread r owns key kb * 128 + r; the first four warps store dV, the others dK
     const int kj = kb * kBk + r;
     const long long row = (long long)s * p.T + (long long)b * p.seq_len + kj;
-    uint4* dst_k = reinterpret_cast<uint4*>(p.d_qkv + row * p.nq + p.a_sub + kvp * kDh);
-    uint4* dst_v = reinterpret_cast<uint4*>(p.d_qkv + row * p.nq + p.a_sub + (p.kv_max + kvp) * kDh);
+    __nv_bfloat16* dst = p.d_qkv + row * p.nq + p.a_sub + ((half ? 0 : p.kv_max) + kvp) * kDh;
     if (total == 0) {                                    // a KV position this subnet does not hold: zero gradient
       if (kj < p.seq_len)
-        for (int c = 0; c < kDh / 8; ++c) { dst_k[c] = make_uint4(0, 0, 0, 0); dst_v[c] = make_uint4(0, 0, 0, 0); }
+        for (int c = 0; c < kDh / 8; ++c) reinterpret_cast<uint4*>(dst)[c] = make_uint4(0, 0, 0, 0);
     } else if (ok && __all_sync(0xffffffffu, mbar_wait(bar(7), 0, abort_flag, status))) {
       tc_fence_after();
-      const float sc = p.scale_log2 * 0.6931471805599453f;
+      const float sc = half ? p.scale_log2 * 0.6931471805599453f : 1.f;          // dK carries 1 / sqrt(d_head)
 #pragma unroll
       for (int c = 0; c < kDh / 32; ++c) {
-        uint32_t vv[32], vk[32];
-        tc_ld32(tm_dv + lane_off + 32 * c, vv);
-        tc_ld32(tm_dk + lane_off + 32 * c, vk);
+        uint32_t v[32];
+        tc_ld32((half ? tm_dk : tm_dv) + lane_off + 32 * c, v);
         tc_wait_ld();
-        if (kj < p.seq_len) {
-#pragma unroll
-          for (int q4 = 0; q4 < 4; ++q4) {
-            dst_v[4 * c + q4] = make_uint4(pack2(__uint_as_float(vv[8 * q4]), __uint_as_float(vv[8 * q4 + 1])),
-                                           pack2(__uint_as_float(vv[8 * q4 + 2]), __uint_as_float(vv[8 * q4 + 3])),
-                                           pack2(__uint_as_float(vv[8 * q4 + 4]), __uint_as_float(vv[8 * q4 + 5])),
-                                           pack2(__uint_as_float(vv[8 * q4 + 6]), __uint_as_float(vv[8 * q4 + 7])));
-            dst_k[4 * c + q4] = make_uint4(pack2(sc * __uint_as_float(vk[8 * q4]), sc * __uint_as_float(vk[8 * q4 + 1])),
-                                           pack2(sc * __uint_as_float(vk[8 * q4 + 2]), sc * __uint_as_float(vk[8 * q4 + 3])),
-                                           pack2(sc * __uint_as_float(vk[8 * q4 + 4]), sc * __uint_as_float(vk[8 * q4 + 5])),
-                                           pack2(sc * __uint_as_float(vk[8 * q4 + 6]), sc * __uint_as_float(vk[8 * q4 + 7])));
-          }
-        }
+        if (kj < p.seq_len) store_acc32(dst + 32 * c, v, sc);
       }
     }
   }
@@ -601,7 +588,7 @@ __global__ void __launch_bounds__(kFwdThreads) attn_dkv_tc_kernel(const __grid_c
     while (global_timer_ns() - t0 < 2000000ull) __nanosleep(1000);
     __syncthreads();
   }
-  if (warp == 4) {
+  if (warp == 8) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"((uint32_t)kBwdTmemCols) : "memory");
   }
@@ -634,9 +621,9 @@ int attn_bwd_tc(const AttnParams& p, int n_subnets, cudaStream_t st) {
   int* status = device_status_ptr();
   if (!status) return TWIST_ERR_CUDA;
   const int nb = (p.seq_len + kBq - 1) / kBq;
-  attn_dq_tc_kernel<<<dim3(nb, p.heads, n_subnets * p.n_seqs), kFwdThreads, kDqSmem, st>>>(tq, tdo, p, status);
+  attn_dq_tc_kernel<<<dim3(nb, p.heads, n_subnets * p.n_seqs), kBwdThreads, kDqSmem, st>>>(tq, tdo, p, status);
   TWIST_LAUNCH_CHECK();
-  attn_dkv_tc_kernel<<<dim3(nb, p.kv_max, n_subnets * p.n_seqs), kFwdThreads, kDkvSmem, st>>>(tq, tdo, p, status);
+  attn_dkv_tc_kernel<<<dim3(nb, p.kv_max, n_subnets * p.n_seqs), kBwdThreads, kDkvSmem, st>>>(tq, tdo, p, status);
   TWIST_LAUNCH_CHECK();
   return TWIST_OK;
 }
