@@ -105,10 +105,8 @@ int make_epilogue_maps(int epi, const GemmParams& p, const CUtensorMap& filler, 
   };
   switch (epi) {
     case EPI_STORE: mk(0, p.out0, N, N); break;
-    case EPI_MSE:
-      mk(0, p.in0, N, N); mk(1, p.out1, N, N);
-      if (p.out0) mk(2, p.out0, N, N);
-      break;
+    case EPI_MSE: mk(0, p.in0, N, N); mk(1, p.out1, N, N); mk(2, p.out0, N, N); break;
+    case EPI_MSE_NOY: mk(0, p.in0, N, N); mk(1, p.out1, N, N); break;
     case EPI_SWIGLU_FWD: mk(0, p.out0, N, 2LL * N); mk(1, p.out0 + N, N, 2LL * N); mk(2, p.out1, N, N); break;
     case EPI_ACT_FWD: mk(0, p.out0, N, N); mk(1, p.out1, N, N); break;
     case EPI_DSWIGLU:
@@ -212,11 +210,13 @@ int launch_gemm_bf16(int layout, int epi, const GemmOperand& A, const GemmOperan
       case EPI_DSWIGLU: return launch<MAJOR_K, MAJOR_K, EPI_DSWIGLU>(ta, tb, p, st);
       case EPI_DACT: return launch<MAJOR_K, MAJOR_K, EPI_DACT>(ta, tb, p, st);
       case EPI_MSE: return launch<MAJOR_K, MAJOR_K, EPI_MSE>(ta, tb, p, st);
+      case EPI_MSE_NOY: return launch<MAJOR_K, MAJOR_K, EPI_MSE_NOY>(ta, tb, p, st);
       default: return TWIST_ERR_UNSUPPORTED;
     }
   }
   if (layout == 1 && epi == EPI_STORE) return launch<MAJOR_K, MAJOR_MN, EPI_STORE>(ta, tb, p, st);
   if (layout == 1 && epi == EPI_MSE) return launch<MAJOR_K, MAJOR_MN, EPI_MSE>(ta, tb, p, st);
+  if (layout == 1 && epi == EPI_MSE_NOY) return launch<MAJOR_K, MAJOR_MN, EPI_MSE_NOY>(ta, tb, p, st);
   if (layout == 1 && epi == EPI_RESID) return launch<MAJOR_K, MAJOR_MN, EPI_RESID>(ta, tb, p, st);
   if (layout == 2 && epi == EPI_SGD) return launch<MAJOR_MN, MAJOR_MN, EPI_SGD>(ta, tb, p, st);
   return TWIST_ERR_UNSUPPORTED;

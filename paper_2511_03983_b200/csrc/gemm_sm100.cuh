@@ -32,7 +32,8 @@
 namespace twist {
 
 enum { MAJOR_K = 0, MAJOR_MN = 1 };
-enum { EPI_STORE = 0, EPI_SWIGLU_FWD = 1, EPI_ACT_FWD = 2, EPI_DSWIGLU = 3, EPI_DACT = 4, EPI_SGD = 5, EPI_MSE = 6, EPI_RESID = 7 };
+enum { EPI_STORE = 0, EPI_SWIGLU_FWD = 1, EPI_ACT_FWD = 2, EPI_DSWIGLU = 3, EPI_DACT = 4, EPI_SGD = 5, EPI_MSE = 6, EPI_RESID = 7,
+       EPI_MSE_NOY = 8 /* EPI_MSE without storing D: one box per chunk, so twice as many chunk buffers */ };
 
 constexpr int kBM = 256, kBN = 256, kBK = 64, kUmmaK = 16;   // tile of a CTA pair
 constexpr int kCtaM = kBM / 2, kCtaN = kBN / 2;   // rows of A / columns of B that one CTA of the pair loads
@@ -46,7 +47,7 @@ constexpr int kGemmThreads = 192;
 constexpr int kEpiBoxBytes = 32 * 32 * 2;
 constexpr int kEpiWarpBytes = 16384;
 constexpr int kEpiBytes = 4 * kEpiWarpBytes;
-constexpr int kCtrlBytes = 384;
+constexpr int kCtrlBytes = 512;
 // Operand ring: 5 stages of 32 KB beside the epilogue staging.  The weight-gradient kernel stages nothing and
 // could hold 7, but measured no faster with them (it is bound by power, not by latency), so it keeps 5 too.
 __host__ __device__ constexpr int gemm_stages(bool /*staged_epilogue*/) { return 5; }
@@ -85,9 +86,9 @@ __host__ __device__ constexpr int epi_slots(int epi) {
   return epi == EPI_SWIGLU_FWD ? 3 : (epi == EPI_MSE || epi == EPI_ACT_FWD || epi == EPI_DSWIGLU) ? 2 : 1;
 }
 __host__ __device__ constexpr int epi_in_slots(int epi) {
-  return epi == EPI_DSWIGLU ? 2 : (epi == EPI_MSE || epi == EPI_DACT || epi == EPI_RESID) ? 1 : 0;
+  return epi == EPI_DSWIGLU ? 2 : (epi == EPI_MSE || epi == EPI_MSE_NOY || epi == EPI_DACT || epi == EPI_RESID) ? 1 : 0;
 }
-__host__ __device__ constexpr int epi_bufs(int epi) { return epi_slots(epi) == 3 ? 2 : 4; }
+__host__ __device__ constexpr int epi_bufs(int epi) { return epi_slots(epi) == 3 ? 2 : epi_slots(epi) == 2 ? 4 : 8; }
 
 // Registers of one 32-column chunk of accumulator words.
 template <int EPI> struct EpiAcc { uint32_t r0[32]; };
@@ -208,8 +209,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   volatile uint32_t* ctrl = reinterpret_cast<volatile uint32_t*>(smem_gen + kStages * kStageBytes + (kStaged ? kEpiBytes : 0));
   // control block: 8-byte barriers full[kStages], empty[kStages], tmem_full[2], tmem_empty[2]; then the TMEM base
   // address and the abort flag (4 bytes each, within the first 160 bytes for at most 7 stages); at byte 192 the
-  // 16 "box arrived" barriers of the epilogue warps (4 per warp).  Same offsets in both CTAs of the pair.
-  auto in_bar = [&](int w, uint32_t buf) { return bar_base + 192u + 8u * (4u * w + buf); };
+  // 32 "box arrived" barriers of the epilogue warps (8 per warp).  Same offsets in both CTAs of the pair.
+  auto in_bar = [&](int w, uint32_t buf) { return bar_base + 192u + 8u * (8u * w + buf); };
   auto full_bar = [&](int i) { return bar_base + 8u * i; };
   auto empty_bar = [&](int i) { return bar_base + 8u * (kStages + i); };
   auto tfull_bar = [&](int i) { return bar_base + 8u * (2 * kStages + i); };
@@ -230,7 +231,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     for (int i = 0; i < 2; ++i) { mbar_init(tfull_bar(i), 1); mbar_init(tempty_bar(i), 8); }   // 4 epilogue warps x 2 CTAs
     if (kStaged)
       for (int w = 0; w < 4; ++w)
-        for (int b = 0; b < 4; ++b) mbar_init(in_bar(w, b), 1);
+        for (int b = 0; b < 8; ++b) mbar_init(in_bar(w, b), 1);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -387,50 +388,63 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       }
     } else {
       // Staged epilogues.  Chunk number gc (counted over all tiles of this CTA) uses buffer gc % kBufs of the
-      // warp: kSlots boxes of 2 KB.  Boxes the chunk reads are requested kBufs - 1 chunks ahead, results are
+      // warp: kSlots boxes of 2 KB.  Boxes the chunk reads are requested kBufs / 2 chunks ahead, results are
       // written over them in place (each thread touches only its own row) and leave as bulk stores; a buffer
       // is refilled or rewritten only after the bulk store that last read it has finished reading.
       constexpr int kSlots = epi_slots(EPI), kIn = epi_in_slots(EPI), kBufs = epi_bufs(EPI);
+      constexpr bool kIsMse = EPI == EPI_MSE || EPI == EPI_MSE_NOY;
+      // Inputs are requested kAhead chunks ahead into the buffer that chunk gc + kAhead - kBufs used; only that
+      // chunk's store has to be finished, so up to kBufs - kAhead younger stores may still be reading.
+      constexpr int kAhead = kBufs / 2;
       const uint32_t wbase = epi_base + (uint32_t)warp * kEpiWarpBytes;
       auto box = [&](uint32_t gc, int slot) { return wbase + ((gc & (kBufs - 1)) * kSlots + slot) * kEpiBoxBytes; };
       // 16-byte piece q (0..3) of this thread's row inside a box (64-byte rows, 64-byte swizzle)
       const uint32_t row_off = (uint32_t)lane * 64u;
       const uint32_t sw = ((uint32_t)lane >> 1) & 3u;
       auto piece = [&](uint32_t box_addr, int q) { return box_addr + row_off + ((((uint32_t)q) ^ sw) << 4); };
-      // (group, first row of this warp, first column) of chunk gc; false past the CTA's last tile
-      auto chunk_coords = [&](uint32_t gc, int& g, int& row0, int& n) {
-        const int tile = pair + (int)(gc / kChunks) * num_pairs;
-        if (tile >= total_tiles) return false;
-        int mt, nt;
-        tile_coords(p, tile, g, mt, nt);
-        row0 = mt * kBM + (int)rank * kCtaM + warp * 32;
-        n = nt * kTileN + 32 * (int)(gc % kChunks);
-        return true;
+      // Coordinates (group, first row of this warp, first column) of the tile being processed and of the CTA's next
+      // tile, so that requesting a chunk's inputs costs no index arithmetic (kAhead < kChunks: a requested chunk
+      // lies in one of the two).
+      struct TileAt { int g, row0, n0; bool valid; };
+      auto locate = [&](int tile) {
+        TileAt t;
+        t.valid = tile < total_tiles;
+        t.g = 0; t.row0 = 0; t.n0 = 0;
+        if (t.valid) {
+          int mt, nt;
+          tile_coords(p, tile, t.g, mt, nt);
+          t.row0 = mt * kBM + (int)rank * kCtaM + warp * 32;
+          t.n0 = nt * kTileN;
+        }
+        return t;
       };
-      auto request_inputs = [&](uint32_t gc) {      // lane 0 only
-        int g, row0, n;
-        if (kIn == 0 || !chunk_coords(gc, g, row0, n)) return;
+      TileAt cur = locate(pair), nxt = locate(pair + num_pairs);
+      auto request_inputs = [&](uint32_t gc) {      // lane 0 only; gc / kChunks is tl or tl + 1
+        if (kIn == 0) return;
+        const TileAt& t = (gc / kChunks == tl) ? cur : nxt;
+        if (!t.valid) return;
         const uint32_t bar = in_bar(warp, gc & (kBufs - 1));
         mbar_expect_tx(bar, kIn * kEpiBoxBytes);
+        const int n = t.n0 + 32 * (int)(gc % kChunks);
 #pragma unroll
-        for (int i = 0; i < kIn; ++i) tma_load_3d_local(box(gc, i), &tmE.m[i], bar, n, row0, g);
+        for (int i = 0; i < kIn; ++i) tma_load_3d_local(box(gc, i), &tmE.m[i], bar, n, t.row0, t.g);
       };
       if (lane == 0) {
-        for (uint32_t gc = 0; gc + 1 < (uint32_t)kBufs; ++gc) request_inputs(gc);
+        for (uint32_t gc = 0; gc < (uint32_t)kAhead; ++gc) request_inputs(gc);
       }
 
       for (int tile = pair; ok && tile < total_tiles; tile += num_pairs, ++tl) {
-        int g, mt, nt;
-        tile_coords(p, tile, g, mt, nt);
+        if (tl > 0) { cur = nxt; nxt = locate(tile + num_pairs); }
+        const int g = cur.g, nt_n0 = cur.n0;
         const uint32_t slot = tl & 1u, acc_phase = (tl >> 1) & 1u;
-        const int row0 = mt * kBM + (int)rank * kCtaM + warp * 32;
+        const int row0 = cur.row0;
         const bool row_ok = row0 + lane < p.M;
         const uint32_t t_row = tmem_base + slot * kBN + ((uint32_t)(warp * 32) << 16);
-        const int n_base = nt * kTileN;
+        const int n_base = nt_n0;
         EpiAcc<EPI> acc[2];
         float loss_acc = 0.f, kfac = 0.f;
         int vc = 0;
-        if constexpr (EPI == EPI_MSE) {
+        if constexpr (kIsMse) {
           vc = p.valid_cols ? p.valid_cols[g] : p.seg_width;
           const int n_valid = p.seg_begin + ((p.N - p.seg_begin) / p.seg_width) * vc;
           kfac = 2.0f / ((float)p.M * (float)n_valid);
@@ -466,12 +480,17 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                                               pack2(p.scale * __uint_as_float(r[2]), p.scale * __uint_as_float(r[3])),
                                               pack2(p.scale * __uint_as_float(r[4]), p.scale * __uint_as_float(r[5])),
                                               pack2(p.scale * __uint_as_float(r[6]), p.scale * __uint_as_float(r[7]))));
-            } else if constexpr (EPI == EPI_MSE) {
+            } else if constexpr (kIsMse) {
               const uint4 tv = lds128(piece(b0, q));
               const uint32_t tw[4] = {tv.x, tv.y, tv.z, tv.w};
               // validity is constant over aligned groups of 8 columns (seg_begin, seg_width, vc are multiples of 8)
               const int col = n + 8 * q;
-              const bool cv = row_ok && col < p.N && (col < p.seg_begin || (col - p.seg_begin) % p.seg_width < vc);
+              bool cv = row_ok && col < p.N;
+              if (p.valid_cols && col >= p.seg_begin) {     // masked column groups (uniform branch; few groups: no division)
+                int rel = col - p.seg_begin;
+                while (rel >= p.seg_width) rel -= p.seg_width;
+                cv = cv && rel < vc;
+              }
               uint32_t wy[4], wd[4];
 #pragma unroll
               for (int h = 0; h < 4; ++h) {
@@ -482,7 +501,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                 wd[h] = pack2(kfac * d0, kfac * d1);
               }
               sts128(piece(b0, q), make_uint4(wd[0], wd[1], wd[2], wd[3]));
-              if (p.out0) sts128(piece(b1, q), make_uint4(wy[0], wy[1], wy[2], wy[3]));
+              if constexpr (EPI == EPI_MSE) sts128(piece(b1, q), make_uint4(wy[0], wy[1], wy[2], wy[3]));
             } else if constexpr (EPI == EPI_SWIGLU_FWD) {
               const uint32_t* ru = a.r1 + 8 * q;
               uint32_t wg[4], wu[4], wh[4];
@@ -556,9 +575,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             const int rr = row0, gg = g;
             if constexpr (EPI == EPI_STORE) {
               tma_store_3d(&tmE.m[0], b0, n, rr, gg);
-            } else if constexpr (EPI == EPI_MSE) {
+            } else if constexpr (kIsMse) {
               tma_store_3d(&tmE.m[1], b0, n, rr, gg);
-              if (p.out0) tma_store_3d(&tmE.m[2], b1, n, rr, gg);
+              if constexpr (EPI == EPI_MSE) tma_store_3d(&tmE.m[2], b1, n, rr, gg);
             } else if constexpr (EPI == EPI_SWIGLU_FWD) {
               tma_store_3d(&tmE.m[0], b0, n, rr, gg);
               tma_store_3d(&tmE.m[1], b1, n, rr, gg);
@@ -573,9 +592,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
               tma_store_3d(&tmE.m[1], b0, n, rr, gg);
             }
             bulk_commit();
-            if (kIn > 0) {     // the previous chunk's store has finished reading its buffer: refill it
-              bulk_wait_read<1>();
-              request_inputs(gc + kBufs - 1);
+            if (kIn > 0) {     // refill the buffer whose store is old enough to have finished reading
+              bulk_wait_read<kBufs - kAhead>();
+              request_inputs(gc + kAhead);
             }
           }
         }
@@ -584,7 +603,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive_cluster(tempty_leader[slot]);
-        if constexpr (EPI == EPI_MSE) {   // per-warp partial sum of squared errors, fixed order
+        if constexpr (kIsMse) {   // per-warp partial sum of squared errors, fixed order
           for (int o = 16; o > 0; o >>= 1) loss_acc += __shfl_xor_sync(0xffffffffu, loss_acc, o);
           if (lane == 0) p.dw[((long long)tile * 2 + rank) * 4 + warp] = loss_acc;
         }

@@ -47,7 +47,7 @@ int launch_fused_loss(int layout, const GemmOperand& A, const GemmOperand& B, Ge
   p.valid_cols = valid_cols;
   p.seg_begin = valid_cols ? seg_begin : 0;
   p.seg_width = valid_cols ? seg_width : p.N;
-  TWIST_TRY(launch_gemm_bf16(layout, EPI_MSE, A, B, p, st));
+  TWIST_TRY(launch_gemm_bf16(layout, out ? EPI_MSE : EPI_MSE_NOY, A, B, p, st));
   return finish_fused_loss(p.dw, p.groups, p.M, p.N, valid_cols, p.seg_begin, p.seg_width, loss, st);
 }
 
