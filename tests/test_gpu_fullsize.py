@@ -1,5 +1,6 @@
 """Parity at the full sizes of the 7B-shaped workload (S=8, T=32768, d=4096, F=11008 -> f'=2752,
-8 of 32 heads), in the launch configuration bench.py times, on outputs the oracle can compute one
+8 of 32 heads) and of the TinyLlama-shaped one (S=4, T=32768, d=2048, F=5632 -> f'=2816, 16 of 32 heads in
+4 KV groups), in the launch configuration bench.py times, on outputs the oracle can compute one
 by one: sampled token rows of every activation, sampled weight rows of every fused-SGD update
 (full-length contractions over all 32768 tokens), whole blueprints, whole gathered slices of
 sampled subnets, and the whole aggregate.  Inputs are seeded draws made on the device; the oracle
@@ -16,7 +17,7 @@ from paper_2511_03983_b200 import inputs as I
 pytestmark = pytest.mark.gpu
 
 TOL = 2e-2
-SUBNETS = (1, 6)          # subnets whose activations / updates are checked
+SUBNETS = {4: (1, 6), 3: (0, 3)}   # subnets whose activations / updates are checked, per workload
 N_ROWS, N_WROWS = 40, 12  # sampled token rows, sampled weight rows
 
 
@@ -28,12 +29,12 @@ def f64(t):
     return t.detach().float().cpu().numpy().astype(np.float64)
 
 
-@pytest.fixture(scope="module")
-def setup():
+@pytest.fixture(scope="module", params=[4, 3])
+def setup(request):
     from paper_2511_03983_b200 import binding as B
     from paper_2511_03983_b200.engine import RoundEngine
     B.lib()
-    w = replace(I.PRESETS[4], n_layers=1, local_steps=1)
+    w = replace(I.PRESETS[request.param], n_layers=1, local_steps=1)
     eng = RoundEngine(w, keep_f32_full=True)
     gen = torch.Generator(device="cuda")
     gen.manual_seed(w.seed_w)
@@ -50,7 +51,11 @@ def setup():
     bp = o.layer_blueprints(w, 0, 0)
     rng = np.random.default_rng(5)
     rows = np.sort(rng.choice(T, N_ROWS, replace=False))
-    return dict(B=B, eng=eng, w=w, full=full_np, bp=bp, rows=rows, rng=rng, gen=gen, rnd=rnd)
+    # the device pads K / V to the maximum group count; these workloads keep every group, so the layouts coincide
+    assert np.all(bp["kv_count"] == eng.kv_max)
+    yield dict(B=B, eng=eng, w=w, full=full_np, bp=bp, rows=rows, rng=rng, gen=gen, rnd=rnd, subnets=SUBNETS[request.param])
+    del eng
+    torch.cuda.empty_cache()
 
 
 def test_blueprints_and_index_data_bit_exact(setup):
@@ -63,14 +68,14 @@ def test_blueprints_and_index_data_bit_exact(setup):
     c, _, p = o.cover_and_pos(bp["head"], w.n_heads)
     assert np.array_equal(eng.cover_head[0].cpu().numpy().view(np.uint32), c)
     assert np.array_equal(eng.pos_head[0].cpu().numpy(), p)
-    assert np.array_equal(eng.kv_idx[0].cpu().numpy()[:, : w.head_keep], bp["kv_idx"][:, : w.head_keep])
+    assert np.array_equal(eng.kv_idx[0].cpu().numpy(), bp["kv_idx"])
     assert np.array_equal(eng.kv_count[0].cpu().numpy(), bp["kv_count"])
 
 
 def test_gathered_slices_bit_exact(setup):
     eng, w, bp, full = setup["eng"], setup["w"], setup["bp"], setup["full"]
     f = w.f_sub
-    for s in SUBNETS:
+    for s in setup["subnets"]:
         sl = o.gather_layer(w, full, bp, s)
         want = {"w_gu": np.concatenate([sl["gate"], sl["up"]]), "w_down": sl["down"], "w_qkv": sl["qkv"], "w_o": sl["o"]}
         for name, arr in want.items():
@@ -97,7 +102,7 @@ def test_ffn_forward_backward_sampled(setup):
     B.twist_subnet_ffn_bwd(a)
     torch.cuda.synchronize()
     assert B.twist_device_status() == 0
-    for s in SUBNETS:
+    for s in setup["subnets"]:
         sl = _sl64(setup, s)
         X = f64(eng.X[0][s])
         dYs = f64(dY[s])
@@ -142,7 +147,7 @@ def test_projections_forward_backward_sampled(setup):
     torch.cuda.synchronize()
     assert B.twist_device_status() == 0
     r = torch.from_numpy(rows).cuda()
-    for s in SUBNETS:
+    for s in setup["subnets"]:
         sl = _sl64(setup, s)
         X, A = f64(eng.X[0][s]), f64(eng.A[0][s])
         dQs, dYs = f64(dQ[s]), f64(dYo[s])
@@ -166,7 +171,8 @@ def test_aggregate_whole_layer(setup):
         m.copy_(torch.randn(m.shape, generator=gen, device="cuda") * 0.02)
     eng.aggregate_layer(0)
     torch.cuda.synchronize()
-    f, a_sub, dh, H = w.f_sub, eng.a_sub, w.d_head, w.n_heads
+    f, a_sub, dh, H, Hkv = w.f_sub, eng.a_sub, w.d_head, w.n_heads, w.n_kv_heads
+    kvw = eng.kv_max * dh
     gu, down, qkv, wo = (t.cpu().numpy().astype(np.float64) for t in (eng.w_gu_m, eng.w_down_m, eng.w_qkv_m, eng.w_o_m))
     kvs = [bp["kv_idx"][s][: bp["kv_count"][s]] for s in range(S)]
     cases = [
@@ -174,8 +180,8 @@ def test_aggregate_whole_layer(setup):
         ("up", [gu[s, f:] for s in range(S)], bp["ffn"], 1, 0, slice(0, w.d_ff)),
         ("down", [down[s] for s in range(S)], bp["ffn"], 1, 0, slice(0, w.d_ff)),
         ("qkv", [qkv[s, :a_sub] for s in range(S)], bp["head"], dh, 0, slice(0, H * dh)),
-        ("qkv", [qkv[s, a_sub:2 * a_sub] for s in range(S)], kvs, dh, H * dh, slice(H * dh, 2 * H * dh)),
-        ("qkv", [qkv[s, 2 * a_sub:] for s in range(S)], kvs, dh, 2 * H * dh, slice(2 * H * dh, 3 * H * dh)),
+        ("qkv", [qkv[s, a_sub:a_sub + kvw] for s in range(S)], kvs, dh, H * dh, slice(H * dh, (H + Hkv) * dh)),
+        ("qkv", [qkv[s, a_sub + kvw:] for s in range(S)], kvs, dh, (H + Hkv) * dh, slice((H + Hkv) * dh, (H + 2 * Hkv) * dh)),
         ("o", [wo[s] for s in range(S)], bp["head"], dh, 0, slice(0, H * dh)),
     ]
     for name, subs, blue, br, off, rows in cases:
@@ -214,7 +220,7 @@ def test_fused_loss_at_full_size(setup):
     assert torch.equal(eng.dy, dy_b)
     assert torch.allclose(loss_a, loss_b, rtol=1e-5, atol=0)
     r = torch.from_numpy(rows).cuda()
-    for s in SUBNETS:
+    for s in setup["subnets"]:
         sl = _sl64(setup, s)
         Yw, _ = o.ffn_fwd(f64(eng.X[0][s][r]), sl["up"], sl["gate"], sl["down"], w.ffn_kind, eng.alpha_f, True)
         want_dy = o.round_bf16(2.0 * (Yw - f64(eng.Td[0][s][r])) / (T * d))
