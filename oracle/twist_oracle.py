@@ -296,6 +296,43 @@ def sgd(master, dW, lr, lowp):
     return new, _q(new, lowp)
 
 
+def adam(master, m, v, dW, step, lr, beta1, beta2, eps, lowp):
+    """One Adam step (the optimiser of the paper's experiments, Sec. 5 Setup), in its standard form:
+        m <- b1 m + (1 - b1) g,   v <- b2 v + (1 - b2) g^2,
+        w <- w - lr (m / (1 - b1^t)) / (sqrt(v / (1 - b2^t)) + eps),        t = step = 1, 2, ...
+    Returns (new master, new m, new v, compute copy in stored precision)."""
+    m = beta1 * m + (1.0 - beta1) * dW
+    v = beta2 * v + (1.0 - beta2) * dW * dW
+    m_hat = m / (1.0 - beta1 ** step)
+    v_hat = v / (1.0 - beta2 ** step)
+    new = master - lr * m_hat / (np.sqrt(v_hat) + eps)
+    return new, m, v, _q(new, lowp)
+
+
+class _Optimizer:
+    """Applies the workload's optimiser to a dict of masters.  Adam moments belong to the worker's copy of the
+    slice: they start at zero when the slices are dispatched and are not aggregated (the paper exchanges
+    parameters only)."""
+
+    def __init__(self, spec):
+        self.kind = getattr(spec, "optimizer", "sgd")
+        self.spec = spec
+        self.state = {}
+        self.t = 0
+
+    def begin_step(self):
+        self.t += 1
+
+    def update(self, key, master, dW, lowp):
+        sp = self.spec
+        if self.kind == "sgd":
+            return sgd(master, dW, sp.lr, lowp)[0]
+        m, v = self.state.get(key, (np.zeros_like(master), np.zeros_like(master)))
+        new, m, v, _ = adam(master, m, v, dW, self.t, sp.lr, sp.beta1, sp.beta2, sp.adam_eps, lowp)
+        self.state[key] = (m, v)
+        return new
+
+
 # ----------------------------------------------------------------------------------------
 # Aggregator (Sec. 3.3): p <- sum_i p_i 1[p in W_i] / sum_i 1[p in W_i].
 # ----------------------------------------------------------------------------------------
@@ -360,7 +397,9 @@ def local_steps_blockwise(spec, sl, get_batch, rnd, s, lowp):
     d = spec.d_model
     alpha_f = act_scale(spec.d_ff // spec.ffn_block, spec.ffn_keep)
     losses = {"ffn": [], "qkv": [], "o": []}
+    opt = _Optimizer(spec)
     for k in range(spec.local_steps):
+        opt.begin_step()
         X = get_batch(0, rnd, s, k, d).astype(np.float64)
         Td = get_batch(1, rnd, s, k, d).astype(np.float64)
         cw = {m: _q(v, lowp) for m, v in sl.items()}            # compute copies
@@ -368,10 +407,10 @@ def local_steps_blockwise(spec, sl, get_batch, rnd, s, lowp):
         loss, dY = mse(Y, Td, lowp)
         _, dWu, dWg, dWd = ffn_bwd(dY, X, saved, cw["up"], cw.get("gate"), cw["down"], spec.ffn_kind, alpha_f, lowp)
         losses["ffn"].append(loss)
-        sl["up"], _ = sgd(sl["up"], dWu, spec.lr, lowp)
-        sl["down"], _ = sgd(sl["down"], dWd, spec.lr, lowp)
+        sl["up"] = opt.update("up", sl["up"], dWu, lowp)
+        sl["down"] = opt.update("down", sl["down"], dWd, lowp)
         if dWg is not None:
-            sl["gate"], _ = sgd(sl["gate"], dWg, spec.lr, lowp)
+            sl["gate"] = opt.update("gate", sl["gate"], dWg, lowp)
         if spec.n_heads:
             alpha_a = act_scale(spec.n_heads, spec.head_keep)
             nq = sl["qkv"].shape[0]
@@ -380,13 +419,13 @@ def local_steps_blockwise(spec, sl, get_batch, rnd, s, lowp):
             loss, dQKV = mse(QKV, Tq, lowp)
             _, dWq = qkv_bwd(dQKV, X, cw["qkv"], lowp)
             losses["qkv"].append(loss)
-            sl["qkv"], _ = sgd(sl["qkv"], dWq, spec.lr, lowp)
+            sl["qkv"] = opt.update("qkv", sl["qkv"], dWq, lowp)
             A = get_batch(3, rnd, s, k, sl["o"].shape[0]).astype(np.float64)
             Yo = o_fwd(A, cw["o"], alpha_a, lowp)
             loss, dYo = mse(Yo, Td, lowp)
             _, dWo = o_bwd(dYo, A, cw["o"], alpha_a, lowp)
             losses["o"].append(loss)
-            sl["o"], _ = sgd(sl["o"], dWo, spec.lr, lowp)
+            sl["o"] = opt.update("o", sl["o"], dWo, lowp)
     return losses
 
 
@@ -542,7 +581,9 @@ def local_steps_stack(spec, slices, head_kv, get_batch, rnd, s, n_seqs, seq_len,
     """K local SGD steps of subnet s through the whole stack (masters `slices[l]`, float64,
     updated in place).  Batch kinds: 0 input X of width d, 1 target of width d.  Returns the losses."""
     losses = []
+    opt = _Optimizer(spec)
     for k in range(spec.local_steps):
+        opt.begin_step()
         X0 = get_batch(0, rnd, s, k, spec.d_model).astype(np.float64)
         Tgt = get_batch(1, rnd, s, k, spec.d_model).astype(np.float64)
         layers = [{m: _q(v, lowp) for m, v in sl.items()} for sl in slices]
@@ -550,9 +591,9 @@ def local_steps_stack(spec, slices, head_kv, get_batch, rnd, s, n_seqs, seq_len,
         loss, dX = mse(xL, Tgt, lowp)
         grads, _ = stack_bwd(spec, layers, head_kv, saved, dX, n_seqs, seq_len, lowp)
         losses.append(loss)
-        for sl, g in zip(slices, grads):
+        for l, (sl, g) in enumerate(zip(slices, grads)):
             for m in sl:
-                sl[m], _ = sgd(sl[m], g[m], spec.lr, lowp)
+                sl[m] = opt.update((l, m), sl[m], g[m], lowp)
     return losses
 
 

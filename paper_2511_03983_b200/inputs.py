@@ -51,6 +51,10 @@ class Workload:
     seed_mask: int = 3000
     common_ffn: Tuple[int, ...] = field(default_factory=tuple)
     common_heads: Tuple[int, ...] = field(default_factory=tuple)
+    optimizer: str = "sgd"   # "sgd" (the workloads) or "adam" (the optimiser of the paper's experiments)
+    beta1: float = 0.9
+    beta2: float = 0.999
+    adam_eps: float = 1e-8
     n_seqs: int = 1       # sequences per batch (tokens = n_seqs * sequence length); matters to the attention core only
 
     @property

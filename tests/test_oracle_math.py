@@ -374,3 +374,41 @@ def test_lowp_mirror_stays_close_to_exact_and_is_bf16_representable():
     assert np.linalg.norm(Y - Ye) / np.linalg.norm(Ye) < 1e-2
     for a in (Y, saved["G"], saved["U"], saved["Hh"]):
         assert np.array_equal(o.round_bf16(a), a)
+
+
+# ------------------------------------------------------------------ Adam (the optimiser of the paper's experiments)
+
+def test_adam_steps_match_torch_optim_adam():
+    r = _rng(40)
+    w0 = r.standard_normal((5, 7))
+    grads = [r.standard_normal((5, 7)) * s for s in (1.0, 1e-3, 5.0, 0.0, 2.0)]
+    lr, b1, b2, eps = 3e-2, 0.9, 0.95, 1e-8
+    wt = torch.from_numpy(w0.copy()).requires_grad_(True)
+    opt = torch.optim.Adam([wt], lr=lr, betas=(b1, b2), eps=eps)
+    w, m, v = w0.copy(), np.zeros_like(w0), np.zeros_like(w0)
+    for t, g in enumerate(grads, start=1):
+        wt.grad = torch.from_numpy(g.copy())
+        opt.step()
+        w, m, v, _ = o.adam(w, m, v, g, t, lr, b1, b2, eps, lowp=False)
+        assert np.allclose(w, wt.detach().numpy(), rtol=1e-12, atol=1e-14), t
+
+
+def test_blockwise_local_steps_with_adam_equal_torch_adam_on_the_dense_model():
+    """S = 1 keeping everything, K = 3 steps with Adam = 3 torch.optim.Adam steps on the dense FFN block."""
+    spec = SimpleNamespace(d_model=6, d_ff=10, ffn_block=1, ffn_keep=10, ffn_kind=o.FFN_GELU, n_heads=0, local_steps=3,
+                           lr=1e-2, optimizer="adam", beta1=0.9, beta2=0.999, adam_eps=1e-8)
+    r = _rng(41)
+    sl = {"up": r.standard_normal((10, 6)) * 0.3, "down": r.standard_normal((10, 6)) * 0.3}
+    batches = {(kind, k): r.standard_normal((9, 6)) for kind in (0, 1) for k in range(3)}
+    tw = {m: torch.from_numpy(v.copy()).requires_grad_(True) for m, v in sl.items()}
+    losses = o.local_steps_blockwise(spec, sl, lambda kind, rnd, s, k, w: batches[(kind, k)], 0, 0, lowp=False)
+    opt = torch.optim.Adam(list(tw.values()), lr=1e-2, betas=(0.9, 0.999), eps=1e-8)
+    for k in range(3):
+        X, Tg = torch.from_numpy(batches[(0, k)]), torch.from_numpy(batches[(1, k)])
+        loss = torch.mean((torch.nn.functional.gelu(X @ tw["up"].T) @ tw["down"] - Tg) ** 2)
+        assert abs(loss.item() - losses["ffn"][k]) < 1e-12
+        opt.zero_grad()
+        loss.backward()
+        opt.step()
+    for m in sl:
+        assert np.allclose(sl[m], tw[m].detach().numpy(), rtol=1e-9, atol=1e-12), m
