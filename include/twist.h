@@ -177,6 +177,18 @@ int32_t twist_aggregate(const twist_aggregate_segment* segs /*host*/, int32_t n_
  *   dX = dpre W_gu;  dW_gu = dpre^T X;  dW_down = out_scale * hh^T dY;
  *   if lr != 0:  master -= lr * dW (fp32), compute copy = round(master)   [plain SGD]
  */
+/* Optimiser of the fused weight update.  TWIST_OPT_SGD (the zero-initialised default): w <- w - lr dW.
+ * TWIST_OPT_ADAM (the optimiser of the paper's experiments, Sec. 5 Setup; bf16 dtype only), in its standard form:
+ *   m <- beta1 m + (1 - beta1) g;  v <- beta2 v + (1 - beta2) g^2;
+ *   w <- w - lr (m / (1 - beta1^step)) / (sqrt(v / (1 - beta2^step)) + eps),   step = 1, 2, ... within a round.
+ * The moments are fp32 arrays shaped like the masters, owned by the caller; they belong to the worker's copy of
+ * the slice: zero them when the slices are gathered (the paper exchanges parameters only, never optimiser state). */
+enum { TWIST_OPT_SGD = 0, TWIST_OPT_ADAM = 1 };
+typedef struct {
+  int32_t kind, step;
+  float beta1, beta2, eps;
+} twist_optimizer;
+
 typedef struct {
   int32_t ffn_kind, dtype, n_subnets, tokens, d_model, f_sub;
   float out_scale, lr;
@@ -204,6 +216,9 @@ typedef struct {
    * Not combinable with the fused loss. */
   const void* y_residual;   /* device [S][T][d] */
   const void* dx_residual;  /* device [S][T][d] */
+  twist_optimizer opt;      /* bwd: optimiser of the fused update */
+  float *m_gu, *v_gu;       /* device fp32 Adam moments of w_gu   [S][g*f_sub][d] */
+  float *m_down, *v_down;   /* device fp32 Adam moments of w_down [S][f_sub][d] */
 } twist_ffn_args;
 
 /* Fused loss.  When `tgt` is set, twist_subnet_ffn_fwd / twist_subnet_attn_proj_fwd also evaluate the loss
@@ -244,6 +259,8 @@ typedef struct {
    * TWIST_PROJ_QKV bwd: d_in = d_in_residual + d_out W.  NULL: no addend.  Not combinable with the fused loss. */
   const void* out_residual;    /* device [S][T][d] */
   const void* d_in_residual;   /* device [S][T][d] */
+  twist_optimizer opt;         /* bwd: optimiser of the fused update */
+  float *m, *v;                /* device fp32 Adam moments of w [S][n][d] */
 } twist_proj_args;
 
 int32_t twist_subnet_attn_proj_fwd(const twist_proj_args* a /*host*/, void* stream);

@@ -53,6 +53,17 @@ class AggregateSegment(C.Structure):
                 ("sub_subnet_stride", C.c_int64), ("sub_row_offset", C.c_int64)]
 
 
+class Optimizer(C.Structure):
+    _fields_ = [("kind", C.c_int32), ("step", C.c_int32), ("beta1", C.c_float), ("beta2", C.c_float), ("eps", C.c_float)]
+
+
+OPT_SGD, OPT_ADAM = 0, 1
+
+
+def adam(step: int, beta1: float = 0.9, beta2: float = 0.999, eps: float = 1e-8) -> Optimizer:
+    return Optimizer(OPT_ADAM, step, beta1, beta2, eps)
+
+
 class FfnArgs(C.Structure):
     _fields_ = [("ffn_kind", C.c_int32), ("dtype", C.c_int32), ("n_subnets", C.c_int32), ("tokens", C.c_int32),
                 ("d_model", C.c_int32), ("f_sub", C.c_int32), ("out_scale", C.c_float), ("lr", C.c_float),
@@ -60,7 +71,9 @@ class FfnArgs(C.Structure):
                 ("w_down_master", C.c_void_p), ("pre", C.c_void_p), ("hh", C.c_void_p), ("y", C.c_void_p),
                 ("dy", C.c_void_p), ("dpre", C.c_void_p), ("dx", C.c_void_p), ("dw_gu", C.c_void_p),
                 ("dw_down", C.c_void_p), ("tgt", C.c_void_p), ("loss", C.c_void_p), ("loss_ws", C.c_void_p),
-                ("loss_ws_bytes", C.c_size_t), ("y_residual", C.c_void_p), ("dx_residual", C.c_void_p)]
+                ("loss_ws_bytes", C.c_size_t), ("y_residual", C.c_void_p), ("dx_residual", C.c_void_p),
+                ("opt", Optimizer), ("m_gu", C.c_void_p), ("v_gu", C.c_void_p), ("m_down", C.c_void_p),
+                ("v_down", C.c_void_p)]
 
 
 class ProjArgs(C.Structure):
@@ -70,7 +83,8 @@ class ProjArgs(C.Structure):
                 ("d_out", C.c_void_p), ("d_in", C.c_void_p), ("dw", C.c_void_p), ("tgt", C.c_void_p),
                 ("loss", C.c_void_p), ("loss_ws", C.c_void_p), ("loss_ws_bytes", C.c_size_t),
                 ("valid_cols", C.c_void_p), ("seg_begin", C.c_int32), ("seg_width", C.c_int32),
-                ("out_residual", C.c_void_p), ("d_in_residual", C.c_void_p)]
+                ("out_residual", C.c_void_p), ("d_in_residual", C.c_void_p), ("opt", Optimizer), ("m", C.c_void_p),
+                ("v", C.c_void_p)]
 
 
 class AttnCoreArgs(C.Structure):
@@ -201,14 +215,19 @@ def _ws_bytes(ws) -> int:
     return 0 if ws is None else ws.numel() * ws.element_size()
 
 
-def ffn_args(ffn_kind, dtype, n_subnets, tokens, d_model, f_sub, out_scale, lr=0.0, **t) -> FfnArgs:
+def ffn_args(ffn_kind, dtype, n_subnets, tokens, d_model, f_sub, out_scale, lr=0.0, opt: Optional[Optimizer] = None,
+             **t) -> FfnArgs:
     """Marshals twist_ffn_args.  tgt / loss / loss_ws request the fused loss of the forward call."""
     names = ["x", "w_gu", "w_down", "w_gu_master", "w_down_master", "pre", "hh", "y", "dy", "dpre", "dx", "dw_gu",
              "dw_down", "tgt", "loss", "loss_ws"]
-    unknown = set(t) - set(names) - {"y_residual", "dx_residual"}
+    moments = ["m_gu", "v_gu", "m_down", "v_down"]
+    unknown = set(t) - set(names) - {"y_residual", "dx_residual"} - set(moments)
     assert not unknown, unknown
-    return FfnArgs(ffn_kind, dtype, n_subnets, tokens, d_model, f_sub, out_scale, lr, *[_ptr(t.get(n)) for n in names],
-                   _ws_bytes(t.get("loss_ws")), _ptr(t.get("y_residual")), _ptr(t.get("dx_residual")))
+    a = FfnArgs(ffn_kind, dtype, n_subnets, tokens, d_model, f_sub, out_scale, lr, *[_ptr(t.get(n)) for n in names],
+                _ws_bytes(t.get("loss_ws")), _ptr(t.get("y_residual")), _ptr(t.get("dx_residual")),
+                opt if opt is not None else Optimizer(), *[_ptr(t.get(n)) for n in moments])
+    a._keepalive = list(t.values())      # the struct holds raw addresses: keep the tensors alive as long as it lives
+    return a
 
 
 def twist_subnet_ffn_fwd(a: FfnArgs):
@@ -219,15 +238,19 @@ def twist_subnet_ffn_bwd(a: FfnArgs):
     _check(lib().twist_subnet_ffn_bwd(C.byref(a), _stream()), "twist_subnet_ffn_bwd")
 
 
-def proj_args(which, dtype, n_subnets, tokens, d_model, n, out_scale, lr=0.0, seg_begin=0, seg_width=0, **t) -> ProjArgs:
+def proj_args(which, dtype, n_subnets, tokens, d_model, n, out_scale, lr=0.0, seg_begin=0, seg_width=0,
+              opt: Optional[Optimizer] = None, **t) -> ProjArgs:
     """Marshals twist_proj_args.  tgt / loss / loss_ws (and the optional column mask valid_cols,
     seg_begin, seg_width) request the fused loss of the forward call."""
     names = ["in_", "w", "w_master", "out", "d_out", "d_in", "dw", "tgt", "loss", "loss_ws"]
-    unknown = set(t) - set(names) - {"valid_cols", "out_residual", "d_in_residual"}
+    unknown = set(t) - set(names) - {"valid_cols", "out_residual", "d_in_residual", "m", "v"}
     assert not unknown, unknown
-    return ProjArgs(which, dtype, n_subnets, tokens, d_model, n, out_scale, lr, *[_ptr(t.get(n)) for n in names],
-                    _ws_bytes(t.get("loss_ws")), _ptr(t.get("valid_cols")), seg_begin, seg_width,
-                    _ptr(t.get("out_residual")), _ptr(t.get("d_in_residual")))
+    a = ProjArgs(which, dtype, n_subnets, tokens, d_model, n, out_scale, lr, *[_ptr(t.get(n)) for n in names],
+                 _ws_bytes(t.get("loss_ws")), _ptr(t.get("valid_cols")), seg_begin, seg_width,
+                 _ptr(t.get("out_residual")), _ptr(t.get("d_in_residual")), opt if opt is not None else Optimizer(),
+                 _ptr(t.get("m")), _ptr(t.get("v")))
+    a._keepalive = list(t.values())
+    return a
 
 
 def twist_subnet_attn_proj_fwd(a: ProjArgs):
@@ -243,8 +266,10 @@ def attn_core_args(dtype, n_subnets, n_seqs, seq_len, head_keep, kv_max, d_head,
     names = ["qkv", "out", "lse", "d_out", "d_qkv", "delta", "head_idx", "kv_pos", "kv_count"]
     unknown = set(t) - set(names)
     assert not unknown, unknown
-    return AttnCoreArgs(dtype, n_subnets, n_seqs, seq_len, head_keep, kv_max, d_head, n_heads, n_kv_heads,
-                        *[_ptr(t.get(n)) for n in names])
+    a = AttnCoreArgs(dtype, n_subnets, n_seqs, seq_len, head_keep, kv_max, d_head, n_heads, n_kv_heads,
+                     *[_ptr(t.get(n)) for n in names])
+    a._keepalive = list(t.values())
+    return a
 
 
 def twist_attn_core_fwd(a: AttnCoreArgs):

@@ -52,12 +52,12 @@ int resident_pairs(int* out) {
   if (dev < 0 || dev >= 64) return TWIST_ERR_UNSUPPORTED;
   if (cached[dev] == 0) {
     TWIST_CUDA_TRY(cudaFuncSetAttribute(gemm_kernel<AM, BM_, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                        gemm_smem_bytes(EPI != EPI_SGD)));
+                                        gemm_smem_bytes(EPI != EPI_SGD && EPI != EPI_ADAM)));
     cudaLaunchConfig_t cfg;
     memset(&cfg, 0, sizeof(cfg));
     cfg.gridDim = dim3(2 * (sm_count() / 2));
     cfg.blockDim = dim3(kGemmThreads);
-    cfg.dynamicSmemBytes = gemm_smem_bytes(EPI != EPI_SGD);
+    cfg.dynamicSmemBytes = gemm_smem_bytes(EPI != EPI_SGD && EPI != EPI_ADAM);
     cudaLaunchAttribute attr;
     attr.id = cudaLaunchAttributeClusterDimension;
     attr.val.clusterDim.x = 2; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
@@ -130,7 +130,7 @@ int launch(const CUtensorMap& ta, const CUtensorMap& tb, const GemmParams& p, cu
   EpiMaps te;
   rc = make_epilogue_maps(EPI, p, ta, &te);
   if (rc != TWIST_OK) return rc;
-  gemm_kernel<AM, BM_, EPI><<<grid, kGemmThreads, gemm_smem_bytes(EPI != EPI_SGD), st>>>(ta, tb, te, p);
+  gemm_kernel<AM, BM_, EPI><<<grid, kGemmThreads, gemm_smem_bytes(EPI != EPI_SGD && EPI != EPI_ADAM), st>>>(ta, tb, te, p);
   TWIST_LAUNCH_CHECK();
   return TWIST_OK;
 }
@@ -219,6 +219,7 @@ int launch_gemm_bf16(int layout, int epi, const GemmOperand& A, const GemmOperan
   if (layout == 1 && epi == EPI_MSE_NOY) return launch<MAJOR_K, MAJOR_MN, EPI_MSE_NOY>(ta, tb, p, st);
   if (layout == 1 && epi == EPI_RESID) return launch<MAJOR_K, MAJOR_MN, EPI_RESID>(ta, tb, p, st);
   if (layout == 2 && epi == EPI_SGD) return launch<MAJOR_MN, MAJOR_MN, EPI_SGD>(ta, tb, p, st);
+  if (layout == 2 && epi == EPI_ADAM) return launch<MAJOR_MN, MAJOR_MN, EPI_ADAM>(ta, tb, p, st);
   return TWIST_ERR_UNSUPPORTED;
 }
 

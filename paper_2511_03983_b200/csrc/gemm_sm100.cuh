@@ -33,7 +33,8 @@ namespace twist {
 
 enum { MAJOR_K = 0, MAJOR_MN = 1 };
 enum { EPI_STORE = 0, EPI_SWIGLU_FWD = 1, EPI_ACT_FWD = 2, EPI_DSWIGLU = 3, EPI_DACT = 4, EPI_SGD = 5, EPI_MSE = 6, EPI_RESID = 7,
-       EPI_MSE_NOY = 8 /* EPI_MSE without storing D: one box per chunk, so twice as many chunk buffers */ };
+       EPI_MSE_NOY = 8 /* EPI_MSE without storing D: one box per chunk, so twice as many chunk buffers */,
+       EPI_ADAM = 9 /* weight gradient with the Adam update fused, like EPI_SGD */ };
 
 constexpr int kBM = 256, kBN = 256, kBK = 64, kUmmaK = 16;   // tile of a CTA pair
 constexpr int kCtaM = kBM / 2, kCtaN = kBN / 2;   // rows of A / columns of B that one CTA of the pair loads
@@ -68,6 +69,9 @@ struct GemmParams {
   __nv_bfloat16* out1;  // *_FWD: hh [g][M][f_sub].  MSE: gradient of the loss w.r.t. D, [g][M][N]
   const __nv_bfloat16* in0;   // DSWIGLU / DACT: pre.  MSE: target [g][M][N].  RESID: addend [g][M][N]
   float* master;        // SGD: fp32 master weights [g][M][N] (updated when lr != 0)
+  float* adam_m;        // ADAM: first / second moment of the group's weights, fp32 [g][M][N]
+  float* adam_v;
+  float beta1, beta2, adam_eps, bias1, bias2;   // ADAM: decay rates, epsilon, 1 / (1 - beta^t)
   float* dw;            // SGD: optional fp32 gradient dump [g][M][N].  MSE: partial sums, 8 per tile (2 CTAs x 4 warps)
   const int32_t* valid_cols;   // MSE: valid columns per column group and subnet [groups], or null (all valid)
   int seg_begin, seg_width;    // MSE: columns [0, seg_begin) valid, then groups of seg_width columns (see twist_mse_fwd_bwd)
@@ -199,7 +203,7 @@ template <int A_MAJOR, int B_MAJOR, int EPI>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
             const __grid_constant__ EpiMaps tmE, const GemmParams p) {
-  constexpr bool kStaged = EPI != EPI_SGD;
+  constexpr bool kStaged = EPI != EPI_SGD && EPI != EPI_ADAM;
   constexpr int kStages = gemm_stages(kStaged);
   extern __shared__ unsigned char smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -327,7 +331,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     uint32_t tl = 0;
     bool ok = true;
 
-    if constexpr (EPI == EPI_SGD) {
+    if constexpr (EPI == EPI_SGD || EPI == EPI_ADAM) {
       // Weight-gradient tiles (contraction over all tokens, so this epilogue is rare): plain vector accesses
       // to the fp32 master rows; the master values of the next chunk are loaded ahead.
       for (int tile = pair; ok && tile < total_tiles; tile += num_pairs, ++tl) {
@@ -372,9 +376,26 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                 const float4 gq = make_float4(p.scale * __uint_as_float(r[4 * q]), p.scale * __uint_as_float(r[4 * q + 1]),
                                               p.scale * __uint_as_float(r[4 * q + 2]), p.scale * __uint_as_float(r[4 * q + 3]));
                 if (dw) *reinterpret_cast<float4*>(dw + 4 * q) = gq;
-                if (p.lr != 0.f) {      // master -= lr * dW (fp32); compute copy = bf16(master)
+                if (p.lr != 0.f) {      // master -= lr * step (fp32); compute copy = bf16(master)
                   float4 m = mv[c & 1][q];
-                  m.x -= p.lr * gq.x; m.y -= p.lr * gq.y; m.z -= p.lr * gq.z; m.w -= p.lr * gq.w;
+                  if constexpr (EPI == EPI_ADAM) {
+                    // m1 <- b1 m1 + (1 - b1) g;  m2 <- b2 m2 + (1 - b2) g^2;  step = (m1 / (1 - b1^t)) / (sqrt(m2 / (1 - b2^t)) + eps)
+                    float* pm1 = p.adam_m + grow * p.N + n + 4 * q;
+                    float* pm2 = p.adam_v + grow * p.N + n + 4 * q;
+                    float4 m1 = *reinterpret_cast<const float4*>(pm1), m2 = *reinterpret_cast<const float4*>(pm2);
+                    const float gv[4] = {gq.x, gq.y, gq.z, gq.w};
+                    float* a1 = &m1.x; float* a2 = &m2.x; float* wv = &m.x;
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                      a1[e] = fmaf(p.beta1, a1[e], (1.f - p.beta1) * gv[e]);
+                      a2[e] = fmaf(p.beta2, a2[e], (1.f - p.beta2) * gv[e] * gv[e]);
+                      wv[e] -= p.lr * (a1[e] * p.bias1) / (sqrtf(a2[e] * p.bias2) + p.adam_eps);
+                    }
+                    *reinterpret_cast<float4*>(pm1) = m1;
+                    *reinterpret_cast<float4*>(pm2) = m2;
+                  } else {
+                    m.x -= p.lr * gq.x; m.y -= p.lr * gq.y; m.z -= p.lr * gq.z; m.w -= p.lr * gq.w;
+                  }
                   *reinterpret_cast<float4*>(master + 4 * q) = m;
                   *reinterpret_cast<uint2*>(w16 + 4 * q) = make_uint2(pack2(m.x, m.y), pack2(m.z, m.w));
                 }

@@ -2,6 +2,8 @@
 // S subnets on their dense slices (FFN of App. A: y = C act(W x); projections of the multi-head
 // attention definition).  bf16: grouped tcgen05 GEMMs with fused epilogues.  fp32: plain SIMT
 // kernels (tiny correctness workload only).
+#include <math.h>
+
 #include "gemm_sm100.cuh"
 #include "glue.cuh"
 
@@ -49,6 +51,21 @@ int launch_fused_loss(int layout, const GemmOperand& A, const GemmOperand& B, Ge
   p.seg_width = valid_cols ? seg_width : p.N;
   TWIST_TRY(launch_gemm_bf16(layout, out ? EPI_MSE : EPI_MSE_NOY, A, B, p, st));
   return finish_fused_loss(p.dw, p.groups, p.M, p.N, valid_cols, p.seg_begin, p.seg_width, loss, st);
+}
+
+// Fills the optimiser part of a weight-gradient launch; returns the epilogue to use or a negative status.
+int optimizer_epilogue(const twist_optimizer& o, float lr, float* m, float* v, GemmParams* p) {
+  if (o.kind == TWIST_OPT_SGD) return EPI_SGD;
+  if (o.kind != TWIST_OPT_ADAM) return TWIST_ERR_SHAPE;
+  if (lr == 0.f) return EPI_SGD;                                   // nothing to update: plain gradient launch
+  if (!m || !v) return TWIST_ERR_NULL;
+  if (o.step < 1 || !(o.beta1 >= 0.f && o.beta1 < 1.f) || !(o.beta2 >= 0.f && o.beta2 < 1.f) || !(o.eps >= 0.f))
+    return TWIST_ERR_SHAPE;
+  p->adam_m = m; p->adam_v = v;
+  p->beta1 = o.beta1; p->beta2 = o.beta2; p->adam_eps = o.eps;
+  p->bias1 = (float)(1.0 / (1.0 - pow((double)o.beta1, (double)o.step)));
+  p->bias2 = (float)(1.0 / (1.0 - pow((double)o.beta2, (double)o.step)));
+  return EPI_ADAM;
 }
 
 GemmParams base_params(int M, int N, int K, int groups, float scale) {
@@ -123,7 +140,7 @@ extern "C" int32_t twist_subnet_ffn_bwd(const twist_ffn_args* a, void* stream) {
   const int gf = swiglu ? 2 * f : f;
   if (a->dtype == TWIST_FP32) {
     if (!a->dw_gu || !a->dw_down) return TWIST_ERR_NULL;
-    if (a->dx_residual) return TWIST_ERR_UNSUPPORTED;
+    if (a->dx_residual || a->opt.kind != TWIST_OPT_SGD) return TWIST_ERR_UNSUPPORTED;
     const float* x = static_cast<const float*>(a->x);
     const float* dy = static_cast<const float*>(a->dy);
     const float* pre = static_cast<const float*>(a->pre);
@@ -171,14 +188,18 @@ extern "C" int32_t twist_subnet_ffn_bwd(const twist_ffn_args* a, void* stream) {
   r.master = a->w_down_master;
   r.dw = a->dw_down;
   r.lr = a->lr;
-  TWIST_TRY(launch_gemm_bf16(2, EPI_SGD, GemmOperand{a->hh, T, f}, GemmOperand{a->dy, T, d}, r, st));
+  int epi = optimizer_epilogue(a->opt, a->lr, a->m_down, a->v_down, &r);
+  if (epi < 0) return epi;
+  TWIST_TRY(launch_gemm_bf16(2, epi, GemmOperand{a->hh, T, f}, GemmOperand{a->dy, T, d}, r, st));
   // dW_gu = dpre^T X, fused SGD
   GemmParams u = base_params(gf, d, T, S, 1.f);
   u.out0 = static_cast<__nv_bfloat16*>(a->w_gu);
   u.master = a->w_gu_master;
   u.dw = a->dw_gu;
   u.lr = a->lr;
-  return launch_gemm_bf16(2, EPI_SGD, GemmOperand{a->dpre, T, gf}, GemmOperand{a->x, T, d}, u, st);
+  epi = optimizer_epilogue(a->opt, a->lr, a->m_gu, a->v_gu, &u);
+  if (epi < 0) return epi;
+  return launch_gemm_bf16(2, epi, GemmOperand{a->dpre, T, gf}, GemmOperand{a->x, T, d}, u, st);
 }
 
 static int check_proj(const twist_proj_args* a) {
@@ -237,7 +258,7 @@ extern "C" int32_t twist_subnet_attn_proj_bwd(const twist_proj_args* a, void* st
   const int w_out = qkv ? n : d;      // width of `d_out`
   if (a->dtype == TWIST_FP32) {
     if (!a->dw) return TWIST_ERR_NULL;
-    if (a->d_in_residual) return TWIST_ERR_UNSUPPORTED;
+    if (a->d_in_residual || a->opt.kind != TWIST_OPT_SGD) return TWIST_ERR_UNSUPPORTED;
     const float* in = static_cast<const float*>(a->in);
     const float* dout = static_cast<const float*>(a->d_out);
     float* w = static_cast<float*>(a->w);
@@ -278,6 +299,8 @@ extern "C" int32_t twist_subnet_attn_proj_bwd(const twist_proj_args* a, void* st
   r.master = a->w_master;
   r.dw = a->dw;
   r.lr = a->lr;
-  if (qkv) return launch_gemm_bf16(2, EPI_SGD, GemmOperand{a->d_out, T, w_out}, GemmOperand{a->in, T, w_in}, r, st);
-  return launch_gemm_bf16(2, EPI_SGD, GemmOperand{a->in, T, w_in}, GemmOperand{a->d_out, T, w_out}, r, st);
+  const int epi = optimizer_epilogue(a->opt, a->lr, a->m, a->v, &r);
+  if (epi < 0) return epi;
+  if (qkv) return launch_gemm_bf16(2, epi, GemmOperand{a->d_out, T, w_out}, GemmOperand{a->in, T, w_in}, r, st);
+  return launch_gemm_bf16(2, epi, GemmOperand{a->in, T, w_in}, GemmOperand{a->d_out, T, w_out}, r, st);
 }

@@ -82,6 +82,15 @@ class RoundEngine:
         if self.has_attn:
             self.w_qkv, self.w_qkv_m = sl(self.nq)
             self.w_o, self.w_o_m = sl(self.a_sub)
+        # Adam moments live with the worker's copy of the slice: allocated here, zeroed at every gather
+        self.adam = w.optimizer == "adam"
+        assert not self.adam or bf16, "the fused Adam update exists for the bf16 dtype"
+        self.moment_names = []
+        if self.adam:
+            for n in ("w_gu", "w_down") + (("w_qkv", "w_o") if self.has_attn else ()):
+                for tag in ("_m1", "_m2"):
+                    setattr(self, n + tag, torch.zeros_like(getattr(self, n + "_m")))
+                    self.moment_names.append(n + tag)
         # activations of one (layer, step)
         act = lambda width: torch.empty(S, T, width, dtype=td, device=dev)
         self.pre, self.dpre, self.hh = act(gf), act(gf), act(f)
@@ -167,6 +176,8 @@ class RoundEngine:
                                          w.head_keep, dh, 0, self.a_sub * d, 0))
         with self._timed("gather"):
             B.twist_gather_subnets(segs, w.n_subnets, d, w.dtype)
+            for n in self.moment_names:        # a fresh worker state: first and second moments start at zero
+                getattr(self, n).zero_()
         self.launches += 1
 
     def aggregate_layer(self, l: int, live: int = 0xFFFFFFFF, which=("ffn", "attn")):
@@ -201,6 +212,17 @@ class RoundEngine:
             B.twist_aggregate(segs, w.n_subnets, d, w.dtype, live)
         self.launches += 1
 
+    def _opt(self, k: int, *names):
+        """Optimiser arguments of local step k (0-based) for the slices `names`: (opt, moments...) keyword args."""
+        if not self.adam:
+            return {}
+        w = self.w
+        kw = {"opt": B.adam(k + 1, w.beta1, w.beta2, w.adam_eps)}
+        for arg, n in names:
+            kw["m" + arg] = getattr(self, n + "_m1")
+            kw["v" + arg] = getattr(self, n + "_m2")
+        return kw
+
     def _mse(self, y, tgt, dy, loss, width, valid_cols=None, seg_begin=0, seg_width=0):
         w = self.w
         with self._timed("mse"):
@@ -216,7 +238,8 @@ class RoundEngine:
                        x=self.X[k], w_gu=self.w_gu, w_down=self.w_down, w_gu_master=self.w_gu_m,
                        w_down_master=self.w_down_m, pre=self.pre, hh=self.hh,
                        y=self.y if self.store_outputs else None, dy=self.dy, dpre=self.dpre,
-                       dx=self.dx, dw_gu=self.dw_gu, dw_down=self.dw_down, **fused)
+                       dx=self.dx, dw_gu=self.dw_gu, dw_down=self.dw_down, **fused,
+                       **self._opt(k, ("_gu", "w_gu"), ("_down", "w_down")))
         with self._timed("ffn_fwd"):
             B.twist_subnet_ffn_fwd(a)
         if self.fuse_loss:
@@ -236,7 +259,7 @@ class RoundEngine:
         fused = dict(tgt=self.Tq[k], loss=self.loss[l, 1, k], loss_ws=self.ws, **mask) if self.fuse_loss else {}
         a = B.proj_args(B.PROJ_QKV, w.dtype, w.n_subnets, w.tokens, w.d_model, self.nq, 1.0, lr, in_=self.X[k],
                         w=self.w_qkv, w_master=self.w_qkv_m, out=self.qkv_out if self.store_outputs else None,
-                        d_out=self.dqkv, d_in=self.dx, dw=self.dw_qkv, **fused)
+                        d_out=self.dqkv, d_in=self.dx, dw=self.dw_qkv, **fused, **self._opt(k, ("", "w_qkv")))
         with self._timed("qkv_fwd"):
             B.twist_subnet_attn_proj_fwd(a)
         if self.fuse_loss:
@@ -254,7 +277,7 @@ class RoundEngine:
         fused = dict(tgt=self.Td[k], loss=self.loss[l, 2, k], loss_ws=self.ws) if self.fuse_loss else {}
         a = B.proj_args(B.PROJ_O, w.dtype, w.n_subnets, w.tokens, w.d_model, self.a_sub, self.alpha_a, lr,
                         in_=self.A[k], w=self.w_o, w_master=self.w_o_m, out=self.y if self.store_outputs else None,
-                        d_out=self.dy, d_in=self.da, dw=self.dw_o, **fused)
+                        d_out=self.dy, d_in=self.da, dw=self.dw_o, **fused, **self._opt(k, ("", "w_o")))
         with self._timed("o_fwd"):
             B.twist_subnet_attn_proj_fwd(a)
         if self.fuse_loss:
@@ -297,7 +320,7 @@ class StackEngine(RoundEngine):
         S, T, d, L = w.n_subnets, w.tokens, w.d_model, w.n_layers
         gf, f = self.g * w.f_sub, w.f_sub
         dev, bf = self.dev, torch.bfloat16
-        names = ("w_gu", "w_gu_m", "w_down", "w_down_m", "w_qkv", "w_qkv_m", "w_o", "w_o_m")
+        names = ("w_gu", "w_gu_m", "w_down", "w_down_m", "w_qkv", "w_qkv_m", "w_o", "w_o_m") + tuple(self.moment_names)
         self.slices = [{n: (getattr(self, n) if l == 0 else torch.empty_like(getattr(self, n))) for n in names}
                        for l in range(L)]
         act = lambda width: torch.empty(S, T, width, dtype=bf, device=dev)
@@ -356,18 +379,19 @@ class StackEngine(RoundEngine):
                                                   x=self.x_mid[l], w_gu=self.w_gu, w_down=self.w_down,
                                                   w_gu_master=self.w_gu_m, w_down_master=self.w_down_m,
                                                   pre=self.pre_l[l], hh=self.hh_l[l], dy=g, dpre=self.dpre, dx=g_mid,
-                                                  dx_residual=g, dw_gu=self.dw_gu, dw_down=self.dw_down))
+                                                  dx_residual=g, dw_gu=self.dw_gu, dw_down=self.dw_down,
+                                                  **self._opt(k, ("_gu", "w_gu"), ("_down", "w_down"))))
             with self._timed("o_bwd"):
                 B.twist_subnet_attn_proj_bwd(B.proj_args(B.PROJ_O, w.dtype, S, T, d, self.a_sub, self.alpha_a, lr,
                                                          in_=self.a_l[l], w=self.w_o, w_master=self.w_o_m, d_out=g_mid,
-                                                         d_in=self.da, dw=self.dw_o))
+                                                         d_in=self.da, dw=self.dw_o, **self._opt(k, ("", "w_o"))))
             with self._timed("core_bwd"):
                 B.twist_attn_core_bwd(self._core_args(l, qkv=self.qkv_l[l], out=self.a_l[l], lse=self.lse[l],
                                                       d_out=self.da, d_qkv=self.dqkv, delta=self.delta))
             with self._timed("qkv_bwd"):
                 B.twist_subnet_attn_proj_bwd(B.proj_args(B.PROJ_QKV, w.dtype, S, T, d, self.nq, 1.0, lr, in_=self.x[l],
                                                          w=self.w_qkv, w_master=self.w_qkv_m, d_out=self.dqkv, d_in=g,
-                                                         d_in_residual=g_mid, dw=self.dw_qkv))
+                                                         d_in_residual=g_mid, dw=self.dw_qkv, **self._opt(k, ("", "w_qkv"))))
             self.launches += 4 + 2 + 3 + 2
 
     def local_step(self, k: int, lr: Optional[float] = None):

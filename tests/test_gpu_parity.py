@@ -487,3 +487,87 @@ def test_round_with_zero_lr_is_identity_on_the_bf16_model(B):
     torch.cuda.synchronize()
     for m in before:      # aggregation of identical (untrained) subnets is the identity
         assert torch.equal(before[m], eng.full[m]), m
+
+
+# --------------------------------------------------------------------------------------------- Adam
+
+def test_fused_adam_update_matches_the_oracle(B):
+    """Two consecutive steps of the fused Adam update (FFN block).  The moments are linear /
+    quadratic in the gradient, so they carry the 2e-2 bar; the weight step, which is close to a sign function of
+    the gradient where the gradient is small, is checked exactly against the formula applied to the device's own
+    moments."""
+    bf, dtype, kind, alpha = torch.bfloat16, I.DTYPE_BF16, I.FFN_SWIGLU, 2.0
+    S, T, d, f = 2, 200, 328, 344
+    lr, b1, b2, eps = 1e-3, 0.9, 0.95, 1e-8
+    X = I.normal(95, 1, (S, T, d), 1.0, dtype)
+    Wgu = I.normal(95, 2, (S, 2 * f, d), 0.05, dtype)
+    Wd = I.normal(95, 3, (S, f, d), 0.05, dtype)
+    dY = I.normal(95, 4, (S, T, d), 1e-3, dtype)
+    t = lambda *s: torch.zeros(*s, dtype=bf, device="cuda")
+    w_gu, w_down = dev(Wgu, bf), dev(Wd, bf)
+    m_gu, m_down = w_gu.float(), w_down.float()
+    mom = {n: torch.zeros_like(m_gu if "gu" in n else m_down) for n in ("m_gu", "v_gu", "m_down", "v_down")}
+    dw_gu = torch.zeros(S, 2 * f, d, dtype=torch.float32, device="cuda")
+    dw_down = torch.zeros(S, f, d, dtype=torch.float32, device="cuda")
+    pre, hh, y, dpre = t(S, T, 2 * f), t(S, T, f), t(S, T, d), t(S, T, 2 * f)
+    x_dev, dy_dev = dev(X, bf), dev(dY, bf)          # kept alive: the argument struct holds raw pointers only
+    for step in (1, 2):
+        a = B.ffn_args(kind, dtype, S, T, d, f, alpha, lr, opt=B.adam(step, b1, b2, eps), x=x_dev, w_gu=w_gu,
+                       w_down=w_down, w_gu_master=m_gu, w_down_master=m_down, pre=pre, hh=hh, y=y, dy=dy_dev,
+                       dpre=dpre, dw_gu=dw_gu, dw_down=dw_down, **mom)
+        before = {"gu": (m_gu.clone(), mom["m_gu"].clone(), mom["v_gu"].clone()),
+                  "down": (m_down.clone(), mom["m_down"].clone(), mom["v_down"].clone())}
+        B.twist_subnet_ffn_fwd(a)
+        B.twist_subnet_ffn_bwd(a)
+        torch.cuda.synchronize()
+        check_status(B)
+        for name, master, grad in (("gu", m_gu, dw_gu), ("down", m_down, dw_down)):
+            w0, m0, v0 = (x.double().cpu().numpy() for x in before[name])
+            g = grad.double().cpu().numpy()                       # the device's own gradient
+            new, m1, v1, _ = o.adam(w0, m0, v0, g, step, lr, b1, b2, eps, True)
+            assert rel_fro(host(mom["m_" + name]), m1) < 1e-5 and rel_fro(host(mom["v_" + name]), v1) < 1e-5
+            assert rel_fro(host(master) - w0, new - w0) < 1e-3, (name, step)     # fp32 sqrt / divide vs fp64
+        if step == 1:      # fresh moments against the oracle's own gradients: m = (1 - b1) g, v = (1 - b2) g^2
+            for s in range(S):
+                Wg_s, Wu_s, Wd_s = Wgu[s, :f].astype(np.float64), Wgu[s, f:].astype(np.float64), Wd[s].astype(np.float64)
+                Xs, dYs = X[s].astype(np.float64), dY[s].astype(np.float64)
+                _, saved = o.ffn_fwd(Xs, Wu_s, Wg_s, Wd_s, kind, alpha, True)
+                _, dWu, dWg, dWd = o.ffn_bwd(dYs, Xs, saved, Wu_s, Wg_s, Wd_s, kind, alpha, True)
+                dWgu = np.concatenate([dWg, dWu], axis=0)
+                assert rel_fro(host(mom["m_down"][s]), (1 - b1) * dWd) < GEMM_TOL
+                assert rel_fro(host(mom["v_down"][s]), (1 - b2) * dWd * dWd) < 2 * GEMM_TOL
+                assert rel_fro(host(mom["m_gu"][s]), (1 - b1) * dWgu) < GEMM_TOL
+                assert rel_fro(host(mom["v_gu"][s]), (1 - b2) * dWgu * dWgu) < 2 * GEMM_TOL
+
+
+def test_scaled_twin_round_with_adam_matches_oracle(B):
+    """A free-running BLOCKWISE round with Adam; eps is large against sqrt(v) here, so the step is nearly linear
+    in the gradient and the 5e-2 bar on the weight change is meaningful (with a tiny eps the step is a sign
+    function of gradients that are themselves only known to 2e-2)."""
+    w = replace(I.scaled_twin(I.PRESETS[3], d_model=256, d_ff=688, d_head=8, tokens=256, n_layers=1, local_steps=3),
+                optimizer="adam", lr=1e-3, beta1=0.9, beta2=0.99, adam_eps=3e-3)
+    _run_round_and_compare(B, w)
+
+
+def test_stack_round_with_adam_runs_and_matches_losses(B):
+    from paper_2511_03983_b200.engine import StackEngine
+    w = replace(I.scaled_twin(I.PRESETS[2], d_model=192, d_ff=528, d_head=16, tokens=192, n_layers=2, local_steps=3),
+                optimizer="adam", lr=1e-3, adam_eps=3e-3)
+    eng = StackEngine(w, 2, 96, keep_f32_full=True)
+    full_np = _load_full(eng, w)
+    store = {}
+    for k in range(w.local_steps):
+        for kind, dst in ((I.BATCH_X, eng.X), (I.BATCH_TGT_D, eng.Td)):
+            arr = np.stack([I.batch(w, kind, 0, s, k, w.d_model) for s in range(w.n_subnets)])
+            store[(kind, k)] = arr
+            dst.append(dev(arr, torch.bfloat16))
+    eng.run_round(0)
+    torch.cuda.synchronize()
+    check_status(B)
+    full64 = [{m: v.astype(np.float64) for m, v in layer.items()} for layer in full_np]
+    new, _, losses = o.round_stack(w, full64, lambda kind, rnd, s, k, width: store[(kind, k)][s], 0, 2, 96, True)
+    assert np.allclose(eng.stack_loss[: w.local_steps].cpu().numpy(), np.array(losses).T, rtol=2e-2)
+    for l in range(w.n_layers):
+        for m in eng.full:
+            res = eng.full_f32[m][l].cpu().numpy().astype(np.float64)
+            assert rel_fro(res - full64[l][m], new[l][m] - full64[l][m]) < 5e-2, (l, m)
