@@ -174,7 +174,7 @@ int encode_map_3d_bf16(CUtensorMap* map, const void* ptr, const unsigned long lo
 
 size_t fused_loss_partials(int groups, int M, int N) {
   const size_t m_tiles = (size_t)(M + kBM - 1) / kBM, n_tiles = (size_t)(N + kBN - 1) / kBN;
-  return (size_t)groups * m_tiles * n_tiles * 8;
+  return (size_t)groups * m_tiles * n_tiles * 2 * kEpiWarps;
 }
 
 int finish_fused_loss(const float* partial, int groups, int M, int N, const int32_t* valid_cols, int seg_begin,

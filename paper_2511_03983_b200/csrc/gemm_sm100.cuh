@@ -17,8 +17,10 @@
 //   NN (A K-major, B MN-major)  h W              : down / o forward, dX
 //   TN (A MN-major, B MN-major) act^T other      : every weight gradient (contraction over tokens)
 //
-// Warp roles (192 threads per CTA): warps 0-3 epilogue (warp w owns TMEM lanes 32w..32w+31), warp 4 TMA
-// producer (one lane), warp 5 TMEM allocator (both CTAs) + MMA issuer (one lane, leader CTA only).
+// Warp roles (320 threads per CTA): warps 0-7 epilogue (warp w owns TMEM lanes 32 (w & 3) .. +31 and half w >> 2 of
+// the columns), warp 8 TMA producer (one lane), warp 9 TMEM allocator (both CTAs) + MMA issuer (one lane, leader
+// CTA only).  Eight epilogue warps, two per scheduler: a single warp per scheduler cannot hide the latency of its
+// own dependent instructions, and short-K tiles were bound by the epilogue's issue rate.
 // Barriers: both producers' copies complete on the leader's "full" barrier; the leader's
 // tcgen05.commit signals "stage empty" and "accumulator full" in both CTAs; the epilogue warps of both
 // CTAs arrive on the leader's "accumulator empty" barrier.
@@ -41,13 +43,14 @@ constexpr int kCtaM = kBM / 2, kCtaN = kBN / 2;   // rows of A / columns of B th
 constexpr int kABytes = kCtaM * kBK * 2;          // 16 KB
 constexpr int kBBytes = kCtaN * kBK * 2;          // 16 KB
 constexpr int kStageBytes = kABytes + kBBytes;    // 32 KB per CTA and stage
-constexpr int kGemmThreads = 192;
-// Epilogue staging: every epilogue warp owns 16 KB in which 32-row x 32-column bf16 boxes (2 KB, 64-byte rows,
+constexpr int kEpiWarps = 8;                      // epilogue warps: two per tensor-memory lane quarter
+constexpr int kGemmThreads = (kEpiWarps + 2) * 32;
+// Epilogue staging: every epilogue warp owns 8 KB in which 32-row x 32-column bf16 boxes (2 KB, 64-byte rows,
 // 64-byte swizzle) travel between global memory and the warp by TMA: operands the epilogue reads arrive as boxes,
 // results leave as boxes, so every global access of the epilogue is a full-line bulk transfer.
 constexpr int kEpiBoxBytes = 32 * 32 * 2;
-constexpr int kEpiWarpBytes = 16384;
-constexpr int kEpiBytes = 4 * kEpiWarpBytes;
+constexpr int kEpiWarpBytes = 8192;
+constexpr int kEpiBytes = kEpiWarps * kEpiWarpBytes;
 constexpr int kCtrlBytes = 512;
 // Operand ring: 5 stages of 32 KB beside the epilogue staging.  The weight-gradient kernel stages nothing and
 // could hold 7, but measured no faster with them (it is bound by power, not by latency), so it keeps 5 too.
@@ -72,7 +75,7 @@ struct GemmParams {
   float* adam_m;        // ADAM: first / second moment of the group's weights, fp32 [g][M][N]
   float* adam_v;
   float beta1, beta2, adam_eps, bias1, bias2;   // ADAM: decay rates, epsilon, 1 / (1 - beta^t)
-  float* dw;            // SGD: optional fp32 gradient dump [g][M][N].  MSE: partial sums, 8 per tile (2 CTAs x 4 warps)
+  float* dw;            // SGD: optional fp32 gradient dump [g][M][N].  MSE: partial sums, 16 per tile (2 CTAs x 8 warps)
   const int32_t* valid_cols;   // MSE: valid columns per column group and subnet [groups], or null (all valid)
   int seg_begin, seg_width;    // MSE: columns [0, seg_begin) valid, then groups of seg_width columns (see twist_mse_fwd_bwd)
   int* status;          // device status word
@@ -92,7 +95,7 @@ __host__ __device__ constexpr int epi_slots(int epi) {
 __host__ __device__ constexpr int epi_in_slots(int epi) {
   return epi == EPI_DSWIGLU ? 2 : (epi == EPI_MSE || epi == EPI_MSE_NOY || epi == EPI_DACT || epi == EPI_RESID) ? 1 : 0;
 }
-__host__ __device__ constexpr int epi_bufs(int epi) { return epi_slots(epi) == 3 ? 2 : epi_slots(epi) == 2 ? 4 : 8; }
+__host__ __device__ constexpr int epi_bufs(int epi) { return epi_slots(epi) == 3 ? 1 : epi_slots(epi) == 2 ? 2 : 4; }
 
 // Registers of one 32-column chunk of accumulator words.
 template <int EPI> struct EpiAcc { uint32_t r0[32]; };
@@ -259,7 +262,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   // control block: 8-byte barriers full[kStages], empty[kStages], tmem_full[2], tmem_empty[2]; then the TMEM base
   // address and the abort flag (4 bytes each, within the first 160 bytes for at most 7 stages); at byte 192 the
   // 32 "box arrived" barriers of the epilogue warps (8 per warp).  Same offsets in both CTAs of the pair.
-  auto in_bar = [&](int w, uint32_t buf) { return bar_base + 192u + 8u * (8u * w + buf); };
+  auto in_bar = [&](int w, uint32_t buf) { return bar_base + 192u + 8u * (4u * w + buf); };
   auto full_bar = [&](int i) { return bar_base + 8u * i; };
   auto empty_bar = [&](int i) { return bar_base + 8u * (kStages + i); };
   auto tfull_bar = [&](int i) { return bar_base + 8u * (2 * kStages + i); };
@@ -273,19 +276,19 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   const int total_tiles = p.groups * p.m_tiles * p.n_tiles;
   const int num_kb = (p.K + kBK - 1) / kBK;
 
-  if (warp == 4 && lane == 0) {
+  if (warp == kEpiWarps && lane == 0) {
     tma_prefetch_desc(&tmA);
     tma_prefetch_desc(&tmB);
     for (int i = 0; i < kStages; ++i) { mbar_init(full_bar(i), 1); mbar_init(empty_bar(i), 1); }
-    for (int i = 0; i < 2; ++i) { mbar_init(tfull_bar(i), 1); mbar_init(tempty_bar(i), 8); }   // 4 epilogue warps x 2 CTAs
+    for (int i = 0; i < 2; ++i) { mbar_init(tfull_bar(i), 1); mbar_init(tempty_bar(i), 2 * kEpiWarps); }   // epilogue warps of both CTAs
     if (kStaged)
-      for (int w = 0; w < 4; ++w)
-        for (int b = 0; b < 8; ++b) mbar_init(in_bar(w, b), 1);
+      for (int w = 0; w < kEpiWarps; ++w)
+        for (int b = 0; b < 4; ++b) mbar_init(in_bar(w, b), 1);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
-  if (warp == 5) {   // the same warp of both CTAs allocates the pair's tensor memory together
+  if (warp == kEpiWarps + 1) {   // the same warp of both CTAs allocates the pair's tensor memory together
     asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;"
                  ::"r"(smem_u32(const_cast<uint32_t*>(tmem_slot))), "r"((uint32_t)kTmemCols) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
@@ -296,7 +299,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
-  if (warp == 4) {
+  if (warp == kEpiWarps) {
     // ------------------------------------------------------------------ TMA producer (both CTAs)
     if (lane == 0) {
       uint32_t it = 0;
@@ -332,7 +335,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         }
       }
     }
-  } else if (warp == 5) {
+  } else if (warp == kEpiWarps + 1) {
     // ------------------------------------------------------------------ MMA issuer (leader CTA only)
     if (lane == 0 && rank == 0) {
       constexpr uint32_t idesc = instr_desc(A_MAJOR, B_MAJOR);
@@ -370,8 +373,12 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     // ------------------------------------------------------------------ epilogue warps 0..3
     // Thread (warp w, lane l) owns accumulator row 32 w + l of this CTA and walks it in chunks of 32 columns;
     // the tensor-memory load of chunk c + 1 is in flight while chunk c is processed.
-    constexpr int kChunks = (EPI == EPI_SWIGLU_FWD) ? kCtaN / 32 : kBN / 32;
+    // Warp w reads tensor-memory lanes 32 (w & 3) .. +31 (the rows of that quarter) and the columns of half w >> 2:
+    // 128 of the tile's 256 output columns (SwiGLU forward: 64 of its 128 neurons, as 64 G and 64 U columns).
     constexpr int kTileN = (EPI == EPI_SWIGLU_FWD) ? kCtaN : kBN;     // output columns (neurons) per tile
+    constexpr int kHalfN = kTileN / 2;                                // ... per warp
+    constexpr int kChunks = kHalfN / 32;
+    const int quarter = warp & 3, half = warp >> 2;
     const uint32_t tempty_leader[2] = {map_to_cta(tempty_bar(0), 0), map_to_cta(tempty_bar(1), 0)};
     uint32_t tl = 0;
     bool ok = true;
@@ -383,11 +390,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         int g, mt, nt;
         tile_coords(p, tile, g, mt, nt);
         const uint32_t slot = tl & 1u, acc_phase = (tl >> 1) & 1u;
-        const int row = mt * kBM + (int)rank * kCtaM + warp * 32 + lane;
+        const int row = mt * kBM + (int)rank * kCtaM + quarter * 32 + lane;
         const bool row_ok = row < p.M;
-        const uint32_t t_row = tmem_base + slot * kBN + ((uint32_t)(warp * 32) << 16);
+        const uint32_t t_row = tmem_base + slot * kBN + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(half * kHalfN);
         const long long grow = (long long)g * p.M + row;      // row index over all groups
-        const int n_base = nt * kBN;
+        const int n_base = nt * kBN + half * kHalfN;
         float4 mv[2][8];
         EpiAcc<EPI> acc[2];
         auto load_master = [&](int c, float4 (&m)[8]) {
@@ -461,7 +468,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       constexpr bool kIsMse = EPI == EPI_MSE || EPI == EPI_MSE_NOY;
       // Inputs are requested kAhead chunks ahead into the buffer that chunk gc + kAhead - kBufs used; only that
       // chunk's store has to be finished, so up to kBufs - kAhead younger stores may still be reading.
-      constexpr int kAhead = kBufs / 2;
+      constexpr int kAhead = kBufs > 1 ? kBufs / 2 : 1;
       const uint32_t wbase = epi_base + (uint32_t)warp * kEpiWarpBytes;
       auto box = [&](uint32_t gc, int slot) { return wbase + ((gc & (kBufs - 1)) * kSlots + slot) * kEpiBoxBytes; };
       // 16-byte piece q (0..3) of this thread's row inside a box (64-byte rows, 64-byte swizzle)
@@ -479,8 +486,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         if (t.valid) {
           int mt, nt;
           tile_coords(p, tile, t.g, mt, nt);
-          t.row0 = mt * kBM + (int)rank * kCtaM + warp * 32;
-          t.n0 = nt * kTileN;
+          t.row0 = mt * kBM + (int)rank * kCtaM + quarter * 32;
+          t.n0 = nt * kTileN + half * kHalfN;
         }
         return t;
       };
@@ -505,7 +512,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         const uint32_t slot = tl & 1u, acc_phase = (tl >> 1) & 1u;
         const int row0 = cur.row0;
         const bool row_ok = row0 + lane < p.M;
-        const uint32_t t_row = tmem_base + slot * kBN + ((uint32_t)(warp * 32) << 16);
+        const uint32_t t_row = tmem_base + slot * kBN + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(half * kHalfN);
         const int n_base = nt_n0;
         EpiAcc<EPI> acc[2];
         float loss_acc = 0.f, kfac = 0.f;
@@ -517,7 +524,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         }
         auto load_acc = [&](int c, EpiAcc<EPI>& a) {
           tc_ld32(t_row + 32 * c, a.r0);
-          if constexpr (EPI == EPI_SWIGLU_FWD) tc_ld32(t_row + kCtaN + 32 * c, a.r1);
+          if constexpr (EPI == EPI_SWIGLU_FWD) tc_ld32(t_row + kCtaN + 32 * c, a.r1);      // U: 128 columns after G
         };
         if (!__all_sync(0xffffffffu, mbar_wait(tfull_bar(slot), acc_phase, abort_flag, p.status))) { ok = false; break; }
         tc_fence_after();
@@ -678,7 +685,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         if (lane == 0) mbar_arrive_cluster(tempty_leader[slot]);
         if constexpr (kIsMse) {   // per-warp partial sum of squared errors, fixed order
           for (int o = 16; o > 0; o >>= 1) loss_acc += __shfl_xor_sync(0xffffffffu, loss_acc, o);
-          if (lane == 0) p.dw[((long long)tile * 2 + rank) * 4 + warp] = loss_acc;
+          if (lane == 0) p.dw[((long long)tile * 2 + rank) * kEpiWarps + warp] = loss_acc;
         }
       }
       if (lane == 0) bulk_wait_read<0>();      // shared memory stays valid until the last store has read it
@@ -698,7 +705,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   // Neither CTA leaves (nor frees tensor memory) while the other may still signal its barriers, read
   // its shared memory or write its accumulators.
   cluster_sync_all();
-  if (warp == 5) {
+  if (warp == kEpiWarps + 1) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)kTmemCols) : "memory");
   }
