@@ -51,6 +51,81 @@ __device__ inline uint32_t pack2(float lo, float hi) {
   __nv_bfloat162 t = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<uint32_t*>(&t);
 }
+// 2^x by the special-function unit (about 2 ulp, flushes denormals, 2^-inf = 0): exp2f() would wrap the same
+// instruction in range fix-ups that cost more issue slots than the rest of the softmax.
+__device__ inline float ex2_fast(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+// Softmax of one 128-key block for this thread's query row: reads the row of S from tensor memory twice (maximum,
+// then exponentials), updates the running maximum m (log2 domain) and sum l, writes P (bf16) into the A-operand
+// tile and returns the factor by which the running output shrinks.  MASKED: only columns <= k_lim are visible
+// (the diagonal block); the other blocks carry no per-element predicate.  The tensor-memory load of the next
+// 32-column chunk is in flight while the current one is processed.
+template <bool MASKED>
+__device__ inline float softmax_block(uint32_t t_s, uint32_t p_row, uint32_t sw, int k_lim, float scale_log2, float& m,
+                                      float& l) {
+  uint32_t va[32], vb[32];
+  float mx = -INFINITY;
+  auto fold_max = [&](const uint32_t (&v)[32], int c) {
+#pragma unroll
+    for (int i = 0; i < 32; ++i)
+      if (!MASKED || 32 * c + i <= k_lim) mx = fmaxf(mx, __uint_as_float(v[i]));
+  };
+  tc_ld32(t_s, va);
+  tc_wait_ld();
+  tc_ld32(t_s + 32, vb);
+  fold_max(va, 0);
+  tc_wait_ld();
+  tc_ld32(t_s + 64, va);
+  fold_max(vb, 1);
+  tc_wait_ld();
+  tc_ld32(t_s + 96, vb);
+  fold_max(va, 2);
+  tc_wait_ld();
+  tc_ld32(t_s, va);                                    // first chunk of the second pass
+  fold_max(vb, 3);
+  const float m_new = fmaxf(m, mx * scale_log2);       // scale > 0: the maximum commutes with the scaling
+  const float corr = ex2_fast(m - m_new);
+  float sum = 0.f;
+  auto emit = [&](const uint32_t (&v)[32], int c) {
+    uint32_t w[16];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+      float p0 = ex2_fast(fmaf(__uint_as_float(v[2 * i]), scale_log2, -m_new));
+      float p1 = ex2_fast(fmaf(__uint_as_float(v[2 * i + 1]), scale_log2, -m_new));
+      if (MASKED) {
+        p0 = (32 * c + 2 * i <= k_lim) ? p0 : 0.f;
+        p1 = (32 * c + 2 * i + 1 <= k_lim) ? p1 : 0.f;
+      }
+      sum += p0 + p1;
+      w[i] = pack2(p0, p1);
+    }
+    const uint32_t half = p_row + (uint32_t)(c >> 1) * (kPBytes / 2);
+#pragma unroll
+    for (int q4 = 0; q4 < 4; ++q4) {
+      const uint32_t piece = (uint32_t)((c & 1) * 4 + q4);
+      sts128(half + ((piece ^ sw) << 4), make_uint4(w[4 * q4], w[4 * q4 + 1], w[4 * q4 + 2], w[4 * q4 + 3]));
+    }
+  };
+  tc_wait_ld();
+  tc_ld32(t_s + 32, vb);
+  emit(va, 0);
+  tc_wait_ld();
+  tc_ld32(t_s + 64, va);
+  emit(vb, 1);
+  tc_wait_ld();
+  tc_ld32(t_s + 96, vb);
+  emit(va, 2);
+  tc_wait_ld();
+  emit(vb, 3);
+  l = l * corr + sum;
+  m = m_new;
+  return corr;
+}
+
 __device__ inline int kv_position(const AttnParams& p, int s, int hq) {
   if (!p.head_idx) return hq;
   const int g = p.head_idx[(long long)s * p.heads + hq] / p.per_group;
@@ -163,42 +238,8 @@ __global__ void __launch_bounds__(kFwdThreads, 2) attn_fwd_tc_kernel(const __gri
     for (int j = 0; j < nblk; ++j) {
       if (!__all_sync(0xffffffffu, mbar_wait(bar(5), j & 1, abort_flag, status))) { ok = false; break; }
       tc_fence_after();
-      const int k_lim = (j == qb) ? qi - j * kBk : kBk;                           // columns <= k_lim are visible
-      // pass 1: row maximum (scores scaled into the log2 domain)
-      float mx = -INFINITY;
-#pragma unroll
-      for (int c = 0; c < kBk / 32; ++c) {
-        uint32_t v[32];
-        tc_ld32(t_s + 32 * c, v);
-        tc_wait_ld();
-#pragma unroll
-        for (int i = 0; i < 32; ++i)
-          if (32 * c + i <= k_lim) mx = fmaxf(mx, __uint_as_float(v[i]));
-      }
-      const float m_new = fmaxf(m, mx * p.scale_log2);
-      const float corr = exp2f(m - m_new);
-      l *= corr;
-      // pass 2: exponentials -> P (bf16) in shared memory, row sum
-#pragma unroll
-      for (int c = 0; c < kBk / 32; ++c) {
-        uint32_t v[32];
-        tc_ld32(t_s + 32 * c, v);
-        tc_wait_ld();
-        uint32_t w[16];
-#pragma unroll
-        for (int i = 0; i < 16; ++i) {
-          const float p0 = (32 * c + 2 * i <= k_lim) ? exp2f(fmaf(__uint_as_float(v[2 * i]), p.scale_log2, -m_new)) : 0.f;
-          const float p1 = (32 * c + 2 * i + 1 <= k_lim) ? exp2f(fmaf(__uint_as_float(v[2 * i + 1]), p.scale_log2, -m_new)) : 0.f;
-          l += p0 + p1;
-          w[i] = pack2(p0, p1);
-        }
-        const uint32_t half = p_row + (uint32_t)(c >> 1) * (kPBytes / 2);
-#pragma unroll
-        for (int q4 = 0; q4 < 4; ++q4) {
-          const uint32_t piece = (uint32_t)((c & 1) * 4 + q4);
-          sts128(half + ((piece ^ sw) << 4), make_uint4(w[4 * q4], w[4 * q4 + 1], w[4 * q4 + 2], w[4 * q4 + 3]));
-        }
-      }
+      const float corr = (j == qb) ? softmax_block<true>(t_s, p_row, sw, qi - j * kBk, p.scale_log2, m, l)
+                                   : softmax_block<false>(t_s, p_row, sw, kBk, p.scale_log2, m, l);
       fence_async_smem();                                                         // P: generic writes -> MMA reads
       tc_fence_before();
       mbar_arrive(bar(6));
@@ -212,7 +253,6 @@ __global__ void __launch_bounds__(kFwdThreads, 2) attn_fwd_tc_kernel(const __gri
 #pragma unroll
         for (int i = 0; i < 32; ++i) o[32 * c + i] = fmaf(o[32 * c + i], corr, __uint_as_float(v[i]));
       }
-      m = m_new;
     }
     if (ok && qi < p.seq_len) {
       const float inv = 1.f / l;
@@ -258,7 +298,7 @@ constexpr int kDkvSmem = kTileBytes * 6 + 4 * kPBytes + 1024 + 256;   // K, V, Q
 // Element-wise step shared by the two backward kernels: for this thread's row and its 64 columns (two 32-column
 // chunks starting at chunk c0) of S and dP in tensor memory, P = exp2(S * scale - lse2) where visible (column <=
 // k_lim), dS = P * (dP - dl); dS (and P when WRITE_P) go to the operand tiles in shared memory.
-template <bool WRITE_P>
+template <bool WRITE_P, bool MASKED>
 __device__ inline void probs_and_ds(uint32_t t_s, uint32_t t_dp, int c0, int r, int k_lim, float scale_log2, float lse2,
                                     float dl, uint32_t p_tile, uint32_t ds_tile) {
 #pragma unroll
@@ -275,7 +315,8 @@ __device__ inline void probs_and_ds(uint32_t t_s, uint32_t t_dp, int c0, int r, 
 #pragma unroll
       for (int h = 0; h < 2; ++h) {
         const int col = 32 * c + 2 * e + h;
-        pr[h] = col <= k_lim ? exp2f(fmaf(__uint_as_float(vs[2 * e + h]), scale_log2, -lse2)) : 0.f;
+        pr[h] = ex2_fast(fmaf(__uint_as_float(vs[2 * e + h]), scale_log2, -lse2));
+        if (MASKED) pr[h] = col <= k_lim ? pr[h] : 0.f;
         d2[h] = pr[h] * (__uint_as_float(vd[2 * e + h]) - dl);
       }
       wp[e] = pack2(pr[0], pr[1]);
@@ -405,8 +446,12 @@ __global__ void __launch_bounds__(kBwdThreads) attn_dq_tc_kernel(const __grid_co
       if (!__all_sync(0xffffffffu, mbar_wait(bar(5), j & 1, abort_flag, status))) { ok = false; break; }
       tc_fence_after();
       const int k_lim = !row_ok ? -1 : ((j == qb) ? qi - j * kBk : kBk);
-      probs_and_ds<false>(tm_s + lane_off, tm_dp + lane_off, 2 * half, r, k_lim, p.scale_log2, lse2, dl, 0u,
-                          ds_s + (j & 1) * kPBytes);
+      if (__any_sync(0xffffffffu, k_lim < kBk))      // warp-uniform: the tensor-memory loads inside are warp-wide
+        probs_and_ds<false, true>(tm_s + lane_off, tm_dp + lane_off, 2 * half, r, k_lim, p.scale_log2, lse2, dl, 0u,
+                                  ds_s + (j & 1) * kPBytes);
+      else
+        probs_and_ds<false, false>(tm_s + lane_off, tm_dp + lane_off, 2 * half, r, k_lim, p.scale_log2, lse2, dl, 0u,
+                                   ds_s + (j & 1) * kPBytes);
       fence_async_smem();
       tc_fence_before();
       mbar_arrive(bar(6));
@@ -556,8 +601,12 @@ __global__ void __launch_bounds__(kBwdThreads) attn_dkv_tc_kernel(const __grid_c
       if (!__all_sync(0xffffffffu, mbar_wait(bar(5), n & 1, abort_flag, status))) { ok = false; break; }
       tc_fence_after();
       const int k_lim = !row_ok ? -1 : ((i == kb) ? r : kBk);                     // diagonal block: keys <= query
-      probs_and_ds<true>(tm_s + lane_off, tm_dp + lane_off, 2 * half, r, k_lim, p.scale_log2, lse2, dl,
-                         p_s + (n & 1) * kPBytes, ds_s + (n & 1) * kPBytes);
+      if (__any_sync(0xffffffffu, k_lim < kBk))      // warp-uniform: the tensor-memory loads inside are warp-wide
+        probs_and_ds<true, true>(tm_s + lane_off, tm_dp + lane_off, 2 * half, r, k_lim, p.scale_log2, lse2, dl,
+                                 p_s + (n & 1) * kPBytes, ds_s + (n & 1) * kPBytes);
+      else
+        probs_and_ds<true, false>(tm_s + lane_off, tm_dp + lane_off, 2 * half, r, k_lim, p.scale_log2, lse2, dl,
+                                  p_s + (n & 1) * kPBytes, ds_s + (n & 1) * kPBytes);
       fence_async_smem();
       tc_fence_before();
       mbar_arrive(bar(6));

@@ -26,6 +26,8 @@ struct AggParams {
   int n_subnets;
   uint32_t live;
   long long total_rows;
+  int parts;          // work item = one of `parts` equal spans of a row
+  int part_chunks;    // float4 chunks per span
 };
 
 __device__ inline uint4 ld_nc(const uint4* p) {
@@ -49,12 +51,26 @@ __device__ inline uint4 widen_hi(uint4 v) {   // bf16 elements 4..7
 }
 
 constexpr int kUnroll = 4;
+#ifndef TWIST_AGG_PART_CHUNKS
+#define TWIST_AGG_PART_CHUNKS 256
+#endif
+constexpr int kAggPartChunks = TWIST_AGG_PART_CHUNKS;
 
-constexpr int kGatherWarps = 8;          // warps per CTA
-constexpr int kGatherPieceBytes = 4096;  // a row travels in pieces of at most this many bytes
+#ifndef TWIST_GATHER_WARPS
+#define TWIST_GATHER_WARPS 8
+#define TWIST_GATHER_BUFS 2
+#define TWIST_GATHER_AHEAD 1
+#define TWIST_GATHER_PIECE 4096
+#endif
+constexpr int kGatherWarps = TWIST_GATHER_WARPS;        // warps per CTA
+constexpr int kGatherBufs = TWIST_GATHER_BUFS;          // shared-memory buffers per warp
+constexpr int kGatherAhead = TWIST_GATHER_AHEAD;        // a piece's load is requested this many items early
+constexpr int kGatherPending = kGatherBufs - 1 - kGatherAhead;   // store groups that may still be reading shared memory
+constexpr int kGatherPieceBytes = TWIST_GATHER_PIECE;   // a row travels in pieces of at most this many bytes
+static_assert(kGatherAhead >= 1 && kGatherPending >= 0, "buffer ring too short for the lookahead");
 
-// Work item = (destination row, piece of the row); one warp per item at a time, two buffers per warp so
-// the load of the next item overlaps the widening and the stores of the current one.
+// Work item = (destination row, piece of the row); one warp per item at a time, a ring of buffers per warp so
+// the loads of the next items overlap the widening and the stores of the current one.
 // Shared memory per warp and buffer: the piece as loaded [piece bytes] and, when masters are written,
 // its fp32 widening [2 x piece bytes].  ELEM = 2 (bf16) or 4 (fp32) bytes.
 template <int ELEM>
@@ -62,18 +78,17 @@ __global__ void __launch_bounds__(kGatherWarps * 32) gather_rows_kernel(const __
                                                                         int piece_bytes, int pieces, int buf_bytes,
                                                                         int* status) {
   extern __shared__ __align__(128) unsigned char gsm[];
-  __shared__ __align__(8) unsigned long long bars[kGatherWarps][2];
+  __shared__ __align__(8) unsigned long long bars[kGatherWarps][kGatherBufs];
   __shared__ int abort_flag;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (threadIdx.x == 0) abort_flag = 0;
   if (lane == 0) {
-    mbar_init(smem_u32(&bars[warp][0]), 1);
-    mbar_init(smem_u32(&bars[warp][1]), 1);
+    for (int i = 0; i < kGatherBufs; ++i) mbar_init(smem_u32(&bars[warp][i]), 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     fence_async_smem();
   }
   __syncthreads();
-  const uint32_t wbase = smem_u32(gsm) + (uint32_t)warp * 2u * (uint32_t)buf_bytes;
+  const uint32_t wbase = smem_u32(gsm) + (uint32_t)warp * (uint32_t)kGatherBufs * (uint32_t)buf_bytes;
   const int row_bytes = p.d * ELEM;
   const long long items = p.total_rows * pieces;
   const long long wid0 = (long long)blockIdx.x * kGatherWarps + warp;
@@ -123,24 +138,29 @@ __global__ void __launch_bounds__(kGatherWarps * 32) gather_rows_kernel(const __
     bulk_load(wbase + (uint32_t)b * buf_bytes, src, (uint32_t)o.bytes, bar);
   };
 
-  uint32_t uses0 = 0, uses1 = 0;                       // completed phases of each buffer's barrier
-  Item cur = decode(wid0);
-  if (lane == 0 && wid0 < items) request(cur, 0);
-  Item nxt = decode(wid0 + stride);
-  int n = 0;
-  for (long long it = wid0; it < items; it += stride, ++n) {
-    const int b = n & 1;
-    const Item nxt2 = decode(it + 2 * stride);         // its index load is in flight during this iteration
+  // Ring discipline: item n lives in buffer n % kGatherBufs and commits exactly one store group (an empty one for
+  // a padding row), so "at most kGatherPending groups still reading" frees the buffer of item n + kGatherAhead.
+  uint32_t phase = 0;                                  // bit b: parity of buffer b's barrier
+  Item q[kGatherAhead + 1];                            // q[0] current, q[1..] requested, q[kGatherAhead] decoded only
+#pragma unroll
+  for (int i = 0; i <= kGatherAhead; ++i) q[i] = decode(wid0 + i * stride);
+#pragma unroll
+  for (int i = 0; i < kGatherAhead; ++i)
+    if (lane == 0) request(q[i], i % kGatherBufs);
+  int b = 0, b_req = kGatherAhead % kGatherBufs;
+  for (long long it = wid0; it < items; it += stride) {
+    const Item fresh = decode(it + (kGatherAhead + 1) * stride);   // its index load is in flight during this iteration
     if (lane == 0) {
-      bulk_wait_read<0>();                             // the stores that read the other buffer are done with it
-      if (it + stride < items) request(nxt, b ^ 1);
+      bulk_wait_read<kGatherPending>();                // the stores that read buffer b_req are done with it
+      request(q[kGatherAhead], b_req);
     }
+    const Item cur = q[0];
     const uint32_t in = wbase + (uint32_t)b * buf_bytes;
     if (cur.src_base) {
-      const uint32_t parity = (b ? uses1 : uses0) & 1u;
+      const uint32_t parity = (phase >> b) & 1u;
       // warp-uniform outcome: either every lane goes on or every lane leaves
       if (!__all_sync(0xffffffffu, mbar_wait(smem_u32(&bars[warp][b]), parity, &abort_flag, status))) break;
-      if (b) ++uses1; else ++uses0;
+      phase ^= 1u << b;
       if (lane == 0) bulk_store(cur.dst, in, (uint32_t)cur.bytes);
       if (cur.mst) {                                   // exact widening bf16 -> fp32, staged in shared memory
         const uint32_t out = in + (uint32_t)piece_bytes;
@@ -153,7 +173,6 @@ __global__ void __launch_bounds__(kGatherWarps * 32) gather_rows_kernel(const __
         __syncwarp();
         if (lane == 0) bulk_store(cur.mst, out, 2u * (uint32_t)cur.bytes);
       }
-      if (lane == 0) bulk_commit();
     } else {                                           // padding row: zeros, plain stores
       for (int c = lane; c < cur.bytes / 16; c += 32) {
         st_cs(reinterpret_cast<uint4*>(cur.dst) + c, make_uint4(0, 0, 0, 0));
@@ -163,9 +182,13 @@ __global__ void __launch_bounds__(kGatherWarps * 32) gather_rows_kernel(const __
         }
       }
     }
+    if (lane == 0) bulk_commit();
     __syncwarp();
-    cur = nxt;
-    nxt = nxt2;
+#pragma unroll
+    for (int i = 0; i < kGatherAhead; ++i) q[i] = q[i + 1];
+    q[kGatherAhead] = fresh;
+    b = b + 1 == kGatherBufs ? 0 : b + 1;
+    b_req = b_req + 1 == kGatherBufs ? 0 : b_req + 1;
   }
   if (lane == 0) bulk_wait_read<0>();
   __syncthreads();
@@ -189,7 +212,11 @@ __global__ void __launch_bounds__(256) aggregate_rows_kernel(const __grid_consta
   const long long warp0 = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   const long long nwarps = ((long long)gridDim.x * blockDim.x) >> 5;
   const int chunks = p.d / 4;                          // float4 chunks per row
-  for (long long r = warp0; r < p.total_rows; r += nwarps) {
+  const long long items = p.total_rows * p.parts;
+  for (long long it = warp0; it < items; it += nwarps) {
+    const long long r = it / p.parts;
+    const int c_begin = (int)(it - r * p.parts) * p.part_chunks;
+    const int c_end = c_begin + p.part_chunks < chunks ? c_begin + p.part_chunks : chunks;
     int g = 0;
     while (g + 1 < p.n_segs && r >= p.row_end[g]) ++g;
     const twist_aggregate_segment& sg = p.seg[g];
@@ -213,7 +240,7 @@ __global__ void __launch_bounds__(256) aggregate_rows_kernel(const __grid_consta
       const float q = a * rden;
       return fmaf(fmaf(-q, denom, a), rden, q);
     };
-    for (int c0 = lane; c0 < chunks; c0 += 32 * kUnroll) {
+    for (int c0 = c_begin + lane; c0 < c_end; c0 += 32 * kUnroll) {
       float4 acc[kUnroll];
 #pragma unroll
       for (int u = 0; u < kUnroll; ++u) acc[u] = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -222,7 +249,7 @@ __global__ void __launch_bounds__(256) aggregate_rows_kernel(const __grid_consta
 #pragma unroll
         for (int u = 0; u < kUnroll; ++u) {
           const int c = c0 + 32 * u;
-          if (c < chunks) {
+          if (c < c_end) {
             uint4 raw = ld_nc(reinterpret_cast<const uint4*>(ptr + c));
             acc[u].x += __uint_as_float(raw.x);
             acc[u].y += __uint_as_float(raw.y);
@@ -234,7 +261,7 @@ __global__ void __launch_bounds__(256) aggregate_rows_kernel(const __grid_consta
 #pragma unroll
       for (int u = 0; u < kUnroll; ++u) {
         const int c = c0 + 32 * u;
-        if (c < chunks) {
+        if (c < c_end) {
           float4 q = make_float4(quot(acc[u].x), quot(acc[u].y), quot(acc[u].z), quot(acc[u].w));
           uint4 qb = make_uint4(__float_as_uint(q.x), __float_as_uint(q.y), __float_as_uint(q.z), __float_as_uint(q.w));
           if (BF16) {
@@ -250,9 +277,9 @@ __global__ void __launch_bounds__(256) aggregate_rows_kernel(const __grid_consta
   }
 }
 
-int grid_for_rows(long long rows) {
+int grid_for_items(long long items) {
   const long long warps_per_cta = 8;
-  long long want = (rows + warps_per_cta - 1) / warps_per_cta;
+  long long want = (items + warps_per_cta - 1) / warps_per_cta;
   long long cap = (long long)sm_count() * 8;          // 8 resident CTAs of 256 threads per SM
   return (int)(want < cap ? (want > 0 ? want : 1) : cap);
 }
@@ -293,13 +320,13 @@ extern "C" int32_t twist_gather_subnets(const twist_gather_segment* segs, int32_
   const int piece_bytes = row_bytes < kGatherPieceBytes ? row_bytes : kGatherPieceBytes;
   const int pieces = (row_bytes + piece_bytes - 1) / piece_bytes;
   const int buf_bytes = piece_bytes * (any_master ? 3 : 1);          // the piece + its fp32 widening
-  const int smem = kGatherWarps * 2 * buf_bytes;
+  const int smem = kGatherWarps * kGatherBufs * buf_bytes;
   static bool configured = false;
   if (!configured) {
     TWIST_CUDA_TRY(cudaFuncSetAttribute(gather_rows_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                        kGatherWarps * 2 * 3 * kGatherPieceBytes));
+                                        kGatherWarps * kGatherBufs * 3 * kGatherPieceBytes));
     TWIST_CUDA_TRY(cudaFuncSetAttribute(gather_rows_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                        kGatherWarps * 2 * kGatherPieceBytes));
+                                        kGatherWarps * kGatherBufs * kGatherPieceBytes));
     configured = true;
   }
   // persistent grid: as many CTAs per SM as the shared memory allows (at most 8), or fewer for small inputs
@@ -348,7 +375,11 @@ extern "C" int32_t twist_aggregate(const twist_aggregate_segment* segs, int32_t 
   p.live = n_subnets >= 32 ? live_subnets : (live_subnets & ((1u << n_subnets) - 1u));
   p.total_rows = total;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  const int grid = grid_for_rows(total);
+  // A row is split into spans of kAggPartChunks float4 chunks: with whole rows as items a warp of the persistent
+  // grid gets only a handful, and the slowest warp (one row more, or rows with more covering subnets) sets the time.
+  p.part_chunks = kAggPartChunks;
+  p.parts = (d / 4 + kAggPartChunks - 1) / kAggPartChunks;
+  const int grid = grid_for_items(total * p.parts);
   if (dtype == TWIST_BF16) aggregate_rows_kernel<true><<<grid, 256, 0, st>>>(p);
   else aggregate_rows_kernel<false><<<grid, 256, 0, st>>>(p);
   TWIST_LAUNCH_CHECK();
