@@ -6,10 +6,14 @@
 //   softmax          thread = query row: the row of S is read from tensor memory twice (maximum, then
 //                    exponentials), running maximum / sum kept in registers, P written to shared memory as the
 //                    bf16 A operand of the next MMA
-//   O_blk = P V      128 x 64 x 128 MMA chain, V as the MN-major B operand (rows = keys as they lie in memory)
-//   O = O * corr + O_blk in registers (64 fp32 per thread), so tensor memory never needs rescaling.
-// The MMA of the next block's S is issued as soon as P of the current block is consumed, so it overlaps the
-// threads' accumulation of O.  Warps 0-3: softmax / output; warp 4, one lane: TMA and MMA issue.
+//   O += P V         128 x 64 x 128 MMA chain accumulating in tensor memory, V as the MN-major B operand (rows =
+//                    keys as they lie in memory)
+// P and O are expressed relative to a reference maximum that follows the running maximum lazily: only when a
+// row's maximum has grown by more than kRescaleLog2 since the reference was set does its warp rescale O in
+// tensor memory (and the running sum); otherwise P = 2^(s - ref) <= 2^kRescaleLog2 simply accumulates.  O / l is
+// the same quotient for any reference.  The threads therefore never wait for an output block: per key block
+// they read S, write P and go on.  The next block's S is issued ahead of O += P V.
+// Warps 0-3: softmax / output; warp 4, one lane: TMA and MMA issue.
 // Backward (same tile sizes; probabilities recomputed from the stored log-sum-exp, dS = P (dP - delta)):
 //   dQ kernel     one CTA per query block: per key block S = Q K^T and dP = dO V^T into tensor memory, the threads
 //                 write dS (bf16) to shared memory, dQ += dS K accumulates in tensor memory over the key blocks.
@@ -30,7 +34,8 @@ constexpr int kTileBytes = 128 * kDh * 2;            // a 128-row tile of Q, K o
 constexpr int kPBytes = kBq * kBk * 2;               // P: 32 KB (two 64-key halves of 16 KB)
 constexpr int kFwdThreads = 160;
 constexpr int kFwdSmem = kTileBytes * 4 + kPBytes + 1024 + 128;   // Q, K[2], V, P, alignment, barriers: two CTAs per SM
-constexpr int kFwdTmemCols = 256;       // S: columns 0..127, O_blk: columns 128..191
+constexpr int kFwdTmemCols = 256;       // S: columns 0..127, O: columns 128..191
+constexpr float kRescaleLog2 = 8.f;     // growth of a row maximum (log2 domain) tolerated before O is rescaled
 
 __device__ inline void mma1(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
   asm volatile(
@@ -60,19 +65,20 @@ __device__ inline float ex2_fast(float x) {
 }
 
 // Softmax of one 128-key block for this thread's query row: reads the row of S from tensor memory twice (maximum,
-// then exponentials), updates the running maximum m (log2 domain) and sum l, writes P (bf16) into the A-operand
-// tile and returns the factor by which the running output shrinks.  MASKED: only columns <= k_lim are visible
-// (the diagonal block); the other blocks carry no per-element predicate.  The tensor-memory load of the next
-// 32-column chunk is in flight while the current one is processed.
-template <bool MASKED>
-__device__ inline float softmax_block(uint32_t t_s, uint32_t p_row, uint32_t sw, int k_lim, float scale_log2, float& m,
-                                      float& l) {
+// then exponentials), keeps the reference maximum m (log2 domain) and the sum l relative to it, and writes
+// P = 2^(s * scale - m) (bf16) into the A-operand tile.  MASKED: only columns <= k_lim are visible (the diagonal
+// block); the other blocks carry no per-element predicate.  The tensor-memory load of the next 32-column chunk is
+// in flight while the current one is processed.  `rescale(corr)` is called (by the whole warp) between the two
+// passes when some row of the warp moves its reference; it multiplies the row's O by corr.
+template <bool MASKED, typename Rescale>
+__device__ inline void softmax_block(uint32_t t_s, uint32_t p_row, uint32_t sw, int k_lim, float scale_log2, float& m,
+                                     float& l, Rescale&& rescale) {
   uint32_t va[32], vb[32];
-  float mx = -INFINITY;
+  float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};   // four independent chains
   auto fold_max = [&](const uint32_t (&v)[32], int c) {
 #pragma unroll
     for (int i = 0; i < 32; ++i)
-      if (!MASKED || 32 * c + i <= k_lim) mx = fmaxf(mx, __uint_as_float(v[i]));
+      if (!MASKED || 32 * c + i <= k_lim) mx4[i & 3] = fmaxf(mx4[i & 3], __uint_as_float(v[i]));
   };
   tc_ld32(t_s, va);
   tc_wait_ld();
@@ -85,22 +91,29 @@ __device__ inline float softmax_block(uint32_t t_s, uint32_t p_row, uint32_t sw,
   tc_ld32(t_s + 96, vb);
   fold_max(va, 2);
   tc_wait_ld();
-  tc_ld32(t_s, va);                                    // first chunk of the second pass
   fold_max(vb, 3);
-  const float m_new = fmaxf(m, mx * scale_log2);       // scale > 0: the maximum commutes with the scaling
-  const float corr = ex2_fast(m - m_new);
-  float sum = 0.f;
+  const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+  const float m_blk = mx * scale_log2;                 // scale > 0: the maximum commutes with the scaling
+  if (__any_sync(0xffffffffu, m_blk > m + kRescaleLog2)) {
+    const float m_new = fmaxf(m, m_blk);
+    const float corr = ex2_fast(m - m_new);            // 0 for a first block (m = -inf), 1 where nothing moved
+    l *= corr;
+    m = m_new;
+    rescale(corr);
+  }
+  tc_ld32(t_s, va);
+  float sum4[4] = {0.f, 0.f, 0.f, 0.f};
   auto emit = [&](const uint32_t (&v)[32], int c) {
     uint32_t w[16];
 #pragma unroll
     for (int i = 0; i < 16; ++i) {
-      float p0 = ex2_fast(fmaf(__uint_as_float(v[2 * i]), scale_log2, -m_new));
-      float p1 = ex2_fast(fmaf(__uint_as_float(v[2 * i + 1]), scale_log2, -m_new));
+      float p0 = ex2_fast(fmaf(__uint_as_float(v[2 * i]), scale_log2, -m));
+      float p1 = ex2_fast(fmaf(__uint_as_float(v[2 * i + 1]), scale_log2, -m));
       if (MASKED) {
         p0 = (32 * c + 2 * i <= k_lim) ? p0 : 0.f;
         p1 = (32 * c + 2 * i + 1 <= k_lim) ? p1 : 0.f;
       }
-      sum += p0 + p1;
+      sum4[i & 3] += p0 + p1;
       w[i] = pack2(p0, p1);
     }
     const uint32_t half = p_row + (uint32_t)(c >> 1) * (kPBytes / 2);
@@ -121,9 +134,18 @@ __device__ inline float softmax_block(uint32_t t_s, uint32_t p_row, uint32_t sw,
   emit(va, 2);
   tc_wait_ld();
   emit(vb, 3);
-  l = l * corr + sum;
-  m = m_new;
-  return corr;
+  l += (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
+}
+
+// Stores 32 accumulator columns (scaled) of this thread's row as bf16.
+__device__ inline void store_acc32(__nv_bfloat16* dst, const uint32_t (&v)[32], float sc) {
+  uint4* d = reinterpret_cast<uint4*>(dst);
+#pragma unroll
+  for (int q4 = 0; q4 < 4; ++q4)
+    d[q4] = make_uint4(pack2(sc * __uint_as_float(v[8 * q4]), sc * __uint_as_float(v[8 * q4 + 1])),
+                       pack2(sc * __uint_as_float(v[8 * q4 + 2]), sc * __uint_as_float(v[8 * q4 + 3])),
+                       pack2(sc * __uint_as_float(v[8 * q4 + 4]), sc * __uint_as_float(v[8 * q4 + 5])),
+                       pack2(sc * __uint_as_float(v[8 * q4 + 6]), sc * __uint_as_float(v[8 * q4 + 7])));
 }
 
 __device__ inline int kv_position(const AttnParams& p, int s, int hq) {
@@ -133,7 +155,7 @@ __device__ inline int kv_position(const AttnParams& p, int s, int hq) {
 }
 
 // qkv viewed as [S * n_seqs][seq_len][nq]: rows past the end of a sequence read as zeros.
-__global__ void __launch_bounds__(kFwdThreads, 2) attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQKV,
+__global__ void __maxnreg__(200) attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQKV,
                                                                      const AttnParams p, int* status) {
   extern __shared__ unsigned char smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -209,14 +231,14 @@ __global__ void __launch_bounds__(kFwdThreads, 2) attn_fwd_tc_kernel(const __gri
 #pragma unroll
         for (int k = 0; k < kBk / 16; ++k) {
           const uint64_t a = smem_desc(p_s + (k >> 2) * (kPBytes / 2), 16u, 1024u) + 2u * (k & 3);
-          mma1(tm_o, a, bd + (uint64_t)((k * 16 * 128) >> 4), idesc_o, k != 0);
+          mma1(tm_o, a, bd + (uint64_t)((k * 16 * 128) >> 4), idesc_o, (j | k) != 0);
         }
-        commit1(bar(7));                                                          // O_blk complete
         commit1(bar(4));                                                          // V buffer free
+        if (j + 1 == nblk) commit1(bar(7));                                       // O complete
         if (j + 1 < nblk) {
           if (!mbar_wait(bar(1 + ((j + 1) & 1)), ((j + 1) >> 1) & 1, abort_flag, status)) break;
           tc_fence_after();
-          mma_s(j + 1);                                                           // overlaps the threads' work on O
+          mma_s(j + 1);              // its commit also tells the threads that O += P V (j) is done with P and O
           if (!mbar_wait(bar(4), j & 1, abort_flag, status)) break;
           load_v(j + 1);
         }
@@ -230,39 +252,44 @@ __global__ void __launch_bounds__(kFwdThreads, 2) attn_fwd_tc_kernel(const __gri
     // 16-byte piece c (0..7) of this row inside a 64-key half of P (128-byte rows, 128-byte swizzle)
     const uint32_t p_row = p_s + (uint32_t)(r >> 3) * 1024u + (uint32_t)(r & 7) * 128u;
     const uint32_t sw = (uint32_t)(r & 7);
-    float o[kDh];
-#pragma unroll
-    for (int i = 0; i < kDh; ++i) o[i] = 0.f;
     float m = -INFINITY, l = 0.f;
     bool ok = true;
     for (int j = 0; j < nblk; ++j) {
+      // S(j) is complete, and so is every earlier MMA: P and O are at rest until this warp arrives below
       if (!__all_sync(0xffffffffu, mbar_wait(bar(5), j & 1, abort_flag, status))) { ok = false; break; }
       tc_fence_after();
-      const float corr = (j == qb) ? softmax_block<true>(t_s, p_row, sw, qi - j * kBk, p.scale_log2, m, l)
-                                   : softmax_block<false>(t_s, p_row, sw, kBk, p.scale_log2, m, l);
+      auto rescale = [&](float corr) {                   // whole warp: O row *= corr in tensor memory
+        if (j == 0) return;                              // nothing accumulated yet
+#pragma unroll
+        for (int c = 0; c < kDh / 32; ++c) {
+          uint32_t v[32];
+          tc_ld32(t_o + 32 * c, v);
+          tc_wait_ld();
+#pragma unroll
+          for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) * corr);
+          tc_st32(t_o + 32 * c, v);
+        }
+        tc_wait_st();
+      };
+      if (j == qb) softmax_block<true>(t_s, p_row, sw, qi - j * kBk, p.scale_log2, m, l, rescale);
+      else softmax_block<false>(t_s, p_row, sw, kBk, p.scale_log2, m, l, rescale);
       fence_async_smem();                                                         // P: generic writes -> MMA reads
       tc_fence_before();
       mbar_arrive(bar(6));
-      if (!__all_sync(0xffffffffu, mbar_wait(bar(7), j & 1, abort_flag, status))) { ok = false; break; }
+    }
+    if (ok && __all_sync(0xffffffffu, mbar_wait(bar(7), 0, abort_flag, status))) {
       tc_fence_after();
+      const float inv = 1.f / l;
+      const long long row = (long long)s * p.T + (long long)b * p.seq_len + qi;
 #pragma unroll
       for (int c = 0; c < kDh / 32; ++c) {
         uint32_t v[32];
         tc_ld32(t_o + 32 * c, v);
         tc_wait_ld();
-#pragma unroll
-        for (int i = 0; i < 32; ++i) o[32 * c + i] = fmaf(o[32 * c + i], corr, __uint_as_float(v[i]));
+        if (qi < p.seq_len) store_acc32(p.out + row * p.a_sub + hq * kDh + 32 * c, v, inv);
       }
-    }
-    if (ok && qi < p.seq_len) {
-      const float inv = 1.f / l;
-      const long long row = (long long)s * p.T + (long long)b * p.seq_len + qi;
-      uint4* dst = reinterpret_cast<uint4*>(p.out + row * p.a_sub + hq * kDh);
-#pragma unroll
-      for (int c = 0; c < kDh / 8; ++c)
-        dst[c] = make_uint4(pack2(o[8 * c] * inv, o[8 * c + 1] * inv), pack2(o[8 * c + 2] * inv, o[8 * c + 3] * inv),
-                            pack2(o[8 * c + 4] * inv, o[8 * c + 5] * inv), pack2(o[8 * c + 6] * inv, o[8 * c + 7] * inv));
-      p.lse[((long long)s * p.heads + hq) * p.T + (long long)b * p.seq_len + qi] = (m + log2f(l)) * 0.6931471805599453f;
+      if (qi < p.seq_len)
+        p.lse[((long long)s * p.heads + hq) * p.T + (long long)b * p.seq_len + qi] = (m + log2f(l)) * 0.6931471805599453f;
     }
   }
   tc_fence_before();
@@ -298,15 +325,17 @@ constexpr int kDkvSmem = kTileBytes * 6 + 4 * kPBytes + 1024 + 256;   // K, V, Q
 // Element-wise step shared by the two backward kernels: for this thread's row and its 64 columns (two 32-column
 // chunks starting at chunk c0) of S and dP in tensor memory, P = exp2(S * scale - lse2) where visible (column <=
 // k_lim), dS = P * (dP - dl); dS (and P when WRITE_P) go to the operand tiles in shared memory.
-template <bool WRITE_P, bool MASKED>
+// NCHUNK chunks starting at chunk c0 of the 128-key block; the chunk's data sit at column 32 * (c - c_base) of
+// t_s / t_dp (c_base = 0 when a whole block lies in tensor memory, = first chunk of a half block otherwise).
+template <bool WRITE_P, bool MASKED, int NCHUNK = 2>
 __device__ inline void probs_and_ds(uint32_t t_s, uint32_t t_dp, int c0, int r, int k_lim, float scale_log2, float lse2,
-                                    float dl, uint32_t p_tile, uint32_t ds_tile) {
+                                    float dl, uint32_t p_tile, uint32_t ds_tile, int c_base = 0) {
 #pragma unroll
-  for (int cc = 0; cc < 2; ++cc) {
+  for (int cc = 0; cc < NCHUNK; ++cc) {
     const int c = c0 + cc;
     uint32_t vs[32], vd[32];
-    tc_ld32(t_s + 32 * c, vs);
-    tc_ld32(t_dp + 32 * c, vd);
+    tc_ld32(t_s + 32 * (c - c_base), vs);
+    tc_ld32(t_dp + 32 * (c - c_base), vd);
     tc_wait_ld();
     uint32_t wp[16], wd[16];
 #pragma unroll
@@ -325,17 +354,6 @@ __device__ inline void probs_and_ds(uint32_t t_s, uint32_t t_dp, int c0, int r, 
     if (WRITE_P) store_row_chunk32(p_tile, r, c, wp);
     store_row_chunk32(ds_tile, r, c, wd);
   }
-}
-
-// Stores 32 accumulator columns (scaled) of this thread's row as bf16.
-__device__ inline void store_acc32(__nv_bfloat16* dst, const uint32_t (&v)[32], float sc) {
-  uint4* d = reinterpret_cast<uint4*>(dst);
-#pragma unroll
-  for (int q4 = 0; q4 < 4; ++q4)
-    d[q4] = make_uint4(pack2(sc * __uint_as_float(v[8 * q4]), sc * __uint_as_float(v[8 * q4 + 1])),
-                       pack2(sc * __uint_as_float(v[8 * q4 + 2]), sc * __uint_as_float(v[8 * q4 + 3])),
-                       pack2(sc * __uint_as_float(v[8 * q4 + 4]), sc * __uint_as_float(v[8 * q4 + 5])),
-                       pack2(sc * __uint_as_float(v[8 * q4 + 6]), sc * __uint_as_float(v[8 * q4 + 7])));
 }
 
 // ---- dQ: grid (query blocks, kept heads, S * n_seqs).  S / dP of block j + 1 are issued before dQ += dS K of block j

@@ -38,14 +38,19 @@ def rel_fro(got, want):
 
 
 # head_map: per subnet, (kept head ids, kept KV group list) under n_heads / n_kv_heads sharing; None = no sharing
-@pytest.mark.parametrize("S,n_seqs,N,H,dh,gqa", [
-    (2, 2, 64, 2, 64, None),            # whole tiles, two threads per query
-    (2, 3, 77, 3, 16, None),            # ragged sequence length, one thread per query
-    (1, 1, 200, 2, 128, None),          # several key tiles, four threads per query
-    (3, 2, 150, 4, 8, (8, 2)),          # grouped-query sharing: 8 heads in 2 groups, ragged group counts
-    (2, 1, 130, 4, 32, (8, 4)),
+@pytest.mark.parametrize("S,n_seqs,N,H,dh,gqa,ramp", [
+    (2, 2, 64, 2, 64, None, 0.0),       # whole tiles, two threads per query
+    (2, 3, 77, 3, 16, None, 0.0),       # ragged sequence length, one thread per query
+    (1, 1, 200, 2, 128, None, 0.0),     # several key tiles, four threads per query
+    (3, 2, 150, 4, 8, (8, 2), 0.0),     # grouped-query sharing: 8 heads in 2 groups, ragged group counts
+    (2, 1, 130, 4, 32, (8, 4), 0.0),
+    (2, 2, 300, 3, 64, None, 0.0),      # tensor-core path: three key blocks, ragged last block
+    (2, 1, 333, 4, 64, (8, 2), 0.0),    # tensor-core path with grouped-query sharing
+    (1, 2, 640, 2, 64, None, 6.0),      # keys grow along the sequence: the row maxima keep rising, so the
+                                        # lazily updated reference maximum has to move several times
+    (1, 1, 100, 2, 32, None, 6.0),
 ])
-def test_attention_core_parity(B, S, n_seqs, N, H, dh, gqa):
+def test_attention_core_parity(B, S, n_seqs, N, H, dh, gqa, ramp):
     bf = torch.bfloat16
     T = n_seqs * N
     if gqa is None:
@@ -67,6 +72,12 @@ def test_attention_core_parity(B, S, n_seqs, N, H, dh, gqa):
     a, kvw = H * dh, kv_max * dh
     nq = a + 2 * kvw
     QKV = I.normal(81, 1, (S, T, nq), 1.0, I.DTYPE_BF16)
+    if ramp:
+        pos = (np.arange(T) % N) / N
+        QKV = QKV.copy()
+        QKV[:, :, :a] *= 3.0
+        QKV[:, :, a:a + kvw] *= (1.0 + ramp * pos)[None, :, None]
+        QKV = I.f32_from_bf16_bits(I.bf16_bits_from_f32(QKV.astype(np.float32)))      # back onto the bf16 grid
     dA = I.normal(81, 2, (S, T, a), 1.0, I.DTYPE_BF16)
     qkv, d_out = dev(QKV, bf), dev(dA, bf)
     out = torch.zeros(S, T, a, dtype=bf, device="cuda")
