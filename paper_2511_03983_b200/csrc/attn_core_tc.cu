@@ -319,66 +319,85 @@ __device__ inline void store_row_chunk32(uint32_t tile, int r, int c, const uint
 
 constexpr int kBwdTmemCols = 512;
 constexpr int kBwdThreads = 288;        // 8 element-wise warps (two per tensor-memory lane quarter) + the control warp
-constexpr int kDqSmem = kTileBytes * 6 + 2 * kPBytes + 1024 + 128;    // Q, dO, K[2], V[2], dS[2]
-constexpr int kDkvSmem = kTileBytes * 6 + 4 * kPBytes + 1024 + 256;   // K, V, Q[2], dO[2], P[2], dS[2]
 
-// Element-wise step shared by the two backward kernels: for this thread's row and its 64 columns (two 32-column
-// chunks starting at chunk c0) of S and dP in tensor memory, P = exp2(S * scale - lse2) where visible (column <=
-// k_lim), dS = P * (dP - dl); dS (and P when WRITE_P) go to the operand tiles in shared memory.
-// NCHUNK chunks starting at chunk c0 of the 128-key block; the chunk's data sit at column 32 * (c - c_base) of
-// t_s / t_dp (c_base = 0 when a whole block lies in tensor memory, = first chunk of a half block otherwise).
-template <bool WRITE_P, bool MASKED, int NCHUNK = 2>
-__device__ inline void probs_and_ds(uint32_t t_s, uint32_t t_dp, int c0, int r, int k_lim, float scale_log2, float lse2,
-                                    float dl, uint32_t p_tile, uint32_t ds_tile, int c_base = 0) {
-#pragma unroll
-  for (int cc = 0; cc < NCHUNK; ++cc) {
+// Element-wise steps shared by the two backward kernels, for this thread's row and its 64 columns (chunks c0 and
+// c0 + 1 of 32 columns).  They are split so that the tensor pipe can work on dP while the threads are busy with
+// the exponentials:
+//   probs_from_s   P = exp2(S * scale - lse2) where visible (column <= k_lim), kept in registers (fp32) and, when
+//                  WRITE_P, written as bf16 into the operand tile;
+//   ds_from_dp     dS = P * (dP - dl), written as bf16 into the operand tile.
+template <bool WRITE_P, bool MASKED>
+__device__ inline void probs_from_s(uint32_t t_s, int c0, int r, int k_lim, float scale_log2, float lse2, uint32_t p_tile,
+                                    float (&pr)[64]) {
+  uint32_t va[32], vb[32];
+  tc_ld32(t_s + 32 * c0, va);
+  tc_wait_ld();
+  tc_ld32(t_s + 32 * (c0 + 1), vb);
+  auto chunk = [&](const uint32_t (&v)[32], int cc) {
     const int c = c0 + cc;
-    uint32_t vs[32], vd[32];
-    tc_ld32(t_s + 32 * (c - c_base), vs);
-    tc_ld32(t_dp + 32 * (c - c_base), vd);
-    tc_wait_ld();
-    uint32_t wp[16], wd[16];
 #pragma unroll
-    for (int e = 0; e < 16; ++e) {
-      float pr[2], d2[2];
-#pragma unroll
-      for (int h = 0; h < 2; ++h) {
-        const int col = 32 * c + 2 * e + h;
-        pr[h] = ex2_fast(fmaf(__uint_as_float(vs[2 * e + h]), scale_log2, -lse2));
-        if (MASKED) pr[h] = col <= k_lim ? pr[h] : 0.f;
-        d2[h] = pr[h] * (__uint_as_float(vd[2 * e + h]) - dl);
-      }
-      wp[e] = pack2(pr[0], pr[1]);
-      wd[e] = pack2(d2[0], d2[1]);
+    for (int i = 0; i < 32; ++i) {
+      float x = ex2_fast(fmaf(__uint_as_float(v[i]), scale_log2, -lse2));
+      if (MASKED) x = (32 * c + i <= k_lim) ? x : 0.f;
+      pr[32 * cc + i] = x;
     }
-    if (WRITE_P) store_row_chunk32(p_tile, r, c, wp);
-    store_row_chunk32(ds_tile, r, c, wd);
-  }
+    if (WRITE_P) {
+      uint32_t w[16];
+#pragma unroll
+      for (int e = 0; e < 16; ++e) w[e] = pack2(pr[32 * cc + 2 * e], pr[32 * cc + 2 * e + 1]);
+      store_row_chunk32(p_tile, r, c, w);
+    }
+  };
+  chunk(va, 0);
+  tc_wait_ld();
+  chunk(vb, 1);
+}
+__device__ inline void ds_from_dp(uint32_t t_dp, int c0, int r, float dl, uint32_t ds_tile, const float (&pr)[64]) {
+  uint32_t va[32], vb[32];
+  tc_ld32(t_dp + 32 * c0, va);
+  tc_wait_ld();
+  tc_ld32(t_dp + 32 * (c0 + 1), vb);
+  auto chunk = [&](const uint32_t (&v)[32], int cc) {
+    uint32_t w[16];
+#pragma unroll
+    for (int e = 0; e < 16; ++e)
+      w[e] = pack2(pr[32 * cc + 2 * e] * (__uint_as_float(v[2 * e]) - dl),
+                   pr[32 * cc + 2 * e + 1] * (__uint_as_float(v[2 * e + 1]) - dl));
+    store_row_chunk32(ds_tile, r, c0 + cc, w);
+  };
+  chunk(va, 0);
+  tc_wait_ld();
+  chunk(vb, 1);
 }
 
-// ---- dQ: grid (query blocks, kept heads, S * n_seqs).  S / dP of block j + 1 are issued before dQ += dS K of block j
-// (dS is double-buffered), so the MMAs of one block run while the threads work on the next.
+// ---- dQ: grid (query blocks, kept heads, S * n_seqs).  Per key block j: S = Q K^T and dP = dO V^T (128 x 128)
+// into tensor memory, the threads write dS (bf16) into shared memory, dQ += dS K accumulates in tensor memory.
+// S is double-buffered in tensor memory and issued two blocks ahead, dP one block ahead right after the threads
+// released it, so both are complete before the threads need them: the threads turn S(j) into probabilities (the
+// expensive half of their work) while dP(j) is still being computed.  K / V blocks are triple-buffered.
+constexpr int kDqStages = 3;
+constexpr int kDqSmem = kTileBytes * (2 + 2 * kDqStages) + 2 * kPBytes + 1024 + 256;    // Q, dO, K[3], V[3], dS[2]
 __global__ void __launch_bounds__(kBwdThreads) attn_dq_tc_kernel(const __grid_constant__ CUtensorMap tmQKV,
                                                                  const __grid_constant__ CUtensorMap tmDO,
                                                                  const AttnParams p, int* status) {
   extern __shared__ unsigned char smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   unsigned char* gen = smem_raw + (base - smem_u32(smem_raw));
-  const uint32_t q_s = base, do_s = base + kTileBytes, k_s = base + 2 * kTileBytes, v_s = base + 4 * kTileBytes,
-                 ds_s = base + 6 * kTileBytes;
+  const uint32_t q_s = base, do_s = base + kTileBytes, k_s = base + 2 * kTileBytes,
+                 v_s = k_s + kDqStages * kTileBytes, ds_s = v_s + kDqStages * kTileBytes;
   const uint32_t bar0 = ds_s + 2 * kPBytes;
-  volatile uint32_t* ctrl = reinterpret_cast<volatile uint32_t*>(gen + 6 * kTileBytes + 2 * kPBytes);
-  // barriers: 0 q_full, 1-2 kv_full, 3-4 kv_free, 5 sdp_full, 6 ds_ready, 7 dq_full
+  volatile uint32_t* ctrl = reinterpret_cast<volatile uint32_t*>(gen + (2 + 2 * kDqStages) * kTileBytes + 2 * kPBytes);
+  // barriers: 0 q_full, 1-3 kv_full, 4-6 kv_free, 7-8 s_full, 9 dp_full, 10 ds_ready, 11 dq_full
   auto bar = [&](int i) { return bar0 + 8u * i; };
-  volatile uint32_t* tmem_slot = ctrl + 16;
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(ctrl + 17);
+  volatile uint32_t* tmem_slot = ctrl + 32;
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(ctrl + 33);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int qb = blockIdx.x, hq = blockIdx.y, s = blockIdx.z / p.n_seqs, b = blockIdx.z - s * p.n_seqs;
   const int nblk = qb + 1;
   if (threadIdx.x == 256) {
     tma_prefetch_desc(&tmQKV);
     tma_prefetch_desc(&tmDO);
-    for (int i = 0; i < 8; ++i) mbar_init(bar(i), i == 6 ? 256 : 1);
+    for (int i = 0; i < 12; ++i) mbar_init(bar(i), i == 10 ? 256 : 1);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     fence_async_smem();
@@ -392,7 +411,7 @@ __global__ void __launch_bounds__(kBwdThreads) attn_dq_tc_kernel(const __grid_co
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
-  const uint32_t tm_s = tmem, tm_dp = tmem + 128, tm_dq = tmem + 256;
+  const uint32_t tm_dp = tmem + 256, tm_dq = tmem + 384;      // S(j) at columns 128 (j & 1)
 
   if (warp == 8) {
     if (lane == 0) {
@@ -400,7 +419,7 @@ __global__ void __launch_bounds__(kBwdThreads) attn_dq_tc_kernel(const __grid_co
       const int z = blockIdx.z;
       const int k_col = p.a_sub + kvp * kDh, v_col = k_col + p.kv_max * kDh;
       auto load_kv = [&](int j) {
-        const int st = j & 1;
+        const int st = j % kDqStages;
         mbar_expect_tx(bar(1 + st), 2 * kTileBytes);
         tma_load_3d_local(k_s + st * kTileBytes, &tmQKV, bar(1 + st), k_col, j * kBk, z);
         tma_load_3d_local(v_s + st * kTileBytes, &tmQKV, bar(1 + st), v_col, j * kBk, z);
@@ -408,45 +427,58 @@ __global__ void __launch_bounds__(kBwdThreads) attn_dq_tc_kernel(const __grid_co
       mbar_expect_tx(bar(0), 2 * kTileBytes);
       tma_load_3d_local(q_s, &tmQKV, bar(0), hq * kDh, qb * kBq, z);
       tma_load_3d_local(do_s, &tmDO, bar(0), hq * kDh, qb * kBq, z);
-      load_kv(0);
-      if (nblk > 1) load_kv(1);
+      for (int j = 0; j < kDqStages && j < nblk; ++j) load_kv(j);
       constexpr uint32_t idesc_s = idesc_bf16(0, 0, kBq, kBk);       // S = Q K^T, dP = dO V^T : both K-major
       constexpr uint32_t idesc_q = idesc_bf16(0, 1, kBq, kDh);       // dQ = dS K : K as the MN-major B operand
-      auto mma_sdp = [&](int j) {
-        const uint64_t aq = smem_desc(q_s, 16u, 1024u), ao = smem_desc(do_s, 16u, 1024u);
-        const uint64_t bk = smem_desc(k_s + (j & 1) * kTileBytes, 16u, 1024u), bv = smem_desc(v_s + (j & 1) * kTileBytes, 16u, 1024u);
+      auto mma_s = [&](int j) {
+        const uint64_t aq = smem_desc(q_s, 16u, 1024u), bk = smem_desc(k_s + (j % kDqStages) * kTileBytes, 16u, 1024u);
 #pragma unroll
-        for (int k = 0; k < kDh / 16; ++k) mma1(tm_s, aq + 2u * k, bk + 2u * k, idesc_s, k != 0);
+        for (int k = 0; k < kDh / 16; ++k) mma1(tmem + 128u * (j & 1), aq + 2u * k, bk + 2u * k, idesc_s, k != 0);
+        commit1(bar(7 + (j & 1)));
+      };
+      auto mma_dp = [&](int j) {
+        const uint64_t ao = smem_desc(do_s, 16u, 1024u), bv = smem_desc(v_s + (j % kDqStages) * kTileBytes, 16u, 1024u);
 #pragma unroll
         for (int k = 0; k < kDh / 16; ++k) mma1(tm_dp, ao + 2u * k, bv + 2u * k, idesc_s, k != 0);
-        commit1(bar(5));
+        commit1(bar(9));
       };
       bool ok = mbar_wait(bar(0), 0, abort_flag, status) && mbar_wait(bar(1), 0, abort_flag, status);
       if (ok) {
         tc_fence_after();
-        mma_sdp(0);
+        mma_s(0);
+        mma_dp(0);
+        if (nblk > 1) {
+          ok = mbar_wait(bar(2), 0, abort_flag, status);
+          if (ok) {
+            tc_fence_after();
+            mma_s(1);
+          }
+        }
       }
       for (int j = 0; ok && j < nblk; ++j) {
-        const int st = j & 1;
-        if (!mbar_wait(bar(6), j & 1, abort_flag, status)) break;                 // dS of block j is in shared memory,
-        tc_fence_after();                                                         // S / dP of block j have been read
-        if (j + 1 < nblk) {
-          if (!mbar_wait(bar(1 + ((j + 1) & 1)), ((j + 1) >> 1) & 1, abort_flag, status)) break;
-          tc_fence_after();
-          mma_sdp(j + 1);
-        }
+        const int st = j % kDqStages;
+        // dS(j) is in shared memory; S(j) and dP(j) have been read (the threads read S before dP)
+        if (!mbar_wait(bar(10), j & 1, abort_flag, status)) break;
+        tc_fence_after();
+        if (j + 1 < nblk) mma_dp(j + 1);                 // block j + 1 arrived before S(j + 1) was issued
         const uint64_t bd = smem_desc(k_s + st * kTileBytes, (uint32_t)kDh * 128u, 1024u);
-        const uint32_t ds_j = ds_s + st * kPBytes;
+        const uint32_t ds_j = ds_s + (j & 1) * kPBytes;
 #pragma unroll
         for (int k = 0; k < kBk / 16; ++k) {
           const uint64_t a = smem_desc(ds_j + (k >> 2) * (kPBytes / 2), 16u, 1024u) + 2u * (k & 3);
           mma1(tm_dq, a, bd + (uint64_t)((k * 16 * 128) >> 4), idesc_q, (j | k) != 0);
         }
-        commit1(bar(3 + st));
-        if (j + 1 == nblk) commit1(bar(7));
+        commit1(bar(4 + st));                            // block j's K / V are consumed
+        if (j + 1 == nblk) commit1(bar(11));
         if (j + 2 < nblk) {
-          if (!mbar_wait(bar(3 + st), (j >> 1) & 1, abort_flag, status)) break;
-          load_kv(j + 2);
+          const int j2 = j + 2;
+          if (!mbar_wait(bar(1 + j2 % kDqStages), (j2 / kDqStages) & 1, abort_flag, status)) break;
+          tc_fence_after();
+          mma_s(j2);                                     // into the buffer S(j) has just left
+        }
+        if (j + kDqStages < nblk) {
+          if (!mbar_wait(bar(4 + st), (j / kDqStages) & 1, abort_flag, status)) break;
+          load_kv(j + kDqStages);
         }
       }
     }
@@ -461,20 +493,23 @@ __global__ void __launch_bounds__(kBwdThreads) attn_dq_tc_kernel(const __grid_co
     const float dl = row_ok ? p.delta[stat] : 0.f;
     bool ok = true;
     for (int j = 0; j < nblk; ++j) {
-      if (!__all_sync(0xffffffffu, mbar_wait(bar(5), j & 1, abort_flag, status))) { ok = false; break; }
+      float pr[64];
+      if (!__all_sync(0xffffffffu, mbar_wait(bar(7 + (j & 1)), (j >> 1) & 1, abort_flag, status))) { ok = false; break; }
       tc_fence_after();
       const int k_lim = !row_ok ? -1 : ((j == qb) ? qi - j * kBk : kBk);
+      const uint32_t t_s = tmem + lane_off + 128u * (j & 1);
       if (__any_sync(0xffffffffu, k_lim < kBk))      // warp-uniform: the tensor-memory loads inside are warp-wide
-        probs_and_ds<false, true>(tm_s + lane_off, tm_dp + lane_off, 2 * half, r, k_lim, p.scale_log2, lse2, dl, 0u,
-                                  ds_s + (j & 1) * kPBytes);
+        probs_from_s<false, true>(t_s, 2 * half, r, k_lim, p.scale_log2, lse2, 0u, pr);
       else
-        probs_and_ds<false, false>(tm_s + lane_off, tm_dp + lane_off, 2 * half, r, k_lim, p.scale_log2, lse2, dl, 0u,
-                                   ds_s + (j & 1) * kPBytes);
+        probs_from_s<false, false>(t_s, 2 * half, r, k_lim, p.scale_log2, lse2, 0u, pr);
+      if (!__all_sync(0xffffffffu, mbar_wait(bar(9), j & 1, abort_flag, status))) { ok = false; break; }
+      tc_fence_after();
+      ds_from_dp(tm_dp + lane_off, 2 * half, r, dl, ds_s + (j & 1) * kPBytes, pr);
       fence_async_smem();
       tc_fence_before();
-      mbar_arrive(bar(6));
+      mbar_arrive(bar(10));
     }
-    if (ok && __all_sync(0xffffffffu, mbar_wait(bar(7), 0, abort_flag, status))) {
+    if (ok && __all_sync(0xffffffffu, mbar_wait(bar(11), 0, abort_flag, status))) {
       tc_fence_after();
       uint32_t v[32];
       tc_ld32(tm_dq + lane_off + 32 * half, v);
@@ -498,8 +533,12 @@ __global__ void __launch_bounds__(kBwdThreads) attn_dq_tc_kernel(const __grid_co
   }
 }
 
-// ---- dK, dV: grid (key blocks, KV positions, S * n_seqs).  Units (kept head, query block) stream through; S / dP
-// of unit n + 1 are issued before dV += P^T dO, dK += dS^T Q of unit n (P and dS are double-buffered).
+// ---- dK, dV: grid (key blocks, KV positions, S * n_seqs).  Units (kept head, query block) stream through with the
+// same schedule as the dQ kernel: S two units ahead into one of two tensor-memory buffers, dP one unit ahead, the
+// threads form P from S while dP is computed; dV += P^T dO and dK += dS^T Q accumulate in tensor memory.  P is
+// double-buffered in shared memory; dS has one tile, rewritten once the previous unit's MMAs are done with it.
+constexpr int kDkvStages = 3;
+constexpr int kDkvSmem = kTileBytes * (2 + 2 * kDkvStages) + 3 * kPBytes + 1024 + 256;   // K, V, Q[3], dO[3], P[2], dS
 __global__ void __launch_bounds__(kBwdThreads) attn_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmQKV,
                                                                   const __grid_constant__ CUtensorMap tmDO,
                                                                   const AttnParams p, int* status) {
@@ -508,14 +547,14 @@ __global__ void __launch_bounds__(kBwdThreads) attn_dkv_tc_kernel(const __grid_c
   __shared__ int n_match_s;
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   unsigned char* gen = smem_raw + (base - smem_u32(smem_raw));
-  const uint32_t k_s = base, v_s = base + kTileBytes, q_s = base + 2 * kTileBytes, do_s = base + 4 * kTileBytes,
-                 p_s = base + 6 * kTileBytes, ds_s = p_s + 2 * kPBytes;
-  const uint32_t bar0 = ds_s + 2 * kPBytes;
-  volatile uint32_t* ctrl = reinterpret_cast<volatile uint32_t*>(gen + 6 * kTileBytes + 4 * kPBytes);
-  // barriers: 0 kv_full, 1-2 q_full, 3-4 q_free, 5 sdp_full, 6 pds_ready, 7 acc_full
+  const uint32_t k_s = base, v_s = base + kTileBytes, q_s = base + 2 * kTileBytes,
+                 do_s = q_s + kDkvStages * kTileBytes, p_s = do_s + kDkvStages * kTileBytes, ds_s = p_s + 2 * kPBytes;
+  const uint32_t bar0 = ds_s + kPBytes;
+  volatile uint32_t* ctrl = reinterpret_cast<volatile uint32_t*>(gen + (2 + 2 * kDkvStages) * kTileBytes + 3 * kPBytes);
+  // barriers: 0 kv_full, 1-3 q_full, 4-6 q_free, 7-8 s_full, 9 dp_full, 10 pds_ready, 11 acc_full, 12 acc_done
   auto bar = [&](int i) { return bar0 + 8u * i; };
-  volatile uint32_t* tmem_slot = ctrl + 16;
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(ctrl + 17);
+  volatile uint32_t* tmem_slot = ctrl + 32;
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(ctrl + 33);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int kb = blockIdx.x, kvp = blockIdx.y, s = blockIdx.z / p.n_seqs, b = blockIdx.z - s * p.n_seqs;
   const int nqb = (p.seq_len + kBq - 1) / kBq;
@@ -523,7 +562,7 @@ __global__ void __launch_bounds__(kBwdThreads) attn_dkv_tc_kernel(const __grid_c
   if (threadIdx.x == 256) {
     tma_prefetch_desc(&tmQKV);
     tma_prefetch_desc(&tmDO);
-    for (int i = 0; i < 8; ++i) mbar_init(bar(i), i == 6 ? 256 : 1);
+    for (int i = 0; i < 13; ++i) mbar_init(bar(i), i == 10 ? 256 : 1);
     *abort_flag = 0;
     int n = 0;
     if (kvp < held)
@@ -542,7 +581,7 @@ __global__ void __launch_bounds__(kBwdThreads) attn_dkv_tc_kernel(const __grid_c
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
-  const uint32_t tm_s = tmem, tm_dp = tmem + 128, tm_dv = tmem + 256, tm_dk = tmem + 320;
+  const uint32_t tm_dp = tmem + 256, tm_dv = tmem + 384, tm_dk = tmem + 448;   // S(n) at columns 128 (n & 1)
   const int per_head = nqb - kb;                         // query blocks kb .. nqb-1
   const int total = n_match_s * per_head;                // units (head, query block)
 
@@ -550,7 +589,7 @@ __global__ void __launch_bounds__(kBwdThreads) attn_dkv_tc_kernel(const __grid_c
     if (lane == 0 && total > 0) {
       const int z = blockIdx.z;
       auto load_q = [&](int n) {
-        const int st = n & 1, hq = match[n / per_head], i = kb + n % per_head;
+        const int st = n % kDkvStages, hq = match[n / per_head], i = kb + n % per_head;
         mbar_expect_tx(bar(1 + st), 2 * kTileBytes);
         tma_load_3d_local(q_s + st * kTileBytes, &tmQKV, bar(1 + st), hq * kDh, i * kBq, z);
         tma_load_3d_local(do_s + st * kTileBytes, &tmDO, bar(1 + st), hq * kDh, i * kBq, z);
@@ -558,49 +597,62 @@ __global__ void __launch_bounds__(kBwdThreads) attn_dkv_tc_kernel(const __grid_c
       mbar_expect_tx(bar(0), 2 * kTileBytes);
       tma_load_3d_local(k_s, &tmQKV, bar(0), p.a_sub + kvp * kDh, kb * kBk, z);
       tma_load_3d_local(v_s, &tmQKV, bar(0), p.a_sub + (p.kv_max + kvp) * kDh, kb * kBk, z);
-      load_q(0);
-      if (total > 1) load_q(1);
+      for (int n = 0; n < kDkvStages && n < total; ++n) load_q(n);
       constexpr uint32_t idesc_s = idesc_bf16(0, 0, kBq, kBk);       // S = Q K^T, dP = dO V^T
       constexpr uint32_t idesc_t = idesc_bf16(1, 1, kBk, kDh);       // dV = P^T dO, dK = dS^T Q : both MN-major
-      auto mma_sdp = [&](int n) {
-        const int st = n & 1;
-        const uint64_t aq = smem_desc(q_s + st * kTileBytes, 16u, 1024u), ao = smem_desc(do_s + st * kTileBytes, 16u, 1024u);
-        const uint64_t bk = smem_desc(k_s, 16u, 1024u), bv = smem_desc(v_s, 16u, 1024u);
+      auto mma_s = [&](int n) {
+        const uint64_t aq = smem_desc(q_s + (n % kDkvStages) * kTileBytes, 16u, 1024u), bk = smem_desc(k_s, 16u, 1024u);
 #pragma unroll
-        for (int k = 0; k < kDh / 16; ++k) mma1(tm_s, aq + 2u * k, bk + 2u * k, idesc_s, k != 0);
+        for (int k = 0; k < kDh / 16; ++k) mma1(tmem + 128u * (n & 1), aq + 2u * k, bk + 2u * k, idesc_s, k != 0);
+        commit1(bar(7 + (n & 1)));
+      };
+      auto mma_dp = [&](int n) {
+        const uint64_t ao = smem_desc(do_s + (n % kDkvStages) * kTileBytes, 16u, 1024u), bv = smem_desc(v_s, 16u, 1024u);
 #pragma unroll
         for (int k = 0; k < kDh / 16; ++k) mma1(tm_dp, ao + 2u * k, bv + 2u * k, idesc_s, k != 0);
-        commit1(bar(5));
+        commit1(bar(9));
       };
       bool ok = mbar_wait(bar(0), 0, abort_flag, status) && mbar_wait(bar(1), 0, abort_flag, status);
       if (ok) {
         tc_fence_after();
-        mma_sdp(0);
+        mma_s(0);
+        mma_dp(0);
+        if (total > 1) {
+          ok = mbar_wait(bar(2), 0, abort_flag, status);
+          if (ok) {
+            tc_fence_after();
+            mma_s(1);
+          }
+        }
       }
       for (int n = 0; ok && n < total; ++n) {
-        const int st = n & 1;
-        if (!mbar_wait(bar(6), n & 1, abort_flag, status)) break;                 // P and dS of unit n are in shared memory,
-        tc_fence_after();                                                         // S / dP of unit n have been read
-        if (n + 1 < total) {
-          if (!mbar_wait(bar(1 + ((n + 1) & 1)), ((n + 1) >> 1) & 1, abort_flag, status)) break;
-          tc_fence_after();
-          mma_sdp(n + 1);
-        }
+        const int st = n % kDkvStages;
+        // P and dS of unit n are in shared memory; S(n) and dP(n) have been read (the threads read S before dP)
+        if (!mbar_wait(bar(10), n & 1, abort_flag, status)) break;
+        tc_fence_after();
+        if (n + 1 < total) mma_dp(n + 1);                // unit n + 1 arrived before S(n + 1) was issued
         // A = P^T / dS^T: rows of the tile are the contraction index (queries), 64 keys per 128-byte row, the two
         // 64-key halves 16 KB apart; B = dO / Q with rows = queries.
-        const uint64_t ap = smem_desc(p_s + st * kPBytes, (uint32_t)(kPBytes / 2), 1024u);
-        const uint64_t ad = smem_desc(ds_s + st * kPBytes, (uint32_t)(kPBytes / 2), 1024u);
+        const uint64_t ap = smem_desc(p_s + (n & 1) * kPBytes, (uint32_t)(kPBytes / 2), 1024u);
+        const uint64_t ad = smem_desc(ds_s, (uint32_t)(kPBytes / 2), 1024u);
         const uint64_t bo = smem_desc(do_s + st * kTileBytes, (uint32_t)kDh * 128u, 1024u);
         const uint64_t bq = smem_desc(q_s + st * kTileBytes, (uint32_t)kDh * 128u, 1024u);
 #pragma unroll
         for (int k = 0; k < kBq / 16; ++k) mma1(tm_dv, ap + (uint64_t)(k * 128), bo + (uint64_t)(k * 128), idesc_t, (n | k) != 0);
 #pragma unroll
         for (int k = 0; k < kBq / 16; ++k) mma1(tm_dk, ad + (uint64_t)(k * 128), bq + (uint64_t)(k * 128), idesc_t, (n | k) != 0);
-        commit1(bar(3 + st));
-        if (n + 1 == total) commit1(bar(7));
+        commit1(bar(12));                                // the dS tile may be rewritten
+        commit1(bar(4 + st));                            // unit n's Q / dO are consumed
+        if (n + 1 == total) commit1(bar(11));
         if (n + 2 < total) {
-          if (!mbar_wait(bar(3 + st), (n >> 1) & 1, abort_flag, status)) break;
-          load_q(n + 2);
+          const int n2 = n + 2;
+          if (!mbar_wait(bar(1 + n2 % kDkvStages), (n2 / kDkvStages) & 1, abort_flag, status)) break;
+          tc_fence_after();
+          mma_s(n2);                                     // into the buffer S(n) has just left; P(n & 1) is free after it
+        }
+        if (n + kDkvStages < total) {
+          if (!mbar_wait(bar(4 + st), (n / kDkvStages) & 1, abort_flag, status)) break;
+          load_q(n + kDkvStages);
         }
       }
     }
@@ -610,24 +662,28 @@ __global__ void __launch_bounds__(kBwdThreads) attn_dkv_tc_kernel(const __grid_c
     const uint32_t lane_off = (uint32_t)(quarter * 32) << 16;
     bool ok = true;
     for (int n = 0; n < total; ++n) {
+      float pr[64];
       const int hq = match[n / per_head], i = kb + n % per_head;
       const int qi = i * kBq + r;
       const bool row_ok = qi < p.seq_len;
       const long long stat = ((long long)s * p.heads + hq) * p.T + (long long)b * p.seq_len + qi;
       const float lse2 = row_ok ? p.lse[stat] * 1.4426950408889634f : 0.f;
       const float dl = row_ok ? p.delta[stat] : 0.f;
-      if (!__all_sync(0xffffffffu, mbar_wait(bar(5), n & 1, abort_flag, status))) { ok = false; break; }
+      if (!__all_sync(0xffffffffu, mbar_wait(bar(7 + (n & 1)), (n >> 1) & 1, abort_flag, status))) { ok = false; break; }
       tc_fence_after();
       const int k_lim = !row_ok ? -1 : ((i == kb) ? r : kBk);                     // diagonal block: keys <= query
+      const uint32_t t_s = tmem + lane_off + 128u * (n & 1);
       if (__any_sync(0xffffffffu, k_lim < kBk))      // warp-uniform: the tensor-memory loads inside are warp-wide
-        probs_and_ds<true, true>(tm_s + lane_off, tm_dp + lane_off, 2 * half, r, k_lim, p.scale_log2, lse2, dl,
-                                 p_s + (n & 1) * kPBytes, ds_s + (n & 1) * kPBytes);
+        probs_from_s<true, true>(t_s, 2 * half, r, k_lim, p.scale_log2, lse2, p_s + (n & 1) * kPBytes, pr);
       else
-        probs_and_ds<true, false>(tm_s + lane_off, tm_dp + lane_off, 2 * half, r, k_lim, p.scale_log2, lse2, dl,
-                                  p_s + (n & 1) * kPBytes, ds_s + (n & 1) * kPBytes);
+        probs_from_s<true, false>(t_s, 2 * half, r, k_lim, p.scale_log2, lse2, p_s + (n & 1) * kPBytes, pr);
+      if (!__all_sync(0xffffffffu, mbar_wait(bar(9), n & 1, abort_flag, status))) { ok = false; break; }
+      if (n > 0 && !__all_sync(0xffffffffu, mbar_wait(bar(12), (n - 1) & 1, abort_flag, status))) { ok = false; break; }
+      tc_fence_after();
+      ds_from_dp(tm_dp + lane_off, 2 * half, r, dl, ds_s, pr);
       fence_async_smem();
       tc_fence_before();
-      mbar_arrive(bar(6));
+      mbar_arrive(bar(10));
     }
     // accumulator rows are keys now: thread r owns key kb * 128 + r; the first four warps store dV, the others dK
     const int kj = kb * kBk + r;
@@ -636,7 +692,7 @@ __global__ void __launch_bounds__(kBwdThreads) attn_dkv_tc_kernel(const __grid_c
     if (total == 0) {                                    // a KV position this subnet does not hold: zero gradient
       if (kj < p.seq_len)
         for (int c = 0; c < kDh / 8; ++c) reinterpret_cast<uint4*>(dst)[c] = make_uint4(0, 0, 0, 0);
-    } else if (ok && __all_sync(0xffffffffu, mbar_wait(bar(7), 0, abort_flag, status))) {
+    } else if (ok && __all_sync(0xffffffffu, mbar_wait(bar(11), 0, abort_flag, status))) {
       tc_fence_after();
       const float sc = half ? p.scale_log2 * 0.6931471805599453f : 1.f;          // dK carries 1 / sqrt(d_head)
 #pragma unroll
