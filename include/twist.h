@@ -219,6 +219,12 @@ typedef struct {
   twist_optimizer opt;      /* bwd: optimiser of the fused update */
   float *m_gu, *v_gu;       /* device fp32 Adam moments of w_gu   [S][g*f_sub][d] */
   float *m_down, *v_down;   /* device fp32 Adam moments of w_down [S][f_sub][d] */
+  /* Optional activation mask (Sec. 4.1, Masked TwIST: y = M * f(x)): device uint8 [S][f_sub], 1 = neuron active,
+   * 0 = masked out.  The weights are then the full-width model (f_sub = all neurons) and worker s behaves like
+   * the subnet of its active neurons: fwd hh = mask * act(pre) (pre is stored unmasked), bwd dHh = mask * dHh, so
+   * the gradients of masked neurons' rows are exactly zero and the fused update leaves them untouched (Hybrid
+   * TwIST's central model trains this way on its full copy).  NULL: no mask.  bf16 dtype only. */
+  const uint8_t* hidden_mask;
 } twist_ffn_args;
 
 /* Fused loss.  When `tgt` is set, twist_subnet_ffn_fwd / twist_subnet_attn_proj_fwd also evaluate the loss

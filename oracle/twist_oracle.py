@@ -222,25 +222,30 @@ def _plus(v, residual):
     return v if residual is None else v + residual
 
 
-def ffn_fwd(X, W_up, W_gate, W_down, kind, alpha, lowp, residual=None):
+def ffn_fwd(X, W_up, W_gate, W_down, kind, alpha, lowp, residual=None, hidden_mask=None):
     """Y = alpha * act(X W_up^T) W_down  (MLP)  or  alpha * (silu(X W_gate^T) * (X W_up^T)) W_down.
     Returns Y [T, d] and the tensors kept for the backward pass (stored precision).
-    `residual` (App. A, Transformer Layer Architecture, final output) is added before Y is stored."""
+    `residual` (App. A, Transformer Layer Architecture, final output) is added before Y is stored.
+    `hidden_mask` [f] of 0/1 (Sec. 4.1, Masked TwIST): the activations are multiplied by it, y = M * f(x)."""
     U = X @ W_up.T
+    mask = 1.0 if hidden_mask is None else np.asarray(hidden_mask, dtype=np.float64)[None, :]
     if kind == FFN_SWIGLU:
         G = X @ W_gate.T
-        Hh = (G * _sigmoid(G)) * U
+        Hh = mask * ((G * _sigmoid(G)) * U)
         saved = {"G": _q(G, lowp), "U": _q(U, lowp), "Hh": _q(Hh, lowp)}
     else:
-        saved = {"U": _q(U, lowp), "Hh": _q(_act(U, kind), lowp)}
+        saved = {"U": _q(U, lowp), "Hh": _q(mask * _act(U, kind), lowp)}
     Y = _q(_plus(alpha * (saved["Hh"] @ W_down), residual), lowp)
     return Y, saved
 
 
-def ffn_bwd(dY, X, saved, W_up, W_gate, W_down, kind, alpha, lowp, residual=None):
+def ffn_bwd(dY, X, saved, W_up, W_gate, W_down, kind, alpha, lowp, residual=None, hidden_mask=None):
     """Exact chain rule through ffn_fwd.  Returns dX and dW_up, dW_gate, dW_down ([f', d] each).
-    `residual`: gradient arriving over the skip connection, added to dX before it is stored."""
+    `residual`: gradient arriving over the skip connection, added to dX before it is stored.
+    `hidden_mask`: the mask of the forward pass; the gradient reaching the activations is multiplied by it."""
     dHh = alpha * (dY @ W_down.T)
+    if hidden_mask is not None:
+        dHh = dHh * np.asarray(hidden_mask, dtype=np.float64)[None, :]
     dW_down = alpha * (saved["Hh"].T @ dY)
     if kind == FFN_SWIGLU:
         G, U = saved["G"], saved["U"]

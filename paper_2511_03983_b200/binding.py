@@ -73,7 +73,7 @@ class FfnArgs(C.Structure):
                 ("dw_down", C.c_void_p), ("tgt", C.c_void_p), ("loss", C.c_void_p), ("loss_ws", C.c_void_p),
                 ("loss_ws_bytes", C.c_size_t), ("y_residual", C.c_void_p), ("dx_residual", C.c_void_p),
                 ("opt", Optimizer), ("m_gu", C.c_void_p), ("v_gu", C.c_void_p), ("m_down", C.c_void_p),
-                ("v_down", C.c_void_p)]
+                ("v_down", C.c_void_p), ("hidden_mask", C.c_void_p)]
 
 
 class ProjArgs(C.Structure):
@@ -217,15 +217,17 @@ def _ws_bytes(ws) -> int:
 
 def ffn_args(ffn_kind, dtype, n_subnets, tokens, d_model, f_sub, out_scale, lr=0.0, opt: Optional[Optimizer] = None,
              **t) -> FfnArgs:
-    """Marshals twist_ffn_args.  tgt / loss / loss_ws request the fused loss of the forward call."""
+    """Marshals twist_ffn_args.  tgt / loss / loss_ws request the fused loss of the forward call; hidden_mask
+    (uint8 [S][f_sub]) the activation mask of Masked TwIST."""
     names = ["x", "w_gu", "w_down", "w_gu_master", "w_down_master", "pre", "hh", "y", "dy", "dpre", "dx", "dw_gu",
              "dw_down", "tgt", "loss", "loss_ws"]
     moments = ["m_gu", "v_gu", "m_down", "v_down"]
-    unknown = set(t) - set(names) - {"y_residual", "dx_residual"} - set(moments)
+    unknown = set(t) - set(names) - {"y_residual", "dx_residual", "hidden_mask"} - set(moments)
     assert not unknown, unknown
     a = FfnArgs(ffn_kind, dtype, n_subnets, tokens, d_model, f_sub, out_scale, lr, *[_ptr(t.get(n)) for n in names],
                 _ws_bytes(t.get("loss_ws")), _ptr(t.get("y_residual")), _ptr(t.get("dx_residual")),
-                opt if opt is not None else Optimizer(), *[_ptr(t.get(n)) for n in moments])
+                opt if opt is not None else Optimizer(), *[_ptr(t.get(n)) for n in moments],
+                _ptr(t.get("hidden_mask")))
     a._keepalive = list(t.values())      # the struct holds raw addresses: keep the tensors alive as long as it lives
     return a
 

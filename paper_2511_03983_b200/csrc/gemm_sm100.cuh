@@ -75,6 +75,7 @@ struct GemmParams {
   float* adam_m;        // ADAM: first / second moment of the group's weights, fp32 [g][M][N]
   float* adam_v;
   float beta1, beta2, adam_eps, bias1, bias2;   // ADAM: decay rates, epsilon, 1 / (1 - beta^t)
+  const uint8_t* hmask;  // activation epilogues: per group N bytes, 1 = column active, 0 = masked out; may be null
   float* dw;            // SGD: optional fp32 gradient dump [g][M][N].  MSE: partial sums, 16 per tile (2 CTAs x 8 warps)
   const int32_t* valid_cols;   // MSE: valid columns per column group and subnet [groups], or null (all valid)
   int seg_begin, seg_width;    // MSE: columns [0, seg_begin) valid, then groups of seg_width columns (see twist_mse_fwd_bwd)
@@ -99,6 +100,16 @@ __host__ __device__ constexpr int epi_bufs(int epi) { return epi_slots(epi) == 3
 
 // Registers of one 32-column chunk of accumulator words.
 template <int EPI> struct EpiAcc { uint32_t r0[32]; };
+// Eight consecutive mask bytes of group g starting at column `col` (a multiple of 8, col + 8 <= N) as factors.
+__device__ inline void mask8(const uint8_t* hmask, int g, int N, int col, float (&m)[8]) {
+  uint2 w;
+  asm volatile("ld.global.nc.v2.u32 {%0,%1}, [%2];" : "=r"(w.x), "=r"(w.y) : "l"(hmask + (long long)g * N + col));
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    m[i] = (float)((w.x >> (8 * i)) & 1u);
+    m[4 + i] = (float)((w.y >> (8 * i)) & 1u);
+  }
+}
 template <> struct EpiAcc<EPI_SWIGLU_FWD> { uint32_t r0[32], r1[32]; };
 
 // ---------------------------------------------------------------------------------------------
@@ -548,6 +559,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
 #pragma unroll
           for (int q = 0; q < 4; ++q) {
             const uint32_t* r = a.r0 + 8 * q;
+            float hm[8] = {1.f, 1.f, 1.f, 1.f, 1.f, 1.f, 1.f, 1.f};
+            if constexpr (EPI == EPI_SWIGLU_FWD || EPI == EPI_ACT_FWD || EPI == EPI_DSWIGLU || EPI == EPI_DACT) {
+              if (p.hmask && n + 8 * q < p.N) mask8(p.hmask, g, p.N, n + 8 * q, hm);     // uniform branch
+            }
             if constexpr (EPI == EPI_STORE) {
               sts128(piece(b0, q), make_uint4(pack2(p.scale * __uint_as_float(r[0]), p.scale * __uint_as_float(r[1])),
                                               pack2(p.scale * __uint_as_float(r[2]), p.scale * __uint_as_float(r[3])),
@@ -584,7 +599,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                 const float u0 = __uint_as_float(ru[2 * h]), u1 = __uint_as_float(ru[2 * h + 1]);
                 wg[h] = pack2(g0, g1);
                 wu[h] = pack2(u0, u1);
-                wh[h] = pack2(g0 * sigmoid_fast(g0) * u0, g1 * sigmoid_fast(g1) * u1);
+                wh[h] = pack2(g0 * sigmoid_fast(g0) * u0 * hm[2 * h], g1 * sigmoid_fast(g1) * u1 * hm[2 * h + 1]);
               }
               sts128(piece(b0, q), make_uint4(wg[0], wg[1], wg[2], wg[3]));
               sts128(piece(b1, q), make_uint4(wu[0], wu[1], wu[2], wu[3]));
@@ -598,7 +613,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
 #pragma unroll
               for (int h = 0; h < 4; ++h) {
                 wp[h] = pack2(xin[2 * h], xin[2 * h + 1]);
-                wh[h] = pack2(yv[2 * h], yv[2 * h + 1]);
+                wh[h] = pack2(yv[2 * h] * hm[2 * h], yv[2 * h + 1] * hm[2 * h + 1]);
               }
               sts128(piece(b0, q), make_uint4(wp[0], wp[1], wp[2], wp[3]));
               sts128(piece(b1, q), make_uint4(wh[0], wh[1], wh[2], wh[3]));
@@ -611,7 +626,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                 float dg[2], du[2];
 #pragma unroll
                 for (int e = 0; e < 2; ++e) {
-                  const float dh = p.scale * __uint_as_float(r[2 * h + e]);
+                  const float dh = p.scale * __uint_as_float(r[2 * h + e]) * hm[2 * h + e];
                   const float gt = e ? bf_hi(pg[h]) : bf_lo(pg[h]);
                   const float up = e ? bf_hi(pu[h]) : bf_lo(pu[h]);
                   const float sg = sigmoid_fast(gt);
@@ -642,8 +657,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
               act_grad8(xin, p.act_kind, gv);
 #pragma unroll
               for (int h = 0; h < 4; ++h)
-                w[h] = pack2(p.scale * __uint_as_float(r[2 * h]) * gv[2 * h],
-                             p.scale * __uint_as_float(r[2 * h + 1]) * gv[2 * h + 1]);
+                w[h] = pack2(p.scale * __uint_as_float(r[2 * h]) * gv[2 * h] * hm[2 * h],
+                             p.scale * __uint_as_float(r[2 * h + 1]) * gv[2 * h + 1] * hm[2 * h + 1]);
               sts128(piece(b0, q), make_uint4(w[0], w[1], w[2], w[3]));
             }
           }

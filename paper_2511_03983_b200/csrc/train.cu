@@ -95,6 +95,7 @@ extern "C" int32_t twist_subnet_ffn_fwd(const twist_ffn_args* a, void* stream) {
   if (!a->x || !a->w_gu || !a->w_down || !a->pre || !a->hh || (!a->y && !fused)) return TWIST_ERR_NULL;
   if (a->dtype == TWIST_FP32 && !a->y) return TWIST_ERR_NULL;
   if (a->y_residual && (fused || a->dtype == TWIST_FP32)) return TWIST_ERR_UNSUPPORTED;
+  if (a->hidden_mask && a->dtype == TWIST_FP32) return TWIST_ERR_UNSUPPORTED;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const int S = a->n_subnets, T = a->tokens, d = a->d_model, f = a->f_sub;
   const bool swiglu = a->ffn_kind == TWIST_FFN_SWIGLU;
@@ -118,6 +119,7 @@ extern "C" int32_t twist_subnet_ffn_fwd(const twist_ffn_args* a, void* stream) {
   p.out1 = static_cast<__nv_bfloat16*>(a->hh);
   p.b_split = f;
   p.act_kind = a->ffn_kind;
+  p.hmask = a->hidden_mask;
   TWIST_TRY(launch_gemm_bf16(0, swiglu ? EPI_SWIGLU_FWD : EPI_ACT_FWD, GemmOperand{a->x, T, d},
                              GemmOperand{a->w_gu, gf, d}, p, st));
   // Y = out_scale * hh W_down  (+ loss and dY in the same epilogue when requested)
@@ -140,7 +142,7 @@ extern "C" int32_t twist_subnet_ffn_bwd(const twist_ffn_args* a, void* stream) {
   const int gf = swiglu ? 2 * f : f;
   if (a->dtype == TWIST_FP32) {
     if (!a->dw_gu || !a->dw_down) return TWIST_ERR_NULL;
-    if (a->dx_residual || a->opt.kind != TWIST_OPT_SGD) return TWIST_ERR_UNSUPPORTED;
+    if (a->dx_residual || a->opt.kind != TWIST_OPT_SGD || a->hidden_mask) return TWIST_ERR_UNSUPPORTED;
     const float* x = static_cast<const float*>(a->x);
     const float* dy = static_cast<const float*>(a->dy);
     const float* pre = static_cast<const float*>(a->pre);
@@ -172,6 +174,7 @@ extern "C" int32_t twist_subnet_ffn_bwd(const twist_ffn_args* a, void* stream) {
   p.out0 = static_cast<__nv_bfloat16*>(a->dpre);
   p.in0 = static_cast<const __nv_bfloat16*>(a->pre);
   p.act_kind = a->ffn_kind;
+  p.hmask = a->hidden_mask;
   TWIST_TRY(launch_gemm_bf16(0, swiglu ? EPI_DSWIGLU : EPI_DACT, GemmOperand{a->dy, T, d}, GemmOperand{a->w_down, f, d},
                              p, st));
   // dX = dpre W_gu   (before the weights are updated)

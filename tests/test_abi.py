@@ -80,7 +80,10 @@ def test_host_side_argument_checks():
     a = B.FfnArgs(B.FFN_SWIGLU, B.BF16, 2, 128, 64, 96, 1.0, 0.0, 0x1000, 0x1000, 0x1000, None, None, 0x1000, 0x1000,
                   0x1000, 0x1000, None, None, None, None, 0x1000, 0x1000, 0x1000, 1 << 30, 0x1000, None)
     assert h.twist_subnet_ffn_fwd(C.byref(a), None) == B.ERR_UNSUPPORTED
-
+    # the activation mask of Masked TwIST exists in the bf16 path only
+    a = B.FfnArgs(B.FFN_SWIGLU, B.FP32, 2, 128, 64, 96, 1.0, 0.0, 0x1000, 0x1000, 0x1000, None, None, 0x1000, 0x1000, 0x1000)
+    a.hidden_mask = 0x1000
+    assert h.twist_subnet_ffn_fwd(C.byref(a), None) == B.ERR_UNSUPPORTED
 
 
 def test_missing_library_fails_loudly(monkeypatch, tmp_path):

@@ -213,7 +213,7 @@ def test_mse_parity(B, dtype):
 
 # --------------------------------------------------------------------------------------------- FFN / projections
 
-def _ffn_case(B, kind, dtype, S, T, d, f, alpha, lr, seed):
+def _ffn_case(B, kind, dtype, S, T, d, f, alpha, lr, seed, mask_keep=0):
     lowp = dtype == I.DTYPE_BF16
     td = torch.bfloat16 if lowp else torch.float32
     g = 2 if kind == I.FFN_SWIGLU else 1
@@ -227,9 +227,16 @@ def _ffn_case(B, kind, dtype, S, T, d, f, alpha, lr, seed):
     pre, hh, y, dpre, dx = t(S, T, g * f), t(S, T, f), t(S, T, d), t(S, T, g * f), t(S, T, d)
     dw_gu = torch.zeros(S, g * f, d, dtype=torch.float32, device="cuda")
     dw_down = torch.zeros(S, f, d, dtype=torch.float32, device="cuda")
+    masks, extra = [None] * S, {}
+    if mask_keep:          # Masked TwIST (Sec. 4.1): worker s sees only its active neurons of the full-width model
+        rng = np.random.default_rng(seed)
+        masks = [np.zeros(f, dtype=np.uint8) for _ in range(S)]
+        for s in range(S):
+            masks[s][rng.choice(f, mask_keep, replace=False)] = 1
+        extra = dict(hidden_mask=dev(np.stack(masks)))
     a = B.ffn_args(kind, dtype, S, T, d, f, alpha, lr, x=dev(X, td), w_gu=w_gu, w_down=w_down, w_gu_master=m_gu,
                    w_down_master=m_down, pre=pre, hh=hh, y=y, dy=dev(dY, td), dpre=dpre, dx=dx, dw_gu=dw_gu,
-                   dw_down=dw_down)
+                   dw_down=dw_down, **extra)
     B.twist_subnet_ffn_fwd(a)
     B.twist_subnet_ffn_bwd(a)
     torch.cuda.synchronize()
@@ -240,8 +247,14 @@ def _ffn_case(B, kind, dtype, S, T, d, f, alpha, lr, seed):
         Wu_s = Wgu[s, (g - 1) * f:].astype(np.float64)
         Wd_s = Wd[s].astype(np.float64)
         Xs, dYs = X[s].astype(np.float64), dY[s].astype(np.float64)
-        Yw, saved = o.ffn_fwd(Xs, Wu_s, Wg_s, Wd_s, kind, alpha, lowp)
-        dXw, dWu, dWg, dWd = o.ffn_bwd(dYs, Xs, saved, Wu_s, Wg_s, Wd_s, kind, alpha, lowp)
+        Yw, saved = o.ffn_fwd(Xs, Wu_s, Wg_s, Wd_s, kind, alpha, lowp, hidden_mask=masks[s])
+        dXw, dWu, dWg, dWd = o.ffn_bwd(dYs, Xs, saved, Wu_s, Wg_s, Wd_s, kind, alpha, lowp, hidden_mask=masks[s])
+        if mask_keep:      # masked-out neurons: zero activation, exactly zero gradient rows, weights untouched
+            off = np.flatnonzero(masks[s] == 0)
+            rows = np.concatenate([off, off + f]) if g == 2 else off
+            assert np.all(host(hh[s])[:, off] == 0)
+            assert np.all(host(dw_gu[s])[rows] == 0) and np.all(host(dw_down[s])[off] == 0)
+            assert np.array_equal(host(m_gu[s])[rows], Wgu[s][rows]) and np.array_equal(host(m_down[s])[off], Wd[s][off])
         pre_w = np.concatenate([saved["G"], saved["U"]], axis=1) if g == 2 else saved["U"]
         dWgu = np.concatenate([dWg, dWu], axis=0) if g == 2 else dWu
         assert rel_fro(host(pre[s]), pre_w) < tol, ("pre", s)
@@ -276,6 +289,53 @@ def test_ffn_fp32_parity(B, kind):
 ])
 def test_ffn_bf16_parity(B, kind, S, T, d, f):
     _ffn_case(B, kind, I.DTYPE_BF16, S, T, d, f, alpha=2.0, lr=0.5, seed=41)
+
+
+@pytest.mark.parametrize("kind,S,T,d,f,keep", [
+    (I.FFN_SWIGLU, 2, 300, 264, 392, 96),      # ragged tiles, a quarter of the neurons active
+    (I.FFN_GELU, 3, 130, 136, 264, 128),
+    (I.FFN_RELU, 1, 257, 72, 520, 8),
+])
+def test_masked_twist_ffn_parity(B, kind, S, T, d, f, keep):
+    """Masked TwIST (Sec. 4.1): the full-width model with an activation mask per worker, against the oracle's
+    masked model; the scale is the one of a subnet with `keep` of f neurons (Sec. 3.4)."""
+    _ffn_case(B, kind, I.DTYPE_BF16, S, T, d, f, o.act_scale(f, keep), 0.05, 33, mask_keep=keep)
+
+
+def test_masked_twist_equals_the_gathered_subnet_on_the_gpu(B):
+    """The same subnet once as a gathered dense slice and once as the masked full-width model: outputs and input
+    gradients agree to rounding (the contraction merely runs over more, zeroed, terms)."""
+    kind, T, d, F, keep = I.FFN_SWIGLU, 260, 136, 256, 64
+    bf = torch.bfloat16
+    rng = np.random.default_rng(3)
+    kept = np.sort(rng.choice(F, keep, replace=False))
+    X = I.normal(44, 1, (1, T, d), 1.0, I.DTYPE_BF16)
+    Wgu = I.normal(44, 2, (1, 2 * F, d), 0.05, I.DTYPE_BF16)
+    Wd = I.normal(44, 3, (1, F, d), 0.05, I.DTYPE_BF16)
+    dY = I.normal(44, 4, (1, T, d), 1e-3, I.DTYPE_BF16)
+    alpha = o.act_scale(F, keep)
+    outs = []
+    for masked in (True, False):
+        f = F if masked else keep
+        rows = np.arange(2 * F) if masked else np.concatenate([kept, kept + F])
+        w_gu, w_down = dev(Wgu[:, rows], bf), dev(Wd[:, np.arange(F) if masked else kept], bf)
+        t = lambda *s: torch.zeros(*s, dtype=bf, device="cuda")
+        pre, hh, y, dpre, dx = t(1, T, 2 * f), t(1, T, f), t(1, T, d), t(1, T, 2 * f), t(1, T, d)
+        extra = {}
+        if masked:
+            m = np.zeros((1, F), dtype=np.uint8)
+            m[0, kept] = 1
+            extra = dict(hidden_mask=dev(m))
+        a = B.ffn_args(kind, I.DTYPE_BF16, 1, T, d, f, alpha, 0.0, x=dev(X, bf), w_gu=w_gu, w_down=w_down, pre=pre, hh=hh,
+                       y=y, dy=dev(dY, bf), dpre=dpre, dx=dx, **extra)
+        B.twist_subnet_ffn_fwd(a)
+        B.twist_subnet_ffn_bwd(a)
+        torch.cuda.synchronize()
+        check_status(B)
+        outs.append((host(y[0]), host(dx[0]), host(hh[0])[:, kept] if masked else host(hh[0])))
+    (ym, dxm, hm), (yg, dxg, hg) = outs
+    assert np.array_equal(hm, hg)                    # the kept activations are the same numbers
+    assert rel_fro(ym, yg) < 4e-3 and rel_fro(dxm, dxg) < 4e-3     # one bf16 rounding apart at most
 
 
 @pytest.mark.parametrize("dtype,S,T,d,n", [(I.DTYPE_FP32, 2, 33, 24, 16), (I.DTYPE_BF16, 2, 200, 328, 200),

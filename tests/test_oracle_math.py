@@ -158,6 +158,35 @@ def test_masked_full_model_equals_gathered_slice(kind):
         assert np.all(full.numpy()[dropped] == 0)
 
 
+@pytest.mark.parametrize("kind", KINDS)
+def test_oracle_hidden_mask_matches_autograd_of_the_masked_model(kind):
+    """y = M * f(x) (Sec. 4.1) through the oracle's own mask option: forward, dX and every weight gradient equal
+    torch autograd on the masked full model; rows of masked-out neurons get exactly zero gradient."""
+    r = _rng(14)
+    T, d, F = 5, 8, 16
+    kept = np.array(sorted(r.choice(F, 6, replace=False)))
+    alpha = o.act_scale(F, len(kept))
+    X, Wu, Wg, Wd, Tgt = (r.standard_normal(s) for s in [(T, d), (F, d), (F, d), (F, d), (T, d)])
+    m = np.zeros(F)
+    m[kept] = 1.0
+    Y, saved = o.ffn_fwd(X, Wu, Wg, Wd, kind, alpha, lowp=False, hidden_mask=m)
+    _, dY = o.mse(Y, Tgt, lowp=False)
+    dX, dWu, dWg, dWd = o.ffn_bwd(dY, X, saved, Wu, Wg, Wd, kind, alpha, lowp=False, hidden_mask=m)
+    tX, tWu, tWg, tWd = (torch.tensor(a, requires_grad=True) for a in (X, Wu, Wg, Wd))
+    tY = _dense_ffn_torch(kind, tX, tWu, tWg, tWd, alpha, torch.from_numpy(m))
+    torch.mean((tY - torch.from_numpy(Tgt)) ** 2).backward()
+    assert np.allclose(Y, tY.detach().numpy(), atol=1e-12)
+    assert np.allclose(dX, tX.grad.numpy(), atol=1e-13)
+    dropped = np.setdiff1d(np.arange(F), kept)
+    for got, full in [(dWu, tWu.grad), (dWd, tWd.grad)] + ([(dWg, tWg.grad)] if kind == 2 else []):
+        assert np.allclose(got, full.numpy(), atol=1e-13)
+        assert np.all(got[dropped] == 0)
+    # and the mask of all ones is the unmasked model
+    Y1, _ = o.ffn_fwd(X, Wu, Wg, Wd, kind, alpha, lowp=False, hidden_mask=np.ones(F))
+    Y0, _ = o.ffn_fwd(X, Wu, Wg, Wd, kind, alpha, lowp=False)
+    assert np.array_equal(Y1, Y0)
+
+
 # ------------------------------------------------------------------ aggregator (Sec. 3.3)
 
 def test_aggregate_hand_example():
