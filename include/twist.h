@@ -100,6 +100,12 @@ int32_t twist_sample_masks(uint64_t seed, uint64_t round, int32_t layer_begin, i
  * query heads is.  Writes kv_idx [n_layers][S][n_kv_heads] (sorted kept groups, then -1),
  * kv_count [n_layers][S], kv_cols [n_layers][S] = kv_count * d_head (valid K or V columns of the
  * subnet's projection), kv_cover [n_layers][n_kv_heads], kv_pos [n_layers][S][n_kv_heads]; all device. */
+/* Activation masks of Masked / Hybrid TwIST (Sec. 4.1) from the aggregator's cover masks: for the subnets
+ * subnet_begin .. subnet_begin + n_subnets - 1,  mask[s][b*block_rows + i] = 1 if subnet s holds block b, else 0.
+ *   cover [n_full] device uint32 (one layer);  mask [n_subnets][n_full*block_rows] device uint8: out. */
+int32_t twist_hidden_mask(const uint32_t* cover /*device*/, int32_t n_full, int32_t block_rows, int32_t subnet_begin,
+                          int32_t n_subnets, uint8_t* mask /*device*/, void* stream);
+
 int32_t twist_kv_groups(const int32_t* head_idx, int32_t n_layers, int32_t n_subnets, int32_t head_keep,
                         int32_t n_heads, int32_t n_kv_heads, int32_t d_head, int32_t* kv_idx, int32_t* kv_count,
                         int32_t* kv_cols, uint32_t* kv_cover, int32_t* kv_pos, void* stream);
@@ -158,6 +164,12 @@ typedef struct {
   int64_t dst_row_offset;     /* first row of the partitioned range inside dst */
   int64_t sub_subnet_stride;  /* elements between subnets in sub */
   int64_t sub_row_offset;     /* first row of this segment inside a subnet's slice */
+  /* Hybrid TwIST (Sec. 4.1): the worker `central_subnet` trained its blocks in place on a full-width fp32
+   * matrix under an activation mask instead of on a slice; its row for (block b, row i) is
+   * central[(dst_row_offset + b*block_rows + i)*d + :].  central may be dst_f32 itself (every element is read
+   * before it is written, by the same thread).  NULL: every subnet is read from `sub`. */
+  const float* central;
+  int32_t central_subnet;
 } twist_aggregate_segment;
 
 int32_t twist_aggregate(const twist_aggregate_segment* segs /*host*/, int32_t n_segs, int32_t n_subnets,

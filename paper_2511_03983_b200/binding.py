@@ -31,6 +31,7 @@ EXPORTS = [
     "twist_kv_groups", "twist_gather_subnets", "twist_aggregate", "twist_subnet_ffn_fwd", "twist_subnet_ffn_bwd",
     "twist_subnet_attn_proj_fwd", "twist_subnet_attn_proj_bwd", "twist_mse_workspace_bytes", "twist_mse_fwd_bwd",
     "twist_mse_fwd_bwd_noalloc", "twist_fused_loss_workspace_bytes", "twist_attn_core_fwd", "twist_attn_core_bwd",
+    "twist_hidden_mask",
 ]
 
 
@@ -50,7 +51,8 @@ class GatherSegment(C.Structure):
 class AggregateSegment(C.Structure):
     _fields_ = [("dst", C.c_void_p), ("dst_f32", C.c_void_p), ("sub", C.c_void_p), ("cover", C.c_void_p),
                 ("pos", C.c_void_p), ("n_full", C.c_int32), ("block_rows", C.c_int32), ("dst_row_offset", C.c_int64),
-                ("sub_subnet_stride", C.c_int64), ("sub_row_offset", C.c_int64)]
+                ("sub_subnet_stride", C.c_int64), ("sub_row_offset", C.c_int64), ("central", C.c_void_p),
+                ("central_subnet", C.c_int32)]
 
 
 class Optimizer(C.Structure):
@@ -116,6 +118,7 @@ def lib() -> C.CDLL:
                                          C.c_void_p, C.c_void_p]
         h.twist_kv_groups.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int32,
                                       C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+        h.twist_hidden_mask.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p]
         h.twist_gather_subnets.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_void_p]
         h.twist_aggregate.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_uint32, C.c_void_p]
         for name in ("twist_subnet_ffn_fwd", "twist_subnet_ffn_bwd", "twist_subnet_attn_proj_fwd",
@@ -199,10 +202,15 @@ def twist_gather_subnets(segs: Sequence[GatherSegment], n_subnets, d, dtype):
 
 
 def aggregate_segment(dst, dst_f32, sub, cover, pos, n_full, block_rows, dst_row_offset, sub_subnet_stride,
-                      sub_row_offset) -> AggregateSegment:
+                      sub_row_offset, central=None, central_subnet=0) -> AggregateSegment:
     a = lambda v: v if (v is None or isinstance(v, int)) else _ptr(v)
     return AggregateSegment(a(dst), a(dst_f32), a(sub), a(cover), a(pos), n_full, block_rows, dst_row_offset,
-                            sub_subnet_stride, sub_row_offset)
+                            sub_subnet_stride, sub_row_offset, a(central), central_subnet)
+
+
+def twist_hidden_mask(cover, n_full, block_rows, subnet_begin, n_subnets, mask):
+    _check(lib().twist_hidden_mask(_ptr(cover), n_full, block_rows, subnet_begin, n_subnets, _ptr(mask), _stream()),
+           "twist_hidden_mask")
 
 
 def twist_aggregate(segs: Sequence[AggregateSegment], n_subnets, d, dtype, live_subnets=0xFFFFFFFF):

@@ -226,12 +226,16 @@ __global__ void __launch_bounds__(256) aggregate_rows_kernel(const __grid_consta
     if (m == 0) continue;                              // held by no live subnet: untouched
     const int cnt = __popc(m);
     const float4* mine = nullptr;                      // lane k holds the row pointer of the k-th covering subnet
+    const long long drow = sg.dst_row_offset + rl;
     if (lane < cnt) {
       const int s = __fns(m, 0, lane + 1);
-      const long long srow = sg.sub_row_offset + (long long)sg.pos[(long long)s * sg.n_full + b] * sg.block_rows + i;
-      mine = reinterpret_cast<const float4*>(sg.sub + (long long)s * sg.sub_subnet_stride + srow * p.d);
+      if (sg.central && s == sg.central_subnet) {        // trained in place on the full-width matrix
+        mine = reinterpret_cast<const float4*>(sg.central + drow * p.d);
+      } else {
+        const long long srow = sg.sub_row_offset + (long long)sg.pos[(long long)s * sg.n_full + b] * sg.block_rows + i;
+        mine = reinterpret_cast<const float4*>(sg.sub + (long long)s * sg.sub_subnet_stride + srow * p.d);
+      }
     }
-    const long long drow = sg.dst_row_offset + rl;
     // Quotient by the coverage count: reciprocal product corrected with the exact remainder, which gives
     // the correctly rounded quotient (the same bits as an IEEE division) at a fraction of its cost.
     const float denom = (float)cnt;
@@ -363,7 +367,8 @@ extern "C" int32_t twist_aggregate(const twist_aggregate_segment* segs, int32_t 
     if (s.n_full <= 0 || s.block_rows <= 0 || s.dst_row_offset < 0 || s.sub_row_offset < 0 ||
         s.sub_subnet_stride < 0 || s.sub_subnet_stride % 4 != 0)
       return TWIST_ERR_SHAPE;
-    if (!aligned16(s.dst) || !aligned16(s.sub) || !aligned16(s.dst_f32)) return TWIST_ERR_SHAPE;
+    if (!aligned16(s.dst) || !aligned16(s.sub) || !aligned16(s.dst_f32) || !aligned16(s.central)) return TWIST_ERR_SHAPE;
+    if (s.central && (s.central_subnet < 0 || s.central_subnet >= n_subnets)) return TWIST_ERR_BAD_INDEX;
     if (dtype == TWIST_FP32 && s.dst_f32) return TWIST_ERR_UNSUPPORTED;      // dst already is the fp32 result
     p.seg[g] = s;
     total += (long long)s.n_full * s.block_rows;

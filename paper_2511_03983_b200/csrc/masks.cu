@@ -158,6 +158,15 @@ __global__ void cover_pos_kernel(const int32_t* __restrict__ idx, const int32_t*
   cover[(size_t)l * n_full + b] = mask;
 }
 
+// mask[s][r] = bit (subnet_begin + s) of cover[r / block_rows]
+__global__ void hidden_mask_kernel(const uint32_t* __restrict__ cover, long long rows, int block_rows, int subnet_begin,
+                                   int n_subnets, uint8_t* __restrict__ mask) {
+  const long long r = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (r >= rows) return;
+  const uint32_t c = cover[r / block_rows];
+  for (int s = 0; s < n_subnets; ++s) mask[(long long)s * rows + r] = (uint8_t)((c >> (subnet_begin + s)) & 1u);
+}
+
 // One thread per (layer, subnet): kept KV groups of the sorted kept heads.
 __global__ void kv_groups_kernel(const int32_t* __restrict__ head_idx, int total, int head_keep, int per_group,
                                  int n_kv, int d_head, int32_t* __restrict__ kv_idx, int32_t* __restrict__ kv_count,
@@ -215,6 +224,19 @@ extern "C" int32_t twist_sample_masks(uint64_t seed, uint64_t round, int32_t lay
   TWIST_LAUNCH_CHECK();
   cover_pos_kernel<<<dim3((n_full + 255) / 256, n_layers), 256, 0, st>>>(idx, nullptr, n_full, n_subnets, n_sub,
                                                                          cover, pos);
+  TWIST_LAUNCH_CHECK();
+  return TWIST_OK;
+}
+
+extern "C" int32_t twist_hidden_mask(const uint32_t* cover, int32_t n_full, int32_t block_rows, int32_t subnet_begin,
+                                     int32_t n_subnets, uint8_t* mask, void* stream) {
+  using namespace twist;
+  if (!cover || !mask) return TWIST_ERR_NULL;
+  if (n_full <= 0 || block_rows <= 0 || subnet_begin < 0 || n_subnets <= 0) return TWIST_ERR_SHAPE;
+  if (subnet_begin + n_subnets > TWIST_MAX_SUBNETS) return TWIST_ERR_UNSUPPORTED;
+  const long long rows = (long long)n_full * block_rows;
+  hidden_mask_kernel<<<(unsigned)((rows + 255) / 256), 256, 0, static_cast<cudaStream_t>(stream)>>>(
+      cover, rows, block_rows, subnet_begin, n_subnets, mask);
   TWIST_LAUNCH_CHECK();
   return TWIST_OK;
 }

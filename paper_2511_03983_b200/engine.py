@@ -304,6 +304,86 @@ class RoundEngine:
             self.run_layer(l)
 
 
+class HybridRoundEngine(RoundEngine):
+    """Hybrid TwIST (Sec. 4.1) for the FFN blocks: worker 0 is the central model.  It keeps no slice: it trains its
+    subnet in place on the full-width matrices under an activation mask (twist_ffn_args.hidden_mask), while workers
+    1 .. S-1 train gathered dense slices as in RoundEngine; the aggregator reads worker 0's rows from the full fp32
+    matrices (twist_aggregate_segment.central).  In exact arithmetic the round equals RoundEngine's.
+    Gate and up rows of a layer are laid out back to back so that the full model is a valid w_gu operand."""
+
+    def __init__(self, w: Workload, device: str = "cuda", **kw):
+        assert w.dtype == DTYPE_BF16 and w.n_heads == 0 and w.n_subnets >= 2, "bf16 FFN-only workloads"
+        assert w.optimizer != "adam", "the central model's moments would need full-width arrays"
+        super().__init__(w, device=device, keep_f32_full=True, **kw)
+        L, F, d, T = w.n_layers, w.d_ff, w.d_model, w.tokens
+        g, dev = self.g, self.dev
+        bf = torch.bfloat16
+        # [L][g F][d]: gate rows then up rows of a layer are contiguous; the dictionaries keep their per-matrix views
+        self.full_gu = torch.empty(L, g * F, d, dtype=bf, device=dev)
+        self.full_gu_f32 = torch.empty(L, g * F, d, dtype=torch.float32, device=dev)
+        for store, buf in ((self.full, self.full_gu), (self.full_f32, self.full_gu_f32)):
+            if g == 2:
+                store["gate"] = buf[:, :F]
+            store["up"] = buf[:, (g - 1) * F:]
+        act = lambda width: torch.empty(1, T, width, dtype=bf, device=dev)
+        self.c_pre, self.c_dpre, self.c_hh = act(g * F), act(g * F), act(F)
+        self.c_mask = torch.zeros(1, F, dtype=torch.uint8, device=dev)
+
+    def gather_layer(self, l: int, which=("ffn",)):
+        """Slices of workers 1 .. S-1 only; the central worker's activation mask for this layer."""
+        w, d = self.w, self.w.d_model
+        f, gf = w.f_sub, self.g * w.f_sub
+        idx = self.idx_ffn[l, 1:]
+        segs = []
+        for m, off, dst, dst_m, stride in ([("gate", 0, self.w_gu, self.w_gu_m, gf)] if self.g == 2 else []) + [
+                ("up", f if self.g == 2 else 0, self.w_gu, self.w_gu_m, gf), ("down", 0, self.w_down, self.w_down_m, f)]:
+            segs.append(B.gather_segment(self.full[m][l], dst[1:], dst_m[1:], idx, None, w.ffn_keep, w.ffn_keep,
+                                         w.ffn_block, 0, stride * d, off))
+        with self._timed("gather"):
+            B.twist_gather_subnets(segs, w.n_subnets - 1, d, w.dtype)
+            B.twist_hidden_mask(self.cover_ffn[l], w.n_ffn_blocks, w.ffn_block, 0, 1, self.c_mask)
+        self.launches += 2
+
+    def ffn_step(self, l: int, k: int, lr: Optional[float] = None):
+        w = self.w
+        lr = w.lr if lr is None else lr
+        S, T, d, F = w.n_subnets, w.tokens, w.d_model, w.d_ff
+        # central worker: the full-width layer under its mask, updated in place
+        c = B.ffn_args(w.ffn_kind, w.dtype, 1, T, d, F, self.alpha_f, lr, x=self.X[k][:1], w_gu=self.full_gu[l],
+                       w_down=self.full["down"][l], w_gu_master=self.full_gu_f32[l],
+                       w_down_master=self.full_f32["down"][l], pre=self.c_pre, hh=self.c_hh,
+                       y=self.y[:1] if self.store_outputs else None, dy=self.dy[:1], dpre=self.c_dpre,
+                       dx=self.dx[:1] if self.dx is not None else None, hidden_mask=self.c_mask,
+                       tgt=self.Td[k][:1], loss=self.loss[l, 0, k][:1], loss_ws=self.ws)
+        # workers 1 .. S-1: gathered slices
+        o = B.ffn_args(w.ffn_kind, w.dtype, S - 1, T, d, w.f_sub, self.alpha_f, lr, x=self.X[k][1:], w_gu=self.w_gu[1:],
+                       w_down=self.w_down[1:], w_gu_master=self.w_gu_m[1:], w_down_master=self.w_down_m[1:],
+                       pre=self.pre[1:], hh=self.hh[1:], y=self.y[1:] if self.store_outputs else None, dy=self.dy[1:],
+                       dpre=self.dpre[1:], dx=self.dx[1:] if self.dx is not None else None, tgt=self.Td[k][1:],
+                       loss=self.loss[l, 0, k][1:], loss_ws=self.ws)
+        with self._timed("ffn_fwd"):
+            B.twist_subnet_ffn_fwd(c)
+            B.twist_subnet_ffn_fwd(o)
+        with self._timed("ffn_bwd"):
+            B.twist_subnet_ffn_bwd(c)
+            B.twist_subnet_ffn_bwd(o)
+        self.launches += 2 * (2 + 1 + 3 + (1 if self.compute_dx else 0))
+
+    def aggregate_layer(self, l: int, live: int = 0xFFFFFFFF, which=("ffn",)):
+        w, d = self.w, self.w.d_model
+        f, gf = w.f_sub, self.g * w.f_sub
+        nb = w.n_ffn_blocks
+        segs = []
+        for m, off, sub, stride in ([("gate", 0, self.w_gu_m, gf)] if self.g == 2 else []) + [
+                ("up", f if self.g == 2 else 0, self.w_gu_m, gf), ("down", 0, self.w_down_m, f)]:
+            segs.append(B.aggregate_segment(self.full[m][l], self.full_f32[m][l], sub, self.cover_ffn[l], self.pos_ffn[l],
+                                            nb, w.ffn_block, 0, stride * d, off, central=self.full_f32[m][l],
+                                            central_subnet=0))
+        with self._timed("aggregate"):
+            B.twist_aggregate(segs, w.n_subnets, d, w.dtype, live)
+        self.launches += 1
+
+
 class StackEngine(RoundEngine):
     """One TwIST round in the chained (STACK) composition: every local step runs all layers,
     x <- x + alpha_a * O(core(QKV(x))),  x <- x + alpha_f * FFN(x),  with one loss on the final x.

@@ -24,6 +24,11 @@ def test_library_exports_every_declared_symbol():
         assert hasattr(h, n), n
     assert sorted(B.EXPORTS) == names
     assert B.twist_abi_version() == 1
+    # every entry point that takes arguments declares their C types: a device address passed without them
+    # would be truncated to 32 bits
+    for n in names:
+        if n not in ("twist_abi_version", "twist_last_cuda_error"):
+            assert getattr(h, n).argtypes is not None, n
 
 
 def test_status_strings():

@@ -474,11 +474,14 @@ def _load_batches(eng, w, rnd):
     return store
 
 
-def _run_round_and_compare(B, w, rnd=0, tol_dw=5e-2, **engine_kw):
+def _run_round_and_compare(B, w, rnd=0, tol_dw=5e-2, engine_cls=None, **engine_kw):
     from paper_2511_03983_b200.engine import RoundEngine
     lowp = w.dtype == I.DTYPE_BF16
-    eng = RoundEngine(w, keep_f32_full=True, **engine_kw)
+    eng = RoundEngine(w, keep_f32_full=True, **engine_kw) if engine_cls is None else engine_cls(w, **engine_kw)
     full_np = _load_full(eng, w)
+    if eng.full_f32 is not None:       # the fp32 full model starts as the exact widening of the bf16 one
+        for m in eng.full:
+            eng.full_f32[m].copy_(eng.full[m].float())
     store = _load_batches(eng, w, rnd)
     before = {m: v.clone() for m, v in eng.full.items()}
     eng.run_round(rnd)
@@ -527,6 +530,26 @@ def test_config1_fp32_round_matches_oracle_everywhere(B):
 def test_scaled_twin_rounds_match_oracle(B, cfg, dims):
     w = I.scaled_twin(I.PRESETS[cfg], **dims)
     _run_round_and_compare(B, w)
+
+
+@pytest.mark.parametrize("kind,mode", [(I.FFN_SWIGLU, I.MODE_COVER), (I.FFN_GELU, I.MODE_IID)])
+def test_hybrid_twist_round_matches_the_oracle_round(B, kind, mode):
+    """Hybrid TwIST (Sec. 4.1): worker 0 trains in place on the full-width model under its activation mask, the
+    others on gathered slices; the round is the same function as the all-gathered round the oracle computes."""
+    from paper_2511_03983_b200.engine import HybridRoundEngine
+    w = replace(I.scaled_twin(I.PRESETS[5], d_model=136, d_ff=544, d_head=0, tokens=200, n_layers=2, local_steps=2),
+                n_subnets=4, ffn_kind=kind, sample_mode=mode, lr=0.05)
+    eng, before = _run_round_and_compare(B, w, engine_cls=HybridRoundEngine)
+    assert any(not torch.equal(eng.full[m], before[m]) for m in before)        # the round did train
+
+
+def test_hidden_mask_from_cover_bits(B):
+    cover = np.array([0b101, 0b010, 0, 0b111, 0b100], dtype=np.uint32)
+    mask = torch.zeros(2, 15, dtype=torch.uint8, device="cuda")
+    B.twist_hidden_mask(dev(cover.view(np.int32)), 5, 3, 1, 2, mask)
+    torch.cuda.synchronize()
+    want = np.array([[(c >> s) & 1 for c in cover for _ in range(3)] for s in (1, 2)], dtype=np.uint8)
+    assert np.array_equal(mask.cpu().numpy(), want)
 
 
 @pytest.mark.parametrize("engine_kw", [dict(fuse_loss=False), dict(store_outputs=False)])
