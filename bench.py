@@ -214,9 +214,12 @@ def workload_config(w, args):
                 "tokens_per_round": w.tokens_per_round, "mode": "stack, all layers resident",
                 "l2_policy": "working set exceeds L2 across the layers of a round",
                 "parallelism": "replicas only" if args.gpus > 1 else "single GPU"}
-    return {"workload": f"configs[{args.config - 1}] {w.name}: BLOCKWISE round, L={w.n_layers} d={w.d_model} "
+    hybrid = getattr(args, "mode", "blockwise") == "hybrid"
+    return {"workload": f"configs[{args.config - 1}] {w.name}: {'HYBRID ' if hybrid else ''}BLOCKWISE round, L={w.n_layers} d={w.d_model} "
                         f"F={w.d_ff} f'={w.f_sub} H'={w.head_keep}/{w.n_heads} S={w.n_subnets} T={w.tokens} K={w.local_steps}",
-            "tokens_per_round": w.tokens_per_round, "mode": "blockwise, layers streamed",
+            "tokens_per_round": w.tokens_per_round,
+            "mode": ("hybrid: worker 0 masked on the full-width model in place, the others on gathered slices; flops "
+                     "counted are those of the gathered subnets" if hybrid else "blockwise, layers streamed"),
             "l2_policy": "inputs larger than L2 (every tensor a kernel reads is >= 4x the 126 MB L2)"
                          if w.d_model >= 2048 else "working set exceeds L2 across the layers of a round",
             "parallelism": "replicas only" if args.gpus > 1 else "single GPU"}
@@ -232,7 +235,7 @@ def run_ours(args, w):
 
     from paper_2511_03983_b200 import binding as B
     from paper_2511_03983_b200 import inputs as I
-    from paper_2511_03983_b200.engine import RoundEngine, StackEngine
+    from paper_2511_03983_b200.engine import HybridRoundEngine, RoundEngine, StackEngine
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -250,6 +253,10 @@ def run_ours(args, w):
         if not (w.n_heads and bf16 and w.tokens % w.n_seqs == 0):
             raise SystemExit("--mode stack needs a bf16 workload with attention heads")
         eng = StackEngine(w, w.n_seqs, w.tokens // w.n_seqs, keep_f32_full=True)
+    elif args.mode == "hybrid":
+        if w.n_heads or not bf16:
+            raise SystemExit("--mode hybrid needs a bf16 FFN-only workload (--config 5)")
+        eng = HybridRoundEngine(w, compute_dx=True, fuse_loss=True, store_outputs=False)
     else:
         eng = RoundEngine(w, keep_f32_full=True, compute_dx=True, fuse_loss=True, store_outputs=False)
     gen = torch.Generator(device="cuda")
@@ -257,6 +264,8 @@ def run_ours(args, w):
     for m, v in eng.full.items():                         # weights ~ N(0, 0.02^2), one matrix at a time
         for l in range(w.n_layers):
             v[l].copy_((torch.randn(v[l].shape, generator=gen, device="cuda", dtype=torch.float32) * 0.02).to(td))
+            if args.mode == "hybrid":                     # the central worker trains on the fp32 full model in place
+                eng.full_f32[m][l].copy_(v[l])
     gen.manual_seed(replica_seed(w.seed_x, rank))
     S, T, K = w.n_subnets, w.tokens, w.local_steps
     widths = [("X", w.d_model), ("Td", w.d_model)] + ([("Tq", eng.nq), ("A", eng.a_sub)]
@@ -366,6 +375,8 @@ def run_ours(args, w):
 
     peaks = measured_peaks()
     work = round_work(w)
+    if args.mode == "hybrid":                             # worker 0 has no slice: S - 1 subnets are gathered
+        work["gather_bytes"] *= (w.n_subnets - 1) / w.n_subnets
     gemm_names = [n for n in ("ffn_fwd", "ffn_bwd", "qkv_fwd", "qkv_bwd", "o_fwd", "o_bwd") if n in phases]
     gemm_ms = sum(phases[n][0] for n in gemm_names)
     gemm_launches_per_round = w.n_layers * K * ((2 + 4) + ((1 + 2 + 1 + 2) if eng.has_attn else 0))
@@ -490,8 +501,9 @@ def main():
     ap.add_argument("--layers", type=int, default=0, help="override the layer count (profiling on a small case)")
     ap.add_argument("--tokens", type=int, default=0, help="override tokens per subnet-step (profiling on a small case)")
     ap.add_argument("--local-steps", type=int, default=0)
-    ap.add_argument("--mode", default="blockwise", choices=["blockwise", "stack"],
-                    help="stack: chained layers with the attention core (workloads 2 and 3)")
+    ap.add_argument("--mode", default="blockwise", choices=["blockwise", "stack", "hybrid"],
+                    help="stack: chained layers with the attention core (workloads 2 and 3); hybrid: worker 0 trains "
+                         "the full-width model under a mask (FFN-only workload 5)")
     ap.add_argument("--sweep", action="store_true", help="workload 5: all 12 (S, keep) cells, gather / aggregate GB/s")
     args = ap.parse_args()
     from dataclasses import replace
