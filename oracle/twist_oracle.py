@@ -11,7 +11,7 @@ Every function cites the passage of the paper it follows.  TwIST is an
 iteration, not a shortcut to a closed form, so each function takes the
 algorithm's steps in the paper's order and notation.
 
-Storage convention (a choice of this build, the paper fixes only mathematical
+Storage convention (a choice of this implementation, the paper fixes only mathematical
 shapes in its Problem formulation): every partitioned matrix is stored with one
 row per neuron / head-dimension and d_model contiguous, so a block is a run of
 whole rows ("a block is a chunk of parameters in memory", Sec. 3.1):
@@ -45,7 +45,7 @@ _M2 = _U64(0x94D049BB133111EB)
 # ----------------------------------------------------------------------------------------
 # Counter-based integer hash used for every random draw of the sampler.
 # The paper leaves the generator open (Algorithm 1 calls it "unique_choice" and
-# Sec. 3.1 says "uniformly at random"); this build fixes a 64-bit avalanche
+# Sec. 3.1 says "uniformly at random"); this implementation fixes a 64-bit avalanche
 # mixer (the published splitmix64 finaliser) applied to the counter tuple.
 # ----------------------------------------------------------------------------------------
 

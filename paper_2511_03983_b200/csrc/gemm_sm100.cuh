@@ -197,13 +197,16 @@ __device__ inline float sigmoid_fast(float x) { return __fdividef(1.f, 1.f + __e
 // the epilogue.)  The eight elements advance stage by stage: an epilogue warp has its scheduler to itself, so the
 // only latency hiding there is comes from independent instructions of the same warp.
 __device__ inline void gelu_parts8(const float (&x)[8], float (&cdf)[8], float (&pdf_x)[8]) {
-  float z[8], t[8], e[8], poly[8];
+  // v = |x| sqrt(log2(e) / 2): exp(-x^2 / 2) = 2^(-v^2), and the rational argument p |x| / sqrt(2) = kP v
+  constexpr float kV = 0.84932180028801904f;           // sqrt(log2(e) / 2)
+  constexpr float kP = 0.3275911f / 1.2011224087864498f;   // p / sqrt(log2(e))
+  float v[8], t[8], e[8], poly[8];
 #pragma unroll
-  for (int i = 0; i < 8; ++i) z[i] = fabsf(x[i]) * 0.70710678118654752f;          // |x| / sqrt(2)
+  for (int i = 0; i < 8; ++i) v[i] = fabsf(x[i]) * kV;
 #pragma unroll
-  for (int i = 0; i < 8; ++i) t[i] = __fdividef(1.f, fmaf(0.3275911f, z[i], 1.f));
+  for (int i = 0; i < 8; ++i) asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(t[i]) : "f"(fmaf(kP, v[i], 1.f)));
 #pragma unroll
-  for (int i = 0; i < 8; ++i) e[i] = __expf(-z[i] * z[i]);                         // exp(-x^2 / 2)
+  for (int i = 0; i < 8; ++i) asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e[i]) : "f"(-v[i] * v[i]));   // exp(-x^2 / 2)
 #pragma unroll
   for (int i = 0; i < 8; ++i) poly[i] = fmaf(t[i], 1.061405429f, -1.453152027f);
 #pragma unroll
@@ -214,8 +217,8 @@ __device__ inline void gelu_parts8(const float (&x)[8], float (&cdf)[8], float (
   for (int i = 0; i < 8; ++i) poly[i] = fmaf(t[i], poly[i], 0.254829592f);
 #pragma unroll
   for (int i = 0; i < 8; ++i) {
-    const float erf_abs = fmaf(-poly[i] * t[i], e[i], 1.f);                        // erf(|x| / sqrt(2))
-    cdf[i] = 0.5f * (1.f + copysignf(erf_abs, x[i]));
+    const float half_erf = fmaf(-0.5f * poly[i] * t[i], e[i], 0.5f);               // erf(|x| / sqrt(2)) / 2
+    cdf[i] = 0.5f + copysignf(half_erf, x[i]);
     pdf_x[i] = x[i] * 0.3989422804014327f * e[i];                                  // x phi(x)
   }
 }
