@@ -45,10 +45,13 @@ class RoundEngine:
         self.has_attn = w.n_heads > 0
         bf16 = w.dtype == DTYPE_BF16
         # full model (the central model of the paper's server)
-        self.full: Dict[str, torch.Tensor] = {"up": torch.empty(L, F, d, dtype=td, device=dev),
+        # gate rows then up rows of a layer lie back to back ([L][g F][d]), so that a full-width layer is itself a
+        # valid w_gu operand (Masked / Hybrid TwIST, evaluation of the full model); the dictionary holds views
+        self.full_gu = torch.empty(L, self.g * F, d, dtype=td, device=dev)
+        self.full: Dict[str, torch.Tensor] = {"up": self.full_gu[:, (self.g - 1) * F:],
                                               "down": torch.empty(L, F, d, dtype=td, device=dev)}
         if self.g == 2:
-            self.full["gate"] = torch.empty(L, F, d, dtype=td, device=dev)
+            self.full["gate"] = self.full_gu[:, :F]
         if self.has_attn:
             H, Hkv, dh = w.n_heads, w.n_kv_heads, w.d_head
             self.kv_max = min(Hkv, w.head_keep)
@@ -56,8 +59,12 @@ class RoundEngine:
             self.nq = self.a_sub + 2 * self.kv_max * dh
             self.full["qkv"] = torch.empty(L, (H + 2 * Hkv) * dh, d, dtype=td, device=dev)
             self.full["o"] = torch.empty(L, H * dh, d, dtype=td, device=dev)
-        self.full_f32 = ({m: torch.empty(v.shape, dtype=torch.float32, device=dev) for m, v in self.full.items()}
-                         if (keep_f32_full and bf16) else None)
+        self.full_f32, self.full_gu_f32 = None, None
+        if keep_f32_full and bf16:
+            self.full_gu_f32 = torch.empty(L, self.g * F, d, dtype=torch.float32, device=dev)
+            self.full_f32 = {m: (self.full_gu_f32[:, (self.g - 1) * F:] if m == "up" else
+                                 self.full_gu_f32[:, :F] if m == "gate" else
+                                 torch.empty(v.shape, dtype=torch.float32, device=dev)) for m, v in self.full.items()}
         # blueprints and aggregator index data, all layers
         nb = w.n_ffn_blocks
         i32 = dict(dtype=torch.int32, device=dev)
@@ -288,6 +295,60 @@ class RoundEngine:
             B.twist_subnet_attn_proj_bwd(a)
         self.launches += 1 + 1 + (1 if self.compute_dx else 0) + (0 if w.dtype == DTYPE_BF16 else 1)
 
+    # ------------------------------------------------------------------ deployment / evaluation (Sec. 4.2)
+    def export_subnet(self, s: int) -> Dict[str, torch.Tensor]:
+        """The dense smaller model of subnet s for the layer gathered last (Sec. 4.2, Deployment: the pruned model
+        mirrors the subnet generation of training): copies of its slices, w_gu = gate rows then up rows."""
+        out = {"w_gu": self.w_gu[s].clone(), "w_down": self.w_down[s].clone()}
+        if self.has_attn:
+            out.update(w_qkv=self.w_qkv[s].clone(), w_o=self.w_o[s].clone())
+        return out
+
+    def evaluate_subnets(self, l: int, k: int) -> torch.Tensor:
+        """Evaluation mode for subnets (Sec. 4.2): forward only, on the slices gathered for layer l, with the
+        subnet's own scale (an engine built with other keep counts than the training run evaluates a mismatched
+        subnet ratio).  Returns the losses [blocks][S] (device); the caller averages over the workers."""
+        w = self.w
+        assert self.fuse_loss, "evaluation uses the loss fused into the forward kernels"
+        a = B.ffn_args(w.ffn_kind, w.dtype, w.n_subnets, w.tokens, w.d_model, w.f_sub, self.alpha_f, 0.0, x=self.X[k],
+                       w_gu=self.w_gu, w_down=self.w_down, pre=self.pre, hh=self.hh,
+                       y=self.y if self.store_outputs else None, dy=self.dy, tgt=self.Td[k], loss=self.loss[l, 0, k],
+                       loss_ws=self.ws)
+        B.twist_subnet_ffn_fwd(a)
+        self.launches += 2
+        if self.has_attn:
+            ragged = w.n_kv_heads != w.n_heads
+            mask = dict(valid_cols=self.kv_cols[l], seg_begin=self.a_sub, seg_width=self.kv_max * w.d_head) if ragged else {}
+            q = B.proj_args(B.PROJ_QKV, w.dtype, w.n_subnets, w.tokens, w.d_model, self.nq, 1.0, 0.0, in_=self.X[k],
+                            w=self.w_qkv, out=self.qkv_out if self.store_outputs else None, d_out=self.dqkv,
+                            tgt=self.Tq[k], loss=self.loss[l, 1, k], loss_ws=self.ws, **mask)
+            B.twist_subnet_attn_proj_fwd(q)
+            o = B.proj_args(B.PROJ_O, w.dtype, w.n_subnets, w.tokens, w.d_model, self.a_sub, self.alpha_a, 0.0,
+                            in_=self.A[k], w=self.w_o, out=self.y if self.store_outputs else None, d_out=self.dy,
+                            tgt=self.Td[k], loss=self.loss[l, 2, k], loss_ws=self.ws)
+            B.twist_subnet_attn_proj_fwd(o)
+            self.launches += 2
+        return self.loss[l, : 3 if self.has_attn else 1, k]
+
+    def evaluate_full_ffn(self, l: int, k: int) -> torch.Tensor:
+        """Evaluation mode for the full model (Sec. 4.2: assessed directly, no scaling, no masking), FFN block of
+        layer l on every worker's batch k.  Returns the losses [S] (device)."""
+        w = self.w
+        assert w.dtype == DTYPE_BF16, "the full-width evaluation runs the bf16 kernels"
+        T, d, F = w.tokens, w.d_model, w.d_ff
+        if not hasattr(self, "e_pre"):
+            bf = torch.bfloat16
+            self.e_pre = torch.empty(1, T, self.g * F, dtype=bf, device=self.dev)
+            self.e_hh = torch.empty(1, T, F, dtype=bf, device=self.dev)
+            self.e_loss = torch.zeros(w.n_subnets, dtype=torch.float32, device=self.dev)
+        for s in range(w.n_subnets):
+            a = B.ffn_args(w.ffn_kind, w.dtype, 1, T, d, F, 1.0, 0.0, x=self.X[k][s:s + 1], w_gu=self.full_gu[l],
+                           w_down=self.full["down"][l], pre=self.e_pre, hh=self.e_hh, y=None, dy=self.dy[s:s + 1],
+                           tgt=self.Td[k][s:s + 1], loss=self.e_loss[s:s + 1], loss_ws=self.ws)
+            B.twist_subnet_ffn_fwd(a)
+            self.launches += 2
+        return self.e_loss
+
     def run_layer(self, l: int):
         self.gather_layer(l)
         for k in range(self.w.local_steps):
@@ -309,22 +370,15 @@ class HybridRoundEngine(RoundEngine):
     subnet in place on the full-width matrices under an activation mask (twist_ffn_args.hidden_mask), while workers
     1 .. S-1 train gathered dense slices as in RoundEngine; the aggregator reads worker 0's rows from the full fp32
     matrices (twist_aggregate_segment.central).  In exact arithmetic the round equals RoundEngine's.
-    Gate and up rows of a layer are laid out back to back so that the full model is a valid w_gu operand."""
+    (The full model's gate and up rows lie back to back, so a full-width layer is a valid w_gu operand.)"""
 
     def __init__(self, w: Workload, device: str = "cuda", **kw):
         assert w.dtype == DTYPE_BF16 and w.n_heads == 0 and w.n_subnets >= 2, "bf16 FFN-only workloads"
         assert w.optimizer != "adam", "the central model's moments would need full-width arrays"
         super().__init__(w, device=device, keep_f32_full=True, **kw)
-        L, F, d, T = w.n_layers, w.d_ff, w.d_model, w.tokens
+        F, T = w.d_ff, w.tokens
         g, dev = self.g, self.dev
         bf = torch.bfloat16
-        # [L][g F][d]: gate rows then up rows of a layer are contiguous; the dictionaries keep their per-matrix views
-        self.full_gu = torch.empty(L, g * F, d, dtype=bf, device=dev)
-        self.full_gu_f32 = torch.empty(L, g * F, d, dtype=torch.float32, device=dev)
-        for store, buf in ((self.full, self.full_gu), (self.full_f32, self.full_gu_f32)):
-            if g == 2:
-                store["gate"] = buf[:, :F]
-            store["up"] = buf[:, (g - 1) * F:]
         act = lambda width: torch.empty(1, T, width, dtype=bf, device=dev)
         self.c_pre, self.c_dpre, self.c_hh = act(g * F), act(g * F), act(F)
         self.c_mask = torch.zeros(1, F, dtype=torch.uint8, device=dev)

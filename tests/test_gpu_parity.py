@@ -543,6 +543,43 @@ def test_hybrid_twist_round_matches_the_oracle_round(B, kind, mode):
     assert any(not torch.equal(eng.full[m], before[m]) for m in before)        # the round did train
 
 
+@pytest.mark.parametrize("eval_keep_ratio", [0.25, 0.5])
+def test_deployment_extraction_and_evaluation_modes(B, eval_keep_ratio):
+    """Sec. 4.2: a subnet extracted with the sampler's procedure at a subnet ratio that need not be the training one,
+    evaluated forward-only with its own scale; the full model evaluated directly (no scale, no mask)."""
+    from paper_2511_03983_b200.engine import RoundEngine
+    base = I.scaled_twin(I.PRESETS[4], d_model=136, d_ff=544, d_head=8, tokens=200, n_layers=1, local_steps=1)
+    w = replace(base, ffn_keep=int(base.n_ffn_blocks * eval_keep_ratio), sample_mode=I.MODE_IID)
+    eng = RoundEngine(w)
+    full_np = _load_full(eng, w)
+    store = _load_batches(eng, w, 0)
+    eng.sample_masks(0)
+    eng.gather_layer(0)
+    got = eng.evaluate_subnets(0, 0).cpu().numpy()
+    got_full = eng.evaluate_full_ffn(0, 0).cpu().numpy()
+    dense = eng.export_subnet(1)
+    torch.cuda.synchronize()
+    check_status(B)
+    bp = o.layer_blueprints(w, 0, 0)
+    alpha = o.act_scale(w.n_ffn_blocks, w.ffn_keep)
+    F = w.d_ff
+    for s in range(w.n_subnets):
+        sl = {m: v.astype(np.float64) for m, v in o.gather_layer(w, full_np[0], bp, s).items()}
+        X, Tg = store[(I.BATCH_X, 0)][s].astype(np.float64), store[(I.BATCH_TGT_D, 0)][s].astype(np.float64)
+        Y, _ = o.ffn_fwd(X, sl["up"], sl["gate"], sl["down"], w.ffn_kind, alpha, True)
+        want, _ = o.mse(Y, Tg, True)
+        assert abs(got[0, s] - want) <= 2e-2 * want, (s, got[0, s], want)
+        fm = {m: full_np[0][m].astype(np.float64) for m in ("up", "gate", "down")}
+        Yf, _ = o.ffn_fwd(X, fm["up"], fm["gate"], fm["down"], w.ffn_kind, 1.0, True)
+        want_f, _ = o.mse(Yf, Tg, True)
+        assert abs(got_full[s] - want_f) <= 2e-2 * want_f, (s, got_full[s], want_f)
+        if s == 1:      # the exported dense model is the gathered slice, bit for bit
+            f = w.f_sub
+            assert np.array_equal(host(dense["w_gu"][:f]), sl["gate"]) and np.array_equal(host(dense["w_gu"][f:]), sl["up"])
+            assert np.array_equal(host(dense["w_down"]), sl["down"])
+    assert F // w.ffn_block == w.n_ffn_blocks
+
+
 def test_hidden_mask_from_cover_bits(B):
     cover = np.array([0b101, 0b010, 0, 0b111, 0b100], dtype=np.uint32)
     mask = torch.zeros(2, 15, dtype=torch.uint8, device="cuda")
