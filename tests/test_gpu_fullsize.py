@@ -17,7 +17,7 @@ from paper_2511_03983_b200 import inputs as I
 pytestmark = pytest.mark.gpu
 
 TOL = 2e-2
-SUBNETS = {4: (1, 6), 3: (0, 3)}   # subnets whose activations / updates are checked, per workload
+SUBNETS = {4: (1, 6), 3: (0, 3), 2: (0, 2)}   # subnets whose activations / updates are checked, per workload
 N_ROWS, N_WROWS = 40, 12  # sampled token rows, sampled weight rows
 
 
@@ -29,7 +29,7 @@ def f64(t):
     return t.detach().float().cpu().numpy().astype(np.float64)
 
 
-@pytest.fixture(scope="module", params=[4, 3])
+@pytest.fixture(scope="module", params=[4, 3, 2])
 def setup(request):
     from paper_2511_03983_b200 import binding as B
     from paper_2511_03983_b200.engine import RoundEngine
@@ -77,7 +77,8 @@ def test_gathered_slices_bit_exact(setup):
     f = w.f_sub
     for s in setup["subnets"]:
         sl = o.gather_layer(w, full, bp, s)
-        want = {"w_gu": np.concatenate([sl["gate"], sl["up"]]), "w_down": sl["down"], "w_qkv": sl["qkv"], "w_o": sl["o"]}
+        w_gu = np.concatenate([sl["gate"], sl["up"]]) if "gate" in sl else sl["up"]
+        want = {"w_gu": w_gu, "w_down": sl["down"], "w_qkv": sl["qkv"], "w_o": sl["o"]}
         for name, arr in want.items():
             got16 = getattr(eng, name)[s].float().cpu().numpy()
             got32 = getattr(eng, name + "_m")[s].cpu().numpy()
@@ -107,24 +108,28 @@ def test_ffn_forward_backward_sampled(setup):
         X = f64(eng.X[0][s])
         dYs = f64(dY[s])
         # sampled token rows: every activation of the chain
-        Yw, saved = o.ffn_fwd(X[rows], sl["up"], sl["gate"], sl["down"], w.ffn_kind, eng.alpha_f, True)
-        dXw, _, _, _ = o.ffn_bwd(dYs[rows], X[rows], saved, sl["up"], sl["gate"], sl["down"], w.ffn_kind, eng.alpha_f, True)
+        gated = "gate" in sl                      # SwiGLU: gate and up matrices; otherwise one matrix
+        gate = sl["gate"] if gated else None
+        Yw, saved = o.ffn_fwd(X[rows], sl["up"], gate, sl["down"], w.ffn_kind, eng.alpha_f, True)
+        dXw, _, _, _ = o.ffn_bwd(dYs[rows], X[rows], saved, sl["up"], gate, sl["down"], w.ffn_kind, eng.alpha_f, True)
         r = torch.from_numpy(rows).cuda()
-        assert rel_fro(f64(eng.pre[s][r]), np.concatenate([saved["G"], saved["U"]], axis=1)) < TOL
+        pre_w = np.concatenate([saved["G"], saved["U"]], axis=1) if gated else saved["U"]
+        assert rel_fro(f64(eng.pre[s][r]), pre_w) < TOL
         assert rel_fro(f64(eng.hh[s][r]), saved["Hh"]) < TOL
         assert rel_fro(f64(eng.y[s][r]), Yw) < TOL
         assert rel_fro(f64(eng.dx[s][r]), dXw) < TOL
         # sampled neurons: weight gradients with the full-length contraction over all T tokens; the
         # FFN is separable per neuron except for Y and dX, so restricting the slices to J is exact
         J = np.sort(rng.choice(f, N_WROWS, replace=False))
-        _, savedJ = o.ffn_fwd(X, sl["up"][J], sl["gate"][J], sl["down"][J], w.ffn_kind, eng.alpha_f, True)
-        _, dWu, dWg, dWd = o.ffn_bwd(dYs, X, savedJ, sl["up"][J], sl["gate"][J], sl["down"][J], w.ffn_kind,
-                                     eng.alpha_f, True)
+        gateJ = sl["gate"][J] if gated else None
+        _, savedJ = o.ffn_fwd(X, sl["up"][J], gateJ, sl["down"][J], w.ffn_kind, eng.alpha_f, True)
+        _, dWu, dWg, dWd = o.ffn_bwd(dYs, X, savedJ, sl["up"][J], gateJ, sl["down"][J], w.ffn_kind, eng.alpha_f, True)
         Jt = torch.from_numpy(J).cuda()
-        upd_gate = f64(eng.w_gu_m[s][Jt]) - sl["gate"][J]
-        upd_up = f64(eng.w_gu_m[s][Jt + f]) - sl["up"][J]
+        upd_up = f64(eng.w_gu_m[s][Jt + (f if gated else 0)]) - sl["up"][J]
         upd_down = f64(eng.w_down_m[s][Jt]) - sl["down"][J]
-        assert rel_fro(upd_gate, -lr * dWg) < TOL, (s, "gate")
+        if gated:
+            upd_gate = f64(eng.w_gu_m[s][Jt]) - sl["gate"][J]
+            assert rel_fro(upd_gate, -lr * dWg) < TOL, (s, "gate")
         assert rel_fro(upd_up, -lr * dWu) < TOL, (s, "up")
         assert rel_fro(upd_down, -lr * dWd) < TOL, (s, "down")
         assert torch.equal(eng.w_gu[s][Jt], eng.w_gu_m[s][Jt].to(torch.bfloat16))
@@ -175,9 +180,9 @@ def test_aggregate_whole_layer(setup):
     kvw = eng.kv_max * dh
     gu, down, qkv, wo = (t.cpu().numpy().astype(np.float64) for t in (eng.w_gu_m, eng.w_down_m, eng.w_qkv_m, eng.w_o_m))
     kvs = [bp["kv_idx"][s][: bp["kv_count"][s]] for s in range(S)]
-    cases = [
-        ("gate", [gu[s, :f] for s in range(S)], bp["ffn"], 1, 0, slice(0, w.d_ff)),
-        ("up", [gu[s, f:] for s in range(S)], bp["ffn"], 1, 0, slice(0, w.d_ff)),
+    gated = "gate" in full
+    cases = ([("gate", [gu[s, :f] for s in range(S)], bp["ffn"], 1, 0, slice(0, w.d_ff))] if gated else []) + [
+        ("up", [gu[s, (f if gated else 0):] for s in range(S)], bp["ffn"], 1, 0, slice(0, w.d_ff)),
         ("down", [down[s] for s in range(S)], bp["ffn"], 1, 0, slice(0, w.d_ff)),
         ("qkv", [qkv[s, :a_sub] for s in range(S)], bp["head"], dh, 0, slice(0, H * dh)),
         ("qkv", [qkv[s, a_sub:a_sub + kvw] for s in range(S)], kvs, dh, H * dh, slice(H * dh, (H + Hkv) * dh)),
@@ -222,7 +227,7 @@ def test_fused_loss_at_full_size(setup):
     r = torch.from_numpy(rows).cuda()
     for s in setup["subnets"]:
         sl = _sl64(setup, s)
-        Yw, _ = o.ffn_fwd(f64(eng.X[0][s][r]), sl["up"], sl["gate"], sl["down"], w.ffn_kind, eng.alpha_f, True)
+        Yw, _ = o.ffn_fwd(f64(eng.X[0][s][r]), sl["up"], sl.get("gate"), sl["down"], w.ffn_kind, eng.alpha_f, True)
         want_dy = o.round_bf16(2.0 * (Yw - f64(eng.Td[0][s][r])) / (T * d))
         assert rel_fro(f64(dy_b[s][r]), want_dy) < TOL
         # the reduction: mean squared error over ALL T x d elements, recomputed in fp64 from the stored y
