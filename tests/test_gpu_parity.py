@@ -589,6 +589,18 @@ def test_hidden_mask_from_cover_bits(B):
     assert np.array_equal(mask.cpu().numpy(), want)
 
 
+def test_scaled_twin_round_with_common_blocks_matches_oracle(B):
+    """Common blocks (Sec. 3.1: blocks every subnet holds) in both partitioned kinds: their rows are averaged over
+    all S workers; the cover construction of Algorithm 1 runs over the remaining blocks."""
+    w = replace(I.scaled_twin(I.PRESETS[3], d_model=256, d_ff=688, d_head=8, tokens=256, n_layers=2, local_steps=2),
+                common_ffn=(0, 5, 17, 400, 687), common_heads=(1, 30))
+    eng, _ = _run_round_and_compare(B, w)
+    cover = eng.cover_ffn.cpu().numpy().view(np.uint32)
+    full_mask = (1 << w.n_subnets) - 1
+    assert np.all(cover[:, list(w.common_ffn)] == full_mask)
+    assert np.all(eng.cover_head.cpu().numpy().view(np.uint32)[:, list(w.common_heads)] == full_mask)
+
+
 @pytest.mark.parametrize("engine_kw", [dict(fuse_loss=False), dict(store_outputs=False)])
 def test_scaled_twin_round_with_standalone_loss_and_without_stored_outputs(B, engine_kw):
     w = I.scaled_twin(I.PRESETS[3], d_model=256, d_ff=688, d_head=8, tokens=256, n_layers=1, local_steps=2)
