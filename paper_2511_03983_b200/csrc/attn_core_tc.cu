@@ -735,11 +735,12 @@ int attn_bwd_tc(const AttnParams& p, int n_subnets, cudaStream_t st) {
   if (rc != TWIST_OK) return rc;
   rc = sequence_map(&tdo, p.d_out, p.a_sub, p, n_subnets);
   if (rc != TWIST_OK) return rc;
-  static bool configured = false;
-  if (!configured) {
+  static bool configured[64] = {false};
+  const int slot = device_slot();
+  if (!configured[slot]) {
     TWIST_CUDA_TRY(cudaFuncSetAttribute(attn_dq_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kDqSmem));
     TWIST_CUDA_TRY(cudaFuncSetAttribute(attn_dkv_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kDkvSmem));
-    configured = true;
+    configured[slot] = true;
   }
   int* status = device_status_ptr();
   if (!status) return TWIST_ERR_CUDA;
@@ -756,10 +757,11 @@ int attn_fwd_tc(const AttnParams& p, int n_subnets, cudaStream_t st) {
   CUtensorMap tm;
   int rc = sequence_map(&tm, p.qkv, p.nq, p, n_subnets);
   if (rc != TWIST_OK) return rc;
-  static bool configured = false;
-  if (!configured) {
+  static bool configured[64] = {false};
+  const int slot = device_slot();
+  if (!configured[slot]) {
     TWIST_CUDA_TRY(cudaFuncSetAttribute(attn_fwd_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kFwdSmem));
-    configured = true;
+    configured[slot] = true;
   }
   int* status = device_status_ptr();
   if (!status) return TWIST_ERR_CUDA;

@@ -16,6 +16,13 @@ int* device_status_ptr();
 
 void note_cuda_error(cudaError_t e, const char* where);
 int sm_count();
+// Index of the current device for per-device caches (kernel attributes are per device), 0 when it cannot be read
+// or exceeds the cache size.
+inline int device_slot() {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 0;
+  return dev;
+}
 
 #define TWIST_CUDA_TRY(expr)                                   \
   do {                                                         \

@@ -225,15 +225,17 @@ __global__ void __launch_bounds__(256) aggregate_rows_kernel(const __grid_consta
     const uint32_t m = sg.cover[b] & p.live;
     if (m == 0) continue;                              // held by no live subnet: untouched
     const int cnt = __popc(m);
-    const float4* mine = nullptr;                      // lane k holds the row pointer of the k-th covering subnet
+    // lane k holds the row pointer of the k-th covering subnet; bit 0 marks a row of the full-width matrix itself
+    // (it may be the destination, so it is read with an ordinary load, not through the read-only path)
+    unsigned long long mine = 0;
     const long long drow = sg.dst_row_offset + rl;
     if (lane < cnt) {
       const int s = __fns(m, 0, lane + 1);
       if (sg.central && s == sg.central_subnet) {        // trained in place on the full-width matrix
-        mine = reinterpret_cast<const float4*>(sg.central + drow * p.d);
+        mine = reinterpret_cast<unsigned long long>(sg.central + drow * p.d) | 1ull;
       } else {
         const long long srow = sg.sub_row_offset + (long long)sg.pos[(long long)s * sg.n_full + b] * sg.block_rows + i;
-        mine = reinterpret_cast<const float4*>(sg.sub + (long long)s * sg.sub_subnet_stride + srow * p.d);
+        mine = reinterpret_cast<unsigned long long>(sg.sub + (long long)s * sg.sub_subnet_stride + srow * p.d);
       }
     }
     // Quotient by the coverage count: reciprocal product corrected with the exact remainder, which gives
@@ -249,17 +251,25 @@ __global__ void __launch_bounds__(256) aggregate_rows_kernel(const __grid_consta
 #pragma unroll
       for (int u = 0; u < kUnroll; ++u) acc[u] = make_float4(0.f, 0.f, 0.f, 0.f);
       for (int k = 0; k < cnt; ++k) {
-        const float4* ptr = reinterpret_cast<const float4*>(__shfl_sync(0xffffffffu, (unsigned long long)mine, k));
+        const unsigned long long bits = __shfl_sync(0xffffffffu, mine, k);
+        const uint4* ptr = reinterpret_cast<const uint4*>(bits & ~1ull);
+        const bool in_place = (bits & 1ull) != 0;        // warp-uniform
+        uint4 raw[kUnroll];
+        if (!in_place) {                                 // the loads of one source are issued together
+#pragma unroll
+          for (int u = 0; u < kUnroll; ++u)
+            raw[u] = (c0 + 32 * u < c_end) ? ld_nc(ptr + c0 + 32 * u) : make_uint4(0, 0, 0, 0);
+        } else {
+#pragma unroll
+          for (int u = 0; u < kUnroll; ++u)
+            raw[u] = (c0 + 32 * u < c_end) ? *(ptr + c0 + 32 * u) : make_uint4(0, 0, 0, 0);
+        }
 #pragma unroll
         for (int u = 0; u < kUnroll; ++u) {
-          const int c = c0 + 32 * u;
-          if (c < c_end) {
-            uint4 raw = ld_nc(reinterpret_cast<const uint4*>(ptr + c));
-            acc[u].x += __uint_as_float(raw.x);
-            acc[u].y += __uint_as_float(raw.y);
-            acc[u].z += __uint_as_float(raw.z);
-            acc[u].w += __uint_as_float(raw.w);
-          }
+          acc[u].x += __uint_as_float(raw[u].x);
+          acc[u].y += __uint_as_float(raw[u].y);
+          acc[u].z += __uint_as_float(raw[u].z);
+          acc[u].w += __uint_as_float(raw[u].w);
         }
       }
 #pragma unroll
@@ -325,13 +335,14 @@ extern "C" int32_t twist_gather_subnets(const twist_gather_segment* segs, int32_
   const int pieces = (row_bytes + piece_bytes - 1) / piece_bytes;
   const int buf_bytes = piece_bytes * (any_master ? 3 : 1);          // the piece + its fp32 widening
   const int smem = kGatherWarps * kGatherBufs * buf_bytes;
-  static bool configured = false;
-  if (!configured) {
+  static bool configured[64] = {false};
+  const int slot = device_slot();
+  if (!configured[slot]) {
     TWIST_CUDA_TRY(cudaFuncSetAttribute(gather_rows_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         kGatherWarps * kGatherBufs * 3 * kGatherPieceBytes));
     TWIST_CUDA_TRY(cudaFuncSetAttribute(gather_rows_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         kGatherWarps * kGatherBufs * kGatherPieceBytes));
-    configured = true;
+    configured[slot] = true;
   }
   // persistent grid: as many CTAs per SM as the shared memory allows (at most 8), or fewer for small inputs
   int per_sm = (220 * 1024) / (smem + 1024);
