@@ -188,3 +188,37 @@ def test_stack_round_of_a_scaled_twin_matches_the_oracle(B, cfg, dims, n_seqs):
             res = eng.full_f32[m][l].cpu().numpy().astype(np.float64)
             dw, dg = new[l][m] - full64[l][m], res - full64[l][m]
             assert rel_fro(dg, dw) < 5e-2, (l, m, rel_fro(dg, dw))
+
+
+@pytest.mark.parametrize("mode", ["stack", "blockwise"])
+def test_rounds_are_bit_reproducible(B, mode):
+    """No kernel of the path uses atomics or an order that depends on scheduling (one writer per result, fixed
+    summation orders): the same round from the same state gives the same bits - weights, masters and losses.
+    The twin uses d_head = 64, so the STACK round runs the tensor-core attention kernels."""
+    from paper_2511_03983_b200.engine import RoundEngine, StackEngine
+    w = I.scaled_twin(I.PRESETS[3], d_model=256, d_ff=688, d_head=64, tokens=512, n_layers=2, local_steps=2)
+    eng = StackEngine(w, 2, 256, keep_f32_full=True) if mode == "stack" else RoundEngine(w, keep_f32_full=True)
+    mats = {"gate": I.MAT_GATE, "up": I.MAT_UP, "down": I.MAT_DOWN, "qkv": I.MAT_QKV, "o": I.MAT_O}
+    init = {m: torch.stack([dev(I.weight(w, l, mats[m]), torch.bfloat16) for l in range(w.n_layers)]) for m in eng.full}
+    for k in range(w.local_steps):
+        widths = [(I.BATCH_X, w.d_model, eng.X), (I.BATCH_TGT_D, w.d_model, eng.Td)]
+        if mode == "blockwise":
+            widths += [(I.BATCH_TGT_QKV, eng.nq, eng.Tq), (I.BATCH_A, eng.a_sub, eng.A)]
+        for kind, width, dst in widths:
+            dst.append(dev(np.stack([I.batch(w, kind, 0, s, k, width) for s in range(w.n_subnets)]), torch.bfloat16))
+    runs = []
+    for _ in range(2):
+        for m in eng.full:
+            eng.full[m].copy_(init[m])
+            eng.full_f32[m].copy_(init[m].float())
+        eng.run_round(0)
+        torch.cuda.synchronize()
+        assert B.twist_device_status() == 0
+        loss = eng.stack_loss if mode == "stack" else eng.loss
+        runs.append(({m: v.clone() for m, v in eng.full.items()}, {m: v.clone() for m, v in eng.full_f32.items()},
+                     loss.clone()))
+    (a16, a32, la), (b16, b32, lb) = runs
+    assert any(not torch.equal(a16[m], init[m]) for m in a16)          # the round did train
+    for m in a16:
+        assert torch.equal(a16[m], b16[m]) and torch.equal(a32[m], b32[m]), m
+    assert torch.equal(la, lb)
