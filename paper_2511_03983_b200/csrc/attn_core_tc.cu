@@ -4,15 +4,17 @@
 // One CTA per (block of 128 queries, kept head, sequence).  Per block of 128 keys:
 //   S = Q K^T        one 128 x 128 x 64 MMA chain, Q and K tiles brought by TMA (K-major, 128-byte swizzle)
 //   softmax          thread = query row: the row of S is read from tensor memory twice (maximum, then
-//                    exponentials), running maximum / sum kept in registers, P written to shared memory as the
-//                    bf16 A operand of the next MMA
+//                    exponentials), running maximum / sum kept in registers, P written to tensor memory (bf16
+//                    pairs, lane = query row) as the A operand of the next MMA: it never passes through shared
+//                    memory, whose bandwidth the operand reads of the MMAs already load
 //   O += P V         128 x 64 x 128 MMA chain accumulating in tensor memory, V as the MN-major B operand (rows =
 //                    keys as they lie in memory)
 // P and O are expressed relative to a reference maximum that follows the running maximum lazily: only when a
 // row's maximum has grown by more than kRescaleLog2 since the reference was set does its warp rescale O in
 // tensor memory (and the running sum); otherwise P = 2^(s - ref) <= 2^kRescaleLog2 simply accumulates.  O / l is
-// the same quotient for any reference.  The threads therefore never wait for an output block: per key block
-// they read S, write P and go on.  The next block's S is issued ahead of O += P V.
+// the same quotient for any reference.  The threads therefore never read an output block: per key block they
+// read S, write P and go on.  S of the next block is issued before O += P V of the current one (the threads need
+// it first); between its two passes a thread only checks that the previous O += P V is done with P and O.
 // Warps 0-3: softmax / output; warp 4, one lane: TMA and MMA issue.
 // Backward (same tile sizes; probabilities recomputed from the stored log-sum-exp, dS = P (dP - delta)):
 //   dQ kernel     one CTA per query block: per key block S = Q K^T and dP = dO V^T into tensor memory, the threads
@@ -33,8 +35,8 @@ constexpr int kBq = 128, kBk = 128;     // queries per CTA, keys per block
 constexpr int kTileBytes = 128 * kDh * 2;            // a 128-row tile of Q, K or V: 16 KB
 constexpr int kPBytes = kBq * kBk * 2;               // P: 32 KB (two 64-key halves of 16 KB)
 constexpr int kFwdThreads = 160;
-constexpr int kFwdSmem = kTileBytes * 4 + kPBytes + 1024 + 128;   // Q, K[2], V, P, alignment, barriers: two CTAs per SM
-constexpr int kFwdTmemCols = 256;       // S: columns 0..127, O: columns 128..191
+constexpr int kFwdSmem = kTileBytes * 5 + 1024 + 256;   // Q, K[2], V[2], alignment, barriers: two CTAs per SM
+constexpr int kFwdTmemCols = 256;       // S: columns 0..127, O: columns 128..191, P (bf16 pairs): columns 192..255
 constexpr float kRescaleLog2 = 8.f;     // growth of a row maximum (log2 domain) tolerated before O is rescaled
 
 __device__ inline void mma1(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
@@ -43,6 +45,14 @@ __device__ inline void mma1(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, u
       "setp.ne.b32 p, %4, 0;\n\t"
       "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
       ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// A operand in tensor memory (lane = row of A, two 16-bit elements of the contraction per 32-bit column)
+__device__ inline void mma1_ta(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
 }
 __device__ inline void commit1(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
@@ -66,13 +76,13 @@ __device__ inline float ex2_fast(float x) {
 
 // Softmax of one 128-key block for this thread's query row: reads the row of S from tensor memory twice (maximum,
 // then exponentials), keeps the reference maximum m (log2 domain) and the sum l relative to it, and writes
-// P = 2^(s * scale - m) (bf16) into the A-operand tile.  MASKED: only columns <= k_lim are visible (the diagonal
+// P = 2^(s * scale - m) (bf16 pairs) into the A operand in tensor memory.  MASKED: only columns <= k_lim are visible (the diagonal
 // block); the other blocks carry no per-element predicate.  The tensor-memory load of the next 32-column chunk is
 // in flight while the current one is processed.  `rescale(corr)` is called (by the whole warp) between the two
 // passes when some row of the warp moves its reference; it multiplies the row's O by corr.
-template <bool MASKED, typename Rescale>
-__device__ inline void softmax_block(uint32_t t_s, uint32_t p_row, uint32_t sw, int k_lim, float scale_log2, float& m,
-                                     float& l, Rescale&& rescale) {
+template <bool MASKED, typename BeforeP, typename Rescale>
+__device__ inline bool softmax_block(uint32_t t_s, uint32_t t_p, int k_lim, float scale_log2, float& m, float& l,
+                                     BeforeP&& before_p, Rescale&& rescale) {
   uint32_t va[32], vb[32];
   float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};   // four independent chains
   auto fold_max = [&](const uint32_t (&v)[32], int c) {
@@ -94,6 +104,7 @@ __device__ inline void softmax_block(uint32_t t_s, uint32_t p_row, uint32_t sw, 
   fold_max(vb, 3);
   const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
   const float m_blk = mx * scale_log2;                 // scale > 0: the maximum commutes with the scaling
+  if (!before_p()) return false;                       // warp-uniform
   if (__any_sync(0xffffffffu, m_blk > m + kRescaleLog2)) {
     const float m_new = fmaxf(m, m_blk);
     const float corr = ex2_fast(m - m_new);            // 0 for a first block (m = -inf), 1 where nothing moved
@@ -116,12 +127,7 @@ __device__ inline void softmax_block(uint32_t t_s, uint32_t p_row, uint32_t sw, 
       sum4[i & 3] += p0 + p1;
       w[i] = pack2(p0, p1);
     }
-    const uint32_t half = p_row + (uint32_t)(c >> 1) * (kPBytes / 2);
-#pragma unroll
-    for (int q4 = 0; q4 < 4; ++q4) {
-      const uint32_t piece = (uint32_t)((c & 1) * 4 + q4);
-      sts128(half + ((piece ^ sw) << 4), make_uint4(w[4 * q4], w[4 * q4 + 1], w[4 * q4 + 2], w[4 * q4 + 3]));
-    }
+    tc_st16(t_p + 16 * c, w);                          // 32 keys = 16 columns of packed bf16 pairs
   };
   tc_wait_ld();
   tc_ld32(t_s + 32, vb);
@@ -134,7 +140,9 @@ __device__ inline void softmax_block(uint32_t t_s, uint32_t p_row, uint32_t sw, 
   emit(va, 2);
   tc_wait_ld();
   emit(vb, 3);
+  tc_wait_st();
   l += (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
+  return true;
 }
 
 // Stores 32 accumulator columns (scaled) of this thread's row as bf16.
@@ -160,21 +168,22 @@ __global__ void __maxnreg__(200) attn_fwd_tc_kernel(const __grid_constant__ CUte
   extern __shared__ unsigned char smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   unsigned char* gen = smem_raw + (base - smem_u32(smem_raw));
-  const uint32_t q_s = base, k_s = base + kTileBytes, v_s = base + 3 * kTileBytes, p_s = base + 4 * kTileBytes;
-  const uint32_t bar0 = p_s + kPBytes;
-  volatile uint32_t* ctrl = reinterpret_cast<volatile uint32_t*>(gen + 4 * kTileBytes + kPBytes);
-  // Two CTAs share an SM (their startup, softmax and MMA phases interleave), so K is double-buffered and V is not.
-  // barriers (8 bytes each): 0 q_full, 1-2 k_full, 3 v_full, 4 v_free, 5 s_full, 6 p_ready, 7 o_full; then TMEM base, abort flag
+  const uint32_t q_s = base, k_s = base + kTileBytes, v_s = base + 3 * kTileBytes;
+  const uint32_t bar0 = base + 5 * kTileBytes;
+  volatile uint32_t* ctrl = reinterpret_cast<volatile uint32_t*>(gen + 5 * kTileBytes);
+  // Two CTAs share an SM (their startup, softmax and MMA phases interleave); K and V are double-buffered.
+  // barriers (8 bytes each): 0 q_full, 1-2 k_full, 3-4 v_full, 5-6 v_free, 7 s_full, 8 p_ready, 9 o_done;
+  // then the TMEM base address and the abort flag
   auto bar = [&](int i) { return bar0 + 8u * i; };
-  volatile uint32_t* tmem_slot = ctrl + 16;
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(ctrl + 17);
+  volatile uint32_t* tmem_slot = ctrl + 32;
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(ctrl + 33);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int qb = blockIdx.x, hq = blockIdx.y, s = blockIdx.z / p.n_seqs, b = blockIdx.z - s * p.n_seqs;
   const int nblk = qb + 1;                               // causal: key blocks 0 .. qb
   if (threadIdx.x == 128) {
     tma_prefetch_desc(&tmQKV);
-    for (int i = 0; i < 8; ++i) mbar_init(bar(i), i == 6 ? 128 : 1);
+    for (int i = 0; i < 10; ++i) mbar_init(bar(i), i == 8 ? 128 : 1);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     fence_async_smem();
@@ -188,7 +197,7 @@ __global__ void __maxnreg__(200) attn_fwd_tc_kernel(const __grid_constant__ CUte
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
-  const uint32_t tm_s = tmem, tm_o = tmem + 128;
+  const uint32_t tm_s = tmem, tm_o = tmem + 128, tm_p = tmem + 192;
 
   if (warp == 4) {
     if (lane == 0) {
@@ -201,21 +210,22 @@ __global__ void __maxnreg__(200) attn_fwd_tc_kernel(const __grid_constant__ CUte
         tma_load_3d_local(k_s + st * kTileBytes, &tmQKV, bar(1 + st), k_col, j * kBk, z);
       };
       auto load_v = [&](int j) {
-        mbar_expect_tx(bar(3), kTileBytes);
-        tma_load_3d_local(v_s, &tmQKV, bar(3), v_col, j * kBk, z);
+        const int st = j & 1;
+        mbar_expect_tx(bar(3 + st), kTileBytes);
+        tma_load_3d_local(v_s + st * kTileBytes, &tmQKV, bar(3 + st), v_col, j * kBk, z);
       };
       mbar_expect_tx(bar(0), kTileBytes);
       tma_load_3d_local(q_s, &tmQKV, bar(0), hq * kDh, qb * kBq, z);
       load_k(0);
       load_v(0);
-      if (nblk > 1) load_k(1);
+      if (nblk > 1) { load_k(1); load_v(1); }
       constexpr uint32_t idesc_s = idesc_bf16(0, 0, kBq, kBk);       // S = Q K^T : both K-major
       constexpr uint32_t idesc_o = idesc_bf16(0, 1, kBq, kDh);       // O = P V   : V MN-major
       auto mma_s = [&](int j) {
         const uint64_t a = smem_desc(q_s, 16u, 1024u), bd = smem_desc(k_s + (j & 1) * kTileBytes, 16u, 1024u);
 #pragma unroll
         for (int k = 0; k < kDh / 16; ++k) mma1(tm_s, a + 2u * k, bd + 2u * k, idesc_s, k != 0);
-        commit1(bar(5));
+        commit1(bar(7));
       };
       bool ok = mbar_wait(bar(0), 0, abort_flag, status) && mbar_wait(bar(1), 0, abort_flag, status);
       if (ok) {
@@ -223,24 +233,27 @@ __global__ void __maxnreg__(200) attn_fwd_tc_kernel(const __grid_constant__ CUte
         mma_s(0);
       }
       for (int j = 0; ok && j < nblk; ++j) {
-        if (!mbar_wait(bar(6), j & 1, abort_flag, status)) break;                 // P of block j is in shared memory:
-        if (j + 2 < nblk) load_k(j + 2);                                          // S(j) was read, so K(j)'s buffer is free
-        if (!mbar_wait(bar(3), j & 1, abort_flag, status)) break;                 // V of block j
+        const int st = j & 1;
+        // P of block j is in tensor memory and S(j) has been read: K(j)'s buffer and the S columns are free
+        if (!mbar_wait(bar(8), j & 1, abort_flag, status)) break;
         tc_fence_after();
-        const uint64_t bd = smem_desc(v_s, (uint32_t)kDh * 128u, 1024u);
-#pragma unroll
-        for (int k = 0; k < kBk / 16; ++k) {
-          const uint64_t a = smem_desc(p_s + (k >> 2) * (kPBytes / 2), 16u, 1024u) + 2u * (k & 3);
-          mma1(tm_o, a, bd + (uint64_t)((k * 16 * 128) >> 4), idesc_o, (j | k) != 0);
-        }
-        commit1(bar(4));                                                          // V buffer free
-        if (j + 1 == nblk) commit1(bar(7));                                       // O complete
-        if (j + 1 < nblk) {
+        if (j + 2 < nblk) load_k(j + 2);
+        if (j + 1 < nblk) {                                // S of the next block first: the threads need it soonest
           if (!mbar_wait(bar(1 + ((j + 1) & 1)), ((j + 1) >> 1) & 1, abort_flag, status)) break;
           tc_fence_after();
-          mma_s(j + 1);              // its commit also tells the threads that O += P V (j) is done with P and O
-          if (!mbar_wait(bar(4), j & 1, abort_flag, status)) break;
-          load_v(j + 1);
+          mma_s(j + 1);
+        }
+        if (!mbar_wait(bar(3 + st), (j >> 1) & 1, abort_flag, status)) break;     // V of block j
+        tc_fence_after();
+        const uint64_t bd = smem_desc(v_s + st * kTileBytes, (uint32_t)kDh * 128u, 1024u);
+#pragma unroll
+        for (int k = 0; k < kBk / 16; ++k)                                        // 16 keys = 8 columns of P
+          mma1_ta(tm_o, tm_p + 8u * k, bd + (uint64_t)((k * 16 * 128) >> 4), idesc_o, (j | k) != 0);
+        commit1(bar(5 + st));                                                     // V buffer free
+        commit1(bar(9));                                                          // P consumed, O at rest again
+        if (j + 2 < nblk) {
+          if (!mbar_wait(bar(5 + st), (j >> 1) & 1, abort_flag, status)) break;
+          load_v(j + 2);
         }
       }
     }
@@ -248,16 +261,21 @@ __global__ void __maxnreg__(200) attn_fwd_tc_kernel(const __grid_constant__ CUte
     // ---- softmax warps: thread = query row
     const int r = warp * 32 + lane;
     const int qi = qb * kBq + r;
-    const uint32_t t_s = tm_s + ((uint32_t)(warp * 32) << 16), t_o = tm_o + ((uint32_t)(warp * 32) << 16);
-    // 16-byte piece c (0..7) of this row inside a 64-key half of P (128-byte rows, 128-byte swizzle)
-    const uint32_t p_row = p_s + (uint32_t)(r >> 3) * 1024u + (uint32_t)(r & 7) * 128u;
-    const uint32_t sw = (uint32_t)(r & 7);
+    const uint32_t lane_off = (uint32_t)(warp * 32) << 16;
+    const uint32_t t_s = tm_s + lane_off, t_o = tm_o + lane_off, t_p = tm_p + lane_off;
     float m = -INFINITY, l = 0.f;
     bool ok = true;
     for (int j = 0; j < nblk; ++j) {
-      // S(j) is complete, and so is every earlier MMA: P and O are at rest until this warp arrives below
-      if (!__all_sync(0xffffffffu, mbar_wait(bar(5), j & 1, abort_flag, status))) { ok = false; break; }
+      if (!__all_sync(0xffffffffu, mbar_wait(bar(7), j & 1, abort_flag, status))) { ok = false; break; }      // S(j)
       tc_fence_after();
+      // called between the two passes: O += P V of the previous block must be done before P is overwritten and
+      // before O may be rescaled; it was issued right after S(j), so it is usually complete by now
+      auto before_p = [&]() {
+        if (j == 0) return true;
+        const bool done = __all_sync(0xffffffffu, mbar_wait(bar(9), (j - 1) & 1, abort_flag, status));
+        tc_fence_after();
+        return done;
+      };
       auto rescale = [&](float corr) {                   // whole warp: O row *= corr in tensor memory
         if (j == 0) return;                              // nothing accumulated yet
 #pragma unroll
@@ -271,13 +289,14 @@ __global__ void __maxnreg__(200) attn_fwd_tc_kernel(const __grid_constant__ CUte
         }
         tc_wait_st();
       };
-      if (j == qb) softmax_block<true>(t_s, p_row, sw, qi - j * kBk, p.scale_log2, m, l, rescale);
-      else softmax_block<false>(t_s, p_row, sw, kBk, p.scale_log2, m, l, rescale);
-      fence_async_smem();                                                         // P: generic writes -> MMA reads
+      bool fine;
+      if (j == qb) fine = softmax_block<true>(t_s, t_p, qi - j * kBk, p.scale_log2, m, l, before_p, rescale);
+      else fine = softmax_block<false>(t_s, t_p, kBk, p.scale_log2, m, l, before_p, rescale);
+      if (!fine) { ok = false; break; }
       tc_fence_before();
-      mbar_arrive(bar(6));
+      mbar_arrive(bar(8));
     }
-    if (ok && __all_sync(0xffffffffu, mbar_wait(bar(7), 0, abort_flag, status))) {
+    if (ok && __all_sync(0xffffffffu, mbar_wait(bar(9), (nblk - 1) & 1, abort_flag, status))) {
       tc_fence_after();
       const float inv = 1.f / l;
       const long long row = (long long)s * p.T + (long long)b * p.seq_len + qi;
