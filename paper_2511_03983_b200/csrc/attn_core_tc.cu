@@ -371,7 +371,10 @@ __device__ inline void probs_from_s(uint32_t t_s, int c0, int r, int k_lim, floa
   tc_wait_ld();
   chunk(vb, 1);
 }
-__device__ inline void ds_from_dp(uint32_t t_dp, int c0, int r, float dl, uint32_t ds_tile, const float (&pr)[64]) {
+// TO_TMEM: dS goes to tensor memory at column 16 c of `ds` (packed bf16 pairs, the A operand of dQ += dS K);
+// otherwise `ds` is the operand tile in shared memory.
+template <bool TO_TMEM>
+__device__ inline void ds_from_dp(uint32_t t_dp, int c0, int r, float dl, uint32_t ds, const float (&pr)[64]) {
   uint32_t va[32], vb[32];
   tc_ld32(t_dp + 32 * c0, va);
   tc_wait_ld();
@@ -382,20 +385,23 @@ __device__ inline void ds_from_dp(uint32_t t_dp, int c0, int r, float dl, uint32
     for (int e = 0; e < 16; ++e)
       w[e] = pack2(pr[32 * cc + 2 * e] * (__uint_as_float(v[2 * e]) - dl),
                    pr[32 * cc + 2 * e + 1] * (__uint_as_float(v[2 * e + 1]) - dl));
-    store_row_chunk32(ds_tile, r, c0 + cc, w);
+    if (TO_TMEM) tc_st16(ds + 16 * (c0 + cc), w);
+    else store_row_chunk32(ds, r, c0 + cc, w);
   };
   chunk(va, 0);
   tc_wait_ld();
   chunk(vb, 1);
+  if (TO_TMEM) tc_wait_st();
 }
 
 // ---- dQ: grid (query blocks, kept heads, S * n_seqs).  Per key block j: S = Q K^T and dP = dO V^T (128 x 128)
-// into tensor memory, the threads write dS (bf16) into shared memory, dQ += dS K accumulates in tensor memory.
+// into tensor memory, the threads write dS (bf16 pairs) into tensor memory as the A operand, dQ += dS K accumulates
+// in tensor memory.
 // S is double-buffered in tensor memory and issued two blocks ahead, dP one block ahead right after the threads
 // released it, so both are complete before the threads need them: the threads turn S(j) into probabilities (the
 // expensive half of their work) while dP(j) is still being computed.  K / V blocks are triple-buffered.
 constexpr int kDqStages = 3;
-constexpr int kDqSmem = kTileBytes * (2 + 2 * kDqStages) + 2 * kPBytes + 1024 + 256;    // Q, dO, K[3], V[3], dS[2]
+constexpr int kDqSmem = kTileBytes * (2 + 2 * kDqStages) + 1024 + 256;    // Q, dO, K[3], V[3]
 __global__ void __launch_bounds__(kBwdThreads) attn_dq_tc_kernel(const __grid_constant__ CUtensorMap tmQKV,
                                                                  const __grid_constant__ CUtensorMap tmDO,
                                                                  const AttnParams p, int* status) {
@@ -403,9 +409,9 @@ __global__ void __launch_bounds__(kBwdThreads) attn_dq_tc_kernel(const __grid_co
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   unsigned char* gen = smem_raw + (base - smem_u32(smem_raw));
   const uint32_t q_s = base, do_s = base + kTileBytes, k_s = base + 2 * kTileBytes,
-                 v_s = k_s + kDqStages * kTileBytes, ds_s = v_s + kDqStages * kTileBytes;
-  const uint32_t bar0 = ds_s + 2 * kPBytes;
-  volatile uint32_t* ctrl = reinterpret_cast<volatile uint32_t*>(gen + (2 + 2 * kDqStages) * kTileBytes + 2 * kPBytes);
+                 v_s = k_s + kDqStages * kTileBytes;
+  const uint32_t bar0 = v_s + kDqStages * kTileBytes;
+  volatile uint32_t* ctrl = reinterpret_cast<volatile uint32_t*>(gen + (2 + 2 * kDqStages) * kTileBytes);
   // barriers: 0 q_full, 1-3 kv_full, 4-6 kv_free, 7-8 s_full, 9 dp_full, 10 ds_ready, 11 dq_full
   auto bar = [&](int i) { return bar0 + 8u * i; };
   volatile uint32_t* tmem_slot = ctrl + 32;
@@ -430,7 +436,7 @@ __global__ void __launch_bounds__(kBwdThreads) attn_dq_tc_kernel(const __grid_co
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
-  const uint32_t tm_dp = tmem + 256, tm_dq = tmem + 384;      // S(j) at columns 128 (j & 1)
+  const uint32_t tm_dp = tmem + 256, tm_dq = tmem + 384, tm_ds = tmem + 448;      // S(j) at columns 128 (j & 1)
 
   if (warp == 8) {
     if (lane == 0) {
@@ -476,19 +482,18 @@ __global__ void __launch_bounds__(kBwdThreads) attn_dq_tc_kernel(const __grid_co
       }
       for (int j = 0; ok && j < nblk; ++j) {
         const int st = j % kDqStages;
-        // dS(j) is in shared memory; S(j) and dP(j) have been read (the threads read S before dP)
+        // dS(j) is in tensor memory; S(j) and dP(j) have been read (the threads read S before dP)
         if (!mbar_wait(bar(10), j & 1, abort_flag, status)) break;
         tc_fence_after();
-        if (j + 1 < nblk) mma_dp(j + 1);                 // block j + 1 arrived before S(j + 1) was issued
         const uint64_t bd = smem_desc(k_s + st * kTileBytes, (uint32_t)kDh * 128u, 1024u);
-        const uint32_t ds_j = ds_s + (j & 1) * kPBytes;
 #pragma unroll
-        for (int k = 0; k < kBk / 16; ++k) {
-          const uint64_t a = smem_desc(ds_j + (k >> 2) * (kPBytes / 2), 16u, 1024u) + 2u * (k & 3);
-          mma1(tm_dq, a, bd + (uint64_t)((k * 16 * 128) >> 4), idesc_q, (j | k) != 0);
-        }
+        for (int k = 0; k < kBk / 16; ++k)               // 16 keys = 8 columns of dS
+          mma1_ta(tm_dq, tm_ds + 8u * k, bd + (uint64_t)((k * 16 * 128) >> 4), idesc_q, (j | k) != 0);
         commit1(bar(4 + st));                            // block j's K / V are consumed
         if (j + 1 == nblk) commit1(bar(11));
+        // dP of the next block after dQ of this one: its commit then also tells the threads that dS may be rewritten
+        // (block j + 1 arrived before S(j + 1) was issued)
+        if (j + 1 < nblk) mma_dp(j + 1);
         if (j + 2 < nblk) {
           const int j2 = j + 2;
           if (!mbar_wait(bar(1 + j2 % kDqStages), (j2 / kDqStages) & 1, abort_flag, status)) break;
@@ -523,8 +528,7 @@ __global__ void __launch_bounds__(kBwdThreads) attn_dq_tc_kernel(const __grid_co
         probs_from_s<false, false>(t_s, 2 * half, r, k_lim, p.scale_log2, lse2, 0u, pr);
       if (!__all_sync(0xffffffffu, mbar_wait(bar(9), j & 1, abort_flag, status))) { ok = false; break; }
       tc_fence_after();
-      ds_from_dp(tm_dp + lane_off, 2 * half, r, dl, ds_s + (j & 1) * kPBytes, pr);
-      fence_async_smem();
+      ds_from_dp<true>(tm_dp + lane_off, 2 * half, r, dl, tm_ds + lane_off, pr);
       tc_fence_before();
       mbar_arrive(bar(10));
     }
@@ -699,7 +703,7 @@ __global__ void __launch_bounds__(kBwdThreads) attn_dkv_tc_kernel(const __grid_c
       if (!__all_sync(0xffffffffu, mbar_wait(bar(9), n & 1, abort_flag, status))) { ok = false; break; }
       if (n > 0 && !__all_sync(0xffffffffu, mbar_wait(bar(12), (n - 1) & 1, abort_flag, status))) { ok = false; break; }
       tc_fence_after();
-      ds_from_dp(tm_dp + lane_off, 2 * half, r, dl, ds_s, pr);
+      ds_from_dp<false>(tm_dp + lane_off, 2 * half, r, dl, ds_s, pr);
       fence_async_smem();
       tc_fence_before();
       mbar_arrive(bar(10));
