@@ -18,11 +18,14 @@
 // Warps 0-3: softmax / output; warp 4, one lane: TMA and MMA issue.
 // Backward (same tile sizes; probabilities recomputed from the stored log-sum-exp, dS = P (dP - delta)):
 //   dQ kernel     one CTA per query block: per key block S = Q K^T and dP = dO V^T into tensor memory, the threads
-//                 write dS (bf16) to shared memory, dQ += dS K accumulates in tensor memory over the key blocks.
+//                 write dS (bf16 pairs) into tensor memory as the A operand, dQ += dS K accumulates in tensor memory
+//                 over the key blocks.
 //   dK/dV kernel  one CTA per (key block, KV position): for every kept head that reads the position and every
-//                 query block at or after the key block, S and dP as above, the threads write P and dS, and
-//                 dV += P^T dO, dK += dS^T Q accumulate in tensor memory (P and dS are read as MN-major A
-//                 operands: the same bytes, no transpose).
+//                 query block at or after the key block, the transposed tiles S^T = K Q^T and dP^T = V dO^T (rows =
+//                 keys), the threads write P^T and dS^T back into tensor memory as A operands, and dV += P^T dO,
+//                 dK += dS^T Q accumulate in tensor memory.
+// No probability or score gradient ever passes through shared memory: its bandwidth is what the operand reads of
+// the MMAs need.
 // Every wait is bounded; on expiry the CTA records TWIST_ERR_DEVICE_TIMEOUT and leaves.
 #include "attn_core.cuh"
 #include "ptx.cuh"
@@ -33,7 +36,6 @@ namespace {
 constexpr int kDh = 64;                 // head dimension of this kernel
 constexpr int kBq = 128, kBk = 128;     // queries per CTA, keys per block
 constexpr int kTileBytes = 128 * kDh * 2;            // a 128-row tile of Q, K or V: 16 KB
-constexpr int kPBytes = kBq * kBk * 2;               // P: 32 KB (two 64-key halves of 16 KB)
 constexpr int kFwdThreads = 160;
 constexpr int kFwdSmem = kTileBytes * 5 + 1024 + 256;   // Q, K[2], V[2], alignment, barriers: two CTAs per SM
 constexpr int kFwdTmemCols = 256;       // S: columns 0..127, O: columns 128..191, P (bf16 pairs): columns 192..255
@@ -324,30 +326,16 @@ __global__ void __maxnreg__(200) attn_fwd_tc_kernel(const __grid_constant__ CUte
   }
 }
 
-// 16-byte pieces of row r of a [128 rows][2 x 64 columns] bf16 operand tile (two halves of 16 KB, 128-byte rows,
-// 128-byte swizzle): the layout of P and dS, readable as a K-major A operand (rows = M) or an MN-major one (rows = K).
-__device__ inline void store_row_chunk32(uint32_t tile, int r, int c, const uint32_t (&w)[16]) {
-  const uint32_t half = tile + (uint32_t)(c >> 1) * (kPBytes / 2) + (uint32_t)(r >> 3) * 1024u + (uint32_t)(r & 7) * 128u;
-  const uint32_t sw = (uint32_t)(r & 7);
-#pragma unroll
-  for (int q4 = 0; q4 < 4; ++q4) {
-    const uint32_t piece = (uint32_t)((c & 1) * 4 + q4);
-    sts128(half + ((piece ^ sw) << 4), make_uint4(w[4 * q4], w[4 * q4 + 1], w[4 * q4 + 2], w[4 * q4 + 3]));
-  }
-}
-
 constexpr int kBwdTmemCols = 512;
 constexpr int kBwdThreads = 288;        // 8 element-wise warps (two per tensor-memory lane quarter) + the control warp
 
-// Element-wise steps shared by the two backward kernels, for this thread's row and its 64 columns (chunks c0 and
-// c0 + 1 of 32 columns).  They are split so that the tensor pipe can work on dP while the threads are busy with
-// the exponentials:
-//   probs_from_s   P = exp2(S * scale - lse2) where visible (column <= k_lim), kept in registers (fp32) and, when
-//                  WRITE_P, written as bf16 into the operand tile;
-//   ds_from_dp     dS = P * (dP - dl), written as bf16 into the operand tile.
-template <bool WRITE_P, bool MASKED>
-__device__ inline void probs_from_s(uint32_t t_s, int c0, int r, int k_lim, float scale_log2, float lse2, uint32_t p_tile,
-                                    float (&pr)[64]) {
+// Element-wise steps of the dQ kernel, for this thread's query row and its 64 key columns (chunks c0 and c0 + 1 of 32
+// columns).  They are split so that the tensor pipe can work on dP while the threads are busy with the exponentials:
+//   probs_from_s   P = exp2(S * scale - lse2) where visible (column <= k_lim), kept in registers (fp32);
+//   ds_from_dp     dS = P * (dP - dl), packed bf16 pairs into tensor memory at column 16 c of `ds` (the A operand of
+//                  dQ += dS K).
+template <bool MASKED>
+__device__ inline void probs_from_s(uint32_t t_s, int c0, int k_lim, float scale_log2, float lse2, float (&pr)[64]) {
   uint32_t va[32], vb[32];
   tc_ld32(t_s + 32 * c0, va);
   tc_wait_ld();
@@ -360,21 +348,12 @@ __device__ inline void probs_from_s(uint32_t t_s, int c0, int r, int k_lim, floa
       if (MASKED) x = (32 * c + i <= k_lim) ? x : 0.f;
       pr[32 * cc + i] = x;
     }
-    if (WRITE_P) {
-      uint32_t w[16];
-#pragma unroll
-      for (int e = 0; e < 16; ++e) w[e] = pack2(pr[32 * cc + 2 * e], pr[32 * cc + 2 * e + 1]);
-      store_row_chunk32(p_tile, r, c, w);
-    }
   };
   chunk(va, 0);
   tc_wait_ld();
   chunk(vb, 1);
 }
-// TO_TMEM: dS goes to tensor memory at column 16 c of `ds` (packed bf16 pairs, the A operand of dQ += dS K);
-// otherwise `ds` is the operand tile in shared memory.
-template <bool TO_TMEM>
-__device__ inline void ds_from_dp(uint32_t t_dp, int c0, int r, float dl, uint32_t ds, const float (&pr)[64]) {
+__device__ inline void ds_from_dp(uint32_t t_dp, int c0, float dl, uint32_t ds, const float (&pr)[64]) {
   uint32_t va[32], vb[32];
   tc_ld32(t_dp + 32 * c0, va);
   tc_wait_ld();
@@ -385,13 +364,12 @@ __device__ inline void ds_from_dp(uint32_t t_dp, int c0, int r, float dl, uint32
     for (int e = 0; e < 16; ++e)
       w[e] = pack2(pr[32 * cc + 2 * e] * (__uint_as_float(v[2 * e]) - dl),
                    pr[32 * cc + 2 * e + 1] * (__uint_as_float(v[2 * e + 1]) - dl));
-    if (TO_TMEM) tc_st16(ds + 16 * (c0 + cc), w);
-    else store_row_chunk32(ds, r, c0 + cc, w);
+    tc_st16(ds + 16 * (c0 + cc), w);
   };
   chunk(va, 0);
   tc_wait_ld();
   chunk(vb, 1);
-  if (TO_TMEM) tc_wait_st();
+  tc_wait_st();
 }
 
 // ---- dQ: grid (query blocks, kept heads, S * n_seqs).  Per key block j: S = Q K^T and dP = dO V^T (128 x 128)
@@ -523,12 +501,12 @@ __global__ void __launch_bounds__(kBwdThreads) attn_dq_tc_kernel(const __grid_co
       const int k_lim = !row_ok ? -1 : ((j == qb) ? qi - j * kBk : kBk);
       const uint32_t t_s = tmem + lane_off + 128u * (j & 1);
       if (__any_sync(0xffffffffu, k_lim < kBk))      // warp-uniform: the tensor-memory loads inside are warp-wide
-        probs_from_s<false, true>(t_s, 2 * half, r, k_lim, p.scale_log2, lse2, 0u, pr);
+        probs_from_s<true>(t_s, 2 * half, k_lim, p.scale_log2, lse2, pr);
       else
-        probs_from_s<false, false>(t_s, 2 * half, r, k_lim, p.scale_log2, lse2, 0u, pr);
+        probs_from_s<false>(t_s, 2 * half, k_lim, p.scale_log2, lse2, pr);
       if (!__all_sync(0xffffffffu, mbar_wait(bar(9), j & 1, abort_flag, status))) { ok = false; break; }
       tc_fence_after();
-      ds_from_dp<true>(tm_dp + lane_off, 2 * half, r, dl, tm_ds + lane_off, pr);
+      ds_from_dp(tm_dp + lane_off, 2 * half, dl, tm_ds + lane_off, pr);
       tc_fence_before();
       mbar_arrive(bar(10));
     }
@@ -557,24 +535,84 @@ __global__ void __launch_bounds__(kBwdThreads) attn_dq_tc_kernel(const __grid_co
 }
 
 // ---- dK, dV: grid (key blocks, KV positions, S * n_seqs).  Units (kept head, query block) stream through with the
-// same schedule as the dQ kernel: S two units ahead into one of two tensor-memory buffers, dP one unit ahead, the
-// threads form P from S while dP is computed; dV += P^T dO and dK += dS^T Q accumulate in tensor memory.  P is
-// double-buffered in shared memory; dS has one tile, rewritten once the previous unit's MMAs are done with it.
+// same schedule as the dQ kernel (S two units ahead, dP one).  The score tiles are computed with the keys as rows, S^T = K Q^T and dP^T = V dO^T (128 keys x 128 queries), so that the thread that owns
+// tensor-memory lane r owns key r: the probabilities it forms are rows of P^T and dS^T, which is exactly the A operand
+// of dV += P^T dO and dK += dS^T Q.  They are written back into tensor memory (packed bf16 pairs, over the first half
+// of the thread's own 64 score columns) and never touch shared memory; the softmax statistics, now per column, are
+// staged in shared memory once per unit.  Per unit the MMAs read 96 KB of operands from shared memory instead of 160
+// KB and the threads write none.
 constexpr int kDkvStages = 3;
-constexpr int kDkvSmem = kTileBytes * (2 + 2 * kDkvStages) + 3 * kPBytes + 1024 + 256;   // K, V, Q[3], dO[3], P[2], dS
+constexpr int kDkvSmem = kTileBytes * (2 + 2 * kDkvStages) + 1024 + 256;   // K, V, Q[3], dO[3]
+
+// Thread = key row r, 64 query columns starting at col0 (= 64 (warp >> 2)); `stat` = shared-memory address of the 64
+// per-query values (log-sum-exp in the log2 domain, +inf for queries past the sequence end).  P^T goes to registers
+// and, packed, to columns 0..31 of the thread's own score columns at t_s.
+template <bool MASKED>
+__device__ inline void probs_from_st(uint32_t t_s, uint32_t stat, int r, int col0, float scale_log2, float (&pr)[64]) {
+  uint32_t va[32], vb[32];
+  tc_ld32(t_s, va);
+  tc_wait_ld();
+  tc_ld32(t_s + 32, vb);
+  auto chunk = [&](const uint32_t (&v)[32], int cc) {
+#pragma unroll
+    for (int q4 = 0; q4 < 8; ++q4) {
+      const uint4 lv = lds128(stat + 16u * (8 * cc + q4));
+      const float l4[4] = {__uint_as_float(lv.x), __uint_as_float(lv.y), __uint_as_float(lv.z), __uint_as_float(lv.w)};
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const int i = 4 * q4 + e;
+        float x = ex2_fast(fmaf(__uint_as_float(v[i]), scale_log2, -l4[e]));
+        if (MASKED) x = (col0 + 32 * cc + i >= r) ? x : 0.f;       // causal: key <= query
+        pr[32 * cc + i] = x;
+      }
+    }
+    uint32_t w[16];
+#pragma unroll
+    for (int e = 0; e < 16; ++e) w[e] = pack2(pr[32 * cc + 2 * e], pr[32 * cc + 2 * e + 1]);
+    tc_st16(t_s + 16 * cc, w);          // over score columns this thread has already read
+  };
+  chunk(va, 0);
+  tc_wait_ld();
+  chunk(vb, 1);
+}
+// dS^T = P^T * (dP^T - delta[query]), packed over the first half of the thread's own dP^T columns.
+__device__ inline void ds_from_dpt(uint32_t t_dp, uint32_t stat, const float (&pr)[64]) {
+  uint32_t va[32], vb[32];
+  tc_ld32(t_dp, va);
+  tc_wait_ld();
+  tc_ld32(t_dp + 32, vb);
+  auto chunk = [&](const uint32_t (&v)[32], int cc) {
+    uint32_t w[16];
+#pragma unroll
+    for (int q4 = 0; q4 < 8; ++q4) {
+      const uint4 dv = lds128(stat + 16u * (8 * cc + q4));
+      const int i = 4 * q4;
+      w[2 * q4] = pack2(pr[32 * cc + i] * (__uint_as_float(v[i]) - __uint_as_float(dv.x)),
+                        pr[32 * cc + i + 1] * (__uint_as_float(v[i + 1]) - __uint_as_float(dv.y)));
+      w[2 * q4 + 1] = pack2(pr[32 * cc + i + 2] * (__uint_as_float(v[i + 2]) - __uint_as_float(dv.z)),
+                            pr[32 * cc + i + 3] * (__uint_as_float(v[i + 3]) - __uint_as_float(dv.w)));
+    }
+    tc_st16(t_dp + 16 * cc, w);
+  };
+  chunk(va, 0);
+  tc_wait_ld();
+  chunk(vb, 1);
+  tc_wait_st();
+}
+
 __global__ void __launch_bounds__(kBwdThreads) attn_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmQKV,
-                                                                  const __grid_constant__ CUtensorMap tmDO,
-                                                                  const AttnParams p, int* status) {
+                                                                    const __grid_constant__ CUtensorMap tmDO,
+                                                                    const AttnParams p, int* status) {
   extern __shared__ unsigned char smem_raw[];
   __shared__ int match[64];
   __shared__ int n_match_s;
+  __shared__ __align__(16) float stat_w[8][2][64];       // per element-wise warp: [lse2 | delta][its 64 queries]
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   unsigned char* gen = smem_raw + (base - smem_u32(smem_raw));
-  const uint32_t k_s = base, v_s = base + kTileBytes, q_s = base + 2 * kTileBytes,
-                 do_s = q_s + kDkvStages * kTileBytes, p_s = do_s + kDkvStages * kTileBytes, ds_s = p_s + 2 * kPBytes;
-  const uint32_t bar0 = ds_s + kPBytes;
-  volatile uint32_t* ctrl = reinterpret_cast<volatile uint32_t*>(gen + (2 + 2 * kDkvStages) * kTileBytes + 3 * kPBytes);
-  // barriers: 0 kv_full, 1-3 q_full, 4-6 q_free, 7-8 s_full, 9 dp_full, 10 pds_ready, 11 acc_full, 12 acc_done
+  const uint32_t k_s = base, v_s = base + kTileBytes, q_s = base + 2 * kTileBytes, do_s = q_s + kDkvStages * kTileBytes;
+  const uint32_t bar0 = do_s + kDkvStages * kTileBytes;
+  volatile uint32_t* ctrl = reinterpret_cast<volatile uint32_t*>(gen + (2 + 2 * kDkvStages) * kTileBytes);
+  // barriers: 0 kv_full, 1-3 q_full, 4-6 q_free, 7-8 s_full, 9 dp_full, 10 pds_ready, 11 acc_full
   auto bar = [&](int i) { return bar0 + 8u * i; };
   volatile uint32_t* tmem_slot = ctrl + 32;
   volatile int* abort_flag = reinterpret_cast<volatile int*>(ctrl + 33);
@@ -585,7 +623,7 @@ __global__ void __launch_bounds__(kBwdThreads) attn_dkv_tc_kernel(const __grid_c
   if (threadIdx.x == 256) {
     tma_prefetch_desc(&tmQKV);
     tma_prefetch_desc(&tmDO);
-    for (int i = 0; i < 13; ++i) mbar_init(bar(i), i == 10 ? 256 : 1);
+    for (int i = 0; i < 12; ++i) mbar_init(bar(i), i == 10 ? 256 : 1);
     *abort_flag = 0;
     int n = 0;
     if (kvp < held)
@@ -604,7 +642,7 @@ __global__ void __launch_bounds__(kBwdThreads) attn_dkv_tc_kernel(const __grid_c
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
-  const uint32_t tm_dp = tmem + 256, tm_dv = tmem + 384, tm_dk = tmem + 448;   // S(n) at columns 128 (n & 1)
+  const uint32_t tm_dp = tmem + 256, tm_dv = tmem + 384, tm_dk = tmem + 448;   // S^T(n) at columns 128 (n & 1)
   const int per_head = nqb - kb;                         // query blocks kb .. nqb-1
   const int total = n_match_s * per_head;                // units (head, query block)
 
@@ -621,18 +659,18 @@ __global__ void __launch_bounds__(kBwdThreads) attn_dkv_tc_kernel(const __grid_c
       tma_load_3d_local(k_s, &tmQKV, bar(0), p.a_sub + kvp * kDh, kb * kBk, z);
       tma_load_3d_local(v_s, &tmQKV, bar(0), p.a_sub + (p.kv_max + kvp) * kDh, kb * kBk, z);
       for (int n = 0; n < kDkvStages && n < total; ++n) load_q(n);
-      constexpr uint32_t idesc_s = idesc_bf16(0, 0, kBq, kBk);       // S = Q K^T, dP = dO V^T
-      constexpr uint32_t idesc_t = idesc_bf16(1, 1, kBk, kDh);       // dV = P^T dO, dK = dS^T Q : both MN-major
+      constexpr uint32_t idesc_s = idesc_bf16(0, 0, kBk, kBq);       // S^T = K Q^T, dP^T = V dO^T : both K-major
+      constexpr uint32_t idesc_a = idesc_bf16(0, 1, kBk, kDh);       // dV += P^T dO, dK += dS^T Q : B MN-major
       auto mma_s = [&](int n) {
-        const uint64_t aq = smem_desc(q_s + (n % kDkvStages) * kTileBytes, 16u, 1024u), bk = smem_desc(k_s, 16u, 1024u);
+        const uint64_t ak = smem_desc(k_s, 16u, 1024u), bq = smem_desc(q_s + (n % kDkvStages) * kTileBytes, 16u, 1024u);
 #pragma unroll
-        for (int k = 0; k < kDh / 16; ++k) mma1(tmem + 128u * (n & 1), aq + 2u * k, bk + 2u * k, idesc_s, k != 0);
+        for (int k = 0; k < kDh / 16; ++k) mma1(tmem + 128u * (n & 1), ak + 2u * k, bq + 2u * k, idesc_s, k != 0);
         commit1(bar(7 + (n & 1)));
       };
       auto mma_dp = [&](int n) {
-        const uint64_t ao = smem_desc(do_s + (n % kDkvStages) * kTileBytes, 16u, 1024u), bv = smem_desc(v_s, 16u, 1024u);
+        const uint64_t av = smem_desc(v_s, 16u, 1024u), bo = smem_desc(do_s + (n % kDkvStages) * kTileBytes, 16u, 1024u);
 #pragma unroll
-        for (int k = 0; k < kDh / 16; ++k) mma1(tm_dp, ao + 2u * k, bv + 2u * k, idesc_s, k != 0);
+        for (int k = 0; k < kDh / 16; ++k) mma1(tm_dp, av + 2u * k, bo + 2u * k, idesc_s, k != 0);
         commit1(bar(9));
       };
       bool ok = mbar_wait(bar(0), 0, abort_flag, status) && mbar_wait(bar(1), 0, abort_flag, status);
@@ -650,28 +688,28 @@ __global__ void __launch_bounds__(kBwdThreads) attn_dkv_tc_kernel(const __grid_c
       }
       for (int n = 0; ok && n < total; ++n) {
         const int st = n % kDkvStages;
-        // P and dS of unit n are in shared memory; S(n) and dP(n) have been read (the threads read S before dP)
+        // P^T and dS^T of unit n are in tensor memory (inside the S^T(n) and dP^T columns)
         if (!mbar_wait(bar(10), n & 1, abort_flag, status)) break;
         tc_fence_after();
-        if (n + 1 < total) mma_dp(n + 1);                // unit n + 1 arrived before S(n + 1) was issued
-        // A = P^T / dS^T: rows of the tile are the contraction index (queries), 64 keys per 128-byte row, the two
-        // 64-key halves 16 KB apart; B = dO / Q with rows = queries.
-        const uint64_t ap = smem_desc(p_s + (n & 1) * kPBytes, (uint32_t)(kPBytes / 2), 1024u);
-        const uint64_t ad = smem_desc(ds_s, (uint32_t)(kPBytes / 2), 1024u);
+        const uint32_t t_p = tmem + 128u * (n & 1);
         const uint64_t bo = smem_desc(do_s + st * kTileBytes, (uint32_t)kDh * 128u, 1024u);
         const uint64_t bq = smem_desc(q_s + st * kTileBytes, (uint32_t)kDh * 128u, 1024u);
+        // contraction over the 128 queries, 16 per step: 8 packed columns, the two 64-query halves 64 columns apart
 #pragma unroll
-        for (int k = 0; k < kBq / 16; ++k) mma1(tm_dv, ap + (uint64_t)(k * 128), bo + (uint64_t)(k * 128), idesc_t, (n | k) != 0);
+        for (int k = 0; k < kBq / 16; ++k)
+          mma1_ta(tm_dv, t_p + 64u * (k >> 2) + 8u * (k & 3), bo + (uint64_t)(k * 128), idesc_a, (n | k) != 0);
 #pragma unroll
-        for (int k = 0; k < kBq / 16; ++k) mma1(tm_dk, ad + (uint64_t)(k * 128), bq + (uint64_t)(k * 128), idesc_t, (n | k) != 0);
-        commit1(bar(12));                                // the dS tile may be rewritten
+        for (int k = 0; k < kBq / 16; ++k)
+          mma1_ta(tm_dk, tm_dp + 64u * (k >> 2) + 8u * (k & 3), bq + (uint64_t)(k * 128), idesc_a, (n | k) != 0);
         commit1(bar(4 + st));                            // unit n's Q / dO are consumed
         if (n + 1 == total) commit1(bar(11));
+        // in issue order behind the MMAs that read dS^T(n) / P^T(n) out of the columns they overwrite
+        if (n + 1 < total) mma_dp(n + 1);                // unit n + 1 arrived before S^T(n + 1) was issued
         if (n + 2 < total) {
           const int n2 = n + 2;
           if (!mbar_wait(bar(1 + n2 % kDkvStages), (n2 / kDkvStages) & 1, abort_flag, status)) break;
           tc_fence_after();
-          mma_s(n2);                                     // into the buffer S(n) has just left; P(n & 1) is free after it
+          mma_s(n2);
         }
         if (n + kDkvStages < total) {
           if (!mbar_wait(bar(4 + st), (n / kDkvStages) & 1, abort_flag, status)) break;
@@ -681,34 +719,47 @@ __global__ void __launch_bounds__(kBwdThreads) attn_dkv_tc_kernel(const __grid_c
     }
   } else {
     const int quarter = warp & 3, half = warp >> 2;
-    const int r = quarter * 32 + lane;
+    const int r = quarter * 32 + lane;                   // key row of this thread
     const uint32_t lane_off = (uint32_t)(quarter * 32) << 16;
+    // Each warp stages the statistics of its own 64 queries (lane l: queries l and l + 32 of its half), one unit
+    // ahead in registers, so no barrier between warps is needed.
+    struct Stat { float l0, l1, d0, d1; };
+    auto load_stat = [&](int n) {
+      Stat o;
+      o.l0 = INFINITY; o.l1 = INFINITY; o.d0 = 0.f; o.d1 = 0.f;      // no probability mass past the sequence end
+      if (n >= total) return o;
+      const int hq = match[n / per_head], i = kb + n % per_head;
+      const int q0 = i * kBq + 64 * half + lane;
+      const long long at = ((long long)s * p.heads + hq) * p.T + (long long)b * p.seq_len + q0;
+      if (q0 < p.seq_len) { o.l0 = p.lse[at] * 1.4426950408889634f; o.d0 = p.delta[at]; }
+      if (q0 + 32 < p.seq_len) { o.l1 = p.lse[at + 32] * 1.4426950408889634f; o.d1 = p.delta[at + 32]; }
+      return o;
+    };
+    Stat staged = load_stat(0);
+    const uint32_t st_lse = smem_u32(&stat_w[warp][0][0]), st_dl = smem_u32(&stat_w[warp][1][0]);
     bool ok = true;
     for (int n = 0; n < total; ++n) {
       float pr[64];
-      const int hq = match[n / per_head], i = kb + n % per_head;
-      const int qi = i * kBq + r;
-      const bool row_ok = qi < p.seq_len;
-      const long long stat = ((long long)s * p.heads + hq) * p.T + (long long)b * p.seq_len + qi;
-      const float lse2 = row_ok ? p.lse[stat] * 1.4426950408889634f : 0.f;
-      const float dl = row_ok ? p.delta[stat] : 0.f;
+      __syncwarp();                                      // the previous unit's reads of the staging area are done
+      stat_w[warp][0][lane] = staged.l0;
+      stat_w[warp][0][lane + 32] = staged.l1;
+      stat_w[warp][1][lane] = staged.d0;
+      stat_w[warp][1][lane + 32] = staged.d1;
+      __syncwarp();
+      staged = load_stat(n + 1);                         // in flight during this unit
+      const int i = kb + n % per_head;
       if (!__all_sync(0xffffffffu, mbar_wait(bar(7 + (n & 1)), (n >> 1) & 1, abort_flag, status))) { ok = false; break; }
       tc_fence_after();
-      const int k_lim = !row_ok ? -1 : ((i == kb) ? r : kBk);                     // diagonal block: keys <= query
-      const uint32_t t_s = tmem + lane_off + 128u * (n & 1);
-      if (__any_sync(0xffffffffu, k_lim < kBk))      // warp-uniform: the tensor-memory loads inside are warp-wide
-        probs_from_s<true, true>(t_s, 2 * half, r, k_lim, p.scale_log2, lse2, p_s + (n & 1) * kPBytes, pr);
-      else
-        probs_from_s<true, false>(t_s, 2 * half, r, k_lim, p.scale_log2, lse2, p_s + (n & 1) * kPBytes, pr);
+      const uint32_t t_s = tmem + lane_off + 128u * (n & 1) + 64u * half;
+      if (i == kb) probs_from_st<true>(t_s, st_lse, r, 64 * half, p.scale_log2, pr);      // diagonal block
+      else probs_from_st<false>(t_s, st_lse, r, 64 * half, p.scale_log2, pr);
       if (!__all_sync(0xffffffffu, mbar_wait(bar(9), n & 1, abort_flag, status))) { ok = false; break; }
-      if (n > 0 && !__all_sync(0xffffffffu, mbar_wait(bar(12), (n - 1) & 1, abort_flag, status))) { ok = false; break; }
       tc_fence_after();
-      ds_from_dp<false>(tm_dp + lane_off, 2 * half, r, dl, ds_s, pr);
-      fence_async_smem();
+      ds_from_dpt(tm_dp + lane_off + 64u * half, st_dl, pr);
       tc_fence_before();
       mbar_arrive(bar(10));
     }
-    // accumulator rows are keys now: thread r owns key kb * 128 + r; the first four warps store dV, the others dK
+    // thread r owns key kb * 128 + r; the first four warps store dV, the others dK
     const int kj = kb * kBk + r;
     const long long row = (long long)s * p.T + (long long)b * p.seq_len + kj;
     __nv_bfloat16* dst = p.d_qkv + row * p.nq + p.a_sub + ((half ? 0 : p.kv_max) + kvp) * kDh;
