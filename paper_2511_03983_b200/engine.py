@@ -374,7 +374,6 @@ class HybridRoundEngine(RoundEngine):
 
     def __init__(self, w: Workload, device: str = "cuda", **kw):
         assert w.dtype == DTYPE_BF16 and w.n_heads == 0 and w.n_subnets >= 2, "bf16 FFN-only workloads"
-        assert w.optimizer != "adam", "the central model's moments would need full-width arrays"
         super().__init__(w, device=device, keep_f32_full=True, **kw)
         F, T = w.d_ff, w.tokens
         g, dev = self.g, self.dev
@@ -382,6 +381,9 @@ class HybridRoundEngine(RoundEngine):
         act = lambda width: torch.empty(1, T, width, dtype=bf, device=dev)
         self.c_pre, self.c_dpre, self.c_hh = act(g * F), act(g * F), act(F)
         self.c_mask = torch.zeros(1, F, dtype=torch.uint8, device=dev)
+        if self.adam:      # the central worker's moments are full-width like its weights; zeroed when its layer starts
+            f32 = lambda rows: torch.zeros(1, rows, w.d_model, dtype=torch.float32, device=dev)
+            self.c_gu_m1, self.c_gu_m2, self.c_down_m1, self.c_down_m2 = f32(g * F), f32(g * F), f32(F), f32(F)
 
     def gather_layer(self, l: int, which=("ffn",)):
         """Slices of workers 1 .. S-1 only; the central worker's activation mask for this layer."""
@@ -396,25 +398,36 @@ class HybridRoundEngine(RoundEngine):
         with self._timed("gather"):
             B.twist_gather_subnets(segs, w.n_subnets - 1, d, w.dtype)
             B.twist_hidden_mask(self.cover_ffn[l], w.n_ffn_blocks, w.ffn_block, 0, 1, self.c_mask)
+            for n in self.moment_names:        # a fresh worker state, also for the central worker
+                getattr(self, n).zero_()
+            if self.adam:
+                for t in (self.c_gu_m1, self.c_gu_m2, self.c_down_m1, self.c_down_m2):
+                    t.zero_()
         self.launches += 2
 
     def ffn_step(self, l: int, k: int, lr: Optional[float] = None):
         w = self.w
         lr = w.lr if lr is None else lr
         S, T, d, F = w.n_subnets, w.tokens, w.d_model, w.d_ff
+        central_opt, others_opt = {}, {}
+        if self.adam:
+            opt = B.adam(k + 1, w.beta1, w.beta2, w.adam_eps)
+            central_opt = dict(opt=opt, m_gu=self.c_gu_m1, v_gu=self.c_gu_m2, m_down=self.c_down_m1, v_down=self.c_down_m2)
+            others_opt = dict(opt=opt, m_gu=self.w_gu_m1[1:], v_gu=self.w_gu_m2[1:], m_down=self.w_down_m1[1:],
+                              v_down=self.w_down_m2[1:])
         # central worker: the full-width layer under its mask, updated in place
         c = B.ffn_args(w.ffn_kind, w.dtype, 1, T, d, F, self.alpha_f, lr, x=self.X[k][:1], w_gu=self.full_gu[l],
                        w_down=self.full["down"][l], w_gu_master=self.full_gu_f32[l],
                        w_down_master=self.full_f32["down"][l], pre=self.c_pre, hh=self.c_hh,
                        y=self.y[:1] if self.store_outputs else None, dy=self.dy[:1], dpre=self.c_dpre,
                        dx=self.dx[:1] if self.dx is not None else None, hidden_mask=self.c_mask,
-                       tgt=self.Td[k][:1], loss=self.loss[l, 0, k][:1], loss_ws=self.ws)
+                       tgt=self.Td[k][:1], loss=self.loss[l, 0, k][:1], loss_ws=self.ws, **central_opt)
         # workers 1 .. S-1: gathered slices
         o = B.ffn_args(w.ffn_kind, w.dtype, S - 1, T, d, w.f_sub, self.alpha_f, lr, x=self.X[k][1:], w_gu=self.w_gu[1:],
                        w_down=self.w_down[1:], w_gu_master=self.w_gu_m[1:], w_down_master=self.w_down_m[1:],
                        pre=self.pre[1:], hh=self.hh[1:], y=self.y[1:] if self.store_outputs else None, dy=self.dy[1:],
                        dpre=self.dpre[1:], dx=self.dx[1:] if self.dx is not None else None, tgt=self.Td[k][1:],
-                       loss=self.loss[l, 0, k][1:], loss_ws=self.ws)
+                       loss=self.loss[l, 0, k][1:], loss_ws=self.ws, **others_opt)
         with self._timed("ffn_fwd"):
             B.twist_subnet_ffn_fwd(c)
             B.twist_subnet_ffn_fwd(o)

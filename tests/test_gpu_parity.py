@@ -580,6 +580,15 @@ def test_deployment_extraction_and_evaluation_modes(B, eval_keep_ratio):
     assert F // w.ffn_block == w.n_ffn_blocks
 
 
+def test_hybrid_twist_round_with_adam_matches_the_oracle_round(B):
+    """Hybrid TwIST with the paper's optimiser: the central worker's moments are full-width and start at zero like
+    the slices' moments; a masked neuron's zero gradient gives a zero Adam step."""
+    from paper_2511_03983_b200.engine import HybridRoundEngine
+    w = replace(I.scaled_twin(I.PRESETS[5], d_model=136, d_ff=544, d_head=0, tokens=200, n_layers=2, local_steps=3),
+                n_subnets=4, sample_mode=I.MODE_COVER, optimizer="adam", lr=1e-3, beta1=0.9, beta2=0.99, adam_eps=3e-3)
+    _run_round_and_compare(B, w, engine_cls=HybridRoundEngine)
+
+
 def test_hidden_mask_from_cover_bits(B):
     cover = np.array([0b101, 0b010, 0, 0b111, 0b100], dtype=np.uint32)
     mask = torch.zeros(2, 15, dtype=torch.uint8, device="cuda")
