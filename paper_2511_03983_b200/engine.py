@@ -124,6 +124,9 @@ class RoundEngine:
         self.Tq: List[torch.Tensor] = []
         self.A: List[torch.Tensor] = []
         self.launches = 0
+        # what the gather reads as blueprint, what the aggregate reads as ranks, and the activation mask of the FFN
+        # calls: the sampler's outputs and none, unless a subclass (Masked TwIST) substitutes its own
+        self.gather_idx_ffn, self.agg_pos_ffn, self.h_mask = self.idx_ffn, self.pos_ffn, None
         # optional per-phase CUDA-event timing (events on the launching stream)
         self.timing = False
         self.events: Dict[str, List[Tuple[torch.cuda.Event, torch.cuda.Event]]] = {}
@@ -164,11 +167,11 @@ class RoundEngine:
         segs = []
         if "ffn" in which:
             if self.g == 2:
-                segs.append(B.gather_segment(self.full["gate"][l], self.w_gu, self.w_gu_m, self.idx_ffn[l], None,
+                segs.append(B.gather_segment(self.full["gate"][l], self.w_gu, self.w_gu_m, self.gather_idx_ffn[l], None,
                                              w.ffn_keep, w.ffn_keep, w.ffn_block, 0, gf * d, 0))
-            segs.append(B.gather_segment(self.full["up"][l], self.w_gu, self.w_gu_m, self.idx_ffn[l], None,
+            segs.append(B.gather_segment(self.full["up"][l], self.w_gu, self.w_gu_m, self.gather_idx_ffn[l], None,
                                          w.ffn_keep, w.ffn_keep, w.ffn_block, 0, gf * d, f if self.g == 2 else 0))
-            segs.append(B.gather_segment(self.full["down"][l], self.w_down, self.w_down_m, self.idx_ffn[l], None,
+            segs.append(B.gather_segment(self.full["down"][l], self.w_down, self.w_down_m, self.gather_idx_ffn[l], None,
                                          w.ffn_keep, w.ffn_keep, w.ffn_block, 0, f * d, 0))
         if self.has_attn and "attn" in which:
             H, Hkv, dh = w.n_heads, w.n_kv_heads, w.d_head
@@ -198,12 +201,12 @@ class RoundEngine:
         if "ffn" in which:
             if self.g == 2:
                 segs.append(B.aggregate_segment(self.full["gate"][l], f32("gate"), sub(self.w_gu, self.w_gu_m),
-                                                self.cover_ffn[l], self.pos_ffn[l], nb, w.ffn_block, 0, gf * d, 0))
+                                                self.cover_ffn[l], self.agg_pos_ffn[l], nb, w.ffn_block, 0, gf * d, 0))
             segs.append(B.aggregate_segment(self.full["up"][l], f32("up"), sub(self.w_gu, self.w_gu_m),
-                                            self.cover_ffn[l], self.pos_ffn[l], nb, w.ffn_block, 0, gf * d,
+                                            self.cover_ffn[l], self.agg_pos_ffn[l], nb, w.ffn_block, 0, gf * d,
                                             f if self.g == 2 else 0))
             segs.append(B.aggregate_segment(self.full["down"][l], f32("down"), sub(self.w_down, self.w_down_m),
-                                            self.cover_ffn[l], self.pos_ffn[l], nb, w.ffn_block, 0, f * d, 0))
+                                            self.cover_ffn[l], self.agg_pos_ffn[l], nb, w.ffn_block, 0, f * d, 0))
         if self.has_attn and "attn" in which:
             H, Hkv, dh = w.n_heads, w.n_kv_heads, w.d_head
             q_sub = sub(self.w_qkv, self.w_qkv_m)
@@ -245,7 +248,7 @@ class RoundEngine:
                        x=self.X[k], w_gu=self.w_gu, w_down=self.w_down, w_gu_master=self.w_gu_m,
                        w_down_master=self.w_down_m, pre=self.pre, hh=self.hh,
                        y=self.y if self.store_outputs else None, dy=self.dy, dpre=self.dpre,
-                       dx=self.dx, dw_gu=self.dw_gu, dw_down=self.dw_down, **fused,
+                       dx=self.dx, dw_gu=self.dw_gu, dw_down=self.dw_down, hidden_mask=self.h_mask, **fused,
                        **self._opt(k, ("_gu", "w_gu"), ("_down", "w_down")))
         with self._timed("ffn_fwd"):
             B.twist_subnet_ffn_fwd(a)
@@ -363,6 +366,42 @@ class RoundEngine:
         self.sample_masks(rnd)
         for l in range(self.w.n_layers):
             self.run_layer(l)
+
+
+class MaskedRoundEngine(RoundEngine):
+    """Masked TwIST (Sec. 4.1) for the FFN blocks: every worker holds a full-width copy of the layer and is turned
+    into its subnet by an activation mask; nothing is physically smaller.  The "gather" is a copy of the whole layer
+    to every worker (the identity blueprint), the masks come from the sampled blueprints' cover bits, and the
+    aggregator averages every block over the workers whose blueprint holds it.  In exact arithmetic the round
+    equals RoundEngine's, at N_full / N_sub times its flops and S full copies of a layer: a simulation mode and an
+    on-device check of "masked = gathered", not a fast path."""
+
+    def __init__(self, w: Workload, device: str = "cuda", **kw):
+        from dataclasses import replace as _replace
+        assert w.dtype == DTYPE_BF16 and w.n_heads == 0, "bf16 FFN-only workloads"
+        nb = w.n_ffn_blocks
+        super().__init__(_replace(w, ffn_keep=nb), device=device, **kw)      # storage: full-width slices
+        self.true_w = w
+        L, S = w.n_layers, w.n_subnets
+        i32 = dict(dtype=torch.int32, device=self.dev)
+        self.idx_ffn = torch.empty(L, S, w.ffn_keep, **i32)                   # the sampled blueprints
+        ident = torch.arange(nb, **i32).expand(L, S, nb).contiguous()
+        self.gather_idx_ffn, self.agg_pos_ffn = ident, ident                  # every worker copies / returns every block
+        self.h_mask = torch.zeros(S, w.d_ff, dtype=torch.uint8, device=self.dev)
+        self.alpha_f = math.sqrt(nb / w.ffn_keep)                             # the subnet's scale (Sec. 3.4)
+
+    def sample_masks(self, rnd: int):
+        w = self.true_w
+        with self._timed("sample_masks"):
+            B.twist_sample_masks(w.seed_mask, rnd, 0, w.n_layers, B.KIND_FFN, w.n_ffn_blocks, w.n_subnets, w.ffn_keep,
+                                 list(w.common_ffn), w.sample_mode, self.idx_ffn, self.cover_ffn, self.pos_ffn)
+        self.launches += 2
+
+    def gather_layer(self, l: int, which=("ffn",)):
+        super().gather_layer(l, which=("ffn",))
+        w = self.true_w
+        B.twist_hidden_mask(self.cover_ffn[l], w.n_ffn_blocks, w.ffn_block, 0, w.n_subnets, self.h_mask)
+        self.launches += 1
 
 
 class HybridRoundEngine(RoundEngine):

@@ -580,6 +580,17 @@ def test_deployment_extraction_and_evaluation_modes(B, eval_keep_ratio):
     assert F // w.ffn_block == w.n_ffn_blocks
 
 
+@pytest.mark.parametrize("kind,mode", [(I.FFN_SWIGLU, I.MODE_COVER), (I.FFN_RELU, I.MODE_IID)])
+def test_masked_twist_round_matches_the_oracle_round(B, kind, mode):
+    """Masked TwIST (Sec. 4.1) as a whole round: every worker a full-width copy under its activation mask; the
+    round is the same function as the gathered round the oracle computes."""
+    from paper_2511_03983_b200.engine import MaskedRoundEngine
+    w = replace(I.scaled_twin(I.PRESETS[5], d_model=136, d_ff=544, d_head=0, tokens=200, n_layers=2, local_steps=2),
+                n_subnets=4, ffn_kind=kind, sample_mode=mode, lr=0.05)
+    eng, before = _run_round_and_compare(B, w, engine_cls=MaskedRoundEngine, keep_f32_full=True)
+    assert eng.w_gu.shape[1] == eng.g * w.d_ff            # nothing is physically smaller
+
+
 def test_hybrid_twist_round_with_adam_matches_the_oracle_round(B):
     """Hybrid TwIST with the paper's optimiser: the central worker's moments are full-width and start at zero like
     the slices' moments; a masked neuron's zero gradient gives a zero Adam step."""
