@@ -589,6 +589,25 @@ class StackEngine(RoundEngine):
         self.launches += 2
         self.backward(k, lr)
 
+    def extract(self, rnd: int):
+        """Deployment (Sec. 4.2): sample blueprints as in training and gather every layer's dense slices; the S
+        extracted subnets are then resident (self.slices) for forward-only inference."""
+        self.sample_masks(rnd)
+        for l in range(self.w.n_layers):
+            self._bind(l)
+            self.gather_layer(l)
+
+    def evaluate(self, k: int) -> torch.Tensor:
+        """Evaluation mode for subnets (Sec. 4.2): forward only through the whole stack of every extracted subnet on
+        batch k with the subnets' own scales, no update.  An engine built with keep counts other than the training
+        run's evaluates a mismatched subnet ratio.  Returns the losses [S] (device); callers average over workers."""
+        w = self.w
+        self.forward(k)
+        B.twist_mse_fwd_bwd(self.x[w.n_layers], self.Td[k], self.grad[0], self.stack_loss[k], w.n_subnets, w.tokens,
+                            w.d_model, None, 0, 0, w.dtype, self.ws)
+        self.launches += 2
+        return self.stack_loss[k]
+
     def run_round(self, rnd: int):
         """Resample, gather every layer, K local steps through the whole stack, aggregate every layer."""
         w = self.w

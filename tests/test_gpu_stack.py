@@ -222,3 +222,41 @@ def test_rounds_are_bit_reproducible(B, mode):
     for m in a16:
         assert torch.equal(a16[m], b16[m]) and torch.equal(a32[m], b32[m]), m
     assert torch.equal(la, lb)
+
+
+@pytest.mark.parametrize("head_keep,ffn_ratio", [(16, 0.5), (24, 0.75)])
+def test_extracted_subnets_forward_only_at_any_ratio(B, head_keep, ffn_ratio):
+    """Sec. 4.2: subnets extracted with the sampler's procedure at a ratio that need not be the training one run
+    forward only through the whole chained stack with their own scales; losses match the oracle's stack forward."""
+    from paper_2511_03983_b200.engine import StackEngine
+    base = I.scaled_twin(I.PRESETS[3], d_model=256, d_ff=688, d_head=8, tokens=200, n_layers=2, local_steps=1)
+    w = replace(base, head_keep=head_keep, ffn_keep=int(base.n_ffn_blocks * ffn_ratio) // 8 * 8)
+    n_seqs, seq_len = 2, 100
+    eng = StackEngine(w, n_seqs, seq_len)
+    mats = {"gate": I.MAT_GATE, "up": I.MAT_UP, "down": I.MAT_DOWN, "qkv": I.MAT_QKV, "o": I.MAT_O}
+    full_np = []
+    for l in range(w.n_layers):
+        layer = {m: I.weight(w, l, mats[m]) for m in eng.full}
+        for m, v in layer.items():
+            eng.full[m][l].copy_(dev(v, torch.bfloat16))
+        full_np.append(layer)
+    X = np.stack([I.batch(w, I.BATCH_X, 0, s, 0, w.d_model) for s in range(w.n_subnets)])
+    Tg = np.stack([I.batch(w, I.BATCH_TGT_D, 0, s, 0, w.d_model) for s in range(w.n_subnets)])
+    eng.X.append(dev(X, torch.bfloat16))
+    eng.Td.append(dev(Tg, torch.bfloat16))
+    before = {m: v.clone() for m, v in eng.full.items()}
+    eng.extract(0)
+    got = eng.evaluate(0).cpu().numpy()
+    torch.cuda.synchronize()
+    assert B.twist_device_status() == 0
+    for m in before:                                      # inference leaves the model alone
+        assert torch.equal(before[m], eng.full[m])
+    for s in range(w.n_subnets):
+        bps = [o.layer_blueprints(w, 0, l) for l in range(w.n_layers)]
+        layers = [{m: v.astype(np.float64) for m, v in o.gather_layer(w, full_np[l], bps[l], s).items()}
+                  for l in range(w.n_layers)]
+        head_kv = [o.head_kv_positions(bps[l], w, s) for l in range(w.n_layers)]
+        out = o.stack_fwd(w, layers, head_kv, X[s].astype(np.float64), n_seqs, seq_len, True)
+        y = out[0] if isinstance(out, tuple) else out
+        want, _ = o.mse(y, Tg[s].astype(np.float64), True)
+        assert abs(got[s] - want) <= 2e-2 * want, (s, got[s], want)
