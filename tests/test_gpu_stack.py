@@ -49,6 +49,9 @@ def rel_fro(got, want):
     (1, 2, 640, 2, 64, None, 6.0),      # keys grow along the sequence: the row maxima keep rising, so the
                                         # lazily updated reference maximum has to move several times
     (1, 1, 100, 2, 32, None, 6.0),
+    (1, 2, 1, 1, 64, None, 0.0),        # tensor-core path, degenerate sizes: one token per sequence,
+    (1, 1, 127, 1, 64, None, 0.0),      # one block minus a row,
+    (2, 1, 129, 2, 64, None, 0.0),      # one block plus a row
 ])
 def test_attention_core_parity(B, S, n_seqs, N, H, dh, gqa, ramp):
     bf = torch.bfloat16
@@ -101,7 +104,10 @@ def test_attention_core_parity(B, S, n_seqs, N, H, dh, gqa, ramp):
         got = host(d_qkv[s])
         got_z = np.concatenate([got[:, :a], got[:, a:a + kc], got[:, a + kvw:a + kvw + kc]], axis=1)
         for name, cols in (("dq", slice(0, a)), ("dk", slice(a, a + kc)), ("dv", slice(a + kc, a + 2 * kc))):
-            assert rel_fro(got_z[:, cols], dZ[:, cols]) < GEMM_TOL, (name, s)
+            # a gradient that is exactly zero (one visible key: dS = P (dP - delta) = 0) is met up to the rounding of
+            # delta, so the error is measured against the larger of its norm and a sliver of the incoming gradient's
+            err = np.linalg.norm(got_z[:, cols] - dZ[:, cols])
+            assert err < GEMM_TOL * max(np.linalg.norm(dZ[:, cols]), 1e-3 * np.linalg.norm(dA[s])), (name, s)
         assert np.all(got[:, a + kc:a + kvw] == 0) and np.all(got[:, a + kvw + kc:] == 0)     # padding columns
         # log-sum-exp of the first position of every sequence: a single score
         for b in range(n_seqs):
