@@ -215,11 +215,14 @@ def workload_config(w, args):
                 "l2_policy": "working set exceeds L2 across the layers of a round",
                 "parallelism": "replicas only" if args.gpus > 1 else "single GPU"}
     hybrid = getattr(args, "mode", "blockwise") == "hybrid"
-    return {"workload": f"configs[{args.config - 1}] {w.name}: {'HYBRID ' if hybrid else ''}BLOCKWISE round, L={w.n_layers} d={w.d_model} "
+    masked = getattr(args, "mode", "blockwise") == "masked"
+    return {"workload": f"configs[{args.config - 1}] {w.name}: {'HYBRID ' if hybrid else 'MASKED ' if masked else ''}BLOCKWISE round, L={w.n_layers} d={w.d_model} "
                         f"F={w.d_ff} f'={w.f_sub} H'={w.head_keep}/{w.n_heads} S={w.n_subnets} T={w.tokens} K={w.local_steps}",
             "tokens_per_round": w.tokens_per_round,
             "mode": ("hybrid: worker 0 masked on the full-width model in place, the others on gathered slices; flops "
-                     "counted are those of the gathered subnets" if hybrid else "blockwise, layers streamed"),
+                     "counted are those of the gathered subnets" if hybrid else
+                     "masked: every worker a full-width copy under its activation mask; flops counted are those of the "
+                     "gathered subnets" if masked else "blockwise, layers streamed"),
             "l2_policy": "inputs larger than L2 (every tensor a kernel reads is >= 4x the 126 MB L2)"
                          if w.d_model >= 2048 else "working set exceeds L2 across the layers of a round",
             "parallelism": "replicas only" if args.gpus > 1 else "single GPU"}
@@ -235,7 +238,7 @@ def run_ours(args, w):
 
     from paper_2511_03983_b200 import binding as B
     from paper_2511_03983_b200 import inputs as I
-    from paper_2511_03983_b200.engine import HybridRoundEngine, RoundEngine, StackEngine
+    from paper_2511_03983_b200.engine import HybridRoundEngine, MaskedRoundEngine, RoundEngine, StackEngine
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -253,10 +256,13 @@ def run_ours(args, w):
         if not (w.n_heads and bf16 and w.tokens % w.n_seqs == 0):
             raise SystemExit("--mode stack needs a bf16 workload with attention heads")
         eng = StackEngine(w, w.n_seqs, w.tokens // w.n_seqs, keep_f32_full=True)
-    elif args.mode == "hybrid":
+    elif args.mode in ("hybrid", "masked"):
         if w.n_heads or not bf16:
-            raise SystemExit("--mode hybrid needs a bf16 FFN-only workload (--config 5)")
-        eng = HybridRoundEngine(w, compute_dx=True, fuse_loss=True, store_outputs=False)
+            raise SystemExit(f"--mode {args.mode} needs a bf16 FFN-only workload (--config 5)")
+        if args.mode == "hybrid":
+            eng = HybridRoundEngine(w, compute_dx=True, fuse_loss=True, store_outputs=False)
+        else:
+            eng = MaskedRoundEngine(w, keep_f32_full=True, compute_dx=True, fuse_loss=True, store_outputs=False)
     else:
         eng = RoundEngine(w, keep_f32_full=True, compute_dx=True, fuse_loss=True, store_outputs=False)
     gen = torch.Generator(device="cuda")
@@ -377,6 +383,9 @@ def run_ours(args, w):
     work = round_work(w)
     if args.mode == "hybrid":                             # worker 0 has no slice: S - 1 subnets are gathered
         work["gather_bytes"] *= (w.n_subnets - 1) / w.n_subnets
+    if args.mode == "masked":                             # every worker copies and returns the whole layer
+        full_over_kept = w.n_ffn_blocks / w.ffn_keep
+        work["gather_bytes"] *= full_over_kept            # (the aggregate reads the same rows as in the gathered round)
     gemm_names = [n for n in ("ffn_fwd", "ffn_bwd", "qkv_fwd", "qkv_bwd", "o_fwd", "o_bwd") if n in phases]
     gemm_ms = sum(phases[n][0] for n in gemm_names)
     gemm_launches_per_round = w.n_layers * K * ((2 + 4) + ((1 + 2 + 1 + 2) if eng.has_attn else 0))
@@ -501,9 +510,9 @@ def main():
     ap.add_argument("--layers", type=int, default=0, help="override the layer count (profiling on a small case)")
     ap.add_argument("--tokens", type=int, default=0, help="override tokens per subnet-step (profiling on a small case)")
     ap.add_argument("--local-steps", type=int, default=0)
-    ap.add_argument("--mode", default="blockwise", choices=["blockwise", "stack", "hybrid"],
+    ap.add_argument("--mode", default="blockwise", choices=["blockwise", "stack", "hybrid", "masked"],
                     help="stack: chained layers with the attention core (workloads 2 and 3); hybrid: worker 0 trains "
-                         "the full-width model under a mask (FFN-only workload 5)")
+                         "the full-width model under a mask; masked: every worker does (FFN-only workload 5)")
     ap.add_argument("--sweep", action="store_true", help="workload 5: all 12 (S, keep) cells, gather / aggregate GB/s")
     args = ap.parse_args()
     from dataclasses import replace
