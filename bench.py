@@ -402,7 +402,11 @@ def run_ours(args, w):
         peak = peaks[peak_key]
         roofline = {"bound": "tensor", "kernel": "gemm_kernel (grouped tcgen05 GEMM, all layouts/epilogues)",
                     "achieved": tflops, "peak": peak, "unit": "TFLOP/s", "frac": tflops / peak,
-                    "peak_source": f"{peak_key} of {peaks['source']}", "traffic": None,
+                    "peak_source": f"{peak_key} of {peaks['source']}",
+                    # dram read + write bytes per launch, averaged over the launches of a layer-step, from the
+                    # single-pass ncu capture at this exact size (profiles/gemm_kernel_cfg4_full_size_dram.txt);
+                    # any other workload has no capture
+                    "traffic": 13.3e9 if (args.config == 4 and not args.tokens and args.mode == "blockwise") else None,
                     "flops_per_launch": work["gemm_flops"] / gemm_launches_per_round,
                     "avg_launch_ms": gemm_ms / args.steps / gemm_launches_per_round,
                     "share_of_step": gemm_ms / ms_total}
