@@ -406,7 +406,7 @@ def run_ours(args, w):
                     # dram read + write bytes per launch, averaged over the launches of a layer-step, from the
                     # single-pass ncu capture at this exact size (profiles/gemm_kernel_cfg4_full_size_dram.txt);
                     # any other workload has no capture
-                    "traffic": 13.3e9 if (args.config == 4 and not args.tokens and args.mode == "blockwise") else None,
+                    "traffic": 12.5e9 if (args.config == 4 and not args.tokens and args.mode == "blockwise") else None,
                     "flops_per_launch": work["gemm_flops"] / gemm_launches_per_round,
                     "avg_launch_ms": gemm_ms / args.steps / gemm_launches_per_round,
                     "share_of_step": gemm_ms / ms_total}

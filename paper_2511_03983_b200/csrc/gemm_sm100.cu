@@ -195,6 +195,7 @@ int launch_gemm_bf16(int layout, int epi, const GemmOperand& A, const GemmOperan
   p.m_tiles = (p.M + kBM - 1) / kBM;
   p.n_tiles = epi == EPI_SWIGLU_FWD ? (p.N + kCtaN - 1) / kCtaN : (p.N + kBN - 1) / kBN;
   if ((long long)p.groups * p.m_tiles * p.n_tiles > 0x7fffffffLL) return TWIST_ERR_UNSUPPORTED;
+  p.raster_m = layout == 2 ? 8 : 1;      // see tile_coords
   p.status = device_status_ptr();
   if (!p.status) return TWIST_ERR_CUDA;
   CUtensorMap ta, tb;

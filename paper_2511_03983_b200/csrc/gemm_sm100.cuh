@@ -59,12 +59,12 @@ __host__ __device__ constexpr int gemm_smem_bytes(bool staged_epilogue) {
   return gemm_stages(staged_epilogue) * kStageBytes + (staged_epilogue ? kEpiBytes : 0) + 1024 /*alignment slack*/ + kCtrlBytes;
 }
 constexpr int kTmemCols = 512;                    // two 128 x 256 fp32 accumulators per CTA
-constexpr int kRasterGroupM = 8;                  // m-tiles per raster group (L2 reuse of A and B tiles)
 
 struct GemmParams {
   int M, N, K;          // per group.  EPI_SWIGLU_FWD: N = f_sub (neurons); the tile holds 128 gate + 128 up columns
   int groups;
   int m_tiles, n_tiles;
+  int raster_m;         // m-tiles per raster band (set by the launcher from the operand layout)
   int b_split;          // EPI_SWIGLU_FWD: row of the first "up" weight inside B (= f_sub)
   int act_kind;         // TWIST_FFN_*
   float scale, lr;
@@ -246,17 +246,23 @@ __device__ inline void act_grad8(const float (&x)[8], int kind, float (&g)[8]) {
   for (int i = 0; i < 8; ++i) g[i] = cdf[i] + pdf_x[i];
 }
 
-// Tile index -> (group, m_tile, n_tile): groups outermost; inside a group, raster groups of
-// kRasterGroupM m-tiles, n-tiles next, m-tiles innermost, so that concurrently running CTAs share
-// a small set of A and B tiles in L2.
+// Tile index -> (group, m_tile, n_tile): groups outermost; inside a group, bands of raster_m m-tiles, n-tiles
+// next, m-tiles innermost.  The 74 tiles in flight stream their operands through L2 together, so what a wave reads
+// from DRAM is one copy of the A rows and B columns it spans, plus whatever of them did not stay in L2 since the
+// last wave.  Measured on the 7B-shaped launches (DRAM bytes read per layer-step, round time):
+//   token-major launches (M = tokens, B = a weight slice): raster_m = 1, i.e. a wave is "a few m-tiles x every
+//     n-tile" - A streams through once, B is shared by the whole wave; bands of 8 read 25 % more, panels of 4 - 12
+//     n-tiles 10 - 100 % more;
+//   weight-gradient launches (both operands activations streamed along a long contraction): the squarest wave,
+//     bands of 8 m-tiles (8 x 9 tiles), reads least.
 __device__ inline void tile_coords(const GemmParams& p, int tile, int& g, int& mt, int& nt) {
   const int per_group = p.m_tiles * p.n_tiles;
   g = tile / per_group;
   const int r = tile - g * per_group;
-  const int band = r / (kRasterGroupM * p.n_tiles);
-  const int m_first = band * kRasterGroupM;
-  const int band_h = min(kRasterGroupM, p.m_tiles - m_first);
-  const int rr = r - band * kRasterGroupM * p.n_tiles;
+  const int band = r / (p.raster_m * p.n_tiles);
+  const int m_first = band * p.raster_m;
+  const int band_h = min(p.raster_m, p.m_tiles - m_first);
+  const int rr = r - band * p.raster_m * p.n_tiles;
   nt = rr / band_h;
   mt = m_first + (rr - nt * band_h);
 }
