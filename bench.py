@@ -25,6 +25,10 @@ if ROOT not in sys.path:
 
 METRIC = "twist_round_tokens_per_s"
 UNIT = "tokens/s"
+# Nominal peaks of the part (dense bf16 tensor throughput, HBM3e bandwidth); fractions against them are reported
+# beside the fractions against the peaks measured on the machine.
+NOMINAL_BF16_TFLOPS = 2250.0
+NOMINAL_HBM_GBS = 8000.0
 
 
 def measured_peaks():
@@ -403,6 +407,11 @@ def run_ours(args, w):
         roofline = {"bound": "tensor", "kernel": "gemm_kernel (grouped tcgen05 GEMM, all layouts/epilogues)",
                     "achieved": tflops, "peak": peak, "unit": "TFLOP/s", "frac": tflops / peak,
                     "peak_source": f"{peak_key} of {peaks['source']}",
+                    "frac_of_nominal": tflops / NOMINAL_BF16_TFLOPS, "nominal_peak": NOMINAL_BF16_TFLOPS,
+                    # what the same kernels would give at the maximum SM clock, if throughput followed the clock
+                    # (the step runs under the power cap): achieved x max MHz / median MHz
+                    "achieved_at_max_clock": (tflops * clocks["sm_max_mhz"] / clocks["sm_mhz"]
+                                              if clocks and clocks.get("sm_mhz") and clocks.get("sm_max_mhz") else None),
                     # dram read + write bytes per launch, averaged over the launches of a layer-step, from the
                     # single-pass ncu capture at this exact size (profiles/gemm_kernel_cfg4_full_size_dram.txt);
                     # any other workload has no capture
@@ -417,7 +426,8 @@ def run_ours(args, w):
         if name in phases and phases[name][0] > 0:
             gbs = work[key] * args.steps / (phases[name][0] / 1e3) / 1e9
             hbm[name] = {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                         "frac": gbs / peaks["hbm_gbs"], "bytes_per_launch": work[key] / w.n_layers,
+                         "frac": gbs / peaks["hbm_gbs"], "frac_of_nominal": gbs / NOMINAL_HBM_GBS,
+                         "nominal_peak": NOMINAL_HBM_GBS, "bytes_per_launch": work[key] / w.n_layers,
                          "traffic": ncu_traffic.get(name)}
     if roofline is None and "aggregate" in hbm:
         roofline = dict(hbm["aggregate"], kernel="aggregate_rows_kernel")

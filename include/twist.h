@@ -14,10 +14,11 @@
  *    (a cudaStream_t passed as void*; NULL is the default stream).
  *  - "device" pointers are CUDA device memory owned by the caller; they must stay
  *    valid until the stream has run the call.  "host" pointers are read during the
- *    call only.  Base pointers must be 16-byte aligned.
+ *    call only.  Base pointers must be 16-byte aligned (byte masks: 8-byte); a misaligned
+ *    pointer returns TWIST_ERR_SHAPE, it is never dereferenced.
  *  - Storage layout: every partitioned matrix is row-major with one row per hidden
- *    neuron / head dimension and d_model contiguous ("a block is a chunk of
- *    parameters in memory", Sec. 3.1):
+ *    neuron / head dimension and d_model contiguous, so that a block -- a run of whole rows --
+ *    is one contiguous piece of memory (block definition of Sec. 3.1):
  *        W_gate, W_up, W_down : [F, d];  W_qkv : [(H + 2 H_kv) d_head, d];  W_o : [H d_head, d].
  *    up/gate/qkv rows are output features (y = x W^T), down/o rows are input features (y = h W).
  *    Slices and activations of the S subnets are packed [S][rows][cols], dense.
@@ -65,9 +66,16 @@ uint32_t twist_abi_version(void);
 const char* twist_strerror(int32_t status);
 /* Text of the last CUDA error this library saw on the calling thread ("" if none). */
 const char* twist_last_cuda_error(void);
-/* Reads (and clears) the device status word.  Synchronises the device.  *code is TWIST_OK or
- * TWIST_ERR_DEVICE_TIMEOUT. */
+/* Reads (and clears) the device status word.  Synchronises the device.  *code is TWIST_OK,
+ * TWIST_ERR_DEVICE_TIMEOUT (a bounded wait of a kernel ran out) or TWIST_ERR_BAD_INDEX (a kernel met an
+ * index entry outside its range and skipped it); the time-out wins when both happened. */
 int32_t twist_device_status(int32_t* code);
+/* Self-test of the give-up path of the kernels' bounded waits (the paper has no counterpart; for tests and
+ * bring-up).  Launches one CTA pair with the roles, barriers and exit sequence of the GEMM kernel whose
+ * barriers nobody arrives at; every wait gives up after limit_ns (1 .. 100 000 000) of wall time, the pair
+ * drains, frees its tensor memory and returns.  Afterwards twist_device_status reports
+ * TWIST_ERR_DEVICE_TIMEOUT once, and the device stays usable. */
+int32_t twist_selftest_wait(uint64_t limit_ns, void* stream);
 
 /* ---------------------------------------------------------------------------------------------
  * twist_sample_masks -- subnet generator, Algorithm 1 ("Generate Training Subnet Blueprint").
@@ -95,17 +103,17 @@ int32_t twist_sample_masks(uint64_t seed, uint64_t round, int32_t layer_begin, i
                            const int32_t* common, int32_t n_common, int32_t sample_mode,
                            int32_t* idx, uint32_t* cover, int32_t* pos, void* stream);
 
-/* KV groups under grouped-query attention (an extension; the paper's attention is plain
- * multi-head, App. A): group g = h / (n_heads / n_kv_heads) is held by subnet s iff one of its
- * query heads is.  Writes kv_idx [n_layers][S][n_kv_heads] (sorted kept groups, then -1),
- * kv_count [n_layers][S], kv_cols [n_layers][S] = kv_count * d_head (valid K or V columns of the
- * subnet's projection), kv_cover [n_layers][n_kv_heads], kv_pos [n_layers][S][n_kv_heads]; all device. */
 /* Activation masks of Masked / Hybrid TwIST (Sec. 4.1) from the aggregator's cover masks: for the subnets
  * subnet_begin .. subnet_begin + n_subnets - 1,  mask[s][b*block_rows + i] = 1 if subnet s holds block b, else 0.
  *   cover [n_full] device uint32 (one layer);  mask [n_subnets][n_full*block_rows] device uint8: out. */
 int32_t twist_hidden_mask(const uint32_t* cover /*device*/, int32_t n_full, int32_t block_rows, int32_t subnet_begin,
                           int32_t n_subnets, uint8_t* mask /*device*/, void* stream);
 
+/* KV groups under grouped-query attention (an extension; the paper's attention is plain
+ * multi-head, App. A): group g = h / (n_heads / n_kv_heads) is held by subnet s iff one of its
+ * query heads is.  Writes kv_idx [n_layers][S][n_kv_heads] (sorted kept groups, then -1),
+ * kv_count [n_layers][S], kv_cols [n_layers][S] = kv_count * d_head (valid K or V columns of the
+ * subnet's projection), kv_cover [n_layers][n_kv_heads], kv_pos [n_layers][S][n_kv_heads]; all device. */
 int32_t twist_kv_groups(const int32_t* head_idx, int32_t n_layers, int32_t n_subnets, int32_t head_keep,
                         int32_t n_heads, int32_t n_kv_heads, int32_t d_head, int32_t* kv_idx, int32_t* kv_count,
                         int32_t* kv_cols, uint32_t* kv_cover, int32_t* kv_pos, void* stream);
@@ -121,6 +129,9 @@ int32_t twist_kv_groups(const int32_t* head_idx, int32_t n_layers, int32_t n_sub
  *       = src[(src_row_offset + idx[s*idx_stride + j]*block_rows + i)*d + :]
  * (bit copy); the same values widened to fp32 go to dst_master when it is not NULL.  Entries
  * j >= count[s] (count may be NULL = all valid) are written as zeros (padding of ragged KV rows).
+ * Index data is checked on the device: a valid entry idx[..] outside [0, n_blocks) is not followed -- its
+ * destination rows are left untouched and TWIST_ERR_BAD_INDEX is recorded in the device status word
+ * (twist_device_status); the other rows are gathered as usual.
  */
 #define TWIST_MAX_SEGMENTS 8
 typedef struct {
@@ -132,7 +143,7 @@ typedef struct {
   int32_t idx_stride;
   int32_t n_keep;             /* entries written per subnet */
   int32_t block_rows;         /* rows per block */
-  int32_t reserved;
+  int32_t n_blocks;           /* blocks in the partitioned range of src: every idx entry must lie in [0, n_blocks) */
   int64_t src_row_offset;     /* first row of the partitioned range inside src */
   int64_t dst_subnet_stride;  /* elements between consecutive subnets in dst / dst_master */
   int64_t dst_row_offset;     /* first destination row inside a subnet's slice */
@@ -152,6 +163,9 @@ int32_t twist_gather_subnets(const twist_gather_segment* segs /*host*/, int32_t 
  * order, no atomics: results are deterministic.
  *   src (subnet s, block b at rank pos[s][b]) row i:
  *       sub[s*sub_subnet_stride + (sub_row_offset + pos[s*n_full + b]*block_rows + i)*d + :]
+ * Index data is checked on the device: when cover says subnet s holds block b but pos[s][b] is outside
+ * [0, n_keep), the block's rows are left untouched and TWIST_ERR_BAD_INDEX is recorded in the device
+ * status word; the other rows are aggregated as usual.
  */
 typedef struct {
   void* dst;                  /* device, full matrix in `dtype` (bf16: rounded shadow; fp32: the result) */
@@ -170,6 +184,7 @@ typedef struct {
    * before it is written, by the same thread).  NULL: every subnet is read from `sub`. */
   const float* central;
   int32_t central_subnet;
+  int32_t n_keep;             /* blocks of this segment in a subnet's slice: pos of a held block must lie in [0, n_keep) */
 } twist_aggregate_segment;
 
 int32_t twist_aggregate(const twist_aggregate_segment* segs /*host*/, int32_t n_segs, int32_t n_subnets,
@@ -346,7 +361,9 @@ int32_t twist_mse_fwd_bwd(const void* y, const void* tgt, void* dy, float* loss,
  *  - n_subnets > TWIST_NOALLOC_MAX_SUBNETS returns TWIST_ERR_UNSUPPORTED; nothing is launched.
  *  - No cudaMalloc, cudaFree or other allocating call is made, here or in a library on its behalf.
  *  - The first call on each device looks up the array's device address (once per device, with that
- *    device current).  Make that first call outside any stream capture.
+ *    device current).  Make that first call outside any stream capture.  The address is remembered for
+ *    as long as the device's primary context lives; a process that destroys that context
+ *    (cudaDeviceReset) must not call this entry point on the device again.
  *  - All calls share the one array, which keeps whatever the previous call left in it.  Nothing in it
  *    has to start at zero: each call overwrites every partial sum it later reads.  Two calls that
  *    overlap on the GPU (different streams, or different host threads without ordering) race on the

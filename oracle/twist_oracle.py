@@ -14,7 +14,7 @@ algorithm's steps in the paper's order and notation.
 Storage convention (a choice of this implementation, the paper fixes only mathematical
 shapes in its Problem formulation): every partitioned matrix is stored with one
 row per neuron / head-dimension and d_model contiguous, so a block is a run of
-whole rows ("a block is a chunk of parameters in memory", Sec. 3.1):
+whole rows, contiguous in memory (block definition of Sec. 3.1):
     W_up, W_gate : [F, d]   (paper's W^ffn,  rows = hidden neurons)
     W_down       : [F, d]   (paper's C^ffn transposed, rows = hidden neurons)
     W_qkv        : [(H + 2 H_kv) d_head, d]  (transposed W^Q_h | W^K_h | W^V_h, head after head)
@@ -44,8 +44,8 @@ _M2 = _U64(0x94D049BB133111EB)
 
 # ----------------------------------------------------------------------------------------
 # Counter-based integer hash used for every random draw of the sampler.
-# The paper leaves the generator open (Algorithm 1 calls it "unique_choice" and
-# Sec. 3.1 says "uniformly at random"); this implementation fixes a 64-bit avalanche
+# The paper leaves the generator open (Algorithm 1 only names a routine that draws distinct
+# blocks, and Sec. 3.1 asks for a uniform draw); this implementation fixes a 64-bit avalanche
 # mixer (the published splitmix64 finaliser) applied to the counter tuple.
 # ----------------------------------------------------------------------------------------
 

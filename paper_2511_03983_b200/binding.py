@@ -31,7 +31,7 @@ EXPORTS = [
     "twist_kv_groups", "twist_gather_subnets", "twist_aggregate", "twist_subnet_ffn_fwd", "twist_subnet_ffn_bwd",
     "twist_subnet_attn_proj_fwd", "twist_subnet_attn_proj_bwd", "twist_mse_workspace_bytes", "twist_mse_fwd_bwd",
     "twist_mse_fwd_bwd_noalloc", "twist_fused_loss_workspace_bytes", "twist_attn_core_fwd", "twist_attn_core_bwd",
-    "twist_hidden_mask",
+    "twist_hidden_mask", "twist_selftest_wait",
 ]
 
 
@@ -44,7 +44,7 @@ class TwistError(RuntimeError):
 class GatherSegment(C.Structure):
     _fields_ = [("src", C.c_void_p), ("dst", C.c_void_p), ("dst_master", C.c_void_p), ("idx", C.c_void_p),
                 ("count", C.c_void_p), ("idx_stride", C.c_int32), ("n_keep", C.c_int32), ("block_rows", C.c_int32),
-                ("reserved", C.c_int32), ("src_row_offset", C.c_int64), ("dst_subnet_stride", C.c_int64),
+                ("n_blocks", C.c_int32), ("src_row_offset", C.c_int64), ("dst_subnet_stride", C.c_int64),
                 ("dst_row_offset", C.c_int64)]
 
 
@@ -52,7 +52,7 @@ class AggregateSegment(C.Structure):
     _fields_ = [("dst", C.c_void_p), ("dst_f32", C.c_void_p), ("sub", C.c_void_p), ("cover", C.c_void_p),
                 ("pos", C.c_void_p), ("n_full", C.c_int32), ("block_rows", C.c_int32), ("dst_row_offset", C.c_int64),
                 ("sub_subnet_stride", C.c_int64), ("sub_row_offset", C.c_int64), ("central", C.c_void_p),
-                ("central_subnet", C.c_int32)]
+                ("central_subnet", C.c_int32), ("n_keep", C.c_int32)]
 
 
 class Optimizer(C.Structure):
@@ -113,6 +113,7 @@ def lib() -> C.CDLL:
         h.twist_strerror.argtypes = [C.c_int32]
         h.twist_last_cuda_error.restype = C.c_char_p
         h.twist_device_status.argtypes = [C.POINTER(C.c_int32)]
+        h.twist_selftest_wait.argtypes = [C.c_uint64, C.c_void_p]
         h.twist_sample_masks.argtypes = [C.c_uint64, C.c_uint64, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int32,
                                          C.c_int32, C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p,
                                          C.c_void_p, C.c_void_p]
@@ -172,6 +173,12 @@ def twist_device_status() -> int:
     return code.value
 
 
+def twist_selftest_wait(limit_ns: int):
+    """Runs the library's bounded waits on barriers nobody arrives at (test / bring-up only); afterwards
+    twist_device_status() reports ERR_DEVICE_TIMEOUT once."""
+    _check(lib().twist_selftest_wait(limit_ns, _stream()), "twist_selftest_wait")
+
+
 def twist_sample_masks(seed, rnd, layer_begin, n_layers, kind, n_full, n_subnets, n_sub, common: Sequence[int],
                        sample_mode, idx, cover, pos):
     arr = (C.c_int32 * max(1, len(common)))(*common)
@@ -188,10 +195,11 @@ def twist_kv_groups(head_idx, n_layers, n_subnets, head_keep, n_heads, n_kv_head
 
 
 def gather_segment(src, dst, dst_master, idx, count, idx_stride, n_keep, block_rows, src_row_offset,
-                   dst_subnet_stride, dst_row_offset) -> GatherSegment:
-    """Marshals one twist_gather_segment.  src/dst/... may be tensors or raw device addresses (ints)."""
+                   dst_subnet_stride, dst_row_offset, n_blocks) -> GatherSegment:
+    """Marshals one twist_gather_segment.  src/dst/... may be tensors or raw device addresses (ints).
+    n_blocks: blocks in the partitioned range of src (the range idx entries are checked against)."""
     a = lambda v: v if (v is None or isinstance(v, int)) else _ptr(v)
-    return GatherSegment(a(src), a(dst), a(dst_master), a(idx), a(count), idx_stride, n_keep, block_rows, 0,
+    return GatherSegment(a(src), a(dst), a(dst_master), a(idx), a(count), idx_stride, n_keep, block_rows, n_blocks,
                          src_row_offset, dst_subnet_stride, dst_row_offset)
 
 
@@ -202,10 +210,12 @@ def twist_gather_subnets(segs: Sequence[GatherSegment], n_subnets, d, dtype):
 
 
 def aggregate_segment(dst, dst_f32, sub, cover, pos, n_full, block_rows, dst_row_offset, sub_subnet_stride,
-                      sub_row_offset, central=None, central_subnet=0) -> AggregateSegment:
+                      sub_row_offset, n_keep, central=None, central_subnet=0) -> AggregateSegment:
+    """Marshals one twist_aggregate_segment.  n_keep: blocks of the segment in a subnet's slice (the range the
+    ranks in pos are checked against)."""
     a = lambda v: v if (v is None or isinstance(v, int)) else _ptr(v)
     return AggregateSegment(a(dst), a(dst_f32), a(sub), a(cover), a(pos), n_full, block_rows, dst_row_offset,
-                            sub_subnet_stride, sub_row_offset, a(central), central_subnet)
+                            sub_subnet_stride, sub_row_offset, a(central), central_subnet, n_keep)
 
 
 def twist_hidden_mask(cover, n_full, block_rows, subnet_begin, n_subnets, mask):

@@ -26,12 +26,6 @@ __device__ inline uint32_t pack2(float lo, float hi) {
   return *reinterpret_cast<uint32_t*>(&t);
 }
 
-__device__ inline int kv_position(const AttnParams& p, int s, int hq) {
-  if (!p.head_idx) return hq;
-  const int g = p.head_idx[(long long)s * p.heads + hq] / p.per_group;
-  return p.kv_pos[(long long)s * p.n_kv_heads + g];
-}
-
 // Loads DPT bf16 values (a thread's part of a row) from global memory as floats; zeros when !ok.
 template <int DPT>
 __device__ inline void load_part(const __nv_bfloat16* src, float (&v)[DPT], bool ok) {
@@ -322,6 +316,7 @@ AttnParams make_params(const twist_attn_core_args* a) {
   p.nq = p.a_sub + 2 * a->kv_max * a->d_head;
   p.T = a->n_seqs * a->seq_len;
   p.scale_log2 = kLog2e / sqrtf((float)a->d_head);
+  p.status = device_status_ptr();
   return p;
 }
 
@@ -347,6 +342,7 @@ int run(const AttnParams& p, int n_subnets, bool backward, cudaStream_t st) {
 }
 
 int dispatch(const AttnParams& p, int n_subnets, bool backward, cudaStream_t st) {
+  if (!p.status) return TWIST_ERR_CUDA;
   switch (p.d_head) {
     case 8: return run<8, 1>(p, n_subnets, backward, st);
     case 16: return run<16, 1>(p, n_subnets, backward, st);

@@ -18,7 +18,20 @@ struct AttnParams {
   int n_seqs, seq_len, heads, kv_max, d_head, per_group, n_kv_heads;
   int a_sub, nq, T;
   float scale_log2;           // log2(e) / sqrt(d_head)
+  int* status;                // device status word
 };
+
+// KV position (among the subnet's kept groups) that kept head hq of subnet s reads.  The two index arrays are
+// checked on the way: an entry outside its range is replaced by 0 (so that nothing is read or written out of
+// bounds) and TWIST_ERR_BAD_INDEX is recorded in the status word.
+__device__ inline int kv_position(const AttnParams& p, int s, int hq) {
+  if (!p.head_idx) return hq;
+  int g = p.head_idx[(long long)s * p.heads + hq] / p.per_group;
+  if ((unsigned)g >= (unsigned)p.n_kv_heads) { atomicMin(p.status, (int)TWIST_ERR_BAD_INDEX); g = 0; }
+  int pos = p.kv_pos[(long long)s * p.n_kv_heads + g];
+  if ((unsigned)pos >= (unsigned)p.kv_max) { atomicMin(p.status, (int)TWIST_ERR_BAD_INDEX); pos = 0; }
+  return pos;
+}
 
 
 // Tensor-core kernels (d_head = 64), defined in attn_core_tc.cu.  The backward expects delta to be filled.

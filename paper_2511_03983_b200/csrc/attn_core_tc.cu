@@ -158,12 +158,6 @@ __device__ inline void store_acc32(__nv_bfloat16* dst, const uint32_t (&v)[32], 
                        pack2(sc * __uint_as_float(v[8 * q4 + 6]), sc * __uint_as_float(v[8 * q4 + 7])));
 }
 
-__device__ inline int kv_position(const AttnParams& p, int s, int hq) {
-  if (!p.head_idx) return hq;
-  const int g = p.head_idx[(long long)s * p.heads + hq] / p.per_group;
-  return p.kv_pos[(long long)s * p.n_kv_heads + g];
-}
-
 // qkv viewed as [S * n_seqs][seq_len][nq]: rows past the end of a sequence read as zeros.
 __global__ void __maxnreg__(200) attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQKV,
                                                                      const AttnParams p, int* status) {

@@ -99,12 +99,14 @@ __global__ void __launch_bounds__(kGatherWarps * 32) gather_rows_kernel(const __
   struct Item {
     const char* src_base;   // null: a padding row, written as zeros
     long long src_row;      // row of the source piece before the block index is applied
-    int block_rows, idxv, off;
+    int block_rows, idxv, n_blocks, off;
     char* dst; char* mst; int bytes;
   };
+  // A kept-block id outside the source's block range: the row is neither read nor written, the status word says so.
+  auto bad_index = [](const Item& o) { return o.src_base && (unsigned)o.idxv >= (unsigned)o.n_blocks; };
   auto decode = [&](long long it) {
     Item o;
-    o.src_base = nullptr; o.src_row = 0; o.block_rows = 0; o.idxv = 0; o.off = 0; o.dst = nullptr; o.mst = nullptr; o.bytes = 0;
+    o.src_base = nullptr; o.src_row = 0; o.block_rows = 0; o.idxv = 0; o.n_blocks = 0; o.off = 0; o.dst = nullptr; o.mst = nullptr; o.bytes = 0;
     if (it >= items) return o;
     const long long r = it / pieces;
     const int pc = (int)(it - r * pieces);
@@ -126,12 +128,13 @@ __global__ void __launch_bounds__(kGatherWarps * 32) gather_rows_kernel(const __
       o.src_base = static_cast<const char*>(sg.src);
       o.src_row = sg.src_row_offset + i;
       o.block_rows = sg.block_rows;
+      o.n_blocks = sg.n_blocks;
       asm volatile("ld.global.nc.s32 %0, [%1];" : "=r"(o.idxv) : "l"(sg.idx + (long long)s * sg.idx_stride + j));
     }
     return o;
   };
   auto request = [&](const Item& o, int b) {          // lane 0
-    if (!o.src_base) return;
+    if (!o.src_base || bad_index(o)) return;
     const uint32_t bar = smem_u32(&bars[warp][b]);
     const char* src = o.src_base + (o.src_row + (long long)o.idxv * o.block_rows) * row_bytes + o.off;
     mbar_expect_tx(bar, (uint32_t)o.bytes);
@@ -156,7 +159,9 @@ __global__ void __launch_bounds__(kGatherWarps * 32) gather_rows_kernel(const __
     }
     const Item cur = q[0];
     const uint32_t in = wbase + (uint32_t)b * buf_bytes;
-    if (cur.src_base) {
+    if (bad_index(cur)) {                              // skipped: destination row left as it was
+      if (lane == 0) note_status(status, (int)TWIST_ERR_BAD_INDEX);
+    } else if (cur.src_base) {
       const uint32_t parity = (phase >> b) & 1u;
       // warp-uniform outcome: either every lane goes on or every lane leaves
       if (!__all_sync(0xffffffffu, mbar_wait(smem_u32(&bars[warp][b]), parity, &abort_flag, status))) break;
@@ -192,10 +197,7 @@ __global__ void __launch_bounds__(kGatherWarps * 32) gather_rows_kernel(const __
   }
   if (lane == 0) bulk_wait_read<0>();
   __syncthreads();
-  if (abort_flag) {     // a wait expired: let a copy that may still be in flight land before shared memory is released
-    const uint64_t t0 = global_timer_ns();
-    while (global_timer_ns() - t0 < 2000000ull) __nanosleep(1000);
-  }
+  drain_after_abort(&abort_flag);     // a wait expired: a copy may still be in flight towards shared memory
 }
 
 __device__ inline uint32_t pack_bf16x2_rn(float lo, float hi) {
@@ -207,7 +209,7 @@ __device__ inline uint32_t pack_bf16x2_rn(float lo, float hi) {
 // covering subnets in ascending order, correctly rounded quotient.  (A bulk-copy version of this kernel, like the
 // gather's, measured slower: 2 KB pieces keep too few bytes in flight per SM.)
 template <bool BF16>
-__global__ void __launch_bounds__(256) aggregate_rows_kernel(const __grid_constant__ AggParams p) {
+__global__ void __launch_bounds__(256) aggregate_rows_kernel(const __grid_constant__ AggParams p, int* status) {
   const int lane = threadIdx.x & 31;
   const long long warp0 = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   const long long nwarps = ((long long)gridDim.x * blockDim.x) >> 5;
@@ -229,14 +231,21 @@ __global__ void __launch_bounds__(256) aggregate_rows_kernel(const __grid_consta
     // (it may be the destination, so it is read with an ordinary load, not through the read-only path)
     unsigned long long mine = 0;
     const long long drow = sg.dst_row_offset + rl;
+    bool bad = false;
     if (lane < cnt) {
       const int s = __fns(m, 0, lane + 1);
       if (sg.central && s == sg.central_subnet) {        // trained in place on the full-width matrix
         mine = reinterpret_cast<unsigned long long>(sg.central + drow * p.d) | 1ull;
       } else {
-        const long long srow = sg.sub_row_offset + (long long)sg.pos[(long long)s * sg.n_full + b] * sg.block_rows + i;
+        const int rank = sg.pos[(long long)s * sg.n_full + b];
+        bad = (unsigned)rank >= (unsigned)sg.n_keep;     // not a row of the subnet's slice
+        const long long srow = sg.sub_row_offset + (long long)rank * sg.block_rows + i;
         mine = reinterpret_cast<unsigned long long>(sg.sub + (long long)s * sg.sub_subnet_stride + srow * p.d);
       }
+    }
+    if (__any_sync(0xffffffffu, bad)) {                  // row left as it was, the status word says so
+      if (lane == 0) note_status(status, (int)TWIST_ERR_BAD_INDEX);
+      continue;
     }
     // Quotient by the coverage count: reciprocal product corrected with the exact remainder, which gives
     // the correctly rounded quotient (the same bits as an IEEE division) at a fraction of its cost.
@@ -315,7 +324,7 @@ extern "C" int32_t twist_gather_subnets(const twist_gather_segment* segs, int32_
   for (int g = 0; g < n_segs; ++g) {
     const twist_gather_segment& s = segs[g];
     if (!s.src || !s.dst || !s.idx) return TWIST_ERR_NULL;
-    if (s.n_keep <= 0 || s.block_rows <= 0 || s.idx_stride < s.n_keep || s.src_row_offset < 0 ||
+    if (s.n_keep <= 0 || s.block_rows <= 0 || s.n_blocks <= 0 || s.idx_stride < s.n_keep || s.src_row_offset < 0 ||
         s.dst_row_offset < 0 || s.dst_subnet_stride < 0 || (s.dst_subnet_stride * elem) % 16 != 0)
       return TWIST_ERR_SHAPE;
     if (!aligned16(s.src) || !aligned16(s.dst) || !aligned16(s.dst_master)) return TWIST_ERR_SHAPE;
@@ -375,7 +384,7 @@ extern "C" int32_t twist_aggregate(const twist_aggregate_segment* segs, int32_t 
   for (int g = 0; g < n_segs; ++g) {
     const twist_aggregate_segment& s = segs[g];
     if (!s.dst || !s.sub || !s.cover || !s.pos) return TWIST_ERR_NULL;
-    if (s.n_full <= 0 || s.block_rows <= 0 || s.dst_row_offset < 0 || s.sub_row_offset < 0 ||
+    if (s.n_full <= 0 || s.block_rows <= 0 || s.n_keep <= 0 || s.dst_row_offset < 0 || s.sub_row_offset < 0 ||
         s.sub_subnet_stride < 0 || s.sub_subnet_stride % 4 != 0)
       return TWIST_ERR_SHAPE;
     if (!aligned16(s.dst) || !aligned16(s.sub) || !aligned16(s.dst_f32) || !aligned16(s.central)) return TWIST_ERR_SHAPE;
@@ -396,8 +405,10 @@ extern "C" int32_t twist_aggregate(const twist_aggregate_segment* segs, int32_t 
   p.part_chunks = kAggPartChunks;
   p.parts = (d / 4 + kAggPartChunks - 1) / kAggPartChunks;
   const int grid = grid_for_items(total * p.parts);
-  if (dtype == TWIST_BF16) aggregate_rows_kernel<true><<<grid, 256, 0, st>>>(p);
-  else aggregate_rows_kernel<false><<<grid, 256, 0, st>>>(p);
+  int* status = device_status_ptr();
+  if (!status) return TWIST_ERR_CUDA;
+  if (dtype == TWIST_BF16) aggregate_rows_kernel<true><<<grid, 256, 0, st>>>(p, status);
+  else aggregate_rows_kernel<false><<<grid, 256, 0, st>>>(p, status);
   TWIST_LAUNCH_CHECK();
   return TWIST_OK;
 }

@@ -145,10 +145,41 @@ __global__ void fused_loss_finish_kernel(const float* __restrict__ partial, long
   for (long long i = lane; i < per_group; i += 32) acc += (double)src[i];
   for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
   if (lane == 0) {
-    const int vc = valid_cols ? valid_cols[g] : seg_width;
+    const int vc = valid_cols ? min(max(valid_cols[g], 0), seg_width) : seg_width;
     const long long n_valid = seg_begin + (long long)((width - seg_begin) / seg_width) * vc;
-    loss[g] = (float)(acc / ((double)tokens * (double)n_valid));
+    loss[g] = n_valid > 0 ? (float)(acc / ((double)tokens * (double)n_valid)) : 0.f;
   }
+}
+
+// Self-test of the give-up path: a CTA pair with the GEMM's roles, barriers nobody ever arrives at, the same bounded
+// wait (with a short limit) and the same exit (abort flag, drain, pair barrier, tensor-memory release).
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 1)
+selftest_wait_kernel(unsigned long long limit_ns, int* status) {
+  __shared__ __align__(8) unsigned long long bars[3];
+  __shared__ uint32_t tmem_slot_s;
+  __shared__ int abort_s;
+  volatile uint32_t* tmem_slot = &tmem_slot_s;
+  volatile int* abort_flag = &abort_s;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (warp == kEpiWarps && lane == 0) {
+    for (int i = 0; i < 3; ++i) mbar_init(smem_u32(&bars[i]), 1);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == kEpiWarps + 1) pair_tmem_alloc(tmem_slot, 32u);
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  if (warp == kEpiWarps) {                       // producer role: "stage empty" never comes
+    if (lane == 0) mbar_wait_for(smem_u32(&bars[0]), 0, abort_flag, status, limit_ns);
+  } else if (warp == kEpiWarps + 1) {            // MMA issuer role (leader only): "stage full" never comes
+    if (lane == 0 && cluster_rank() == 0) mbar_wait_for(smem_u32(&bars[1]), 0, abort_flag, status, limit_ns);
+  } else {                                       // epilogue role: "accumulator full" never comes; warp-uniform outcome
+    (void)__all_sync(0xffffffffu, mbar_wait_for(smem_u32(&bars[2]), 0, abort_flag, status, limit_ns));
+  }
+  pair_teardown(abort_flag, warp == kEpiWarps + 1, tmem_base, 32u);
 }
 
 }  // namespace
@@ -225,3 +256,13 @@ int launch_gemm_bf16(int layout, int epi, const GemmOperand& A, const GemmOperan
 }
 
 }  // namespace twist
+
+extern "C" int32_t twist_selftest_wait(uint64_t limit_ns, void* stream) {
+  using namespace twist;
+  if (limit_ns == 0 || limit_ns > 100000000ull) return TWIST_ERR_SHAPE;       // at most 0.1 s
+  int* status = device_status_ptr();
+  if (!status) return TWIST_ERR_CUDA;
+  selftest_wait_kernel<<<2, kGemmThreads, 0, static_cast<cudaStream_t>(stream)>>>(limit_ns, status);
+  TWIST_LAUNCH_CHECK();
+  return TWIST_OK;
+}

@@ -133,6 +133,29 @@ __device__ inline void mbar_arrive_cluster(uint32_t cluster_addr) {
 __device__ inline void cluster_sync_all() {
   asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
+// Tensor memory of a CTA pair: the same warp of both CTAs allocates `cols` columns together and writes the base
+// address to `slot` (shared memory); pair_teardown is the common exit of such a pair.
+__device__ inline void pair_tmem_alloc(volatile uint32_t* slot, uint32_t cols) {
+  asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;"
+               ::"r"(smem_u32(const_cast<uint32_t*>(slot))), "r"(cols) : "memory");
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+// Called by every thread of both CTAs once their roles are done (or gave up).  If a wait ran out, copies that
+// may still be in flight get time to land before shared memory is released.  Neither CTA leaves (nor frees
+// tensor memory) while the other may still signal its barriers, read its shared memory or write its accumulators.
+__device__ inline void pair_teardown(volatile int* abort_flag, bool alloc_warp, uint32_t tmem_base, uint32_t cols) {
+  tc_fence_before();
+  __syncthreads();
+  if (*abort_flag) {
+    drain_after_abort(abort_flag);
+    __syncthreads();
+  }
+  cluster_sync_all();
+  if (alloc_warp) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(cols) : "memory");
+  }
+}
 // Tiled copy into this CTA's shared memory; completion bytes are counted on `bar`, which may be a
 // barrier of the other CTA of the pair (cluster-window address).
 __device__ inline void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2) {
@@ -308,11 +331,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
-  if (warp == kEpiWarps + 1) {   // the same warp of both CTAs allocates the pair's tensor memory together
-    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;"
-                 ::"r"(smem_u32(const_cast<uint32_t*>(tmem_slot))), "r"((uint32_t)kTmemCols) : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
-  }
+  if (warp == kEpiWarps + 1) pair_tmem_alloc(tmem_slot, (uint32_t)kTmemCols);
   tc_fence_before();
   __syncthreads();
   cluster_sync_all();          // the peer's barriers exist before anything is signalled across the pair
@@ -538,9 +557,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         float loss_acc = 0.f, kfac = 0.f;
         int vc = 0;
         if constexpr (kIsMse) {
-          vc = p.valid_cols ? p.valid_cols[g] : p.seg_width;
+          vc = p.valid_cols ? min(max(p.valid_cols[g], 0), p.seg_width) : p.seg_width;
           const int n_valid = p.seg_begin + ((p.N - p.seg_begin) / p.seg_width) * vc;
-          kfac = 2.0f / ((float)p.M * (float)n_valid);
+          kfac = n_valid > 0 ? 2.0f / ((float)p.M * (float)n_valid) : 0.f;      // no valid column: zero loss, zero gradient
         }
         auto load_acc = [&](int c, EpiAcc<EPI>& a) {
           tc_ld32(t_row + 32 * c, a.r0);
@@ -718,21 +737,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   }
 
   // ------------------------------------------------------------------ teardown
-  tc_fence_before();
-  __syncthreads();
-  if (*abort_flag) {
-    // a wait expired: give copies that may still be in flight time to land before shared memory is released
-    const uint64_t t0 = global_timer_ns();
-    while (global_timer_ns() - t0 < 2000000ull) __nanosleep(1000);
-    __syncthreads();
-  }
-  // Neither CTA leaves (nor frees tensor memory) while the other may still signal its barriers, read
-  // its shared memory or write its accumulators.
-  cluster_sync_all();
-  if (warp == kEpiWarps + 1) {
-    tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)kTmemCols) : "memory");
-  }
+  pair_teardown(abort_flag, warp == kEpiWarps + 1, tmem_base, (uint32_t)kTmemCols);
 }
 
 // Host side ------------------------------------------------------------------------------------

@@ -38,9 +38,10 @@ __global__ void __launch_bounds__(256) mse_kernel(const void* __restrict__ y_, c
                                                   float* __restrict__ partial) {
   __shared__ float scratch[8];
   const int s = blockIdx.y;
-  const int vc = valid_cols ? valid_cols[s] : seg_width;
+  const int vc = valid_cols ? min(max(valid_cols[s], 0), seg_width) : seg_width;
   const long long n = (long long)tokens * width;
-  const float k = 2.0f / ((float)tokens * (float)valid_count(width, seg_begin, seg_width, vc));
+  const int n_valid = valid_count(width, seg_begin, seg_width, vc);
+  const float k = n_valid > 0 ? 2.0f / ((float)tokens * (float)n_valid) : 0.f;     // no valid column: zero gradient
   float acc = 0.f;
   if (BF16) {
     const uint4* y = reinterpret_cast<const uint4*>(static_cast<const __nv_bfloat16*>(y_) + (long long)s * n);
@@ -87,8 +88,9 @@ __global__ void mse_finish_kernel(const float* __restrict__ partial, int nblocks
   for (int i = lane; i < nblocks; i += 32) acc += (double)partial[(long long)s * kMseBlocks + i];
   for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
   if (lane == 0) {
-    const int vc = valid_cols ? valid_cols[s] : seg_width;
-    loss[s] = (float)(acc / ((double)tokens * (double)valid_count(width, seg_begin, seg_width, vc)));
+    const int vc = valid_cols ? min(max(valid_cols[s], 0), seg_width) : seg_width;
+    const int n_valid = valid_count(width, seg_begin, seg_width, vc);
+    loss[s] = n_valid > 0 ? (float)(acc / ((double)tokens * (double)n_valid)) : 0.f;
   }
 }
 

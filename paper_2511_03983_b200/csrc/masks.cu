@@ -218,7 +218,15 @@ extern "C" int32_t twist_sample_masks(uint64_t seed, uint64_t round, int32_t lay
   const int threads = np >= 4096 ? 1024 : 256;
   const size_t smem = (size_t)np * 8 + 64 * 4 + (size_t)n_full;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  TWIST_CUDA_TRY(cudaFuncSetAttribute(sample_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  // The shared-memory limit is raised once per device to what the largest block count needs: setting it per call
+  // would let two host threads with different sizes lower it between one thread's set and its launch.
+  static bool configured[64] = {false};
+  const int slot = device_slot();
+  if (!configured[slot]) {
+    TWIST_CUDA_TRY(cudaFuncSetAttribute(sample_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        TWIST_MAX_BLOCKS * 8 + 64 * 4 + TWIST_MAX_BLOCKS));
+    configured[slot] = true;
+  }
   sample_rows_kernel<<<dim3(n_subnets, n_layers), threads, smem, st>>>(seed, round, layer_begin, kind, n_full,
                                                                        n_subnets, n_sub, sample_mode, np, cl, idx);
   TWIST_LAUNCH_CHECK();

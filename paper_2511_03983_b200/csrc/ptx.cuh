@@ -33,19 +33,37 @@ __device__ inline uint64_t global_timer_ns() {
   return t;
 }
 
-// Bounded wait: gives up after ~2 s of wall time or as soon as another role of the CTA gave up.
-__device__ inline bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status) {
+// Records a status code in the device status word.  Codes are negative; the most negative one wins, so a wait
+// that ran out is not hidden by a bad index seen later.
+__device__ inline void note_status(int* status, int code) { atomicMin(status, code); }
+
+// Bounded wait: gives up after `limit_ns` of wall time or as soon as another role of the CTA gave up.
+constexpr uint64_t kWaitLimitNs = 2000000000ull;      // 2 s: far beyond any launch of this library
+__device__ inline bool mbar_wait_for(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status,
+                                     uint64_t limit_ns) {
   if (mbar_try_wait(bar, parity)) return true;
   const uint64_t t0 = global_timer_ns();
   for (uint32_t it = 1;; ++it) {
     if (mbar_try_wait(bar, parity)) return true;
     if ((it & 255u) == 0) {
-      if (*abort_flag || global_timer_ns() - t0 > 2000000000ull) {
+      if (*abort_flag || global_timer_ns() - t0 > limit_ns) {
         *abort_flag = 1;
-        atomicExch(status, (int)TWIST_ERR_DEVICE_TIMEOUT);
+        note_status(status, (int)TWIST_ERR_DEVICE_TIMEOUT);
         return false;
       }
     }
+  }
+}
+__device__ inline bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status) {
+  return mbar_wait_for(bar, parity, abort_flag, status, kWaitLimitNs);
+}
+
+// After a wait ran out somewhere in the CTA: copies that were requested may still be in flight, so shared memory
+// must not be released yet.  Sleeps long enough for them to land (call by every thread, between CTA barriers).
+__device__ inline void drain_after_abort(volatile int* abort_flag) {
+  if (*abort_flag) {
+    const uint64_t t0 = global_timer_ns();
+    while (global_timer_ns() - t0 < 2000000ull) __nanosleep(1000);
   }
 }
 

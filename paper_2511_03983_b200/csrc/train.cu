@@ -4,6 +4,8 @@
 // kernels (tiny correctness workload only).
 #include <math.h>
 
+#include <initializer_list>
+
 #include "gemm_sm100.cuh"
 #include "glue.cuh"
 
@@ -16,12 +18,25 @@ namespace {
     if (rc__ != TWIST_OK) return rc__;\
   } while (0)
 
+// The kernels touch these arrays with 16-byte (the byte mask: 8-byte) vector accesses; a pointer that breaks the
+// rule is refused here instead of faulting on the device.  NULL passes (absence is checked where it matters).
+bool all_aligned16(std::initializer_list<const void*> ptrs) {
+  for (const void* p : ptrs)
+    if (!aligned16(p)) return false;
+  return true;
+}
+bool aligned8(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 7u) == 0; }
+
 int check_ffn(const twist_ffn_args* a) {
   if (!a) return TWIST_ERR_NULL;
   if (a->n_subnets <= 0 || a->tokens <= 0 || a->d_model <= 0 || a->f_sub <= 0) return TWIST_ERR_SHAPE;
   if (a->ffn_kind < TWIST_FFN_RELU || a->ffn_kind > TWIST_FFN_SWIGLU) return TWIST_ERR_SHAPE;
   if (a->dtype != TWIST_FP32 && a->dtype != TWIST_BF16) return TWIST_ERR_SHAPE;
   if (a->dtype == TWIST_BF16 && (a->d_model % 8 || a->f_sub % 8)) return TWIST_ERR_SHAPE;
+  if (!all_aligned16({a->x, a->w_gu, a->w_down, a->w_gu_master, a->w_down_master, a->pre, a->hh, a->y, a->dy, a->dpre,
+                      a->dx, a->dw_gu, a->dw_down, a->tgt, a->loss_ws, a->y_residual, a->dx_residual, a->m_gu, a->v_gu,
+                      a->m_down, a->v_down}) || !aligned8(a->hidden_mask))
+    return TWIST_ERR_SHAPE;
   return TWIST_OK;
 }
 
@@ -211,6 +226,9 @@ static int check_proj(const twist_proj_args* a) {
   if (a->which != TWIST_PROJ_QKV && a->which != TWIST_PROJ_O) return TWIST_ERR_SHAPE;
   if (a->dtype != TWIST_FP32 && a->dtype != TWIST_BF16) return TWIST_ERR_SHAPE;
   if (a->dtype == TWIST_BF16 && (a->d_model % 8 || a->n % 8)) return TWIST_ERR_SHAPE;
+  if (!all_aligned16({a->in, a->w, a->w_master, a->out, a->d_out, a->d_in, a->dw, a->tgt, a->loss_ws, a->out_residual,
+                      a->d_in_residual, a->m, a->v}))
+    return TWIST_ERR_SHAPE;
   return TWIST_OK;
 }
 

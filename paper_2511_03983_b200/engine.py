@@ -168,22 +168,24 @@ class RoundEngine:
         if "ffn" in which:
             if self.g == 2:
                 segs.append(B.gather_segment(self.full["gate"][l], self.w_gu, self.w_gu_m, self.gather_idx_ffn[l], None,
-                                             w.ffn_keep, w.ffn_keep, w.ffn_block, 0, gf * d, 0))
+                                             w.ffn_keep, w.ffn_keep, w.ffn_block, 0, gf * d, 0, w.n_ffn_blocks))
             segs.append(B.gather_segment(self.full["up"][l], self.w_gu, self.w_gu_m, self.gather_idx_ffn[l], None,
-                                         w.ffn_keep, w.ffn_keep, w.ffn_block, 0, gf * d, f if self.g == 2 else 0))
+                                         w.ffn_keep, w.ffn_keep, w.ffn_block, 0, gf * d, f if self.g == 2 else 0,
+                                         w.n_ffn_blocks))
             segs.append(B.gather_segment(self.full["down"][l], self.w_down, self.w_down_m, self.gather_idx_ffn[l], None,
-                                         w.ffn_keep, w.ffn_keep, w.ffn_block, 0, f * d, 0))
+                                         w.ffn_keep, w.ffn_keep, w.ffn_block, 0, f * d, 0, w.n_ffn_blocks))
         if self.has_attn and "attn" in which:
             H, Hkv, dh = w.n_heads, w.n_kv_heads, w.d_head
             qkv = self.full["qkv"][l]
             segs.append(B.gather_segment(qkv, self.w_qkv, self.w_qkv_m, self.idx_head[l], None, w.head_keep,
-                                         w.head_keep, dh, 0, self.nq * d, 0))
+                                         w.head_keep, dh, 0, self.nq * d, 0, H))
             segs.append(B.gather_segment(qkv, self.w_qkv, self.w_qkv_m, self.kv_idx[l], self.kv_count[l], Hkv,
-                                         self.kv_max, dh, H * dh, self.nq * d, self.a_sub))
+                                         self.kv_max, dh, H * dh, self.nq * d, self.a_sub, Hkv))
             segs.append(B.gather_segment(qkv, self.w_qkv, self.w_qkv_m, self.kv_idx[l], self.kv_count[l], Hkv,
-                                         self.kv_max, dh, (H + Hkv) * dh, self.nq * d, self.a_sub + self.kv_max * dh))
+                                         self.kv_max, dh, (H + Hkv) * dh, self.nq * d, self.a_sub + self.kv_max * dh,
+                                         Hkv))
             segs.append(B.gather_segment(self.full["o"][l], self.w_o, self.w_o_m, self.idx_head[l], None, w.head_keep,
-                                         w.head_keep, dh, 0, self.a_sub * d, 0))
+                                         w.head_keep, dh, 0, self.a_sub * d, 0, H))
         with self._timed("gather"):
             B.twist_gather_subnets(segs, w.n_subnets, d, w.dtype)
             for n in self.moment_names:        # a fresh worker state: first and second moments start at zero
@@ -201,23 +203,26 @@ class RoundEngine:
         if "ffn" in which:
             if self.g == 2:
                 segs.append(B.aggregate_segment(self.full["gate"][l], f32("gate"), sub(self.w_gu, self.w_gu_m),
-                                                self.cover_ffn[l], self.agg_pos_ffn[l], nb, w.ffn_block, 0, gf * d, 0))
+                                                self.cover_ffn[l], self.agg_pos_ffn[l], nb, w.ffn_block, 0, gf * d, 0,
+                                                w.ffn_keep))
             segs.append(B.aggregate_segment(self.full["up"][l], f32("up"), sub(self.w_gu, self.w_gu_m),
                                             self.cover_ffn[l], self.agg_pos_ffn[l], nb, w.ffn_block, 0, gf * d,
-                                            f if self.g == 2 else 0))
+                                            f if self.g == 2 else 0, w.ffn_keep))
             segs.append(B.aggregate_segment(self.full["down"][l], f32("down"), sub(self.w_down, self.w_down_m),
-                                            self.cover_ffn[l], self.agg_pos_ffn[l], nb, w.ffn_block, 0, f * d, 0))
+                                            self.cover_ffn[l], self.agg_pos_ffn[l], nb, w.ffn_block, 0, f * d, 0,
+                                            w.ffn_keep))
         if self.has_attn and "attn" in which:
             H, Hkv, dh = w.n_heads, w.n_kv_heads, w.d_head
             q_sub = sub(self.w_qkv, self.w_qkv_m)
             segs.append(B.aggregate_segment(self.full["qkv"][l], f32("qkv"), q_sub, self.cover_head[l],
-                                            self.pos_head[l], H, dh, 0, self.nq * d, 0))
+                                            self.pos_head[l], H, dh, 0, self.nq * d, 0, w.head_keep))
             segs.append(B.aggregate_segment(self.full["qkv"][l], f32("qkv"), q_sub, self.kv_cover[l], self.kv_pos[l],
-                                            Hkv, dh, H * dh, self.nq * d, self.a_sub))
+                                            Hkv, dh, H * dh, self.nq * d, self.a_sub, self.kv_max))
             segs.append(B.aggregate_segment(self.full["qkv"][l], f32("qkv"), q_sub, self.kv_cover[l], self.kv_pos[l],
-                                            Hkv, dh, (H + Hkv) * dh, self.nq * d, self.a_sub + self.kv_max * dh))
+                                            Hkv, dh, (H + Hkv) * dh, self.nq * d, self.a_sub + self.kv_max * dh,
+                                            self.kv_max))
             segs.append(B.aggregate_segment(self.full["o"][l], f32("o"), sub(self.w_o, self.w_o_m), self.cover_head[l],
-                                            self.pos_head[l], H, dh, 0, self.a_sub * d, 0))
+                                            self.pos_head[l], H, dh, 0, self.a_sub * d, 0, w.head_keep))
         with self._timed("aggregate"):
             B.twist_aggregate(segs, w.n_subnets, d, w.dtype, live)
         self.launches += 1
@@ -433,7 +438,7 @@ class HybridRoundEngine(RoundEngine):
         for m, off, dst, dst_m, stride in ([("gate", 0, self.w_gu, self.w_gu_m, gf)] if self.g == 2 else []) + [
                 ("up", f if self.g == 2 else 0, self.w_gu, self.w_gu_m, gf), ("down", 0, self.w_down, self.w_down_m, f)]:
             segs.append(B.gather_segment(self.full[m][l], dst[1:], dst_m[1:], idx, None, w.ffn_keep, w.ffn_keep,
-                                         w.ffn_block, 0, stride * d, off))
+                                         w.ffn_block, 0, stride * d, off, w.n_ffn_blocks))
         with self._timed("gather"):
             B.twist_gather_subnets(segs, w.n_subnets - 1, d, w.dtype)
             B.twist_hidden_mask(self.cover_ffn[l], w.n_ffn_blocks, w.ffn_block, 0, 1, self.c_mask)
@@ -483,8 +488,8 @@ class HybridRoundEngine(RoundEngine):
         for m, off, sub, stride in ([("gate", 0, self.w_gu_m, gf)] if self.g == 2 else []) + [
                 ("up", f if self.g == 2 else 0, self.w_gu_m, gf), ("down", 0, self.w_down_m, f)]:
             segs.append(B.aggregate_segment(self.full[m][l], self.full_f32[m][l], sub, self.cover_ffn[l], self.pos_ffn[l],
-                                            nb, w.ffn_block, 0, stride * d, off, central=self.full_f32[m][l],
-                                            central_subnet=0))
+                                            nb, w.ffn_block, 0, stride * d, off, w.ffn_keep,
+                                            central=self.full_f32[m][l], central_subnet=0))
         with self._timed("aggregate"):
             B.twist_aggregate(segs, w.n_subnets, d, w.dtype, live)
         self.launches += 1

@@ -23,7 +23,7 @@ def test_library_exports_every_declared_symbol():
     for n in names:
         assert hasattr(h, n), n
     assert sorted(B.EXPORTS) == names
-    assert B.twist_abi_version() == 1
+    assert B.twist_abi_version() == 2
     # every entry point that takes arguments declares their C types: a device address passed without them
     # would be truncated to 32 bits
     for n in names:
@@ -55,11 +55,17 @@ def test_host_side_argument_checks():
     assert f(1, 0, 0, 1, 0, 12, 4, 6, C.cast(bad, C.c_void_p), 2, 0, dummy, dummy, dummy, None) == B.ERR_BAD_INDEX
     # gather / aggregate
     assert h.twist_gather_subnets(None, 1, 2, 64, B.BF16, None) == B.ERR_NULL
-    seg = B.GatherSegment(0x1000, 0x2000, None, 0x3000, None, 4, 4, 1, 0, 0, 256, 0)
+    seg = B.GatherSegment(0x1000, 0x2000, None, 0x3000, None, 4, 4, 1, 16, 0, 256, 0)
     arr = (B.GatherSegment * 1)(seg)
     assert h.twist_gather_subnets(C.cast(arr, C.c_void_p), 1, 2, 63, B.BF16, None) == B.ERR_SHAPE     # row not 16 B
     assert h.twist_gather_subnets(C.cast(arr, C.c_void_p), 9, 2, 64, B.BF16, None) == B.ERR_SHAPE     # too many segments
+    seg0 = B.GatherSegment(0x1000, 0x2000, None, 0x3000, None, 4, 4, 1, 0, 0, 256, 0)     # source block count missing
+    arr0 = (B.GatherSegment * 1)(seg0)
+    assert h.twist_gather_subnets(C.cast(arr0, C.c_void_p), 1, 2, 64, B.BF16, None) == B.ERR_SHAPE
     assert h.twist_aggregate(None, 1, 2, 64, B.BF16, 3, None) == B.ERR_NULL
+    ag = (B.AggregateSegment * 1)(B.AggregateSegment(0x1000, None, 0x2000, 0x3000, 0x4000, 8, 1, 0, 256, 0, None, 0, 0))
+    assert h.twist_aggregate(C.cast(ag, C.c_void_p), 1, 2, 64, B.BF16, 3, None) == B.ERR_SHAPE   # slice block count missing
+    assert h.twist_selftest_wait(0, None) == B.ERR_SHAPE and h.twist_selftest_wait(10 ** 9, None) == B.ERR_SHAPE
     # local steps
     a = B.FfnArgs(B.FFN_SWIGLU, B.BF16, 2, 128, 64, 100, 1.0, 0.0)       # f_sub not a multiple of 8
     assert h.twist_subnet_ffn_fwd(C.byref(a), None) == B.ERR_SHAPE
@@ -89,6 +95,37 @@ def test_host_side_argument_checks():
     a = B.FfnArgs(B.FFN_SWIGLU, B.FP32, 2, 128, 64, 96, 1.0, 0.0, 0x1000, 0x1000, 0x1000, None, None, 0x1000, 0x1000, 0x1000)
     a.hidden_mask = 0x1000
     assert h.twist_subnet_ffn_fwd(C.byref(a), None) == B.ERR_UNSUPPORTED
+
+
+def test_misaligned_pointers_are_refused_before_any_launch():
+    """The kernels use 16-byte (the activation mask: 8-byte) vector accesses; a pointer that breaks the rule must
+    come back as a status, never reach the device."""
+    from paper_2511_03983_b200 import binding as B
+    h = B.lib()
+    ok = 0x10000
+    names = ["x", "w_gu", "w_down", "w_gu_master", "w_down_master", "pre", "hh", "y", "dy", "dpre", "dx", "dw_gu",
+             "dw_down", "tgt", "loss_ws", "y_residual", "dx_residual", "m_gu", "v_gu", "m_down", "v_down"]
+    for n in names:
+        a = B.FfnArgs(B.FFN_SWIGLU, B.BF16, 2, 128, 64, 96, 1.0, 0.0)
+        for m in names:
+            setattr(a, m, ok)
+        setattr(a, n, ok + (8 if n != "x" else 2))
+        assert h.twist_subnet_ffn_fwd(C.byref(a), None) == B.ERR_SHAPE, n
+        assert h.twist_subnet_ffn_bwd(C.byref(a), None) == B.ERR_SHAPE, n
+    a = B.FfnArgs(B.FFN_SWIGLU, B.BF16, 2, 128, 64, 96, 1.0, 0.0)
+    for m in names:
+        setattr(a, m, ok)
+    a.hidden_mask = ok + 4                                   # byte mask: 8-byte rule
+    assert h.twist_subnet_ffn_fwd(C.byref(a), None) == B.ERR_SHAPE
+    pnames = ["in_", "w", "w_master", "out", "d_out", "d_in", "dw", "tgt", "loss_ws", "out_residual", "d_in_residual",
+              "m", "v"]
+    for n in pnames:
+        p = B.ProjArgs(B.PROJ_O, B.BF16, 2, 128, 64, 64, 1.0, 0.0)
+        for m in pnames:
+            setattr(p, m, ok)
+        setattr(p, n, ok + 4)
+        assert h.twist_subnet_attn_proj_fwd(C.byref(p), None) == B.ERR_SHAPE, n
+        assert h.twist_subnet_attn_proj_bwd(C.byref(p), None) == B.ERR_SHAPE, n
 
 
 def test_missing_library_fails_loudly(monkeypatch, tmp_path):

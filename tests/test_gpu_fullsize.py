@@ -11,6 +11,7 @@ import numpy as np
 import pytest
 import torch
 
+from fp32_mirror import aggregate_f32
 from oracle import twist_oracle as o
 from paper_2511_03983_b200 import inputs as I
 
@@ -198,6 +199,10 @@ def test_aggregate_whole_layer(setup):
         assert held.any()
         err = np.abs(got[held] - want[held]) / np.maximum(mag[held], 1e-30)
         assert err.max() <= 1e-6, (name, err.max())
+        # bit for bit the fp32 evaluation in the fixed order (ascending subnets, one IEEE division)
+        mirror = aggregate_f32(full[name], [v.astype(np.float32) for v in subs], blue, br, row_offset=off)[rows]
+        got32 = eng.full_f32[name][0].cpu().numpy()[rows]
+        assert np.array_equal(got32[held].view(np.uint32), mirror[held].view(np.uint32)), name
         shadow = eng.full[name][0][rows]
         assert torch.equal(shadow[torch.from_numpy(held).cuda()],
                            eng.full_f32[name][0][rows][torch.from_numpy(held).cuda()].to(torch.bfloat16))
@@ -292,3 +297,154 @@ def test_attention_core_at_stack_workload_sizes(cfg):
         assert rel_fro(got[:, :nqh], dZ[:, :nqh]) < TOL, "dq"
         assert rel_fro(got[:, nqh:nqh + dh], dZ[:, nqh:nqh + dh]) < TOL, "dk"
         assert rel_fro(got[:, nqh + dh:], dZ[:, nqh + dh:]) < TOL, "dv"
+
+
+# ---------------------------------------------------------------------------------------------------------------
+# The gather / aggregate sweep workload (7B FFN shapes, IID masks, 1024 tokens per subnet) at full block counts:
+# the cell with rows no subnet holds (S = 2, keep 1/4), the cell with up to 16 subnets per row and the widest
+# slices (S = 16, keep 3/4: f' = 8256), and the f' = 5504 cell (S = 4, keep 1/2).  One layer.
+# ---------------------------------------------------------------------------------------------------------------
+
+CELLS5 = [(2, 0.25), (16, 0.75), (4, 0.5)]
+
+
+@pytest.fixture(scope="module", params=CELLS5, ids=lambda c: f"S{c[0]}-keep{c[1]}")
+def cell(request):
+    from paper_2511_03983_b200 import binding as B
+    from paper_2511_03983_b200.engine import RoundEngine
+    B.lib()
+    S, keep = request.param
+    base = I.PRESETS[5]
+    w = replace(base, n_subnets=S, ffn_keep=int(np.floor(keep * base.n_ffn_blocks)), n_layers=1, local_steps=1,
+                name=f"cfg5-S{S}-keep{keep}")
+    eng = RoundEngine(w, keep_f32_full=True)
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(w.seed_w + S)
+    for m, v in eng.full.items():
+        v[0].copy_((torch.randn(v[0].shape, generator=gen, device="cuda") * 0.02).to(torch.bfloat16))
+    for m in eng.full:                    # the fp32 result starts as a recognisable value: untouched rows keep it
+        eng.full_f32[m].fill_(123.0)
+    T, d = w.tokens, w.d_model
+    rnd = lambda width, std=1.0: (torch.randn(S, T, width, generator=gen, device="cuda") * std).to(torch.bfloat16)
+    eng.X, eng.Td = [rnd(d)], [rnd(d)]
+    full_np = {m: v[0].float().cpu().numpy() for m, v in eng.full.items()}
+    eng.sample_masks(0)
+    eng.gather_layer(0)
+    torch.cuda.synchronize()
+    bp = o.layer_blueprints(w, 0, 0)
+    yield dict(B=B, eng=eng, w=w, full=full_np, bp=bp, gen=gen, rnd=rnd, rng=np.random.default_rng(7 + S))
+    del eng
+    torch.cuda.empty_cache()
+
+
+def test_sweep_cell_blueprints_bit_exact(cell):
+    eng, w, bp = cell["eng"], cell["w"], cell["bp"]
+    assert np.array_equal(eng.idx_ffn[0].cpu().numpy(), bp["ffn"])
+    c, count, p = o.cover_and_pos(bp["ffn"], w.n_ffn_blocks)
+    assert np.array_equal(eng.cover_ffn[0].cpu().numpy().view(np.uint32), c)
+    assert np.array_equal(eng.pos_ffn[0].cpu().numpy(), p)
+    if w.n_subnets == 2:
+        assert (count == 0).mean() > 0.4          # independent quarters leave (3/4)^2 of the blocks unheld
+    if w.n_subnets == 16:
+        assert count.max() == 16                  # some block is held by every subnet
+
+
+def test_sweep_cell_gathered_slices_bit_exact(cell):
+    eng, w, bp, full = cell["eng"], cell["w"], cell["bp"], cell["full"]
+    for s in sorted({0, w.n_subnets - 1}):
+        sl = o.gather_layer(w, full, bp, s)
+        want = {"w_gu": np.concatenate([sl["gate"], sl["up"]]), "w_down": sl["down"]}
+        for name, arr in want.items():
+            got16 = getattr(eng, name)[s].float().cpu().numpy()
+            got32 = getattr(eng, name + "_m")[s].cpu().numpy()
+            assert np.array_equal(got16.view(np.uint32), arr.view(np.uint32)), (s, name)
+            assert np.array_equal(got32.view(np.uint32), arr.view(np.uint32)), (s, name, "master")
+
+
+def test_sweep_cell_ffn_forward_backward_sampled(cell):
+    B, eng, w, rng = cell["B"], cell["eng"], cell["w"], cell["rng"]
+    S, T, d, f = w.n_subnets, w.tokens, w.d_model, w.f_sub
+    lr = w.lr
+    dY = cell["rnd"](d, 1e-4)
+    a = B.ffn_args(w.ffn_kind, w.dtype, S, T, d, f, eng.alpha_f, lr, x=eng.X[0], w_gu=eng.w_gu, w_down=eng.w_down,
+                   w_gu_master=eng.w_gu_m, w_down_master=eng.w_down_m, pre=eng.pre, hh=eng.hh, y=eng.y, dy=dY,
+                   dpre=eng.dpre, dx=eng.dx)
+    B.twist_subnet_ffn_fwd(a)
+    B.twist_subnet_ffn_bwd(a)
+    torch.cuda.synchronize()
+    assert B.twist_device_status() == 0
+    rows = np.sort(rng.choice(T, N_ROWS, replace=False))
+    r = torch.from_numpy(rows).cuda()
+    for s in sorted({0, S - 1}):
+        sl = {m: v.astype(np.float64) for m, v in o.gather_layer(w, cell["full"], cell["bp"], s).items()}
+        X, dYs = f64(eng.X[0][s]), f64(dY[s])
+        Yw, saved = o.ffn_fwd(X[rows], sl["up"], sl["gate"], sl["down"], w.ffn_kind, eng.alpha_f, True)
+        dXw, _, _, _ = o.ffn_bwd(dYs[rows], X[rows], saved, sl["up"], sl["gate"], sl["down"], w.ffn_kind, eng.alpha_f, True)
+        assert rel_fro(f64(eng.pre[s][r]), np.concatenate([saved["G"], saved["U"]], axis=1)) < TOL
+        assert rel_fro(f64(eng.hh[s][r]), saved["Hh"]) < TOL
+        assert rel_fro(f64(eng.y[s][r]), Yw) < TOL
+        assert rel_fro(f64(eng.dx[s][r]), dXw) < TOL
+        J = np.sort(np.concatenate([rng.choice(f, N_WROWS - 2, replace=False), [0, f - 1]]))     # incl. the ragged last tile
+        J = np.unique(J)
+        _, savedJ = o.ffn_fwd(X, sl["up"][J], sl["gate"][J], sl["down"][J], w.ffn_kind, eng.alpha_f, True)
+        _, dWu, dWg, dWd = o.ffn_bwd(dYs, X, savedJ, sl["up"][J], sl["gate"][J], sl["down"][J], w.ffn_kind, eng.alpha_f, True)
+        Jt = torch.from_numpy(J).cuda()
+        assert rel_fro(f64(eng.w_gu_m[s][Jt]) - sl["gate"][J], -lr * dWg) < TOL, (s, "gate")
+        assert rel_fro(f64(eng.w_gu_m[s][Jt + f]) - sl["up"][J], -lr * dWu) < TOL, (s, "up")
+        assert rel_fro(f64(eng.w_down_m[s][Jt]) - sl["down"][J], -lr * dWd) < TOL, (s, "down")
+        assert torch.equal(eng.w_gu[s][Jt], eng.w_gu_m[s][Jt].to(torch.bfloat16))
+
+
+def test_sweep_cell_aggregate_whole_layer(cell):
+    """The whole layer's aggregate.  The operation is independent per column, so the oracle (float64) and the fp32
+    mirror evaluate every row on a sample of columns (all lanes and row spans of the kernel occur among them) and
+    every column on a sample of rows: within 1e-6 of the oracle relative to the mean magnitude of the averaged
+    values (the (count + 1) 2^-24 bound of the fp32 evaluation where count reaches 16), bit for bit equal to the fp32
+    evaluation in the fixed order, and rows nobody holds untouched in both outputs."""
+    eng, w, bp, full, gen, rng = cell["eng"], cell["w"], cell["bp"], cell["full"], cell["gen"], cell["rng"]
+    S, f, d, F = w.n_subnets, w.f_sub, w.d_model, w.d_ff
+    for m in (eng.w_gu_m, eng.w_down_m):
+        m.copy_(torch.randn(m.shape, generator=gen, device="cuda") * 0.02)
+    before16 = {m: eng.full[m][0].clone() for m in eng.full}
+    eng.aggregate_layer(0)
+    torch.cuda.synchronize()
+    _, count, _ = o.cover_and_pos(bp["ffn"], w.n_ffn_blocks)
+    held = count > 0
+    cols = np.unique(np.concatenate([rng.choice(d, 254, replace=False), [0, d - 1]]))
+    rows = np.unique(np.concatenate([rng.choice(F, 30, replace=False), [0, F - 1]]))
+    ct, rt = torch.from_numpy(cols).cuda(), torch.from_numpy(rows).cuda()
+    cases = [("gate", eng.w_gu_m[:, :f]), ("up", eng.w_gu_m[:, f:]), ("down", eng.w_down_m)]
+    for name, master in cases:
+        # (1) every row, sampled columns
+        subs32 = master[:, :, ct].cpu().numpy()
+        W0 = full[name][:, cols]
+        want = o.aggregate(W0.astype(np.float64), [subs32[s].astype(np.float64) for s in range(S)], bp["ffn"], 1)
+        mag = o.aggregate(np.abs(W0).astype(np.float64), [np.abs(subs32[s]).astype(np.float64) for s in range(S)],
+                          bp["ffn"], 1)
+        mirror = aggregate_f32(W0, [subs32[s] for s in range(S)], bp["ffn"], 1)
+        got = eng.full_f32[name][0][:, ct].cpu().numpy()
+        err = np.abs(got[held].astype(np.float64) - want[held]) / np.maximum(mag[held], 1e-30)
+        assert err.max() <= max(1e-6, (count.max() + 1) * 2.0 ** -24), (name, err.max())
+        assert np.array_equal(got[held].view(np.uint32), mirror[held].view(np.uint32)), name
+        assert np.all(got[~held] == 123.0), name                                  # rows nobody holds: not written
+        # (2) sampled rows, every column
+        subs_r = []
+        kept_rows = []
+        for s in range(S):
+            pos = np.searchsorted(bp["ffn"][s], rows)
+            pos = np.where((pos < f) & (bp["ffn"][s][np.minimum(pos, f - 1)] == rows), pos, -1)
+            kept_rows.append(pos)
+        got_r = eng.full_f32[name][0][rt].cpu().numpy()
+        for i, rr in enumerate(rows):
+            holders = [s for s in range(S) if kept_rows[s][i] >= 0]
+            if not holders:
+                assert np.all(got_r[i] == 123.0)
+                continue
+            acc = np.zeros(d, dtype=np.float32)
+            for s in holders:                                                     # ascending s, float32
+                acc = acc + master[s, int(kept_rows[s][i])].cpu().numpy()
+            assert np.array_equal(got_r[i].view(np.uint32), (acc / np.float32(len(holders))).view(np.uint32)), (name, rr)
+        # the bf16 model: rounded result on held rows, previous bytes elsewhere
+        ht = torch.from_numpy(held).cuda()
+        assert torch.equal(eng.full[name][0][ht], eng.full_f32[name][0][ht].to(torch.bfloat16))
+        assert torch.equal(eng.full[name][0][~ht], before16[name][~ht])

@@ -441,3 +441,29 @@ def test_blockwise_local_steps_with_adam_equal_torch_adam_on_the_dense_model():
         opt.step()
     for m in sl:
         assert np.allclose(sl[m], tw[m].detach().numpy(), rtol=1e-9, atol=1e-12), m
+
+
+def test_fp32_mirror_of_the_aggregator_agrees_with_the_float64_oracle():
+    """tests/fp32_mirror.py (the fixed-order float32 evaluation the GPU result must equal bit for bit) against the
+    float64 aggregator: same rows held, same untouched rows, and every averaged element within the rounding of
+    count float32 additions and one division, (count + 1) 2^-24, relative to the mean magnitude of the values
+    averaged.  A hand case fixes its order of operations."""
+    from fp32_mirror import aggregate_f32
+    rng = np.random.default_rng(3)
+    n_full, S, n_sub, br, d = 40, 16, 30, 2, 24
+    A = np.stack([np.sort(rng.choice(n_full, n_sub, replace=False)) for _ in range(S)])
+    W = rng.standard_normal((n_full * br + 3, d)).astype(np.float32)
+    subs = [rng.standard_normal((n_sub * br, d)).astype(np.float32) for _ in range(S)]
+    for live in (None, 0b1010011):
+        got = aggregate_f32(W, subs, A, br, live_mask=live, row_offset=3)
+        want = o.aggregate(W.astype(np.float64), subs, A, br, live_mask=live, row_offset=3)
+        mag = o.aggregate(np.abs(W).astype(np.float64), [np.abs(v) for v in subs], A, br, live_mask=live, row_offset=3)
+        touched = np.any(want != W, axis=1)
+        assert np.array_equal(got[~touched], W[~touched]) and touched[:3].sum() == 0
+        assert np.max(np.abs(got[touched] - want[touched]) / mag[touched]) <= (S + 1) * 2.0 ** -24
+    # order of operations: ((a + b) + c) / 3 in float32, not a + (b + c), not a product with a rounded 1/3
+    a, b, c = np.float32(1.0), np.float32(2.0 ** -24), np.float32(2.0 ** -24)
+    got = aggregate_f32(np.zeros((1, 1), np.float32), [np.full((1, 1), v, np.float32) for v in (a, b, c)],
+                        [[0], [0], [0]], 1)
+    assert got[0, 0] == np.float32((np.float32(a + b) + c) / np.float32(3.0)) == np.float32(1.0) / np.float32(3.0)
+    assert got[0, 0] != np.float32(a + np.float32(b + c)) / np.float32(3.0)

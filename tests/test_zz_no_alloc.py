@@ -46,6 +46,27 @@ def test_noalloc_matches_workspace_entry_point_twice_in_a_row():
     assert B.twist_device_status() == 0
 
 
+def test_noalloc_call_allocates_no_device_memory():
+    """What the entry point is for: once its first call on the device has happened, a call leaves the device's free
+    memory and the allocator's books exactly as they were."""
+    from paper_2511_03983_b200 import binding as B
+    B.lib()
+    S, T, width = 4, 256, 128
+    y = torch.randn(S, T, width, device="cuda").to(torch.bfloat16)
+    t = torch.randn(S, T, width, device="cuda").to(torch.bfloat16)
+    dy = torch.zeros_like(y)
+    loss = torch.zeros(S, dtype=torch.float32, device="cuda")
+    B.twist_mse_fwd_bwd_noalloc(y, t, dy, loss, S, T, width, None, 0, 0, I.DTYPE_BF16)      # warm-up: first call
+    torch.cuda.synchronize()
+    free0, alloc0, reserved0 = torch.cuda.mem_get_info()[0], torch.cuda.memory_allocated(), torch.cuda.memory_reserved()
+    for _ in range(3):
+        B.twist_mse_fwd_bwd_noalloc(y, t, dy, loss, S, T, width, None, 0, 0, I.DTYPE_BF16)
+    torch.cuda.synchronize()
+    assert torch.cuda.mem_get_info()[0] == free0
+    assert torch.cuda.memory_allocated() == alloc0 and torch.cuda.memory_reserved() == reserved0
+    assert float(loss.min()) > 0.5
+
+
 def test_noalloc_rejects_more_subnets_than_its_scratch_holds():
     from paper_2511_03983_b200 import binding as B
     h = B.lib()
