@@ -255,7 +255,9 @@ __global__ void __launch_bounds__(256) aggregate_rows_kernel(const __grid_consta
       const float q = a * rden;
       return fmaf(fmaf(-q, denom, a), rden, q);
     };
-    for (int c0 = c_begin + lane; c0 < c_end; c0 += 32 * kUnroll) {
+    // warp-uniform trip count (the shuffles below need every lane): lanes past the end of the span load nothing
+    for (int cb = c_begin; cb < c_end; cb += 32 * kUnroll) {
+      const int c0 = cb + lane;
       float4 acc[kUnroll];
 #pragma unroll
       for (int u = 0; u < kUnroll; ++u) acc[u] = make_float4(0.f, 0.f, 0.f, 0.f);

@@ -796,9 +796,13 @@ def test_two_chained_rounds_gather_the_previous_rounds_shadow(B):
             for m in eng.full:
                 got = eng.full[m][l].float().cpu().numpy().astype(np.float64)
                 differ = got != free_shadow[m]
-                ulp = np.abs(free_shadow[m]) * 2.0 ** -7 + 1e-30
+                # one bf16 ulp at the magnitude of the weight (of the old one where the update nearly cancels it)
+                ulp = np.maximum(np.abs(free_shadow[m]), np.abs(oracle_shadow[l][m])) * 2.0 ** -7 + 1e-30
                 assert differ.mean() < (0.02 if rnd == 0 else 0.06), (rnd, l, m, differ.mean())
-                assert np.all(np.abs(got - free_shadow[m])[differ] <= 2.0 * ulp[differ]), (rnd, l, m)
+                # a rounding flip per round, plus (for weights much smaller than their update) the 2e-2-level
+                # difference of the updates themselves
+                bound = 2.0 * (rnd + 1) * ulp + 0.1 * np.abs(free_shadow[m] - oracle_shadow[l][m])
+                assert np.all(np.abs(got - free_shadow[m])[differ] <= bound[differ]), (rnd, l, m)
             oracle_shadow[l] = free_shadow
         changed = np.mean([np.mean(eng.full[m][l].float().cpu().numpy() != full_np[l][m]) for m in eng.full
                            for l in range(w.n_layers)])
