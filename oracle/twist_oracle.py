@@ -194,6 +194,38 @@ def act_scale(n_full, n_sub):
 
 
 # ----------------------------------------------------------------------------------------
+# Layer normalisation (App. A, Layer Normalization): z = (x - mu) / sigma with mu, sigma the mean and the
+# standard deviation of the d_model elements of a token, y = gamma * z + b.  The paper's formula has no
+# stabiliser; sigma is taken as sqrt(var + eps) with a small eps (the usual convention; eps = 0 gives the
+# printed formula).  gamma and b are shared parameters: every worker gets a copy and trains it.
+# ----------------------------------------------------------------------------------------
+
+LN_EPS = 1e-5
+
+
+def layer_norm_fwd(X, gamma, beta, lowp, eps=LN_EPS):
+    """Y [T, d] (stored precision) and what the backward pass needs: the normalised rows z and 1 / sigma."""
+    mu = X.mean(axis=1, keepdims=True)
+    var = ((X - mu) ** 2).mean(axis=1, keepdims=True)
+    rstd = 1.0 / np.sqrt(var + eps)
+    z = (X - mu) * rstd
+    return _q(gamma[None, :] * z + beta[None, :], lowp), {"z": z, "rstd": rstd}
+
+
+def layer_norm_bwd(dY, saved, gamma, lowp, residual=None):
+    """Exact chain rule through layer_norm_fwd: with dz = dY * gamma,
+        dX = (dz - mean(dz) - z mean(dz * z)) / sigma,   dgamma = sum_t dY * z,   db = sum_t dY.
+    `residual`: gradient arriving over the skip connection around the normalised block, added before dX is stored."""
+    z, rstd = saved["z"], saved["rstd"]
+    dz = dY * gamma[None, :]
+    dX = rstd * (dz - dz.mean(axis=1, keepdims=True) - z * (dz * z).mean(axis=1, keepdims=True))
+    return _q(_plus(dX, residual), lowp), np.sum(dY * z, axis=0), np.sum(dY, axis=0)
+
+
+LN_PARAMS = ("ln_a_g", "ln_a_b", "ln_f_g", "ln_f_b")     # gamma / b of the attention and the FFN normalisation
+
+
+# ----------------------------------------------------------------------------------------
 # FFN block on a dense slice.  Paper (App. A, Feedforward): y = C relu(W x).
 # GELU (exact, x Phi(x)) and SwiGLU (silu(gate) * up) are the workloads' variants.
 # ----------------------------------------------------------------------------------------
@@ -284,14 +316,20 @@ def o_bwd(dY, A, W_o, alpha, lowp):
 # Loss and optimiser of the local steps: mean squared error, plain SGD.
 # ----------------------------------------------------------------------------------------
 
-def mse(Y, Tgt, lowp, valid_cols=None):
+def mse(Y, Tgt, lowp, valid_cols=None, col_mask=None):
     """loss = mean over the T x width elements of (y - t)^2 (no 1/2); dY = 2 (y - t) / (T width).
-    valid_cols restricts both to the leading columns (zero gradient elsewhere)."""
+    valid_cols restricts both to the leading columns, col_mask [width] of 0/1 to the columns it marks (zero
+    gradient elsewhere; the mean runs over the valid elements).  No valid column: loss 0, gradient 0."""
     T, width = Y.shape
-    vc = width if valid_cols is None else valid_cols
+    if col_mask is not None:
+        cols = np.flatnonzero(np.asarray(col_mask) != 0)
+    else:
+        cols = np.arange(width if valid_cols is None else valid_cols)
     diff = np.zeros_like(Y, dtype=np.float64)
-    diff[:, :vc] = Y[:, :vc] - Tgt[:, :vc]
-    n = T * vc
+    diff[:, cols] = Y[:, cols] - Tgt[:, cols]
+    n = T * len(cols)
+    if n == 0:
+        return 0.0, diff
     return float(np.sum(diff * diff) / n), _q(2.0 * diff / n, lowp)
 
 
@@ -366,13 +404,22 @@ def aggregate(W_full, subs, blueprints, block_rows, live_mask=None, row_offset=0
 # dispatch, local training for the repartition interval, aggregate, resample).
 # ----------------------------------------------------------------------------------------
 
+def layer_keeps(spec, layer):
+    """(N_sub for the FFN blocks, N_sub for the heads) of one layer.  A shared layer (Sec. 5 Setup: the first and
+    the last two layers of the paper's runs) has N_sub = N_full in both kinds: every worker holds all of it."""
+    if layer in getattr(spec, "shared_layers", ()):
+        return spec.d_ff // spec.ffn_block, spec.n_heads
+    return spec.ffn_keep, spec.head_keep
+
+
 def layer_blueprints(spec, rnd, layer):
     """Blueprints of one layer for one round: FFN blocks, heads, KV groups."""
     out = {}
-    out["ffn"] = sample_blueprint(spec.d_ff // spec.ffn_block, spec.n_subnets, spec.ffn_keep, spec.common_ffn,
+    ffn_keep, head_keep = layer_keeps(spec, layer)
+    out["ffn"] = sample_blueprint(spec.d_ff // spec.ffn_block, spec.n_subnets, ffn_keep, spec.common_ffn,
                                   spec.seed_mask, rnd, layer, KIND_FFN, spec.sample_mode)
     if spec.n_heads:
-        out["head"] = sample_blueprint(spec.n_heads, spec.n_subnets, spec.head_keep, spec.common_heads,
+        out["head"] = sample_blueprint(spec.n_heads, spec.n_subnets, head_keep, spec.common_heads,
                                        spec.seed_mask, rnd, layer, KIND_HEAD, spec.sample_mode)
         out["kv_idx"], out["kv_count"] = kv_groups(out["head"], spec.n_heads, spec.n_kv_heads)
     return out
@@ -392,6 +439,9 @@ def gather_layer(spec, full, bp, s):
                                     gather_rows(full["qkv"], kv, dh, H * dh),
                                     gather_rows(full["qkv"], kv, dh, (H + Hkv) * dh)], axis=0)
         sl["o"] = gather_rows(full["o"], bp["head"][s], dh)
+    for m in LN_PARAMS:          # shared parameters are broadcast whole (Sec. 3.2)
+        if m in full:
+            sl[m] = np.array(full[m], copy=True)
     return sl
 
 
@@ -400,7 +450,7 @@ def local_steps_blockwise(spec, sl, get_batch, rnd, s, lowp):
     place).  get_batch(kind, rnd, s, k, width) -> [T, width].  Returns the losses
     {block: [K]}.  Batch kinds: 0 X, 1 target of width d, 2 target of QKV width, 3 A."""
     d = spec.d_model
-    alpha_f = act_scale(spec.d_ff // spec.ffn_block, spec.ffn_keep)
+    alpha_f = act_scale(spec.d_ff, sl["up"].shape[0])          # N_full / N_sub of this layer (Sec. 3.4)
     losses = {"ffn": [], "qkv": [], "o": []}
     opt = _Optimizer(spec)
     for k in range(spec.local_steps):
@@ -417,7 +467,7 @@ def local_steps_blockwise(spec, sl, get_batch, rnd, s, lowp):
         if dWg is not None:
             sl["gate"] = opt.update("gate", sl["gate"], dWg, lowp)
         if spec.n_heads:
-            alpha_a = act_scale(spec.n_heads, spec.head_keep)
+            alpha_a = act_scale(spec.n_heads * spec.d_head, sl["o"].shape[0])
             nq = sl["qkv"].shape[0]
             Tq = get_batch(2, rnd, s, k, nq).astype(np.float64)
             QKV = qkv_fwd(X, cw["qkv"], lowp)
@@ -440,9 +490,12 @@ def aggregate_layer(spec, full, slices, bp):
     new = {}
     for m in ("up", "down") + (("gate",) if spec.ffn_kind == FFN_SWIGLU else ()):
         new[m] = aggregate(full[m], [slices[s][m] for s in range(S)], bp["ffn"], spec.ffn_block)
+    for m in LN_PARAMS:          # held by every subnet: the aggregator formula is the plain mean over S
+        if m in full:
+            new[m] = aggregate(np.asarray(full[m])[None, :], [slices[s][m][None, :] for s in range(S)], [[0]] * S, 1)[0]
     if spec.n_heads:
         dh, H, Hkv = spec.d_head, spec.n_heads, spec.n_kv_heads
-        a_sub = spec.head_keep * dh
+        a_sub = len(bp["head"][0]) * dh
         kvs = [bp["kv_idx"][s][: bp["kv_count"][s]] for s in range(S)]
         qkv = aggregate(full["qkv"], [slices[s]["qkv"][:a_sub] for s in range(S)], bp["head"], dh)
         qkv = aggregate(qkv, [slices[s]["qkv"][a_sub:a_sub + len(kvs[s]) * dh] for s in range(S)], kvs, dh,
@@ -548,17 +601,27 @@ def head_kv_positions(bp, spec, s):
 def stack_fwd(spec, layers, head_kv, X0, n_seqs, seq_len, lowp):
     """layers[l] = compute copies {gate, up, down, qkv, o} of one subnet; head_kv[l] as above.
     Returns the final x and what the backward pass needs per layer."""
-    alpha_f = act_scale(spec.d_ff // spec.ffn_block, spec.ffn_keep)
-    alpha_a = act_scale(spec.n_heads, spec.head_keep)
     x, saved = X0, []
     for l, W in enumerate(layers):
+        alpha_f = act_scale(spec.d_ff, W["up"].shape[0])                        # per layer: N_full / N_sub
+        alpha_a = act_scale(spec.n_heads * spec.d_head, W["o"].shape[0])
         kvw = (W["qkv"].shape[0] - W["o"].shape[0]) // 2
-        QKV = qkv_fwd(x, W["qkv"], lowp)
+        sv = {"x": x, "kvw": kvw}
+        if "ln_a_g" in W:            # pre-LN layer (App. A, Transformer Layer Architecture, steps 1 and 4)
+            x_a, sv["ln_a"] = layer_norm_fwd(x, W["ln_a_g"], W["ln_a_b"], lowp)
+        else:
+            x_a = x
+        QKV = qkv_fwd(x_a, W["qkv"], lowp)
         A = attn_core_fwd(QKV, n_seqs, seq_len, spec.d_head, head_kv[l], kvw, lowp)
         x_mid = o_fwd(A, W["o"], alpha_a, lowp, residual=x)
-        x_out, ffn_saved = ffn_fwd(x_mid, W["up"], W.get("gate"), W["down"], spec.ffn_kind, alpha_f, lowp,
+        if "ln_f_g" in W:
+            x_f, sv["ln_f"] = layer_norm_fwd(x_mid, W["ln_f_g"], W["ln_f_b"], lowp)
+        else:
+            x_f = x_mid
+        x_out, ffn_saved = ffn_fwd(x_f, W["up"], W.get("gate"), W["down"], spec.ffn_kind, alpha_f, lowp,
                                    residual=x_mid)
-        saved.append({"x": x, "QKV": QKV, "A": A, "x_mid": x_mid, "ffn": ffn_saved, "kvw": kvw})
+        sv.update({"x_a": x_a, "QKV": QKV, "A": A, "x_mid": x_mid, "x_f": x_f, "ffn": ffn_saved})
+        saved.append(sv)
         x = x_out
     return x, saved
 
@@ -567,18 +630,29 @@ def stack_bwd(spec, layers, head_kv, saved, dX, n_seqs, seq_len, lowp):
     """Gradients of every layer's slices for the loss gradient dX at the output; also returns
     the gradient with respect to the input.  The gradient of each residual sum flows both
     through the block and over the skip connection."""
-    alpha_f = act_scale(spec.d_ff // spec.ffn_block, spec.ffn_keep)
-    alpha_a = act_scale(spec.n_heads, spec.head_keep)
     grads = [None] * len(layers)
     dx = dX
     for l in reversed(range(len(layers))):
         W, sv = layers[l], saved[l]
-        dx_mid, dWu, dWg, dWd = ffn_bwd(dx, sv["x_mid"], sv["ffn"], W["up"], W.get("gate"), W["down"],
-                                        spec.ffn_kind, alpha_f, lowp, residual=dx)
+        alpha_f = act_scale(spec.d_ff, W["up"].shape[0])
+        alpha_a = act_scale(spec.n_heads * spec.d_head, W["o"].shape[0])
+        g = {}
+        if "ln_f" in sv:     # the skip connection's gradient joins the normalised branch's at the normalisation's input
+            d_f, dWu, dWg, dWd = ffn_bwd(dx, sv["x_f"], sv["ffn"], W["up"], W.get("gate"), W["down"],
+                                         spec.ffn_kind, alpha_f, lowp)
+            dx_mid, g["ln_f_g"], g["ln_f_b"] = layer_norm_bwd(d_f, sv["ln_f"], W["ln_f_g"], lowp, residual=dx)
+        else:
+            dx_mid, dWu, dWg, dWd = ffn_bwd(dx, sv["x_mid"], sv["ffn"], W["up"], W.get("gate"), W["down"],
+                                            spec.ffn_kind, alpha_f, lowp, residual=dx)
         dA, dWo = o_bwd(dx_mid, sv["A"], W["o"], alpha_a, lowp)
         dQKV = attn_core_bwd(dA, sv["QKV"], n_seqs, seq_len, spec.d_head, head_kv[l], sv["kvw"], lowp)
-        dx, dWq = qkv_bwd(dQKV, sv["x"], W["qkv"], lowp, residual=dx_mid)
-        grads[l] = {"up": dWu, "gate": dWg, "down": dWd, "qkv": dWq, "o": dWo}
+        if "ln_a" in sv:
+            d_a, dWq = qkv_bwd(dQKV, sv["x_a"], W["qkv"], lowp)
+            dx, g["ln_a_g"], g["ln_a_b"] = layer_norm_bwd(d_a, sv["ln_a"], W["ln_a_g"], lowp, residual=dx_mid)
+        else:
+            dx, dWq = qkv_bwd(dQKV, sv["x"], W["qkv"], lowp, residual=dx_mid)
+        g.update({"up": dWu, "gate": dWg, "down": dWd, "qkv": dWq, "o": dWo})
+        grads[l] = g
     return grads, dx
 
 
@@ -591,14 +665,15 @@ def local_steps_stack(spec, slices, head_kv, get_batch, rnd, s, n_seqs, seq_len,
         opt.begin_step()
         X0 = get_batch(0, rnd, s, k, spec.d_model).astype(np.float64)
         Tgt = get_batch(1, rnd, s, k, spec.d_model).astype(np.float64)
-        layers = [{m: _q(v, lowp) for m, v in sl.items()} for sl in slices]
+        # compute copies: the partitioned matrices in stored precision; the normalisation's parameters stay wide
+        layers = [{m: (v if m in LN_PARAMS else _q(v, lowp)) for m, v in sl.items()} for sl in slices]
         xL, saved = stack_fwd(spec, layers, head_kv, X0, n_seqs, seq_len, lowp)
         loss, dX = mse(xL, Tgt, lowp)
         grads, _ = stack_bwd(spec, layers, head_kv, saved, dX, n_seqs, seq_len, lowp)
         losses.append(loss)
         for l, (sl, g) in enumerate(zip(slices, grads)):
             for m in sl:
-                sl[m] = opt.update((l, m), sl[m], g[m], lowp)
+                sl[m] = opt.update((l, m), sl[m], g[m], lowp and m not in LN_PARAMS)
     return losses
 
 

@@ -467,3 +467,153 @@ def test_fp32_mirror_of_the_aggregator_agrees_with_the_float64_oracle():
                         [[0], [0], [0]], 1)
     assert got[0, 0] == np.float32((np.float32(a + b) + c) / np.float32(3.0)) == np.float32(1.0) / np.float32(3.0)
     assert got[0, 0] != np.float32(a + np.float32(b + c)) / np.float32(3.0)
+
+
+# ------------------------------------------------------------------ layer normalisation (App. A)
+
+def test_layer_norm_matches_torch_forward_and_autograd():
+    r = _rng(31)
+    T, d = 7, 12
+    X, g, b = r.standard_normal((T, d)) * 2 + 0.5, r.standard_normal(d) + 1.0, r.standard_normal(d)
+    dY, res = r.standard_normal((T, d)), r.standard_normal((T, d))
+    Y, saved = o.layer_norm_fwd(X, g, b, lowp=False)
+    tx, tg, tb = (torch.tensor(v, requires_grad=True) for v in (X, g, b))
+    want = torch.nn.functional.layer_norm(tx, (d,), tg, tb, eps=o.LN_EPS)
+    assert np.allclose(Y, want.detach().numpy(), rtol=1e-12, atol=1e-13)
+    (want * torch.from_numpy(dY)).sum().backward()
+    dX, dg, db = o.layer_norm_bwd(dY, saved, g, lowp=False)
+    assert np.allclose(dX, tx.grad.numpy(), rtol=1e-10, atol=1e-12)
+    assert np.allclose(dg, tg.grad.numpy(), rtol=1e-10, atol=1e-12)
+    assert np.allclose(db, tb.grad.numpy(), rtol=1e-10, atol=1e-12)
+    dXr, _, _ = o.layer_norm_bwd(dY, saved, g, lowp=False, residual=res)       # the skip connection's gradient
+    assert np.allclose(dXr, dX + res, rtol=0, atol=1e-14)
+
+
+def test_layer_norm_definition_and_finite_differences():
+    """App. A, Layer Normalization: z = (x - mu) / sigma has zero mean and unit variance per token, and with the
+    initial parameters (gamma = 1, b = 0: App. A, Initialization) the output is z itself; y is invariant to a
+    shift and to a positive scaling of the token; the gradient passes a central-difference check."""
+    r = _rng(32)
+    T, d = 5, 16
+    X = r.standard_normal((T, d)) * 3 + 1
+    Y, saved = o.layer_norm_fwd(X, np.ones(d), np.zeros(d), lowp=False, eps=0.0)
+    assert np.allclose(Y.mean(axis=1), 0, atol=1e-13) and np.allclose(Y.var(axis=1), 1, atol=1e-12)
+    assert np.array_equal(Y, saved["z"])
+    Y2, _ = o.layer_norm_fwd(4.0 * X + 7.0, np.ones(d), np.zeros(d), lowp=False, eps=0.0)
+    assert np.allclose(Y, Y2, atol=1e-12)
+    g, b, dY = r.standard_normal(d), r.standard_normal(d), r.standard_normal((T, d))
+    f = lambda Z, gg, bb: float(np.sum(o.layer_norm_fwd(Z, gg, bb, False)[0] * dY))
+    _, sv = o.layer_norm_fwd(X, g, b, False)
+    dX, dg, db = o.layer_norm_bwd(dY, sv, g, False)
+    eps = 1e-6
+    for (i, j) in [(0, 0), (2, 5), (4, 15)]:
+        Zp, Zm = X.copy(), X.copy()
+        Zp[i, j] += eps; Zm[i, j] -= eps
+        assert abs((f(Zp, g, b) - f(Zm, g, b)) / (2 * eps) - dX[i, j]) < 1e-6 * max(1.0, abs(dX[i, j]))
+    for j in (0, 7):
+        gp, gm = g.copy(), g.copy()
+        gp[j] += eps; gm[j] -= eps
+        assert abs((f(X, gp, b) - f(X, gm, b)) / (2 * eps) - dg[j]) < 1e-6 * max(1.0, abs(dg[j]))
+        bp_, bm = b.copy(), b.copy()
+        bp_[j] += eps; bm[j] -= eps
+        assert abs((f(X, g, bp_) - f(X, g, bm)) / (2 * eps) - db[j]) < 1e-6 * max(1.0, abs(db[j]))
+
+
+def test_layer_norm_parameter_count_is_two_d_model():
+    """App. C: N_ln = 2 d_model per normalisation (gamma and b)."""
+    d = 768
+    _, saved = o.layer_norm_fwd(np.zeros((1, d)) + np.arange(d), np.ones(d), np.zeros(d), False)
+    assert saved["z"].shape == (1, d) and np.ones(d).size + np.zeros(d).size == 2 * d
+
+
+# ------------------------------------------------------------------ column-mask loss, masked attention worker (Sec. 4.1)
+
+def test_mse_with_a_column_mask_and_with_no_valid_column():
+    r = _rng(33)
+    Y, Tg = r.standard_normal((6, 10)), r.standard_normal((6, 10))
+    mask = np.array([1, 0, 0, 1, 1, 0, 1, 0, 0, 0])
+    cols = np.flatnonzero(mask)
+    loss, dY = o.mse(Y, Tg, False, col_mask=mask)
+    assert loss == pytest.approx(np.mean((Y[:, cols] - Tg[:, cols]) ** 2), rel=1e-13)
+    assert np.allclose(dY[:, cols], 2 * (Y[:, cols] - Tg[:, cols]) / (6 * len(cols))) and np.all(dY[:, mask == 0] == 0)
+    l2, d2 = o.mse(Y[:, :4], Tg[:, :4], False, col_mask=np.ones(4))
+    l3, d3 = o.mse(Y[:, :4], Tg[:, :4], False)
+    assert l2 == l3 and np.array_equal(d2, d3)
+    l0, d0 = o.mse(Y, Tg, False, col_mask=np.zeros(10))
+    assert l0 == 0.0 and np.all(d0 == 0)
+
+
+def test_head_masked_projections_equal_the_gathered_slices():
+    """Sec. 4.1, Masked TwIST for attention: on the full-width projections with the dropped heads masked out (their
+    query / key / value columns out of the loss; their head outputs zeroed before the output projection) the kept
+    rows see the gathered subnet's outputs, losses and gradients, and the dropped rows get exactly zero gradient.
+    Checked with torch autograd on the masked full matrices."""
+    r = _rng(34)
+    T, d, H, dh = 9, 10, 6, 4
+    kept = np.array([1, 2, 5])
+    rows = np.concatenate([np.arange(h * dh, (h + 1) * dh) for h in kept])
+    qrows = np.concatenate([rows, H * dh + rows, 2 * H * dh + rows])          # Q, K, V rows of the kept heads
+    Wqkv, Wo = r.standard_normal((3 * H * dh, d)), r.standard_normal((H * dh, d))
+    X = r.standard_normal((T, d))
+    Tq_full, A_full, Td = r.standard_normal((T, 3 * H * dh)), r.standard_normal((T, H * dh)), r.standard_normal((T, d))
+    cmask = np.zeros(3 * H * dh); cmask[qrows] = 1
+    amask = np.zeros(H * dh); amask[rows] = 1
+    alpha = o.act_scale(H, len(kept))
+    # gathered subnet
+    out_g = o.qkv_fwd(X, Wqkv[qrows], False)
+    loss_g, dq_g = o.mse(out_g, Tq_full[:, qrows], False)
+    dx_g, dWq_g = o.qkv_bwd(dq_g, X, Wqkv[qrows], False)
+    y_g = o.o_fwd(A_full[:, rows], Wo[rows], alpha, False)
+    loss_o, dy = o.mse(y_g, Td, False)
+    dA_g, dWo_g = o.o_bwd(dy, A_full[:, rows], Wo[rows], alpha, False)
+    # masked full-width worker, by the oracle ...
+    out_m = o.qkv_fwd(X, Wqkv, False)
+    loss_m, dq_m = o.mse(out_m, Tq_full, False, col_mask=cmask)
+    dx_m, dWq_m = o.qkv_bwd(dq_m, X, Wqkv, False)
+    y_m = o.o_fwd(A_full * amask, Wo, alpha, False)
+    _, dWo_m = o.o_bwd(dy, A_full * amask, Wo, alpha, False)
+    assert loss_m == pytest.approx(loss_g, rel=1e-13) and np.allclose(dx_m, dx_g, atol=1e-14)
+    assert np.allclose(dWq_m[qrows], dWq_g, atol=1e-14) and np.all(np.delete(dWq_m, qrows, axis=0) == 0)
+    assert np.allclose(y_m, y_g, atol=1e-13)
+    assert np.allclose(dWo_m[rows], dWo_g, atol=1e-14) and np.all(np.delete(dWo_m, rows, axis=0) == 0)
+    # ... and by autograd on the masked model
+    tq, to = torch.tensor(Wqkv, requires_grad=True), torch.tensor(Wo, requires_grad=True)
+    tm = torch.from_numpy(cmask)
+    lq = (((torch.from_numpy(X) @ tq.T - torch.from_numpy(Tq_full)) * tm) ** 2).sum() / (T * tm.sum())
+    lo = torch.mean((alpha * ((torch.from_numpy(A_full) * torch.from_numpy(amask)) @ to) - torch.from_numpy(Td)) ** 2)
+    (lq + lo).backward()
+    assert lq.item() == pytest.approx(loss_m, rel=1e-12) and lo.item() == pytest.approx(loss_o, rel=1e-12)
+    assert np.allclose(tq.grad.numpy(), dWq_m, atol=1e-13) and np.allclose(to.grad.numpy(), dWo_m, atol=1e-13)
+
+
+# ------------------------------------------------------------------ shared layers (Sec. 5 Setup: N_sub = N_full)
+
+def test_shared_layer_is_held_by_every_worker_and_averaged_over_all_of_them():
+    r = _rng(35)
+    spec = _spec(n_layers=2, n_subnets=3, ffn_keep=6, ffn_kind=o.FFN_GELU, n_heads=4, n_kv_heads=4, d_head=2,
+                 head_keep=2, local_steps=1, tokens=6, shared_layers=(1,))
+    assert o.layer_keeps(spec, 0) == (6, 2) and o.layer_keeps(spec, 1) == (16, 4)
+    bp = o.layer_blueprints(spec, 0, 1)
+    assert all(np.array_equal(row, np.arange(16)) for row in bp["ffn"])
+    assert all(np.array_equal(row, np.arange(4)) for row in bp["head"])
+    assert o.layer_blueprints(spec, 0, 0)["ffn"].shape == (3, 6)
+    d, F, a = 8, 16, 8
+    full = {"up": r.standard_normal((F, d)), "down": r.standard_normal((F, d)),
+            "qkv": r.standard_normal((3 * a, d)), "o": r.standard_normal((a, d))}
+    data = {}
+    get_batch = lambda kd, rnd, s, k, width: data.setdefault((kd, s, width),
+                                                             _rng(200 + 10 * kd + s).standard_normal((spec.tokens, width)))
+    new, _, _, losses = o.round_blockwise_layer(spec, full, get_batch, 0, 1, lowp=False)
+    # every worker trains the whole dense layer (scale 1) on its own batch; the aggregate is the plain mean
+    mean = {m: np.zeros_like(v) for m, v in full.items()}
+    for s in range(3):
+        t = {m: torch.tensor(v, requires_grad=True) for m, v in full.items()}
+        X, Td = torch.from_numpy(get_batch(0, 0, s, 0, d)), torch.from_numpy(get_batch(1, 0, s, 0, d))
+        Tq, A = torch.from_numpy(get_batch(2, 0, s, 0, 3 * a)), torch.from_numpy(get_batch(3, 0, s, 0, a))
+        l_ffn = torch.mean((_dense_ffn_torch(o.FFN_GELU, X, t["up"], None, t["down"], 1.0) - Td) ** 2)
+        (l_ffn + torch.mean((X @ t["qkv"].T - Tq) ** 2) + torch.mean((A @ t["o"] - Td) ** 2)).backward()
+        assert losses[s]["ffn"][0] == pytest.approx(l_ffn.item(), rel=1e-12)
+        for m in full:
+            mean[m] += (full[m] - spec.lr * t[m].grad.numpy()) / 3
+    for m in full:
+        assert np.allclose(new[m], mean[m], rtol=1e-11, atol=1e-13), m

@@ -108,10 +108,15 @@ def _torch_stack(spec, full, masks, X, n_seqs, N):
     masked out (Sec. 4.1: masked and gathered subnets compute the same function)."""
     H, Hkv, dh = spec.n_heads, spec.n_kv_heads, spec.d_head
     per = H // Hkv
-    alpha_f = (spec.d_ff / spec.ffn_keep) ** 0.5
-    alpha_a = (H / spec.head_keep) ** 0.5
     x = X
+    ln = lambda v, g, b: torch.nn.functional.layer_norm(v, (v.shape[1],), g, b, eps=o.LN_EPS)
     for l, W in enumerate(full):
+        ffn_keep, head_keep = o.layer_keeps(spec, l)
+        alpha_f = (spec.d_ff / ffn_keep) ** 0.5
+        alpha_a = (H / head_keep) ** 0.5
+        x_in = x
+        if "ln_a_g" in W:
+            x = ln(x, W["ln_a_g"], W["ln_a_b"])
         qkv = x @ W["qkv"].T
         heads = []
         for b in range(n_seqs):
@@ -121,9 +126,10 @@ def _torch_stack(spec, full, masks, X, n_seqs, N):
             V = torch.stack([r[:, (H + Hkv + h // per) * dh:(H + Hkv + h // per + 1) * dh] for h in range(H)])
             O = _sdpa(Q, K, V) * masks[l]["head"][:, None, None]
             heads.append(torch.cat([O[h] for h in range(H)], dim=1))
-        x = x + alpha_a * (torch.cat(heads, dim=0) @ W["o"])
-        U = x @ W["up"].T
-        G = x @ W["gate"].T if "gate" in W else None
+        x = x_in + alpha_a * (torch.cat(heads, dim=0) @ W["o"])
+        x_f = ln(x, W["ln_f_g"], W["ln_f_b"]) if "ln_f_g" in W else x
+        U = x_f @ W["up"].T
+        G = x_f @ W["gate"].T if "gate" in W else None
         x = x + alpha_f * ((_torch_act(spec.ffn_kind, U, G) * masks[l]["ffn"]) @ W["down"])
     return x
 
@@ -207,3 +213,85 @@ def test_stack_round_with_one_full_subnet_is_dense_training():
         for m in rows:
             want = full[l][m] - spec.lr * tw[l][m].grad.numpy()
             assert np.allclose(new[l][m], want, rtol=1e-10, atol=1e-12), (l, m)
+
+
+@pytest.mark.parametrize("shared", [(), (1,)])
+def test_pre_ln_stack_equals_masked_full_model_with_layer_norm_under_autograd(shared):
+    """App. A, Transformer Layer Architecture: LN -> attention -> skip -> LN -> FFN -> skip.  K local steps of a
+    gathered subnet through the pre-LN stack = K SGD steps of the masked full model written with torch's own
+    layer_norm, on the kept rows AND on the (shared, whole) normalisation parameters.  With a shared layer
+    (N_sub = N_full, Sec. 5 Setup) that layer's slices are the whole matrices and its scales are 1."""
+    spec = _spec(ffn_kind=o.FFN_SWIGLU, n_kv_heads=2, shared_layers=shared)
+    r = _rng(16)
+    L, d, F, H, dh, hkv = spec.n_layers, spec.d_model, spec.d_ff, spec.n_heads, spec.d_head, spec.n_kv_heads
+    n_seqs, N = 2, 5
+    rows = {"up": F, "down": F, "gate": F, "qkv": (H + 2 * hkv) * dh, "o": H * dh}
+    full = []
+    for _ in range(L):
+        layer = {m: r.standard_normal((rows[m], d)) * 0.3 for m in rows}
+        layer.update(ln_a_g=1 + 0.2 * r.standard_normal(d), ln_a_b=0.1 * r.standard_normal(d),
+                     ln_f_g=1 + 0.2 * r.standard_normal(d), ln_f_b=0.1 * r.standard_normal(d))
+        full.append(layer)
+    batches = {(kd, k): r.standard_normal((n_seqs * N, d)) for kd in (0, 1) for k in range(spec.local_steps)}
+    get_batch = lambda kd, rnd, s, k, width: batches[(kd, k)]
+    s = 1
+    bps = [o.layer_blueprints(spec, 0, l) for l in range(L)]
+    slices = [{m: v.astype(np.float64) for m, v in o.gather_layer(spec, full[l], bps[l], s).items()} for l in range(L)]
+    for l in range(L):
+        assert all(m in slices[l] for m in o.LN_PARAMS)
+        if l in shared:
+            assert slices[l]["up"].shape[0] == F and slices[l]["o"].shape[0] == H * dh
+    head_kv = [o.head_kv_positions(bps[l], spec, s) for l in range(L)]
+    losses = o.local_steps_stack(spec, slices, head_kv, get_batch, 0, s, n_seqs, N, lowp=False)
+    tw = [{m: torch.from_numpy(v.copy()).requires_grad_(True) for m, v in full[l].items()} for l in range(L)]
+    masks = []
+    for l in range(L):
+        fm = torch.zeros(F, dtype=torch.float64); fm[torch.from_numpy(bps[l]["ffn"][s].astype(np.int64))] = 1
+        hm = torch.zeros(H, dtype=torch.float64); hm[torch.from_numpy(bps[l]["head"][s].astype(np.int64))] = 1
+        masks.append({"ffn": fm, "head": hm})
+    for k in range(spec.local_steps):
+        y = _torch_stack(spec, tw, masks, torch.from_numpy(batches[(0, k)]), n_seqs, N)
+        loss = torch.mean((y - torch.from_numpy(batches[(1, k)])) ** 2)
+        assert abs(loss.item() - losses[k]) < 1e-10 * max(1.0, loss.item())
+        loss.backward()
+        with torch.no_grad():
+            for W in tw:
+                for v in W.values():
+                    v -= spec.lr * v.grad
+                    v.grad = None
+    for l in range(L):
+        kept_f = bps[l]["ffn"][s]
+        for m in ("up", "down", "gate"):
+            assert np.allclose(slices[l][m], tw[l][m].detach().numpy()[kept_f], rtol=1e-9, atol=1e-11), (l, m)
+        for m in o.LN_PARAMS:
+            assert np.allclose(slices[l][m], tw[l][m].detach().numpy(), rtol=1e-9, atol=1e-11), (l, m)
+            assert not np.allclose(slices[l][m], full[l][m])                       # they were trained
+        heads = bps[l]["head"][s]
+        q_rows = np.concatenate([np.arange(h * dh, (h + 1) * dh) for h in heads])
+        assert np.allclose(slices[l]["o"], tw[l]["o"].detach().numpy()[q_rows], rtol=1e-9, atol=1e-11)
+
+
+def test_round_stack_aggregates_the_normalisation_parameters_as_a_plain_mean():
+    spec = _spec(ffn_kind=o.FFN_GELU, n_kv_heads=4, n_subnets=3, local_steps=1)
+    r = _rng(17)
+    L, d, F, H, dh = spec.n_layers, spec.d_model, spec.d_ff, spec.n_heads, spec.d_head
+    n_seqs, N = 1, 4
+    rows = {"up": F, "down": F, "qkv": 3 * H * dh, "o": H * dh}
+    full = []
+    for _ in range(L):
+        layer = {m: r.standard_normal((rows[m], d)) * 0.3 for m in rows}
+        layer.update(ln_a_g=np.ones(d), ln_a_b=np.zeros(d), ln_f_g=np.ones(d), ln_f_b=np.zeros(d))
+        full.append(layer)
+    data = {}
+    get_batch = lambda kd, rnd, s, k, w: data.setdefault((kd, s), _rng(300 + 10 * kd + s).standard_normal((N, d)))
+    new, bps, _ = o.round_stack(spec, full, get_batch, 0, n_seqs, N, False)
+    for l in range(L):
+        per_worker = []
+        for s in range(spec.n_subnets):
+            sl = [{m: v.astype(np.float64) for m, v in o.gather_layer(spec, full[j], bps[j], s).items()} for j in range(L)]
+            hk = [o.head_kv_positions(bps[j], spec, s) for j in range(L)]
+            o.local_steps_stack(spec, sl, hk, get_batch, 0, s, n_seqs, N, False)
+            per_worker.append(sl[l])
+        for m in o.LN_PARAMS:
+            assert np.allclose(new[l][m], np.mean([pw[m] for pw in per_worker], axis=0), rtol=1e-13, atol=1e-15)
+            assert new[l][m].shape == (d,)
