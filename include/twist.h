@@ -330,6 +330,45 @@ int32_t twist_attn_core_fwd(const twist_attn_core_args* a /*host*/, void* stream
 int32_t twist_attn_core_bwd(const twist_attn_core_args* a /*host*/, void* stream);
 
 /* ---------------------------------------------------------------------------------------------
+ * Layer normalisation of the pre-LN transformer layer (App. A, Layer Normalization: z = (x - mu) / sigma with
+ * mu, sigma the mean and standard deviation of a token's d_model elements, y = gamma * z + b; Transformer
+ * Layer Architecture: one normalisation before the attention block, one before the FFN block, the skip
+ * connections around them).  sigma = sqrt(var + eps); eps = 0 is the printed formula.  Used by the chained
+ * (STACK) composition.  gamma and b are shared parameters (Sec. 3.1: everything outside the blocks is shared):
+ * every worker holds a copy, gamma / beta [S][d_model] fp32, trains it, and the aggregator averages the copies
+ * (twist_gather_subnets / twist_aggregate in TWIST_FP32 with one block held by all subnets).
+ *   fwd:  y [S][T][d] = gamma[s] * (x - mean) * rstd + beta[s];  mean, rstd [S][T] fp32 are written (bwd reads them)
+ *   bwd:  dx = (dz - mean_d(dz) - z mean_d(dz z)) * rstd (+ dx_residual, one rounding for the sum), dz = dy * gamma,
+ *         dgamma[s] = sum_t dy z,  dbeta[s] = sum_t dy  (fixed summation order: deterministic), then the optimiser
+ *         step on gamma / beta when lr != 0 (twist_optimizer as in the GEMM calls; moments [S][d] fp32).
+ *         dx may alias dy or dx_residual.
+ * dtype TWIST_BF16 only (bf16 activations, fp32 arithmetic); d_model a multiple of 8, at most 4096.
+ * ws: device scratch of at least twist_layernorm_workspace_bytes(S, T, d) bytes (bwd only). */
+typedef struct {
+  int32_t dtype, n_subnets, tokens, d_model;
+  float eps, lr;
+  const void* x;            /* device [S][T][d] */
+  void* y;                  /* device [S][T][d]   fwd: out */
+  float* mean;              /* device [S][T]      fwd: out, bwd: in */
+  float* rstd;              /* device [S][T]      fwd: out, bwd: in */
+  float* gamma;             /* device [S][d]      bwd: updated when lr != 0 */
+  float* beta;              /* device [S][d] */
+  const void* dy;           /* device [S][T][d]   bwd: in, gradient w.r.t. y */
+  void* dx;                 /* device [S][T][d]   bwd: out */
+  const void* dx_residual;  /* device [S][T][d]   bwd: optional addend (gradient over the skip connection) */
+  float* dgamma;            /* device [S][d]      bwd: optional gradient dumps */
+  float* dbeta;
+  void* ws;                 /* device scratch (bwd) */
+  size_t ws_bytes;
+  twist_optimizer opt;
+  float *m_gamma, *v_gamma, *m_beta, *v_beta;   /* device fp32 Adam moments [S][d] */
+} twist_layernorm_args;
+
+size_t twist_layernorm_workspace_bytes(int32_t n_subnets, int32_t tokens, int32_t d_model);
+int32_t twist_layernorm_fwd(const twist_layernorm_args* a /*host*/, void* stream);
+int32_t twist_layernorm_bwd(const twist_layernorm_args* a /*host*/, void* stream);
+
+/* ---------------------------------------------------------------------------------------------
  * Loss of the local steps: mean squared error against a target, per subnet, and its gradient.
  *   loss[s] = mean over the valid elements of (y - t)^2;   dy = 2 (y - t) / n_valid  (zero where invalid)
  * Valid columns: all `width` columns when valid_cols is NULL.  Otherwise columns [0, seg_begin) are

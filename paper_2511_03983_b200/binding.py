@@ -31,7 +31,8 @@ EXPORTS = [
     "twist_kv_groups", "twist_gather_subnets", "twist_aggregate", "twist_subnet_ffn_fwd", "twist_subnet_ffn_bwd",
     "twist_subnet_attn_proj_fwd", "twist_subnet_attn_proj_bwd", "twist_mse_workspace_bytes", "twist_mse_fwd_bwd",
     "twist_mse_fwd_bwd_noalloc", "twist_fused_loss_workspace_bytes", "twist_attn_core_fwd", "twist_attn_core_bwd",
-    "twist_hidden_mask", "twist_selftest_wait",
+    "twist_hidden_mask", "twist_selftest_wait", "twist_layernorm_workspace_bytes", "twist_layernorm_fwd",
+    "twist_layernorm_bwd",
 ]
 
 
@@ -97,6 +98,15 @@ class AttnCoreArgs(C.Structure):
                 ("kv_pos", C.c_void_p), ("kv_count", C.c_void_p)]
 
 
+class LayerNormArgs(C.Structure):
+    _fields_ = [("dtype", C.c_int32), ("n_subnets", C.c_int32), ("tokens", C.c_int32), ("d_model", C.c_int32),
+                ("eps", C.c_float), ("lr", C.c_float), ("x", C.c_void_p), ("y", C.c_void_p), ("mean", C.c_void_p),
+                ("rstd", C.c_void_p), ("gamma", C.c_void_p), ("beta", C.c_void_p), ("dy", C.c_void_p),
+                ("dx", C.c_void_p), ("dx_residual", C.c_void_p), ("dgamma", C.c_void_p), ("dbeta", C.c_void_p),
+                ("ws", C.c_void_p), ("ws_bytes", C.c_size_t), ("opt", Optimizer), ("m_gamma", C.c_void_p),
+                ("v_gamma", C.c_void_p), ("m_beta", C.c_void_p), ("v_beta", C.c_void_p)]
+
+
 _lib_handle = None
 
 
@@ -122,8 +132,11 @@ def lib() -> C.CDLL:
         h.twist_hidden_mask.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p]
         h.twist_gather_subnets.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_void_p]
         h.twist_aggregate.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_uint32, C.c_void_p]
+        h.twist_layernorm_workspace_bytes.restype = C.c_size_t
+        h.twist_layernorm_workspace_bytes.argtypes = [C.c_int32, C.c_int32, C.c_int32]
         for name in ("twist_subnet_ffn_fwd", "twist_subnet_ffn_bwd", "twist_subnet_attn_proj_fwd",
-                     "twist_subnet_attn_proj_bwd", "twist_attn_core_fwd", "twist_attn_core_bwd"):
+                     "twist_subnet_attn_proj_bwd", "twist_attn_core_fwd", "twist_attn_core_bwd",
+                     "twist_layernorm_fwd", "twist_layernorm_bwd"):
             getattr(h, name).argtypes = [C.c_void_p, C.c_void_p]
         h.twist_mse_workspace_bytes.restype = C.c_size_t
         h.twist_mse_workspace_bytes.argtypes = [C.c_int32]
@@ -137,7 +150,8 @@ def lib() -> C.CDLL:
         for name in EXPORTS:
             f = getattr(h, name)
             if name not in ("twist_abi_version", "twist_strerror", "twist_last_cuda_error",
-                            "twist_mse_workspace_bytes", "twist_fused_loss_workspace_bytes"):
+                            "twist_mse_workspace_bytes", "twist_fused_loss_workspace_bytes",
+                            "twist_layernorm_workspace_bytes"):
                 f.restype = C.c_int32
         _lib_handle = h
     return _lib_handle
@@ -298,6 +312,31 @@ def twist_attn_core_fwd(a: AttnCoreArgs):
 
 def twist_attn_core_bwd(a: AttnCoreArgs):
     _check(lib().twist_attn_core_bwd(C.byref(a), _stream()), "twist_attn_core_bwd")
+
+
+def layernorm_args(dtype, n_subnets, tokens, d_model, eps, lr=0.0, opt: Optional[Optimizer] = None, **t) -> LayerNormArgs:
+    """Marshals twist_layernorm_args (tensors by keyword: x, y, mean, rstd, gamma, beta, dy, dx, dx_residual,
+    dgamma, dbeta, ws, m_gamma, v_gamma, m_beta, v_beta)."""
+    names = ["x", "y", "mean", "rstd", "gamma", "beta", "dy", "dx", "dx_residual", "dgamma", "dbeta", "ws"]
+    moments = ["m_gamma", "v_gamma", "m_beta", "v_beta"]
+    unknown = set(t) - set(names) - set(moments)
+    assert not unknown, unknown
+    a = LayerNormArgs(dtype, n_subnets, tokens, d_model, eps, lr, *[_ptr(t.get(n)) for n in names],
+                      _ws_bytes(t.get("ws")), opt if opt is not None else Optimizer(), *[_ptr(t.get(n)) for n in moments])
+    a._keepalive = list(t.values())
+    return a
+
+
+def twist_layernorm_workspace_bytes(n_subnets: int, tokens: int, d_model: int) -> int:
+    return lib().twist_layernorm_workspace_bytes(n_subnets, tokens, d_model)
+
+
+def twist_layernorm_fwd(a: LayerNormArgs):
+    _check(lib().twist_layernorm_fwd(C.byref(a), _stream()), "twist_layernorm_fwd")
+
+
+def twist_layernorm_bwd(a: LayerNormArgs):
+    _check(lib().twist_layernorm_bwd(C.byref(a), _stream()), "twist_layernorm_bwd")
 
 
 def twist_mse_workspace_bytes(n_subnets: int) -> int:

@@ -1,13 +1,19 @@
-"""Sequencing of one TwIST round on one GPU (BLOCKWISE composition).
+"""Sequencing of one TwIST round on one GPU.
 
 This module only allocates device buffers (torch) and calls the C ABI in order:
 sample masks -> per layer { gather -> K local steps (forward, MSE, backward with fused
 SGD) for the FFN block, the QKV projection and the output projection -> aggregate }.
 Every arithmetic step runs in the CUDA library; nothing here computes on tensors.
 
-Layers are streamed: slices, masters and activations exist for one layer at a time,
-which is what lets the 7B-shaped workloads fit (per layer ~2.4 GB of slices + masters
-at S=8, keep 25%, instead of 78 GB for all 32 layers).
+Layers are streamed (BLOCKWISE, RoundEngine): slices, masters and activations exist for one
+layer at a time, which is what lets the 7B-shaped workloads fit (per layer ~2.4 GB of slices
++ masters at S=8, keep 25%, instead of 78 GB for all 32 layers).  StackEngine chains the
+layers (attention core, skip connections, optionally the two layer normalisations).
+
+A layer is either partitioned (N_sub = the workload's keep counts) or shared (N_sub = N_full
+in both kinds: every worker holds the whole layer and the aggregate is the plain mean); the two
+kinds have different slice sizes, so the engine keeps one set of buffers per kind ("geometry")
+and binds the set of the layer it is working on.
 """
 from __future__ import annotations
 
@@ -18,11 +24,32 @@ from typing import Dict, List, Optional, Tuple
 import torch
 
 from . import binding as B
-from .inputs import DTYPE_BF16, FFN_SWIGLU, Workload
+from .inputs import DTYPE_BF16, FFN_SWIGLU, LN_PARAMS, Workload
 
 
 def _tdtype(w: Workload):
     return torch.bfloat16 if w.dtype == DTYPE_BF16 else torch.float32
+
+
+class Geometry:
+    """Slice sizes and output scales of a layer whose subnets keep `ffn_keep` FFN blocks and `head_keep` heads."""
+
+    def __init__(self, w: Workload, ffn_keep: int, head_keep: int):
+        self.ffn_keep, self.head_keep = ffn_keep, head_keep
+        self.f_sub = ffn_keep * w.ffn_block
+        self.g = 2 if w.ffn_kind == FFN_SWIGLU else 1
+        self.gf = self.g * self.f_sub
+        self.alpha_f = math.sqrt(w.n_ffn_blocks / ffn_keep)            # activation-shift scale, Sec. 3.4
+        self.kv_max = self.a_sub = self.nq = 0
+        self.alpha_a = 1.0
+        if w.n_heads > 0:
+            self.kv_max = min(w.n_kv_heads, head_keep)
+            self.a_sub = head_keep * w.d_head
+            self.nq = self.a_sub + 2 * self.kv_max * w.d_head
+            self.alpha_a = math.sqrt(w.n_heads / head_keep)
+
+
+_SLICES = ("w_gu", "w_down", "w_qkv", "w_o")
 
 
 class RoundEngine:
@@ -38,9 +65,8 @@ class RoundEngine:
         self.fuse_loss = fuse_loss
         self.store_outputs = store_outputs or not fuse_loss or w.dtype != DTYPE_BF16
         td, dev = _tdtype(w), self.dev
-        S, T, d, f = w.n_subnets, w.tokens, w.d_model, w.f_sub
+        S, T, d = w.n_subnets, w.tokens, w.d_model
         self.g = 2 if w.ffn_kind == FFN_SWIGLU else 1
-        gf = self.g * f
         L, F = w.n_layers, w.d_ff
         self.has_attn = w.n_heads > 0
         bf16 = w.dtype == DTYPE_BF16
@@ -54,9 +80,6 @@ class RoundEngine:
             self.full["gate"] = self.full_gu[:, :F]
         if self.has_attn:
             H, Hkv, dh = w.n_heads, w.n_kv_heads, w.d_head
-            self.kv_max = min(Hkv, w.head_keep)
-            self.a_sub = w.head_keep * dh
-            self.nq = self.a_sub + 2 * self.kv_max * dh
             self.full["qkv"] = torch.empty(L, (H + 2 * Hkv) * dh, d, dtype=td, device=dev)
             self.full["o"] = torch.empty(L, H * dh, d, dtype=td, device=dev)
         self.full_f32, self.full_gu_f32 = None, None
@@ -65,14 +88,12 @@ class RoundEngine:
             self.full_f32 = {m: (self.full_gu_f32[:, (self.g - 1) * F:] if m == "up" else
                                  self.full_gu_f32[:, :F] if m == "gate" else
                                  torch.empty(v.shape, dtype=torch.float32, device=dev)) for m, v in self.full.items()}
-        # blueprints and aggregator index data, all layers
+        # aggregator index data (the same shape for every layer), all layers
         nb = w.n_ffn_blocks
         i32 = dict(dtype=torch.int32, device=dev)
-        self.idx_ffn = torch.empty(L, S, w.ffn_keep, **i32)
         self.cover_ffn = torch.empty(L, nb, **i32)
         self.pos_ffn = torch.empty(L, S, nb, **i32)
         if self.has_attn:
-            self.idx_head = torch.empty(L, S, w.head_keep, **i32)
             self.cover_head = torch.empty(L, w.n_heads, **i32)
             self.pos_head = torch.empty(L, S, w.n_heads, **i32)
             self.kv_idx = torch.empty(L, S, w.n_kv_heads, **i32)
@@ -80,56 +101,109 @@ class RoundEngine:
             self.kv_cols = torch.empty(L, S, **i32)
             self.kv_cover = torch.empty(L, w.n_kv_heads, **i32)
             self.kv_pos = torch.empty(L, S, w.n_kv_heads, **i32)
-        # slices of one layer (+ fp32 masters in bf16 mode)
-        def sl(rows):
-            t = torch.empty(S, rows, d, dtype=td, device=dev)
-            return t, (torch.empty(S, rows, d, dtype=torch.float32, device=dev) if bf16 else None)
-        self.w_gu, self.w_gu_m = sl(gf)
-        self.w_down, self.w_down_m = sl(f)
-        if self.has_attn:
-            self.w_qkv, self.w_qkv_m = sl(self.nq)
-            self.w_o, self.w_o_m = sl(self.a_sub)
-        # Adam moments live with the worker's copy of the slice: allocated here, zeroed at every gather
         self.adam = w.optimizer == "adam"
         assert not self.adam or bf16, "the fused Adam update exists for the bf16 dtype"
-        self.moment_names = []
-        if self.adam:
-            for n in ("w_gu", "w_down") + (("w_qkv", "w_o") if self.has_attn else ()):
-                for tag in ("_m1", "_m2"):
-                    setattr(self, n + tag, torch.zeros_like(getattr(self, n + "_m")))
-                    self.moment_names.append(n + tag)
-        # activations of one (layer, step)
+        # geometries: partitioned layers, and shared layers (N_sub = N_full) if the workload has any
+        self.shared_layers = frozenset(w.shared_layers)
+        assert all(0 <= l < L for l in self.shared_layers)
+        self.geo: Dict[str, Geometry] = {"part": Geometry(w, w.ffn_keep, w.head_keep)}
+        if self.shared_layers:
+            self.geo["shared"] = Geometry(w, w.n_ffn_blocks, w.n_heads)
+        self.bufs: Dict[str, Dict[str, object]] = {}
+        self.batches: Dict[str, Dict[str, List[torch.Tensor]]] = {k: {"Tq": [], "A": []} for k in self.geo}
+        # activations of one (layer, step) whose size does not depend on the geometry
         act = lambda width: torch.empty(S, T, width, dtype=td, device=dev)
-        self.pre, self.dpre, self.hh = act(gf), act(gf), act(f)
         self.y, self.dy = act(d), act(d)
         self.dx = act(d) if compute_dx else None
-        if self.has_attn:
-            self.qkv_out, self.dqkv = act(self.nq), act(self.nq)
-            self.da = act(self.a_sub) if compute_dx else None
-        f32 = lambda *shape: torch.empty(*shape, dtype=torch.float32, device=dev)
-        self.dw_gu = f32(S, gf, d) if self.dump_grads else None
-        self.dw_down = f32(S, f, d) if self.dump_grads else None
-        if self.has_attn:
-            self.dw_qkv = f32(S, self.nq, d) if self.dump_grads else None
-            self.dw_o = f32(S, self.a_sub, d) if self.dump_grads else None
         self.loss = torch.zeros(L, 3, max(1, w.local_steps), S, dtype=torch.float32, device=dev)
-        ws_bytes = max(B.twist_mse_workspace_bytes(S),
-                       B.twist_fused_loss_workspace_bytes(S, T, max(d, self.nq if self.has_attn else 0)))
+        nq_max = max(gm.nq for gm in self.geo.values())
+        ws_bytes = max(B.twist_mse_workspace_bytes(S), B.twist_fused_loss_workspace_bytes(S, T, max(d, nq_max)))
         self.ws = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
-        self.alpha_f = math.sqrt(w.n_ffn_blocks / w.ffn_keep)
-        self.alpha_a = math.sqrt(w.n_heads / w.head_keep) if self.has_attn else 1.0
-        # batches: lists over the local step k of [S][T][width] tensors
+        # batches: lists over the local step k of [S][T][width] tensors (Tq and A: per geometry, see the properties)
         self.X: List[torch.Tensor] = []
         self.Td: List[torch.Tensor] = []
-        self.Tq: List[torch.Tensor] = []
-        self.A: List[torch.Tensor] = []
         self.launches = 0
         # what the gather reads as blueprint, what the aggregate reads as ranks, and the activation mask of the FFN
         # calls: the sampler's outputs and none, unless a subclass (Masked TwIST) substitutes its own
-        self.gather_idx_ffn, self.agg_pos_ffn, self.h_mask = self.idx_ffn, self.pos_ffn, None
+        self._gather_idx_override, self._agg_pos_override, self.h_mask = None, None, None
         # optional per-phase CUDA-event timing (events on the launching stream)
         self.timing = False
         self.events: Dict[str, List[Tuple[torch.cuda.Event, torch.cuda.Event]]] = {}
+        self._cur = None
+        self._use_kind("part")
+
+    # ------------------------------------------------------------------ geometries
+    def _alloc(self, kind: str) -> Dict[str, object]:
+        """Buffers of one geometry: blueprints, slices (+ fp32 masters and Adam moments in bf16 mode), the
+        activations and gradient dumps whose width depends on the kept sizes."""
+        w, gm, dev, td = self.w, self.geo[kind], self.dev, _tdtype(self.w)
+        S, T, d, L = w.n_subnets, w.tokens, w.d_model, w.n_layers
+        bf16 = w.dtype == DTYPE_BF16
+        i32 = dict(dtype=torch.int32, device=dev)
+        b: Dict[str, object] = {"idx_ffn": torch.empty(L, S, gm.ffn_keep, **i32)}
+        if self.has_attn:
+            b["idx_head"] = torch.empty(L, S, gm.head_keep, **i32)
+        rows = {"w_gu": gm.gf, "w_down": gm.f_sub, "w_qkv": gm.nq, "w_o": gm.a_sub}
+        names = _SLICES if self.has_attn else _SLICES[:2]
+        moments = []
+        for n in names:
+            b[n] = torch.empty(S, rows[n], d, dtype=td, device=dev)
+            b[n + "_m"] = torch.empty(S, rows[n], d, dtype=torch.float32, device=dev) if bf16 else None
+            if self.adam:      # Adam moments live with the worker's copy of the slice: zeroed at every gather
+                for tag in ("_m1", "_m2"):
+                    b[n + tag] = torch.zeros_like(b[n + "_m"])
+                    moments.append(n + tag)
+            b["d" + n] = torch.empty(S, rows[n], d, dtype=torch.float32, device=dev) if self.dump_grads else None
+        b["moment_names"] = moments
+        act = lambda width: torch.empty(S, T, width, dtype=td, device=dev)
+        b["pre"], b["dpre"], b["hh"] = act(gm.gf), act(gm.gf), act(gm.f_sub)
+        if self.has_attn:
+            b["qkv_out"], b["dqkv"] = act(gm.nq), act(gm.nq)
+            b["da"] = act(gm.a_sub) if self.compute_dx else None
+        return b
+
+    def _use_kind(self, kind: str):
+        if kind == self._cur:
+            return
+        if kind not in self.bufs:
+            self.bufs[kind] = self._alloc(kind)
+        gm = self.geo[kind]
+        for n in ("f_sub", "gf", "a_sub", "nq", "kv_max", "alpha_f", "alpha_a", "ffn_keep", "head_keep"):
+            setattr(self, n, getattr(gm, n))
+        for n, t in self.bufs[kind].items():
+            setattr(self, n, t)
+        self._cur = kind
+
+    def kind_of(self, l: int) -> str:
+        return "shared" if l in self.shared_layers else "part"
+
+    def _use(self, l: int):
+        """Binds the sizes and buffers of layer l's geometry onto the engine."""
+        self._use_kind(self.kind_of(l))
+
+    @property
+    def Tq(self) -> List[torch.Tensor]:      # targets of the QKV block (width nq) of the bound geometry
+        return self.batches[self._cur]["Tq"]
+
+    @Tq.setter
+    def Tq(self, v):
+        self.batches[self._cur]["Tq"] = v
+
+    @property
+    def A(self) -> List[torch.Tensor]:       # inputs of the output projection (width a') of the bound geometry
+        return self.batches[self._cur]["A"]
+
+    @A.setter
+    def A(self, v):
+        self.batches[self._cur]["A"] = v
+
+    @property
+    def gather_idx_ffn(self):
+        return self.idx_ffn if self._gather_idx_override is None else self._gather_idx_override
+
+    @property
+    def agg_pos_ffn(self):
+        return self.pos_ffn if self._agg_pos_override is None else self._agg_pos_override
 
     @contextmanager
     def _timed(self, name: str):
@@ -147,45 +221,62 @@ class RoundEngine:
         return {k: (sum(a.elapsed_time(b) for a, b in v), len(v)) for k, v in self.events.items()}
 
     # ------------------------------------------------------------------ steps of the round
+    def _layer_runs(self):
+        """Maximal runs of consecutive layers of the same kind: (first layer, count, kind)."""
+        runs, l, L = [], 0, self.w.n_layers
+        while l < L:
+            k, n = self.kind_of(l), 1
+            while l + n < L and self.kind_of(l + n) == k:
+                n += 1
+            runs.append((l, n, k))
+            l += n
+        return runs
+
     def sample_masks(self, rnd: int):
         w = self.w
         with self._timed("sample_masks"):
-            B.twist_sample_masks(w.seed_mask, rnd, 0, w.n_layers, B.KIND_FFN, w.n_ffn_blocks, w.n_subnets, w.ffn_keep,
-                                 list(w.common_ffn), w.sample_mode, self.idx_ffn, self.cover_ffn, self.pos_ffn)
-            self.launches += 2
-            if self.has_attn:
-                B.twist_sample_masks(w.seed_mask, rnd, 0, w.n_layers, B.KIND_HEAD, w.n_heads, w.n_subnets,
-                                     w.head_keep, list(w.common_heads), w.sample_mode, self.idx_head, self.cover_head,
-                                     self.pos_head)
-                B.twist_kv_groups(self.idx_head, w.n_layers, w.n_subnets, w.head_keep, w.n_heads, w.n_kv_heads,
-                                  w.d_head, self.kv_idx, self.kv_count, self.kv_cols, self.kv_cover, self.kv_pos)
-                self.launches += 4
+            for l0, n, kind in self._layer_runs():
+                self._use_kind(kind)
+                sl = slice(l0, l0 + n)
+                B.twist_sample_masks(w.seed_mask, rnd, l0, n, B.KIND_FFN, w.n_ffn_blocks, w.n_subnets, self.ffn_keep,
+                                     list(w.common_ffn), w.sample_mode, self.idx_ffn[sl], self.cover_ffn[sl],
+                                     self.pos_ffn[sl])
+                self.launches += 2
+                if self.has_attn:
+                    B.twist_sample_masks(w.seed_mask, rnd, l0, n, B.KIND_HEAD, w.n_heads, w.n_subnets, self.head_keep,
+                                         list(w.common_heads), w.sample_mode, self.idx_head[sl], self.cover_head[sl],
+                                         self.pos_head[sl])
+                    B.twist_kv_groups(self.idx_head[sl], n, w.n_subnets, self.head_keep, w.n_heads, w.n_kv_heads,
+                                      w.d_head, self.kv_idx[sl], self.kv_count[sl], self.kv_cols[sl], self.kv_cover[sl],
+                                      self.kv_pos[sl])
+                    self.launches += 4
 
     def gather_layer(self, l: int, which=("ffn", "attn")):
+        self._use(l)
         w, d = self.w, self.w.d_model
-        f, gf = w.f_sub, self.g * w.f_sub
+        f, gf, keep = self.f_sub, self.gf, self.ffn_keep
+        nb = w.n_ffn_blocks
         segs = []
         if "ffn" in which:
             if self.g == 2:
                 segs.append(B.gather_segment(self.full["gate"][l], self.w_gu, self.w_gu_m, self.gather_idx_ffn[l], None,
-                                             w.ffn_keep, w.ffn_keep, w.ffn_block, 0, gf * d, 0, w.n_ffn_blocks))
+                                             keep, keep, w.ffn_block, 0, gf * d, 0, nb))
             segs.append(B.gather_segment(self.full["up"][l], self.w_gu, self.w_gu_m, self.gather_idx_ffn[l], None,
-                                         w.ffn_keep, w.ffn_keep, w.ffn_block, 0, gf * d, f if self.g == 2 else 0,
-                                         w.n_ffn_blocks))
+                                         keep, keep, w.ffn_block, 0, gf * d, f if self.g == 2 else 0, nb))
             segs.append(B.gather_segment(self.full["down"][l], self.w_down, self.w_down_m, self.gather_idx_ffn[l], None,
-                                         w.ffn_keep, w.ffn_keep, w.ffn_block, 0, f * d, 0, w.n_ffn_blocks))
+                                         keep, keep, w.ffn_block, 0, f * d, 0, nb))
         if self.has_attn and "attn" in which:
-            H, Hkv, dh = w.n_heads, w.n_kv_heads, w.d_head
+            H, Hkv, dh, hk = w.n_heads, w.n_kv_heads, w.d_head, self.head_keep
             qkv = self.full["qkv"][l]
-            segs.append(B.gather_segment(qkv, self.w_qkv, self.w_qkv_m, self.idx_head[l], None, w.head_keep,
-                                         w.head_keep, dh, 0, self.nq * d, 0, H))
+            segs.append(B.gather_segment(qkv, self.w_qkv, self.w_qkv_m, self.idx_head[l], None, hk, hk, dh, 0,
+                                         self.nq * d, 0, H))
             segs.append(B.gather_segment(qkv, self.w_qkv, self.w_qkv_m, self.kv_idx[l], self.kv_count[l], Hkv,
                                          self.kv_max, dh, H * dh, self.nq * d, self.a_sub, Hkv))
             segs.append(B.gather_segment(qkv, self.w_qkv, self.w_qkv_m, self.kv_idx[l], self.kv_count[l], Hkv,
                                          self.kv_max, dh, (H + Hkv) * dh, self.nq * d, self.a_sub + self.kv_max * dh,
                                          Hkv))
-            segs.append(B.gather_segment(self.full["o"][l], self.w_o, self.w_o_m, self.idx_head[l], None, w.head_keep,
-                                         w.head_keep, dh, 0, self.a_sub * d, 0, H))
+            segs.append(B.gather_segment(self.full["o"][l], self.w_o, self.w_o_m, self.idx_head[l], None, hk, hk, dh, 0,
+                                         self.a_sub * d, 0, H))
         with self._timed("gather"):
             B.twist_gather_subnets(segs, w.n_subnets, d, w.dtype)
             for n in self.moment_names:        # a fresh worker state: first and second moments start at zero
@@ -193,8 +284,9 @@ class RoundEngine:
         self.launches += 1
 
     def aggregate_layer(self, l: int, live: int = 0xFFFFFFFF, which=("ffn", "attn")):
+        self._use(l)
         w, d = self.w, self.w.d_model
-        f, gf = w.f_sub, self.g * w.f_sub
+        f, gf, keep = self.f_sub, self.gf, self.ffn_keep
         bf16 = w.dtype == DTYPE_BF16
         f32 = (lambda m: self.full_f32[m][l]) if self.full_f32 is not None else (lambda m: None)
         sub = lambda lo, master: master if bf16 else lo
@@ -204,25 +296,25 @@ class RoundEngine:
             if self.g == 2:
                 segs.append(B.aggregate_segment(self.full["gate"][l], f32("gate"), sub(self.w_gu, self.w_gu_m),
                                                 self.cover_ffn[l], self.agg_pos_ffn[l], nb, w.ffn_block, 0, gf * d, 0,
-                                                w.ffn_keep))
+                                                keep))
             segs.append(B.aggregate_segment(self.full["up"][l], f32("up"), sub(self.w_gu, self.w_gu_m),
                                             self.cover_ffn[l], self.agg_pos_ffn[l], nb, w.ffn_block, 0, gf * d,
-                                            f if self.g == 2 else 0, w.ffn_keep))
+                                            f if self.g == 2 else 0, keep))
             segs.append(B.aggregate_segment(self.full["down"][l], f32("down"), sub(self.w_down, self.w_down_m),
                                             self.cover_ffn[l], self.agg_pos_ffn[l], nb, w.ffn_block, 0, f * d, 0,
-                                            w.ffn_keep))
+                                            keep))
         if self.has_attn and "attn" in which:
             H, Hkv, dh = w.n_heads, w.n_kv_heads, w.d_head
             q_sub = sub(self.w_qkv, self.w_qkv_m)
             segs.append(B.aggregate_segment(self.full["qkv"][l], f32("qkv"), q_sub, self.cover_head[l],
-                                            self.pos_head[l], H, dh, 0, self.nq * d, 0, w.head_keep))
+                                            self.pos_head[l], H, dh, 0, self.nq * d, 0, self.head_keep))
             segs.append(B.aggregate_segment(self.full["qkv"][l], f32("qkv"), q_sub, self.kv_cover[l], self.kv_pos[l],
                                             Hkv, dh, H * dh, self.nq * d, self.a_sub, self.kv_max))
             segs.append(B.aggregate_segment(self.full["qkv"][l], f32("qkv"), q_sub, self.kv_cover[l], self.kv_pos[l],
                                             Hkv, dh, (H + Hkv) * dh, self.nq * d, self.a_sub + self.kv_max * dh,
                                             self.kv_max))
             segs.append(B.aggregate_segment(self.full["o"][l], f32("o"), sub(self.w_o, self.w_o_m), self.cover_head[l],
-                                            self.pos_head[l], H, dh, 0, self.a_sub * d, 0, w.head_keep))
+                                            self.pos_head[l], H, dh, 0, self.a_sub * d, 0, self.head_keep))
         with self._timed("aggregate"):
             B.twist_aggregate(segs, w.n_subnets, d, w.dtype, live)
         self.launches += 1
@@ -246,10 +338,11 @@ class RoundEngine:
         self.launches += 2
 
     def ffn_step(self, l: int, k: int, lr: Optional[float] = None):
+        self._use(l)
         w = self.w
         lr = w.lr if lr is None else lr
         fused = dict(tgt=self.Td[k], loss=self.loss[l, 0, k], loss_ws=self.ws) if self.fuse_loss else {}
-        a = B.ffn_args(w.ffn_kind, w.dtype, w.n_subnets, w.tokens, w.d_model, w.f_sub, self.alpha_f, lr,
+        a = B.ffn_args(w.ffn_kind, w.dtype, w.n_subnets, w.tokens, w.d_model, self.f_sub, self.alpha_f, lr,
                        x=self.X[k], w_gu=self.w_gu, w_down=self.w_down, w_gu_master=self.w_gu_m,
                        w_down_master=self.w_down_m, pre=self.pre, hh=self.hh,
                        y=self.y if self.store_outputs else None, dy=self.dy, dpre=self.dpre,
@@ -267,6 +360,7 @@ class RoundEngine:
         self.launches += (2 + 3 + (1 if self.compute_dx else 0)) if bf16 else (3 + 4 + (1 if self.compute_dx else 0) + 2)
 
     def qkv_step(self, l: int, k: int, lr: Optional[float] = None):
+        self._use(l)
         w = self.w
         lr = w.lr if lr is None else lr
         ragged = self.w.n_kv_heads != self.w.n_heads
@@ -287,6 +381,7 @@ class RoundEngine:
         self.launches += 1 + 1 + (1 if self.compute_dx else 0) + (0 if w.dtype == DTYPE_BF16 else 1)
 
     def o_step(self, l: int, k: int, lr: Optional[float] = None):
+        self._use(l)
         w = self.w
         lr = w.lr if lr is None else lr
         fused = dict(tgt=self.Td[k], loss=self.loss[l, 2, k], loss_ws=self.ws) if self.fuse_loss else {}
@@ -316,9 +411,10 @@ class RoundEngine:
         """Evaluation mode for subnets (Sec. 4.2): forward only, on the slices gathered for layer l, with the
         subnet's own scale (an engine built with other keep counts than the training run evaluates a mismatched
         subnet ratio).  Returns the losses [blocks][S] (device); the caller averages over the workers."""
+        self._use(l)
         w = self.w
         assert self.fuse_loss, "evaluation uses the loss fused into the forward kernels"
-        a = B.ffn_args(w.ffn_kind, w.dtype, w.n_subnets, w.tokens, w.d_model, w.f_sub, self.alpha_f, 0.0, x=self.X[k],
+        a = B.ffn_args(w.ffn_kind, w.dtype, w.n_subnets, w.tokens, w.d_model, self.f_sub, self.alpha_f, 0.0, x=self.X[k],
                        w_gu=self.w_gu, w_down=self.w_down, pre=self.pre, hh=self.hh,
                        y=self.y if self.store_outputs else None, dy=self.dy, tgt=self.Td[k], loss=self.loss[l, 0, k],
                        loss_ws=self.ws)
@@ -383,17 +479,18 @@ class MaskedRoundEngine(RoundEngine):
 
     def __init__(self, w: Workload, device: str = "cuda", **kw):
         from dataclasses import replace as _replace
-        assert w.dtype == DTYPE_BF16 and w.n_heads == 0, "bf16 FFN-only workloads"
+        assert w.dtype == DTYPE_BF16 and w.n_heads == 0 and not w.shared_layers, "bf16 FFN-only workloads"
         nb = w.n_ffn_blocks
         super().__init__(_replace(w, ffn_keep=nb), device=device, **kw)      # storage: full-width slices
         self.true_w = w
         L, S = w.n_layers, w.n_subnets
         i32 = dict(dtype=torch.int32, device=self.dev)
         self.idx_ffn = torch.empty(L, S, w.ffn_keep, **i32)                   # the sampled blueprints
+        self.bufs["part"]["idx_ffn"] = self.idx_ffn
         ident = torch.arange(nb, **i32).expand(L, S, nb).contiguous()
-        self.gather_idx_ffn, self.agg_pos_ffn = ident, ident                  # every worker copies / returns every block
+        self._gather_idx_override, self._agg_pos_override = ident, ident      # every worker copies / returns every block
         self.h_mask = torch.zeros(S, w.d_ff, dtype=torch.uint8, device=self.dev)
-        self.alpha_f = math.sqrt(nb / w.ffn_keep)                             # the subnet's scale (Sec. 3.4)
+        self.alpha_f = self.geo["part"].alpha_f = math.sqrt(nb / w.ffn_keep)  # the subnet's scale (Sec. 3.4)
 
     def sample_masks(self, rnd: int):
         w = self.true_w
@@ -417,7 +514,8 @@ class HybridRoundEngine(RoundEngine):
     (The full model's gate and up rows lie back to back, so a full-width layer is a valid w_gu operand.)"""
 
     def __init__(self, w: Workload, device: str = "cuda", **kw):
-        assert w.dtype == DTYPE_BF16 and w.n_heads == 0 and w.n_subnets >= 2, "bf16 FFN-only workloads"
+        assert w.dtype == DTYPE_BF16 and w.n_heads == 0 and w.n_subnets >= 2 and not w.shared_layers, \
+            "bf16 FFN-only workloads"
         super().__init__(w, device=device, keep_f32_full=True, **kw)
         F, T = w.d_ff, w.tokens
         g, dev = self.g, self.dev
@@ -432,7 +530,7 @@ class HybridRoundEngine(RoundEngine):
     def gather_layer(self, l: int, which=("ffn",)):
         """Slices of workers 1 .. S-1 only; the central worker's activation mask for this layer."""
         w, d = self.w, self.w.d_model
-        f, gf = w.f_sub, self.g * w.f_sub
+        f, gf = self.f_sub, self.gf
         idx = self.idx_ffn[l, 1:]
         segs = []
         for m, off, dst, dst_m, stride in ([("gate", 0, self.w_gu, self.w_gu_m, gf)] if self.g == 2 else []) + [
@@ -482,7 +580,7 @@ class HybridRoundEngine(RoundEngine):
 
     def aggregate_layer(self, l: int, live: int = 0xFFFFFFFF, which=("ffn",)):
         w, d = self.w, self.w.d_model
-        f, gf = w.f_sub, self.g * w.f_sub
+        f, gf = self.f_sub, self.gf
         nb = w.n_ffn_blocks
         segs = []
         for m, off, sub, stride in ([("gate", 0, self.w_gu_m, gf)] if self.g == 2 else []) + [
@@ -497,11 +595,13 @@ class HybridRoundEngine(RoundEngine):
 
 class StackEngine(RoundEngine):
     """One TwIST round in the chained (STACK) composition: every local step runs all layers,
-    x <- x + alpha_a * O(core(QKV(x))),  x <- x + alpha_f * FFN(x),  with one loss on the final x.
+    x <- x + alpha_a * O(core(QKV(LN_a(x)))),  x <- x + alpha_f * FFN(LN_f(x)),  with one loss on the final x
+    (App. A, Transformer Layer Architecture; the two layer normalisations only when the workload asks for them).
 
     All layers' slices and saved activations are resident at once (the backward pass needs them), so
     this engine is for the stack-shaped workloads whose activations fit; the streamed RoundEngine
     covers the per-block workloads.  Like RoundEngine it only allocates buffers and calls the C ABI.
+    The normalised activations are not kept: the backward pass forms them again from the saved inputs.
     """
 
     def __init__(self, w: Workload, n_seqs: int, seq_len: int, device: str = "cuda", keep_f32_full: bool = False):
@@ -509,42 +609,111 @@ class StackEngine(RoundEngine):
         super().__init__(w, device=device, keep_f32_full=keep_f32_full, compute_dx=True, fuse_loss=False)
         self.n_seqs, self.seq_len = n_seqs, seq_len
         S, T, d, L = w.n_subnets, w.tokens, w.d_model, w.n_layers
-        gf, f = self.g * w.f_sub, w.f_sub
         dev, bf = self.dev, torch.bfloat16
-        names = ("w_gu", "w_gu_m", "w_down", "w_down_m", "w_qkv", "w_qkv_m", "w_o", "w_o_m") + tuple(self.moment_names)
-        self.slices = [{n: (getattr(self, n) if l == 0 else torch.empty_like(getattr(self, n))) for n in names}
-                       for l in range(L)]
+        for kind in self.geo:
+            self._use_kind(kind)
+        self._use_kind("part")
+        # slices of every layer: the first layer of a kind uses the geometry's own buffers
+        self.slices: List[Dict[str, torch.Tensor]] = []
+        seen = set()
+        for l in range(L):
+            kind = self.kind_of(l)
+            b = self.bufs[kind]
+            names = [n for n in b if (n in _SLICES or n.endswith(("_m", "_m1", "_m2"))) and torch.is_tensor(b[n])]
+            self.slices.append({n: (b[n] if kind not in seen else torch.empty_like(b[n])) for n in names})
+            seen.add(kind)
         act = lambda width: torch.empty(S, T, width, dtype=bf, device=dev)
+        geo = [self.geo[self.kind_of(l)] for l in range(L)]
         self.x = [act(d) for _ in range(L + 1)]
         self.x_mid = [act(d) for _ in range(L)]
-        self.qkv_l = [act(self.nq) for _ in range(L)]
-        self.a_l = [act(self.a_sub) for _ in range(L)]
-        self.pre_l = [act(gf) for _ in range(L)]
-        self.hh_l = [act(f) for _ in range(L)]
-        self.lse = [torch.empty(S, w.head_keep, T, dtype=torch.float32, device=dev) for _ in range(L)]
-        self.delta = torch.empty(S, w.head_keep, T, dtype=torch.float32, device=dev)
+        self.qkv_l = [act(geo[l].nq) for l in range(L)]
+        self.a_l = [act(geo[l].a_sub) for l in range(L)]
+        self.pre_l = [act(geo[l].gf) for l in range(L)]
+        self.hh_l = [act(geo[l].f_sub) for l in range(L)]
+        self.lse = [torch.empty(S, geo[l].head_keep, T, dtype=torch.float32, device=dev) for l in range(L)]
+        self.delta = torch.empty(S, max(gm.head_keep for gm in geo), T, dtype=torch.float32, device=dev)
         self.grad = [act(d), act(d)]            # gradient w.r.t. the residual stream (ping-pong)
         self.stack_loss = torch.zeros(max(1, w.local_steps), S, dtype=torch.float32, device=dev)
         self.gqa = w.n_kv_heads != w.n_heads
+        # layer normalisation (App. A): shared parameters, one copy per worker and layer, statistics per token
+        self.ln = w.layer_norm
+        if self.ln:
+            f32 = lambda *shape: torch.empty(*shape, dtype=torch.float32, device=dev)
+            self.full_ln = {n: f32(L, d) for n in LN_PARAMS}
+            self.ln_w = [{n: f32(S, d) for n in LN_PARAMS} for _ in range(L)]
+            self.ln_mom = [{n + t: torch.zeros(S, d, dtype=torch.float32, device=dev) for n in LN_PARAMS
+                            for t in ("_m1", "_m2")} if self.adam else {} for _ in range(L)]
+            self.ln_stat = [{n: f32(S, T) for n in ("mean_a", "rstd_a", "mean_f", "rstd_f")} for _ in range(L)]
+            self.x_ln, self.d_ln = act(d), act(d)         # a normalised activation / the gradient w.r.t. one
+            self.ln_ws = torch.empty(B.twist_layernorm_workspace_bytes(S, T, d), dtype=torch.uint8, device=dev)
+            self.ln_zero_idx = torch.zeros(S, 1, dtype=torch.int32, device=dev)
+            mask = (1 << S) - 1
+            self.ln_cover = torch.tensor([mask - (1 << 32) if mask >= (1 << 31) else mask], dtype=torch.int32, device=dev)
 
     def _bind(self, l: int):
+        self._use(l)
         for n, t in self.slices[l].items():
             setattr(self, n, t)
 
     def _core_args(self, l: int, **t):
         w = self.w
         extra = dict(head_idx=self.idx_head[l], kv_pos=self.kv_pos[l], kv_count=self.kv_count[l]) if self.gqa else {}
-        return B.attn_core_args(w.dtype, w.n_subnets, self.n_seqs, self.seq_len, w.head_keep, self.kv_max, w.d_head,
+        return B.attn_core_args(w.dtype, w.n_subnets, self.n_seqs, self.seq_len, self.head_keep, self.kv_max, w.d_head,
                                 w.n_heads, w.n_kv_heads, **extra, **t)
 
+    # ------------------------------------------------------------------ layer normalisation
+    def _ln_args(self, l: int, which: str, lr: float = 0.0, k: int = 0, **t):
+        w = self.w
+        p, st = self.ln_w[l], self.ln_stat[l]
+        kw = {}
+        if self.adam and lr != 0.0:
+            m = self.ln_mom[l]
+            kw = dict(opt=B.adam(k + 1, w.beta1, w.beta2, w.adam_eps), m_gamma=m[f"ln_{which}_g_m1"],
+                      v_gamma=m[f"ln_{which}_g_m2"], m_beta=m[f"ln_{which}_b_m1"], v_beta=m[f"ln_{which}_b_m2"])
+        return B.layernorm_args(w.dtype, w.n_subnets, w.tokens, w.d_model, w.ln_eps, lr, gamma=p[f"ln_{which}_g"],
+                                beta=p[f"ln_{which}_b"], mean=st["mean_" + which], rstd=st["rstd_" + which], **kw, **t)
+
+    def _ln_fwd(self, l: int, which: str, x, y):
+        with self._timed("ln_fwd"):
+            B.twist_layernorm_fwd(self._ln_args(l, which, x=x, y=y))
+        self.launches += 1
+
+    def _ln_bwd(self, l: int, which: str, k: int, lr: float, x, dy, dx, residual):
+        with self._timed("ln_bwd"):
+            B.twist_layernorm_bwd(self._ln_args(l, which, lr, k, x=x, dy=dy, dx=dx, dx_residual=residual, ws=self.ln_ws))
+        self.launches += 3
+
+    def gather_ln(self, l: int):
+        """The shared normalisation parameters are broadcast: every worker gets a copy (Sec. 3.2)."""
+        w, d = self.w, self.w.d_model
+        segs = [B.gather_segment(self.full_ln[n][l], self.ln_w[l][n], None, self.ln_zero_idx, None, 1, 1, 1, 0, d, 0, 1)
+                for n in LN_PARAMS]
+        B.twist_gather_subnets(segs, w.n_subnets, d, B.FP32)
+        for t in self.ln_mom[l].values():
+            t.zero_()
+        self.launches += 1
+
+    def aggregate_ln(self, l: int, live: int = 0xFFFFFFFF):
+        """Held by every worker: the aggregator's formula (Sec. 3.3) is the plain mean over the S copies."""
+        w, d = self.w, self.w.d_model
+        segs = [B.aggregate_segment(self.full_ln[n][l], None, self.ln_w[l][n], self.ln_cover, self.ln_zero_idx, 1, 1, 0,
+                                    d, 0, 1) for n in LN_PARAMS]
+        B.twist_aggregate(segs, w.n_subnets, d, B.FP32, live)
+        self.launches += 1
+
+    # ------------------------------------------------------------------ the chained local step
     def forward(self, k: int):
         w = self.w
         S, T, d = w.n_subnets, w.tokens, w.d_model
         self.x[0].copy_(self.X[k])
         for l in range(w.n_layers):
             self._bind(l)
+            x_a = self.x[l]
+            if self.ln:
+                self._ln_fwd(l, "a", self.x[l], self.x_ln)
+                x_a = self.x_ln
             with self._timed("qkv_fwd"):
-                B.twist_subnet_attn_proj_fwd(B.proj_args(B.PROJ_QKV, w.dtype, S, T, d, self.nq, 1.0, 0.0, in_=self.x[l],
+                B.twist_subnet_attn_proj_fwd(B.proj_args(B.PROJ_QKV, w.dtype, S, T, d, self.nq, 1.0, 0.0, in_=x_a,
                                                          w=self.w_qkv, out=self.qkv_l[l]))
             with self._timed("core_fwd"):
                 B.twist_attn_core_fwd(self._core_args(l, qkv=self.qkv_l[l], out=self.a_l[l], lse=self.lse[l]))
@@ -552,9 +721,13 @@ class StackEngine(RoundEngine):
                 B.twist_subnet_attn_proj_fwd(B.proj_args(B.PROJ_O, w.dtype, S, T, d, self.a_sub, self.alpha_a, 0.0,
                                                          in_=self.a_l[l], w=self.w_o, out=self.x_mid[l],
                                                          out_residual=self.x[l]))
+            x_f = self.x_mid[l]
+            if self.ln:
+                self._ln_fwd(l, "f", self.x_mid[l], self.x_ln)
+                x_f = self.x_ln
             with self._timed("ffn_fwd"):
-                B.twist_subnet_ffn_fwd(B.ffn_args(w.ffn_kind, w.dtype, S, T, d, w.f_sub, self.alpha_f, 0.0,
-                                                  x=self.x_mid[l], w_gu=self.w_gu, w_down=self.w_down, pre=self.pre_l[l],
+                B.twist_subnet_ffn_fwd(B.ffn_args(w.ffn_kind, w.dtype, S, T, d, self.f_sub, self.alpha_f, 0.0,
+                                                  x=x_f, w_gu=self.w_gu, w_down=self.w_down, pre=self.pre_l[l],
                                                   hh=self.hh_l[l], y=self.x[l + 1], y_residual=self.x_mid[l]))
             self.launches += 5
 
@@ -565,13 +738,23 @@ class StackEngine(RoundEngine):
         g, g_mid = self.grad
         for l in reversed(range(w.n_layers)):
             self._bind(l)
+            # FFN block.  With the normalisation: its input is formed again, its input gradient goes through the
+            # normalisation's backward, which also adds the gradient arriving over the skip connection.
+            x_f = self.x_mid[l]
+            if self.ln:
+                self._ln_fwd(l, "f", self.x_mid[l], self.x_ln)
+                x_f = self.x_ln
             with self._timed("ffn_bwd"):
-                B.twist_subnet_ffn_bwd(B.ffn_args(w.ffn_kind, w.dtype, S, T, d, w.f_sub, self.alpha_f, lr,
-                                                  x=self.x_mid[l], w_gu=self.w_gu, w_down=self.w_down,
+                B.twist_subnet_ffn_bwd(B.ffn_args(w.ffn_kind, w.dtype, S, T, d, self.f_sub, self.alpha_f, lr,
+                                                  x=x_f, w_gu=self.w_gu, w_down=self.w_down,
                                                   w_gu_master=self.w_gu_m, w_down_master=self.w_down_m,
-                                                  pre=self.pre_l[l], hh=self.hh_l[l], dy=g, dpre=self.dpre, dx=g_mid,
-                                                  dx_residual=g, dw_gu=self.dw_gu, dw_down=self.dw_down,
+                                                  pre=self.pre_l[l], hh=self.hh_l[l], dy=g, dpre=self.dpre,
+                                                  dx=self.d_ln if self.ln else g_mid,
+                                                  dx_residual=None if self.ln else g, dw_gu=self.dw_gu,
+                                                  dw_down=self.dw_down,
                                                   **self._opt(k, ("_gu", "w_gu"), ("_down", "w_down"))))
+            if self.ln:
+                self._ln_bwd(l, "f", k, lr, self.x_mid[l], self.d_ln, g_mid, g)
             with self._timed("o_bwd"):
                 B.twist_subnet_attn_proj_bwd(B.proj_args(B.PROJ_O, w.dtype, S, T, d, self.a_sub, self.alpha_a, lr,
                                                          in_=self.a_l[l], w=self.w_o, w_master=self.w_o_m, d_out=g_mid,
@@ -579,10 +762,18 @@ class StackEngine(RoundEngine):
             with self._timed("core_bwd"):
                 B.twist_attn_core_bwd(self._core_args(l, qkv=self.qkv_l[l], out=self.a_l[l], lse=self.lse[l],
                                                       d_out=self.da, d_qkv=self.dqkv, delta=self.delta))
+            x_a = self.x[l]
+            if self.ln:
+                self._ln_fwd(l, "a", self.x[l], self.x_ln)
+                x_a = self.x_ln
             with self._timed("qkv_bwd"):
-                B.twist_subnet_attn_proj_bwd(B.proj_args(B.PROJ_QKV, w.dtype, S, T, d, self.nq, 1.0, lr, in_=self.x[l],
-                                                         w=self.w_qkv, w_master=self.w_qkv_m, d_out=self.dqkv, d_in=g,
-                                                         d_in_residual=g_mid, dw=self.dw_qkv, **self._opt(k, ("", "w_qkv"))))
+                B.twist_subnet_attn_proj_bwd(B.proj_args(B.PROJ_QKV, w.dtype, S, T, d, self.nq, 1.0, lr, in_=x_a,
+                                                         w=self.w_qkv, w_master=self.w_qkv_m, d_out=self.dqkv,
+                                                         d_in=self.d_ln if self.ln else g,
+                                                         d_in_residual=None if self.ln else g_mid, dw=self.dw_qkv,
+                                                         **self._opt(k, ("", "w_qkv"))))
+            if self.ln:
+                self._ln_bwd(l, "a", k, lr, self.x[l], self.d_ln, g, g_mid)
             self.launches += 4 + 2 + 3 + 2
 
     def local_step(self, k: int, lr: Optional[float] = None):
@@ -594,13 +785,18 @@ class StackEngine(RoundEngine):
         self.launches += 2
         self.backward(k, lr)
 
+    def _gather_all(self):
+        for l in range(self.w.n_layers):
+            self._bind(l)
+            self.gather_layer(l)
+            if self.ln:
+                self.gather_ln(l)
+
     def extract(self, rnd: int):
         """Deployment (Sec. 4.2): sample blueprints as in training and gather every layer's dense slices; the S
         extracted subnets are then resident (self.slices) for forward-only inference."""
         self.sample_masks(rnd)
-        for l in range(self.w.n_layers):
-            self._bind(l)
-            self.gather_layer(l)
+        self._gather_all()
 
     def evaluate(self, k: int) -> torch.Tensor:
         """Evaluation mode for subnets (Sec. 4.2): forward only through the whole stack of every extracted subnet on
@@ -617,11 +813,11 @@ class StackEngine(RoundEngine):
         """Resample, gather every layer, K local steps through the whole stack, aggregate every layer."""
         w = self.w
         self.sample_masks(rnd)
-        for l in range(w.n_layers):
-            self._bind(l)
-            self.gather_layer(l)
+        self._gather_all()
         for k in range(w.local_steps):
             self.local_step(k)
         for l in range(w.n_layers):
             self._bind(l)
             self.aggregate_layer(l)
+            if self.ln:
+                self.aggregate_ln(l)

@@ -56,6 +56,9 @@ class Workload:
     beta2: float = 0.999
     adam_eps: float = 1e-8
     n_seqs: int = 1       # sequences per batch (tokens = n_seqs * sequence length); matters to the attention core only
+    shared_layers: Tuple[int, ...] = field(default_factory=tuple)   # layers every worker holds whole (N_sub = N_full)
+    layer_norm: bool = False   # chained composition only: the two layer normalisations of the pre-LN layer
+    ln_eps: float = 1e-5
 
     @property
     def n_ffn_blocks(self) -> int:
@@ -162,6 +165,19 @@ def weight(w: Workload, layer: int, mat: int) -> np.ndarray:
     rows = {MAT_GATE: w.d_ff, MAT_UP: w.d_ff, MAT_DOWN: w.d_ff,
             MAT_QKV: (w.n_heads + 2 * w.n_kv_heads) * w.d_head, MAT_O: w.n_heads * w.d_head}[mat]
     return normal(w.seed_w, layer * 8 + mat, (rows, w.d_model), 0.02, w.dtype)
+
+
+LN_PARAMS = ("ln_a_g", "ln_a_b", "ln_f_g", "ln_f_b")     # gain / bias of the attention and the FFN normalisation
+
+
+def ln_param(w: Workload, layer: int, name: str, spread: float = 0.1) -> np.ndarray:
+    """Layer-normalisation parameter [d_model] (float32).  The customary initial values are gain 1 and bias 0;
+    `spread` adds a seeded N(0, spread^2) perturbation so that tests can tell the parameters apart (0: exact
+    initial values)."""
+    base = np.float32(1.0 if name.endswith("_g") else 0.0)
+    if spread == 0:
+        return np.full(w.d_model, base, dtype=np.float32)
+    return base + normal(w.seed_w, layer * 8 + 5 + 65536 * (1 + LN_PARAMS.index(name)), (w.d_model,), spread, DTYPE_FP32)
 
 
 def batch(w: Workload, kind: int, rnd: int, subnet: int, step: int, width: int, tokens: int | None = None):

@@ -494,16 +494,27 @@ def _load_full(eng, w):
 
 
 def _load_batches(eng, w, rnd):
+    """Seeded batches of round rnd on the device and, for the oracle, on the host: store[(kind, k)] for the
+    partitioned layers' widths, store[(kind, k, width)] for every width (shared layers have their own QKV / A widths)."""
     td = torch.bfloat16 if w.dtype == I.DTYPE_BF16 else torch.float32
     S = w.n_subnets
-    eng.X, eng.Td, eng.Tq, eng.A = [], [], [], []
+    eng.X, eng.Td = [], []
     store = {}
     for k in range(w.local_steps):
-        for kind, width, dst in ((I.BATCH_X, w.d_model, eng.X), (I.BATCH_TGT_D, w.d_model, eng.Td)) + (
-                ((I.BATCH_TGT_QKV, eng.nq, eng.Tq), (I.BATCH_A, eng.a_sub, eng.A)) if eng.has_attn else ()):
-            arr = np.stack([I.batch(w, kind, rnd, s, k, width) for s in range(S)])
-            store[(kind, k)] = arr
+        for kind, dst in ((I.BATCH_X, eng.X), (I.BATCH_TGT_D, eng.Td)):
+            arr = np.stack([I.batch(w, kind, rnd, s, k, w.d_model) for s in range(S)])
+            store[(kind, k)] = store[(kind, k, w.d_model)] = arr
             dst.append(dev(arr, td))
+    if eng.has_attn:
+        for gk, gm in eng.geo.items():
+            eng.batches[gk] = {"Tq": [], "A": []}
+            for k in range(w.local_steps):
+                for kind, width, name in ((I.BATCH_TGT_QKV, gm.nq, "Tq"), (I.BATCH_A, gm.a_sub, "A")):
+                    arr = np.stack([I.batch(w, kind, rnd, s, k, width) for s in range(S)])
+                    store[(kind, k, width)] = arr
+                    if gk == "part":
+                        store[(kind, k)] = arr
+                    eng.batches[gk][name].append(dev(arr, td))
     return store
 
 
@@ -524,18 +535,20 @@ def _run_round_and_compare(B, w, rnd=0, tol_dw=5e-2, engine_cls=None, **engine_k
     for l in range(w.n_layers):
         bp = o.layer_blueprints(w, rnd, l)
 
-        def get_batch(kind, rnd_, s, k, width):
-            arr = store[(kind, k)][s]
+        gm = eng.geo[eng.kind_of(l)]
+
+        def get_batch(kind, rnd_, s, k, width, bp=bp, gm=gm):
             if kind == I.BATCH_TGT_QKV and ragged:     # device layout [Q | K pad | V pad] -> oracle [Q | K | V]
+                arr = store[(kind, k, gm.nq)][s]
                 kc = bp["kv_count"][s] * w.d_head
-                kvw = eng.kv_max * w.d_head
-                return np.concatenate([arr[:, :eng.a_sub], arr[:, eng.a_sub:eng.a_sub + kc],
-                                       arr[:, eng.a_sub + kvw:eng.a_sub + kvw + kc]], axis=1)
-            return arr
+                kvw = gm.kv_max * w.d_head
+                return np.concatenate([arr[:, :gm.a_sub], arr[:, gm.a_sub:gm.a_sub + kc],
+                                       arr[:, gm.a_sub + kvw:gm.a_sub + kvw + kc]], axis=1)
+            return store[(kind, k, width)][s]
 
         full64 = {m: v.astype(np.float64) for m, v in full_np[l].items()}
         new, new_shadow, _, losses = o.round_blockwise_layer(w, full64, get_batch, rnd, l, lowp)
-        assert np.array_equal(eng.idx_ffn[l].cpu().numpy(), bp["ffn"])
+        assert np.array_equal(eng.bufs[eng.kind_of(l)]["idx_ffn"][l].cpu().numpy(), bp["ffn"])
         for m in eng.full:
             res = (eng.full_f32[m][l] if lowp else eng.full[m][l]).cpu().numpy().astype(np.float64)
             delta_w, delta_g = new[m] - full64[m], res - full64[m]
@@ -892,3 +905,78 @@ def test_a_bounded_wait_that_runs_out_reports_a_timeout_and_leaves_the_device_us
         B.twist_selftest_wait(10 ** 10)                         # limits beyond 0.1 s are refused
     _ffn_case(B, I.FFN_SWIGLU, I.DTYPE_BF16, S=2, T=256, d=256, f=256, alpha=2.0, lr=0.5, seed=41)
     check_status(B)
+
+
+def test_blockwise_round_with_a_shared_layer_matches_the_oracle(B):
+    """Sec. 5 Setup: some layers are shared (N_sub = N_full in both kinds): every worker holds and trains the whole
+    layer, scale 1, and the aggregate is the plain mean over the S workers; the other layers are partitioned."""
+    w = replace(I.scaled_twin(I.PRESETS[3], d_model=256, d_ff=688, d_head=8, tokens=256, n_layers=3, local_steps=2),
+                shared_layers=(0, 2))
+    eng, _ = _run_round_and_compare(B, w)
+    full_mask = (1 << w.n_subnets) - 1
+    cover = eng.cover_ffn.cpu().numpy().view(np.uint32)
+    assert np.all(cover[0] == full_mask) and np.all(cover[2] == full_mask) and not np.all(cover[1] == full_mask)
+    assert eng.bufs["shared"]["w_gu"].shape[1] == 2 * w.d_ff and eng.bufs["part"]["w_gu"].shape[1] == 2 * w.f_sub
+    assert eng.geo["shared"].alpha_f == 1.0 and eng.geo["shared"].alpha_a == 1.0
+
+
+# --------------------------------------------------------------------------------------------- layer normalisation
+
+@pytest.mark.parametrize("S,T,d,adam", [(2, 77, 328, False), (3, 300, 768, True), (1, 130, 4096, False), (2, 9, 8, False)])
+def test_layernorm_parity(B, S, T, d, adam):
+    """App. A, Layer Normalization, forward and backward against the oracle: outputs and input gradients (bf16) to the
+    bar of the other stored activations, statistics and parameter gradients (fp32 sums) much tighter, the
+    optimiser step on gamma / b against the oracle's step on the device's own gradients."""
+    bf = torch.bfloat16
+    eps, lr = 1e-5, 0.05
+    X = I.normal(91, 1, (S, T, d), 2.0, I.DTYPE_BF16) + np.float32(0.5)
+    X = I.f32_from_bf16_bits(I.bf16_bits_from_f32(X))
+    dY = I.normal(91, 2, (S, T, d), 1e-2, I.DTYPE_BF16)
+    R = I.normal(91, 3, (S, T, d), 1e-2, I.DTYPE_BF16)
+    g0 = (1.0 + I.normal(91, 4, (S, d), 0.2, I.DTYPE_FP32)).astype(np.float32)
+    b0 = I.normal(91, 5, (S, d), 0.2, I.DTYPE_FP32)
+    x, dy, r = dev(X, bf), dev(dY, bf), dev(R, bf)
+    gamma, beta = dev(g0), dev(b0)
+    y, dx = torch.zeros_like(x), torch.zeros_like(x)
+    mean = torch.zeros(S, T, dtype=torch.float32, device="cuda")
+    rstd = torch.zeros_like(mean)
+    dg, db = torch.zeros_like(gamma), torch.zeros_like(gamma)
+    ws = torch.empty(B.twist_layernorm_workspace_bytes(S, T, d), dtype=torch.uint8, device="cuda")
+    mom = {n: torch.zeros_like(gamma) for n in ("m_gamma", "v_gamma", "m_beta", "v_beta")} if adam else {}
+    opt = dict(opt=B.adam(1, 0.9, 0.99, 1e-3), **mom) if adam else {}
+    a = B.layernorm_args(B.BF16, S, T, d, eps, lr, x=x, y=y, mean=mean, rstd=rstd, gamma=gamma, beta=beta, dy=dy, dx=dx,
+                         dx_residual=r, dgamma=dg, dbeta=db, ws=ws, **opt)
+    B.twist_layernorm_fwd(a)
+    B.twist_layernorm_bwd(a)
+    torch.cuda.synchronize()
+    check_status(B)
+    for s in range(S):
+        Xs = X[s].astype(np.float64)
+        Yw, saved = o.layer_norm_fwd(Xs, g0[s].astype(np.float64), b0[s].astype(np.float64), True, eps)
+        assert close(host(y[s]), Yw, GEMM_TOL) if d >= 32 else rel_fro(host(y[s]), Yw) < GEMM_TOL
+        assert np.allclose(mean[s].cpu().numpy(), Xs.mean(axis=1), rtol=1e-5, atol=1e-6)
+        assert np.allclose(rstd[s].cpu().numpy(), saved["rstd"][:, 0], rtol=1e-5)
+        dXw, dgw, dbw = o.layer_norm_bwd(dY[s].astype(np.float64), saved, g0[s].astype(np.float64), True,
+                                         residual=R[s].astype(np.float64))
+        assert rel_fro(host(dx[s]), dXw) < GEMM_TOL
+        assert rel_fro(host(dx[s]) - R[s], dXw - R[s]) < 4 * GEMM_TOL        # the normalisation's own part of the sum
+        assert rel_fro(host(dg[s]), dgw) < 1e-4 and rel_fro(host(db[s]), dbw) < 1e-4
+        if adam:
+            for name, p0, grad, m_, v_ in (("gamma", g0[s], dg[s], mom["m_gamma"][s], mom["v_gamma"][s]),
+                                           ("beta", b0[s], db[s], mom["m_beta"][s], mom["v_beta"][s])):
+                gdev = grad.double().cpu().numpy()
+                new, m1, v1, _ = o.adam(p0.astype(np.float64), np.zeros(d), np.zeros(d), gdev, 1, lr, 0.9, 0.99, 1e-3, False)
+                got = (gamma if name == "gamma" else beta)[s].double().cpu().numpy()
+                assert rel_fro(got - p0, new - p0) < 1e-3, name
+                assert rel_fro(host(m_), m1) < 1e-5 and rel_fro(host(v_), v1) < 1e-5
+        else:
+            assert rel_fro(host(gamma[s]) - g0[s], -lr * dgw) < 1e-3
+            assert rel_fro(host(beta[s]) - b0[s], -lr * dbw) < 1e-3
+    # in place: dx may overwrite dy
+    dy2 = dy.clone()
+    gamma.copy_(dev(g0)); beta.copy_(dev(b0))
+    a2 = B.layernorm_args(B.BF16, S, T, d, eps, 0.0, x=x, mean=mean, rstd=rstd, gamma=gamma, beta=beta, dy=dy2, dx=dy2,
+                          dx_residual=r, ws=ws)
+    B.twist_layernorm_bwd(a2)
+    torch.cuda.synchronize()
+    assert torch.equal(dy2, dx)

@@ -157,13 +157,22 @@ def test_skip_connection_epilogues(B):
         assert rel_fro(host(d_in[s]), o.qkv_bwd(f64(dQ), f64(X), f64(W), True, residual=f64(R2))[0]) < GEMM_TOL
 
 
-@pytest.mark.parametrize("cfg,dims,n_seqs", [
-    (2, dict(d_model=192, d_ff=528, d_head=16, tokens=192, n_layers=2, local_steps=2), 2),     # GELU, 12 heads keep 6
-    (3, dict(d_model=256, d_ff=688, d_head=8, tokens=200, n_layers=3, local_steps=2), 2),      # SwiGLU, GQA 32 heads / 4 groups
+@pytest.mark.parametrize("cfg,dims,n_seqs,extra", [
+    (2, dict(d_model=192, d_ff=528, d_head=16, tokens=192, n_layers=2, local_steps=2), 2, {}),     # GELU, 12 heads keep 6
+    (3, dict(d_model=256, d_ff=688, d_head=8, tokens=200, n_layers=3, local_steps=2), 2, {}),      # SwiGLU, GQA 32 heads / 4 groups
+    # the pre-LN layer of App. A (both layer normalisations, their parameters trained and averaged)
+    # (a learning rate at which the change of gamma / b is well above the fp32 spacing of their values)
+    (2, dict(d_model=192, d_ff=528, d_head=16, tokens=192, n_layers=2, local_steps=2), 2, dict(layer_norm=True, lr=1.0)),
+    (3, dict(d_model=256, d_ff=688, d_head=8, tokens=200, n_layers=3, local_steps=2), 2,
+     dict(layer_norm=True, optimizer="adam", lr=1e-2, adam_eps=3e-3)),
+    # shared first and last layers (Sec. 5 Setup: N_sub = N_full there), with and without the normalisations
+    (3, dict(d_model=256, d_ff=688, d_head=8, tokens=200, n_layers=3, local_steps=2), 2, dict(shared_layers=(0, 2))),
+    (2, dict(d_model=192, d_ff=528, d_head=16, tokens=192, n_layers=3, local_steps=1), 2,
+     dict(shared_layers=(2,), layer_norm=True, lr=1.0)),
 ])
-def test_stack_round_of_a_scaled_twin_matches_the_oracle(B, cfg, dims, n_seqs):
+def test_stack_round_of_a_scaled_twin_matches_the_oracle(B, cfg, dims, n_seqs, extra):
     from paper_2511_03983_b200.engine import StackEngine
-    w = I.scaled_twin(I.PRESETS[cfg], **dims)
+    w = replace(I.scaled_twin(I.PRESETS[cfg], **dims), **extra)
     seq_len = w.tokens // n_seqs
     eng = StackEngine(w, n_seqs, seq_len, keep_f32_full=True)
     mats = {"gate": I.MAT_GATE, "up": I.MAT_UP, "down": I.MAT_DOWN, "qkv": I.MAT_QKV, "o": I.MAT_O}
@@ -172,6 +181,10 @@ def test_stack_round_of_a_scaled_twin_matches_the_oracle(B, cfg, dims, n_seqs):
         layer = {m: I.weight(w, l, mats[m]) for m in eng.full}
         for m, v in layer.items():
             eng.full[m][l].copy_(dev(v, torch.bfloat16))
+        if w.layer_norm:
+            for n in I.LN_PARAMS:
+                layer[n] = I.ln_param(w, l, n)
+                eng.full_ln[n][l].copy_(dev(layer[n]))
         full_np.append(layer)
     store = {}
     for k in range(w.local_steps):
@@ -188,12 +201,21 @@ def test_stack_round_of_a_scaled_twin_matches_the_oracle(B, cfg, dims, n_seqs):
     want_loss = np.array(losses).T
     assert np.allclose(got_loss, want_loss, rtol=2e-2), (got_loss, want_loss)
     for l in range(w.n_layers):
-        assert np.array_equal(eng.idx_ffn[l].cpu().numpy(), bps[l]["ffn"])
-        assert np.array_equal(eng.idx_head[l].cpu().numpy(), bps[l]["head"])
+        assert np.array_equal(eng.bufs[eng.kind_of(l)]["idx_ffn"][l].cpu().numpy(), bps[l]["ffn"])
+        assert np.array_equal(eng.bufs[eng.kind_of(l)]["idx_head"][l].cpu().numpy(), bps[l]["head"])
+        if l in w.shared_layers:
+            assert bps[l]["ffn"].shape[1] == w.n_ffn_blocks and bps[l]["head"].shape[1] == w.n_heads
         for m in eng.full:
             res = eng.full_f32[m][l].cpu().numpy().astype(np.float64)
             dw, dg = new[l][m] - full64[l][m], res - full64[l][m]
             assert rel_fro(dg, dw) < 5e-2, (l, m, rel_fro(dg, dw))
+        if w.layer_norm:
+            for n in I.LN_PARAMS:
+                res = eng.full_ln[n][l].cpu().numpy().astype(np.float64)
+                dw, dg = new[l][n] - full64[l][n], res - full64[l][n]
+                # stored in fp32: half a spacing of the values themselves is the floor of what a difference can show
+                floor = 2.0 ** -24 * np.linalg.norm(np.maximum(np.abs(full64[l][n]), 2.0 ** -6)) / np.linalg.norm(dw)
+                assert rel_fro(dg, dw) < 5e-2 + floor, (l, n, rel_fro(dg, dw), floor)
 
 
 @pytest.mark.parametrize("mode", ["stack", "blockwise"])
