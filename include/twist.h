@@ -114,6 +114,21 @@ int32_t twist_hidden_mask(const uint32_t* cover /*device*/, int32_t n_full, int3
  * query heads is.  Writes kv_idx [n_layers][S][n_kv_heads] (sorted kept groups, then -1),
  * kv_count [n_layers][S], kv_cols [n_layers][S] = kv_count * d_head (valid K or V columns of the
  * subnet's projection), kv_cover [n_layers][n_kv_heads], kv_pos [n_layers][S][n_kv_heads]; all device. */
+/* Column mask of a masked worker's full-width QKV projection (Sec. 4.1) from the aggregator's cover masks:
+ * for subnets subnet_begin .. +n_subnets-1, mask[s][c] = 1 iff column c of [Q heads | K groups | V groups] belongs to
+ * a head (head_cover, uint32 [n_heads]) or KV group (kv_cover, uint32 [n_kv_heads]) the subnet holds;
+ * count[s] = number of marked columns.  mask [n_subnets][(n_heads + 2 n_kv_heads) d_head] uint8, count [n_subnets]
+ * int32; all device, one layer. */
+int32_t twist_qkv_col_mask(const uint32_t* head_cover, const uint32_t* kv_cover, int32_t n_heads, int32_t n_kv_heads,
+                           int32_t d_head, int32_t subnet_begin, int32_t n_subnets, uint8_t* mask, int32_t* count,
+                           void* stream);
+
+/* Head mask on the attention core's output (Sec. 4.1: the module output is multiplied element-wise by the mask):
+ * out[s][t][c] = mask[s][c] ? in[s][t][c] : 0 for bf16 activations [S][T][width] and a uint8 mask [S][width]
+ * (width a multiple of 8; in == out allowed).  All device. */
+int32_t twist_apply_col_mask(const void* in, const uint8_t* mask, void* out, int32_t n_subnets, int32_t tokens,
+                             int32_t width, void* stream);
+
 int32_t twist_kv_groups(const int32_t* head_idx, int32_t n_layers, int32_t n_subnets, int32_t head_keep,
                         int32_t n_heads, int32_t n_kv_heads, int32_t d_head, int32_t* kv_idx, int32_t* kv_count,
                         int32_t* kv_cols, uint32_t* kv_cover, int32_t* kv_pos, void* stream);
@@ -294,6 +309,16 @@ typedef struct {
   const void* d_in_residual;   /* device [S][T][d] */
   twist_optimizer opt;         /* bwd: optimiser of the fused update */
   float *m, *v;                /* device fp32 Adam moments of w [S][n][d] */
+  /* Optional head mask of a masked worker (Sec. 4.1, Masked TwIST: the worker holds the full-width projections and
+   * behaves like the subnet of the heads it "holds"): device uint8 [S][n], 1 for the rows of W (columns of the QKV
+   * output / of the output projection's input) that belong to held heads, constant over aligned groups of 8.
+   *   TWIST_PROJ_QKV fwd with fused loss: only marked columns count -- loss = mean over T x valid_cols[s] elements,
+   *     zero gradient elsewhere, so the rows of W of the other heads get exactly zero gradient;
+   *     valid_cols[s] must then hold the number of marked columns (twist_qkv_col_mask writes both).
+   *   TWIST_PROJ_O bwd: d_in is multiplied by the mask.  (The output projection's input `in` is expected to be
+   *     masked already, as the attention core's output under a head mask is.)
+   * NULL: no mask.  bf16 dtype only. */
+  const uint8_t* col_mask;
 } twist_proj_args;
 
 int32_t twist_subnet_attn_proj_fwd(const twist_proj_args* a /*host*/, void* stream);

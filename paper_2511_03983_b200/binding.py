@@ -32,7 +32,7 @@ EXPORTS = [
     "twist_subnet_attn_proj_fwd", "twist_subnet_attn_proj_bwd", "twist_mse_workspace_bytes", "twist_mse_fwd_bwd",
     "twist_mse_fwd_bwd_noalloc", "twist_fused_loss_workspace_bytes", "twist_attn_core_fwd", "twist_attn_core_bwd",
     "twist_hidden_mask", "twist_selftest_wait", "twist_layernorm_workspace_bytes", "twist_layernorm_fwd",
-    "twist_layernorm_bwd",
+    "twist_layernorm_bwd", "twist_qkv_col_mask", "twist_apply_col_mask",
 ]
 
 
@@ -87,7 +87,7 @@ class ProjArgs(C.Structure):
                 ("loss", C.c_void_p), ("loss_ws", C.c_void_p), ("loss_ws_bytes", C.c_size_t),
                 ("valid_cols", C.c_void_p), ("seg_begin", C.c_int32), ("seg_width", C.c_int32),
                 ("out_residual", C.c_void_p), ("d_in_residual", C.c_void_p), ("opt", Optimizer), ("m", C.c_void_p),
-                ("v", C.c_void_p)]
+                ("v", C.c_void_p), ("col_mask", C.c_void_p)]
 
 
 class AttnCoreArgs(C.Structure):
@@ -130,6 +130,9 @@ def lib() -> C.CDLL:
         h.twist_kv_groups.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int32,
                                       C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         h.twist_hidden_mask.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p]
+        h.twist_qkv_col_mask.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int32,
+                                         C.c_void_p, C.c_void_p, C.c_void_p]
+        h.twist_apply_col_mask.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_void_p]
         h.twist_gather_subnets.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_void_p]
         h.twist_aggregate.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_uint32, C.c_void_p]
         h.twist_layernorm_workspace_bytes.restype = C.c_size_t
@@ -237,6 +240,16 @@ def twist_hidden_mask(cover, n_full, block_rows, subnet_begin, n_subnets, mask):
            "twist_hidden_mask")
 
 
+def twist_qkv_col_mask(head_cover, kv_cover, n_heads, n_kv_heads, d_head, subnet_begin, n_subnets, mask, count):
+    _check(lib().twist_qkv_col_mask(_ptr(head_cover), _ptr(kv_cover), n_heads, n_kv_heads, d_head, subnet_begin,
+                                    n_subnets, _ptr(mask), _ptr(count), _stream()), "twist_qkv_col_mask")
+
+
+def twist_apply_col_mask(in_, mask, out, n_subnets, tokens, width):
+    _check(lib().twist_apply_col_mask(_ptr(in_), _ptr(mask), _ptr(out), n_subnets, tokens, width, _stream()),
+           "twist_apply_col_mask")
+
+
 def twist_aggregate(segs: Sequence[AggregateSegment], n_subnets, d, dtype, live_subnets=0xFFFFFFFF):
     arr = (AggregateSegment * len(segs))(*segs)
     _check(lib().twist_aggregate(C.cast(arr, C.c_void_p), len(segs), n_subnets, d, dtype, live_subnets, _stream()),
@@ -277,12 +290,12 @@ def proj_args(which, dtype, n_subnets, tokens, d_model, n, out_scale, lr=0.0, se
     """Marshals twist_proj_args.  tgt / loss / loss_ws (and the optional column mask valid_cols,
     seg_begin, seg_width) request the fused loss of the forward call."""
     names = ["in_", "w", "w_master", "out", "d_out", "d_in", "dw", "tgt", "loss", "loss_ws"]
-    unknown = set(t) - set(names) - {"valid_cols", "out_residual", "d_in_residual", "m", "v"}
+    unknown = set(t) - set(names) - {"valid_cols", "out_residual", "d_in_residual", "m", "v", "col_mask"}
     assert not unknown, unknown
     a = ProjArgs(which, dtype, n_subnets, tokens, d_model, n, out_scale, lr, *[_ptr(t.get(n)) for n in names],
                  _ws_bytes(t.get("loss_ws")), _ptr(t.get("valid_cols")), seg_begin, seg_width,
                  _ptr(t.get("out_residual")), _ptr(t.get("d_in_residual")), opt if opt is not None else Optimizer(),
-                 _ptr(t.get("m")), _ptr(t.get("v")))
+                 _ptr(t.get("m")), _ptr(t.get("v")), _ptr(t.get("col_mask")))
     a._keepalive = list(t.values())
     return a
 

@@ -75,7 +75,8 @@ struct GemmParams {
   float* adam_m;        // ADAM: first / second moment of the group's weights, fp32 [g][M][N]
   float* adam_v;
   float beta1, beta2, adam_eps, bias1, bias2;   // ADAM: decay rates, epsilon, 1 / (1 - beta^t)
-  const uint8_t* hmask;  // activation epilogues: per group N bytes, 1 = column active, 0 = masked out; may be null
+  const uint8_t* hmask;  // activation and STORE epilogues: per group N bytes, 1 = column active, 0 = masked out; may be null
+  const uint8_t* col_mask;   // MSE: per group N bytes, 1 = column counts in the loss (valid_cols[g] = how many do); may be null
   float* dw;            // SGD: optional fp32 gradient dump [g][M][N].  MSE: partial sums, 16 per tile (2 CTAs x 8 warps)
   const int32_t* valid_cols;   // MSE: valid columns per column group and subnet [groups], or null (all valid)
   int seg_begin, seg_width;    // MSE: columns [0, seg_begin) valid, then groups of seg_width columns (see twist_mse_fwd_bwd)
@@ -588,21 +589,27 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           for (int q = 0; q < 4; ++q) {
             const uint32_t* r = a.r0 + 8 * q;
             float hm[8] = {1.f, 1.f, 1.f, 1.f, 1.f, 1.f, 1.f, 1.f};
-            if constexpr (EPI == EPI_SWIGLU_FWD || EPI == EPI_ACT_FWD || EPI == EPI_DSWIGLU || EPI == EPI_DACT) {
+            if constexpr (EPI == EPI_SWIGLU_FWD || EPI == EPI_ACT_FWD || EPI == EPI_DSWIGLU || EPI == EPI_DACT ||
+                          EPI == EPI_STORE) {
               if (p.hmask && n + 8 * q < p.N) mask8(p.hmask, g, p.N, n + 8 * q, hm);     // uniform branch
             }
             if constexpr (EPI == EPI_STORE) {
-              sts128(piece(b0, q), make_uint4(pack2(p.scale * __uint_as_float(r[0]), p.scale * __uint_as_float(r[1])),
-                                              pack2(p.scale * __uint_as_float(r[2]), p.scale * __uint_as_float(r[3])),
-                                              pack2(p.scale * __uint_as_float(r[4]), p.scale * __uint_as_float(r[5])),
-                                              pack2(p.scale * __uint_as_float(r[6]), p.scale * __uint_as_float(r[7]))));
+              float sc[8];
+#pragma unroll
+              for (int e = 0; e < 8; ++e) sc[e] = p.scale * hm[e];
+              sts128(piece(b0, q), make_uint4(pack2(sc[0] * __uint_as_float(r[0]), sc[1] * __uint_as_float(r[1])),
+                                              pack2(sc[2] * __uint_as_float(r[2]), sc[3] * __uint_as_float(r[3])),
+                                              pack2(sc[4] * __uint_as_float(r[4]), sc[5] * __uint_as_float(r[5])),
+                                              pack2(sc[6] * __uint_as_float(r[6]), sc[7] * __uint_as_float(r[7]))));
             } else if constexpr (kIsMse) {
               const uint4 tv = lds128(piece(b0, q));
               const uint32_t tw[4] = {tv.x, tv.y, tv.z, tv.w};
               // validity is constant over aligned groups of 8 columns (seg_begin, seg_width, vc are multiples of 8)
               const int col = n + 8 * q;
               bool cv = row_ok && col < p.N;
-              if (p.valid_cols && col >= p.seg_begin) {     // masked column groups (uniform branch; few groups: no division)
+              if (p.col_mask) {                             // arbitrary column set (constant over aligned groups of 8)
+                cv = cv && p.col_mask[(long long)g * p.N + col] != 0;
+              } else if (p.valid_cols && col >= p.seg_begin) {     // masked column groups (uniform branch; few groups: no division)
                 int rel = col - p.seg_begin;
                 while (rel >= p.seg_width) rel -= p.seg_width;
                 cv = cv && rel < vc;

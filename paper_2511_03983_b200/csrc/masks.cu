@@ -167,6 +167,43 @@ __global__ void hidden_mask_kernel(const uint32_t* __restrict__ cover, long long
   for (int s = 0; s < n_subnets; ++s) mask[(long long)s * rows + r] = (uint8_t)((c >> (subnet_begin + s)) & 1u);
 }
 
+// One CTA per subnet: mask over the columns [Q heads | K groups | V groups] and the number of marked columns.
+__global__ void qkv_col_mask_kernel(const uint32_t* __restrict__ head_cover, const uint32_t* __restrict__ kv_cover,
+                                    int n_heads, int n_kv, int d_head, int subnet_begin, uint8_t* __restrict__ mask,
+                                    int32_t* __restrict__ count) {
+  const int s = blockIdx.x, bit = subnet_begin + s;
+  const int width = (n_heads + 2 * n_kv) * d_head;
+  for (int c = threadIdx.x; c < width; c += blockDim.x) {
+    const int blk = c / d_head;
+    const uint32_t cov = blk < n_heads ? head_cover[blk] : kv_cover[(blk - n_heads) % n_kv];
+    mask[(long long)s * width + c] = (uint8_t)((cov >> bit) & 1u);
+  }
+  if (threadIdx.x == 0) {
+    int n = 0;
+    for (int h = 0; h < n_heads; ++h) n += (head_cover[h] >> bit) & 1u;
+    for (int g = 0; g < n_kv; ++g) n += 2 * ((kv_cover[g] >> bit) & 1u);
+    count[s] = n * d_head;
+  }
+}
+
+// out[s][t][c] = mask[s][c] ? in[s][t][c] : 0 for bf16 activations, 8 columns (16 bytes) per thread.
+__global__ void __launch_bounds__(256) apply_col_mask_kernel(const uint4* __restrict__ in, const uint8_t* __restrict__ mask,
+                                                             uint4* __restrict__ out, long long vecs_per_subnet,
+                                                             int vecs_per_row, long long total) {
+  for (long long v = (long long)blockIdx.x * blockDim.x + threadIdx.x; v < total; v += (long long)gridDim.x * blockDim.x) {
+    const long long s = v / vecs_per_subnet;
+    const int c = (int)((v - s * vecs_per_subnet) % vecs_per_row);
+    const uint2 m = *reinterpret_cast<const uint2*>(mask + (s * vecs_per_row + c) * 8);
+    const uint4 x = in[v];
+    uint4 y;
+    y.x = (x.x & ((m.x & 0x000000FFu) ? 0x0000FFFFu : 0u)) | (x.x & ((m.x & 0x0000FF00u) ? 0xFFFF0000u : 0u));
+    y.y = (x.y & ((m.x & 0x00FF0000u) ? 0x0000FFFFu : 0u)) | (x.y & ((m.x & 0xFF000000u) ? 0xFFFF0000u : 0u));
+    y.z = (x.z & ((m.y & 0x000000FFu) ? 0x0000FFFFu : 0u)) | (x.z & ((m.y & 0x0000FF00u) ? 0xFFFF0000u : 0u));
+    y.w = (x.w & ((m.y & 0x00FF0000u) ? 0x0000FFFFu : 0u)) | (x.w & ((m.y & 0xFF000000u) ? 0xFFFF0000u : 0u));
+    out[v] = y;
+  }
+}
+
 // One thread per (layer, subnet): kept KV groups of the sorted kept heads.
 __global__ void kv_groups_kernel(const int32_t* __restrict__ head_idx, int total, int head_keep, int per_group,
                                  int n_kv, int d_head, int32_t* __restrict__ kv_idx, int32_t* __restrict__ kv_count,
@@ -245,6 +282,36 @@ extern "C" int32_t twist_hidden_mask(const uint32_t* cover, int32_t n_full, int3
   const long long rows = (long long)n_full * block_rows;
   hidden_mask_kernel<<<(unsigned)((rows + 255) / 256), 256, 0, static_cast<cudaStream_t>(stream)>>>(
       cover, rows, block_rows, subnet_begin, n_subnets, mask);
+  TWIST_LAUNCH_CHECK();
+  return TWIST_OK;
+}
+
+extern "C" int32_t twist_qkv_col_mask(const uint32_t* head_cover, const uint32_t* kv_cover, int32_t n_heads,
+                                      int32_t n_kv_heads, int32_t d_head, int32_t subnet_begin, int32_t n_subnets,
+                                      uint8_t* mask, int32_t* count, void* stream) {
+  using namespace twist;
+  if (!head_cover || !kv_cover || !mask || !count) return TWIST_ERR_NULL;
+  if (n_heads <= 0 || n_kv_heads <= 0 || d_head <= 0 || subnet_begin < 0 || n_subnets <= 0) return TWIST_ERR_SHAPE;
+  if (subnet_begin + n_subnets > TWIST_MAX_SUBNETS) return TWIST_ERR_UNSUPPORTED;
+  qkv_col_mask_kernel<<<n_subnets, 256, 0, static_cast<cudaStream_t>(stream)>>>(head_cover, kv_cover, n_heads, n_kv_heads,
+                                                                              d_head, subnet_begin, mask, count);
+  TWIST_LAUNCH_CHECK();
+  return TWIST_OK;
+}
+
+extern "C" int32_t twist_apply_col_mask(const void* in, const uint8_t* mask, void* out, int32_t n_subnets, int32_t tokens,
+                                        int32_t width, void* stream) {
+  using namespace twist;
+  if (!in || !mask || !out) return TWIST_ERR_NULL;
+  if (n_subnets <= 0 || tokens <= 0 || width <= 0 || width % 8 != 0) return TWIST_ERR_SHAPE;
+  if (!aligned16(in) || !aligned16(out) || (reinterpret_cast<uintptr_t>(mask) & 7u)) return TWIST_ERR_SHAPE;
+  const int vecs_per_row = width / 8;
+  const long long per_subnet = (long long)tokens * vecs_per_row, total = per_subnet * n_subnets;
+  long long blocks = (total + 255) / 256;
+  const long long cap = (long long)sm_count() * 8;
+  if (blocks > cap) blocks = cap;
+  apply_col_mask_kernel<<<(unsigned)blocks, 256, 0, static_cast<cudaStream_t>(stream)>>>(
+      static_cast<const uint4*>(in), mask, static_cast<uint4*>(out), per_subnet, vecs_per_row, total);
   TWIST_LAUNCH_CHECK();
   return TWIST_OK;
 }

@@ -56,7 +56,8 @@ int check_fused(const void* tgt, float* loss, const void* dgrad, void* ws, size_
 // Output GEMM of a forward call with the loss fused into its epilogue (bf16).
 int launch_fused_loss(int layout, const GemmOperand& A, const GemmOperand& B, GemmParams p, void* out, const void* tgt,
                       void* dgrad, float* loss, void* ws, const int32_t* valid_cols, int seg_begin, int seg_width,
-                      cudaStream_t st) {
+                      cudaStream_t st, const uint8_t* col_mask = nullptr) {
+  p.col_mask = col_mask;
   p.out0 = static_cast<__nv_bfloat16*>(out);
   p.out1 = static_cast<__nv_bfloat16*>(dgrad);
   p.in0 = static_cast<const __nv_bfloat16*>(tgt);
@@ -227,8 +228,9 @@ static int check_proj(const twist_proj_args* a) {
   if (a->dtype != TWIST_FP32 && a->dtype != TWIST_BF16) return TWIST_ERR_SHAPE;
   if (a->dtype == TWIST_BF16 && (a->d_model % 8 || a->n % 8)) return TWIST_ERR_SHAPE;
   if (!all_aligned16({a->in, a->w, a->w_master, a->out, a->d_out, a->d_in, a->dw, a->tgt, a->loss_ws, a->out_residual,
-                      a->d_in_residual, a->m, a->v}))
+                      a->d_in_residual, a->m, a->v}) || !aligned8(a->col_mask))
     return TWIST_ERR_SHAPE;
+  if (a->col_mask && a->dtype != TWIST_BF16) return TWIST_ERR_UNSUPPORTED;
   return TWIST_OK;
 }
 
@@ -238,8 +240,13 @@ extern "C" int32_t twist_subnet_attn_proj_fwd(const twist_proj_args* a, void* st
   const bool qkv = a->which == TWIST_PROJ_QKV;
   const int w_out = qkv ? n : d;      // width of the output
   bool fused = false;
+  // An arbitrary column set for the loss (col_mask, with valid_cols[s] = its size) is a one-group prefix rule
+  // as far as the normaliser goes.
+  const bool by_mask = qkv && a->col_mask != nullptr && a->tgt != nullptr;      // (TWIST_PROJ_O: the mask acts in bwd)
+  const int seg_begin = by_mask ? 0 : a->seg_begin, seg_width = by_mask ? w_out : a->seg_width;
+  if (by_mask && (!a->valid_cols || a->dtype != TWIST_BF16)) return a->valid_cols ? TWIST_ERR_UNSUPPORTED : TWIST_ERR_NULL;
   TWIST_TRY(check_fused(a->tgt, a->loss, a->d_out, a->loss_ws, a->loss_ws_bytes, S, T, w_out, a->valid_cols,
-                        a->seg_begin, a->seg_width, &fused));
+                        seg_begin, seg_width, &fused));
   if (!a->in || !a->w || (!a->out && !fused)) return TWIST_ERR_NULL;
   if (a->out_residual && (fused || qkv || a->dtype == TWIST_FP32)) return TWIST_ERR_UNSUPPORTED;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -263,7 +270,7 @@ extern "C" int32_t twist_subnet_attn_proj_fwd(const twist_proj_args* a, void* st
   const int layout = qkv ? 0 : 1;
   if (fused)
     return launch_fused_loss(layout, A, W, p, a->out, a->tgt, const_cast<void*>(a->d_out), a->loss, a->loss_ws,
-                             a->valid_cols, a->seg_begin, a->seg_width, st);
+                             a->valid_cols, seg_begin, seg_width, st, by_mask ? a->col_mask : nullptr);
   p.out0 = static_cast<__nv_bfloat16*>(a->out);
   p.in0 = static_cast<const __nv_bfloat16*>(a->out_residual);
   return launch_gemm_bf16(layout, a->out_residual ? EPI_RESID : EPI_STORE, A, W, p, st);
@@ -312,6 +319,7 @@ extern "C" int32_t twist_subnet_attn_proj_bwd(const twist_proj_args* a, void* st
     } else {
       GemmParams p = base_params(T, n, d, S, a->out_scale);
       p.out0 = static_cast<__nv_bfloat16*>(a->d_in);
+      p.hmask = a->col_mask;             // a masked worker: no gradient flows into the heads it does not hold
       TWIST_TRY(launch_gemm_bf16(0, EPI_STORE, GemmOperand{a->d_out, T, d}, GemmOperand{a->w, n, d}, p, st));
     }
   }

@@ -359,12 +359,23 @@ class RoundEngine:
         bf16 = w.dtype == DTYPE_BF16
         self.launches += (2 + 3 + (1 if self.compute_dx else 0)) if bf16 else (3 + 4 + (1 if self.compute_dx else 0) + 2)
 
+    def _qkv_loss_mask(self, l: int) -> dict:
+        """Which columns of the QKV block's output count in its loss: all, or (grouped-query attention) the K / V
+        groups each subnet holds."""
+        w = self.w
+        if w.n_kv_heads == w.n_heads:
+            return {}
+        return dict(valid_cols=self.kv_cols[l], seg_begin=self.a_sub, seg_width=self.kv_max * w.d_head)
+
+    def _o_mask(self, l: int) -> dict:
+        return {}
+
     def qkv_step(self, l: int, k: int, lr: Optional[float] = None):
         self._use(l)
         w = self.w
         lr = w.lr if lr is None else lr
-        ragged = self.w.n_kv_heads != self.w.n_heads
-        mask = dict(valid_cols=self.kv_cols[l], seg_begin=self.a_sub, seg_width=self.kv_max * w.d_head) if ragged else {}
+        mask = self._qkv_loss_mask(l)
+        ragged = bool(mask)
         fused = dict(tgt=self.Tq[k], loss=self.loss[l, 1, k], loss_ws=self.ws, **mask) if self.fuse_loss else {}
         a = B.proj_args(B.PROJ_QKV, w.dtype, w.n_subnets, w.tokens, w.d_model, self.nq, 1.0, lr, in_=self.X[k],
                         w=self.w_qkv, w_master=self.w_qkv_m, out=self.qkv_out if self.store_outputs else None,
@@ -387,7 +398,8 @@ class RoundEngine:
         fused = dict(tgt=self.Td[k], loss=self.loss[l, 2, k], loss_ws=self.ws) if self.fuse_loss else {}
         a = B.proj_args(B.PROJ_O, w.dtype, w.n_subnets, w.tokens, w.d_model, self.a_sub, self.alpha_a, lr,
                         in_=self.A[k], w=self.w_o, w_master=self.w_o_m, out=self.y if self.store_outputs else None,
-                        d_out=self.dy, d_in=self.da, dw=self.dw_o, **fused, **self._opt(k, ("", "w_o")))
+                        d_out=self.dy, d_in=self.da, dw=self.dw_o, **fused, **self._o_mask(l),
+                        **self._opt(k, ("", "w_o")))
         with self._timed("o_fwd"):
             B.twist_subnet_attn_proj_fwd(a)
         if self.fuse_loss:
@@ -470,18 +482,23 @@ class RoundEngine:
 
 
 class MaskedRoundEngine(RoundEngine):
-    """Masked TwIST (Sec. 4.1) for the FFN blocks: every worker holds a full-width copy of the layer and is turned
-    into its subnet by an activation mask; nothing is physically smaller.  The "gather" is a copy of the whole layer
-    to every worker (the identity blueprint), the masks come from the sampled blueprints' cover bits, and the
+    """Masked TwIST (Sec. 4.1): every worker holds a full-width copy of the layer and is turned into its subnet by
+    masks; nothing is physically smaller.  FFN blocks: an activation mask (y = M * f(x)).  Attention blocks: a head
+    mask -- the columns of the dropped heads stay out of the QKV block's loss, the dropped heads' outputs are zero
+    at the output projection's input and no gradient flows into them.  The "gather" is a copy of the whole layer to
+    every worker (the identity blueprint), the masks come from the sampled blueprints' cover bits, and the
     aggregator averages every block over the workers whose blueprint holds it.  In exact arithmetic the round
     equals RoundEngine's, at N_full / N_sub times its flops and S full copies of a layer: a simulation mode and an
-    on-device check of "masked = gathered", not a fast path."""
+    on-device check of "masked = gathered", not a fast path.
+    Batches of the attention blocks are full-width: Tq [S][T][(H + 2 H_kv) d_head] (only the held columns are
+    read) and A [S][T][H d_head] (the head mask is applied to it before the output projection)."""
 
     def __init__(self, w: Workload, device: str = "cuda", **kw):
         from dataclasses import replace as _replace
-        assert w.dtype == DTYPE_BF16 and w.n_heads == 0 and not w.shared_layers, "bf16 FFN-only workloads"
-        nb = w.n_ffn_blocks
-        super().__init__(_replace(w, ffn_keep=nb), device=device, **kw)      # storage: full-width slices
+        assert w.dtype == DTYPE_BF16 and not w.shared_layers, "bf16 workloads without shared layers"
+        nb, H, Hkv = w.n_ffn_blocks, w.n_heads, w.n_kv_heads
+        super().__init__(_replace(w, ffn_keep=nb, head_keep=H), device=device, **kw)      # storage: full-width slices
+        assert self.fuse_loss or not self.has_attn, "the head mask of the QKV block acts in the fused loss"
         self.true_w = w
         L, S = w.n_layers, w.n_subnets
         i32 = dict(dtype=torch.int32, device=self.dev)
@@ -491,19 +508,66 @@ class MaskedRoundEngine(RoundEngine):
         self._gather_idx_override, self._agg_pos_override = ident, ident      # every worker copies / returns every block
         self.h_mask = torch.zeros(S, w.d_ff, dtype=torch.uint8, device=self.dev)
         self.alpha_f = self.geo["part"].alpha_f = math.sqrt(nb / w.ffn_keep)  # the subnet's scale (Sec. 3.4)
+        if self.has_attn:
+            self.alpha_a = self.geo["part"].alpha_a = math.sqrt(H / w.head_keep)
+            self.t_idx_head = torch.empty(L, S, w.head_keep, **i32)           # the sampled head blueprints
+            self.t_pos_head = torch.empty(L, S, H, **i32)
+            self.t_kv = [torch.empty(L, S, Hkv, **i32), torch.empty(L, S, **i32), torch.empty(L, S, **i32),
+                         torch.empty(L, S, Hkv, **i32)]                       # kv_idx, kv_count, kv_cols, kv_pos (unused)
+            # what gather and aggregate see: every worker holds every head / group at its own position
+            self.idx_head.copy_(torch.arange(H, **i32).expand(L, S, H))
+            self.pos_head.copy_(torch.arange(H, **i32).expand(L, S, H))
+            self.kv_idx.copy_(torch.arange(Hkv, **i32).expand(L, S, Hkv))
+            self.kv_pos.copy_(torch.arange(Hkv, **i32).expand(L, S, Hkv))
+            self.kv_count.fill_(Hkv)
+            self.kv_cols.fill_(Hkv * w.d_head)
+            self.qkv_mask = torch.zeros(S, self.nq, dtype=torch.uint8, device=self.dev)
+            self.qkv_count = torch.zeros(S, **i32)
+            self.a_mask = torch.zeros(S, self.a_sub, dtype=torch.uint8, device=self.dev)
+            self.a_masked = torch.empty(S, w.tokens, self.a_sub, dtype=torch.bfloat16, device=self.dev)
+
+    def o_step(self, l: int, k: int, lr: Optional[float] = None):
+        """The head mask multiplies the head outputs (Sec. 4.1) before the output projection sees them."""
+        w = self.true_w
+        B.twist_apply_col_mask(self.A[k], self.a_mask, self.a_masked, w.n_subnets, w.tokens, self.a_sub)
+        self.launches += 1
+        plain = self.A[k]
+        self.A[k] = self.a_masked
+        try:
+            super().o_step(l, k, lr)
+        finally:
+            self.A[k] = plain
 
     def sample_masks(self, rnd: int):
         w = self.true_w
         with self._timed("sample_masks"):
             B.twist_sample_masks(w.seed_mask, rnd, 0, w.n_layers, B.KIND_FFN, w.n_ffn_blocks, w.n_subnets, w.ffn_keep,
                                  list(w.common_ffn), w.sample_mode, self.idx_ffn, self.cover_ffn, self.pos_ffn)
-        self.launches += 2
+            self.launches += 2
+            if self.has_attn:
+                B.twist_sample_masks(w.seed_mask, rnd, 0, w.n_layers, B.KIND_HEAD, w.n_heads, w.n_subnets, w.head_keep,
+                                     list(w.common_heads), w.sample_mode, self.t_idx_head, self.cover_head,
+                                     self.t_pos_head)
+                B.twist_kv_groups(self.t_idx_head, w.n_layers, w.n_subnets, w.head_keep, w.n_heads, w.n_kv_heads,
+                                  w.d_head, self.t_kv[0], self.t_kv[1], self.t_kv[2], self.kv_cover, self.t_kv[3])
+                self.launches += 4
 
-    def gather_layer(self, l: int, which=("ffn",)):
-        super().gather_layer(l, which=("ffn",))
+    def gather_layer(self, l: int, which=("ffn", "attn")):
+        super().gather_layer(l, which=which)
         w = self.true_w
         B.twist_hidden_mask(self.cover_ffn[l], w.n_ffn_blocks, w.ffn_block, 0, w.n_subnets, self.h_mask)
         self.launches += 1
+        if self.has_attn:
+            B.twist_qkv_col_mask(self.cover_head[l], self.kv_cover[l], w.n_heads, w.n_kv_heads, w.d_head, 0, w.n_subnets,
+                                 self.qkv_mask, self.qkv_count)
+            B.twist_hidden_mask(self.cover_head[l], w.n_heads, w.d_head, 0, w.n_subnets, self.a_mask)
+            self.launches += 2
+
+    def _qkv_loss_mask(self, l: int) -> dict:
+        return dict(col_mask=self.qkv_mask, valid_cols=self.qkv_count)
+
+    def _o_mask(self, l: int) -> dict:
+        return dict(col_mask=self.a_mask)
 
 
 class HybridRoundEngine(RoundEngine):

@@ -532,12 +532,26 @@ def _run_round_and_compare(B, w, rnd=0, tol_dw=5e-2, engine_cls=None, **engine_k
     torch.cuda.synchronize()
     check_status(B)
     ragged = eng.has_attn and w.n_kv_heads != w.n_heads
+    w = getattr(eng, "true_w", w)
     for l in range(w.n_layers):
         bp = o.layer_blueprints(w, rnd, l)
 
         gm = eng.geo[eng.kind_of(l)]
+        masked_attn = eng.has_attn and hasattr(eng, "true_w")      # full-width batches: the oracle sees the held columns
+
+        def held_cols(bp, s, qkv):
+            dh, H, Hkv = w.d_head, w.n_heads, w.n_kv_heads
+            q = np.concatenate([np.arange(h * dh, (h + 1) * dh) for h in bp["head"][s]])
+            if not qkv:
+                return q
+            groups = bp["kv_idx"][s][: bp["kv_count"][s]]
+            kc = np.concatenate([np.arange((H + g) * dh, (H + g + 1) * dh) for g in groups])
+            return np.concatenate([q, kc, kc + Hkv * dh])
 
         def get_batch(kind, rnd_, s, k, width, bp=bp, gm=gm):
+            if masked_attn and kind in (I.BATCH_TGT_QKV, I.BATCH_A):
+                full_width = gm.nq if kind == I.BATCH_TGT_QKV else gm.a_sub
+                return store[(kind, k, full_width)][s][:, held_cols(bp, s, kind == I.BATCH_TGT_QKV)]
             if kind == I.BATCH_TGT_QKV and ragged:     # device layout [Q | K pad | V pad] -> oracle [Q | K | V]
                 arr = store[(kind, k, gm.nq)][s]
                 kc = bp["kv_count"][s] * w.d_head
@@ -980,3 +994,27 @@ def test_layernorm_parity(B, S, T, d, adam):
     B.twist_layernorm_bwd(a2)
     torch.cuda.synchronize()
     assert torch.equal(dy2, dx)
+
+
+@pytest.mark.parametrize("cfg,dims", [
+    (4, dict(d_model=136, d_ff=544, d_head=8, tokens=200, n_layers=2, local_steps=2)),       # multi-head attention
+    (3, dict(d_model=256, d_ff=688, d_head=8, tokens=256, n_layers=2, local_steps=1)),       # grouped-query: masked KV groups
+])
+def test_masked_twist_round_with_head_masks_matches_the_oracle_round(B, cfg, dims):
+    """Masked TwIST (Sec. 4.1) with attention: FFN activations masked, and a head mask on the attention blocks (the
+    dropped heads' columns out of the QKV block's loss, their outputs zero before the output projection, no gradient
+    into them).  The round equals the gathered round the oracle computes; the rows of dropped heads keep their bytes
+    in every worker's copy."""
+    from paper_2511_03983_b200.engine import MaskedRoundEngine
+    w = replace(I.scaled_twin(I.PRESETS[cfg], **dims), lr=0.05)
+    eng, before = _run_round_and_compare(B, w, engine_cls=MaskedRoundEngine, keep_f32_full=True)
+    assert eng.w_qkv.shape[1] == (w.n_heads + 2 * w.n_kv_heads) * w.d_head        # nothing is physically smaller
+    # the last layer's worker copies: rows of heads a worker does not hold are bit-identical to the gathered model
+    l = w.n_layers - 1
+    bp = o.layer_blueprints(w, 0, l)
+    for s in range(w.n_subnets):
+        dropped = np.setdiff1d(np.arange(w.n_heads), bp["head"][s])
+        rows = np.concatenate([np.arange(h * w.d_head, (h + 1) * w.d_head) for h in dropped])
+        rt = torch.from_numpy(rows).cuda()
+        assert torch.equal(eng.w_qkv_m[s][rt], before["qkv"][l][rt].float())
+        assert torch.equal(eng.w_o_m[s][rt], before["o"][l][rt].float())
