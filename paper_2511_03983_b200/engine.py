@@ -571,28 +571,56 @@ class MaskedRoundEngine(RoundEngine):
 
 
 class HybridRoundEngine(RoundEngine):
-    """Hybrid TwIST (Sec. 4.1) for the FFN blocks: worker 0 is the central model.  It keeps no slice: it trains its
-    subnet in place on the full-width matrices under an activation mask (twist_ffn_args.hidden_mask), while workers
-    1 .. S-1 train gathered dense slices as in RoundEngine; the aggregator reads worker 0's rows from the full fp32
-    matrices (twist_aggregate_segment.central).  In exact arithmetic the round equals RoundEngine's.
-    (The full model's gate and up rows lie back to back, so a full-width layer is a valid w_gu operand.)"""
+    """Hybrid TwIST (Sec. 4.1): worker 0 is the central model.  It keeps no slice: it trains its subnet in place on
+    the full-width matrices under masks (an activation mask on the FFN block, a head mask on the attention blocks,
+    as in MaskedRoundEngine), while workers 1 .. S-1 train gathered dense slices as in RoundEngine; the aggregator
+    reads worker 0's rows from the full fp32 matrices (twist_aggregate_segment.central).  In exact arithmetic the
+    round equals RoundEngine's.  (The full model's gate and up rows lie back to back, so a full-width layer is a
+    valid w_gu operand.)  The central worker's batches of the attention blocks are full-width: Tq_c [1][T][(H + 2
+    H_kv) d_head] (only the held columns are read), A_c [1][T][H d_head] (masked before the output projection)."""
 
     def __init__(self, w: Workload, device: str = "cuda", **kw):
-        assert w.dtype == DTYPE_BF16 and w.n_heads == 0 and w.n_subnets >= 2 and not w.shared_layers, \
-            "bf16 FFN-only workloads"
+        assert w.dtype == DTYPE_BF16 and w.n_subnets >= 2 and not w.shared_layers, "bf16 workloads without shared layers"
         super().__init__(w, device=device, keep_f32_full=True, **kw)
-        F, T = w.d_ff, w.tokens
+        assert self.fuse_loss or not self.has_attn, "the head mask of the QKV block acts in the fused loss"
+        F, T, d = w.d_ff, w.tokens, w.d_model
         g, dev = self.g, self.dev
         bf = torch.bfloat16
         act = lambda width: torch.empty(1, T, width, dtype=bf, device=dev)
         self.c_pre, self.c_dpre, self.c_hh = act(g * F), act(g * F), act(F)
         self.c_mask = torch.zeros(1, F, dtype=torch.uint8, device=dev)
+        f32 = lambda rows: torch.zeros(1, rows, d, dtype=torch.float32, device=dev)
         if self.adam:      # the central worker's moments are full-width like its weights; zeroed when its layer starts
-            f32 = lambda rows: torch.zeros(1, rows, w.d_model, dtype=torch.float32, device=dev)
             self.c_gu_m1, self.c_gu_m2, self.c_down_m1, self.c_down_m2 = f32(g * F), f32(g * F), f32(F), f32(F)
+        if self.has_attn:
+            H, Hkv, dh = w.n_heads, w.n_kv_heads, w.d_head
+            self.c_nq, self.c_a = (H + 2 * Hkv) * dh, H * dh
+            self.c_qkv_mask = torch.zeros(1, self.c_nq, dtype=torch.uint8, device=dev)
+            self.c_qkv_count = torch.zeros(1, dtype=torch.int32, device=dev)
+            self.c_a_mask = torch.zeros(1, self.c_a, dtype=torch.uint8, device=dev)
+            self.c_a_masked, self.c_dqkv = act(self.c_a), act(self.c_nq)
+            self.c_qkv_out = act(self.c_nq) if self.store_outputs else None
+            self.c_da = act(self.c_a) if self.compute_dx else None
+            self.Tq_c: List[torch.Tensor] = []
+            self.A_c: List[torch.Tensor] = []
+            if self.adam:
+                self.c_qkv_m1, self.c_qkv_m2, self.c_o_m1, self.c_o_m2 = f32(self.c_nq), f32(self.c_nq), f32(self.c_a), f32(self.c_a)
 
-    def gather_layer(self, l: int, which=("ffn",)):
-        """Slices of workers 1 .. S-1 only; the central worker's activation mask for this layer."""
+    def _central_opt(self, k: int, *pairs):
+        if not self.adam:
+            return {}
+        w = self.w
+        kw = {"opt": B.adam(k + 1, w.beta1, w.beta2, w.adam_eps)}
+        for arg, name in pairs:
+            kw["m" + arg] = getattr(self, name + "_m1")
+            kw["v" + arg] = getattr(self, name + "_m2")
+        return kw
+
+    def _others_opt(self, k: int, *pairs):
+        return {key: (v if key == "opt" else v[1:]) for key, v in self._opt(k, *pairs).items()}
+
+    def gather_layer(self, l: int, which=("ffn", "attn")):
+        """Slices of workers 1 .. S-1 only; the central worker's masks for this layer."""
         w, d = self.w, self.w.d_model
         f, gf = self.f_sub, self.gf
         idx = self.idx_ffn[l, 1:]
@@ -601,26 +629,38 @@ class HybridRoundEngine(RoundEngine):
                 ("up", f if self.g == 2 else 0, self.w_gu, self.w_gu_m, gf), ("down", 0, self.w_down, self.w_down_m, f)]:
             segs.append(B.gather_segment(self.full[m][l], dst[1:], dst_m[1:], idx, None, w.ffn_keep, w.ffn_keep,
                                          w.ffn_block, 0, stride * d, off, w.n_ffn_blocks))
+        if self.has_attn:
+            H, Hkv, dh, hk = w.n_heads, w.n_kv_heads, w.d_head, w.head_keep
+            qkv, ih, ik, ic = self.full["qkv"][l], self.idx_head[l, 1:], self.kv_idx[l, 1:], self.kv_count[l, 1:]
+            q_dst, q_m = self.w_qkv[1:], self.w_qkv_m[1:]
+            segs.append(B.gather_segment(qkv, q_dst, q_m, ih, None, hk, hk, dh, 0, self.nq * d, 0, H))
+            segs.append(B.gather_segment(qkv, q_dst, q_m, ik, ic, Hkv, self.kv_max, dh, H * dh, self.nq * d, self.a_sub, Hkv))
+            segs.append(B.gather_segment(qkv, q_dst, q_m, ik, ic, Hkv, self.kv_max, dh, (H + Hkv) * dh, self.nq * d,
+                                         self.a_sub + self.kv_max * dh, Hkv))
+            segs.append(B.gather_segment(self.full["o"][l], self.w_o[1:], self.w_o_m[1:], ih, None, hk, hk, dh, 0,
+                                         self.a_sub * d, 0, H))
         with self._timed("gather"):
             B.twist_gather_subnets(segs, w.n_subnets - 1, d, w.dtype)
             B.twist_hidden_mask(self.cover_ffn[l], w.n_ffn_blocks, w.ffn_block, 0, 1, self.c_mask)
+            if self.has_attn:
+                B.twist_qkv_col_mask(self.cover_head[l], self.kv_cover[l], w.n_heads, w.n_kv_heads, w.d_head, 0, 1,
+                                     self.c_qkv_mask, self.c_qkv_count)
+                B.twist_hidden_mask(self.cover_head[l], w.n_heads, w.d_head, 0, 1, self.c_a_mask)
+                self.launches += 2
             for n in self.moment_names:        # a fresh worker state, also for the central worker
                 getattr(self, n).zero_()
             if self.adam:
-                for t in (self.c_gu_m1, self.c_gu_m2, self.c_down_m1, self.c_down_m2):
-                    t.zero_()
+                for n in ("c_gu", "c_down") + (("c_qkv", "c_o") if self.has_attn else ()):
+                    getattr(self, n + "_m1").zero_()
+                    getattr(self, n + "_m2").zero_()
         self.launches += 2
 
     def ffn_step(self, l: int, k: int, lr: Optional[float] = None):
         w = self.w
         lr = w.lr if lr is None else lr
         S, T, d, F = w.n_subnets, w.tokens, w.d_model, w.d_ff
-        central_opt, others_opt = {}, {}
-        if self.adam:
-            opt = B.adam(k + 1, w.beta1, w.beta2, w.adam_eps)
-            central_opt = dict(opt=opt, m_gu=self.c_gu_m1, v_gu=self.c_gu_m2, m_down=self.c_down_m1, v_down=self.c_down_m2)
-            others_opt = dict(opt=opt, m_gu=self.w_gu_m1[1:], v_gu=self.w_gu_m2[1:], m_down=self.w_down_m1[1:],
-                              v_down=self.w_down_m2[1:])
+        central_opt = self._central_opt(k, ("_gu", "c_gu"), ("_down", "c_down"))
+        others_opt = self._others_opt(k, ("_gu", "w_gu"), ("_down", "w_down"))
         # central worker: the full-width layer under its mask, updated in place
         c = B.ffn_args(w.ffn_kind, w.dtype, 1, T, d, F, self.alpha_f, lr, x=self.X[k][:1], w_gu=self.full_gu[l],
                        w_down=self.full["down"][l], w_gu_master=self.full_gu_f32[l],
@@ -642,7 +682,50 @@ class HybridRoundEngine(RoundEngine):
             B.twist_subnet_ffn_bwd(o)
         self.launches += 2 * (2 + 1 + 3 + (1 if self.compute_dx else 0))
 
-    def aggregate_layer(self, l: int, live: int = 0xFFFFFFFF, which=("ffn",)):
+    def qkv_step(self, l: int, k: int, lr: Optional[float] = None):
+        w = self.w
+        lr = w.lr if lr is None else lr
+        S, T, d = w.n_subnets, w.tokens, w.d_model
+        dx = lambda sl: self.dx[sl] if self.dx is not None else None
+        c = B.proj_args(B.PROJ_QKV, w.dtype, 1, T, d, self.c_nq, 1.0, lr, in_=self.X[k][:1], w=self.full["qkv"][l],
+                        w_master=self.full_f32["qkv"][l], out=self.c_qkv_out, d_out=self.c_dqkv, d_in=dx(slice(0, 1)),
+                        tgt=self.Tq_c[k], loss=self.loss[l, 1, k][:1], loss_ws=self.ws, col_mask=self.c_qkv_mask,
+                        valid_cols=self.c_qkv_count, **self._central_opt(k, ("", "c_qkv")))
+        mask = {key: (v[1:] if key == "valid_cols" else v) for key, v in self._qkv_loss_mask(l).items()}
+        o = B.proj_args(B.PROJ_QKV, w.dtype, S - 1, T, d, self.nq, 1.0, lr, in_=self.X[k][1:], w=self.w_qkv[1:],
+                        w_master=self.w_qkv_m[1:], out=self.qkv_out[1:] if self.store_outputs else None,
+                        d_out=self.dqkv[1:], d_in=dx(slice(1, None)), tgt=self.Tq[k][1:], loss=self.loss[l, 1, k][1:],
+                        loss_ws=self.ws, **mask, **self._others_opt(k, ("", "w_qkv")))
+        with self._timed("qkv_fwd"):
+            B.twist_subnet_attn_proj_fwd(c)
+            B.twist_subnet_attn_proj_fwd(o)
+        with self._timed("qkv_bwd"):
+            B.twist_subnet_attn_proj_bwd(c)
+            B.twist_subnet_attn_proj_bwd(o)
+        self.launches += 2 * (2 + 1 + (1 if self.compute_dx else 0))
+
+    def o_step(self, l: int, k: int, lr: Optional[float] = None):
+        w = self.w
+        lr = w.lr if lr is None else lr
+        S, T, d = w.n_subnets, w.tokens, w.d_model
+        B.twist_apply_col_mask(self.A_c[k], self.c_a_mask, self.c_a_masked, 1, T, self.c_a)     # Sec. 4.1: M * f(x)
+        c = B.proj_args(B.PROJ_O, w.dtype, 1, T, d, self.c_a, self.alpha_a, lr, in_=self.c_a_masked, w=self.full["o"][l],
+                        w_master=self.full_f32["o"][l], out=self.y[:1] if self.store_outputs else None,
+                        d_out=self.dy[:1], d_in=self.c_da, tgt=self.Td[k][:1], loss=self.loss[l, 2, k][:1],
+                        loss_ws=self.ws, col_mask=self.c_a_mask, **self._central_opt(k, ("", "c_o")))
+        o = B.proj_args(B.PROJ_O, w.dtype, S - 1, T, d, self.a_sub, self.alpha_a, lr, in_=self.A[k][1:], w=self.w_o[1:],
+                        w_master=self.w_o_m[1:], out=self.y[1:] if self.store_outputs else None, d_out=self.dy[1:],
+                        d_in=self.da[1:] if self.da is not None else None, tgt=self.Td[k][1:],
+                        loss=self.loss[l, 2, k][1:], loss_ws=self.ws, **self._others_opt(k, ("", "w_o")))
+        with self._timed("o_fwd"):
+            B.twist_subnet_attn_proj_fwd(c)
+            B.twist_subnet_attn_proj_fwd(o)
+        with self._timed("o_bwd"):
+            B.twist_subnet_attn_proj_bwd(c)
+            B.twist_subnet_attn_proj_bwd(o)
+        self.launches += 1 + 2 * (2 + 1 + (1 if self.compute_dx else 0))
+
+    def aggregate_layer(self, l: int, live: int = 0xFFFFFFFF, which=("ffn", "attn")):
         w, d = self.w, self.w.d_model
         f, gf = self.f_sub, self.gf
         nb = w.n_ffn_blocks
@@ -652,6 +735,19 @@ class HybridRoundEngine(RoundEngine):
             segs.append(B.aggregate_segment(self.full[m][l], self.full_f32[m][l], sub, self.cover_ffn[l], self.pos_ffn[l],
                                             nb, w.ffn_block, 0, stride * d, off, w.ffn_keep,
                                             central=self.full_f32[m][l], central_subnet=0))
+        if self.has_attn:
+            H, Hkv, dh = w.n_heads, w.n_kv_heads, w.d_head
+            qf, qs = self.full_f32["qkv"][l], self.w_qkv_m
+            c = dict(central=qf, central_subnet=0)
+            segs.append(B.aggregate_segment(self.full["qkv"][l], qf, qs, self.cover_head[l], self.pos_head[l], H, dh, 0,
+                                            self.nq * d, 0, self.head_keep, **c))
+            segs.append(B.aggregate_segment(self.full["qkv"][l], qf, qs, self.kv_cover[l], self.kv_pos[l], Hkv, dh,
+                                            H * dh, self.nq * d, self.a_sub, self.kv_max, **c))
+            segs.append(B.aggregate_segment(self.full["qkv"][l], qf, qs, self.kv_cover[l], self.kv_pos[l], Hkv, dh,
+                                            (H + Hkv) * dh, self.nq * d, self.a_sub + self.kv_max * dh, self.kv_max, **c))
+            segs.append(B.aggregate_segment(self.full["o"][l], self.full_f32["o"][l], self.w_o_m, self.cover_head[l],
+                                            self.pos_head[l], H, dh, 0, self.a_sub * d, 0, self.head_keep,
+                                            central=self.full_f32["o"][l], central_subnet=0))
         with self._timed("aggregate"):
             B.twist_aggregate(segs, w.n_subnets, d, w.dtype, live)
         self.launches += 1

@@ -515,6 +515,13 @@ def _load_batches(eng, w, rnd):
                     if gk == "part":
                         store[(kind, k)] = arr
                     eng.batches[gk][name].append(dev(arr, td))
+    if eng.has_attn and hasattr(eng, "Tq_c"):        # Hybrid TwIST: the central worker's full-width batches
+        eng.Tq_c, eng.A_c = [], []
+        for k in range(w.local_steps):
+            for kind, width, dst in ((I.BATCH_TGT_QKV, eng.c_nq, eng.Tq_c), (I.BATCH_A, eng.c_a, eng.A_c)):
+                arr = I.batch(w, kind + 4, rnd, 0, k, width)[None]
+                store[("central", kind, k)] = arr
+                dst.append(dev(arr, td))
     return store
 
 
@@ -549,6 +556,8 @@ def _run_round_and_compare(B, w, rnd=0, tol_dw=5e-2, engine_cls=None, **engine_k
             return np.concatenate([q, kc, kc + Hkv * dh])
 
         def get_batch(kind, rnd_, s, k, width, bp=bp, gm=gm):
+            if s == 0 and ("central", kind, k) in store:
+                return store[("central", kind, k)][0][:, held_cols(bp, s, kind == I.BATCH_TGT_QKV)]
             if masked_attn and kind in (I.BATCH_TGT_QKV, I.BATCH_A):
                 full_width = gm.nq if kind == I.BATCH_TGT_QKV else gm.a_sub
                 return store[(kind, k, full_width)][s][:, held_cols(bp, s, kind == I.BATCH_TGT_QKV)]
@@ -1018,3 +1027,18 @@ def test_masked_twist_round_with_head_masks_matches_the_oracle_round(B, cfg, dim
         rt = torch.from_numpy(rows).cuda()
         assert torch.equal(eng.w_qkv_m[s][rt], before["qkv"][l][rt].float())
         assert torch.equal(eng.w_o_m[s][rt], before["o"][l][rt].float())
+
+
+@pytest.mark.parametrize("cfg,dims,extra", [
+    (4, dict(d_model=136, d_ff=544, d_head=8, tokens=200, n_layers=2, local_steps=2), dict(lr=0.05)),
+    (3, dict(d_model=256, d_ff=688, d_head=8, tokens=256, n_layers=1, local_steps=2),
+     dict(optimizer="adam", lr=1e-3, beta2=0.99, adam_eps=3e-3)),
+])
+def test_hybrid_twist_round_with_attention_matches_the_oracle_round(B, cfg, dims, extra):
+    """Hybrid TwIST (Sec. 4.1) with attention blocks: the central worker trains the full-width projections in place
+    under its head mask, the others train gathered slices; the aggregate takes the central worker's rows from the
+    full fp32 matrices.  The round equals the all-gathered round of the oracle."""
+    from paper_2511_03983_b200.engine import HybridRoundEngine
+    w = replace(I.scaled_twin(I.PRESETS[cfg], **dims), **extra)
+    eng, before = _run_round_and_compare(B, w, engine_cls=HybridRoundEngine)
+    assert any(not torch.equal(eng.full[m], before[m]) for m in ("qkv", "o"))
