@@ -62,6 +62,40 @@ enum { TWIST_PROJ_QKV = 0, TWIST_PROJ_O = 1 };
 #define TWIST_MAX_BLOCKS 16384   /* blocks per layer and kind the sampler kernel handles */
 #define TWIST_MAX_COMMON 256     /* common blocks |C| per layer and kind */
 
+/* ---------------------------------------------------------------------------------------------
+ * twist_plan -- the shapes of one workload plus a cache of encoded TMA tensor maps (the paper has no counterpart:
+ * it is plumbing of this implementation).  The grouped GEMM and attention kernels address their operands through
+ * tensor maps that the host encodes from (base address, dimensions, box).  Calls that carry a plan
+ * (the `plan` field of their argument struct) look each map up in the plan's cache first, so a training loop that
+ * passes the same buffers every step encodes nothing after its first step.  A cached map never goes stale: it
+ * is a pure function of its key.  Calls without a plan (plan == NULL) encode their maps every time; both forms
+ * compute the same thing.
+ *  - twist_plan_create validates the configuration (TWIST_ERR_SHAPE / _INFEASIBLE / _UNSUPPORTED) and allocates
+ *    host memory only; the plan is owned by the caller and freed with twist_plan_destroy, after which no call may
+ *    carry it.  A plan may be shared by host threads (its cache is locked).
+ *  - twist_workspace_bytes: device scratch that covers every scratch argument (loss_ws, the stand-alone loss's
+ *    ws, the layer normalisation's ws) of the local-step calls of this workload -- partitioned or shared layers,
+ *    gathered or masked workers.
+ *  - twist_plan_stats: maps cached, cache hits and misses so far (any pointer may be NULL). */
+typedef struct twist_plan twist_plan;
+typedef struct {
+  uint32_t struct_size;       /* sizeof(twist_config): versions the struct */
+  int32_t n_layers, d_model, n_heads /* 0: no attention blocks */, n_kv_heads, d_head, d_ff;
+  int32_t ffn_kind;           /* TWIST_FFN_* */
+  int32_t n_subnets;          /* S */
+  int32_t ffn_block;          /* neurons per FFN block (Sec. 3.1: d_inner / R) */
+  int32_t ffn_keep, head_keep;   /* N_sub per kind, in blocks */
+  int32_t sample_mode;        /* TWIST_MODE_* */
+  int32_t dtype;              /* TWIST_FP32 / TWIST_BF16 */
+  int32_t tokens;             /* T: tokens per subnet and local step */
+  int32_t reserved;
+  uint64_t seed;
+} twist_config;
+int32_t twist_plan_create(const twist_config* cfg /*host*/, twist_plan** out);
+int32_t twist_plan_destroy(twist_plan* plan);
+int32_t twist_workspace_bytes(const twist_plan* plan, size_t* bytes);
+int32_t twist_plan_stats(twist_plan* plan, uint64_t* cached, uint64_t* hits, uint64_t* misses);
+
 uint32_t twist_abi_version(void);
 const char* twist_strerror(int32_t status);
 /* Text of the last CUDA error this library saw on the calling thread ("" if none). */
@@ -267,6 +301,7 @@ typedef struct {
    * the gradients of masked neurons' rows are exactly zero and the fused update leaves them untouched (Hybrid
    * TwIST's central model trains this way on its full copy).  NULL: no mask.  bf16 dtype only. */
   const uint8_t* hidden_mask;
+  twist_plan* plan;         /* optional: tensor maps come from this plan's cache (see twist_plan) */
 } twist_ffn_args;
 
 /* Fused loss.  When `tgt` is set, twist_subnet_ffn_fwd / twist_subnet_attn_proj_fwd also evaluate the loss
@@ -319,6 +354,7 @@ typedef struct {
    *     masked already, as the attention core's output under a head mask is.)
    * NULL: no mask.  bf16 dtype only. */
   const uint8_t* col_mask;
+  twist_plan* plan;            /* optional: tensor maps come from this plan's cache */
 } twist_proj_args;
 
 int32_t twist_subnet_attn_proj_fwd(const twist_proj_args* a /*host*/, void* stream);
@@ -349,6 +385,7 @@ typedef struct {
   const int32_t* head_idx;   /* device int32 [S][head_keep] or NULL */
   const int32_t* kv_pos;     /* device int32 [S][n_kv_heads] (required with head_idx) */
   const int32_t* kv_count;   /* device int32 [S] or NULL (every subnet holds kv_max positions) */
+  twist_plan* plan;          /* optional: tensor maps come from this plan's cache */
 } twist_attn_core_args;
 
 int32_t twist_attn_core_fwd(const twist_attn_core_args* a /*host*/, void* stream);

@@ -32,7 +32,8 @@ EXPORTS = [
     "twist_subnet_attn_proj_fwd", "twist_subnet_attn_proj_bwd", "twist_mse_workspace_bytes", "twist_mse_fwd_bwd",
     "twist_mse_fwd_bwd_noalloc", "twist_fused_loss_workspace_bytes", "twist_attn_core_fwd", "twist_attn_core_bwd",
     "twist_hidden_mask", "twist_selftest_wait", "twist_layernorm_workspace_bytes", "twist_layernorm_fwd",
-    "twist_layernorm_bwd", "twist_qkv_col_mask", "twist_apply_col_mask",
+    "twist_layernorm_bwd", "twist_qkv_col_mask", "twist_apply_col_mask", "twist_plan_create", "twist_plan_destroy",
+    "twist_plan_stats", "twist_workspace_bytes",
 ]
 
 
@@ -76,7 +77,7 @@ class FfnArgs(C.Structure):
                 ("dw_down", C.c_void_p), ("tgt", C.c_void_p), ("loss", C.c_void_p), ("loss_ws", C.c_void_p),
                 ("loss_ws_bytes", C.c_size_t), ("y_residual", C.c_void_p), ("dx_residual", C.c_void_p),
                 ("opt", Optimizer), ("m_gu", C.c_void_p), ("v_gu", C.c_void_p), ("m_down", C.c_void_p),
-                ("v_down", C.c_void_p), ("hidden_mask", C.c_void_p)]
+                ("v_down", C.c_void_p), ("hidden_mask", C.c_void_p), ("plan", C.c_void_p)]
 
 
 class ProjArgs(C.Structure):
@@ -87,7 +88,7 @@ class ProjArgs(C.Structure):
                 ("loss", C.c_void_p), ("loss_ws", C.c_void_p), ("loss_ws_bytes", C.c_size_t),
                 ("valid_cols", C.c_void_p), ("seg_begin", C.c_int32), ("seg_width", C.c_int32),
                 ("out_residual", C.c_void_p), ("d_in_residual", C.c_void_p), ("opt", Optimizer), ("m", C.c_void_p),
-                ("v", C.c_void_p), ("col_mask", C.c_void_p)]
+                ("v", C.c_void_p), ("col_mask", C.c_void_p), ("plan", C.c_void_p)]
 
 
 class AttnCoreArgs(C.Structure):
@@ -95,7 +96,51 @@ class AttnCoreArgs(C.Structure):
                 ("head_keep", C.c_int32), ("kv_max", C.c_int32), ("d_head", C.c_int32), ("n_heads", C.c_int32),
                 ("n_kv_heads", C.c_int32), ("qkv", C.c_void_p), ("out", C.c_void_p), ("lse", C.c_void_p),
                 ("d_out", C.c_void_p), ("d_qkv", C.c_void_p), ("delta", C.c_void_p), ("head_idx", C.c_void_p),
-                ("kv_pos", C.c_void_p), ("kv_count", C.c_void_p)]
+                ("kv_pos", C.c_void_p), ("kv_count", C.c_void_p), ("plan", C.c_void_p)]
+
+
+class Config(C.Structure):
+    _fields_ = [("struct_size", C.c_uint32), ("n_layers", C.c_int32), ("d_model", C.c_int32), ("n_heads", C.c_int32),
+                ("n_kv_heads", C.c_int32), ("d_head", C.c_int32), ("d_ff", C.c_int32), ("ffn_kind", C.c_int32),
+                ("n_subnets", C.c_int32), ("ffn_block", C.c_int32), ("ffn_keep", C.c_int32), ("head_keep", C.c_int32),
+                ("sample_mode", C.c_int32), ("dtype", C.c_int32), ("tokens", C.c_int32), ("reserved", C.c_int32),
+                ("seed", C.c_uint64)]
+
+
+class Plan:
+    """Owner of a twist_plan handle (the shapes of a workload and its cache of encoded tensor maps)."""
+
+    def __init__(self, w):
+        cfg = Config(C.sizeof(Config), w.n_layers, w.d_model, w.n_heads, w.n_kv_heads, w.d_head, w.d_ff, w.ffn_kind,
+                     w.n_subnets, w.ffn_block, w.ffn_keep, w.head_keep, w.sample_mode, w.dtype, w.tokens, 0, w.seed_mask)
+        self.handle = C.c_void_p()
+        _check(lib().twist_plan_create(C.byref(cfg), C.byref(self.handle)), "twist_plan_create")
+
+    @property
+    def ptr(self) -> int:
+        return self.handle.value
+
+    def workspace_bytes(self) -> int:
+        n = C.c_size_t(0)
+        _check(lib().twist_workspace_bytes(self.handle, C.byref(n)), "twist_workspace_bytes")
+        return n.value
+
+    def stats(self):
+        """(maps cached, cache hits, cache misses)"""
+        a, b, c = C.c_uint64(0), C.c_uint64(0), C.c_uint64(0)
+        _check(lib().twist_plan_stats(self.handle, C.byref(a), C.byref(b), C.byref(c)), "twist_plan_stats")
+        return a.value, b.value, c.value
+
+    def close(self):
+        if self.handle and self.handle.value:
+            lib().twist_plan_destroy(self.handle)
+            self.handle = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
 
 
 class LayerNormArgs(C.Structure):
@@ -132,6 +177,10 @@ def lib() -> C.CDLL:
         h.twist_hidden_mask.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p]
         h.twist_qkv_col_mask.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int32,
                                          C.c_void_p, C.c_void_p, C.c_void_p]
+        h.twist_plan_create.argtypes = [C.c_void_p, C.c_void_p]
+        h.twist_plan_destroy.argtypes = [C.c_void_p]
+        h.twist_plan_stats.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+        h.twist_workspace_bytes.argtypes = [C.c_void_p, C.c_void_p]
         h.twist_apply_col_mask.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_void_p]
         h.twist_gather_subnets.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_void_p]
         h.twist_aggregate.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_uint32, C.c_void_p]
@@ -260,8 +309,12 @@ def _ws_bytes(ws) -> int:
     return 0 if ws is None else ws.numel() * ws.element_size()
 
 
+def _plan_ptr(plan) -> Optional[int]:
+    return None if plan is None else plan.ptr
+
+
 def ffn_args(ffn_kind, dtype, n_subnets, tokens, d_model, f_sub, out_scale, lr=0.0, opt: Optional[Optimizer] = None,
-             **t) -> FfnArgs:
+             plan: Optional["Plan"] = None, **t) -> FfnArgs:
     """Marshals twist_ffn_args.  tgt / loss / loss_ws request the fused loss of the forward call; hidden_mask
     (uint8 [S][f_sub]) the activation mask of Masked TwIST."""
     names = ["x", "w_gu", "w_down", "w_gu_master", "w_down_master", "pre", "hh", "y", "dy", "dpre", "dx", "dw_gu",
@@ -272,8 +325,8 @@ def ffn_args(ffn_kind, dtype, n_subnets, tokens, d_model, f_sub, out_scale, lr=0
     a = FfnArgs(ffn_kind, dtype, n_subnets, tokens, d_model, f_sub, out_scale, lr, *[_ptr(t.get(n)) for n in names],
                 _ws_bytes(t.get("loss_ws")), _ptr(t.get("y_residual")), _ptr(t.get("dx_residual")),
                 opt if opt is not None else Optimizer(), *[_ptr(t.get(n)) for n in moments],
-                _ptr(t.get("hidden_mask")))
-    a._keepalive = list(t.values())      # the struct holds raw addresses: keep the tensors alive as long as it lives
+                _ptr(t.get("hidden_mask")), _plan_ptr(plan))
+    a._keepalive = list(t.values()) + [plan]      # the struct holds raw addresses: keep their owners alive with it
     return a
 
 
@@ -286,7 +339,7 @@ def twist_subnet_ffn_bwd(a: FfnArgs):
 
 
 def proj_args(which, dtype, n_subnets, tokens, d_model, n, out_scale, lr=0.0, seg_begin=0, seg_width=0,
-              opt: Optional[Optimizer] = None, **t) -> ProjArgs:
+              opt: Optional[Optimizer] = None, plan: Optional["Plan"] = None, **t) -> ProjArgs:
     """Marshals twist_proj_args.  tgt / loss / loss_ws (and the optional column mask valid_cols,
     seg_begin, seg_width) request the fused loss of the forward call."""
     names = ["in_", "w", "w_master", "out", "d_out", "d_in", "dw", "tgt", "loss", "loss_ws"]
@@ -295,8 +348,8 @@ def proj_args(which, dtype, n_subnets, tokens, d_model, n, out_scale, lr=0.0, se
     a = ProjArgs(which, dtype, n_subnets, tokens, d_model, n, out_scale, lr, *[_ptr(t.get(n)) for n in names],
                  _ws_bytes(t.get("loss_ws")), _ptr(t.get("valid_cols")), seg_begin, seg_width,
                  _ptr(t.get("out_residual")), _ptr(t.get("d_in_residual")), opt if opt is not None else Optimizer(),
-                 _ptr(t.get("m")), _ptr(t.get("v")), _ptr(t.get("col_mask")))
-    a._keepalive = list(t.values())
+                 _ptr(t.get("m")), _ptr(t.get("v")), _ptr(t.get("col_mask")), _plan_ptr(plan))
+    a._keepalive = list(t.values()) + [plan]
     return a
 
 
@@ -309,13 +362,13 @@ def twist_subnet_attn_proj_bwd(a: ProjArgs):
 
 
 def attn_core_args(dtype, n_subnets, n_seqs, seq_len, head_keep, kv_max, d_head, n_heads=0, n_kv_heads=0,
-                   **t) -> AttnCoreArgs:
+                   plan: Optional["Plan"] = None, **t) -> AttnCoreArgs:
     names = ["qkv", "out", "lse", "d_out", "d_qkv", "delta", "head_idx", "kv_pos", "kv_count"]
     unknown = set(t) - set(names)
     assert not unknown, unknown
     a = AttnCoreArgs(dtype, n_subnets, n_seqs, seq_len, head_keep, kv_max, d_head, n_heads, n_kv_heads,
-                     *[_ptr(t.get(n)) for n in names])
-    a._keepalive = list(t.values())
+                     *[_ptr(t.get(n)) for n in names], _plan_ptr(plan))
+    a._keepalive = list(t.values()) + [plan]
     return a
 
 

@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libtwist.so")
-SOURCES = ["common.cu", "masks.cu", "gather_aggregate.cu", "glue.cu", "gemm_sm100.cu", "train.cu", "attn_core.cu", "attn_core_tc.cu", "layernorm.cu"]
+SOURCES = ["common.cu", "masks.cu", "gather_aggregate.cu", "glue.cu", "gemm_sm100.cu", "train.cu", "attn_core.cu", "attn_core_tc.cu", "layernorm.cu", "plan.cu"]
 
 
 def _nvcc() -> str:

@@ -11,6 +11,7 @@
 // maximum and sum (one rescale per 8 keys) and stores the log-sum-exp; the backward recomputes
 // the probabilities from it.  Every result has one writer: deterministic, no atomics.
 #include "attn_core.cuh"
+#include "plan.cuh"
 
 namespace twist {
 namespace {
@@ -363,6 +364,7 @@ extern "C" int32_t twist_attn_core_fwd(const twist_attn_core_args* a, void* stre
   int rc = check(a);
   if (rc != TWIST_OK) return rc;
   if (!a->out || !aligned16(a->out)) return a->out ? TWIST_ERR_SHAPE : TWIST_ERR_NULL;
+  PlanScope scope(a->plan);
   return dispatch(make_params(a), a->n_subnets, false, static_cast<cudaStream_t>(stream));
 }
 
@@ -372,5 +374,6 @@ extern "C" int32_t twist_attn_core_bwd(const twist_attn_core_args* a, void* stre
   if (rc != TWIST_OK) return rc;
   if (!a->out || !a->d_out || !a->d_qkv || !a->delta) return TWIST_ERR_NULL;
   if (!aligned16(a->out) || !aligned16(a->d_out) || !aligned16(a->d_qkv)) return TWIST_ERR_SHAPE;
+  PlanScope scope(a->plan);
   return dispatch(make_params(a), a->n_subnets, true, static_cast<cudaStream_t>(stream));
 }

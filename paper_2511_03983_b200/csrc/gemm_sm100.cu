@@ -3,6 +3,8 @@
 
 #include <cudaTypedefs.h>
 
+#include "plan.cuh"
+
 namespace twist {
 namespace {
 
@@ -23,23 +25,38 @@ EncodeTiledFn encode_fn() {
   return fn;
 }
 
+// Encodes a 3-D tiled bf16 tensor map, or takes it from the calling thread's active plan (plan.cuh).
+int encode_or_cached(CUtensorMap* map, const void* ptr, const cuuint64_t dims[3], const cuuint64_t strides[2],
+                     const cuuint32_t box[3], CUtensorMapSwizzle swizzle, CUtensorMapL2promotion promotion,
+                     const char* what) {
+  MapKey key;
+  memset(&key, 0, sizeof(key));
+  key.ptr = ptr;
+  for (int i = 0; i < 3; ++i) { key.dims[i] = dims[i]; key.box[i] = box[i]; }
+  key.strides[0] = strides[0]; key.strides[1] = strides[1];
+  key.swizzle = (unsigned)swizzle; key.promotion = (unsigned)promotion;
+  if (plan_lookup(key, map)) return TWIST_OK;
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) { note_cuda_error(cudaErrorUnknown, "cuTensorMapEncodeTiled entry point"); return TWIST_ERR_CUDA; }
+  cuuint32_t estr[3] = {1, 1, 1};
+  CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle, promotion, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    note_cuda_error(cudaErrorInvalidValue, what);
+    return TWIST_ERR_CUDA;
+  }
+  plan_store(key, *map);
+  return TWIST_OK;
+}
+
 // 3-D map over dense bf16 [groups][rows][cols]; box = 64 contiguous elements x box_rows rows, 128-byte swizzle,
 // out-of-range elements read as zero (ragged M / N / K tails need no special code).
 int make_map(CUtensorMap* map, const GemmOperand& op, int groups, int box_rows) {
-  EncodeTiledFn fn = encode_fn();
-  if (!fn) { note_cuda_error(cudaErrorUnknown, "cuTensorMapEncodeTiled entry point"); return TWIST_ERR_CUDA; }
   cuuint64_t dims[3] = {(cuuint64_t)op.cols, (cuuint64_t)op.rows, (cuuint64_t)groups};
   cuuint64_t strides[2] = {(cuuint64_t)op.cols * 2, (cuuint64_t)op.rows * (cuuint64_t)op.cols * 2};
   cuuint32_t box[3] = {64, (cuuint32_t)box_rows, 1};
-  cuuint32_t estr[3] = {1, 1, 1};
-  CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(op.ptr), dims, strides, box, estr,
-                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  if (r != CUDA_SUCCESS) {
-    note_cuda_error(cudaErrorInvalidValue, "cuTensorMapEncodeTiled");
-    return TWIST_ERR_CUDA;
-  }
-  return TWIST_OK;
+  return encode_or_cached(map, op.ptr, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                          "cuTensorMapEncodeTiled");
 }
 
 // CTA pairs that can be resident at once (one CTA per SM, pairs on neighbouring SMs); queried once per
@@ -78,21 +95,12 @@ int resident_pairs(int* out) {
 // epilogue's 32 x 32 boxes (64-byte rows in shared memory, 64-byte swizzle).  Loads read zeros outside
 // the tensor, stores write nothing there.
 int make_box_map(CUtensorMap* map, const void* ptr, int rows, int cols, long long row_stride, int groups) {
-  EncodeTiledFn fn = encode_fn();
-  if (!fn) { note_cuda_error(cudaErrorUnknown, "cuTensorMapEncodeTiled entry point"); return TWIST_ERR_CUDA; }
   if (!ptr || !aligned16(ptr) || (row_stride * 2) % 16 != 0) return TWIST_ERR_SHAPE;
   cuuint64_t dims[3] = {(cuuint64_t)cols, (cuuint64_t)rows, (cuuint64_t)groups};
   cuuint64_t strides[2] = {(cuuint64_t)row_stride * 2, (cuuint64_t)rows * (cuuint64_t)row_stride * 2};
   cuuint32_t box[3] = {32, 32, 1};
-  cuuint32_t estr[3] = {1, 1, 1};
-  CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, estr,
-                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  if (r != CUDA_SUCCESS) {
-    note_cuda_error(cudaErrorInvalidValue, "cuTensorMapEncodeTiled (epilogue box)");
-    return TWIST_ERR_CUDA;
-  }
-  return TWIST_OK;
+  return encode_or_cached(map, ptr, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                          "cuTensorMapEncodeTiled (epilogue box)");
 }
 
 // Tensor maps of the boxes each epilogue reads and writes (layout of EpiMaps in the kernel header).
@@ -186,21 +194,12 @@ selftest_wait_kernel(unsigned long long limit_ns, int* status) {
 
 int encode_map_3d_bf16(CUtensorMap* map, const void* ptr, const unsigned long long dims[3],
                        const unsigned long long strides[2], const unsigned box[3], int swizzle_bytes) {
-  EncodeTiledFn fn = encode_fn();
-  if (!fn) { note_cuda_error(cudaErrorUnknown, "cuTensorMapEncodeTiled entry point"); return TWIST_ERR_CUDA; }
   if (!ptr || !aligned16(ptr) || strides[0] % 16 || strides[1] % 16) return TWIST_ERR_SHAPE;
   cuuint64_t d[3] = {dims[0], dims[1], dims[2]};
   cuuint64_t st[2] = {strides[0], strides[1]};
   cuuint32_t bx[3] = {box[0], box[1], box[2]};
-  cuuint32_t estr[3] = {1, 1, 1};
-  CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), d, st, bx, estr,
-                  CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B,
-                  CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  if (r != CUDA_SUCCESS) {
-    note_cuda_error(cudaErrorInvalidValue, "cuTensorMapEncodeTiled");
-    return TWIST_ERR_CUDA;
-  }
-  return TWIST_OK;
+  return encode_or_cached(map, ptr, d, st, bx, swizzle_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B,
+                          CU_TENSOR_MAP_L2_PROMOTION_L2_256B, "cuTensorMapEncodeTiled");
 }
 
 size_t fused_loss_partials(int groups, int M, int N) {

@@ -8,6 +8,7 @@
 
 #include "gemm_sm100.cuh"
 #include "glue.cuh"
+#include "plan.cuh"
 
 namespace twist {
 namespace {
@@ -105,6 +106,7 @@ extern "C" size_t twist_fused_loss_workspace_bytes(int32_t n_subnets, int32_t to
 
 extern "C" int32_t twist_subnet_ffn_fwd(const twist_ffn_args* a, void* stream) {
   TWIST_TRY(check_ffn(a));
+  PlanScope scope(a->plan);
   bool fused = false;
   TWIST_TRY(check_fused(a->tgt, a->loss, a->dy, a->loss_ws, a->loss_ws_bytes, a->n_subnets, a->tokens, a->d_model,
                         nullptr, 0, 0, &fused));
@@ -151,6 +153,7 @@ extern "C" int32_t twist_subnet_ffn_fwd(const twist_ffn_args* a, void* stream) {
 
 extern "C" int32_t twist_subnet_ffn_bwd(const twist_ffn_args* a, void* stream) {
   TWIST_TRY(check_ffn(a));
+  PlanScope scope(a->plan);
   if (!a->x || !a->w_gu || !a->w_down || !a->pre || !a->hh || !a->dy || !a->dpre) return TWIST_ERR_NULL;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const int S = a->n_subnets, T = a->tokens, d = a->d_model, f = a->f_sub;
@@ -236,6 +239,7 @@ static int check_proj(const twist_proj_args* a) {
 
 extern "C" int32_t twist_subnet_attn_proj_fwd(const twist_proj_args* a, void* stream) {
   TWIST_TRY(check_proj(a));
+  PlanScope scope(a->plan);
   const int S = a->n_subnets, T = a->tokens, d = a->d_model, n = a->n;
   const bool qkv = a->which == TWIST_PROJ_QKV;
   const int w_out = qkv ? n : d;      // width of the output
@@ -278,6 +282,7 @@ extern "C" int32_t twist_subnet_attn_proj_fwd(const twist_proj_args* a, void* st
 
 extern "C" int32_t twist_subnet_attn_proj_bwd(const twist_proj_args* a, void* stream) {
   TWIST_TRY(check_proj(a));
+  PlanScope scope(a->plan);
   if (!a->in || !a->w || !a->d_out) return TWIST_ERR_NULL;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const int S = a->n_subnets, T = a->tokens, d = a->d_model, n = a->n;

@@ -19,6 +19,7 @@ from __future__ import annotations
 
 import math
 from contextlib import contextmanager
+from functools import partial
 from typing import Dict, List, Optional, Tuple
 
 import torch
@@ -116,9 +117,12 @@ class RoundEngine:
         self.y, self.dy = act(d), act(d)
         self.dx = act(d) if compute_dx else None
         self.loss = torch.zeros(L, 3, max(1, w.local_steps), S, dtype=torch.float32, device=dev)
-        nq_max = max(gm.nq for gm in self.geo.values())
-        ws_bytes = max(B.twist_mse_workspace_bytes(S), B.twist_fused_loss_workspace_bytes(S, T, max(d, nq_max)))
-        self.ws = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
+        # the plan: shapes of the workload and the cache of encoded tensor maps; every GEMM / attention call carries it
+        self.plan = B.Plan(w)
+        self._ffn_args = partial(B.ffn_args, plan=self.plan)
+        self._proj_args = partial(B.proj_args, plan=self.plan)
+        self._attn_core_args = partial(B.attn_core_args, plan=self.plan)
+        self.ws = torch.empty(self.plan.workspace_bytes(), dtype=torch.uint8, device=dev)     # scratch of the loss calls
         # batches: lists over the local step k of [S][T][width] tensors (Tq and A: per geometry, see the properties)
         self.X: List[torch.Tensor] = []
         self.Td: List[torch.Tensor] = []
@@ -342,7 +346,7 @@ class RoundEngine:
         w = self.w
         lr = w.lr if lr is None else lr
         fused = dict(tgt=self.Td[k], loss=self.loss[l, 0, k], loss_ws=self.ws) if self.fuse_loss else {}
-        a = B.ffn_args(w.ffn_kind, w.dtype, w.n_subnets, w.tokens, w.d_model, self.f_sub, self.alpha_f, lr,
+        a = self._ffn_args(w.ffn_kind, w.dtype, w.n_subnets, w.tokens, w.d_model, self.f_sub, self.alpha_f, lr,
                        x=self.X[k], w_gu=self.w_gu, w_down=self.w_down, w_gu_master=self.w_gu_m,
                        w_down_master=self.w_down_m, pre=self.pre, hh=self.hh,
                        y=self.y if self.store_outputs else None, dy=self.dy, dpre=self.dpre,
@@ -377,7 +381,7 @@ class RoundEngine:
         mask = self._qkv_loss_mask(l)
         ragged = bool(mask)
         fused = dict(tgt=self.Tq[k], loss=self.loss[l, 1, k], loss_ws=self.ws, **mask) if self.fuse_loss else {}
-        a = B.proj_args(B.PROJ_QKV, w.dtype, w.n_subnets, w.tokens, w.d_model, self.nq, 1.0, lr, in_=self.X[k],
+        a = self._proj_args(B.PROJ_QKV, w.dtype, w.n_subnets, w.tokens, w.d_model, self.nq, 1.0, lr, in_=self.X[k],
                         w=self.w_qkv, w_master=self.w_qkv_m, out=self.qkv_out if self.store_outputs else None,
                         d_out=self.dqkv, d_in=self.dx, dw=self.dw_qkv, **fused, **self._opt(k, ("", "w_qkv")))
         with self._timed("qkv_fwd"):
@@ -396,7 +400,7 @@ class RoundEngine:
         w = self.w
         lr = w.lr if lr is None else lr
         fused = dict(tgt=self.Td[k], loss=self.loss[l, 2, k], loss_ws=self.ws) if self.fuse_loss else {}
-        a = B.proj_args(B.PROJ_O, w.dtype, w.n_subnets, w.tokens, w.d_model, self.a_sub, self.alpha_a, lr,
+        a = self._proj_args(B.PROJ_O, w.dtype, w.n_subnets, w.tokens, w.d_model, self.a_sub, self.alpha_a, lr,
                         in_=self.A[k], w=self.w_o, w_master=self.w_o_m, out=self.y if self.store_outputs else None,
                         d_out=self.dy, d_in=self.da, dw=self.dw_o, **fused, **self._o_mask(l),
                         **self._opt(k, ("", "w_o")))
@@ -426,7 +430,7 @@ class RoundEngine:
         self._use(l)
         w = self.w
         assert self.fuse_loss, "evaluation uses the loss fused into the forward kernels"
-        a = B.ffn_args(w.ffn_kind, w.dtype, w.n_subnets, w.tokens, w.d_model, self.f_sub, self.alpha_f, 0.0, x=self.X[k],
+        a = self._ffn_args(w.ffn_kind, w.dtype, w.n_subnets, w.tokens, w.d_model, self.f_sub, self.alpha_f, 0.0, x=self.X[k],
                        w_gu=self.w_gu, w_down=self.w_down, pre=self.pre, hh=self.hh,
                        y=self.y if self.store_outputs else None, dy=self.dy, tgt=self.Td[k], loss=self.loss[l, 0, k],
                        loss_ws=self.ws)
@@ -435,11 +439,11 @@ class RoundEngine:
         if self.has_attn:
             ragged = w.n_kv_heads != w.n_heads
             mask = dict(valid_cols=self.kv_cols[l], seg_begin=self.a_sub, seg_width=self.kv_max * w.d_head) if ragged else {}
-            q = B.proj_args(B.PROJ_QKV, w.dtype, w.n_subnets, w.tokens, w.d_model, self.nq, 1.0, 0.0, in_=self.X[k],
+            q = self._proj_args(B.PROJ_QKV, w.dtype, w.n_subnets, w.tokens, w.d_model, self.nq, 1.0, 0.0, in_=self.X[k],
                             w=self.w_qkv, out=self.qkv_out if self.store_outputs else None, d_out=self.dqkv,
                             tgt=self.Tq[k], loss=self.loss[l, 1, k], loss_ws=self.ws, **mask)
             B.twist_subnet_attn_proj_fwd(q)
-            o = B.proj_args(B.PROJ_O, w.dtype, w.n_subnets, w.tokens, w.d_model, self.a_sub, self.alpha_a, 0.0,
+            o = self._proj_args(B.PROJ_O, w.dtype, w.n_subnets, w.tokens, w.d_model, self.a_sub, self.alpha_a, 0.0,
                             in_=self.A[k], w=self.w_o, out=self.y if self.store_outputs else None, d_out=self.dy,
                             tgt=self.Td[k], loss=self.loss[l, 2, k], loss_ws=self.ws)
             B.twist_subnet_attn_proj_fwd(o)
@@ -458,7 +462,7 @@ class RoundEngine:
             self.e_hh = torch.empty(1, T, F, dtype=bf, device=self.dev)
             self.e_loss = torch.zeros(w.n_subnets, dtype=torch.float32, device=self.dev)
         for s in range(w.n_subnets):
-            a = B.ffn_args(w.ffn_kind, w.dtype, 1, T, d, F, 1.0, 0.0, x=self.X[k][s:s + 1], w_gu=self.full_gu[l],
+            a = self._ffn_args(w.ffn_kind, w.dtype, 1, T, d, F, 1.0, 0.0, x=self.X[k][s:s + 1], w_gu=self.full_gu[l],
                            w_down=self.full["down"][l], pre=self.e_pre, hh=self.e_hh, y=None, dy=self.dy[s:s + 1],
                            tgt=self.Td[k][s:s + 1], loss=self.e_loss[s:s + 1], loss_ws=self.ws)
             B.twist_subnet_ffn_fwd(a)
@@ -662,14 +666,14 @@ class HybridRoundEngine(RoundEngine):
         central_opt = self._central_opt(k, ("_gu", "c_gu"), ("_down", "c_down"))
         others_opt = self._others_opt(k, ("_gu", "w_gu"), ("_down", "w_down"))
         # central worker: the full-width layer under its mask, updated in place
-        c = B.ffn_args(w.ffn_kind, w.dtype, 1, T, d, F, self.alpha_f, lr, x=self.X[k][:1], w_gu=self.full_gu[l],
+        c = self._ffn_args(w.ffn_kind, w.dtype, 1, T, d, F, self.alpha_f, lr, x=self.X[k][:1], w_gu=self.full_gu[l],
                        w_down=self.full["down"][l], w_gu_master=self.full_gu_f32[l],
                        w_down_master=self.full_f32["down"][l], pre=self.c_pre, hh=self.c_hh,
                        y=self.y[:1] if self.store_outputs else None, dy=self.dy[:1], dpre=self.c_dpre,
                        dx=self.dx[:1] if self.dx is not None else None, hidden_mask=self.c_mask,
                        tgt=self.Td[k][:1], loss=self.loss[l, 0, k][:1], loss_ws=self.ws, **central_opt)
         # workers 1 .. S-1: gathered slices
-        o = B.ffn_args(w.ffn_kind, w.dtype, S - 1, T, d, w.f_sub, self.alpha_f, lr, x=self.X[k][1:], w_gu=self.w_gu[1:],
+        o = self._ffn_args(w.ffn_kind, w.dtype, S - 1, T, d, w.f_sub, self.alpha_f, lr, x=self.X[k][1:], w_gu=self.w_gu[1:],
                        w_down=self.w_down[1:], w_gu_master=self.w_gu_m[1:], w_down_master=self.w_down_m[1:],
                        pre=self.pre[1:], hh=self.hh[1:], y=self.y[1:] if self.store_outputs else None, dy=self.dy[1:],
                        dpre=self.dpre[1:], dx=self.dx[1:] if self.dx is not None else None, tgt=self.Td[k][1:],
@@ -687,12 +691,12 @@ class HybridRoundEngine(RoundEngine):
         lr = w.lr if lr is None else lr
         S, T, d = w.n_subnets, w.tokens, w.d_model
         dx = lambda sl: self.dx[sl] if self.dx is not None else None
-        c = B.proj_args(B.PROJ_QKV, w.dtype, 1, T, d, self.c_nq, 1.0, lr, in_=self.X[k][:1], w=self.full["qkv"][l],
+        c = self._proj_args(B.PROJ_QKV, w.dtype, 1, T, d, self.c_nq, 1.0, lr, in_=self.X[k][:1], w=self.full["qkv"][l],
                         w_master=self.full_f32["qkv"][l], out=self.c_qkv_out, d_out=self.c_dqkv, d_in=dx(slice(0, 1)),
                         tgt=self.Tq_c[k], loss=self.loss[l, 1, k][:1], loss_ws=self.ws, col_mask=self.c_qkv_mask,
                         valid_cols=self.c_qkv_count, **self._central_opt(k, ("", "c_qkv")))
         mask = {key: (v[1:] if key == "valid_cols" else v) for key, v in self._qkv_loss_mask(l).items()}
-        o = B.proj_args(B.PROJ_QKV, w.dtype, S - 1, T, d, self.nq, 1.0, lr, in_=self.X[k][1:], w=self.w_qkv[1:],
+        o = self._proj_args(B.PROJ_QKV, w.dtype, S - 1, T, d, self.nq, 1.0, lr, in_=self.X[k][1:], w=self.w_qkv[1:],
                         w_master=self.w_qkv_m[1:], out=self.qkv_out[1:] if self.store_outputs else None,
                         d_out=self.dqkv[1:], d_in=dx(slice(1, None)), tgt=self.Tq[k][1:], loss=self.loss[l, 1, k][1:],
                         loss_ws=self.ws, **mask, **self._others_opt(k, ("", "w_qkv")))
@@ -709,11 +713,11 @@ class HybridRoundEngine(RoundEngine):
         lr = w.lr if lr is None else lr
         S, T, d = w.n_subnets, w.tokens, w.d_model
         B.twist_apply_col_mask(self.A_c[k], self.c_a_mask, self.c_a_masked, 1, T, self.c_a)     # Sec. 4.1: M * f(x)
-        c = B.proj_args(B.PROJ_O, w.dtype, 1, T, d, self.c_a, self.alpha_a, lr, in_=self.c_a_masked, w=self.full["o"][l],
+        c = self._proj_args(B.PROJ_O, w.dtype, 1, T, d, self.c_a, self.alpha_a, lr, in_=self.c_a_masked, w=self.full["o"][l],
                         w_master=self.full_f32["o"][l], out=self.y[:1] if self.store_outputs else None,
                         d_out=self.dy[:1], d_in=self.c_da, tgt=self.Td[k][:1], loss=self.loss[l, 2, k][:1],
                         loss_ws=self.ws, col_mask=self.c_a_mask, **self._central_opt(k, ("", "c_o")))
-        o = B.proj_args(B.PROJ_O, w.dtype, S - 1, T, d, self.a_sub, self.alpha_a, lr, in_=self.A[k][1:], w=self.w_o[1:],
+        o = self._proj_args(B.PROJ_O, w.dtype, S - 1, T, d, self.a_sub, self.alpha_a, lr, in_=self.A[k][1:], w=self.w_o[1:],
                         w_master=self.w_o_m[1:], out=self.y[1:] if self.store_outputs else None, d_out=self.dy[1:],
                         d_in=self.da[1:] if self.da is not None else None, tgt=self.Td[k][1:],
                         loss=self.loss[l, 2, k][1:], loss_ws=self.ws, **self._others_opt(k, ("", "w_o")))
@@ -818,7 +822,7 @@ class StackEngine(RoundEngine):
     def _core_args(self, l: int, **t):
         w = self.w
         extra = dict(head_idx=self.idx_head[l], kv_pos=self.kv_pos[l], kv_count=self.kv_count[l]) if self.gqa else {}
-        return B.attn_core_args(w.dtype, w.n_subnets, self.n_seqs, self.seq_len, self.head_keep, self.kv_max, w.d_head,
+        return self._attn_core_args(w.dtype, w.n_subnets, self.n_seqs, self.seq_len, self.head_keep, self.kv_max, w.d_head,
                                 w.n_heads, w.n_kv_heads, **extra, **t)
 
     # ------------------------------------------------------------------ layer normalisation
@@ -873,12 +877,12 @@ class StackEngine(RoundEngine):
                 self._ln_fwd(l, "a", self.x[l], self.x_ln)
                 x_a = self.x_ln
             with self._timed("qkv_fwd"):
-                B.twist_subnet_attn_proj_fwd(B.proj_args(B.PROJ_QKV, w.dtype, S, T, d, self.nq, 1.0, 0.0, in_=x_a,
+                B.twist_subnet_attn_proj_fwd(self._proj_args(B.PROJ_QKV, w.dtype, S, T, d, self.nq, 1.0, 0.0, in_=x_a,
                                                          w=self.w_qkv, out=self.qkv_l[l]))
             with self._timed("core_fwd"):
                 B.twist_attn_core_fwd(self._core_args(l, qkv=self.qkv_l[l], out=self.a_l[l], lse=self.lse[l]))
             with self._timed("o_fwd"):
-                B.twist_subnet_attn_proj_fwd(B.proj_args(B.PROJ_O, w.dtype, S, T, d, self.a_sub, self.alpha_a, 0.0,
+                B.twist_subnet_attn_proj_fwd(self._proj_args(B.PROJ_O, w.dtype, S, T, d, self.a_sub, self.alpha_a, 0.0,
                                                          in_=self.a_l[l], w=self.w_o, out=self.x_mid[l],
                                                          out_residual=self.x[l]))
             x_f = self.x_mid[l]
@@ -886,7 +890,7 @@ class StackEngine(RoundEngine):
                 self._ln_fwd(l, "f", self.x_mid[l], self.x_ln)
                 x_f = self.x_ln
             with self._timed("ffn_fwd"):
-                B.twist_subnet_ffn_fwd(B.ffn_args(w.ffn_kind, w.dtype, S, T, d, self.f_sub, self.alpha_f, 0.0,
+                B.twist_subnet_ffn_fwd(self._ffn_args(w.ffn_kind, w.dtype, S, T, d, self.f_sub, self.alpha_f, 0.0,
                                                   x=x_f, w_gu=self.w_gu, w_down=self.w_down, pre=self.pre_l[l],
                                                   hh=self.hh_l[l], y=self.x[l + 1], y_residual=self.x_mid[l]))
             self.launches += 5
@@ -905,7 +909,7 @@ class StackEngine(RoundEngine):
                 self._ln_fwd(l, "f", self.x_mid[l], self.x_ln)
                 x_f = self.x_ln
             with self._timed("ffn_bwd"):
-                B.twist_subnet_ffn_bwd(B.ffn_args(w.ffn_kind, w.dtype, S, T, d, self.f_sub, self.alpha_f, lr,
+                B.twist_subnet_ffn_bwd(self._ffn_args(w.ffn_kind, w.dtype, S, T, d, self.f_sub, self.alpha_f, lr,
                                                   x=x_f, w_gu=self.w_gu, w_down=self.w_down,
                                                   w_gu_master=self.w_gu_m, w_down_master=self.w_down_m,
                                                   pre=self.pre_l[l], hh=self.hh_l[l], dy=g, dpre=self.dpre,
@@ -916,7 +920,7 @@ class StackEngine(RoundEngine):
             if self.ln:
                 self._ln_bwd(l, "f", k, lr, self.x_mid[l], self.d_ln, g_mid, g)
             with self._timed("o_bwd"):
-                B.twist_subnet_attn_proj_bwd(B.proj_args(B.PROJ_O, w.dtype, S, T, d, self.a_sub, self.alpha_a, lr,
+                B.twist_subnet_attn_proj_bwd(self._proj_args(B.PROJ_O, w.dtype, S, T, d, self.a_sub, self.alpha_a, lr,
                                                          in_=self.a_l[l], w=self.w_o, w_master=self.w_o_m, d_out=g_mid,
                                                          d_in=self.da, dw=self.dw_o, **self._opt(k, ("", "w_o"))))
             with self._timed("core_bwd"):
@@ -927,7 +931,7 @@ class StackEngine(RoundEngine):
                 self._ln_fwd(l, "a", self.x[l], self.x_ln)
                 x_a = self.x_ln
             with self._timed("qkv_bwd"):
-                B.twist_subnet_attn_proj_bwd(B.proj_args(B.PROJ_QKV, w.dtype, S, T, d, self.nq, 1.0, lr, in_=x_a,
+                B.twist_subnet_attn_proj_bwd(self._proj_args(B.PROJ_QKV, w.dtype, S, T, d, self.nq, 1.0, lr, in_=x_a,
                                                          w=self.w_qkv, w_master=self.w_qkv_m, d_out=self.dqkv,
                                                          d_in=self.d_ln if self.ln else g,
                                                          d_in_residual=None if self.ln else g_mid, dw=self.dw_qkv,

@@ -97,6 +97,36 @@ def test_host_side_argument_checks():
     assert h.twist_subnet_ffn_fwd(C.byref(a), None) == B.ERR_UNSUPPORTED
 
 
+def test_plan_object_validates_its_configuration_and_sizes_the_scratch():
+    from paper_2511_03983_b200 import binding as B
+    from paper_2511_03983_b200 import inputs as I
+    h = B.lib()
+    for cfg in (2, 3, 4, 5):
+        w = I.PRESETS[cfg]
+        plan = B.Plan(w)
+        need = plan.workspace_bytes()
+        widths = [w.d_model] + ([(w.n_heads + 2 * w.n_kv_heads) * w.d_head] if w.n_heads else [])
+        assert need >= B.twist_mse_workspace_bytes(w.n_subnets)
+        assert need >= max(B.twist_fused_loss_workspace_bytes(w.n_subnets, w.tokens, x) for x in widths)
+        assert need >= B.twist_layernorm_workspace_bytes(w.n_subnets, w.tokens, w.d_model)
+        assert plan.stats() == (0, 0, 0)
+        plan.close()
+    good = B.Config(C.sizeof(B.Config), 2, 64, 4, 2, 16, 256, B.FFN_SWIGLU, 4, 1, 128, 2, B.MODE_COVER, B.BF16, 128, 0, 7)
+    out = C.c_void_p()
+    assert h.twist_plan_create(C.byref(good), C.byref(out)) == 0 and out.value
+    assert h.twist_plan_destroy(out) == 0
+    assert h.twist_plan_create(None, C.byref(out)) == B.ERR_NULL and h.twist_plan_destroy(None) == B.ERR_NULL
+    import copy
+    for field, value, want in (("struct_size", 8, B.ERR_SHAPE), ("n_subnets", 33, B.ERR_UNSUPPORTED),
+                               ("ffn_keep", 257, B.ERR_INFEASIBLE), ("head_keep", 5, B.ERR_INFEASIBLE),
+                               ("n_kv_heads", 3, B.ERR_SHAPE), ("tokens", 0, B.ERR_SHAPE), ("ffn_block", 3, B.ERR_SHAPE)):
+        bad = copy.copy(good)
+        setattr(bad, field, value)
+        out = C.c_void_p()
+        assert h.twist_plan_create(C.byref(bad), C.byref(out)) == want, field
+        assert not out.value
+
+
 def test_misaligned_pointers_are_refused_before_any_launch():
     """The kernels use 16-byte (the activation mask: 8-byte) vector accesses; a pointer that breaks the rule must
     come back as a status, never reach the device."""

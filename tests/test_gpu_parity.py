@@ -1042,3 +1042,39 @@ def test_hybrid_twist_round_with_attention_matches_the_oracle_round(B, cfg, dims
     w = replace(I.scaled_twin(I.PRESETS[cfg], **dims), **extra)
     eng, before = _run_round_and_compare(B, w, engine_cls=HybridRoundEngine)
     assert any(not torch.equal(eng.full[m], before[m]) for m in ("qkv", "o"))
+
+
+def test_plan_caches_tensor_maps_and_changes_no_result(B):
+    """The same FFN forward / backward on the same buffers without a plan, with a fresh plan, and with the warm plan:
+    bit-identical results; the warm pass encodes no tensor map (every lookup hits)."""
+    S, T, d, f = 2, 200, 328, 344
+    plan = B.Plan(replace(I.PRESETS[5], n_subnets=S, tokens=T, d_model=d, d_ff=4 * f, ffn_keep=f))
+    bf = torch.bfloat16
+    t = lambda *shape: torch.zeros(*shape, dtype=bf, device="cuda")
+    X = dev(I.normal(97, 1, (S, T, d), 1.0, I.DTYPE_BF16), bf)
+    dY = dev(I.normal(97, 4, (S, T, d), 1e-3, I.DTYPE_BF16), bf)
+    Wgu = dev(I.normal(97, 2, (S, 2 * f, d), 0.05, I.DTYPE_BF16), bf)
+    Wd = dev(I.normal(97, 3, (S, f, d), 0.05, I.DTYPE_BF16), bf)
+    buf = dict(w_gu=t(S, 2 * f, d), w_down=t(S, f, d), pre=t(S, T, 2 * f), hh=t(S, T, f), y=t(S, T, d),
+               dpre=t(S, T, 2 * f), dx=t(S, T, d))
+    buf["w_gu_master"] = torch.zeros(S, 2 * f, d, dtype=torch.float32, device="cuda")
+    buf["w_down_master"] = torch.zeros(S, f, d, dtype=torch.float32, device="cuda")
+    results, stats = [], []
+    for use_plan in (None, plan, plan):
+        buf["w_gu"].copy_(Wgu); buf["w_down"].copy_(Wd)
+        buf["w_gu_master"].copy_(Wgu.float()); buf["w_down_master"].copy_(Wd.float())
+        a = B.ffn_args(I.FFN_SWIGLU, I.DTYPE_BF16, S, T, d, f, 2.0, 0.5, plan=use_plan, x=X, dy=dY, **buf)
+        B.twist_subnet_ffn_fwd(a)
+        B.twist_subnet_ffn_bwd(a)
+        torch.cuda.synchronize()
+        check_status(B)
+        results.append({k: v.clone() for k, v in buf.items()})
+        stats.append(plan.stats())
+    for k in buf:
+        assert torch.equal(results[0][k], results[1][k]) and torch.equal(results[0][k], results[2][k]), k
+    assert not torch.equal(results[0]["w_gu"], Wgu)                      # the step did train
+    (c0, h0, m0), (c1, h1, m1), (c2, h2, m2) = stats
+    assert (c0, h0, m0) == (0, 0, 0)                                     # calls without the plan leave it alone
+    assert c1 > 0 and m1 == c1                                           # cold: every distinct map encoded once
+    assert c2 == c1 and m2 == m1 and h2 - h1 == h1 + m1                  # warm: as many lookups, all of them hits
+    plan.close()
