@@ -27,6 +27,9 @@ METRIC = "twist_round_tokens_per_s"
 UNIT = "tokens/s"
 # Nominal peaks of the part (dense bf16 tensor throughput, HBM3e bandwidth); fractions against them are reported
 # beside the fractions against the peaks measured on the machine.
+# dram bytes (read + write) of one 7B-shaped gather launch from the committed ncu capture (profiles/), None while
+# no capture of the current launch exists
+NCU_GATHER_TRAFFIC = None
 NOMINAL_BF16_TFLOPS = 2250.0
 NOMINAL_HBM_GBS = 8000.0
 
@@ -55,7 +58,9 @@ def round_work(w, nq_valid=None):
     flops_attn = 6.0 * T * d * (nq + a) if w.n_heads else 0.0
     gemm_flops = (flops_ffn + flops_attn) * S * K * L
     kept = (w.nmat * f + (nq + a if w.n_heads else 0)) * d    # kept elements per subnet per layer
-    gather_bytes = (2 + 2 + 4) * kept * S * L                 # read bf16, write bf16, write fp32 master
+    # read bf16, write bf16: the fp32 masters are not written by the gather, the first weight update of the round
+    # creates them from the bf16 slice (that update then reads 2 instead of 4 bytes per element)
+    gather_bytes = (2 + 2) * kept * S * L
     # aggregate: read every subnet's master (4 B) + write fp32 result and bf16 shadow for every covered element
     full = (w.nmat * w.d_ff + ((w.n_heads + 2 * w.n_kv_heads + w.n_heads) * w.d_head if w.n_heads else 0)) * d
     agg_bytes = 4 * kept * S * L + (4 + 2) * full * L         # cover mode: every element is covered
@@ -65,6 +70,29 @@ def round_work(w, nq_valid=None):
 # ------------------------------------------------------------------------------------------------
 # N > 1: independent replicas, one process per GPU (the path has no exchange step between GPUs).
 # ------------------------------------------------------------------------------------------------
+
+def spawn_replicas(n: int, argv, extra_env=None, timeout=None) -> int:
+    """Starts n copies of the command `argv`, one per GPU, with the environment a distributed launcher would give
+    them (RANK, LOCAL_RANK, WORLD_SIZE, MASTER_ADDR = 127.0.0.1, a free MASTER_PORT).  Rank 0's standard output
+    passes through (it prints the one JSON line); the others' is dropped.  Returns the largest exit code."""
+    import socket
+    with socket.socket() as sock:
+        sock.bind(("127.0.0.1", 0))
+        port = sock.getsockname()[1]
+    procs = []
+    for r in range(n):
+        env = dict(os.environ, RANK=str(r), LOCAL_RANK=str(r), WORLD_SIZE=str(n), MASTER_ADDR="127.0.0.1",
+                   MASTER_PORT=str(port), **(extra_env or {}))
+        procs.append(subprocess.Popen(argv, env=env, stdout=None if r == 0 else subprocess.DEVNULL))
+    rc = 0
+    for p in procs:
+        try:
+            rc = max(rc, abs(p.wait(timeout=timeout)))
+        except subprocess.TimeoutExpired:
+            p.kill()                       # the exact process this function started
+            rc = max(rc, 124)
+    return rc
+
 
 def replica_seed(base: int, rank: int) -> int:
     """Every replica draws its own weights and batches."""
@@ -331,9 +359,17 @@ def run_ours(args, w):
     # ---- end-to-end: host buffers, copies inside the timed region --------------------------------
     e2e = None
     if not args.no_e2e:
+        # Host side of the copies.  One replica pins all K batches of a round (distinct data per local step).  With
+        # several replicas on one host that would pin N x 25.8 GB, so each then pins one local step's batches and
+        # copies them K times per round: the same bytes cross the bus, the host memory stays bounded.
         pinned = {}
         for name, _ in widths:
-            pinned[name] = [t.cpu().pin_memory() for t in getattr(eng, name)]
+            lst = getattr(eng, name)
+            if world == 1:
+                pinned[name] = [t.cpu().pin_memory() for t in lst]
+            else:
+                one = lst[0].cpu().pin_memory()
+                pinned[name] = [one] * len(lst)
         loss_host = torch.empty(loss_dev.shape, dtype=torch.float32).pin_memory()
         n_e2e = max(1, min(args.steps, args.e2e_steps))
         # Two sets of device batch buffers: while a round runs on one, the next step's batches are copied into
@@ -376,7 +412,8 @@ def run_ours(args, w):
         e2e = {"value": whole_job_value(w.tokens_per_round, world, e2e_ms), "unit": UNIT,
                "h2d_bytes_per_step": h2d_bytes, "d2h_bytes_per_step": d2h_bytes, "steps": n_e2e,
                "note": "pinned host batches copied in (the next step's copy overlaps the current round on a second "
-                       "stream), per-subnet losses copied out, every step"}
+                       "stream), per-subnet losses copied out, every step"
+                       + ("" if world == 1 else "; each replica pins one local step's batches and copies them K times")}
 
     if rank != 0:
         if world > 1:
@@ -421,7 +458,7 @@ def run_ours(args, w):
                     "share_of_step": gemm_ms / ms_total}
     hbm = {}
     # DRAM bytes per launch from the committed ncu capture of one 7B-shaped layer (profiles/); only that launch shape
-    ncu_traffic = {"gather": 3.09e9, "aggregate": 2.79e9} if (args.config == 4 and not stack) else {}
+    ncu_traffic = {"gather": NCU_GATHER_TRAFFIC, "aggregate": 2.79e9} if (args.config == 4 and not stack) else {}
     for name, key in (("gather", "gather_bytes"), ("aggregate", "aggregate_bytes")):
         if name in phases and phases[name][0] > 0:
             gbs = work[key] * args.steps / (phases[name][0] / 1e3) / 1e9
@@ -488,7 +525,7 @@ def run_sweep(args):
             raise SystemExit("device status: a bounded device wait expired")
         kept = w.nmat * w.f_sub * w.d_model                                      # kept elements per subnet and layer
         covered = int((eng.cover_ffn != 0).sum().item()) * w.ffn_block * w.d_model * w.nmat   # last round, all layers
-        gather_b = 8.0 * kept * w.n_subnets * w.n_layers
+        gather_b = 4.0 * kept * w.n_subnets * w.n_layers
         agg_b = 4.0 * kept * w.n_subnets * w.n_layers + 6.0 * covered
         g_gbs = gather_b * args.steps / (ph["gather"][0] / 1e3) / 1e9
         a_gbs = agg_b * args.steps / (ph["aggregate"][0] / 1e3) / 1e9
@@ -505,8 +542,9 @@ def run_sweep(args):
                       "config": {"workload": "configs[4] gather/aggregate sweep on the 7B FFN shapes: d=4096 F=11008 "
                                              f"L={args.layers or 32} bf16 weights, fp32 aggregate, IID masks, K=1, "
                                              "1024 tokens per subnet",
-                                 "bytes": "gather 8 B per kept element (2 read, 2 write, 4 master); aggregate 4 B per "
-                                          "kept master element + 6 B per covered element"},
+                                 "bytes": "gather 4 B per kept element (2 read, 2 write; the fp32 masters are created by "
+                                          "the first weight update); aggregate 4 B per kept master element + 6 B per "
+                                          "covered element"},
                       "cells": cells}))
 
 
@@ -538,6 +576,9 @@ def main():
         w = replace(w, tokens=args.tokens, name=w.name + f"-T{args.tokens}")
     if args.local_steps:
         w = replace(w, local_steps=args.local_steps, name=w.name + f"-K{args.local_steps}")
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and args.impl == "ours" and not args.sweep:
+        # started as a plain command: become the launcher of one replica per GPU (replicas only, no collective)
+        raise SystemExit(spawn_replicas(args.gpus, [sys.executable, os.path.abspath(__file__)] + sys.argv[1:]))
     if args.impl == "reference":
         run_reference(args, w)
     elif args.sweep:

@@ -302,6 +302,11 @@ typedef struct {
    * TwIST's central model trains this way on its full copy).  NULL: no mask.  bf16 dtype only. */
   const uint8_t* hidden_mask;
   twist_plan* plan;         /* optional: tensor maps come from this plan's cache (see twist_plan) */
+  /* bwd, bf16 dtype: non-zero when the fp32 masters hold nothing yet (the slices were gathered without
+   * dst_master).  The update then reads the bf16 weights instead -- a freshly gathered slice's master is exactly
+   * its widening -- and writes the masters, also when lr == 0.  Pass it on the first backward call after a gather,
+   * 0 afterwards.  It saves the gather 4 of its 8 bytes per kept element. */
+  int32_t master_from_slice;
 } twist_ffn_args;
 
 /* Fused loss.  When `tgt` is set, twist_subnet_ffn_fwd / twist_subnet_attn_proj_fwd also evaluate the loss
@@ -355,6 +360,7 @@ typedef struct {
    * NULL: no mask.  bf16 dtype only. */
   const uint8_t* col_mask;
   twist_plan* plan;            /* optional: tensor maps come from this plan's cache */
+  int32_t master_from_slice;   /* bwd: as in twist_ffn_args */
 } twist_proj_args;
 
 int32_t twist_subnet_attn_proj_fwd(const twist_proj_args* a /*host*/, void* stream);

@@ -77,7 +77,8 @@ class FfnArgs(C.Structure):
                 ("dw_down", C.c_void_p), ("tgt", C.c_void_p), ("loss", C.c_void_p), ("loss_ws", C.c_void_p),
                 ("loss_ws_bytes", C.c_size_t), ("y_residual", C.c_void_p), ("dx_residual", C.c_void_p),
                 ("opt", Optimizer), ("m_gu", C.c_void_p), ("v_gu", C.c_void_p), ("m_down", C.c_void_p),
-                ("v_down", C.c_void_p), ("hidden_mask", C.c_void_p), ("plan", C.c_void_p)]
+                ("v_down", C.c_void_p), ("hidden_mask", C.c_void_p), ("plan", C.c_void_p),
+                ("master_from_slice", C.c_int32)]
 
 
 class ProjArgs(C.Structure):
@@ -88,7 +89,8 @@ class ProjArgs(C.Structure):
                 ("loss", C.c_void_p), ("loss_ws", C.c_void_p), ("loss_ws_bytes", C.c_size_t),
                 ("valid_cols", C.c_void_p), ("seg_begin", C.c_int32), ("seg_width", C.c_int32),
                 ("out_residual", C.c_void_p), ("d_in_residual", C.c_void_p), ("opt", Optimizer), ("m", C.c_void_p),
-                ("v", C.c_void_p), ("col_mask", C.c_void_p), ("plan", C.c_void_p)]
+                ("v", C.c_void_p), ("col_mask", C.c_void_p), ("plan", C.c_void_p),
+                ("master_from_slice", C.c_int32)]
 
 
 class AttnCoreArgs(C.Structure):
@@ -314,7 +316,7 @@ def _plan_ptr(plan) -> Optional[int]:
 
 
 def ffn_args(ffn_kind, dtype, n_subnets, tokens, d_model, f_sub, out_scale, lr=0.0, opt: Optional[Optimizer] = None,
-             plan: Optional["Plan"] = None, **t) -> FfnArgs:
+             plan: Optional["Plan"] = None, master_from_slice: bool = False, **t) -> FfnArgs:
     """Marshals twist_ffn_args.  tgt / loss / loss_ws request the fused loss of the forward call; hidden_mask
     (uint8 [S][f_sub]) the activation mask of Masked TwIST."""
     names = ["x", "w_gu", "w_down", "w_gu_master", "w_down_master", "pre", "hh", "y", "dy", "dpre", "dx", "dw_gu",
@@ -325,7 +327,7 @@ def ffn_args(ffn_kind, dtype, n_subnets, tokens, d_model, f_sub, out_scale, lr=0
     a = FfnArgs(ffn_kind, dtype, n_subnets, tokens, d_model, f_sub, out_scale, lr, *[_ptr(t.get(n)) for n in names],
                 _ws_bytes(t.get("loss_ws")), _ptr(t.get("y_residual")), _ptr(t.get("dx_residual")),
                 opt if opt is not None else Optimizer(), *[_ptr(t.get(n)) for n in moments],
-                _ptr(t.get("hidden_mask")), _plan_ptr(plan))
+                _ptr(t.get("hidden_mask")), _plan_ptr(plan), int(master_from_slice))
     a._keepalive = list(t.values()) + [plan]      # the struct holds raw addresses: keep their owners alive with it
     return a
 
@@ -339,7 +341,8 @@ def twist_subnet_ffn_bwd(a: FfnArgs):
 
 
 def proj_args(which, dtype, n_subnets, tokens, d_model, n, out_scale, lr=0.0, seg_begin=0, seg_width=0,
-              opt: Optional[Optimizer] = None, plan: Optional["Plan"] = None, **t) -> ProjArgs:
+              opt: Optional[Optimizer] = None, plan: Optional["Plan"] = None, master_from_slice: bool = False,
+              **t) -> ProjArgs:
     """Marshals twist_proj_args.  tgt / loss / loss_ws (and the optional column mask valid_cols,
     seg_begin, seg_width) request the fused loss of the forward call."""
     names = ["in_", "w", "w_master", "out", "d_out", "d_in", "dw", "tgt", "loss", "loss_ws"]
@@ -348,7 +351,7 @@ def proj_args(which, dtype, n_subnets, tokens, d_model, n, out_scale, lr=0.0, se
     a = ProjArgs(which, dtype, n_subnets, tokens, d_model, n, out_scale, lr, *[_ptr(t.get(n)) for n in names],
                  _ws_bytes(t.get("loss_ws")), _ptr(t.get("valid_cols")), seg_begin, seg_width,
                  _ptr(t.get("out_residual")), _ptr(t.get("d_in_residual")), opt if opt is not None else Optimizer(),
-                 _ptr(t.get("m")), _ptr(t.get("v")), _ptr(t.get("col_mask")), _plan_ptr(plan))
+                 _ptr(t.get("m")), _ptr(t.get("v")), _ptr(t.get("col_mask")), _plan_ptr(plan), int(master_from_slice))
     a._keepalive = list(t.values()) + [plan]
     return a
 

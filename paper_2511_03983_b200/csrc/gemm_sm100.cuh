@@ -72,6 +72,8 @@ struct GemmParams {
   __nv_bfloat16* out1;  // *_FWD: hh [g][M][f_sub].  MSE: gradient of the loss w.r.t. D, [g][M][N]
   const __nv_bfloat16* in0;   // DSWIGLU / DACT: pre.  MSE: target [g][M][N].  RESID: addend [g][M][N]
   float* master;        // SGD: fp32 master weights [g][M][N] (updated when lr != 0)
+  int master_init;      // SGD / ADAM: the masters hold nothing yet - read the bf16 weights (out0) instead, whose exact
+                        // widening they are, and write the masters (also when lr == 0)
   float* adam_m;        // ADAM: first / second moment of the group's weights, fp32 [g][M][N]
   float* adam_v;
   float beta1, beta2, adam_eps, bias1, bias2;   // ADAM: decay rates, epsilon, 1 / (1 - beta^t)
@@ -437,12 +439,23 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         const int n_base = nt * kBN + half * kHalfN;
         float4 mv[2][8];
         EpiAcc<EPI> acc[2];
+        const bool do_update = p.lr != 0.f || p.master_init != 0;
         auto load_master = [&](int c, float4 (&m)[8]) {
           const int n = n_base + 32 * c;
-          const int valid = (row_ok && n < p.N && p.lr != 0.f) ? min(32, p.N - n) : 0;
-          const float4* src = reinterpret_cast<const float4*>(p.master + grow * p.N + n);
+          const int valid = (row_ok && n < p.N && do_update) ? min(32, p.N - n) : 0;
+          if (p.master_init) {      // first update since the slices were gathered: the master is the widened bf16 weight
+            const uint4* src = reinterpret_cast<const uint4*>(p.out0 + grow * p.N + n);
 #pragma unroll
-          for (int q = 0; q < 8; ++q) m[q] = (4 * q < valid) ? src[q] : make_float4(0.f, 0.f, 0.f, 0.f);
+            for (int q = 0; q < 4; ++q) {
+              const uint4 v = (8 * q < valid) ? src[q] : make_uint4(0, 0, 0, 0);
+              m[2 * q] = make_float4(bf_lo(v.x), bf_hi(v.x), bf_lo(v.y), bf_hi(v.y));
+              m[2 * q + 1] = make_float4(bf_lo(v.z), bf_hi(v.z), bf_lo(v.w), bf_hi(v.w));
+            }
+          } else {
+            const float4* src = reinterpret_cast<const float4*>(p.master + grow * p.N + n);
+#pragma unroll
+            for (int q = 0; q < 8; ++q) m[q] = (4 * q < valid) ? src[q] : make_float4(0.f, 0.f, 0.f, 0.f);
+          }
         };
         load_master(0, mv[0]);
         if (!__all_sync(0xffffffffu, mbar_wait(tfull_bar(slot), acc_phase, abort_flag, p.status))) { ok = false; break; }
@@ -468,7 +481,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                 const float4 gq = make_float4(p.scale * __uint_as_float(r[4 * q]), p.scale * __uint_as_float(r[4 * q + 1]),
                                               p.scale * __uint_as_float(r[4 * q + 2]), p.scale * __uint_as_float(r[4 * q + 3]));
                 if (dw) *reinterpret_cast<float4*>(dw + 4 * q) = gq;
-                if (p.lr != 0.f) {      // master -= lr * step (fp32); compute copy = bf16(master)
+                if (do_update) {        // master -= lr * step (fp32); compute copy = bf16(master)
                   float4 m = mv[c & 1][q];
                   if constexpr (EPI == EPI_ADAM) {
                     // m1 <- b1 m1 + (1 - b1) g;  m2 <- b2 m2 + (1 - b2) g^2;  step = (m1 / (1 - b1^t)) / (sqrt(m2 / (1 - b2^t)) + eps)

@@ -186,7 +186,7 @@ extern "C" int32_t twist_subnet_ffn_bwd(const twist_ffn_args* a, void* stream) {
     }
     return TWIST_OK;
   }
-  if (a->lr != 0.f && (!a->w_gu_master || !a->w_down_master)) return TWIST_ERR_NULL;
+  if ((a->lr != 0.f || a->master_from_slice) && (!a->w_gu_master || !a->w_down_master)) return TWIST_ERR_NULL;
   if (a->dx_residual && !a->dx) return TWIST_ERR_NULL;
   // dpre = act'(pre) * (out_scale * dY W_down^T)
   GemmParams p = base_params(T, f, d, S, a->out_scale);
@@ -210,6 +210,7 @@ extern "C" int32_t twist_subnet_ffn_bwd(const twist_ffn_args* a, void* stream) {
   r.master = a->w_down_master;
   r.dw = a->dw_down;
   r.lr = a->lr;
+  r.master_init = a->master_from_slice;
   int epi = optimizer_epilogue(a->opt, a->lr, a->m_down, a->v_down, &r);
   if (epi < 0) return epi;
   TWIST_TRY(launch_gemm_bf16(2, epi, GemmOperand{a->hh, T, f}, GemmOperand{a->dy, T, d}, r, st));
@@ -219,6 +220,7 @@ extern "C" int32_t twist_subnet_ffn_bwd(const twist_ffn_args* a, void* stream) {
   u.master = a->w_gu_master;
   u.dw = a->dw_gu;
   u.lr = a->lr;
+  u.master_init = a->master_from_slice;
   epi = optimizer_epilogue(a->opt, a->lr, a->m_gu, a->v_gu, &u);
   if (epi < 0) return epi;
   return launch_gemm_bf16(2, epi, GemmOperand{a->dpre, T, gf}, GemmOperand{a->x, T, d}, u, st);
@@ -312,7 +314,7 @@ extern "C" int32_t twist_subnet_attn_proj_bwd(const twist_proj_args* a, void* st
     if (a->lr != 0.f) TWIST_TRY(sgd_f32(w, a->dw, a->lr, (long long)S * n * d, st));
     return TWIST_OK;
   }
-  if (a->lr != 0.f && !a->w_master) return TWIST_ERR_NULL;
+  if ((a->lr != 0.f || a->master_from_slice) && !a->w_master) return TWIST_ERR_NULL;
   if (a->d_in_residual && (!qkv || !a->d_in)) return TWIST_ERR_UNSUPPORTED;
   if (a->d_in) {
     if (qkv) {
@@ -333,6 +335,7 @@ extern "C" int32_t twist_subnet_attn_proj_bwd(const twist_proj_args* a, void* st
   r.master = a->w_master;
   r.dw = a->dw;
   r.lr = a->lr;
+  r.master_init = a->master_from_slice;
   const int epi = optimizer_epilogue(a->opt, a->lr, a->m, a->v, &r);
   if (epi < 0) return epi;
   if (qkv) return launch_gemm_bf16(2, epi, GemmOperand{a->d_out, T, w_out}, GemmOperand{a->in, T, w_in}, r, st);

@@ -57,10 +57,13 @@ class RoundEngine:
     BLOCKS = ("ffn", "qkv", "o")
 
     def __init__(self, w: Workload, device: str = "cuda", keep_f32_full: bool = False, compute_dx: bool = True,
-                 dump_grads: bool = False, fuse_loss: bool = True, store_outputs: bool = True):
+                 dump_grads: bool = False, fuse_loss: bool = True, store_outputs: bool = True,
+                 lazy_master: bool = True):
         """fuse_loss: evaluate the loss inside the forward call's output kernel (otherwise with the
         stand-alone twist_mse_fwd_bwd).  store_outputs=False (fused loss, bf16 only) skips storing the
-        block outputs, which nothing reads once the loss gradient exists."""
+        block outputs, which nothing reads once the loss gradient exists.  lazy_master (bf16): the gather
+        writes only the bf16 slices; the fp32 masters come into being in the first weight update of the round,
+        which reads the bf16 slice (exactly the master's value) instead."""
         self.w, self.dev = w, torch.device(device)
         self.compute_dx, self.dump_grads = compute_dx, dump_grads or w.dtype != DTYPE_BF16
         self.fuse_loss = fuse_loss
@@ -104,6 +107,7 @@ class RoundEngine:
             self.kv_pos = torch.empty(L, S, w.n_kv_heads, **i32)
         self.adam = w.optimizer == "adam"
         assert not self.adam or bf16, "the fused Adam update exists for the bf16 dtype"
+        self.lazy_master = lazy_master and bf16 and w.local_steps > 0
         # geometries: partitioned layers, and shared layers (N_sub = N_full) if the workload has any
         self.shared_layers = frozenset(w.shared_layers)
         assert all(0 <= l < L for l in self.shared_layers)
@@ -255,31 +259,40 @@ class RoundEngine:
                                       self.kv_pos[sl])
                     self.launches += 4
 
+    def _gather_master(self, master):
+        """Destination of the gather's fp32 copy: none when the first weight update creates the masters."""
+        return None if self.lazy_master else master
+
+    def _first(self, k: int) -> dict:
+        """Argument of a backward call: the first update after a gather reads the bf16 slice in place of the master."""
+        return dict(master_from_slice=True) if (self.lazy_master and k == 0) else {}
+
     def gather_layer(self, l: int, which=("ffn", "attn")):
         self._use(l)
         w, d = self.w, self.w.d_model
         f, gf, keep = self.f_sub, self.gf, self.ffn_keep
         nb = w.n_ffn_blocks
+        gm = self._gather_master
         segs = []
         if "ffn" in which:
             if self.g == 2:
-                segs.append(B.gather_segment(self.full["gate"][l], self.w_gu, self.w_gu_m, self.gather_idx_ffn[l], None,
+                segs.append(B.gather_segment(self.full["gate"][l], self.w_gu, gm(self.w_gu_m), self.gather_idx_ffn[l], None,
                                              keep, keep, w.ffn_block, 0, gf * d, 0, nb))
-            segs.append(B.gather_segment(self.full["up"][l], self.w_gu, self.w_gu_m, self.gather_idx_ffn[l], None,
+            segs.append(B.gather_segment(self.full["up"][l], self.w_gu, gm(self.w_gu_m), self.gather_idx_ffn[l], None,
                                          keep, keep, w.ffn_block, 0, gf * d, f if self.g == 2 else 0, nb))
-            segs.append(B.gather_segment(self.full["down"][l], self.w_down, self.w_down_m, self.gather_idx_ffn[l], None,
+            segs.append(B.gather_segment(self.full["down"][l], self.w_down, gm(self.w_down_m), self.gather_idx_ffn[l], None,
                                          keep, keep, w.ffn_block, 0, f * d, 0, nb))
         if self.has_attn and "attn" in which:
             H, Hkv, dh, hk = w.n_heads, w.n_kv_heads, w.d_head, self.head_keep
             qkv = self.full["qkv"][l]
-            segs.append(B.gather_segment(qkv, self.w_qkv, self.w_qkv_m, self.idx_head[l], None, hk, hk, dh, 0,
+            segs.append(B.gather_segment(qkv, self.w_qkv, gm(self.w_qkv_m), self.idx_head[l], None, hk, hk, dh, 0,
                                          self.nq * d, 0, H))
-            segs.append(B.gather_segment(qkv, self.w_qkv, self.w_qkv_m, self.kv_idx[l], self.kv_count[l], Hkv,
+            segs.append(B.gather_segment(qkv, self.w_qkv, gm(self.w_qkv_m), self.kv_idx[l], self.kv_count[l], Hkv,
                                          self.kv_max, dh, H * dh, self.nq * d, self.a_sub, Hkv))
-            segs.append(B.gather_segment(qkv, self.w_qkv, self.w_qkv_m, self.kv_idx[l], self.kv_count[l], Hkv,
+            segs.append(B.gather_segment(qkv, self.w_qkv, gm(self.w_qkv_m), self.kv_idx[l], self.kv_count[l], Hkv,
                                          self.kv_max, dh, (H + Hkv) * dh, self.nq * d, self.a_sub + self.kv_max * dh,
                                          Hkv))
-            segs.append(B.gather_segment(self.full["o"][l], self.w_o, self.w_o_m, self.idx_head[l], None, hk, hk, dh, 0,
+            segs.append(B.gather_segment(self.full["o"][l], self.w_o, gm(self.w_o_m), self.idx_head[l], None, hk, hk, dh, 0,
                                          self.a_sub * d, 0, H))
         with self._timed("gather"):
             B.twist_gather_subnets(segs, w.n_subnets, d, w.dtype)
@@ -351,7 +364,7 @@ class RoundEngine:
                        w_down_master=self.w_down_m, pre=self.pre, hh=self.hh,
                        y=self.y if self.store_outputs else None, dy=self.dy, dpre=self.dpre,
                        dx=self.dx, dw_gu=self.dw_gu, dw_down=self.dw_down, hidden_mask=self.h_mask, **fused,
-                       **self._opt(k, ("_gu", "w_gu"), ("_down", "w_down")))
+                       **self._first(k), **self._opt(k, ("_gu", "w_gu"), ("_down", "w_down")))
         with self._timed("ffn_fwd"):
             B.twist_subnet_ffn_fwd(a)
         if self.fuse_loss:
@@ -383,7 +396,8 @@ class RoundEngine:
         fused = dict(tgt=self.Tq[k], loss=self.loss[l, 1, k], loss_ws=self.ws, **mask) if self.fuse_loss else {}
         a = self._proj_args(B.PROJ_QKV, w.dtype, w.n_subnets, w.tokens, w.d_model, self.nq, 1.0, lr, in_=self.X[k],
                         w=self.w_qkv, w_master=self.w_qkv_m, out=self.qkv_out if self.store_outputs else None,
-                        d_out=self.dqkv, d_in=self.dx, dw=self.dw_qkv, **fused, **self._opt(k, ("", "w_qkv")))
+                        d_out=self.dqkv, d_in=self.dx, dw=self.dw_qkv, **fused, **self._first(k),
+                        **self._opt(k, ("", "w_qkv")))
         with self._timed("qkv_fwd"):
             B.twist_subnet_attn_proj_fwd(a)
         if self.fuse_loss:
@@ -402,7 +416,7 @@ class RoundEngine:
         fused = dict(tgt=self.Td[k], loss=self.loss[l, 2, k], loss_ws=self.ws) if self.fuse_loss else {}
         a = self._proj_args(B.PROJ_O, w.dtype, w.n_subnets, w.tokens, w.d_model, self.a_sub, self.alpha_a, lr,
                         in_=self.A[k], w=self.w_o, w_master=self.w_o_m, out=self.y if self.store_outputs else None,
-                        d_out=self.dy, d_in=self.da, dw=self.dw_o, **fused, **self._o_mask(l),
+                        d_out=self.dy, d_in=self.da, dw=self.dw_o, **fused, **self._o_mask(l), **self._first(k),
                         **self._opt(k, ("", "w_o")))
         with self._timed("o_fwd"):
             B.twist_subnet_attn_proj_fwd(a)
@@ -631,18 +645,18 @@ class HybridRoundEngine(RoundEngine):
         segs = []
         for m, off, dst, dst_m, stride in ([("gate", 0, self.w_gu, self.w_gu_m, gf)] if self.g == 2 else []) + [
                 ("up", f if self.g == 2 else 0, self.w_gu, self.w_gu_m, gf), ("down", 0, self.w_down, self.w_down_m, f)]:
-            segs.append(B.gather_segment(self.full[m][l], dst[1:], dst_m[1:], idx, None, w.ffn_keep, w.ffn_keep,
-                                         w.ffn_block, 0, stride * d, off, w.n_ffn_blocks))
+            segs.append(B.gather_segment(self.full[m][l], dst[1:], self._gather_master(dst_m[1:]), idx, None, w.ffn_keep,
+                                         w.ffn_keep, w.ffn_block, 0, stride * d, off, w.n_ffn_blocks))
         if self.has_attn:
             H, Hkv, dh, hk = w.n_heads, w.n_kv_heads, w.d_head, w.head_keep
             qkv, ih, ik, ic = self.full["qkv"][l], self.idx_head[l, 1:], self.kv_idx[l, 1:], self.kv_count[l, 1:]
-            q_dst, q_m = self.w_qkv[1:], self.w_qkv_m[1:]
+            q_dst, q_m = self.w_qkv[1:], self._gather_master(self.w_qkv_m[1:])
             segs.append(B.gather_segment(qkv, q_dst, q_m, ih, None, hk, hk, dh, 0, self.nq * d, 0, H))
             segs.append(B.gather_segment(qkv, q_dst, q_m, ik, ic, Hkv, self.kv_max, dh, H * dh, self.nq * d, self.a_sub, Hkv))
             segs.append(B.gather_segment(qkv, q_dst, q_m, ik, ic, Hkv, self.kv_max, dh, (H + Hkv) * dh, self.nq * d,
                                          self.a_sub + self.kv_max * dh, Hkv))
-            segs.append(B.gather_segment(self.full["o"][l], self.w_o[1:], self.w_o_m[1:], ih, None, hk, hk, dh, 0,
-                                         self.a_sub * d, 0, H))
+            segs.append(B.gather_segment(self.full["o"][l], self.w_o[1:], self._gather_master(self.w_o_m[1:]), ih, None,
+                                         hk, hk, dh, 0, self.a_sub * d, 0, H))
         with self._timed("gather"):
             B.twist_gather_subnets(segs, w.n_subnets - 1, d, w.dtype)
             B.twist_hidden_mask(self.cover_ffn[l], w.n_ffn_blocks, w.ffn_block, 0, 1, self.c_mask)
@@ -677,7 +691,7 @@ class HybridRoundEngine(RoundEngine):
                        w_down=self.w_down[1:], w_gu_master=self.w_gu_m[1:], w_down_master=self.w_down_m[1:],
                        pre=self.pre[1:], hh=self.hh[1:], y=self.y[1:] if self.store_outputs else None, dy=self.dy[1:],
                        dpre=self.dpre[1:], dx=self.dx[1:] if self.dx is not None else None, tgt=self.Td[k][1:],
-                       loss=self.loss[l, 0, k][1:], loss_ws=self.ws, **others_opt)
+                       loss=self.loss[l, 0, k][1:], loss_ws=self.ws, **self._first(k), **others_opt)
         with self._timed("ffn_fwd"):
             B.twist_subnet_ffn_fwd(c)
             B.twist_subnet_ffn_fwd(o)
@@ -699,7 +713,7 @@ class HybridRoundEngine(RoundEngine):
         o = self._proj_args(B.PROJ_QKV, w.dtype, S - 1, T, d, self.nq, 1.0, lr, in_=self.X[k][1:], w=self.w_qkv[1:],
                         w_master=self.w_qkv_m[1:], out=self.qkv_out[1:] if self.store_outputs else None,
                         d_out=self.dqkv[1:], d_in=dx(slice(1, None)), tgt=self.Tq[k][1:], loss=self.loss[l, 1, k][1:],
-                        loss_ws=self.ws, **mask, **self._others_opt(k, ("", "w_qkv")))
+                        loss_ws=self.ws, **mask, **self._first(k), **self._others_opt(k, ("", "w_qkv")))
         with self._timed("qkv_fwd"):
             B.twist_subnet_attn_proj_fwd(c)
             B.twist_subnet_attn_proj_fwd(o)
@@ -720,7 +734,7 @@ class HybridRoundEngine(RoundEngine):
         o = self._proj_args(B.PROJ_O, w.dtype, S - 1, T, d, self.a_sub, self.alpha_a, lr, in_=self.A[k][1:], w=self.w_o[1:],
                         w_master=self.w_o_m[1:], out=self.y[1:] if self.store_outputs else None, d_out=self.dy[1:],
                         d_in=self.da[1:] if self.da is not None else None, tgt=self.Td[k][1:],
-                        loss=self.loss[l, 2, k][1:], loss_ws=self.ws, **self._others_opt(k, ("", "w_o")))
+                        loss=self.loss[l, 2, k][1:], loss_ws=self.ws, **self._first(k), **self._others_opt(k, ("", "w_o")))
         with self._timed("o_fwd"):
             B.twist_subnet_attn_proj_fwd(c)
             B.twist_subnet_attn_proj_fwd(o)
@@ -915,14 +929,15 @@ class StackEngine(RoundEngine):
                                                   pre=self.pre_l[l], hh=self.hh_l[l], dy=g, dpre=self.dpre,
                                                   dx=self.d_ln if self.ln else g_mid,
                                                   dx_residual=None if self.ln else g, dw_gu=self.dw_gu,
-                                                  dw_down=self.dw_down,
+                                                  dw_down=self.dw_down, **self._first(k),
                                                   **self._opt(k, ("_gu", "w_gu"), ("_down", "w_down"))))
             if self.ln:
                 self._ln_bwd(l, "f", k, lr, self.x_mid[l], self.d_ln, g_mid, g)
             with self._timed("o_bwd"):
                 B.twist_subnet_attn_proj_bwd(self._proj_args(B.PROJ_O, w.dtype, S, T, d, self.a_sub, self.alpha_a, lr,
                                                          in_=self.a_l[l], w=self.w_o, w_master=self.w_o_m, d_out=g_mid,
-                                                         d_in=self.da, dw=self.dw_o, **self._opt(k, ("", "w_o"))))
+                                                         d_in=self.da, dw=self.dw_o, **self._first(k),
+                                                         **self._opt(k, ("", "w_o"))))
             with self._timed("core_bwd"):
                 B.twist_attn_core_bwd(self._core_args(l, qkv=self.qkv_l[l], out=self.a_l[l], lse=self.lse[l],
                                                       d_out=self.da, d_qkv=self.dqkv, delta=self.delta))
@@ -935,7 +950,7 @@ class StackEngine(RoundEngine):
                                                          w=self.w_qkv, w_master=self.w_qkv_m, d_out=self.dqkv,
                                                          d_in=self.d_ln if self.ln else g,
                                                          d_in_residual=None if self.ln else g_mid, dw=self.dw_qkv,
-                                                         **self._opt(k, ("", "w_qkv"))))
+                                                         **self._first(k), **self._opt(k, ("", "w_qkv"))))
             if self.ln:
                 self._ln_bwd(l, "a", k, lr, self.x[l], self.d_ln, g, g_mid)
             self.launches += 4 + 2 + 3 + 2

@@ -36,7 +36,7 @@ def setup(request):
     from paper_2511_03983_b200.engine import RoundEngine
     B.lib()
     w = replace(I.PRESETS[request.param], n_layers=1, local_steps=1)
-    eng = RoundEngine(w, keep_f32_full=True)
+    eng = RoundEngine(w, keep_f32_full=True, lazy_master=False)      # the tests below call the C ABI themselves
     gen = torch.Generator(device="cuda")
     gen.manual_seed(w.seed_w)
     for m, v in eng.full.items():
@@ -317,7 +317,7 @@ def cell(request):
     base = I.PRESETS[5]
     w = replace(base, n_subnets=S, ffn_keep=int(np.floor(keep * base.n_ffn_blocks)), n_layers=1, local_steps=1,
                 name=f"cfg5-S{S}-keep{keep}")
-    eng = RoundEngine(w, keep_f32_full=True)
+    eng = RoundEngine(w, keep_f32_full=True, lazy_master=False)      # the tests below call the C ABI themselves
     gen = torch.Generator(device="cuda")
     gen.manual_seed(w.seed_w + S)
     for m, v in eng.full.items():

@@ -1078,3 +1078,33 @@ def test_plan_caches_tensor_maps_and_changes_no_result(B):
     assert c1 > 0 and m1 == c1                                           # cold: every distinct map encoded once
     assert c2 == c1 and m2 == m1 and h2 - h1 == h1 + m1                  # warm: as many lookups, all of them hits
     plan.close()
+
+
+def test_masters_created_by_the_first_update_equal_masters_written_by_the_gather(B):
+    """The gather may leave the fp32 masters unwritten: the first weight update after it reads the bf16 slice, whose
+    exact widening the master is.  Both ways give the same bits everywhere - full model, fp32 result, losses - for
+    SGD and for Adam, with a learning rate and with lr = 0 (where the update only creates the masters)."""
+    from paper_2511_03983_b200.engine import RoundEngine
+    for extra in (dict(), dict(optimizer="adam", lr=1e-3, adam_eps=3e-3), dict(lr=0.0)):
+        w = replace(I.scaled_twin(I.PRESETS[3], d_model=256, d_ff=688, d_head=8, tokens=256, n_layers=2, local_steps=2),
+                    **extra)
+        runs = []
+        for lazy in (True, False):
+            eng = RoundEngine(w, keep_f32_full=True, lazy_master=lazy)
+            assert eng.lazy_master == lazy
+            _load_full(eng, w)
+            for m in eng.full:
+                eng.full_f32[m].copy_(eng.full[m].float())
+            for m in ("w_gu_m", "w_down_m", "w_qkv_m", "w_o_m"):       # whatever was there before must not matter
+                getattr(eng, m).fill_(float("nan"))
+            _load_batches(eng, w, 0)
+            eng.run_round(0)
+            torch.cuda.synchronize()
+            check_status(B)
+            runs.append(({m: v.clone() for m, v in eng.full.items()}, {m: v.clone() for m, v in eng.full_f32.items()},
+                         eng.loss.clone(), eng.w_gu_m.clone()))
+        for a, b in zip(runs[0][:2], runs[1][:2]):
+            for m in a:
+                assert torch.equal(a[m], b[m]), (extra, m)
+        assert torch.equal(runs[0][2], runs[1][2]) and torch.equal(runs[0][3], runs[1][3])
+        assert torch.isfinite(runs[0][3]).all()
