@@ -61,6 +61,7 @@ int32_t twist_device_status(int32_t* code) {
   if (v != 0) {
     int zero = 0;
     TWIST_CUDA_TRY(cudaMemcpyToSymbol(twist::g_device_status, &zero, sizeof(int)));
+    if (v == TWIST_ERR_DEVICE_TIMEOUT) twist::reset_wave_sync();      // a kernel that gave up left its wave count short
   }
   *code = v;
   return TWIST_OK;

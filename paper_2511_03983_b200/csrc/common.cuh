@@ -15,6 +15,8 @@ namespace twist {
 int* device_status_ptr();
 
 void note_cuda_error(cudaError_t e, const char* where);
+// Resets the grouped GEMM's wave-synchronisation counters of the current device (device idle); gemm_sm100.cu.
+void reset_wave_sync();
 int sm_count();
 // Index of the current device for per-device caches (kernel attributes are per device), 0 when it cannot be read
 // or exceeds the cache size.

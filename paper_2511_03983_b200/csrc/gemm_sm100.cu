@@ -3,6 +3,8 @@
 
 #include <cudaTypedefs.h>
 
+#include <mutex>
+
 #include "plan.cuh"
 
 namespace twist {
@@ -128,8 +130,60 @@ int make_epilogue_maps(int epi, const GemmParams& p, const CUtensorMap& filler, 
   return rc;
 }
 
+// Wave synchronisation, host side.  One never-reset device counter per stream (up to kWaveSlots streams per device;
+// further streams run unsynchronised); the host keeps the value each counter will have when the launches issued so
+// far on its stream have finished.  Launches on one stream are ordered, so they can share a counter.
+constexpr int kWaveSlots = 64;
+constexpr int kWaveMinKBlocks = 32;     // contractions shorter than this (K < 2048) lose more to the wait than they save
+__device__ unsigned g_wave_ctr[kWaveSlots];
+struct WaveState {
+  std::mutex mu;
+  unsigned* dev = nullptr;              // device address of g_wave_ctr on this device
+  cudaStream_t owner[kWaveSlots];
+  unsigned base[kWaveSlots];
+  int used = 0;
+};
+WaveState g_wave[64];
+
+// Picks the counter of stream `st` and reserves n_waves * grid arrivals on it.  Returns false when the launch
+// should run without wave synchronisation.
+bool wave_reserve(cudaStream_t st, int n_waves, int grid, GemmParams* p) {
+  cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+  if (cudaStreamIsCapturing(st, &cap) != cudaSuccess || cap != cudaStreamCaptureStatusNone) {
+    cudaGetLastError();
+    return false;                       // the sequence numbers live on the host: not replayable from a graph
+  }
+  WaveState& w = g_wave[device_slot()];
+  std::lock_guard<std::mutex> lock(w.mu);
+  if (!w.dev) {
+    void* ptr = nullptr;
+    if (cudaGetSymbolAddress(&ptr, g_wave_ctr) != cudaSuccess || !ptr) { cudaGetLastError(); return false; }
+    w.dev = static_cast<unsigned*>(ptr);
+  }
+  int slot = -1;
+  for (int i = 0; i < w.used; ++i)
+    if (w.owner[i] == st) { slot = i; break; }
+  if (slot < 0) {
+    if (w.used == kWaveSlots) return false;
+    slot = w.used++;
+    w.owner[slot] = st;
+    w.base[slot] = 0;
+  }
+  p->wave_ctr = w.dev + slot;
+  p->wave_base = w.base[slot];
+  p->n_waves = n_waves;
+  w.base[slot] += (unsigned)n_waves * (unsigned)grid;       // wraps like the device counter
+  return true;
+}
+// Takes a reservation back (the launch did not happen).
+void wave_unreserve(const GemmParams& p, int grid) {
+  WaveState& w = g_wave[device_slot()];
+  std::lock_guard<std::mutex> lock(w.mu);
+  w.base[p.wave_ctr - w.dev] -= (unsigned)p.n_waves * (unsigned)grid;
+}
+
 template <int AM, int BM_, int EPI>
-int launch(const CUtensorMap& ta, const CUtensorMap& tb, const GemmParams& p, cudaStream_t st) {
+int launch(const CUtensorMap& ta, const CUtensorMap& tb, GemmParams p, cudaStream_t st) {
   int pairs = 0;
   int rc = resident_pairs<AM, BM_, EPI>(&pairs);
   if (rc != TWIST_OK) return rc;
@@ -138,7 +192,28 @@ int launch(const CUtensorMap& ta, const CUtensorMap& tb, const GemmParams& p, cu
   EpiMaps te;
   rc = make_epilogue_maps(EPI, p, ta, &te);
   if (rc != TWIST_OK) return rc;
-  gemm_kernel<AM, BM_, EPI><<<grid, kGemmThreads, gemm_smem_bytes(EPI != EPI_SGD && EPI != EPI_ADAM), st>>>(ta, tb, te, p);
+  const int smem = gemm_smem_bytes(EPI != EPI_SGD && EPI != EPI_ADAM);
+  const int n_waves = (tiles + grid / 2 - 1) / (grid / 2);
+  p.wave_ctr = nullptr;
+  if (n_waves >= 2 && (p.K + kBK - 1) / kBK >= kWaveMinKBlocks && wave_reserve(st, n_waves, grid, &p)) {
+    // cooperative: the grid starts only when all of its CTAs can be resident, so the waits cannot starve
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(kGemmThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeCooperative;
+    attr.val.cooperative = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, gemm_kernel<AM, BM_, EPI>, ta, tb, te, p) == cudaSuccess) return TWIST_OK;
+    cudaGetLastError();                 // not launchable that way here: run it unsynchronised
+    wave_unreserve(p, grid);
+    p.wave_ctr = nullptr;
+  }
+  gemm_kernel<AM, BM_, EPI><<<grid, kGemmThreads, smem, st>>>(ta, tb, te, p);
   TWIST_LAUNCH_CHECK();
   return TWIST_OK;
 }
@@ -191,6 +266,16 @@ selftest_wait_kernel(unsigned long long limit_ns, int* status) {
 }
 
 }  // namespace
+
+// After a kernel gave up (a bounded wait ran out) its wave counter is short of what the host booked: start over.
+// Called with the device idle.
+void reset_wave_sync() {
+  WaveState& w = g_wave[device_slot()];
+  std::lock_guard<std::mutex> lock(w.mu);
+  static const unsigned zeros[kWaveSlots] = {0};
+  if (cudaMemcpyToSymbol(g_wave_ctr, zeros, sizeof(zeros)) != cudaSuccess) cudaGetLastError();
+  for (int i = 0; i < kWaveSlots; ++i) w.base[i] = 0;
+}
 
 int encode_map_3d_bf16(CUtensorMap* map, const void* ptr, const unsigned long long dims[3],
                        const unsigned long long strides[2], const unsigned box[3], int swizzle_bytes) {

@@ -83,6 +83,13 @@ struct GemmParams {
   const int32_t* valid_cols;   // MSE: valid columns per column group and subnet [groups], or null (all valid)
   int seg_begin, seg_width;    // MSE: columns [0, seg_begin) valid, then groups of seg_width columns (see twist_mse_fwd_bwd)
   int* status;          // device status word
+  // Wave synchronisation (null: off).  Every CTA of the grid adds one to *wave_ctr per wave (= per tile of its own,
+  // plus once for a last wave it has no tile in); wave w may start once the counter has (nearly) reached
+  // wave_base + (w + 1) * gridDim.x.  The counter is never reset: the host advances wave_base by n_waves * grid
+  // per launch.  Launched cooperatively, so that all CTAs are resident while they wait for one another.
+  unsigned* wave_ctr;
+  unsigned wave_base;
+  int n_waves;
 };
 
 // Tensor maps of the epilogue's boxes (box = 32 columns x 32 rows of a dense bf16 [groups][M][cols] tensor):
@@ -159,6 +166,26 @@ __device__ inline void pair_teardown(volatile int* abort_flag, bool alloc_warp, 
     asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(cols) : "memory");
   }
 }
+// All CTAs of the launch start their next tile together.  Why: the CTA pairs of a wave stream the same operand rows
+// and columns along the contraction and share them through L2 only while they stay within an L2's worth of one
+// another; left alone they drift apart over a long contraction, the same tiles are then fetched from DRAM several
+// times, and the extra DRAM traffic costs power - hence clock - under the board's power cap.  Bounded like every wait.
+__device__ inline bool wave_barrier(unsigned* ctr, unsigned target, volatile int* abort_flag, int* status) {
+  atomicAdd(ctr, 1u);
+  const uint64_t t0 = global_timer_ns();
+  for (uint32_t it = 1;; ++it) {
+    unsigned v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(ctr) : "memory");
+    if ((int)(v - target) >= 0) return true;
+    if ((it & 63u) == 0 && (*abort_flag || global_timer_ns() - t0 > kWaitLimitNs)) {
+      *abort_flag = 1;
+      note_status(status, (int)TWIST_ERR_DEVICE_TIMEOUT);
+      return false;
+    }
+    __nanosleep(200);
+  }
+}
+
 // Tiled copy into this CTA's shared memory; completion bytes are counted on `bar`, which may be a
 // barrier of the other CTA of the pair (cluster-window address).
 __device__ inline void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2) {
@@ -346,9 +373,17 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     if (lane == 0) {
       uint32_t it = 0;
       bool ok = true;
-      for (int tile = pair; ok && tile < total_tiles; tile += num_pairs) {
+      unsigned wave = 0;
+      for (int tile = pair; ok && tile < total_tiles; tile += num_pairs, ++wave) {
         int g, mt, nt;
         tile_coords(p, tile, g, mt, nt);
+        // (the last eighth of the CTAs is not waited for: rough lockstep is all the L2 needs, and the stragglers'
+        // share of a wave would otherwise be idle time for everyone)
+        if (p.wave_ctr && !wave_barrier(p.wave_ctr, p.wave_base + (wave + 1u) * gridDim.x - (gridDim.x >> 3), abort_flag,
+                                        p.status)) {
+          ok = false;
+          break;
+        }
         const int m0 = mt * kBM + (int)rank * kCtaM;
         // B rows (K-major) / columns (MN-major) of this CTA.  SwiGLU forward: the leader loads 128 gate
         // rows, the peer the matching 128 up rows, so accumulator columns 0..127 are G and 128..255 are U.
@@ -376,6 +411,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           }
         }
       }
+      // a wave this CTA has no tile in (the last, partial one) still gets its arrival: the count per wave is uniform
+      if (p.wave_ctr && ok)
+        for (; (int)wave < p.n_waves; ++wave) atomicAdd(p.wave_ctr, 1u);
     }
   } else if (warp == kEpiWarps + 1) {
     // ------------------------------------------------------------------ MMA issuer (leader CTA only)
