@@ -30,18 +30,18 @@ EncodeTiledFn encode_fn() {
 // Encodes a 3-D tiled bf16 tensor map, or takes it from the calling thread's active plan (plan.cuh).
 int encode_or_cached(CUtensorMap* map, const void* ptr, const cuuint64_t dims[3], const cuuint64_t strides[2],
                      const cuuint32_t box[3], CUtensorMapSwizzle swizzle, CUtensorMapL2promotion promotion,
-                     const char* what) {
+                     const char* what, CUtensorMapDataType dtype = CU_TENSOR_MAP_DATA_TYPE_BFLOAT16) {
   MapKey key;
   memset(&key, 0, sizeof(key));
   key.ptr = ptr;
   for (int i = 0; i < 3; ++i) { key.dims[i] = dims[i]; key.box[i] = box[i]; }
   key.strides[0] = strides[0]; key.strides[1] = strides[1];
-  key.swizzle = (unsigned)swizzle; key.promotion = (unsigned)promotion;
+  key.swizzle = (unsigned)swizzle; key.promotion = (unsigned)promotion | ((unsigned)dtype << 16);
   if (plan_lookup(key, map)) return TWIST_OK;
   EncodeTiledFn fn = encode_fn();
   if (!fn) { note_cuda_error(cudaErrorUnknown, "cuTensorMapEncodeTiled entry point"); return TWIST_ERR_CUDA; }
   cuuint32_t estr[3] = {1, 1, 1};
-  CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, estr,
+  CUresult r = fn(map, dtype, 3, const_cast<void*>(ptr), dims, strides, box, estr,
                   CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle, promotion, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) {
     note_cuda_error(cudaErrorInvalidValue, what);
@@ -71,12 +71,12 @@ int resident_pairs(int* out) {
   if (dev < 0 || dev >= 64) return TWIST_ERR_UNSUPPORTED;
   if (cached[dev] == 0) {
     TWIST_CUDA_TRY(cudaFuncSetAttribute(gemm_kernel<AM, BM_, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                        gemm_smem_bytes(EPI != EPI_SGD && EPI != EPI_ADAM)));
+                                        gemm_smem_bytes(EPI)));
     cudaLaunchConfig_t cfg;
     memset(&cfg, 0, sizeof(cfg));
     cfg.gridDim = dim3(2 * (sm_count() / 2));
     cfg.blockDim = dim3(kGemmThreads);
-    cfg.dynamicSmemBytes = gemm_smem_bytes(EPI != EPI_SGD && EPI != EPI_ADAM);
+    cfg.dynamicSmemBytes = gemm_smem_bytes(EPI);
     cudaLaunchAttribute attr;
     attr.id = cudaLaunchAttributeClusterDimension;
     attr.val.clusterDim.x = 2; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
@@ -105,6 +105,16 @@ int make_box_map(CUtensorMap* map, const void* ptr, int rows, int cols, long lon
                           "cuTensorMapEncodeTiled (epilogue box)");
 }
 
+// The same box geometry (64-byte rows, 32 rows, 64-byte swizzle) over an fp32 tensor [groups][rows][cols]: 16 columns.
+int make_box_map_f32(CUtensorMap* map, const void* ptr, int rows, int cols, int groups) {
+  if (!ptr || !aligned16(ptr) || cols % 4 != 0) return TWIST_ERR_SHAPE;
+  cuuint64_t dims[3] = {(cuuint64_t)cols, (cuuint64_t)rows, (cuuint64_t)groups};
+  cuuint64_t strides[2] = {(cuuint64_t)cols * 4, (cuuint64_t)rows * (cuuint64_t)cols * 4};
+  cuuint32_t box[3] = {16, 32, 1};
+  return encode_or_cached(map, ptr, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                          "cuTensorMapEncodeTiled (fp32 epilogue box)", CU_TENSOR_MAP_DATA_TYPE_FLOAT32);
+}
+
 // Tensor maps of the boxes each epilogue reads and writes (layout of EpiMaps in the kernel header).
 int make_epilogue_maps(int epi, const GemmParams& p, const CUtensorMap& filler, EpiMaps* e) {
   for (int i = 0; i < 4; ++i) e->m[i] = filler;          // unused entries stay valid descriptors
@@ -125,7 +135,13 @@ int make_epilogue_maps(int epi, const GemmParams& p, const CUtensorMap& filler, 
       break;
     case EPI_DACT:
     case EPI_RESID: mk(0, p.in0, N, N); mk(1, p.out0, N, N); break;
-    default: break;                                        // EPI_SGD: plain global accesses
+    case EPI_SGD:                                          // staged only when the launch updates the weights
+      if (p.lr != 0.f || p.master_init) {
+        if (rc == TWIST_OK) rc = make_box_map_f32(&e->m[0], p.master, M, N, G);
+        mk(2, p.out0, N, N);
+      }
+      break;
+    default: break;                                        // EPI_ADAM: plain global accesses
   }
   return rc;
 }
@@ -133,6 +149,7 @@ int make_epilogue_maps(int epi, const GemmParams& p, const CUtensorMap& filler, 
 // Wave synchronisation, host side.  One never-reset device counter per stream (up to kWaveSlots streams per device;
 // further streams run unsynchronised); the host keeps the value each counter will have when the launches issued so
 // far on its stream have finished.  Launches on one stream are ordered, so they can share a counter.
+constexpr int kSgdLongK = 16384;        // contraction length from which the fused SGD update runs from registers
 constexpr int kWaveSlots = 64;
 constexpr int kWaveMinKBlocks = 32;     // contractions shorter than this (K < 2048) lose more to the wait than they save
 __device__ unsigned g_wave_ctr[kWaveSlots];
@@ -192,7 +209,7 @@ int launch(const CUtensorMap& ta, const CUtensorMap& tb, GemmParams p, cudaStrea
   EpiMaps te;
   rc = make_epilogue_maps(EPI, p, ta, &te);
   if (rc != TWIST_OK) return rc;
-  const int smem = gemm_smem_bytes(EPI != EPI_SGD && EPI != EPI_ADAM);
+  const int smem = gemm_smem_bytes(EPI);
   const int n_waves = (tiles + grid / 2 - 1) / (grid / 2);
   p.wave_ctr = nullptr;
   if (n_waves >= 2 && (p.K + kBK - 1) / kBK >= kWaveMinKBlocks && wave_reserve(st, n_waves, grid, &p)) {
@@ -334,7 +351,11 @@ int launch_gemm_bf16(int layout, int epi, const GemmOperand& A, const GemmOperan
   if (layout == 1 && epi == EPI_MSE) return launch<MAJOR_K, MAJOR_MN, EPI_MSE>(ta, tb, p, st);
   if (layout == 1 && epi == EPI_MSE_NOY) return launch<MAJOR_K, MAJOR_MN, EPI_MSE_NOY>(ta, tb, p, st);
   if (layout == 1 && epi == EPI_RESID) return launch<MAJOR_K, MAJOR_MN, EPI_RESID>(ta, tb, p, st);
-  if (layout == 2 && epi == EPI_SGD) return launch<MAJOR_MN, MAJOR_MN, EPI_SGD>(ta, tb, p, st);
+  if (layout == 2 && epi == EPI_SGD) {
+    // staged update, except at the longest contractions (see gemm_stages)
+    if (p.K >= kSgdLongK) return launch<MAJOR_MN, MAJOR_MN, EPI_SGD_LONG>(ta, tb, p, st);
+    return launch<MAJOR_MN, MAJOR_MN, EPI_SGD>(ta, tb, p, st);
+  }
   if (layout == 2 && epi == EPI_ADAM) return launch<MAJOR_MN, MAJOR_MN, EPI_ADAM>(ta, tb, p, st);
   return TWIST_ERR_UNSUPPORTED;
 }

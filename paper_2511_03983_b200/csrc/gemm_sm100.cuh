@@ -36,7 +36,8 @@ namespace twist {
 enum { MAJOR_K = 0, MAJOR_MN = 1 };
 enum { EPI_STORE = 0, EPI_SWIGLU_FWD = 1, EPI_ACT_FWD = 2, EPI_DSWIGLU = 3, EPI_DACT = 4, EPI_SGD = 5, EPI_MSE = 6, EPI_RESID = 7,
        EPI_MSE_NOY = 8 /* EPI_MSE without storing D: one box per chunk, so twice as many chunk buffers */,
-       EPI_ADAM = 9 /* weight gradient with the Adam update fused, like EPI_SGD */ };
+       EPI_ADAM = 9 /* weight gradient with the Adam update fused, like EPI_SGD */,
+       EPI_SGD_LONG = 10 /* EPI_SGD for very long contractions: update from registers, full operand ring */ };
 
 constexpr int kBM = 256, kBN = 256, kBK = 64, kUmmaK = 16;   // tile of a CTA pair
 constexpr int kCtaM = kBM / 2, kCtaN = kBN / 2;   // rows of A / columns of B that one CTA of the pair loads
@@ -49,14 +50,20 @@ constexpr int kGemmThreads = (kEpiWarps + 2) * 32;
 // 64-byte swizzle) travel between global memory and the warp by TMA: operands the epilogue reads arrive as boxes,
 // results leave as boxes, so every global access of the epilogue is a full-line bulk transfer.
 constexpr int kEpiBoxBytes = 32 * 32 * 2;
-constexpr int kEpiWarpBytes = 8192;
-constexpr int kEpiBytes = kEpiWarps * kEpiWarpBytes;
 constexpr int kCtrlBytes = 512;
-// Operand ring: 5 stages of 32 KB beside the epilogue staging.  The weight-gradient kernel stages nothing and
-// could hold 7, but measured no faster with them (it is bound by power, not by latency), so it keeps 5 too.
-__host__ __device__ constexpr int gemm_stages(bool /*staged_epilogue*/) { return 5; }
-__host__ __device__ constexpr int gemm_smem_bytes(bool staged_epilogue) {
-  return gemm_stages(staged_epilogue) * kStageBytes + (staged_epilogue ? kEpiBytes : 0) + 1024 /*alignment slack*/ + kCtrlBytes;
+// Shared memory per epilogue (EPI_* values are defined above): the staged epilogues own 8 KB per warp; the fused SGD
+// update, whose chunk is two fp32 master boxes and one bf16 weight box, 12 KB (two chunks in flight) and pays
+// for them with one stage of the operand ring (4 instead of 5: the weight-gradient contraction is the longest of
+// all, while at short contractions its time is the masters' read-modify-write, which staging makes asynchronous:
+// +19 % on the 1024-token workload).  At the longest contractions (32768 tokens) the shorter ring cost the 7B round
+// 2.5 % of its weight-gradient time, so those launches use EPI_SGD_LONG: the update straight from registers, five
+// stages.  The Adam update also works from registers and stages nothing.
+__host__ __device__ constexpr bool epi_staged(int epi) { return epi != 9 /*EPI_ADAM*/ && epi != 10 /*EPI_SGD_LONG*/; }
+__host__ __device__ constexpr int epi_warp_bytes(int epi) { return epi == 5 /*EPI_SGD*/ ? 12288 : 8192; }
+__host__ __device__ constexpr int gemm_stages(int epi) { return epi == 5 /*EPI_SGD*/ ? 4 : 5; }
+__host__ __device__ constexpr int gemm_epi_region(int epi) { return epi_staged(epi) ? kEpiWarps * epi_warp_bytes(epi) : 0; }
+__host__ __device__ constexpr int gemm_smem_bytes(int epi) {
+  return gemm_stages(epi) * kStageBytes + gemm_epi_region(epi) + 1024 /*alignment slack*/ + kCtrlBytes;
 }
 constexpr int kTmemCols = 512;                    // two 128 x 256 fp32 accumulators per CTA
 
@@ -97,16 +104,22 @@ struct GemmParams {
 //   SWIGLU_FWD: 0 G, 1 U (the two halves of pre), 2 hh.        ACT_FWD: 0 pre, 1 hh.
 //   DSWIGLU: 0 G, 1 U (in), 2 dG, 3 dU (out).                  DACT: 0 pre (in), 1 dpre (out).
 //   RESID: 0 addend (in), 1 D (out).
+//   SGD: 0 fp32 masters [groups][M][N] (box = 16 columns x 32 rows, the same 64-byte rows; in and out),
+//        2 bf16 weights (out; in instead of the masters when they are created from the weights).
 struct EpiMaps { CUtensorMap m[4]; };
 
 // Boxes per chunk buffer, how many of them are read from global memory first, and buffers per warp.
 __host__ __device__ constexpr int epi_slots(int epi) {
-  return epi == EPI_SWIGLU_FWD ? 3 : (epi == EPI_MSE || epi == EPI_ACT_FWD || epi == EPI_DSWIGLU) ? 2 : 1;
+  return (epi == EPI_SWIGLU_FWD || epi == EPI_SGD) ? 3 : (epi == EPI_MSE || epi == EPI_ACT_FWD || epi == EPI_DSWIGLU) ? 2 : 1;
 }
 __host__ __device__ constexpr int epi_in_slots(int epi) {
-  return epi == EPI_DSWIGLU ? 2 : (epi == EPI_MSE || epi == EPI_MSE_NOY || epi == EPI_DACT || epi == EPI_RESID) ? 1 : 0;
+  return (epi == EPI_DSWIGLU || epi == EPI_SGD) ? 2
+         : (epi == EPI_MSE || epi == EPI_MSE_NOY || epi == EPI_DACT || epi == EPI_RESID) ? 1 : 0;
 }
-__host__ __device__ constexpr int epi_bufs(int epi) { return epi_slots(epi) == 3 ? 1 : epi_slots(epi) == 2 ? 2 : 4; }
+// chunk buffers per warp: what fits, rounded down to a power of two (4, 2 or 1)
+__host__ __device__ constexpr int epi_bufs(int epi) {
+  return epi_warp_bytes(epi) / (epi_slots(epi) * kEpiBoxBytes) >= 4 ? 4 : epi_warp_bytes(epi) / (epi_slots(epi) * kEpiBoxBytes) >= 2 ? 2 : 1;
+}
 
 // Registers of one 32-column chunk of accumulator words.
 template <int EPI> struct EpiAcc { uint32_t r0[32]; };
@@ -324,14 +337,14 @@ template <int A_MAJOR, int B_MAJOR, int EPI>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
             const __grid_constant__ EpiMaps tmE, const GemmParams p) {
-  constexpr bool kStaged = EPI != EPI_SGD && EPI != EPI_ADAM;
-  constexpr int kStages = gemm_stages(kStaged);
+  constexpr bool kStaged = epi_staged(EPI);
+  constexpr int kStages = gemm_stages(EPI);
   extern __shared__ unsigned char smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   unsigned char* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
   const uint32_t epi_base = smem_base + kStages * kStageBytes;
-  const uint32_t bar_base = epi_base + (kStaged ? kEpiBytes : 0);
-  volatile uint32_t* ctrl = reinterpret_cast<volatile uint32_t*>(smem_gen + kStages * kStageBytes + (kStaged ? kEpiBytes : 0));
+  const uint32_t bar_base = epi_base + gemm_epi_region(EPI);
+  volatile uint32_t* ctrl = reinterpret_cast<volatile uint32_t*>(smem_gen + kStages * kStageBytes + gemm_epi_region(EPI));
   // control block: 8-byte barriers full[kStages], empty[kStages], tmem_full[2], tmem_empty[2]; then the TMEM base
   // address and the abort flag (4 bytes each, within the first 160 bytes for at most 7 stages); at byte 192 the
   // 32 "box arrived" barriers of the epilogue warps (8 per warp).  Same offsets in both CTAs of the pair.
@@ -463,9 +476,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     uint32_t tl = 0;
     bool ok = true;
 
-    if constexpr (EPI == EPI_SGD || EPI == EPI_ADAM) {
-      // Weight-gradient tiles (contraction over all tokens, so this epilogue is rare): plain vector accesses
-      // to the fp32 master rows; the master values of the next chunk are loaded ahead.
+    if constexpr (EPI == EPI_ADAM || EPI == EPI_SGD_LONG) {
+      // Weight-gradient tiles updated from registers - the Adam step (three fp32 streams per weight: too many for
+      // the staging buffers) and SGD at very long contractions, where this epilogue is rare: plain vector accesses
+      // to the fp32 rows; the master values of the next chunk are loaded ahead.
       for (int tile = pair; ok && tile < total_tiles; tile += num_pairs, ++tl) {
         int g, mt, nt;
         tile_coords(p, tile, g, mt, nt);
@@ -560,7 +574,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       // Inputs are requested kAhead chunks ahead into the buffer that chunk gc + kAhead - kBufs used; only that
       // chunk's store has to be finished, so up to kBufs - kAhead younger stores may still be reading.
       constexpr int kAhead = kBufs > 1 ? kBufs / 2 : 1;
-      const uint32_t wbase = epi_base + (uint32_t)warp * kEpiWarpBytes;
+      const uint32_t wbase = epi_base + (uint32_t)warp * epi_warp_bytes(EPI);
       auto box = [&](uint32_t gc, int slot) { return wbase + ((gc & (kBufs - 1)) * kSlots + slot) * kEpiBoxBytes; };
       // 16-byte piece q (0..3) of this thread's row inside a box (64-byte rows, 64-byte swizzle)
       const uint32_t row_off = (uint32_t)lane * 64u;
@@ -583,13 +597,27 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         return t;
       };
       TileAt cur = locate(pair), nxt = locate(pair + num_pairs);
+      // EPI_SGD: whether this launch updates the weights at all (otherwise it only dumps gradients and stages nothing)
+      const bool sgd_update = EPI == EPI_SGD && (p.lr != 0.f || p.master_init != 0);
       auto request_inputs = [&](uint32_t gc) {      // lane 0 only; gc / kChunks is tl or tl + 1
         if (kIn == 0) return;
         const TileAt& t = (gc / kChunks == tl) ? cur : nxt;
         if (!t.valid) return;
         const uint32_t bar = in_bar(warp, gc & (kBufs - 1));
-        mbar_expect_tx(bar, kIn * kEpiBoxBytes);
         const int n = t.n0 + 32 * (int)(gc % kChunks);
+        if constexpr (EPI == EPI_SGD) {
+          if (!sgd_update) return;
+          if (p.master_init) {      // the masters do not exist yet: the bf16 weights, whose widening they are
+            mbar_expect_tx(bar, kEpiBoxBytes);
+            tma_load_3d_local(box(gc, 2), &tmE.m[2], bar, n, t.row0, t.g);
+          } else {                  // two boxes of 16 fp32 columns
+            mbar_expect_tx(bar, 2 * kEpiBoxBytes);
+            tma_load_3d_local(box(gc, 0), &tmE.m[0], bar, n, t.row0, t.g);
+            tma_load_3d_local(box(gc, 1), &tmE.m[0], bar, n + 16, t.row0, t.g);
+          }
+          return;
+        }
+        mbar_expect_tx(bar, kIn * kEpiBoxBytes);
 #pragma unroll
         for (int i = 0; i < kIn; ++i) tma_load_3d_local(box(gc, i), &tmE.m[i], bar, n, t.row0, t.g);
       };
@@ -624,9 +652,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         for (int c = 0; c < kChunks; ++c) {
           const uint32_t gc = tl * kChunks + c;
           const int n = n_base + 32 * c;
-          if (kIn > 0) {      // this chunk's boxes have arrived
+          if (kIn > 0 && (EPI != EPI_SGD || sgd_update)) {      // this chunk's boxes have arrived
             if (!__all_sync(0xffffffffu, mbar_wait(in_bar(warp, gc & (kBufs - 1)), (gc / kBufs) & 1u, abort_flag, p.status))) { ok = false; break; }
-          } else {            // the bulk store that last read this buffer is done with it
+          } else if (EPI != EPI_SGD) {      // the bulk store that last read this buffer is done with it
             if (lane == 0) bulk_wait_read<kBufs - 1>();
             __syncwarp();
           }
@@ -724,6 +752,35 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
               }
               sts128(piece(b0, q), make_uint4(wg[0], wg[1], wg[2], wg[3]));
               sts128(piece(b1, q), make_uint4(wu[0], wu[1], wu[2], wu[3]));
+            } else if constexpr (EPI == EPI_SGD) {
+              // columns 8 q .. 8 q + 7 of the chunk: two 16-byte pieces of a master box, one piece of the weight box
+              float gv[8];
+#pragma unroll
+              for (int e = 0; e < 8; ++e) gv[e] = p.scale * __uint_as_float(r[e]);
+              if (p.dw && row_ok && n + 8 * q < p.N) {      // optional gradient dump (tests, the fp32 parity checks)
+                float* dwp = p.dw + ((long long)g * p.M + row0 + lane) * p.N + n + 8 * q;
+                *reinterpret_cast<float4*>(dwp) = make_float4(gv[0], gv[1], gv[2], gv[3]);
+                *reinterpret_cast<float4*>(dwp + 4) = make_float4(gv[4], gv[5], gv[6], gv[7]);
+              }
+              if (sgd_update) {
+                const uint32_t mb = (q < 2) ? b0 : b1;          // master box holding these columns
+                const int pq = 2 * (q & 1);                      // its first 16-byte piece
+                float m[8];
+                if (p.master_init) {
+                  const uint4 wv = lds128(piece(b2, q));
+                  m[0] = bf_lo(wv.x); m[1] = bf_hi(wv.x); m[2] = bf_lo(wv.y); m[3] = bf_hi(wv.y);
+                  m[4] = bf_lo(wv.z); m[5] = bf_hi(wv.z); m[6] = bf_lo(wv.w); m[7] = bf_hi(wv.w);
+                } else {
+                  const uint4 lo = lds128(piece(mb, pq)), hi = lds128(piece(mb, pq + 1));
+                  m[0] = __uint_as_float(lo.x); m[1] = __uint_as_float(lo.y); m[2] = __uint_as_float(lo.z); m[3] = __uint_as_float(lo.w);
+                  m[4] = __uint_as_float(hi.x); m[5] = __uint_as_float(hi.y); m[6] = __uint_as_float(hi.z); m[7] = __uint_as_float(hi.w);
+                }
+#pragma unroll
+                for (int e = 0; e < 8; ++e) m[e] -= p.lr * gv[e];       // master -= lr * g (fp32)
+                sts128(piece(mb, pq), make_uint4(__float_as_uint(m[0]), __float_as_uint(m[1]), __float_as_uint(m[2]), __float_as_uint(m[3])));
+                sts128(piece(mb, pq + 1), make_uint4(__float_as_uint(m[4]), __float_as_uint(m[5]), __float_as_uint(m[6]), __float_as_uint(m[7])));
+                sts128(piece(b2, q), make_uint4(pack2(m[0], m[1]), pack2(m[2], m[3]), pack2(m[4], m[5]), pack2(m[6], m[7])));   // compute copy
+              }
             } else if constexpr (EPI == EPI_RESID) {   // D = addend + scale * acc, rounded once
               const uint4 av = lds128(piece(b0, q));
               const uint32_t aw[4] = {av.x, av.y, av.z, av.w};
@@ -769,6 +826,12 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             } else if constexpr (EPI == EPI_DSWIGLU) {
               tma_store_3d(&tmE.m[2], b0, n, rr, gg);
               tma_store_3d(&tmE.m[3], b1, n, rr, gg);
+            } else if constexpr (EPI == EPI_SGD) {
+              if (sgd_update) {
+                tma_store_3d(&tmE.m[0], b0, n, rr, gg);
+                tma_store_3d(&tmE.m[0], b1, n + 16, rr, gg);
+                tma_store_3d(&tmE.m[2], b2, n, rr, gg);
+              }
             } else {   // DACT, RESID
               tma_store_3d(&tmE.m[1], b0, n, rr, gg);
             }
