@@ -135,7 +135,8 @@ int make_epilogue_maps(int epi, const GemmParams& p, const CUtensorMap& filler, 
       break;
     case EPI_DACT:
     case EPI_RESID: mk(0, p.in0, N, N); mk(1, p.out0, N, N); break;
-    case EPI_SGD:                                          // staged only when the launch updates the weights
+    case EPI_SGD:
+    case EPI_SGD_LONG:                                     // staged only when the launch updates the weights
       if (p.lr != 0.f || p.master_init) {
         if (rc == TWIST_OK) rc = make_box_map_f32(&e->m[0], p.master, M, N, G);
         mk(2, p.out0, N, N);

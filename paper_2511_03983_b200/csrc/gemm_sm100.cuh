@@ -56,10 +56,11 @@ constexpr int kCtrlBytes = 512;
 // for them with one stage of the operand ring (4 instead of 5: the weight-gradient contraction is the longest of
 // all, while at short contractions its time is the masters' read-modify-write, which staging makes asynchronous:
 // +19 % on the 1024-token workload).  At the longest contractions (32768 tokens) the shorter ring cost the 7B round
-// 2.5 % of its weight-gradient time, so those launches use EPI_SGD_LONG: the update straight from registers, five
-// stages.  The Adam update also works from registers and stages nothing.
-__host__ __device__ constexpr bool epi_staged(int epi) { return epi != 9 /*EPI_ADAM*/ && epi != 10 /*EPI_SGD_LONG*/; }
-__host__ __device__ constexpr int epi_warp_bytes(int epi) { return epi == 5 /*EPI_SGD*/ ? 12288 : 8192; }
+// 2.5 % of its weight-gradient time, so those launches use EPI_SGD_LONG: the same staged update with one chunk
+// buffer per warp (6 KB; the epilogue is rare there and need not overlap its own loads) and all five stages.
+// The Adam update works from registers and stages nothing.
+__host__ __device__ constexpr bool epi_staged(int epi) { return epi != 9 /*EPI_ADAM*/; }
+__host__ __device__ constexpr int epi_warp_bytes(int epi) { return epi == 5 /*EPI_SGD*/ ? 12288 : epi == 10 /*EPI_SGD_LONG*/ ? 6144 : 8192; }
 __host__ __device__ constexpr int gemm_stages(int epi) { return epi == 5 /*EPI_SGD*/ ? 4 : 5; }
 __host__ __device__ constexpr int gemm_epi_region(int epi) { return epi_staged(epi) ? kEpiWarps * epi_warp_bytes(epi) : 0; }
 __host__ __device__ constexpr int gemm_smem_bytes(int epi) {
@@ -110,10 +111,11 @@ struct EpiMaps { CUtensorMap m[4]; };
 
 // Boxes per chunk buffer, how many of them are read from global memory first, and buffers per warp.
 __host__ __device__ constexpr int epi_slots(int epi) {
-  return (epi == EPI_SWIGLU_FWD || epi == EPI_SGD) ? 3 : (epi == EPI_MSE || epi == EPI_ACT_FWD || epi == EPI_DSWIGLU) ? 2 : 1;
+  return (epi == EPI_SWIGLU_FWD || epi == EPI_SGD || epi == EPI_SGD_LONG) ? 3
+         : (epi == EPI_MSE || epi == EPI_ACT_FWD || epi == EPI_DSWIGLU) ? 2 : 1;
 }
 __host__ __device__ constexpr int epi_in_slots(int epi) {
-  return (epi == EPI_DSWIGLU || epi == EPI_SGD) ? 2
+  return (epi == EPI_DSWIGLU || epi == EPI_SGD || epi == EPI_SGD_LONG) ? 2
          : (epi == EPI_MSE || epi == EPI_MSE_NOY || epi == EPI_DACT || epi == EPI_RESID) ? 1 : 0;
 }
 // chunk buffers per warp: what fits, rounded down to a power of two (4, 2 or 1)
@@ -476,10 +478,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     uint32_t tl = 0;
     bool ok = true;
 
-    if constexpr (EPI == EPI_ADAM || EPI == EPI_SGD_LONG) {
-      // Weight-gradient tiles updated from registers - the Adam step (three fp32 streams per weight: too many for
-      // the staging buffers) and SGD at very long contractions, where this epilogue is rare: plain vector accesses
-      // to the fp32 rows; the master values of the next chunk are loaded ahead.
+    if constexpr (EPI == EPI_ADAM) {
+      // Weight-gradient tiles with the Adam step (three fp32 streams per weight: too many for the staging buffers):
+      // plain vector accesses to the fp32 rows; the master values of the next chunk are loaded ahead.
       for (int tile = pair; ok && tile < total_tiles; tile += num_pairs, ++tl) {
         int g, mt, nt;
         tile_coords(p, tile, g, mt, nt);
@@ -598,14 +599,15 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       };
       TileAt cur = locate(pair), nxt = locate(pair + num_pairs);
       // EPI_SGD: whether this launch updates the weights at all (otherwise it only dumps gradients and stages nothing)
-      const bool sgd_update = EPI == EPI_SGD && (p.lr != 0.f || p.master_init != 0);
+      constexpr bool kSgd = EPI == EPI_SGD || EPI == EPI_SGD_LONG;
+      const bool sgd_update = kSgd && (p.lr != 0.f || p.master_init != 0);
       auto request_inputs = [&](uint32_t gc) {      // lane 0 only; gc / kChunks is tl or tl + 1
         if (kIn == 0) return;
         const TileAt& t = (gc / kChunks == tl) ? cur : nxt;
         if (!t.valid) return;
         const uint32_t bar = in_bar(warp, gc & (kBufs - 1));
         const int n = t.n0 + 32 * (int)(gc % kChunks);
-        if constexpr (EPI == EPI_SGD) {
+        if constexpr (kSgd) {
           if (!sgd_update) return;
           if (p.master_init) {      // the masters do not exist yet: the bf16 weights, whose widening they are
             mbar_expect_tx(bar, kEpiBoxBytes);
@@ -652,9 +654,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         for (int c = 0; c < kChunks; ++c) {
           const uint32_t gc = tl * kChunks + c;
           const int n = n_base + 32 * c;
-          if (kIn > 0 && (EPI != EPI_SGD || sgd_update)) {      // this chunk's boxes have arrived
+          if (kIn > 0 && (!kSgd || sgd_update)) {      // this chunk's boxes have arrived
             if (!__all_sync(0xffffffffu, mbar_wait(in_bar(warp, gc & (kBufs - 1)), (gc / kBufs) & 1u, abort_flag, p.status))) { ok = false; break; }
-          } else if (EPI != EPI_SGD) {      // the bulk store that last read this buffer is done with it
+          } else if (!kSgd) {      // the bulk store that last read this buffer is done with it
             if (lane == 0) bulk_wait_read<kBufs - 1>();
             __syncwarp();
           }
@@ -752,7 +754,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
               }
               sts128(piece(b0, q), make_uint4(wg[0], wg[1], wg[2], wg[3]));
               sts128(piece(b1, q), make_uint4(wu[0], wu[1], wu[2], wu[3]));
-            } else if constexpr (EPI == EPI_SGD) {
+            } else if constexpr (kSgd) {
               // columns 8 q .. 8 q + 7 of the chunk: two 16-byte pieces of a master box, one piece of the weight box
               float gv[8];
 #pragma unroll
@@ -826,7 +828,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             } else if constexpr (EPI == EPI_DSWIGLU) {
               tma_store_3d(&tmE.m[2], b0, n, rr, gg);
               tma_store_3d(&tmE.m[3], b1, n, rr, gg);
-            } else if constexpr (EPI == EPI_SGD) {
+            } else if constexpr (kSgd) {
               if (sgd_update) {
                 tma_store_3d(&tmE.m[0], b0, n, rr, gg);
                 tma_store_3d(&tmE.m[0], b1, n + 16, rr, gg);
