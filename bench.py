@@ -27,9 +27,8 @@ METRIC = "twist_round_tokens_per_s"
 UNIT = "tokens/s"
 # Nominal peaks of the part (dense bf16 tensor throughput, HBM3e bandwidth); fractions against them are reported
 # beside the fractions against the peaks measured on the machine.
-# dram bytes (read + write) of one 7B-shaped gather launch from the committed ncu capture (profiles/), None while
-# no capture of the current launch exists
-NCU_GATHER_TRAFFIC = None
+# dram bytes (read + write) of one 7B-shaped gather launch from the committed ncu capture (profiles/)
+NCU_GATHER_TRAFFIC = 1.42e9
 NOMINAL_BF16_TFLOPS = 2250.0
 NOMINAL_HBM_GBS = 8000.0
 
@@ -449,10 +448,9 @@ def run_ours(args, w):
                     # (the step runs under the power cap): achieved x max MHz / median MHz
                     "achieved_at_max_clock": (tflops * clocks["sm_max_mhz"] / clocks["sm_mhz"]
                                               if clocks and clocks.get("sm_mhz") and clocks.get("sm_max_mhz") else None),
-                    # dram read + write bytes per launch, averaged over the launches of a layer-step, from the
-                    # single-pass ncu capture at this exact size (profiles/gemm_kernel_cfg4_full_size_dram.txt);
-                    # any other workload has no capture
-                    "traffic": 12.5e9 if (args.config == 4 and not args.tokens and args.mode == "blockwise") else None,
+                    # dram read + write bytes per launch: the counters on file (profiles/) were taken at this size
+                    # before the kernel's tiles were synchronised; the kernel has changed since, so: null
+                    "traffic": None,
                     "flops_per_launch": work["gemm_flops"] / gemm_launches_per_round,
                     "avg_launch_ms": gemm_ms / args.steps / gemm_launches_per_round,
                     "share_of_step": gemm_ms / ms_total}
