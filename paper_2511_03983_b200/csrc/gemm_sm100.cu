@@ -63,14 +63,14 @@ int make_map(CUtensorMap* map, const GemmOperand& op, int groups, int box_rows) 
 
 // CTA pairs that can be resident at once (one CTA per SM, pairs on neighbouring SMs); queried once per
 // kernel instance and device.  More tiles than pairs: the persistent pairs stride over the tile list.
-template <int AM, int BM_, int EPI>
+template <int AM, int BM_, int EPI, bool HINTED>
 int resident_pairs(int* out) {
   static int cached[64] = {0};
   int dev = 0;
   TWIST_CUDA_TRY(cudaGetDevice(&dev));
   if (dev < 0 || dev >= 64) return TWIST_ERR_UNSUPPORTED;
   if (cached[dev] == 0) {
-    TWIST_CUDA_TRY(cudaFuncSetAttribute(gemm_kernel<AM, BM_, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    TWIST_CUDA_TRY(cudaFuncSetAttribute(gemm_kernel<AM, BM_, EPI, HINTED>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         gemm_smem_bytes(EPI)));
     cudaLaunchConfig_t cfg;
     memset(&cfg, 0, sizeof(cfg));
@@ -83,7 +83,7 @@ int resident_pairs(int* out) {
     cfg.attrs = &attr;
     cfg.numAttrs = 1;
     int n = 0;
-    if (cudaOccupancyMaxActiveClusters(&n, gemm_kernel<AM, BM_, EPI>, &cfg) != cudaSuccess || n <= 0) {
+    if (cudaOccupancyMaxActiveClusters(&n, gemm_kernel<AM, BM_, EPI, HINTED>, &cfg) != cudaSuccess || n <= 0) {
       cudaGetLastError();
       n = sm_count() / 2;
     }
@@ -151,6 +151,7 @@ int make_epilogue_maps(int epi, const GemmParams& p, const CUtensorMap& filler, 
 // further streams run unsynchronised); the host keeps the value each counter will have when the launches issued so
 // far on its stream have finished.  Launches on one stream are ordered, so they can share a counter.
 constexpr int kSgdLongK = 16384;        // contraction length from which the fused SGD update runs from registers
+constexpr size_t kHintMinABytes = (size_t)32 << 20;   // A rows of one group from which a token-major launch uses L2 hints
 constexpr int kWaveSlots = 64;
 constexpr int kWaveMinKBlocks = 32;     // contractions shorter than this (K < 2048) lose more to the wait than they save
 __device__ unsigned g_wave_ctr[kWaveSlots];
@@ -200,10 +201,10 @@ void wave_unreserve(const GemmParams& p, int grid) {
   w.base[p.wave_ctr - w.dev] -= (unsigned)p.n_waves * (unsigned)grid;
 }
 
-template <int AM, int BM_, int EPI>
-int launch(const CUtensorMap& ta, const CUtensorMap& tb, GemmParams p, cudaStream_t st) {
+template <int AM, int BM_, int EPI, bool HINTED>
+int launch_as(const CUtensorMap& ta, const CUtensorMap& tb, GemmParams p, cudaStream_t st) {
   int pairs = 0;
-  int rc = resident_pairs<AM, BM_, EPI>(&pairs);
+  int rc = resident_pairs<AM, BM_, EPI, HINTED>(&pairs);
   if (rc != TWIST_OK) return rc;
   const int tiles = p.groups * p.m_tiles * p.n_tiles;
   const int grid = 2 * (tiles < pairs ? tiles : pairs);
@@ -226,14 +227,36 @@ int launch(const CUtensorMap& ta, const CUtensorMap& tb, GemmParams p, cudaStrea
     attr.val.cooperative = 1;
     cfg.attrs = &attr;
     cfg.numAttrs = 1;
-    if (cudaLaunchKernelEx(&cfg, gemm_kernel<AM, BM_, EPI>, ta, tb, te, p) == cudaSuccess) return TWIST_OK;
+    if (cudaLaunchKernelEx(&cfg, gemm_kernel<AM, BM_, EPI, HINTED>, ta, tb, te, p) == cudaSuccess) return TWIST_OK;
     cudaGetLastError();                 // not launchable that way here: run it unsynchronised
     wave_unreserve(p, grid);
     p.wave_ctr = nullptr;
   }
-  gemm_kernel<AM, BM_, EPI><<<grid, kGemmThreads, smem, st>>>(ta, tb, te, p);
+  gemm_kernel<AM, BM_, EPI, HINTED><<<grid, kGemmThreads, smem, st>>>(ta, tb, te, p);
   TWIST_LAUNCH_CHECK();
   return TWIST_OK;
+}
+
+// L2 eviction priorities, for token-major launches (A = activation rows, B = a weight slice) whose activations do not
+// fit in L2 anyway: the weight slice is what every wave of tiles reads again, the activation rows pass through once,
+// and so does what the epilogue reads and writes - without the hints the stream of activations and results pushes
+// the weights out between waves (7B shapes, 8192 tokens: the up-projection read 2.05 GB from DRAM for 0.9 GB of
+// operands, 1.75 GB with them; the dX launch 2.41 -> 1.63 GB; the 32768-token round gained 0.5 - 0.9 % over the
+// plain copies).  Smaller launches, whose results the next launch finds in L2, lose 1 - 2 % to any hint;
+// weight-gradient launches (both operands stream along the contraction) gain nothing; launches too short for wave
+// synchronisation lose 6 % (their tiles drift apart, and an activation row marked evict-first is gone before the
+// last tile of the wave asks for it).  All of those keep the plain copies.
+template <int AM, int BM_, int EPI>
+int launch(const CUtensorMap& ta, const CUtensorMap& tb, GemmParams p, cudaStream_t st) {
+  if constexpr (AM == MAJOR_K) {
+    if ((size_t)p.M * (size_t)p.K * 2 >= kHintMinABytes && (p.K + kBK - 1) / kBK >= kWaveMinKBlocks) {
+      p.hint_a = L2_EVICT_FIRST;
+      p.hint_b = L2_EVICT_LAST;
+      p.hint_epi = L2_EVICT_FIRST;
+      return launch_as<AM, BM_, EPI, true>(ta, tb, p, st);
+    }
+  }
+  return launch_as<AM, BM_, EPI, false>(ta, tb, p, st);
 }
 
 // loss[g] = (sum of the group's partial sums, fixed order) / (tokens * valid columns of the group)

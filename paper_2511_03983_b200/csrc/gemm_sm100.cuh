@@ -39,6 +39,8 @@ enum { EPI_STORE = 0, EPI_SWIGLU_FWD = 1, EPI_ACT_FWD = 2, EPI_DSWIGLU = 3, EPI_
        EPI_ADAM = 9 /* weight gradient with the Adam update fused, like EPI_SGD */,
        EPI_SGD_LONG = 10 /* EPI_SGD for very long contractions: update from registers, full operand ring */ };
 
+enum { L2_NORMAL = 0, L2_EVICT_FIRST = 1, L2_EVICT_LAST = 2 };
+
 constexpr int kBM = 256, kBN = 256, kBK = 64, kUmmaK = 16;   // tile of a CTA pair
 constexpr int kCtaM = kBM / 2, kCtaN = kBN / 2;   // rows of A / columns of B that one CTA of the pair loads
 constexpr int kABytes = kCtaM * kBK * 2;          // 16 KB
@@ -73,6 +75,8 @@ struct GemmParams {
   int groups;
   int m_tiles, n_tiles;
   int raster_m;         // m-tiles per raster band (set by the launcher from the operand layout)
+  int hint_a, hint_b;   // hinted instantiations: L2 eviction priority of the A / B operand loads (L2_* above)
+  int hint_epi;         // ... and of the boxes the epilogue reads and writes
   int b_split;          // EPI_SWIGLU_FWD: row of the first "up" weight inside B (= f_sub)
   int act_kind;         // TWIST_FFN_*
   float scale, lr;
@@ -208,6 +212,14 @@ __device__ inline void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_
       "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
       ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2) : "memory");
 }
+// The same copy with an L2 eviction policy made by l2_policy().
+__device__ inline void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2,
+                                   uint64_t policy) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint"
+      " [%0], [%1, {%3, %4, %5}], [%2], %6;"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "l"(policy) : "memory");
+}
 // Arrives, once the MMAs issued so far have completed, on the barrier at this shared-memory offset in
 // both CTAs of the pair.
 __device__ inline void tc_commit_pair(uint32_t bar) {
@@ -335,7 +347,10 @@ __device__ inline void tile_coords(const GemmParams& p, int tile, int& g, int& m
   mt = m_first + (rr - nt * band_h);
 }
 
-template <int A_MAJOR, int B_MAJOR, int EPI>
+// HINTED: the operand and epilogue copies carry the L2 eviction policies of GemmParams::hint_* (a separate
+// instantiation, not a run-time choice: the producer's issue latency is on the critical path of the operand ring, and
+// both a branch and a predicated pair of copies per load cost the weight-gradient launches 3 - 10 %).
+template <int A_MAJOR, int B_MAJOR, int EPI, bool HINTED = false>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
             const __grid_constant__ EpiMaps tmE, const GemmParams p) {
@@ -389,6 +404,13 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       uint32_t it = 0;
       bool ok = true;
       unsigned wave = 0;
+      const uint64_t pol_a = HINTED ? l2_policy(p.hint_a) : 0, pol_b = HINTED ? l2_policy(p.hint_b) : 0;
+      auto load_a = [&](uint32_t dst, uint32_t bar, int c0, int c1, int c2) {
+        if constexpr (HINTED) tma_load_3d(dst, &tmA, bar, c0, c1, c2, pol_a); else tma_load_3d(dst, &tmA, bar, c0, c1, c2);
+      };
+      auto load_b = [&](uint32_t dst, uint32_t bar, int c0, int c1, int c2) {
+        if constexpr (HINTED) tma_load_3d(dst, &tmB, bar, c0, c1, c2, pol_b); else tma_load_3d(dst, &tmB, bar, c0, c1, c2);
+      };
       for (int tile = pair; ok && tile < total_tiles; tile += num_pairs, ++wave) {
         int g, mt, nt;
         tile_coords(p, tile, g, mt, nt);
@@ -413,16 +435,16 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           const uint32_t b_dst = a_dst + kABytes;
           const int k0 = kb * kBK;
           if (A_MAJOR == MAJOR_K) {
-            tma_load_3d(a_dst, &tmA, bar, k0, m0, g);                       // box 64 (K) x 128 rows
+            load_a(a_dst, bar, k0, m0, g);                       // box 64 (K) x 128 rows
           } else {
 #pragma unroll
-            for (int j = 0; j < kCtaM / 64; ++j) tma_load_3d(a_dst + j * 8192, &tmA, bar, m0 + 64 * j, k0, g);   // 64 (M) x 64 (K)
+            for (int j = 0; j < kCtaM / 64; ++j) load_a(a_dst + j * 8192, bar, m0 + 64 * j, k0, g);   // 64 (M) x 64 (K)
           }
           if (B_MAJOR == MAJOR_K) {
-            tma_load_3d(b_dst, &tmB, bar, k0, n0, g);                       // box 64 (K) x 128 rows
+            load_b(b_dst, bar, k0, n0, g);                       // box 64 (K) x 128 rows
           } else {
 #pragma unroll
-            for (int j = 0; j < kCtaN / 64; ++j) tma_load_3d(b_dst + j * 8192, &tmB, bar, n0 + 64 * j, k0, g);   // 64 (N) x 64 (K)
+            for (int j = 0; j < kCtaN / 64; ++j) load_b(b_dst + j * 8192, bar, n0 + 64 * j, k0, g);   // 64 (N) x 64 (K)
           }
         }
       }
@@ -601,6 +623,13 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       // EPI_SGD: whether this launch updates the weights at all (otherwise it only dumps gradients and stages nothing)
       constexpr bool kSgd = EPI == EPI_SGD || EPI == EPI_SGD_LONG;
       const bool sgd_update = kSgd && (p.lr != 0.f || p.master_init != 0);
+      const uint64_t pol_epi = HINTED ? l2_policy(p.hint_epi) : 0;
+      auto box_load = [&](uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2) {
+        if constexpr (HINTED) tma_load_3d_local(dst, map, bar, c0, c1, c2, pol_epi); else tma_load_3d_local(dst, map, bar, c0, c1, c2);
+      };
+      auto box_store = [&](const CUtensorMap* map, uint32_t src, int c0, int c1, int c2) {
+        if constexpr (HINTED) tma_store_3d(map, src, c0, c1, c2, pol_epi); else tma_store_3d(map, src, c0, c1, c2);
+      };
       auto request_inputs = [&](uint32_t gc) {      // lane 0 only; gc / kChunks is tl or tl + 1
         if (kIn == 0) return;
         const TileAt& t = (gc / kChunks == tl) ? cur : nxt;
@@ -611,17 +640,17 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           if (!sgd_update) return;
           if (p.master_init) {      // the masters do not exist yet: the bf16 weights, whose widening they are
             mbar_expect_tx(bar, kEpiBoxBytes);
-            tma_load_3d_local(box(gc, 2), &tmE.m[2], bar, n, t.row0, t.g);
+            box_load(box(gc, 2), &tmE.m[2], bar, n, t.row0, t.g);
           } else {                  // two boxes of 16 fp32 columns
             mbar_expect_tx(bar, 2 * kEpiBoxBytes);
-            tma_load_3d_local(box(gc, 0), &tmE.m[0], bar, n, t.row0, t.g);
-            tma_load_3d_local(box(gc, 1), &tmE.m[0], bar, n + 16, t.row0, t.g);
+            box_load(box(gc, 0), &tmE.m[0], bar, n, t.row0, t.g);
+            box_load(box(gc, 1), &tmE.m[0], bar, n + 16, t.row0, t.g);
           }
           return;
         }
         mbar_expect_tx(bar, kIn * kEpiBoxBytes);
 #pragma unroll
-        for (int i = 0; i < kIn; ++i) tma_load_3d_local(box(gc, i), &tmE.m[i], bar, n, t.row0, t.g);
+        for (int i = 0; i < kIn; ++i) box_load(box(gc, i), &tmE.m[i], bar, n, t.row0, t.g);
       };
       if (lane == 0) {
         for (uint32_t gc = 0; gc < (uint32_t)kAhead; ++gc) request_inputs(gc);
@@ -814,28 +843,28 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           if (lane == 0) {
             const int rr = row0, gg = g;
             if constexpr (EPI == EPI_STORE) {
-              tma_store_3d(&tmE.m[0], b0, n, rr, gg);
+              box_store(&tmE.m[0], b0, n, rr, gg);
             } else if constexpr (kIsMse) {
-              tma_store_3d(&tmE.m[1], b0, n, rr, gg);
-              if constexpr (EPI == EPI_MSE) tma_store_3d(&tmE.m[2], b1, n, rr, gg);
+              box_store(&tmE.m[1], b0, n, rr, gg);
+              if constexpr (EPI == EPI_MSE) box_store(&tmE.m[2], b1, n, rr, gg);
             } else if constexpr (EPI == EPI_SWIGLU_FWD) {
-              tma_store_3d(&tmE.m[0], b0, n, rr, gg);
-              tma_store_3d(&tmE.m[1], b1, n, rr, gg);
-              tma_store_3d(&tmE.m[2], b2, n, rr, gg);
+              box_store(&tmE.m[0], b0, n, rr, gg);
+              box_store(&tmE.m[1], b1, n, rr, gg);
+              box_store(&tmE.m[2], b2, n, rr, gg);
             } else if constexpr (EPI == EPI_ACT_FWD) {
-              tma_store_3d(&tmE.m[0], b0, n, rr, gg);
-              tma_store_3d(&tmE.m[1], b1, n, rr, gg);
+              box_store(&tmE.m[0], b0, n, rr, gg);
+              box_store(&tmE.m[1], b1, n, rr, gg);
             } else if constexpr (EPI == EPI_DSWIGLU) {
-              tma_store_3d(&tmE.m[2], b0, n, rr, gg);
-              tma_store_3d(&tmE.m[3], b1, n, rr, gg);
+              box_store(&tmE.m[2], b0, n, rr, gg);
+              box_store(&tmE.m[3], b1, n, rr, gg);
             } else if constexpr (kSgd) {
               if (sgd_update) {
-                tma_store_3d(&tmE.m[0], b0, n, rr, gg);
-                tma_store_3d(&tmE.m[0], b1, n + 16, rr, gg);
-                tma_store_3d(&tmE.m[2], b2, n, rr, gg);
+                box_store(&tmE.m[0], b0, n, rr, gg);
+                box_store(&tmE.m[0], b1, n + 16, rr, gg);
+                box_store(&tmE.m[2], b2, n, rr, gg);
               }
             } else {   // DACT, RESID
-              tma_store_3d(&tmE.m[1], b0, n, rr, gg);
+              box_store(&tmE.m[1], b0, n, rr, gg);
             }
             bulk_commit();
             if (kIn > 0) {     // refill the buffer whose store is old enough to have finished reading
