@@ -150,7 +150,7 @@ int make_epilogue_maps(int epi, const GemmParams& p, const CUtensorMap& filler, 
 // Wave synchronisation, host side.  One never-reset device counter per stream (up to kWaveSlots streams per device;
 // further streams run unsynchronised); the host keeps the value each counter will have when the launches issued so
 // far on its stream have finished.  Launches on one stream are ordered, so they can share a counter.
-constexpr int kSgdLongK = 16384;        // contraction length from which the fused SGD update runs from registers
+constexpr int kSgdLongK = 8192;         // contraction length from which the fused SGD update keeps the full operand ring
 constexpr size_t kHintMinABytes = (size_t)32 << 20;   // A rows of one group from which a token-major launch uses L2 hints
 constexpr int kWaveSlots = 64;
 constexpr int kWaveMinKBlocks = 32;     // contractions shorter than this (K < 2048) lose more to the wait than they save

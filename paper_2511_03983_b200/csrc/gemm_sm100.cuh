@@ -37,7 +37,7 @@ enum { MAJOR_K = 0, MAJOR_MN = 1 };
 enum { EPI_STORE = 0, EPI_SWIGLU_FWD = 1, EPI_ACT_FWD = 2, EPI_DSWIGLU = 3, EPI_DACT = 4, EPI_SGD = 5, EPI_MSE = 6, EPI_RESID = 7,
        EPI_MSE_NOY = 8 /* EPI_MSE without storing D: one box per chunk, so twice as many chunk buffers */,
        EPI_ADAM = 9 /* weight gradient with the Adam update fused, like EPI_SGD */,
-       EPI_SGD_LONG = 10 /* EPI_SGD for very long contractions: update from registers, full operand ring */ };
+       EPI_SGD_LONG = 10 /* EPI_SGD for long contractions: one staged chunk per warp, full operand ring */ };
 
 enum { L2_NORMAL = 0, L2_EVICT_FIRST = 1, L2_EVICT_LAST = 2 };
 
@@ -57,8 +57,8 @@ constexpr int kCtrlBytes = 512;
 // update, whose chunk is two fp32 master boxes and one bf16 weight box, 12 KB (two chunks in flight) and pays
 // for them with one stage of the operand ring (4 instead of 5: the weight-gradient contraction is the longest of
 // all, while at short contractions its time is the masters' read-modify-write, which staging makes asynchronous:
-// +19 % on the 1024-token workload).  At the longest contractions (32768 tokens) the shorter ring cost the 7B round
-// 2.5 % of its weight-gradient time, so those launches use EPI_SGD_LONG: the same staged update with one chunk
+// +19 % on the 1024-token workload).  At long contractions the shorter ring costs more (32768 tokens: 2.5 % of the 7B
+// round's weight-gradient time; 8192 tokens at d = 768: 1.5 - 6 % of the backward phases), so those use EPI_SGD_LONG: the same staged update with one chunk
 // buffer per warp (6 KB; the epilogue is rare there and need not overlap its own loads) and all five stages.
 // The Adam update works from registers and stages nothing.
 __host__ __device__ constexpr bool epi_staged(int epi) { return epi != 9 /*EPI_ADAM*/; }
