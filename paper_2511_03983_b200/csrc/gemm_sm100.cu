@@ -155,9 +155,11 @@ constexpr size_t kHintMinABytes = (size_t)32 << 20;   // A rows of one group fro
 constexpr int kWaveSlots = 64;
 constexpr int kWaveMinKBlocks = 32;     // contractions shorter than this (K < 2048) lose more to the wait than they save
 __device__ unsigned g_wave_ctr[kWaveSlots];
+__device__ unsigned g_done_ctr[kWaveSlots];     // GemmParams::done_ctr, one per stream like the wave counters
 struct WaveState {
   std::mutex mu;
   unsigned* dev = nullptr;              // device address of g_wave_ctr on this device
+  unsigned* done = nullptr;             // ... and of g_done_ctr
   cudaStream_t owner[kWaveSlots];
   unsigned base[kWaveSlots];
   int used = 0;
@@ -166,28 +168,38 @@ WaveState g_wave[64];
 
 // Picks the counter of stream `st` and reserves n_waves * grid arrivals on it.  Returns false when the launch
 // should run without wave synchronisation.
-bool wave_reserve(cudaStream_t st, int n_waves, int grid, GemmParams* p) {
+// Slot of stream `st` in the per-stream counter tables (w.mu held); -1: none left, or the stream is being captured
+// (the counters' sequence lives partly on the host and a captured launch may be replayed on any stream).
+int stream_slot(WaveState& w, cudaStream_t st) {
   cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
   if (cudaStreamIsCapturing(st, &cap) != cudaSuccess || cap != cudaStreamCaptureStatusNone) {
     cudaGetLastError();
-    return false;                       // the sequence numbers live on the host: not replayable from a graph
+    return -1;
   }
+  if (!w.dev) {
+    void *a = nullptr, *b = nullptr;
+    if (cudaGetSymbolAddress(&a, g_wave_ctr) != cudaSuccess || cudaGetSymbolAddress(&b, g_done_ctr) != cudaSuccess || !a || !b) {
+      cudaGetLastError();
+      return -1;
+    }
+    w.dev = static_cast<unsigned*>(a);
+    w.done = static_cast<unsigned*>(b);
+  }
+  for (int i = 0; i < w.used; ++i)
+    if (w.owner[i] == st) return i;
+  if (w.used == kWaveSlots) return -1;
+  w.owner[w.used] = st;
+  w.base[w.used] = 0;
+  return w.used++;
+}
+
+// Picks the counter of stream `st` and reserves n_waves * grid arrivals on it.  Returns false when the launch
+// should run without wave synchronisation.
+bool wave_reserve(cudaStream_t st, int n_waves, int grid, GemmParams* p) {
   WaveState& w = g_wave[device_slot()];
   std::lock_guard<std::mutex> lock(w.mu);
-  if (!w.dev) {
-    void* ptr = nullptr;
-    if (cudaGetSymbolAddress(&ptr, g_wave_ctr) != cudaSuccess || !ptr) { cudaGetLastError(); return false; }
-    w.dev = static_cast<unsigned*>(ptr);
-  }
-  int slot = -1;
-  for (int i = 0; i < w.used; ++i)
-    if (w.owner[i] == st) { slot = i; break; }
-  if (slot < 0) {
-    if (w.used == kWaveSlots) return false;
-    slot = w.used++;
-    w.owner[slot] = st;
-    w.base[slot] = 0;
-  }
+  const int slot = stream_slot(w, st);
+  if (slot < 0) return false;
   p->wave_ctr = w.dev + slot;
   p->wave_base = w.base[slot];
   p->n_waves = n_waves;
@@ -315,6 +327,7 @@ void reset_wave_sync() {
   std::lock_guard<std::mutex> lock(w.mu);
   static const unsigned zeros[kWaveSlots] = {0};
   if (cudaMemcpyToSymbol(g_wave_ctr, zeros, sizeof(zeros)) != cudaSuccess) cudaGetLastError();
+  if (cudaMemcpyToSymbol(g_done_ctr, zeros, sizeof(zeros)) != cudaSuccess) cudaGetLastError();
   for (int i = 0; i < kWaveSlots; ++i) w.base[i] = 0;
 }
 
@@ -331,6 +344,13 @@ int encode_map_3d_bf16(CUtensorMap* map, const void* ptr, const unsigned long lo
 size_t fused_loss_partials(int groups, int M, int N) {
   const size_t m_tiles = (size_t)(M + kBM - 1) / kBM, n_tiles = (size_t)(N + kBN - 1) / kBN;
   return (size_t)groups * m_tiles * n_tiles * 2 * kEpiWarps;
+}
+
+unsigned* fused_loss_counter(cudaStream_t st) {
+  WaveState& w = g_wave[device_slot()];
+  std::lock_guard<std::mutex> lock(w.mu);
+  const int slot = stream_slot(w, st);
+  return slot < 0 ? nullptr : w.done + slot;
 }
 
 int finish_fused_loss(const float* partial, int groups, int M, int N, const int32_t* valid_cols, int seg_begin,

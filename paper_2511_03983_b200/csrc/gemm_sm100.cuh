@@ -95,6 +95,11 @@ struct GemmParams {
   const int32_t* valid_cols;   // MSE: valid columns per column group and subnet [groups], or null (all valid)
   int seg_begin, seg_width;    // MSE: columns [0, seg_begin) valid, then groups of seg_width columns (see twist_mse_fwd_bwd)
   int* status;          // device status word
+  // MSE: when done_ctr is set, the CTA that finishes last reduces the partial sums into loss_out[groups] itself
+  // (same order and arithmetic as finish_fused_loss, which is then not needed).  Every CTA of the grid adds one to
+  // *done_ctr, which wraps to zero at the grid size: launches that share a counter must be ordered (one stream).
+  float* loss_out;
+  unsigned* done_ctr;
   // Wave synchronisation (null: off).  Every CTA of the grid adds one to *wave_ctr per wave (= per tile of its own,
   // plus once for a last wave it has no tile in); wave w may start once the counter has (nearly) reached
   // wave_base + (w + 1) * gridDim.x.  The counter is never reset: the host advances wave_base by n_waves * grid
@@ -888,6 +893,34 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     }
   }
 
+  if constexpr (EPI == EPI_MSE || EPI == EPI_MSE_NOY) {
+    if (p.done_ctr) {      // the last CTA to get here turns the partial sums into the losses
+      __shared__ int last_cta;
+      if (warp < kEpiWarps && lane == 0) __threadfence();        // this warp's partial sums are visible device-wide
+      __syncthreads();
+      if (threadIdx.x == 0) {
+        const unsigned before = atomicInc(p.done_ctr, gridDim.x - 1u);
+        last_cta = before == gridDim.x - 1u;
+      }
+      __syncthreads();
+      if (last_cta && warp < kEpiWarps) {
+        __threadfence();
+        const long long per_group = (long long)p.m_tiles * p.n_tiles * 2 * kEpiWarps;
+        for (int g = warp; g < p.groups; g += kEpiWarps) {
+          const float* src = p.dw + (long long)g * per_group;
+          double acc = 0.0;
+          for (long long i = lane; i < per_group; i += 32) acc += (double)__ldcg(src + i);
+          for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+          if (lane == 0) {
+            const int vc = p.valid_cols ? min(max(p.valid_cols[g], 0), p.seg_width) : p.seg_width;
+            const long long n_valid = p.seg_begin + (long long)((p.N - p.seg_begin) / p.seg_width) * vc;
+            p.loss_out[g] = n_valid > 0 ? (float)(acc / ((double)p.M * (double)n_valid)) : 0.f;
+          }
+        }
+      }
+    }
+  }
+
   // ------------------------------------------------------------------ teardown
   pair_teardown(abort_flag, warp == kEpiWarps + 1, tmem_base, (uint32_t)kTmemCols);
 }
@@ -905,6 +938,9 @@ int launch_gemm_bf16(int layout, int epi, const GemmOperand& A, const GemmOperan
 // EPI_MSE: number of fp32 partial sums the kernel writes (GemmParams::dw) for `groups` problems of M x N,
 // and the fixed-order reduction of those partials into loss[groups].
 size_t fused_loss_partials(int groups, int M, int N);
+// Counter for GemmParams::done_ctr on stream `st`, or null when the launch has to be followed by finish_fused_loss
+// (stream being captured, or more streams in use than there are counters).
+unsigned* fused_loss_counter(cudaStream_t st);
 int finish_fused_loss(const float* partial, int groups, int M, int N, const int32_t* valid_cols, int seg_begin,
                       int seg_width, float* loss, cudaStream_t st);
 

@@ -66,7 +66,12 @@ int launch_fused_loss(int layout, const GemmOperand& A, const GemmOperand& B, Ge
   p.valid_cols = valid_cols;
   p.seg_begin = valid_cols ? seg_begin : 0;
   p.seg_width = valid_cols ? seg_width : p.N;
+  // the last CTA of the launch reduces the partial sums itself; a separate (tiny) launch does it where no per-stream
+  // counter is to be had
+  p.loss_out = loss;
+  p.done_ctr = fused_loss_counter(st);
   TWIST_TRY(launch_gemm_bf16(layout, out ? EPI_MSE : EPI_MSE_NOY, A, B, p, st));
+  if (p.done_ctr) return TWIST_OK;
   return finish_fused_loss(p.dw, p.groups, p.M, p.N, valid_cols, p.seg_begin, p.seg_width, loss, st);
 }
 

@@ -368,7 +368,7 @@ class RoundEngine:
         with self._timed("ffn_fwd"):
             B.twist_subnet_ffn_fwd(a)
         if self.fuse_loss:
-            self.launches += 1 if w.dtype == DTYPE_BF16 else 2
+            self.launches += 0 if w.dtype == DTYPE_BF16 else 2      # bf16: the loss is finished inside the output GEMM
         else:
             self._mse(self.y, self.Td[k], self.dy, self.loss[l, 0, k], w.d_model)
         with self._timed("ffn_bwd"):
@@ -401,7 +401,7 @@ class RoundEngine:
         with self._timed("qkv_fwd"):
             B.twist_subnet_attn_proj_fwd(a)
         if self.fuse_loss:
-            self.launches += 1 if w.dtype == DTYPE_BF16 else 2
+            self.launches += 0 if w.dtype == DTYPE_BF16 else 2      # bf16: the loss is finished inside the output GEMM
         else:
             self._mse(self.qkv_out, self.Tq[k], self.dqkv, self.loss[l, 1, k], self.nq,
                       self.kv_cols[l] if ragged else None, self.a_sub, self.kv_max * w.d_head)
@@ -421,7 +421,7 @@ class RoundEngine:
         with self._timed("o_fwd"):
             B.twist_subnet_attn_proj_fwd(a)
         if self.fuse_loss:
-            self.launches += 1 if w.dtype == DTYPE_BF16 else 2
+            self.launches += 0 if w.dtype == DTYPE_BF16 else 2      # bf16: the loss is finished inside the output GEMM
         else:
             self._mse(self.y, self.Td[k], self.dy, self.loss[l, 2, k], w.d_model)
         with self._timed("o_bwd"):
@@ -698,7 +698,7 @@ class HybridRoundEngine(RoundEngine):
         with self._timed("ffn_bwd"):
             B.twist_subnet_ffn_bwd(c)
             B.twist_subnet_ffn_bwd(o)
-        self.launches += 2 * (2 + 1 + 3 + (1 if self.compute_dx else 0))
+        self.launches += 2 * (2 + 3 + (1 if self.compute_dx else 0))
 
     def qkv_step(self, l: int, k: int, lr: Optional[float] = None):
         w = self.w
@@ -720,7 +720,7 @@ class HybridRoundEngine(RoundEngine):
         with self._timed("qkv_bwd"):
             B.twist_subnet_attn_proj_bwd(c)
             B.twist_subnet_attn_proj_bwd(o)
-        self.launches += 2 * (2 + 1 + (1 if self.compute_dx else 0))
+        self.launches += 2 * (1 + 1 + (1 if self.compute_dx else 0))
 
     def o_step(self, l: int, k: int, lr: Optional[float] = None):
         w = self.w
@@ -741,7 +741,7 @@ class HybridRoundEngine(RoundEngine):
         with self._timed("o_bwd"):
             B.twist_subnet_attn_proj_bwd(c)
             B.twist_subnet_attn_proj_bwd(o)
-        self.launches += 1 + 2 * (2 + 1 + (1 if self.compute_dx else 0))
+        self.launches += 1 + 2 * (1 + 1 + (1 if self.compute_dx else 0))
 
     def aggregate_layer(self, l: int, live: int = 0xFFFFFFFF, which=("ffn", "attn")):
         w, d = self.w, self.w.d_model
