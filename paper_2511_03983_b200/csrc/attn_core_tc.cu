@@ -1,20 +1,21 @@
 // Tensor-core forward of the attention core (App. A: head_h = softmax(Q_h K_h^T / sqrt(d_head)) V_h, causal per
 // sequence) for d_head = 64, on tcgen05 with accumulators in tensor memory.
 //
-// One CTA per (block of 128 queries, kept head, sequence).  Per block of 128 keys:
-//   S = Q K^T        one 128 x 128 x 64 MMA chain, Q and K tiles brought by TMA (K-major, 128-byte swizzle)
-//   softmax          thread = query row: the row of S is read from tensor memory twice (maximum, then
-//                    exponentials), running maximum / sum kept in registers, P written to tensor memory (bf16
-//                    pairs, lane = query row) as the A operand of the next MMA: it never passes through shared
-//                    memory, whose bandwidth the operand reads of the MMAs already load
-//   O += P V         128 x 64 x 128 MMA chain accumulating in tensor memory, V as the MN-major B operand (rows =
-//                    keys as they lie in memory)
+// One CTA per (block of 128 queries, kept head, sequence).  K and V arrive by TMA in tiles of 128 keys (K-major,
+// 128-byte swizzle); the unit of S, P and the softmax is a half block of 64 keys:
+//   S = Q K^T        one 128 x 64 x 64 MMA chain per half block into one of two S buffers in tensor memory, issued two
+//                    half blocks ahead: the threads do not wait for it
+//   softmax          thread = query row: the 64 scores are read from tensor memory once and stay in registers
+//                    (maximum, exponentials), running maximum / sum kept in registers, P written to one of two P
+//                    buffers in tensor memory (bf16 pairs, lane = query row) as the A operand of the next MMA: it
+//                    never passes through shared memory, whose bandwidth the operand reads of the MMAs already load
+//   O += P V         128 x 64 x 64 MMA chain accumulating in tensor memory, V as the MN-major B operand (rows =
+//                    keys as they lie in memory); runs while the threads are at the next half block
 // P and O are expressed relative to a reference maximum that follows the running maximum lazily: only when a
 // row's maximum has grown by more than kRescaleLog2 since the reference was set does its warp rescale O in
-// tensor memory (and the running sum); otherwise P = 2^(s - ref) <= 2^kRescaleLog2 simply accumulates.  O / l is
-// the same quotient for any reference.  The threads therefore never read an output block: per key block they
-// read S, write P and go on.  S of the next block is issued before O += P V of the current one (the threads need
-// it first); between its two passes a thread only checks that the previous O += P V is done with P and O.
+// tensor memory (and the running sum), after waiting for the O += P V issued so far; otherwise
+// P = 2^(s - ref) <= 2^kRescaleLog2 simply accumulates.  O / l is the same quotient for any reference.  The threads
+// therefore never read an output block: per half block they read S, write P and go on.
 // Warps 0-3: softmax / output; warp 4, one lane: TMA and MMA issue.
 // Backward (same tile sizes; probabilities recomputed from the stored log-sum-exp, dS = P (dP - delta)):
 //   dQ kernel     one CTA per query block: per key block S = Q K^T and dP = dO V^T into tensor memory, the threads
@@ -38,7 +39,8 @@ constexpr int kBq = 128, kBk = 128;     // queries per CTA, keys per block
 constexpr int kTileBytes = 128 * kDh * 2;            // a 128-row tile of Q, K or V: 16 KB
 constexpr int kFwdThreads = 160;
 constexpr int kFwdSmem = kTileBytes * 5 + 1024 + 256;   // Q, K[2], V[2], alignment, barriers: two CTAs per SM
-constexpr int kFwdTmemCols = 256;       // S: columns 0..127, O: columns 128..191, P (bf16 pairs): columns 192..255
+constexpr int kHalf = 64;                // forward: keys per S / P half block
+constexpr int kFwdTmemCols = 256;       // S halves: columns 0..63 and 64..127, O: 128..191, P halves (bf16 pairs): 192..223, 224..255
 constexpr float kRescaleLog2 = 8.f;     // growth of a row maximum (log2 domain) tolerated before O is rescaled
 
 __device__ inline void mma1(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
@@ -76,45 +78,36 @@ __device__ inline float ex2_fast(float x) {
   return y;
 }
 
-// Softmax of one 128-key block for this thread's query row: reads the row of S from tensor memory twice (maximum,
-// then exponentials), keeps the reference maximum m (log2 domain) and the sum l relative to it, and writes
-// P = 2^(s * scale - m) (bf16 pairs) into the A operand in tensor memory.  MASKED: only columns <= k_lim are visible (the diagonal
-// block); the other blocks carry no per-element predicate.  The tensor-memory load of the next 32-column chunk is
-// in flight while the current one is processed.  `rescale(corr)` is called (by the whole warp) between the two
-// passes when some row of the warp moves its reference; it multiplies the row's O by corr.
-template <bool MASKED, typename BeforeP, typename Rescale>
-__device__ inline bool softmax_block(uint32_t t_s, uint32_t t_p, int k_lim, float scale_log2, float& m, float& l,
-                                     BeforeP&& before_p, Rescale&& rescale) {
+// Softmax of one half block (64 keys) for this thread's query row.  The 64 scores are read from tensor memory once
+// and stay in registers through the maximum, the (rare) rescale and the exponentials; m is the reference maximum
+// (log2 domain), l the sum relative to it; P = 2^(s * scale - m) goes (bf16 pairs) into the A operand in tensor
+// memory.  MASKED: only columns <= k_lim are visible (the diagonal block; k_lim may be negative); the other blocks
+// carry no per-element predicate.  `p_free()` is called (by the whole warp) before P is overwritten, `rescale(corr)`
+// when some row of the warp moves its reference: it multiplies the row's O by corr.
+template <bool MASKED, typename PFree, typename Rescale>
+__device__ inline bool softmax_half(uint32_t t_s, uint32_t t_p, int k_lim, float scale_log2, float& m, float& l,
+                                    PFree&& p_free, Rescale&& rescale) {
   uint32_t va[32], vb[32];
-  float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};   // four independent chains
-  auto fold_max = [&](const uint32_t (&v)[32], int c) {
-#pragma unroll
-    for (int i = 0; i < 32; ++i)
-      if (!MASKED || 32 * c + i <= k_lim) mx4[i & 3] = fmaxf(mx4[i & 3], __uint_as_float(v[i]));
-  };
   tc_ld32(t_s, va);
-  tc_wait_ld();
   tc_ld32(t_s + 32, vb);
-  fold_max(va, 0);
   tc_wait_ld();
-  tc_ld32(t_s + 64, va);
-  fold_max(vb, 1);
-  tc_wait_ld();
-  tc_ld32(t_s + 96, vb);
-  fold_max(va, 2);
-  tc_wait_ld();
-  fold_max(vb, 3);
+  float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};   // four independent chains
+#pragma unroll
+  for (int i = 0; i < 32; ++i)
+    if (!MASKED || i <= k_lim) mx4[i & 3] = fmaxf(mx4[i & 3], __uint_as_float(va[i]));
+#pragma unroll
+  for (int i = 0; i < 32; ++i)
+    if (!MASKED || 32 + i <= k_lim) mx4[i & 3] = fmaxf(mx4[i & 3], __uint_as_float(vb[i]));
   const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
   const float m_blk = mx * scale_log2;                 // scale > 0: the maximum commutes with the scaling
-  if (!before_p()) return false;                       // warp-uniform
+  if (!p_free()) return false;                         // warp-uniform
   if (__any_sync(0xffffffffu, m_blk > m + kRescaleLog2)) {
     const float m_new = fmaxf(m, m_blk);
     const float corr = ex2_fast(m - m_new);            // 0 for a first block (m = -inf), 1 where nothing moved
     l *= corr;
     m = m_new;
-    rescale(corr);
+    if (!rescale(corr)) return false;
   }
-  tc_ld32(t_s, va);
   float sum4[4] = {0.f, 0.f, 0.f, 0.f};
   auto emit = [&](const uint32_t (&v)[32], int c) {
     uint32_t w[16];
@@ -131,17 +124,8 @@ __device__ inline bool softmax_block(uint32_t t_s, uint32_t t_p, int k_lim, floa
     }
     tc_st16(t_p + 16 * c, w);                          // 32 keys = 16 columns of packed bf16 pairs
   };
-  tc_wait_ld();
-  tc_ld32(t_s + 32, vb);
   emit(va, 0);
-  tc_wait_ld();
-  tc_ld32(t_s + 64, va);
   emit(vb, 1);
-  tc_wait_ld();
-  tc_ld32(t_s + 96, vb);
-  emit(va, 2);
-  tc_wait_ld();
-  emit(vb, 3);
   tc_wait_st();
   l += (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
   return true;
@@ -168,8 +152,9 @@ __global__ void __maxnreg__(200) attn_fwd_tc_kernel(const __grid_constant__ CUte
   const uint32_t bar0 = base + 5 * kTileBytes;
   volatile uint32_t* ctrl = reinterpret_cast<volatile uint32_t*>(gen + 5 * kTileBytes);
   // Two CTAs share an SM (their startup, softmax and MMA phases interleave); K and V are double-buffered.
-  // barriers (8 bytes each): 0 q_full, 1-2 k_full, 3-4 v_full, 5-6 v_free, 7 s_full, 8 p_ready, 9 o_done;
+  // barriers (8 bytes each): 0 q_full, 1-2 k_full, 3-4 v_full, 5-6 v_free, 7-8 s_full, 9-10 p_ready, 11-12 pv_done;
   // then the TMEM base address and the abort flag
+  enum { Q_FULL = 0, K_FULL = 1, V_FULL = 3, V_FREE = 5, S_FULL = 7, P_READY = 9, PV_DONE = 11, N_BARS = 13 };
   auto bar = [&](int i) { return bar0 + 8u * i; };
   volatile uint32_t* tmem_slot = ctrl + 32;
   volatile int* abort_flag = reinterpret_cast<volatile int*>(ctrl + 33);
@@ -177,9 +162,10 @@ __global__ void __maxnreg__(200) attn_fwd_tc_kernel(const __grid_constant__ CUte
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int qb = blockIdx.x, hq = blockIdx.y, s = blockIdx.z / p.n_seqs, b = blockIdx.z - s * p.n_seqs;
   const int nblk = qb + 1;                               // causal: key blocks 0 .. qb
+  const int n_half = 2 * nblk;                           // half blocks of 64 keys: the unit of S, P and the softmax
   if (threadIdx.x == 128) {
     tma_prefetch_desc(&tmQKV);
-    for (int i = 0; i < 10; ++i) mbar_init(bar(i), i == 8 ? 128 : 1);
+    for (int i = 0; i < N_BARS; ++i) mbar_init(bar(i), (i == P_READY || i == P_READY + 1) ? 128 : 1);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     fence_async_smem();
@@ -202,54 +188,61 @@ __global__ void __maxnreg__(200) attn_fwd_tc_kernel(const __grid_constant__ CUte
       const int k_col = p.a_sub + kvp * kDh, v_col = k_col + p.kv_max * kDh;
       auto load_k = [&](int j) {
         const int st = j & 1;
-        mbar_expect_tx(bar(1 + st), kTileBytes);
-        tma_load_3d_local(k_s + st * kTileBytes, &tmQKV, bar(1 + st), k_col, j * kBk, z);
+        mbar_expect_tx(bar(K_FULL + st), kTileBytes);
+        tma_load_3d_local(k_s + st * kTileBytes, &tmQKV, bar(K_FULL + st), k_col, j * kBk, z);
       };
       auto load_v = [&](int j) {
         const int st = j & 1;
-        mbar_expect_tx(bar(3 + st), kTileBytes);
-        tma_load_3d_local(v_s + st * kTileBytes, &tmQKV, bar(3 + st), v_col, j * kBk, z);
+        mbar_expect_tx(bar(V_FULL + st), kTileBytes);
+        tma_load_3d_local(v_s + st * kTileBytes, &tmQKV, bar(V_FULL + st), v_col, j * kBk, z);
       };
-      mbar_expect_tx(bar(0), kTileBytes);
-      tma_load_3d_local(q_s, &tmQKV, bar(0), hq * kDh, qb * kBq, z);
+      mbar_expect_tx(bar(Q_FULL), kTileBytes);
+      tma_load_3d_local(q_s, &tmQKV, bar(Q_FULL), hq * kDh, qb * kBq, z);
       load_k(0);
       load_v(0);
       if (nblk > 1) { load_k(1); load_v(1); }
-      constexpr uint32_t idesc_s = idesc_bf16(0, 0, kBq, kBk);       // S = Q K^T : both K-major
+      constexpr uint32_t idesc_s = idesc_bf16(0, 0, kBq, kHalf);     // S = Q K^T : both K-major
       constexpr uint32_t idesc_o = idesc_bf16(0, 1, kBq, kDh);       // O = P V   : V MN-major
-      auto mma_s = [&](int j) {
-        const uint64_t a = smem_desc(q_s, 16u, 1024u), bd = smem_desc(k_s + (j & 1) * kTileBytes, 16u, 1024u);
+      // S of half block hb: Q against key rows 64 (hb & 1) .. of tile hb / 2 (64 rows of 128 bytes = 8 KB further on)
+      auto mma_s = [&](int hb) {
+        const uint64_t a = smem_desc(q_s, 16u, 1024u);
+        const uint64_t bd = smem_desc(k_s + ((hb >> 1) & 1) * kTileBytes + (hb & 1) * (kHalf * 128), 16u, 1024u);
 #pragma unroll
-        for (int k = 0; k < kDh / 16; ++k) mma1(tm_s, a + 2u * k, bd + 2u * k, idesc_s, k != 0);
-        commit1(bar(7));
+        for (int k = 0; k < kDh / 16; ++k) mma1(tm_s + (uint32_t)(hb & 1) * kHalf, a + 2u * k, bd + 2u * k, idesc_s, k != 0);
+        commit1(bar(S_FULL + (hb & 1)));
       };
-      bool ok = mbar_wait(bar(0), 0, abort_flag, status) && mbar_wait(bar(1), 0, abort_flag, status);
+      bool ok = mbar_wait(bar(Q_FULL), 0, abort_flag, status) && mbar_wait(bar(K_FULL), 0, abort_flag, status);
       if (ok) {
         tc_fence_after();
         mma_s(0);
+        mma_s(1);
       }
-      for (int j = 0; ok && j < nblk; ++j) {
-        const int st = j & 1;
-        // P of block j is in tensor memory and S(j) has been read: K(j)'s buffer and the S columns are free
-        if (!mbar_wait(bar(8), j & 1, abort_flag, status)) break;
+      for (int hb = 0; ok && hb < n_half; ++hb) {
+        const int j = hb >> 1, st = j & 1, h = hb & 1;
+        // P of half block hb is in tensor memory and S(hb) has been read: its S columns are free, and after the
+        // second half so is K(j)'s buffer
+        if (!mbar_wait(bar(P_READY + h), (hb >> 1) & 1, abort_flag, status)) break;
         tc_fence_after();
-        if (j + 2 < nblk) load_k(j + 2);
-        if (j + 1 < nblk) {                                // S of the next block first: the threads need it soonest
-          if (!mbar_wait(bar(1 + ((j + 1) & 1)), ((j + 1) >> 1) & 1, abort_flag, status)) break;
+        if (h == 1 && j + 2 < nblk) load_k(j + 2);
+        if (hb + 2 < n_half) {                             // S two half blocks ahead: the threads never wait for it
+          if (h == 0 && !mbar_wait(bar(K_FULL + ((j + 1) & 1)), ((j + 1) >> 1) & 1, abort_flag, status)) break;
           tc_fence_after();
-          mma_s(j + 1);
+          mma_s(hb + 2);
         }
-        if (!mbar_wait(bar(3 + st), (j >> 1) & 1, abort_flag, status)) break;     // V of block j
+        if (h == 0 && !mbar_wait(bar(V_FULL + st), (j >> 1) & 1, abort_flag, status)) break;     // V of block j
         tc_fence_after();
         const uint64_t bd = smem_desc(v_s + st * kTileBytes, (uint32_t)kDh * 128u, 1024u);
 #pragma unroll
-        for (int k = 0; k < kBk / 16; ++k)                                        // 16 keys = 8 columns of P
-          mma1_ta(tm_o, tm_p + 8u * k, bd + (uint64_t)((k * 16 * 128) >> 4), idesc_o, (j | k) != 0);
-        commit1(bar(5 + st));                                                     // V buffer free
-        commit1(bar(9));                                                          // P consumed, O at rest again
-        if (j + 2 < nblk) {
-          if (!mbar_wait(bar(5 + st), (j >> 1) & 1, abort_flag, status)) break;
-          load_v(j + 2);
+        for (int k = 0; k < kHalf / 16; ++k)                                      // 16 keys = 8 columns of P
+          mma1_ta(tm_o, tm_p + (uint32_t)h * (kHalf / 2) + 8u * k, bd + (uint64_t)(((4 * h + k) * 16 * 128) >> 4), idesc_o,
+                  (hb | k) != 0);
+        commit1(bar(PV_DONE + h));                                                // P(hb) consumed
+        if (h == 1) {
+          commit1(bar(V_FREE + st));                                              // V buffer free
+          if (j + 2 < nblk) {
+            if (!mbar_wait(bar(V_FREE + st), (j >> 1) & 1, abort_flag, status)) break;
+            load_v(j + 2);
+          }
         }
       }
     }
@@ -261,19 +254,24 @@ __global__ void __maxnreg__(200) attn_fwd_tc_kernel(const __grid_constant__ CUte
     const uint32_t t_s = tm_s + lane_off, t_o = tm_o + lane_off, t_p = tm_p + lane_off;
     float m = -INFINITY, l = 0.f;
     bool ok = true;
-    for (int j = 0; j < nblk; ++j) {
-      if (!__all_sync(0xffffffffu, mbar_wait(bar(7), j & 1, abort_flag, status))) { ok = false; break; }      // S(j)
+    for (int hb = 0; hb < n_half; ++hb) {
+      const int h = hb & 1;
+      if (!__all_sync(0xffffffffu, mbar_wait(bar(S_FULL + h), (hb >> 1) & 1, abort_flag, status))) { ok = false; break; }
       tc_fence_after();
-      // called between the two passes: O += P V of the previous block must be done before P is overwritten and
-      // before O may be rescaled; it was issued right after S(j), so it is usually complete by now
-      auto before_p = [&]() {
-        if (j == 0) return true;
-        const bool done = __all_sync(0xffffffffu, mbar_wait(bar(9), (j - 1) & 1, abort_flag, status));
+      // before P (hb & 1) is overwritten, O += P V of half block hb - 2 must have read it: long done as a rule
+      auto p_free = [&]() {
+        if (hb < 2) return true;
+        const bool done = __all_sync(0xffffffffu, mbar_wait(bar(PV_DONE + h), ((hb >> 1) - 1) & 1, abort_flag, status));
         tc_fence_after();
         return done;
       };
-      auto rescale = [&](float corr) {                   // whole warp: O row *= corr in tensor memory
-        if (j == 0) return;                              // nothing accumulated yet
+      // whole warp: O row *= corr in tensor memory, once every O += P V issued so far is complete (the latest is that
+      // of half block hb - 1; the next one is not issued before this warp has delivered P(hb))
+      auto rescale = [&](float corr) {
+        if (hb == 0) return true;                        // nothing accumulated yet
+        if (!__all_sync(0xffffffffu, mbar_wait(bar(PV_DONE + ((hb - 1) & 1)), ((hb - 1) >> 1) & 1, abort_flag, status)))
+          return false;
+        tc_fence_after();
 #pragma unroll
         for (int c = 0; c < kDh / 32; ++c) {
           uint32_t v[32];
@@ -284,15 +282,18 @@ __global__ void __maxnreg__(200) attn_fwd_tc_kernel(const __grid_constant__ CUte
           tc_st32(t_o + 32 * c, v);
         }
         tc_wait_st();
+        return true;
       };
       bool fine;
-      if (j == qb) fine = softmax_block<true>(t_s, t_p, qi - j * kBk, p.scale_log2, m, l, before_p, rescale);
-      else fine = softmax_block<false>(t_s, t_p, kBk, p.scale_log2, m, l, before_p, rescale);
+      const uint32_t ts = t_s + (uint32_t)h * kHalf, tp = t_p + (uint32_t)h * (kHalf / 2);
+      if ((hb >> 1) == qb) fine = softmax_half<true>(ts, tp, qi - (hb >> 1) * kBk - h * kHalf, p.scale_log2, m, l, p_free, rescale);
+      else fine = softmax_half<false>(ts, tp, kHalf, p.scale_log2, m, l, p_free, rescale);
       if (!fine) { ok = false; break; }
       tc_fence_before();
-      mbar_arrive(bar(8));
+      mbar_arrive(bar(P_READY + h));
     }
-    if (ok && __all_sync(0xffffffffu, mbar_wait(bar(9), (nblk - 1) & 1, abort_flag, status))) {
+    // the last O += P V (and with it every earlier one) complete
+    if (ok && __all_sync(0xffffffffu, mbar_wait(bar(PV_DONE + ((n_half - 1) & 1)), ((n_half - 1) >> 1) & 1, abort_flag, status))) {
       tc_fence_after();
       const float inv = 1.f / l;
       const long long row = (long long)s * p.T + (long long)b * p.seq_len + qi;
