@@ -211,7 +211,7 @@ __global__ void __maxnreg__(200) attn_fwd_tc_kernel(const __grid_constant__ CUte
         for (int k = 0; k < kDh / 16; ++k) mma1(tm_s + (uint32_t)(hb & 1) * kHalf, a + 2u * k, bd + 2u * k, idesc_s, k != 0);
         commit1(bar(S_FULL + (hb & 1)));
       };
-      bool ok = mbar_wait(bar(Q_FULL), 0, abort_flag, status) && mbar_wait(bar(K_FULL), 0, abort_flag, status);
+      bool ok = mbar_wait_cta(bar(Q_FULL), 0, abort_flag, status) && mbar_wait_cta(bar(K_FULL), 0, abort_flag, status);
       if (ok) {
         tc_fence_after();
         mma_s(0);
@@ -221,15 +221,10 @@ __global__ void __maxnreg__(200) attn_fwd_tc_kernel(const __grid_constant__ CUte
         const int j = hb >> 1, st = j & 1, h = hb & 1;
         // P of half block hb is in tensor memory and S(hb) has been read: its S columns are free, and after the
         // second half so is K(j)'s buffer
-        if (!mbar_wait(bar(P_READY + h), (hb >> 1) & 1, abort_flag, status)) break;
+        if (!mbar_wait_cta(bar(P_READY + h), (hb >> 1) & 1, abort_flag, status)) break;
         tc_fence_after();
         if (h == 1 && j + 2 < nblk) load_k(j + 2);
-        if (hb + 2 < n_half) {                             // S two half blocks ahead: the threads never wait for it
-          if (h == 0 && !mbar_wait(bar(K_FULL + ((j + 1) & 1)), ((j + 1) >> 1) & 1, abort_flag, status)) break;
-          tc_fence_after();
-          mma_s(hb + 2);
-        }
-        if (h == 0 && !mbar_wait(bar(V_FULL + st), (j >> 1) & 1, abort_flag, status)) break;     // V of block j
+        if (h == 0 && !mbar_wait_cta(bar(V_FULL + st), (j >> 1) & 1, abort_flag, status)) break;     // V of block j
         tc_fence_after();
         const uint64_t bd = smem_desc(v_s + st * kTileBytes, (uint32_t)kDh * 128u, 1024u);
 #pragma unroll
@@ -237,10 +232,18 @@ __global__ void __maxnreg__(200) attn_fwd_tc_kernel(const __grid_constant__ CUte
           mma1_ta(tm_o, tm_p + (uint32_t)h * (kHalf / 2) + 8u * k, bd + (uint64_t)(((4 * h + k) * 16 * 128) >> 4), idesc_o,
                   (hb | k) != 0);
         commit1(bar(PV_DONE + h));                                                // P(hb) consumed
+        // S two half blocks ahead, into the buffer the threads have just read: they never wait for it.  Issued after
+        // O += P V of this half block, so that its completion (S_FULL) also tells the threads that P (hb & 1) has been
+        // read and may be overwritten.
+        if (hb + 2 < n_half) {
+          if (h == 0 && !mbar_wait_cta(bar(K_FULL + ((j + 1) & 1)), ((j + 1) >> 1) & 1, abort_flag, status)) break;
+          tc_fence_after();
+          mma_s(hb + 2);
+        }
         if (h == 1) {
           commit1(bar(V_FREE + st));                                              // V buffer free
           if (j + 2 < nblk) {
-            if (!mbar_wait(bar(V_FREE + st), (j >> 1) & 1, abort_flag, status)) break;
+            if (!mbar_wait_cta(bar(V_FREE + st), (j >> 1) & 1, abort_flag, status)) break;
             load_v(j + 2);
           }
         }
@@ -256,20 +259,16 @@ __global__ void __maxnreg__(200) attn_fwd_tc_kernel(const __grid_constant__ CUte
     bool ok = true;
     for (int hb = 0; hb < n_half; ++hb) {
       const int h = hb & 1;
-      if (!__all_sync(0xffffffffu, mbar_wait(bar(S_FULL + h), (hb >> 1) & 1, abort_flag, status))) { ok = false; break; }
+      if (!__all_sync(0xffffffffu, mbar_wait_cta(bar(S_FULL + h), (hb >> 1) & 1, abort_flag, status))) { ok = false; break; }
       tc_fence_after();
-      // before P (hb & 1) is overwritten, O += P V of half block hb - 2 must have read it: long done as a rule
-      auto p_free = [&]() {
-        if (hb < 2) return true;
-        const bool done = __all_sync(0xffffffffu, mbar_wait(bar(PV_DONE + h), ((hb >> 1) - 1) & 1, abort_flag, status));
-        tc_fence_after();
-        return done;
-      };
+      // P (hb & 1) may be overwritten: O += P V of half block hb - 2 was issued before S(hb), whose completion the
+      // warp has just seen
+      auto p_free = [&]() { return true; };
       // whole warp: O row *= corr in tensor memory, once every O += P V issued so far is complete (the latest is that
       // of half block hb - 1; the next one is not issued before this warp has delivered P(hb))
       auto rescale = [&](float corr) {
         if (hb == 0) return true;                        // nothing accumulated yet
-        if (!__all_sync(0xffffffffu, mbar_wait(bar(PV_DONE + ((hb - 1) & 1)), ((hb - 1) >> 1) & 1, abort_flag, status)))
+        if (!__all_sync(0xffffffffu, mbar_wait_cta(bar(PV_DONE + ((hb - 1) & 1)), ((hb - 1) >> 1) & 1, abort_flag, status)))
           return false;
         tc_fence_after();
 #pragma unroll
@@ -293,7 +292,7 @@ __global__ void __maxnreg__(200) attn_fwd_tc_kernel(const __grid_constant__ CUte
       mbar_arrive(bar(P_READY + h));
     }
     // the last O += P V (and with it every earlier one) complete
-    if (ok && __all_sync(0xffffffffu, mbar_wait(bar(PV_DONE + ((n_half - 1) & 1)), ((n_half - 1) >> 1) & 1, abort_flag, status))) {
+    if (ok && __all_sync(0xffffffffu, mbar_wait_cta(bar(PV_DONE + ((n_half - 1) & 1)), ((n_half - 1) >> 1) & 1, abort_flag, status))) {
       tc_fence_after();
       const float inv = 1.f / l;
       const long long row = (long long)s * p.T + (long long)b * p.seq_len + qi;
@@ -440,13 +439,13 @@ __global__ void __launch_bounds__(kBwdThreads) attn_dq_tc_kernel(const __grid_co
         for (int k = 0; k < kDh / 16; ++k) mma1(tm_dp, ao + 2u * k, bv + 2u * k, idesc_s, k != 0);
         commit1(bar(9));
       };
-      bool ok = mbar_wait(bar(0), 0, abort_flag, status) && mbar_wait(bar(1), 0, abort_flag, status);
+      bool ok = mbar_wait_cta(bar(0), 0, abort_flag, status) && mbar_wait_cta(bar(1), 0, abort_flag, status);
       if (ok) {
         tc_fence_after();
         mma_s(0);
         mma_dp(0);
         if (nblk > 1) {
-          ok = mbar_wait(bar(2), 0, abort_flag, status);
+          ok = mbar_wait_cta(bar(2), 0, abort_flag, status);
           if (ok) {
             tc_fence_after();
             mma_s(1);
@@ -456,7 +455,7 @@ __global__ void __launch_bounds__(kBwdThreads) attn_dq_tc_kernel(const __grid_co
       for (int j = 0; ok && j < nblk; ++j) {
         const int st = j % kDqStages;
         // dS(j) is in tensor memory; S(j) and dP(j) have been read (the threads read S before dP)
-        if (!mbar_wait(bar(10), j & 1, abort_flag, status)) break;
+        if (!mbar_wait_cta(bar(10), j & 1, abort_flag, status)) break;
         tc_fence_after();
         const uint64_t bd = smem_desc(k_s + st * kTileBytes, (uint32_t)kDh * 128u, 1024u);
 #pragma unroll
@@ -469,12 +468,12 @@ __global__ void __launch_bounds__(kBwdThreads) attn_dq_tc_kernel(const __grid_co
         if (j + 1 < nblk) mma_dp(j + 1);
         if (j + 2 < nblk) {
           const int j2 = j + 2;
-          if (!mbar_wait(bar(1 + j2 % kDqStages), (j2 / kDqStages) & 1, abort_flag, status)) break;
+          if (!mbar_wait_cta(bar(1 + j2 % kDqStages), (j2 / kDqStages) & 1, abort_flag, status)) break;
           tc_fence_after();
           mma_s(j2);                                     // into the buffer S(j) has just left
         }
         if (j + kDqStages < nblk) {
-          if (!mbar_wait(bar(4 + st), (j / kDqStages) & 1, abort_flag, status)) break;
+          if (!mbar_wait_cta(bar(4 + st), (j / kDqStages) & 1, abort_flag, status)) break;
           load_kv(j + kDqStages);
         }
       }
@@ -491,7 +490,7 @@ __global__ void __launch_bounds__(kBwdThreads) attn_dq_tc_kernel(const __grid_co
     bool ok = true;
     for (int j = 0; j < nblk; ++j) {
       float pr[64];
-      if (!__all_sync(0xffffffffu, mbar_wait(bar(7 + (j & 1)), (j >> 1) & 1, abort_flag, status))) { ok = false; break; }
+      if (!__all_sync(0xffffffffu, mbar_wait_cta(bar(7 + (j & 1)), (j >> 1) & 1, abort_flag, status))) { ok = false; break; }
       tc_fence_after();
       const int k_lim = !row_ok ? -1 : ((j == qb) ? qi - j * kBk : kBk);
       const uint32_t t_s = tmem + lane_off + 128u * (j & 1);
@@ -499,13 +498,13 @@ __global__ void __launch_bounds__(kBwdThreads) attn_dq_tc_kernel(const __grid_co
         probs_from_s<true>(t_s, 2 * half, k_lim, p.scale_log2, lse2, pr);
       else
         probs_from_s<false>(t_s, 2 * half, k_lim, p.scale_log2, lse2, pr);
-      if (!__all_sync(0xffffffffu, mbar_wait(bar(9), j & 1, abort_flag, status))) { ok = false; break; }
+      if (!__all_sync(0xffffffffu, mbar_wait_cta(bar(9), j & 1, abort_flag, status))) { ok = false; break; }
       tc_fence_after();
       ds_from_dp(tm_dp + lane_off, 2 * half, dl, tm_ds + lane_off, pr);
       tc_fence_before();
       mbar_arrive(bar(10));
     }
-    if (ok && __all_sync(0xffffffffu, mbar_wait(bar(11), 0, abort_flag, status))) {
+    if (ok && __all_sync(0xffffffffu, mbar_wait_cta(bar(11), 0, abort_flag, status))) {
       tc_fence_after();
       uint32_t v[32];
       tc_ld32(tm_dq + lane_off + 32 * half, v);
@@ -668,13 +667,13 @@ __global__ void __launch_bounds__(kBwdThreads) attn_dkv_tc_kernel(const __grid_c
         for (int k = 0; k < kDh / 16; ++k) mma1(tm_dp, av + 2u * k, bo + 2u * k, idesc_s, k != 0);
         commit1(bar(9));
       };
-      bool ok = mbar_wait(bar(0), 0, abort_flag, status) && mbar_wait(bar(1), 0, abort_flag, status);
+      bool ok = mbar_wait_cta(bar(0), 0, abort_flag, status) && mbar_wait_cta(bar(1), 0, abort_flag, status);
       if (ok) {
         tc_fence_after();
         mma_s(0);
         mma_dp(0);
         if (total > 1) {
-          ok = mbar_wait(bar(2), 0, abort_flag, status);
+          ok = mbar_wait_cta(bar(2), 0, abort_flag, status);
           if (ok) {
             tc_fence_after();
             mma_s(1);
@@ -684,7 +683,7 @@ __global__ void __launch_bounds__(kBwdThreads) attn_dkv_tc_kernel(const __grid_c
       for (int n = 0; ok && n < total; ++n) {
         const int st = n % kDkvStages;
         // P^T and dS^T of unit n are in tensor memory (inside the S^T(n) and dP^T columns)
-        if (!mbar_wait(bar(10), n & 1, abort_flag, status)) break;
+        if (!mbar_wait_cta(bar(10), n & 1, abort_flag, status)) break;
         tc_fence_after();
         const uint32_t t_p = tmem + 128u * (n & 1);
         const uint64_t bo = smem_desc(do_s + st * kTileBytes, (uint32_t)kDh * 128u, 1024u);
@@ -702,12 +701,12 @@ __global__ void __launch_bounds__(kBwdThreads) attn_dkv_tc_kernel(const __grid_c
         if (n + 1 < total) mma_dp(n + 1);                // unit n + 1 arrived before S^T(n + 1) was issued
         if (n + 2 < total) {
           const int n2 = n + 2;
-          if (!mbar_wait(bar(1 + n2 % kDkvStages), (n2 / kDkvStages) & 1, abort_flag, status)) break;
+          if (!mbar_wait_cta(bar(1 + n2 % kDkvStages), (n2 / kDkvStages) & 1, abort_flag, status)) break;
           tc_fence_after();
           mma_s(n2);
         }
         if (n + kDkvStages < total) {
-          if (!mbar_wait(bar(4 + st), (n / kDkvStages) & 1, abort_flag, status)) break;
+          if (!mbar_wait_cta(bar(4 + st), (n / kDkvStages) & 1, abort_flag, status)) break;
           load_q(n + kDkvStages);
         }
       }
@@ -743,12 +742,12 @@ __global__ void __launch_bounds__(kBwdThreads) attn_dkv_tc_kernel(const __grid_c
       __syncwarp();
       staged = load_stat(n + 1);                         // in flight during this unit
       const int i = kb + n % per_head;
-      if (!__all_sync(0xffffffffu, mbar_wait(bar(7 + (n & 1)), (n >> 1) & 1, abort_flag, status))) { ok = false; break; }
+      if (!__all_sync(0xffffffffu, mbar_wait_cta(bar(7 + (n & 1)), (n >> 1) & 1, abort_flag, status))) { ok = false; break; }
       tc_fence_after();
       const uint32_t t_s = tmem + lane_off + 128u * (n & 1) + 64u * half;
       if (i == kb) probs_from_st<true>(t_s, st_lse, r, 64 * half, p.scale_log2, pr);      // diagonal block
       else probs_from_st<false>(t_s, st_lse, r, 64 * half, p.scale_log2, pr);
-      if (!__all_sync(0xffffffffu, mbar_wait(bar(9), n & 1, abort_flag, status))) { ok = false; break; }
+      if (!__all_sync(0xffffffffu, mbar_wait_cta(bar(9), n & 1, abort_flag, status))) { ok = false; break; }
       tc_fence_after();
       ds_from_dpt(tm_dp + lane_off + 64u * half, st_dl, pr);
       tc_fence_before();
@@ -761,7 +760,7 @@ __global__ void __launch_bounds__(kBwdThreads) attn_dkv_tc_kernel(const __grid_c
     if (total == 0) {                                    // a KV position this subnet does not hold: zero gradient
       if (kj < p.seq_len)
         for (int c = 0; c < kDh / 8; ++c) reinterpret_cast<uint4*>(dst)[c] = make_uint4(0, 0, 0, 0);
-    } else if (ok && __all_sync(0xffffffffu, mbar_wait(bar(11), 0, abort_flag, status))) {
+    } else if (ok && __all_sync(0xffffffffu, mbar_wait_cta(bar(11), 0, abort_flag, status))) {
       tc_fence_after();
       const float sc = half ? p.scale_log2 * 0.6931471805599453f : 1.f;          // dK carries 1 / sqrt(d_head)
 #pragma unroll

@@ -27,6 +27,17 @@ __device__ inline uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "=r"(done) : "r"(bar), "r"(parity) : "memory");
   return done;
 }
+// The same with CTA scope, for barriers that only this CTA's threads, copies and MMAs arrive at (the cluster-scope
+// acquire costs several tens of cycles more per call).
+__device__ inline uint32_t mbar_try_wait_cta(uint32_t bar, uint32_t parity) {
+  uint32_t done;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.acquire.cta.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+  return done;
+}
 __device__ inline uint64_t global_timer_ns() {
   uint64_t t;
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
@@ -56,6 +67,21 @@ __device__ inline bool mbar_wait_for(uint32_t bar, uint32_t parity, volatile int
 }
 __device__ inline bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status) {
   return mbar_wait_for(bar, parity, abort_flag, status, kWaitLimitNs);
+}
+// Bounded wait with CTA scope (see mbar_try_wait_cta).
+__device__ inline bool mbar_wait_cta(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status) {
+  if (mbar_try_wait_cta(bar, parity)) return true;
+  const uint64_t t0 = global_timer_ns();
+  for (uint32_t it = 1;; ++it) {
+    if (mbar_try_wait_cta(bar, parity)) return true;
+    if ((it & 255u) == 0) {
+      if (*abort_flag || global_timer_ns() - t0 > kWaitLimitNs) {
+        *abort_flag = 1;
+        note_status(status, (int)TWIST_ERR_DEVICE_TIMEOUT);
+        return false;
+      }
+    }
+  }
 }
 
 // After a wait ran out somewhere in the CTA: copies that were requested may still be in flight, so shared memory
