@@ -1080,6 +1080,58 @@ def test_plan_caches_tensor_maps_and_changes_no_result(B):
     plan.close()
 
 
+def test_layer_step_captured_in_a_cuda_graph_replays_bit_identically(B):
+    """A forward + backward FFN step with the fused loss, captured in a CUDA graph after an eager warm-up and replayed
+    twice, gives the bits of the eager step.  Inside a capture the library's host-sequenced device counters are off
+    (no wave synchronisation; the loss is finished by its own small launch), which changes no result; the contraction
+    is long enough (2304, 3 waves of tiles) for the eager step to use both."""
+    S, T, d, f = 4, 2560, 2304, 1280
+    bf, dtype = torch.bfloat16, I.DTYPE_BF16
+    t = lambda *shape: torch.zeros(*shape, dtype=bf, device="cuda")
+    X = dev(I.normal(131, 1, (S, T, d), 1.0, dtype), bf)
+    Tg = dev(I.normal(131, 4, (S, T, d), 1.0, dtype), bf)
+    Wgu = dev(I.normal(131, 2, (S, 2 * f, d), 0.02, dtype), bf)
+    Wd = dev(I.normal(131, 3, (S, f, d), 0.02, dtype), bf)
+    out = dict(pre=t(S, T, 2 * f), hh=t(S, T, f), dy=t(S, T, d), dpre=t(S, T, 2 * f), dx=t(S, T, d),
+               dw_gu=torch.zeros(S, 2 * f, d, dtype=torch.float32, device="cuda"),
+               dw_down=torch.zeros(S, f, d, dtype=torch.float32, device="cuda"),
+               loss=torch.zeros(S, dtype=torch.float32, device="cuda"))
+    ws = torch.empty(B.twist_fused_loss_workspace_bytes(S, T, d), dtype=torch.uint8, device="cuda")
+    a = B.ffn_args(I.FFN_SWIGLU, dtype, S, T, d, f, 2.0, 0.0, x=X, w_gu=Wgu, w_down=Wd, w_gu_master=Wgu.float(),
+                   w_down_master=Wd.float(), y=None, tgt=Tg, loss_ws=ws, **out)
+
+    def step():
+        B.twist_subnet_ffn_fwd(a)
+        B.twist_subnet_ffn_bwd(a)
+
+    def snapshot():
+        torch.cuda.synchronize()
+        check_status(B)
+        got = {k: v.clone() for k, v in out.items()}
+        for v in out.values():
+            v.zero_()
+        return got
+
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        step()                                       # eager, on the stream the capture will use
+        eager = snapshot()
+        assert float(eager["loss"].min()) > 0 and float(eager["dw_gu"].abs().max()) > 0
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            step()
+        snapshot()                                   # capturing runs nothing: the outputs are still zero
+        for _ in range(2):
+            graph.replay()
+            replayed = snapshot()
+            for k in eager:
+                assert torch.equal(eager[k], replayed[k]), k
+        step()                                       # and eager launches work as before afterwards
+        again = snapshot()
+        for k in eager:
+            assert torch.equal(eager[k], again[k]), k
+
+
 def test_masters_created_by_the_first_update_equal_masters_written_by_the_gather(B):
     """The gather may leave the fp32 masters unwritten: the first weight update after it reads the bf16 slice, whose
     exact widening the master is.  Both ways give the same bits everywhere - full model, fp32 result, losses - for
