@@ -63,7 +63,7 @@ def round_work(w, nq_valid=None):
     # aggregate: read every subnet's master (4 B) + write fp32 result and bf16 shadow for every covered element
     full = (w.nmat * w.d_ff + ((w.n_heads + 2 * w.n_kv_heads + w.n_heads) * w.d_head if w.n_heads else 0)) * d
     agg_bytes = 4 * kept * S * L + (4 + 2) * full * L         # cover mode: every element is covered
-    return {"gemm_flops": gemm_flops, "gather_bytes": gather_bytes, "aggregate_bytes": agg_bytes}
+    return {"gemm_flops": gemm_flops, "gather_bytes": gather_bytes, "aggregate_bytes": agg_bytes, "full_elems": full}
 
 
 # ------------------------------------------------------------------------------------------------
@@ -247,16 +247,20 @@ def workload_config(w, args):
                 "parallelism": "replicas only" if args.gpus > 1 else "single GPU"}
     hybrid = getattr(args, "mode", "blockwise") == "hybrid"
     masked = getattr(args, "mode", "blockwise") == "masked"
+    sharded = getattr(args, "mode", "blockwise") == "sharded"
     return {"workload": f"configs[{args.config - 1}] {w.name}: {'HYBRID ' if hybrid else 'MASKED ' if masked else ''}BLOCKWISE round, L={w.n_layers} d={w.d_model} "
                         f"F={w.d_ff} f'={w.f_sub} H'={w.head_keep}/{w.n_heads} S={w.n_subnets} T={w.tokens} K={w.local_steps}",
             "tokens_per_round": w.tokens_per_round,
             "mode": ("hybrid: worker 0 masked on the full-width model in place, the others on gathered slices; flops "
                      "counted are those of the gathered subnets" if hybrid else
                      "masked: every worker a full-width copy under its activation mask; flops counted are those of the "
-                     "gathered subnets" if masked else "blockwise, layers streamed"),
+                     "gathered subnets" if masked else
+                     "blockwise, layers streamed; the S subnets of one round spread over the GPUs, aggregate = partial "
+                     "sums + all-reduce + division" if sharded else "blockwise, layers streamed"),
             "l2_policy": "inputs larger than L2 (every tensor a kernel reads is >= 4x the 126 MB L2)"
                          if w.d_model >= 2048 else "working set exceeds L2 across the layers of a round",
-            "parallelism": "replicas only" if args.gpus > 1 else "single GPU"}
+            "parallelism": (f"subnets sharded over {args.gpus} GPUs" if sharded and args.gpus > 1 else
+                            "replicas only" if args.gpus > 1 else "single GPU")}
 
 
 # ------------------------------------------------------------------------------------------------
@@ -269,7 +273,8 @@ def run_ours(args, w):
 
     from paper_2511_03983_b200 import binding as B
     from paper_2511_03983_b200 import inputs as I
-    from paper_2511_03983_b200.engine import HybridRoundEngine, MaskedRoundEngine, RoundEngine, StackEngine
+    from paper_2511_03983_b200.engine import (HybridRoundEngine, MaskedRoundEngine, RoundEngine, ShardedRoundEngine,
+                                              StackEngine)
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -294,17 +299,21 @@ def run_ours(args, w):
             eng = HybridRoundEngine(w, compute_dx=True, fuse_loss=True, store_outputs=False)
         else:
             eng = MaskedRoundEngine(w, keep_f32_full=True, compute_dx=True, fuse_loss=True, store_outputs=False)
+    elif args.mode == "sharded":                          # the S subnets of ONE round spread over the GPUs
+        eng = ShardedRoundEngine(w, rank=rank, world=world, keep_f32_full=True, compute_dx=True, fuse_loss=True,
+                                 store_outputs=False)
     else:
         eng = RoundEngine(w, keep_f32_full=True, compute_dx=True, fuse_loss=True, store_outputs=False)
+    sharded = args.mode == "sharded"
     gen = torch.Generator(device="cuda")
-    gen.manual_seed(replica_seed(w.seed_w, rank))
+    gen.manual_seed(w.seed_w if sharded else replica_seed(w.seed_w, rank))      # sharded: one model on every GPU
     for m, v in eng.full.items():                         # weights ~ N(0, 0.02^2), one matrix at a time
         for l in range(w.n_layers):
             v[l].copy_((torch.randn(v[l].shape, generator=gen, device="cuda", dtype=torch.float32) * 0.02).to(td))
             if args.mode == "hybrid":                     # the central worker trains on the fp32 full model in place
                 eng.full_f32[m][l].copy_(v[l])
     gen.manual_seed(replica_seed(w.seed_x, rank))
-    S, T, K = w.n_subnets, w.tokens, w.local_steps
+    S, T, K = eng.w.n_subnets, w.tokens, w.local_steps     # (sharded: this GPU's subnets)
     widths = [("X", w.d_model), ("Td", w.d_model)] + ([("Tq", eng.nq), ("A", eng.a_sub)]
                                                       if (eng.has_attn and not stack) else [])
     host = {}
@@ -353,7 +362,9 @@ def run_ours(args, w):
     if status != 0:
         raise SystemExit(f"device status {status}: a bounded device wait expired")
     ms_per_step = max_over_ranks(ms_total) / args.steps
-    value = whole_job_value(w.tokens_per_round, world, ms_per_step)
+    # replicas: every GPU runs a whole round of its own; sharded: all GPUs together run one round
+    job_world = 1 if sharded else world
+    value = whole_job_value(w.tokens_per_round, job_world, ms_per_step)
 
     # ---- end-to-end: host buffers, copies inside the timed region --------------------------------
     e2e = None
@@ -408,7 +419,7 @@ def run_ours(args, w):
         for name, _ in widths:
             setattr(eng, name, sets[0][name])
         e2e_ms = max_over_ranks(e0.elapsed_time(e1)) / n_e2e
-        e2e = {"value": whole_job_value(w.tokens_per_round, world, e2e_ms), "unit": UNIT,
+        e2e = {"value": whole_job_value(w.tokens_per_round, job_world, e2e_ms), "unit": UNIT,
                "h2d_bytes_per_step": h2d_bytes, "d2h_bytes_per_step": d2h_bytes, "steps": n_e2e,
                "note": "pinned host batches copied in (the next step's copy overlaps the current round on a second "
                        "stream), per-subnet losses copied out, every step"
@@ -420,7 +431,12 @@ def run_ours(args, w):
         return
 
     peaks = measured_peaks()
-    work = round_work(w)
+    work = round_work(eng.w)                              # per GPU (sharded: its S / N subnets)
+    if sharded:     # the aggregate in two halves: sums of the GPU's subnets written for the whole layer (4 B per element),
+        full = work.pop("full_elems")     # then the reduced sums read and the fp32 model + bf16 shadow written (4 + 4 + 2)
+        work["aggregate_bytes"] += (4 + 4) * full * w.n_layers
+    else:
+        work.pop("full_elems")
     if args.mode == "hybrid":                             # worker 0 has no slice: S - 1 subnets are gathered
         work["gather_bytes"] *= (w.n_subnets - 1) / w.n_subnets
     if args.mode == "masked":                             # every worker copies and returns the whole layer
@@ -473,7 +489,8 @@ def run_ours(args, w):
         cpu = {k: cpu[k] for k in ("value", "unit", "cores", "kind", "sample")}
 
     out = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
-           "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+           "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "strong" if sharded else "weak",
+           "vs_baseline": None,
            "dtype": "bf16" if bf16 else "f32", "data": "synthetic", "config": workload_config(w, args),
            "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline, "hbm_kernels": hbm,
            "phases": phase_out, "cpu_baseline": cpu}
@@ -560,7 +577,7 @@ def main():
     ap.add_argument("--layers", type=int, default=0, help="override the layer count (profiling on a small case)")
     ap.add_argument("--tokens", type=int, default=0, help="override tokens per subnet-step (profiling on a small case)")
     ap.add_argument("--local-steps", type=int, default=0)
-    ap.add_argument("--mode", default="blockwise", choices=["blockwise", "stack", "hybrid", "masked"],
+    ap.add_argument("--mode", default="blockwise", choices=["blockwise", "stack", "hybrid", "masked", "sharded"],
                     help="stack: chained layers with the attention core (workloads 2 and 3); hybrid: worker 0 trains "
                          "the full-width model under a mask; masked: every worker does (FFN-only workload 5)")
     ap.add_argument("--sweep", action="store_true", help="workload 5: all 12 (S, keep) cells, gather / aggregate GB/s")

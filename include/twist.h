@@ -239,6 +239,28 @@ typedef struct {
 int32_t twist_aggregate(const twist_aggregate_segment* segs /*host*/, int32_t n_segs, int32_t n_subnets,
                         int32_t d, int32_t dtype, uint32_t live_subnets, void* stream);
 
+/* The aggregator in two halves, for subnets spread over several GPUs (Sec. 3.3; the server of Sec. 4.1 receives the
+ * workers' parameters and averages them).  Every GPU holds the whole model, the blueprints of all S subnets (the
+ * sampler is a pure function of the seed) and the slices of its own subnets subnet_begin .. subnet_begin +
+ * n_subnets - 1.
+ *   twist_aggregate_partial: for every block of a segment, each row of dst_f32 (fp32 dtype: of dst) becomes the fp32
+ *     sum, in ascending subnet order, of the rows of this GPU's live holders -- zeros where it has none.  `sub` and
+ *     `pos` hold only this GPU's subnets (numbered from 0), `cover` and live_subnets number the subnets globally.
+ *     dst_f32 (dst) is the GPU's partial-sum buffer, in the geometry of the full matrix; the bf16 dst is not written.
+ *     `central` must be NULL.
+ *   (the caller then adds the partial-sum buffers of all GPUs up, e.g. with an NCCL all-reduce)
+ *   twist_aggregate_finish: `central` holds the reduced sums (full-matrix geometry, like the Hybrid worker's matrix);
+ *     every row of a block held by c > 0 live subnets (of all n_subnets = S) becomes central_row / c (IEEE
+ *     division), written to dst_f32 (if not NULL; it may be `central` itself) and, rounded, to dst; blocks held by
+ *     none are left untouched.  `sub` and `pos` are not read.
+ * The sum over GPUs is associated differently from twist_aggregate's single running sum, so the two agree to fp32
+ * rounding of count additions, not bit for bit; with one GPU (subnet_begin 0, all S subnets) they are bit-identical.
+ * Status codes and index checks as for twist_aggregate. */
+int32_t twist_aggregate_partial(const twist_aggregate_segment* segs /*host*/, int32_t n_segs, int32_t n_subnets,
+                                int32_t subnet_begin, int32_t d, int32_t dtype, uint32_t live_subnets, void* stream);
+int32_t twist_aggregate_finish(const twist_aggregate_segment* segs /*host*/, int32_t n_segs, int32_t n_subnets,
+                               int32_t d, int32_t dtype, uint32_t live_subnets, void* stream);
+
 /* ---------------------------------------------------------------------------------------------
  * Local training on the dense slices (workers of Sec. 4.1 "True TwIST"; FFN of App. A:
  * y = C relu(W x); the GELU and SwiGLU variants are the workloads').  All S subnets run in one

@@ -33,7 +33,7 @@ EXPORTS = [
     "twist_mse_fwd_bwd_noalloc", "twist_fused_loss_workspace_bytes", "twist_attn_core_fwd", "twist_attn_core_bwd",
     "twist_hidden_mask", "twist_selftest_wait", "twist_layernorm_workspace_bytes", "twist_layernorm_fwd",
     "twist_layernorm_bwd", "twist_qkv_col_mask", "twist_apply_col_mask", "twist_plan_create", "twist_plan_destroy",
-    "twist_plan_stats", "twist_workspace_bytes",
+    "twist_plan_stats", "twist_workspace_bytes", "twist_aggregate_partial", "twist_aggregate_finish",
 ]
 
 
@@ -186,6 +186,9 @@ def lib() -> C.CDLL:
         h.twist_apply_col_mask.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_void_p]
         h.twist_gather_subnets.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_void_p]
         h.twist_aggregate.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_uint32, C.c_void_p]
+        h.twist_aggregate_partial.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_uint32,
+                                              C.c_void_p]
+        h.twist_aggregate_finish.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_uint32, C.c_void_p]
         h.twist_layernorm_workspace_bytes.restype = C.c_size_t
         h.twist_layernorm_workspace_bytes.argtypes = [C.c_int32, C.c_int32, C.c_int32]
         for name in ("twist_subnet_ffn_fwd", "twist_subnet_ffn_bwd", "twist_subnet_attn_proj_fwd",
@@ -305,6 +308,18 @@ def twist_aggregate(segs: Sequence[AggregateSegment], n_subnets, d, dtype, live_
     arr = (AggregateSegment * len(segs))(*segs)
     _check(lib().twist_aggregate(C.cast(arr, C.c_void_p), len(segs), n_subnets, d, dtype, live_subnets, _stream()),
            "twist_aggregate")
+
+
+def twist_aggregate_partial(segs: Sequence[AggregateSegment], n_subnets, subnet_begin, d, dtype, live_subnets=0xFFFFFFFF):
+    arr = (AggregateSegment * len(segs))(*segs)
+    _check(lib().twist_aggregate_partial(C.cast(arr, C.c_void_p), len(segs), n_subnets, subnet_begin, d, dtype,
+                                         live_subnets, _stream()), "twist_aggregate_partial")
+
+
+def twist_aggregate_finish(segs: Sequence[AggregateSegment], n_subnets, d, dtype, live_subnets=0xFFFFFFFF):
+    arr = (AggregateSegment * len(segs))(*segs)
+    _check(lib().twist_aggregate_finish(C.cast(arr, C.c_void_p), len(segs), n_subnets, d, dtype, live_subnets, _stream()),
+           "twist_aggregate_finish")
 
 
 def _ws_bytes(ws) -> int:

@@ -34,7 +34,7 @@ int sm_count() {
 
 extern "C" {
 
-uint32_t twist_abi_version(void) { return 2u; }
+uint32_t twist_abi_version(void) { return 3u; }
 
 const char* twist_strerror(int32_t status) {
   switch (status) {

@@ -28,7 +28,11 @@ struct AggParams {
   long long total_rows;
   int parts;          // work item = one of `parts` equal spans of a row
   int part_chunks;    // float4 chunks per span
+  int mode;           // AGG_MEAN: the aggregator; AGG_PARTIAL / AGG_FINISH: its two halves when the subnets are spread
+                      // over several GPUs (sum over this GPU's subnets; division of the reduced sums by the coverage)
+  int subnet_begin;   // AGG_PARTIAL: global index of this GPU's first subnet (bit of the cover masks)
 };
+enum { AGG_MEAN = 0, AGG_PARTIAL = 1, AGG_FINISH = 2 };
 
 __device__ inline uint4 ld_nc(const uint4* p) {
   uint4 v;
@@ -224,17 +228,22 @@ __global__ void __launch_bounds__(256) aggregate_rows_kernel(const __grid_consta
     const twist_aggregate_segment& sg = p.seg[g];
     const long long rl = r - (g ? p.row_end[g - 1] : 0);
     const int b = (int)(rl / sg.block_rows), i = (int)(rl - (long long)b * sg.block_rows);
-    const uint32_t m = sg.cover[b] & p.live;
-    if (m == 0) continue;                              // held by no live subnet: untouched
-    const int cnt = __popc(m);
+    const uint32_t held = sg.cover[b] & p.live;          // subnets (global numbering) that hold the block
+    // the rows this warp adds up: every holder (AGG_MEAN), this GPU's holders (AGG_PARTIAL: bits subnet_begin ..
+    // subnet_begin + n_subnets - 1, renumbered from 0 - sub and pos hold only those), or the one row of reduced
+    // sums (AGG_FINISH)
+    uint32_t m = held;
+    if (p.mode == AGG_PARTIAL) m = (held >> p.subnet_begin) & (p.n_subnets >= 32 ? 0xFFFFFFFFu : ((1u << p.n_subnets) - 1u));
+    if (p.mode != AGG_PARTIAL && held == 0) continue;    // held by no live subnet: untouched
+    const int cnt = p.mode == AGG_FINISH ? 1 : __popc(m);
     // lane k holds the row pointer of the k-th covering subnet; bit 0 marks a row of the full-width matrix itself
     // (it may be the destination, so it is read with an ordinary load, not through the read-only path)
     unsigned long long mine = 0;
     const long long drow = sg.dst_row_offset + rl;
     bool bad = false;
     if (lane < cnt) {
-      const int s = __fns(m, 0, lane + 1);
-      if (sg.central && s == sg.central_subnet) {        // trained in place on the full-width matrix
+      const int s = p.mode == AGG_FINISH ? -1 : __fns(m, 0, lane + 1);
+      if (p.mode == AGG_FINISH || (sg.central && s == sg.central_subnet)) {   // a row in full-matrix geometry
         mine = reinterpret_cast<unsigned long long>(sg.central + drow * p.d) | 1ull;
       } else {
         const int rank = sg.pos[(long long)s * sg.n_full + b];
@@ -249,7 +258,8 @@ __global__ void __launch_bounds__(256) aggregate_rows_kernel(const __grid_consta
     }
     // Quotient by the coverage count: reciprocal product corrected with the exact remainder, which gives
     // the correctly rounded quotient (the same bits as an IEEE division) at a fraction of its cost.
-    const float denom = (float)cnt;
+    // (AGG_PARTIAL divides by one - the sum itself; AGG_FINISH by the number of holders on all GPUs)
+    const float denom = p.mode == AGG_PARTIAL ? 1.f : (float)__popc(held);
     const float rden = 1.0f / denom;
     auto quot = [&](float a) {
       const float q = a * rden;
@@ -291,8 +301,9 @@ __global__ void __launch_bounds__(256) aggregate_rows_kernel(const __grid_consta
           uint4 qb = make_uint4(__float_as_uint(q.x), __float_as_uint(q.y), __float_as_uint(q.z), __float_as_uint(q.w));
           if (BF16) {
             if (sg.dst_f32) st_cs(reinterpret_cast<uint4*>(sg.dst_f32 + drow * p.d) + c, qb);
-            st_cs2(reinterpret_cast<uint2*>(static_cast<__nv_bfloat16*>(sg.dst) + drow * p.d) + c,
-                   make_uint2(pack_bf16x2_rn(q.x, q.y), pack_bf16x2_rn(q.z, q.w)));
+            if (p.mode != AGG_PARTIAL)                   // partial sums are fp32 only
+              st_cs2(reinterpret_cast<uint2*>(static_cast<__nv_bfloat16*>(sg.dst) + drow * p.d) + c,
+                     make_uint2(pack_bf16x2_rn(q.x, q.y), pack_bf16x2_rn(q.z, q.w)));
           } else {
             st_cs(reinterpret_cast<uint4*>(static_cast<float*>(sg.dst) + drow * p.d) + c, qb);
           }
@@ -372,12 +383,14 @@ extern "C" int32_t twist_gather_subnets(const twist_gather_segment* segs, int32_
   return TWIST_OK;
 }
 
-extern "C" int32_t twist_aggregate(const twist_aggregate_segment* segs, int32_t n_segs, int32_t n_subnets, int32_t d,
-                                   int32_t dtype, uint32_t live_subnets, void* stream) {
-  using namespace twist;
+namespace twist {
+namespace {
+int aggregate_launch(const twist_aggregate_segment* segs, int n_segs, int n_subnets, int subnet_begin, int d, int dtype,
+                     uint32_t live_subnets, int mode, void* stream) {
   if (!segs) return TWIST_ERR_NULL;
   if (n_segs <= 0 || n_segs > TWIST_MAX_SEGMENTS || n_subnets <= 0 || n_subnets > TWIST_MAX_SUBNETS || d <= 0)
     return TWIST_ERR_SHAPE;
+  if (subnet_begin < 0 || subnet_begin + n_subnets > TWIST_MAX_SUBNETS) return TWIST_ERR_SHAPE;
   if (dtype != TWIST_FP32 && dtype != TWIST_BF16) return TWIST_ERR_SHAPE;
   if (d % 4 != 0 || (dtype == TWIST_BF16 && d % 8 != 0)) return TWIST_ERR_SHAPE;
   AggParams p;
@@ -385,12 +398,16 @@ extern "C" int32_t twist_aggregate(const twist_aggregate_segment* segs, int32_t 
   long long total = 0;
   for (int g = 0; g < n_segs; ++g) {
     const twist_aggregate_segment& s = segs[g];
-    if (!s.dst || !s.sub || !s.cover || !s.pos) return TWIST_ERR_NULL;
-    if (s.n_full <= 0 || s.block_rows <= 0 || s.n_keep <= 0 || s.dst_row_offset < 0 || s.sub_row_offset < 0 ||
-        s.sub_subnet_stride < 0 || s.sub_subnet_stride % 4 != 0)
+    if (!s.dst || !s.cover) return TWIST_ERR_NULL;
+    if (mode != AGG_FINISH && (!s.sub || !s.pos)) return TWIST_ERR_NULL;
+    if (mode == AGG_FINISH && !s.central) return TWIST_ERR_NULL;                  // the reduced sums
+    if (mode == AGG_PARTIAL && s.central) return TWIST_ERR_UNSUPPORTED;           // no in-place worker on a shard
+    if (mode == AGG_PARTIAL && dtype == TWIST_BF16 && !s.dst_f32) return TWIST_ERR_NULL;   // sums are fp32
+    if (s.n_full <= 0 || s.block_rows <= 0 || s.dst_row_offset < 0) return TWIST_ERR_SHAPE;
+    if (mode != AGG_FINISH && (s.n_keep <= 0 || s.sub_row_offset < 0 || s.sub_subnet_stride < 0 || s.sub_subnet_stride % 4 != 0))
       return TWIST_ERR_SHAPE;
     if (!aligned16(s.dst) || !aligned16(s.sub) || !aligned16(s.dst_f32) || !aligned16(s.central)) return TWIST_ERR_SHAPE;
-    if (s.central && (s.central_subnet < 0 || s.central_subnet >= n_subnets)) return TWIST_ERR_BAD_INDEX;
+    if (mode == AGG_MEAN && s.central && (s.central_subnet < 0 || s.central_subnet >= n_subnets)) return TWIST_ERR_BAD_INDEX;
     if (dtype == TWIST_FP32 && s.dst_f32) return TWIST_ERR_UNSUPPORTED;      // dst already is the fp32 result
     p.seg[g] = s;
     total += (long long)s.n_full * s.block_rows;
@@ -399,7 +416,11 @@ extern "C" int32_t twist_aggregate(const twist_aggregate_segment* segs, int32_t 
   p.n_segs = n_segs;
   p.d = d;
   p.n_subnets = n_subnets;
-  p.live = n_subnets >= 32 ? live_subnets : (live_subnets & ((1u << n_subnets) - 1u));
+  p.mode = mode;
+  p.subnet_begin = subnet_begin;
+  // cover masks number the subnets globally: AGG_MEAN and AGG_FINISH see n_subnets of them from bit 0, AGG_PARTIAL
+  // keeps every live bit and picks its own range in the kernel
+  p.live = (mode == AGG_PARTIAL || n_subnets >= 32) ? live_subnets : (live_subnets & ((1u << n_subnets) - 1u));
   p.total_rows = total;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   // A row is split into spans of kAggPartChunks float4 chunks: with whole rows as items a warp of the persistent
@@ -413,4 +434,22 @@ extern "C" int32_t twist_aggregate(const twist_aggregate_segment* segs, int32_t 
   else aggregate_rows_kernel<false><<<grid, 256, 0, st>>>(p, status);
   TWIST_LAUNCH_CHECK();
   return TWIST_OK;
+}
+}  // namespace
+}  // namespace twist
+
+extern "C" int32_t twist_aggregate(const twist_aggregate_segment* segs, int32_t n_segs, int32_t n_subnets, int32_t d,
+                                   int32_t dtype, uint32_t live_subnets, void* stream) {
+  return twist::aggregate_launch(segs, n_segs, n_subnets, 0, d, dtype, live_subnets, twist::AGG_MEAN, stream);
+}
+
+extern "C" int32_t twist_aggregate_partial(const twist_aggregate_segment* segs, int32_t n_segs, int32_t n_subnets,
+                                           int32_t subnet_begin, int32_t d, int32_t dtype, uint32_t live_subnets,
+                                           void* stream) {
+  return twist::aggregate_launch(segs, n_segs, n_subnets, subnet_begin, d, dtype, live_subnets, twist::AGG_PARTIAL, stream);
+}
+
+extern "C" int32_t twist_aggregate_finish(const twist_aggregate_segment* segs, int32_t n_segs, int32_t n_subnets, int32_t d,
+                                          int32_t dtype, uint32_t live_subnets, void* stream) {
+  return twist::aggregate_launch(segs, n_segs, n_subnets, 0, d, dtype, live_subnets, twist::AGG_FINISH, stream);
 }

@@ -300,40 +300,49 @@ class RoundEngine:
                 getattr(self, n).zero_()
         self.launches += 1
 
-    def aggregate_layer(self, l: int, live: int = 0xFFFFFFFF, which=("ffn", "attn")):
-        self._use(l)
+    def _aggregate_segments(self, l: int, which, dst, f32, central=lambda m: None):
+        """The aggregate's row ranges of layer l.  dst(m) / f32(m): destination of matrix m in the workload's dtype and
+        its fp32 companion (or None); central(m): a source in full-matrix geometry (or None)."""
         w, d = self.w, self.w.d_model
         f, gf, keep = self.f_sub, self.gf, self.ffn_keep
         bf16 = w.dtype == DTYPE_BF16
-        f32 = (lambda m: self.full_f32[m][l]) if self.full_f32 is not None else (lambda m: None)
         sub = lambda lo, master: master if bf16 else lo
         nb = w.n_ffn_blocks
         segs = []
         if "ffn" in which:
             if self.g == 2:
-                segs.append(B.aggregate_segment(self.full["gate"][l], f32("gate"), sub(self.w_gu, self.w_gu_m),
+                segs.append(B.aggregate_segment(dst("gate"), f32("gate"), sub(self.w_gu, self.w_gu_m),
                                                 self.cover_ffn[l], self.agg_pos_ffn[l], nb, w.ffn_block, 0, gf * d, 0,
-                                                keep))
-            segs.append(B.aggregate_segment(self.full["up"][l], f32("up"), sub(self.w_gu, self.w_gu_m),
+                                                keep, central=central("gate")))
+            segs.append(B.aggregate_segment(dst("up"), f32("up"), sub(self.w_gu, self.w_gu_m),
                                             self.cover_ffn[l], self.agg_pos_ffn[l], nb, w.ffn_block, 0, gf * d,
-                                            f if self.g == 2 else 0, keep))
-            segs.append(B.aggregate_segment(self.full["down"][l], f32("down"), sub(self.w_down, self.w_down_m),
+                                            f if self.g == 2 else 0, keep, central=central("up")))
+            segs.append(B.aggregate_segment(dst("down"), f32("down"), sub(self.w_down, self.w_down_m),
                                             self.cover_ffn[l], self.agg_pos_ffn[l], nb, w.ffn_block, 0, f * d, 0,
-                                            keep))
+                                            keep, central=central("down")))
         if self.has_attn and "attn" in which:
             H, Hkv, dh = w.n_heads, w.n_kv_heads, w.d_head
             q_sub = sub(self.w_qkv, self.w_qkv_m)
-            segs.append(B.aggregate_segment(self.full["qkv"][l], f32("qkv"), q_sub, self.cover_head[l],
-                                            self.pos_head[l], H, dh, 0, self.nq * d, 0, self.head_keep))
-            segs.append(B.aggregate_segment(self.full["qkv"][l], f32("qkv"), q_sub, self.kv_cover[l], self.kv_pos[l],
-                                            Hkv, dh, H * dh, self.nq * d, self.a_sub, self.kv_max))
-            segs.append(B.aggregate_segment(self.full["qkv"][l], f32("qkv"), q_sub, self.kv_cover[l], self.kv_pos[l],
+            cq = central("qkv")
+            segs.append(B.aggregate_segment(dst("qkv"), f32("qkv"), q_sub, self.cover_head[l],
+                                            self.pos_head[l], H, dh, 0, self.nq * d, 0, self.head_keep, central=cq))
+            segs.append(B.aggregate_segment(dst("qkv"), f32("qkv"), q_sub, self.kv_cover[l], self.kv_pos[l],
+                                            Hkv, dh, H * dh, self.nq * d, self.a_sub, self.kv_max, central=cq))
+            segs.append(B.aggregate_segment(dst("qkv"), f32("qkv"), q_sub, self.kv_cover[l], self.kv_pos[l],
                                             Hkv, dh, (H + Hkv) * dh, self.nq * d, self.a_sub + self.kv_max * dh,
-                                            self.kv_max))
-            segs.append(B.aggregate_segment(self.full["o"][l], f32("o"), sub(self.w_o, self.w_o_m), self.cover_head[l],
-                                            self.pos_head[l], H, dh, 0, self.a_sub * d, 0, self.head_keep))
+                                            self.kv_max, central=cq))
+            segs.append(B.aggregate_segment(dst("o"), f32("o"), sub(self.w_o, self.w_o_m), self.cover_head[l],
+                                            self.pos_head[l], H, dh, 0, self.a_sub * d, 0, self.head_keep,
+                                            central=central("o")))
+        return segs
+
+    def aggregate_layer(self, l: int, live: int = 0xFFFFFFFF, which=("ffn", "attn")):
+        self._use(l)
+        w = self.w
+        f32 = (lambda m: self.full_f32[m][l]) if self.full_f32 is not None else (lambda m: None)
+        segs = self._aggregate_segments(l, which, lambda m: self.full[m][l], f32)
         with self._timed("aggregate"):
-            B.twist_aggregate(segs, w.n_subnets, d, w.dtype, live)
+            B.twist_aggregate(segs, w.n_subnets, w.d_model, w.dtype, live)
         self.launches += 1
 
     def _opt(self, k: int, *names):
@@ -769,6 +778,123 @@ class HybridRoundEngine(RoundEngine):
         with self._timed("aggregate"):
             B.twist_aggregate(segs, w.n_subnets, d, w.dtype, live)
         self.launches += 1
+
+
+def shard_range(n_subnets: int, rank: int, world: int) -> Tuple[int, int]:
+    """(first subnet, number of subnets) of `rank` when S subnets are spread evenly over `world` GPUs."""
+    if world < 1 or not 0 <= rank < world:
+        raise ValueError("rank %d of %d" % (rank, world))
+    if n_subnets % world != 0:
+        raise ValueError("%d subnets do not divide over %d GPUs" % (n_subnets, world))
+    per = n_subnets // world
+    return rank * per, per
+
+
+class ShardedRoundEngine(RoundEngine):
+    """The S subnets of a round spread over `world` GPUs, one process per GPU (Sec. 4.1: workers train their subnets in
+    parallel and a server averages them; here every GPU is worker for S / world subnets and all of them are the server).
+
+    Every GPU holds the whole model and samples the blueprints of all S subnets (the sampler is a pure function of
+    (seed, round, layer, kind), so nothing is exchanged for that), gathers and trains only its own subnets
+    subnet_begin .. subnet_begin + S / world - 1, and the aggregate runs in two halves around the one exchange of
+    the round: twist_aggregate_partial (fp32 sums of this GPU's subnets, zeros elsewhere, in full-matrix geometry), an
+    all-reduce (sum) of that buffer over the GPUs, twist_aggregate_finish (division by the global coverage counts,
+    written to the fp32 model and its bf16 shadow).  After it every GPU holds the same new model.  `reduce` is the
+    exchange: by default torch.distributed.all_reduce on the process group (NCCL), nothing when world == 1.
+    The batches (X, Td, Tq, A) the caller loads are those of the GPU's own subnets."""
+
+    def __init__(self, w: Workload, rank: int = 0, world: int = 1, reduce=None, device: str = "cuda", **kw):
+        from dataclasses import replace
+        self.global_w = w
+        self.rank, self.world = rank, world
+        self.subnet_begin, self.S_local = shard_range(w.n_subnets, rank, world)
+        self.S_global = w.n_subnets
+        super().__init__(replace(w, n_subnets=self.S_local), device=device, **kw)
+        lw, dev = self.w, self.dev
+        L, S, nb = lw.n_layers, self.S_global, lw.n_ffn_blocks
+        i32 = dict(dtype=torch.int32, device=dev)
+        own = slice(self.subnet_begin, self.subnet_begin + self.S_local)
+        # blueprints and ranks of ALL subnets; what the base class reads are views of this GPU's subnets
+        self.g_pos_ffn = torch.empty(L, S, nb, **i32)
+        self.pos_ffn = self.g_pos_ffn[:, own]
+        self.g_idx_ffn, self.g_idx_head = {}, {}
+        if self.has_attn:
+            H, Hkv = lw.n_heads, lw.n_kv_heads
+            self.g_pos_head = torch.empty(L, S, H, **i32)
+            self.g_kv_idx = torch.empty(L, S, Hkv, **i32)
+            self.g_kv_count = torch.empty(L, S, **i32)
+            self.g_kv_cols = torch.empty(L, S, **i32)
+            self.g_kv_pos = torch.empty(L, S, Hkv, **i32)
+            self.pos_head, self.kv_idx, self.kv_pos = self.g_pos_head[:, own], self.g_kv_idx[:, own], self.g_kv_pos[:, own]
+            self.kv_count, self.kv_cols = self.g_kv_count[:, own], self.g_kv_cols[:, own]
+        for kind, gm in self.geo.items():
+            self._use_kind(kind)
+            self.g_idx_ffn[kind] = torch.empty(L, S, gm.ffn_keep, **i32)
+            self.bufs[kind]["idx_ffn"] = self.idx_ffn = self.g_idx_ffn[kind][:, own]
+            if self.has_attn:
+                self.g_idx_head[kind] = torch.empty(L, S, gm.head_keep, **i32)
+                self.bufs[kind]["idx_head"] = self.idx_head = self.g_idx_head[kind][:, own]
+        self._use_kind("part")
+        # partial sums of one layer, every matrix back to back: one buffer, one exchange
+        rows = {m: v.shape[1] for m, v in self.full.items()}
+        self.part = torch.zeros(sum(rows.values()), lw.d_model, dtype=torch.float32, device=dev)
+        self.part_of, at = {}, 0
+        for m, r in rows.items():
+            self.part_of[m] = self.part[at:at + r]
+            at += r
+        self.reduce = reduce if reduce is not None else self._all_reduce
+
+    def _all_reduce(self, t: torch.Tensor):
+        if self.world > 1:
+            import torch.distributed as dist
+            dist.all_reduce(t, op=dist.ReduceOp.SUM)
+
+    def sample_masks(self, rnd: int):
+        w, S = self.w, self.S_global
+        with self._timed("sample_masks"):
+            for l0, n, kind in self._layer_runs():
+                self._use_kind(kind)
+                sl = slice(l0, l0 + n)
+                B.twist_sample_masks(w.seed_mask, rnd, l0, n, B.KIND_FFN, w.n_ffn_blocks, S, self.ffn_keep,
+                                     list(w.common_ffn), w.sample_mode, self.g_idx_ffn[kind][sl], self.cover_ffn[sl],
+                                     self.g_pos_ffn[sl])
+                self.launches += 2
+                if self.has_attn:
+                    B.twist_sample_masks(w.seed_mask, rnd, l0, n, B.KIND_HEAD, w.n_heads, S, self.head_keep,
+                                         list(w.common_heads), w.sample_mode, self.g_idx_head[kind][sl],
+                                         self.cover_head[sl], self.g_pos_head[sl])
+                    B.twist_kv_groups(self.g_idx_head[kind][sl], n, S, self.head_keep, w.n_heads, w.n_kv_heads,
+                                      w.d_head, self.g_kv_idx[sl], self.g_kv_count[sl], self.g_kv_cols[sl],
+                                      self.kv_cover[sl], self.g_kv_pos[sl])
+                    self.launches += 4
+
+    def aggregate_partial(self, l: int, live: int = 0xFFFFFFFF, which=("ffn", "attn")):
+        """This GPU's fp32 sums of layer l into self.part."""
+        self._use(l)
+        w = self.w
+        if w.dtype == DTYPE_BF16:
+            segs = self._aggregate_segments(l, which, lambda m: self.full[m][l], lambda m: self.part_of[m])
+        else:
+            segs = self._aggregate_segments(l, which, lambda m: self.part_of[m], lambda m: None)
+        with self._timed("aggregate"):
+            B.twist_aggregate_partial(segs, self.S_local, self.subnet_begin, w.d_model, w.dtype, live)
+        self.launches += 1
+
+    def aggregate_finish(self, l: int, live: int = 0xFFFFFFFF, which=("ffn", "attn")):
+        """The reduced sums in self.part divided by the coverage counts into the model."""
+        self._use(l)
+        w = self.w
+        f32 = (lambda m: self.full_f32[m][l]) if self.full_f32 is not None else (lambda m: None)
+        segs = self._aggregate_segments(l, which, lambda m: self.full[m][l], f32, central=lambda m: self.part_of[m])
+        with self._timed("aggregate"):
+            B.twist_aggregate_finish(segs, self.S_global, w.d_model, w.dtype, live)
+        self.launches += 1
+
+    def aggregate_layer(self, l: int, live: int = 0xFFFFFFFF, which=("ffn", "attn")):
+        self.aggregate_partial(l, live, which)
+        with self._timed("exchange"):
+            self.reduce(self.part)
+        self.aggregate_finish(l, live, which)
 
 
 class StackEngine(RoundEngine):

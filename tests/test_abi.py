@@ -23,7 +23,7 @@ def test_library_exports_every_declared_symbol():
     for n in names:
         assert hasattr(h, n), n
     assert sorted(B.EXPORTS) == names
-    assert B.twist_abi_version() == 2
+    assert B.twist_abi_version() == 3
     # every entry point that takes arguments declares their C types: a device address passed without them
     # would be truncated to 32 bits
     for n in names:

@@ -1080,6 +1080,84 @@ def test_plan_caches_tensor_maps_and_changes_no_result(B):
     plan.close()
 
 
+@pytest.mark.parametrize("cfg,dims,world", [
+    (4, dict(d_model=256, d_ff=1024, d_head=16, tokens=256, n_layers=2, local_steps=2), 2),
+    (3, dict(d_model=256, d_ff=688, d_head=8, tokens=256, n_layers=2, local_steps=2), 4),
+    (1, dict(), 2),
+    (4, dict(d_model=256, d_ff=1024, d_head=16, tokens=256, n_layers=1, local_steps=1), 1),
+])
+def test_subnets_sharded_over_several_gpus_match_the_single_gpu_round(B, cfg, dims, world):
+    """The S subnets of a round spread over `world` ranks (Sec. 4.1: workers in parallel, one server average), emulated
+    here as `world` engines in one process whose partial-sum buffers the test adds up in place of the all-reduce.
+    Every rank ends with the same model bit for bit; local training is bit-identical to the single-GPU round (same
+    slices, same batches, same kernels: the losses say so); the new model equals the single-GPU one up to the fp32
+    rounding of a differently associated sum, and the fp64 oracle within the aggregate's bound."""
+    from paper_2511_03983_b200.engine import RoundEngine, ShardedRoundEngine, shard_range
+    w = I.scaled_twin(I.PRESETS[cfg], **dims) if dims else I.PRESETS[cfg]
+    lowp = w.dtype == I.DTYPE_BF16
+    kw = dict(keep_f32_full=True) if lowp else {}
+    ref = RoundEngine(w, **kw)
+    full_np = _load_full(ref, w)
+    if ref.full_f32 is not None:
+        for m in ref.full:
+            ref.full_f32[m].copy_(ref.full[m].float())
+    _load_batches(ref, w, 0)
+    start = {m: v.clone() for m, v in ref.full.items()}
+    ref.run_round(0)
+    ranks = []
+    for r in range(world):
+        e = ShardedRoundEngine(w, rank=r, world=world, reduce=lambda t: None, **kw)
+        s0, n = shard_range(w.n_subnets, r, world)
+        assert (e.subnet_begin, e.S_local) == (s0, n)
+        for m in e.full:
+            e.full[m].copy_(start[m])
+            if e.full_f32 is not None:
+                e.full_f32[m].copy_(start[m].float())
+        own = slice(s0, s0 + n)
+        e.X, e.Td = [t[own].contiguous() for t in ref.X], [t[own].contiguous() for t in ref.Td]
+        if e.has_attn:
+            for gk in e.geo:
+                e.batches[gk] = {name: [t[own].contiguous() for t in ref.batches[gk][name]] for name in ("Tq", "A")}
+        e.sample_masks(0)
+        ranks.append(e)
+    for l in range(w.n_layers):
+        for e in ranks:                                  # each rank's local training, one after the other
+            e.gather_layer(l)
+            for k in range(w.local_steps):
+                e.ffn_step(l, k)
+                if e.has_attn:
+                    e.qkv_step(l, k)
+                    e.o_step(l, k)
+            e.aggregate_partial(l)
+        total = ranks[0].part.clone()                    # the exchange: sum over the ranks, the same bits everywhere
+        for e in ranks[1:]:
+            total += e.part
+        for e in ranks:
+            e.part.copy_(total)
+            e.aggregate_finish(l)
+    torch.cuda.synchronize()
+    check_status(B)
+    for e in ranks:
+        s0 = e.subnet_begin
+        assert torch.equal(e.loss, ref.loss[..., s0:s0 + e.S_local])           # the same local training
+        assert torch.equal(e.cover_ffn, ref.cover_ffn)                         # the same blueprints on every rank
+        for m in e.full:
+            assert torch.equal(e.full[m], ranks[0].full[m]), m                 # one model after the round
+            if e.full_f32 is not None:
+                assert torch.equal(e.full_f32[m], ranks[0].full_f32[m]), m
+    got = ranks[0].full_f32 if lowp else ranks[0].full
+    want = ref.full_f32 if lowp else ref.full
+    for m in got:
+        assert not torch.equal(ranks[0].full[m], start[m])                     # the round did change the model
+        g, r_ = got[m].double(), want[m].double()
+        # differently associated fp32 sums of at most S terms, each of magnitude <= |mean| * count
+        assert float((g - r_).abs().max()) <= 4 * w.n_subnets * 2.0 ** -24 * float(r_.abs().max()), m
+        if lowp:                                                               # shadow = nearest-even rounding of fp32
+            assert torch.equal(ranks[0].full[m], got[m].to(torch.bfloat16))
+        if world == 1:                                                         # one GPU: the two halves are the aggregator
+            assert torch.equal(got[m], want[m]) and torch.equal(ranks[0].full[m], ref.full[m]), m
+
+
 def test_layer_step_captured_in_a_cuda_graph_replays_bit_identically(B):
     """A forward + backward FFN step with the fused loss, captured in a CUDA graph after an eager warm-up and replayed
     twice, gives the bits of the eager step.  Inside a capture the library's host-sequenced device counters are off

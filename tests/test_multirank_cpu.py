@@ -75,3 +75,69 @@ def test_two_gloo_ranks_through_the_spawn_path(tmp_path):
     assert bench.spawn_replicas(2, [sys.executable, "-c", code, str(tmp_path), ROOT], timeout=120) == 0
     got = [json.load(open(tmp_path / f"g{r}.json")) for r in range(2)]
     assert got[0] == got[1] == {"ms": 11.0, "world": 2}
+
+
+def _shard_worker(rank, world, port, out_dir):
+    """One rank of the sharded aggregate on CPU: numpy float32 stands in for the two device halves, the exchange is the
+    engine's own (torch.distributed all-reduce, here on gloo)."""
+    import types
+    import numpy as np
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    sys.path.insert(0, os.path.join(ROOT, "tests"))
+    from paper_2511_03983_b200.engine import ShardedRoundEngine, shard_range
+    S, n_full, n_sub, rows, d = 4, 12, 5, 2, 8
+    rng = np.random.default_rng(7)                       # every rank draws the same blueprints and slices
+    blueprints = [np.sort(rng.choice(n_full, n_sub, replace=False)) for _ in range(S)]
+    subs = [rng.standard_normal((n_sub * rows, d)).astype(np.float32) for _ in range(S)]
+    W_full = rng.standard_normal((n_full * rows, d)).astype(np.float32)
+    s0, n = shard_range(S, rank, world)
+    part = np.zeros_like(W_full)                         # first half: this rank's sums, zeros elsewhere
+    for s in range(s0, s0 + n):                          # ascending subnet order, float32 additions
+        for j, b in enumerate(blueprints[s]):
+            part[b * rows:(b + 1) * rows] += subs[s][j * rows:(j + 1) * rows]
+    t = torch.from_numpy(part)
+    ShardedRoundEngine._all_reduce(types.SimpleNamespace(world=world), t)       # the exchange
+    count = np.zeros(n_full, dtype=np.int64)
+    for bp in blueprints:
+        count[bp] += 1
+    out = W_full.copy()                                  # second half: division by the global coverage
+    held = np.repeat(count > 0, rows)
+    out[held] = t.numpy()[held] / np.repeat(count, rows)[held].astype(np.float32)[:, None]
+    np.save(os.path.join(out_dir, f"shard{rank}.npy"), out)
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_sharded_aggregate_over_two_gloo_ranks_equals_the_aggregator(tmp_path):
+    """Partial sums per rank, the engine's all-reduce, division by the global counts: both ranks end with the same
+    model, which is the aggregator's (Sec. 3.3) result up to the rounding of a differently associated fp32 sum."""
+    import numpy as np
+    sys.path.insert(0, os.path.join(ROOT, "tests"))
+    from fp32_mirror import aggregate_f32
+    from oracle import twist_oracle as o
+    from paper_2511_03983_b200.engine import shard_range
+    port = 31500 + os.getpid() % 2000
+    mp.spawn(_shard_worker, args=(2, port, str(tmp_path)), nprocs=2, join=True)
+    got = [np.load(tmp_path / f"shard{r}.npy") for r in range(2)]
+    assert np.array_equal(got[0], got[1])
+    S, n_full, n_sub, rows, d = 4, 12, 5, 2, 8
+    rng = np.random.default_rng(7)
+    blueprints = [np.sort(rng.choice(n_full, n_sub, replace=False)) for _ in range(S)]
+    subs = [rng.standard_normal((n_sub * rows, d)).astype(np.float32) for _ in range(S)]
+    W_full = rng.standard_normal((n_full * rows, d)).astype(np.float32)
+    mirror = aggregate_f32(W_full, subs, blueprints, rows)
+    assert np.max(np.abs(got[0] - mirror)) <= 4 * 2.0 ** -24 * np.max(np.abs(mirror)) * S
+    want = o.aggregate(W_full.astype(np.float64), [s.astype(np.float64) for s in subs], blueprints, rows)
+    assert np.max(np.abs(got[0] - want)) <= 1e-6 * np.max(np.abs(want)) * S
+    uncovered = np.setdiff1d(np.arange(n_full), np.concatenate(blueprints))
+    for b in uncovered:                                  # rows nobody holds keep their value
+        assert np.array_equal(got[0][b * rows:(b + 1) * rows], W_full[b * rows:(b + 1) * rows])
+    for world in (1, 2, 4):
+        assert [shard_range(8, r, world) for r in range(world)] == [(r * 8 // world, 8 // world) for r in range(world)]
+    for bad in ((8, 0, 3), (8, 2, 2), (8, -1, 2)):
+        try:
+            shard_range(*bad)
+            raise AssertionError(bad)
+        except ValueError:
+            pass
