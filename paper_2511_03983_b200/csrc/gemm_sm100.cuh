@@ -402,6 +402,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   cluster_sync_all();          // the peer's barriers exist before anything is signalled across the pair
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  // The set-up above touches nothing an earlier launch wrote, so it may overlap that launch's tail; from here on
+  // this launch reads its operands.  (Its own successor may in turn be placed as soon as these CTAs have gone.)
+  griddep_launch_dependents();
+  griddep_wait();
 
   if (warp == kEpiWarps) {
     // ------------------------------------------------------------------ TMA producer (both CTAs)

@@ -93,6 +93,13 @@ __device__ inline void drain_after_abort(volatile int* abort_flag) {
   }
 }
 
+// Programmatic dependent launch.  griddep_launch_dependents: the next launch of the stream (if it was launched with
+// programmatic stream serialisation) may place its CTAs wherever these have gone, instead of after the whole grid
+// has drained.  griddep_wait: returns once every launch this one depends on has completed and its writes are
+// visible; a no-op in a launch without that attribute.
+__device__ inline void griddep_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ inline void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 __device__ inline void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 template <int N>
 __device__ inline void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
