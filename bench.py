@@ -431,7 +431,7 @@ def run_ours(args, w):
         return
 
     peaks = measured_peaks()
-    work = round_work(eng.w)                              # per GPU (sharded: its S / N subnets)
+    work = round_work(eng.w if sharded else w)            # per GPU (sharded: its S / N subnets)
     if sharded:     # the aggregate in two halves: sums of the GPU's subnets written for the whole layer (4 B per element),
         full = work.pop("full_elems")     # then the reduced sums read and the fp32 model + bf16 shadow written (4 + 4 + 2)
         work["aggregate_bytes"] += (4 + 4) * full * w.n_layers
