@@ -65,6 +65,17 @@ def test_host_side_argument_checks():
     assert h.twist_aggregate(None, 1, 2, 64, B.BF16, 3, None) == B.ERR_NULL
     ag = (B.AggregateSegment * 1)(B.AggregateSegment(0x1000, None, 0x2000, 0x3000, 0x4000, 8, 1, 0, 256, 0, None, 0, 0))
     assert h.twist_aggregate(C.cast(ag, C.c_void_p), 1, 2, 64, B.BF16, 3, None) == B.ERR_SHAPE   # slice block count missing
+    # the aggregate in two halves (subnets spread over GPUs)
+    ok_seg = lambda **kw: (B.AggregateSegment * 1)(B.AggregateSegment(**dict(dict(
+        dst=0x1000, dst_f32=0x5000, sub=0x2000, cover=0x3000, pos=0x4000, n_full=8, block_rows=1, dst_row_offset=0,
+        sub_subnet_stride=256, sub_row_offset=0, central=None, central_subnet=0, n_keep=4), **kw)))
+    part = lambda seg, n, s0: h.twist_aggregate_partial(C.cast(seg, C.c_void_p), 1, n, s0, 64, B.BF16, 0xFFFFFFFF, None)
+    assert part(ok_seg(), 4, 30) == B.ERR_SHAPE                          # subnets 30..33: beyond the 32 of a cover mask
+    assert part(ok_seg(dst_f32=None), 4, 0) == B.ERR_NULL                # the partial sums are fp32: they need a buffer
+    assert part(ok_seg(central=0x6000), 4, 0) == B.ERR_UNSUPPORTED       # no in-place worker on a shard
+    fin = lambda seg: h.twist_aggregate_finish(C.cast(seg, C.c_void_p), 1, 8, 64, B.BF16, 0xFFFFFFFF, None)
+    assert fin(ok_seg()) == B.ERR_NULL                                   # the reduced sums (central) are missing
+    assert fin(ok_seg(central=0x6004)) == B.ERR_SHAPE                    # ... or not 16-byte aligned
     assert h.twist_selftest_wait(0, None) == B.ERR_SHAPE and h.twist_selftest_wait(10 ** 9, None) == B.ERR_SHAPE
     # local steps
     a = B.FfnArgs(B.FFN_SWIGLU, B.BF16, 2, 128, 64, 100, 1.0, 0.0)       # f_sub not a multiple of 8
